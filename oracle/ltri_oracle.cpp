@@ -1,0 +1,695 @@
+// Ltri-LLM streaming attention -- CPU ORACLE (test infrastructure, not product code).
+//
+// A plain, slow, fp32 restatement of the method's hot path, one thread per query
+// head, written from the paper's equations.  It shares no code with the CUDA path
+// and must never be imported, linked or executed by it.  Only the tests, the smoke
+// check and the benchmark's CPU-baseline leg call into this file.
+//
+// One `Stream` object is one (sequence, layer): the method treats layers and
+// sequences independently.
+//
+// Steps (paper passage each follows):
+//   O1  append K/V of the call                               Sec. 3.4 "Overall Framework"
+//   O2  evict regions that left the window; pick the most     Sec. 3.4 step 1; Eq. 6 (votes v_x),
+//       voted token(s) of each span as its index vector       Sec. 3.3.1 (static index vectors)
+//   O3  local attention rows: softmax over sink+local+cur     Eq. 1-3 restricted to the local map
+//   O4  Q20 fixed-point map, head sum, votes                  Eq. 4 (sum over heads), Eq. 6
+//   O5  threshold theta                                       Eq. 5, App. "Configuration" (quantile)
+//   O6  triangle scores, anti-diagonal filter, greedy NMS     Eq. 4-5, App. "NMS Input Filtration"
+//   O7  query representatives of the call's spans             Sec. 3.4 step 2
+//   O8  similarity of query reps vs span index                Eq. 7
+//   O9  top-k spans                                           Eq. 8 (unit = span)
+//   O10 softmax attention over sink+retrieved+local+cur       Sec. 3.4 step 3
+//   O11 decode step (one query, no eviction, no votes)        Sec. 3.5 "Persistent Mechanism" (the
+//                                                             block becomes a single token)
+//   O12 full causal attention (reference for the pin
+//       "top-k covers every span => method == full attention")
+//
+// Parity status: O3/O10/O12 are pinned by softmax invariants and by the full-attention
+// equivalence; O6 is pinned by brute force, by hand-built block maps and by a library
+// NMS; O8/O9 by brute force.  "parity unpinned" (defined only by this build's readings
+// of passages the paper leaves open, checked by brute force and hand-built cases but by
+// nothing the paper prints): the quantile convention of theta, the Q20 rounding of the
+// map, gap filling, the vote-based choice of representative tokens and its tie rule,
+// the max over query spans of summed representatives, and the decode rules.
+//
+// Build: g++ -O2 -std=c++17 -shared -fPIC -pthread ltri_oracle.cpp -o libltri_oracle.so
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <deque>
+#include <functional>
+#include <thread>
+#include <vector>
+
+namespace {
+
+constexpr int kQ = 20;  // fixed-point fraction bits of the attention map
+constexpr float kQScale = 1048576.0f;
+
+inline float bf16_to_f32(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+
+inline uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40);  // NaN
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7fffu + lsb;
+  return (uint16_t)(u >> 16);
+}
+
+struct Span {
+  int start, len;
+};
+
+struct Region {
+  int start, end;
+  std::vector<Span> spans;
+};
+
+struct Params {
+  int32_t n_q_heads, n_kv_heads, head_dim;
+  int32_t chunk, window, n_sink, top_k;
+  int32_t reps_per_span, max_spans_per_region;
+  int32_t theta_mode;
+  float theta;
+  float softmax_scale;
+  int64_t max_tokens;
+};
+
+// ---------------------------------------------------------------------------
+// O5: threshold in Q20 units of the head-summed map.
+// mode 0: absolute head-mean probability -> theta * Hq * 2^20, rounded to nearest even.
+// mode 1: lower nearest-rank quantile of the causal entries of the region map.
+int64_t theta_q(const int32_t* Mq, int m, int ld, int mode, float theta, int Hq) {
+  if (m <= 0) return 0;
+  if (mode == 0) return (int64_t)std::nearbyint((double)theta * (double)Hq * (double)kQScale);
+  int64_t N = (int64_t)m * (m + 1) / 2;
+  std::vector<int32_t> vals;
+  vals.reserve((size_t)N);
+  for (int i = 0; i < m; ++i)
+    for (int j = 0; j <= i; ++j) vals.push_back(Mq[(size_t)i * ld + j]);
+  int64_t rank = (int64_t)std::floor((double)theta * (double)(N - 1));
+  if (rank < 0) rank = 0;
+  if (rank > N - 1) rank = N - 1;
+  std::nth_element(vals.begin(), vals.begin() + rank, vals.end());
+  return vals[(size_t)rank];
+}
+
+// Eq. 4-5 by the two cumulative sums of Fig. 2: S(x,y) = sum_{x<=j<=i<=y} (Mq[i][j]-theta).
+// Rsuf[i][x] = sum_{j=x..i} D[i][j]  (suffix sum along the row, "sum the right elements"),
+// S(x,y)     = sum_{i=x..y} Rsuf[i][x] (prefix sum down the column, "sum the upper elements").
+// Output S is m x m, entry [x*m+y] defined for x<=y.
+void ta_scores(const int32_t* Mq, int m, int ld, int64_t thq, std::vector<int64_t>& S) {
+  std::vector<int64_t> R((size_t)m * m, 0);
+  for (int i = 0; i < m; ++i) {
+    int64_t acc = 0;
+    for (int x = i; x >= 0; --x) {
+      acc += (int64_t)Mq[(size_t)i * ld + x] - thq;
+      R[(size_t)i * m + x] = acc;
+    }
+  }
+  S.assign((size_t)m * m, 0);
+  for (int x = 0; x < m; ++x) {
+    int64_t acc = 0;
+    for (int y = x; y < m; ++y) {
+      acc += R[(size_t)y * m + x];
+      S[(size_t)x * m + y] = acc;
+    }
+  }
+}
+
+struct Cand {
+  int64_t S;
+  int x, y;
+};
+
+inline double rel_gap(int64_t a, int64_t b) {
+  double da = (double)a, db = (double)b;
+  double den = std::max(std::fabs(da), std::fabs(db));
+  if (den == 0.0) return 0.0;
+  return std::fabs(da - db) / den;
+}
+
+// O6: anti-diagonal filter, sort, greedy disjoint NMS (IoU threshold 0), gap fill.
+// `min_gap` (optional) receives the smallest relative gap between two quantities whose
+// comparison decided something: best vs runner-up on an anti-diagonal that produced a
+// candidate; the best point's triangle mass vs its theta*area (the sign test S>0) on every
+// anti-diagonal; and neighbours in the sorted candidate list up to the last one the
+// greedy pass looked at.
+void segment_map(const int32_t* Mq, int m, int ld, int64_t thq, int C, std::vector<Span>& out,
+                 double* min_gap) {
+  out.clear();
+  double gap = 1.0;
+  if (m <= 0) {
+    if (min_gap) *min_gap = gap;
+    return;
+  }
+  std::vector<int64_t> S;
+  ta_scores(Mq, m, ld, thq, S);
+  std::vector<Cand> cands;
+  for (int c = 0; c <= 2 * m - 2; ++c) {
+    bool have = false;
+    Cand best{0, 0, 0};
+    int64_t second = 0;
+    bool have2 = false;
+    // walk from the shortest interval outwards so that ties keep the shorter span
+    int y0 = (c + 1) / 2;
+    for (int y = y0; y < m && c - y >= 0; ++y) {
+      int x = c - y;
+      int64_t s = S[(size_t)x * m + y];
+      if (!have || s > best.S) {
+        if (have) {
+          second = have2 ? std::max(second, best.S) : best.S;
+          have2 = true;
+        }
+        best = Cand{s, x, y};
+        have = true;
+      } else {
+        second = have2 ? std::max(second, s) : s;
+        have2 = true;
+      }
+    }
+    if (have) {
+      int64_t len = best.y - best.x + 1;
+      int64_t tarea = thq * (len * (len + 1) / 2);
+      gap = std::min(gap, rel_gap(best.S + tarea, tarea));
+    }
+    if (have && best.S > 0) {
+      cands.push_back(best);
+      if (have2) gap = std::min(gap, rel_gap(best.S, second));
+    }
+  }
+  std::sort(cands.begin(), cands.end(), [](const Cand& a, const Cand& b) {
+    if (a.S != b.S) return a.S > b.S;
+    int la = a.y - a.x, lb = b.y - b.x;
+    if (la != lb) return la < lb;
+    return a.x < b.x;
+  });
+  std::vector<Cand> kept;
+  size_t examined = 0;
+  for (size_t ci = 0; ci < cands.size() && (int)kept.size() < C; ++ci) {
+    examined = ci + 1;
+    const Cand& c = cands[ci];
+    bool ok = true;
+    for (const Cand& k : kept)
+      if (!(c.y < k.x || c.x > k.y)) {
+        ok = false;
+        break;
+      }
+    if (ok) kept.push_back(c);
+  }
+  for (size_t ci = 0; ci + 1 < cands.size() && ci < examined; ++ci)
+    gap = std::min(gap, rel_gap(cands[ci].S, cands[ci + 1].S));
+  std::sort(kept.begin(), kept.end(), [](const Cand& a, const Cand& b) { return a.x < b.x; });
+  int pos = 0;
+  for (const Cand& k : kept) {
+    if (k.x > pos) out.push_back(Span{pos, k.x - pos});
+    out.push_back(Span{k.x, k.y - k.x + 1});
+    pos = k.y + 1;
+  }
+  if (pos < m) out.push_back(Span{pos, m - pos});
+  if (min_gap) *min_gap = gap;
+}
+
+// O9: the min(k,n) largest scores, ties -> lower id.  ids in rank order, -1 padded.
+void top_k(const float* score, int n, int k, int* ids, double* cut_gap) {
+  std::vector<int> order(n);
+  for (int i = 0; i < n; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(),
+                   [&](int a, int b) { return score[a] > score[b]; });
+  int kk = std::min(k, n);
+  for (int i = 0; i < k; ++i) ids[i] = i < kk ? order[i] : -1;
+  if (cut_gap) {
+    *cut_gap = 1.0;
+    if (kk < n && kk > 0) {
+      double a = score[order[kk - 1]], b = score[order[kk]];
+      double den = std::max(std::fabs(a), std::fabs(b));
+      *cut_gap = den == 0.0 ? 0.0 : std::fabs(a - b) / den;
+    }
+  }
+}
+
+void run_heads(int H, const std::function<void(int)>& fn) {
+  std::vector<std::thread> th;
+  th.reserve(H);
+  for (int h = 0; h < H; ++h) th.emplace_back(fn, h);
+  for (auto& t : th) t.join();
+}
+
+struct Stream {
+  Params p;
+  int Hq, Hkv, G, d;
+  float scale;
+  int t = 0;  // tokens appended so far
+  int E;      // end of the evicted (indexed) prefix
+  bool decoding = false;
+  std::vector<float> K, V;  // [Hkv][max_tokens][d]
+  std::vector<int64_t> votes;
+  std::deque<Region> pending;
+  std::vector<Span> spans;    // indexed spans, tile [Ls,E)
+  std::vector<uint16_t> KR;   // [span][Hkv][d] bf16 bits
+  // state of the current call
+  int t0 = 0, n = 0;
+  std::vector<float> Q;  // [n][Hq][d]
+  int reg_start = 0, m = 0;
+  std::vector<int32_t> Mq;  // [m][m]
+  int64_t thq = 0;
+  double seg_gap = 1.0;
+  std::vector<float> u;  // [Hkv][J][d]
+  int J = 0;
+  std::vector<float> score;  // [Hkv][Ns]
+  std::vector<int> sel;      // [Hkv][top_k]
+  std::vector<double> cut_gap;  // [Hkv]
+  std::vector<int> qrep_tok;    // [J][reps] absolute tokens, -1 padded
+
+  explicit Stream(const Params& pp) : p(pp) {
+    Hq = p.n_q_heads;
+    Hkv = p.n_kv_heads;
+    G = Hq / Hkv;
+    d = p.head_dim;
+    scale = p.softmax_scale > 0 ? p.softmax_scale : 1.0f / std::sqrt((float)d);
+    E = p.n_sink;
+    K.assign((size_t)Hkv * p.max_tokens * d, 0.f);
+    V.assign((size_t)Hkv * p.max_tokens * d, 0.f);
+    votes.assign((size_t)p.max_tokens, 0);
+    sel.assign((size_t)Hkv * p.top_k, -1);
+    cut_gap.assign(Hkv, 1.0);
+  }
+
+  const float* krow(int g, int tok) const { return &K[((size_t)g * p.max_tokens + tok) * d]; }
+  const float* vrow(int g, int tok) const { return &V[((size_t)g * p.max_tokens + tok) * d]; }
+
+  // O1
+  void append(int cnt, const uint16_t* kb, const uint16_t* vb) {
+    for (int r = 0; r < cnt; ++r)
+      for (int g = 0; g < Hkv; ++g)
+        for (int e = 0; e < d; ++e) {
+          size_t src = ((size_t)r * Hkv + g) * d + e;
+          size_t dst = ((size_t)g * p.max_tokens + (t + r)) * d + e;
+          K[dst] = bf16_to_f32(kb[src]);
+          V[dst] = bf16_to_f32(vb[src]);
+        }
+    t += cnt;
+  }
+
+  // tokens of [lo,hi) with the largest votes, ties -> lower index; returned ascending.
+  std::vector<int> rep_tokens(int lo, int len) const {
+    int cnt = std::min(p.reps_per_span, len);
+    std::vector<int> idx(len);
+    for (int i = 0; i < len; ++i) idx[i] = lo + i;
+    std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) { return votes[a] > votes[b]; });
+    idx.resize(cnt);
+    std::sort(idx.begin(), idx.end());
+    return idx;
+  }
+
+  // O2
+  void evict(int t0_) {
+    while (!pending.empty() && pending.front().end <= t0_ - p.window) {
+      Region& r = pending.front();
+      for (const Span& s : r.spans) {
+        std::vector<int> reps = rep_tokens(s.start, s.len);
+        size_t base = KR.size();
+        KR.resize(base + (size_t)Hkv * d);
+        for (int g = 0; g < Hkv; ++g)
+          for (int e = 0; e < d; ++e) {
+            float acc = 0.f;
+            for (int tok : reps) acc += krow(g, tok)[e];
+            KR[base + (size_t)g * d + e] = f32_to_bf16_rne(acc);
+          }
+        spans.push_back(s);
+      }
+      E = r.end;
+      pending.pop_front();
+    }
+  }
+
+  struct KeySet {
+    // half-open token ranges in the order sink, retrieved..., local, cur
+    std::vector<std::pair<int, int>> ranges;
+  };
+
+  // softmax statistics + probabilities of one (head,row) over a key list; fp32 throughout.
+  void softmax_row(const float* qv, int g, const std::vector<std::pair<int, int>>& ranges,
+                   std::vector<float>& pbuf, float& l_out) const {
+    pbuf.clear();
+    float mx = -INFINITY;
+    for (auto& rg : ranges)
+      for (int j = rg.first; j < rg.second; ++j) {
+        const float* kr = krow(g, j);
+        float acc = 0.f;
+        for (int e = 0; e < d; ++e) acc += qv[e] * kr[e];
+        float s = acc * scale;
+        pbuf.push_back(s);
+        mx = std::max(mx, s);
+      }
+    float l = 0.f;
+    for (float& s : pbuf) {
+      s = std::exp(s - mx);
+      l += s;
+    }
+    l_out = l;
+  }
+
+  // O1-O6
+  int prefill_local(int cnt, const uint16_t* qb, const uint16_t* kb, const uint16_t* vb) {
+    if (decoding) return -3;
+    if (cnt < 1 || cnt > p.chunk || (int64_t)t + cnt > p.max_tokens) return -2;
+    t0 = t;
+    n = cnt;
+    append(cnt, kb, vb);
+    evict(t0);
+    Q.resize((size_t)n * Hq * d);
+    for (size_t i = 0; i < Q.size(); ++i) Q[i] = bf16_to_f32(qb[i]);
+    reg_start = std::max(p.n_sink, t0);
+    m = std::max(0, t0 + n - reg_start);
+    const int sink_end = std::min(p.n_sink, t0);
+    const int loc_begin = std::min(E, t0);
+    std::vector<std::vector<int32_t>> Mh(Hq);
+    std::vector<std::vector<int64_t>> vh(Hq);
+    const int vbase = loc_begin;  // votes touched lie in [loc_begin, t0+n)
+    run_heads(Hq, [&](int h) {
+      int g = h / G;
+      Mh[h].assign((size_t)m * m, 0);
+      vh[h].assign((size_t)(t0 + n - vbase), 0);
+      std::vector<float> pbuf;
+      std::vector<std::pair<int, int>> ranges(3);
+      for (int r = 0; r < n; ++r) {
+        int i = t0 + r;
+        ranges[0] = {0, sink_end};
+        ranges[1] = {loc_begin, t0};
+        ranges[2] = {t0, i + 1};
+        float l;
+        softmax_row(&Q[((size_t)r * Hq + h) * d], g, ranges, pbuf, l);
+        size_t pi = 0;
+        for (auto& rg : ranges)
+          for (int j = rg.first; j < rg.second; ++j, ++pi) {
+            float a = pbuf[pi] / l;
+            int32_t aq = (int32_t)std::nearbyintf(a * kQScale);
+            if (j >= loc_begin && j >= p.n_sink) vh[h][j - vbase] += aq;  // O4 votes (Eq. 6)
+            if (j >= reg_start && i >= reg_start)
+              Mh[h][(size_t)(i - reg_start) * m + (j - reg_start)] += aq;  // O4 map
+          }
+      }
+    });
+    Mq.assign((size_t)m * m, 0);
+    for (int h = 0; h < Hq; ++h) {
+      for (size_t i = 0; i < Mq.size(); ++i) Mq[i] += Mh[h][i];
+      for (size_t i = 0; i < vh[h].size(); ++i) votes[vbase + i] += vh[h][i];
+    }
+    Region reg;
+    reg.start = reg_start;
+    reg.end = t0 + n;
+    if (m > 0) {
+      thq = theta_q(Mq.data(), m, m, p.theta_mode, p.theta, Hq);
+      std::vector<Span> sp;
+      segment_map(Mq.data(), m, m, thq, p.max_spans_per_region, sp, &seg_gap);
+      for (Span& s : sp) s.start += reg_start;
+      reg.spans = sp;
+      pending.push_back(reg);
+    } else {
+      thq = 0;
+      seg_gap = 1.0;
+    }
+    return 0;
+  }
+
+  // O7-O9 for the current prefill call (uses the spans stored for the newest region).
+  void prefill_retrieve() {
+    J = 0;
+    u.clear();
+    qrep_tok.clear();
+    if (m > 0) {
+      const Region& reg = pending.back();
+      J = (int)reg.spans.size();
+      u.assign((size_t)Hkv * J * d, 0.f);
+      qrep_tok.assign((size_t)J * p.reps_per_span, -1);
+      for (int j = 0; j < J; ++j) {
+        std::vector<int> reps = rep_tokens(reg.spans[j].start, reg.spans[j].len);
+        for (size_t r = 0; r < reps.size(); ++r) qrep_tok[(size_t)j * p.reps_per_span + r] = reps[r];
+        for (int g = 0; g < Hkv; ++g)
+          for (int e = 0; e < d; ++e) {
+            float ug = 0.f;
+            for (int h = g * G; h < (g + 1) * G; ++h) {
+              float qr = 0.f;
+              for (int tok : reps) qr += Q[((size_t)(tok - t0) * Hq + h) * d + e];
+              ug += qr;
+            }
+            u[((size_t)g * J + j) * d + e] = ug;
+          }
+      }
+    }
+    score_and_select();
+  }
+
+  // O8 + O9 with the representatives in `u` ([Hkv][J][d]).
+  void score_and_select() {
+    int Ns = (int)spans.size();
+    score.assign((size_t)Hkv * Ns, -INFINITY);
+    for (int g = 0; g < Hkv; ++g) {
+      for (int s = 0; s < Ns; ++s) {
+        float best = -INFINITY;
+        for (int j = 0; j < J; ++j) {
+          const float* uj = &u[((size_t)g * J + j) * d];
+          const uint16_t* kr = &KR[((size_t)s * Hkv + g) * d];
+          float acc = 0.f;
+          for (int e = 0; e < d; ++e) acc += uj[e] * bf16_to_f32(kr[e]);
+          best = std::max(best, acc);
+        }
+        score[(size_t)g * Ns + s] = best;
+      }
+      if (J > 0)
+        top_k(&score[(size_t)g * Ns], Ns, p.top_k, &sel[(size_t)g * p.top_k], &cut_gap[g]);
+      else {
+        for (int i = 0; i < p.top_k; ++i) sel[(size_t)g * p.top_k + i] = -1;
+        cut_gap[g] = 1.0;
+      }
+    }
+  }
+
+  std::vector<std::pair<int, int>> key_ranges(int g, int sink_end, int loc_begin, int loc_end) const {
+    std::vector<std::pair<int, int>> ranges;
+    ranges.push_back({0, sink_end});
+    for (int i = 0; i < p.top_k; ++i) {
+      int s = sel[(size_t)g * p.top_k + i];
+      if (s >= 0) ranges.push_back({spans[s].start, spans[s].start + spans[s].len});
+    }
+    ranges.push_back({loc_begin, loc_end});
+    return ranges;
+  }
+
+  void attend_row(const float* qv, int g, std::vector<std::pair<int, int>>& ranges, float* out) const {
+    std::vector<float> pbuf;
+    float l;
+    softmax_row(qv, g, ranges, pbuf, l);
+    std::vector<float> acc(d, 0.f);
+    size_t pi = 0;
+    for (auto& rg : ranges)
+      for (int j = rg.first; j < rg.second; ++j, ++pi) {
+        const float* vr = vrow(g, j);
+        float pj = pbuf[pi];
+        for (int e = 0; e < d; ++e) acc[e] += pj * vr[e];
+      }
+    for (int e = 0; e < d; ++e) out[e] = acc[e] / l;
+  }
+
+  // O10 for rows [r0,r1) of the current call; out is [r1-r0][Hq][d] fp32.
+  void prefill_attend(int r0, int r1, float* out) const {
+    const int sink_end = std::min(p.n_sink, t0);
+    const int loc_begin = std::min(E, t0);
+    run_heads(Hq, [&](int h) {
+      int g = h / G;
+      for (int r = r0; r < r1; ++r) {
+        auto ranges = key_ranges(g, sink_end, loc_begin, t0);
+        ranges.push_back({t0, t0 + r + 1});
+        attend_row(&Q[((size_t)r * Hq + h) * d], g, ranges, &out[((size_t)(r - r0) * Hq + h) * d]);
+      }
+    });
+  }
+
+  // O11: retrieval part of a decode step.
+  int decode_retrieve(const uint16_t* qb, const uint16_t* kb, const uint16_t* vb) {
+    if ((int64_t)t + 1 > p.max_tokens) return -2;
+    decoding = true;
+    t0 = t;
+    n = 1;
+    m = 0;
+    append(1, kb, vb);
+    Q.resize((size_t)Hq * d);
+    for (size_t i = 0; i < Q.size(); ++i) Q[i] = bf16_to_f32(qb[i]);
+    J = 1;
+    u.assign((size_t)Hkv * d, 0.f);
+    for (int g = 0; g < Hkv; ++g)
+      for (int e = 0; e < d; ++e) {
+        float ug = 0.f;
+        for (int h = g * G; h < (g + 1) * G; ++h) ug += Q[(size_t)h * d + e];
+        u[(size_t)g * d + e] = ug;
+      }
+    score_and_select();
+    return 0;
+  }
+
+  // O11: attention part of a decode step; out is [Hq][d] fp32.
+  void decode_attend(float* out) const {
+    const int pos = t0;  // the decode token's own position
+    const int sink_end = std::min(p.n_sink, pos + 1);
+    const int loc_begin = std::min(E, pos + 1);
+    run_heads(Hq, [&](int h) {
+      int g = h / G;
+      auto ranges = key_ranges(g, sink_end, loc_begin, pos + 1);
+      attend_row(&Q[(size_t)h * d], g, ranges, &out[(size_t)h * d]);
+    });
+  }
+
+  // O12: causal attention over every cached token <= position, for given query rows.
+  void full_attention(int cnt, const int* positions, const uint16_t* qb, float* out) const {
+    std::vector<float> Qf((size_t)cnt * Hq * d);
+    for (size_t i = 0; i < Qf.size(); ++i) Qf[i] = bf16_to_f32(qb[i]);
+    run_heads(Hq, [&](int h) {
+      int g = h / G;
+      for (int r = 0; r < cnt; ++r) {
+        std::vector<std::pair<int, int>> ranges{{0, positions[r] + 1}};
+        attend_row(&Qf[((size_t)r * Hq + h) * d], g, ranges, &out[((size_t)r * Hq + h) * d]);
+      }
+    });
+  }
+};
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// C interface for the ctypes wrapper
+extern "C" {
+
+void* orc_create(const Params* p) {
+  if (!p || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads) return nullptr;
+  if (p->head_dim < 1 || p->chunk < 1 || p->window < 1 || p->n_sink < 1 || p->top_k < 1) return nullptr;
+  if (p->reps_per_span < 1 || p->max_spans_per_region < 1 || p->max_tokens < 1) return nullptr;
+  return new Stream(*p);
+}
+void orc_destroy(void* h) { delete (Stream*)h; }
+
+int orc_prefill_local(void* h, int n, const uint16_t* q, const uint16_t* k, const uint16_t* v) {
+  return ((Stream*)h)->prefill_local(n, q, k, v);
+}
+void orc_prefill_retrieve(void* h) { ((Stream*)h)->prefill_retrieve(); }
+void orc_prefill_attend(void* h, int r0, int r1, float* out) { ((Stream*)h)->prefill_attend(r0, r1, out); }
+int orc_decode_retrieve(void* h, const uint16_t* q, const uint16_t* k, const uint16_t* v) {
+  return ((Stream*)h)->decode_retrieve(q, k, v);
+}
+void orc_decode_attend(void* h, float* out) { ((Stream*)h)->decode_attend(out); }
+void orc_full_attention(void* h, int cnt, const int* pos, const uint16_t* q, float* out) {
+  ((Stream*)h)->full_attention(cnt, pos, q, out);
+}
+
+// --- state access -----------------------------------------------------------
+int orc_tokens(void* h) { return ((Stream*)h)->t; }
+int orc_evicted_end(void* h) { return ((Stream*)h)->E; }
+int orc_num_spans(void* h) { return (int)((Stream*)h)->spans.size(); }
+void orc_get_spans(void* h, int* start_len) {
+  Stream* s = (Stream*)h;
+  for (size_t i = 0; i < s->spans.size(); ++i) {
+    start_len[2 * i] = s->spans[i].start;
+    start_len[2 * i + 1] = s->spans[i].len;
+  }
+}
+void orc_get_index(void* h, uint16_t* kr) {  // [span][Hkv][d] bf16 bits
+  Stream* s = (Stream*)h;
+  std::memcpy(kr, s->KR.data(), s->KR.size() * sizeof(uint16_t));
+}
+int orc_num_pending_regions(void* h) { return (int)((Stream*)h)->pending.size(); }
+// region r of the pending queue (0 = oldest): returns span count, writes {start,end} and spans
+int orc_get_pending(void* h, int r, int* start_end, int* start_len, int cap) {
+  Stream* s = (Stream*)h;
+  if (r < 0 || r >= (int)s->pending.size()) return -1;
+  const Region& reg = s->pending[r];
+  start_end[0] = reg.start;
+  start_end[1] = reg.end;
+  int c = (int)reg.spans.size();
+  for (int i = 0; i < c && i < cap; ++i) {
+    start_len[2 * i] = reg.spans[i].start;
+    start_len[2 * i + 1] = reg.spans[i].len;
+  }
+  return c;
+}
+// replace the spans of the newest pending region (re-synchronisation after a tolerated near-tie)
+int orc_set_newest_spans(void* h, const int* start_len, int cnt) {
+  Stream* s = (Stream*)h;
+  if (s->pending.empty()) return -1;
+  Region& reg = s->pending.back();
+  int pos = reg.start;
+  for (int i = 0; i < cnt; ++i) {
+    if (start_len[2 * i] != pos || start_len[2 * i + 1] < 1) return -1;
+    pos += start_len[2 * i + 1];
+  }
+  if (pos != reg.end) return -1;
+  reg.spans.clear();
+  for (int i = 0; i < cnt; ++i) reg.spans.push_back(Span{start_len[2 * i], start_len[2 * i + 1]});
+  return 0;
+}
+void orc_get_votes(void* h, int lo, int hi, int64_t* out) {
+  Stream* s = (Stream*)h;
+  for (int i = lo; i < hi; ++i) out[i - lo] = s->votes[i];
+}
+// current call
+int orc_region_len(void* h) { return ((Stream*)h)->m; }
+int orc_region_start(void* h) { return ((Stream*)h)->reg_start; }
+void orc_get_map(void* h, int32_t* Mq) {
+  Stream* s = (Stream*)h;
+  std::memcpy(Mq, s->Mq.data(), s->Mq.size() * sizeof(int32_t));
+}
+int64_t orc_get_theta_q(void* h) { return ((Stream*)h)->thq; }
+double orc_get_seg_gap(void* h) { return ((Stream*)h)->seg_gap; }
+int orc_num_query_reps(void* h) { return ((Stream*)h)->J; }
+void orc_get_query_reps(void* h, float* u) {  // [Hkv][J][d]
+  Stream* s = (Stream*)h;
+  std::memcpy(u, s->u.data(), s->u.size() * sizeof(float));
+}
+void orc_get_query_rep_tokens(void* h, int* tok) {  // [J][reps]
+  Stream* s = (Stream*)h;
+  std::memcpy(tok, s->qrep_tok.data(), s->qrep_tok.size() * sizeof(int));
+}
+void orc_get_scores(void* h, float* sc) {  // [Hkv][Ns]
+  Stream* s = (Stream*)h;
+  std::memcpy(sc, s->score.data(), s->score.size() * sizeof(float));
+}
+void orc_get_selected(void* h, int* ids, double* gaps) {  // [Hkv][top_k], [Hkv]
+  Stream* s = (Stream*)h;
+  std::memcpy(ids, s->sel.data(), s->sel.size() * sizeof(int));
+  if (gaps) std::memcpy(gaps, s->cut_gap.data(), s->cut_gap.size() * sizeof(double));
+}
+void orc_set_selected(void* h, const int* ids) {
+  Stream* s = (Stream*)h;
+  std::memcpy(s->sel.data(), ids, s->sel.size() * sizeof(int));
+}
+
+// --- stateless pieces, exposed so that each can be pinned on its own ---------
+int64_t orc_theta_q(const int32_t* Mq, int m, int mode, float theta, int Hq) {
+  return theta_q(Mq, m, m, mode, theta, Hq);
+}
+void orc_ta_scores(const int32_t* Mq, int m, int64_t thq, int64_t* S) {  // S[x*m+y], x<=y
+  std::vector<int64_t> s;
+  ta_scores(Mq, m, m, thq, s);
+  std::memcpy(S, s.data(), s.size() * sizeof(int64_t));
+}
+int orc_segment_map(const int32_t* Mq, int m, int64_t thq, int C, int* start_len, int cap, double* gap) {
+  std::vector<Span> sp;
+  segment_map(Mq, m, m, thq, C, sp, gap);
+  for (size_t i = 0; i < sp.size() && (int)i < cap; ++i) {
+    start_len[2 * i] = sp[i].start;
+    start_len[2 * i + 1] = sp[i].len;
+  }
+  return (int)sp.size();
+}
+void orc_top_k(const float* score, int n, int k, int* ids, double* gap) { top_k(score, n, k, ids, gap); }
+uint16_t orc_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
+
+}  // extern "C"
