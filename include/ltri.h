@@ -1,0 +1,165 @@
+/* ltri.h -- C ABI of the B200 (sm_100a) streaming span-retrieval attention library.
+ *
+ * The library implements, per streamed chunk or decode step, the hot path of Ltri-LLM
+ * (arXiv 2412.04757): segment the KV stream into semantic spans from the triangular
+ * pattern of the local attention map (Sec. 3.2, Eq. 1-5, App. "NMS Input Filtration"),
+ * keep one representative key (or a small key set) per span in a device-resident index
+ * (Sec. 3.3.1, Eq. 6), score the queries against the index and take the top-k spans
+ * (Sec. 3.4 step 2, Eq. 7-8), gather those spans' K/V and run exact softmax attention
+ * over [sink | retrieved spans | local window | current tokens] (Sec. 3.4 step 3).
+ *
+ * Conventions
+ *  - All tensor arguments are DEVICE pointers to bf16 unless stated otherwise, 16-byte
+ *    aligned, dense row-major in the layout written beside the argument.
+ *  - The caller owns every buffer, including the arena all library state lives in; the
+ *    library never allocates or frees device memory.  The handle owns host metadata only.
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*) and return
+ *    without synchronising unless stated.  All calls on one context must use one stream
+ *    (or be ordered by the caller).
+ *  - Return value: 0 (LTRI_OK) or a negative LTRI_E* code.  Parameter, state and capacity
+ *    errors are detected on the host before anything is launched and leave the context
+ *    unchanged.  Device-side checks record a code in a status word read by
+ *    ltri_sync_status; nothing traps or spins without bound.
+ */
+#ifndef LTRI_H_
+#define LTRI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  LTRI_OK = 0,
+  LTRI_EINVAL = -1,    /* bad geometry / parameter / null or misaligned pointer */
+  LTRI_ECAPACITY = -2, /* tokens, sequences, spans or arena size exceeded */
+  LTRI_ESTATE = -3,    /* call order violated (e.g. prefill after decode, layers out of step) */
+  LTRI_ECUDA = -4,     /* a CUDA runtime call failed; see ltri_last_cuda_error */
+  LTRI_EDEVICE = -5,   /* a device-side bounds check failed */
+  LTRI_ETIMEOUT = -6   /* a bounded device-side wait expired */
+};
+
+typedef struct ltri_ctx ltri_ctx; /* opaque host-side handle */
+
+typedef struct {
+  int32_t n_layers, n_q_heads, n_kv_heads, head_dim; /* head_dim must be 128; n_q_heads % n_kv_heads == 0,
+                                                        group size n_q_heads/n_kv_heads in {1,2,4,8} */
+  int32_t max_seqs;                                  /* independent sequences held at once */
+  int64_t max_tokens;                                /* per-sequence capacity, prefill + decode */
+  int32_t chunk;                                     /* max tokens per prefill call, 16..1024, multiple of 16 */
+  int32_t window;                                    /* local window L_win >= 1 (Sec. 3.4) */
+  int32_t n_sink;                                    /* initial tokens L_init, 1..chunk */
+  int32_t top_k;                                     /* spans retrieved per (layer, KV head), 1..64 (Eq. 8) */
+  int32_t reps_per_span;                             /* index vectors per span, 1..8; 0 -> 1 (Sec. 3.3.1) */
+  int32_t max_spans_per_region;                      /* NMS keeps at most this many per call; 0 -> chunk/32 */
+  int32_t theta_mode;                                /* 0: theta is an absolute head-mean probability,
+                                                        1: theta is a quantile level of the region map (Eq. 5) */
+  float theta;                                       /* mode 1 default 0.90 */
+  float softmax_scale;                               /* 0 -> 1/sqrt(head_dim) */
+  uint32_t flags;                                    /* LTRI_FLAG_* */
+  void* arena;                                       /* caller-owned device memory, 256-byte aligned */
+  size_t arena_bytes;                                /* >= ltri_arena_bytes(params) */
+} ltri_params;
+
+enum { LTRI_FLAG_NONE = 0 };
+
+typedef struct {
+  int64_t tokens;          /* tokens appended so far (prefill + decode) */
+  int64_t evicted_end;     /* E: tokens [n_sink, E) are covered by indexed spans */
+  int32_t n_spans;         /* indexed spans N_s */
+  int32_t n_pending_regions;
+  int64_t index_bytes;     /* N_s * n_kv_heads * head_dim * 2 */
+  int64_t retrieved_tokens; /* sum of the lengths of the spans selected by the last call, over KV heads */
+  int32_t last_call_spans; /* spans the last prefill call cut its region into */
+  int32_t reserved;
+} ltri_stats;
+
+/* Bytes of device memory the arena must provide for these parameters (host only; the
+ * `arena` and `arena_bytes` fields are ignored).  Returns 0 if the parameters are invalid. */
+size_t ltri_arena_bytes(const ltri_params* p);
+
+/* Create a context over the caller's arena and initialise its device state on
+ * `cuda_stream` (synchronises that stream once).  Streaming attention with parameters
+ * init / window / chunk / top-K as in Sec. "Implementation Details". */
+int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out);
+
+/* Free the host handle.  Device memory stays with the caller. */
+int ltri_destroy(ltri_ctx* ctx);
+
+/* Forget all tokens of one sequence so that its slot can stream a new context. */
+int ltri_reset_sequence(ltri_ctx* ctx, int seq, void* cuda_stream);
+
+/* One streamed prefill call (Sec. 3.4, steps 1-3) for `n_tokens` (1..chunk) new tokens of
+ * sequence `seq`, for layers [layer_begin, layer_begin+layer_count).
+ *   q   [layer_count][n_tokens][n_q_heads ][head_dim]
+ *   k,v [layer_count][n_tokens][n_kv_heads][head_dim]   (copied into the library's cache)
+ *   out [layer_count][n_tokens][n_q_heads ][head_dim]   (fully overwritten)
+ * Per layer: regions that left the window are indexed (Eq. 6); the local map over
+ * [sink | local | current] is computed and the call's own region is segmented (Eq. 1-5);
+ * query representatives are scored against the index and the top-k spans selected
+ * (Eq. 7-8); attention runs over [sink | selected spans | local | current (causal)].
+ * Each (sequence, layer) is its own stream: its tokens must arrive in order, and a layer
+ * that already decoded cannot prefill again (LTRI_ESTATE).  The layers of one call must
+ * all be at the same position. */
+int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q,
+                       const void* k, const void* v, void* out, void* cuda_stream);
+
+/* One decode step (the block becomes a single token, Sec. 3.5) for `n_seqs` sequences.
+ *   seq_ids  HOST array [n_seqs] of distinct sequence slots
+ *   q   [n_seqs][layer_count][n_q_heads ][head_dim]
+ *   k,v [n_seqs][layer_count][n_kv_heads][head_dim]
+ *   out [n_seqs][layer_count][n_q_heads ][head_dim]
+ * Appends the token, scores the summed query of each KV-head group against the index,
+ * selects top-k spans and attends over [sink | selected spans | every token since the
+ * last eviction].  Decode never evicts, votes or segments. */
+int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int layer_begin, int layer_count,
+                     const void* q, const void* k, const void* v, void* out, void* cuda_stream);
+
+/* ---- introspection (synchronise `cuda_stream`; HOST output buffers) ---- */
+
+/* Indexed spans of (seq, layer) as {start,len} pairs in token order; *n_out = N_s (even if > cap). */
+int ltri_get_spans(ltri_ctx* ctx, int seq, int layer, int32_t* start_len_pairs, int cap, int* n_out, void* cuda_stream);
+/* Spans of the regions still inside the window, oldest first, as {start,len} pairs. */
+int ltri_get_pending_spans(ltri_ctx* ctx, int seq, int layer, int32_t* start_len_pairs, int cap, int* n_out,
+                           void* cuda_stream);
+/* Span ids chosen by the last call, ascending, -1 padded: ids[n_kv_heads][top_k]. */
+int ltri_get_selected(ltri_ctx* ctx, int seq, int layer, int32_t* ids, void* cuda_stream);
+int ltri_get_stats(ltri_ctx* ctx, int seq, int layer, ltri_stats* out, void* cuda_stream);
+/* First device-side error recorded since the last call of this function (then cleared). */
+int ltri_sync_status(ltri_ctx* ctx, void* cuda_stream);
+/* cudaError_t of the last failed runtime call (0 if none). */
+int ltri_last_cuda_error(const ltri_ctx* ctx);
+const char* ltri_strerror(int code);
+
+/* ---- debug / test entry points ---- */
+
+enum {
+  LTRI_BUF_MAP = 1,      /* int32 [chunk][chunk]: the last prefill call's head-summed Q20 region map (row-major,
+                            leading dimension chunk; entries above the diagonal are unspecified) */
+  LTRI_BUF_VOTES = 2,    /* int64 [max_tokens]: accumulated votes v_x in Q20 units (Eq. 6) */
+  LTRI_BUF_INDEX = 3,    /* bf16  [n_kv_heads][span_capacity][head_dim]: the span index K^R */
+  LTRI_BUF_THETA = 4,    /* int64 [1]: theta of the last prefill call in Q20 head-sum units */
+  LTRI_BUF_SCORES = 5,   /* float [n_kv_heads][span_capacity]: similarity scores of the last call (Eq. 7) */
+  LTRI_BUF_QREPS = 6,    /* float [n_kv_heads][2*max_spans_per_region+1][head_dim]: summed query representatives */
+  LTRI_BUF_ROWSTAT = 7   /* float [chunk][n_q_heads][2]: row max (raw dot-product units) and row sum of the
+                            local softmax of the last prefill call */
+};
+/* Copy an internal buffer of (seq, layer) to HOST memory `dst`; *bytes_out = full size.  Synchronises. */
+int ltri_debug_read(ltri_ctx* ctx, int what, int seq, int layer, void* dst, size_t cap_bytes, size_t* bytes_out,
+                    void* cuda_stream);
+/* Span capacity per (seq, layer) (leading dimension of LTRI_BUF_INDEX / LTRI_BUF_SCORES). */
+int ltri_span_capacity(const ltri_ctx* ctx);
+
+/* Run the segmenter (Eq. 4-5 cumulative sums, anti-diagonal filter, greedy NMS with IoU threshold 0, gap
+ * fill) on a caller-supplied HOST map Mq [m][m] int32 row-major (lower triangle used, 1 <= m <= chunk).
+ * theta_mode/theta as in ltri_params, except mode 2: `theta_q` is given directly in map units.
+ * Writes {start,len} pairs (HOST) partitioning [0,m); uses layer 0's scratch of the context.  Synchronises. */
+int ltri_debug_segment_map(ltri_ctx* ctx, const int32_t* Mq, int m, int theta_mode, float theta, int64_t theta_q,
+                           int max_spans, int32_t* start_len_pairs, int cap, int* n_out, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LTRI_H_ */

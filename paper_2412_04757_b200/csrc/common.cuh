@@ -1,0 +1,175 @@
+// Shared declarations of the ltri CUDA library (sm_100a): the device-side view of a
+// context and the host launch wrappers of every kernel file.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ltri {
+
+constexpr int kD = 128;               // head_dim (fixed)
+constexpr int kQBits = 20;            // fixed-point fraction bits of the local attention map
+constexpr float kQScale = 1048576.0f;
+constexpr int kMaxReps = 8;
+constexpr int kMaxTopK = 64;
+constexpr int kMaxDecSplit = 32;
+constexpr int kTokPad = 128;          // rows of slack after every K/V slab so tile over-reads stay inside it
+
+// Device-side view of one context.  Passed to kernels by value.
+struct DevCtx {
+  int NL, Hq, Hkv, G, NS;
+  long long Tpad;        // row capacity of a per-(seq,layer,kv-head) K/V slab (max_tokens + slack)
+  long long Tmax;
+  int chunk, W, Ls, topk, reps, C, Jmax, cap, slots;
+  int theta_mode;
+  float theta, scale;
+  // persistent state
+  __nv_bfloat16* Kc;     // [NS][NL][Hkv][Tpad][128]
+  __nv_bfloat16* Vc;
+  long long* votes;      // [NS][NL][Tpad]
+  int* span_start;       // [NS][NL][cap]
+  int* span_len;
+  int* n_spans;          // [NS][NL]
+  __nv_bfloat16* KR;     // [NS][NL][Hkv][cap][128]
+  int* pend_start;       // [NS][NL][slots][Jmax]
+  int* pend_len;
+  int* pend_cnt;         // [NS][NL][slots]
+  int* sel;              // [NS][NL][Hkv][topk]  ascending ids, -1 padded
+  long long* sel_tokens; // [NS][NL]  retrieved tokens of the last call, summed over KV heads
+  // per-layer scratch of the prefill call in flight
+  int* Mq;               // [NL][chunk][chunk]
+  long long* Rsuf;       // [NL][chunk][chunk]
+  long long* best;       // [NL][2*chunk]
+  long long* thetaq;     // [NL]
+  float2* rowstat;       // [NL][chunk][Hq]   (row max in raw dot units, row sum)
+  float* Oacc;           // [NL][chunk][Hq][128]  unnormalised accumulator of the local part
+  float* u;              // [NL][Hkv][Jmax][128]  summed query representatives
+  int* Jcnt;             // [NL]
+  // per-(seq,layer) scratch
+  float* scores;         // [NS*NL][Hkv][cap]
+  int* rng_start;        // [NS*NL][Hkv][topk+2]
+  int* rng_len;
+  int* rng_cnt;          // [NS*NL][Hkv]
+  float* dec_part;       // [NS*NL][Hq][kMaxDecSplit][128+2]
+  int* status;           // [4]: first error code, detail...
+};
+
+__host__ __device__ inline size_t unit_of(const DevCtx& c, int seq, int layer) { return (size_t)seq * c.NL + layer; }
+
+// Decode batch descriptor (passed by value; at most 64 sequences per launch).
+constexpr int kDecBatch = 64;
+struct DecBatch {
+  int n;
+  int seq[kDecBatch];
+  int pos[kDecBatch];        // position of the new token
+  int loc_begin[kDecBatch];  // E' of the sequence/layer
+  int src[kDecBatch];        // index into the caller's [n_seqs] arrays
+};
+
+struct EvictArgs {
+  int seq, layer_begin;
+  int nslots;
+  int slot[8];
+};
+
+struct PrefillArgs {
+  int seq, layer_begin, layer_count;
+  int n, t0;
+  int sink_end, loc_begin;  // sink = [0,sink_end), local = [loc_begin,t0)
+  int reg_start, m;         // region [reg_start, t0+n), m tokens
+  int slot;                 // pending slot of this region (-1 if the region is empty)
+  const __nv_bfloat16* q;   // [layer_count][n][Hq][128]
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  __nv_bfloat16* out;
+};
+
+// ---- launch wrappers (each returns the cudaError_t of the launch) -------------------
+cudaError_t launch_init(const DevCtx& c, int seq /* -1: all */, cudaStream_t s);
+cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
+cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
+                                 const __nv_bfloat16* k, const __nv_bfloat16* v, cudaStream_t s);
+cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_count, cudaStream_t s);
+// segmenter on Mq of the given layers; writes spans (absolute tokens = reg_start + x) into pending slot `slot`
+// and, when q != nullptr, the summed query representatives of every span.  theta_mode 0/2: theta_q_abs is used.
+cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_count, int m, int reg_start, int slot,
+                           int theta_mode, float theta, long long theta_q_abs, int max_spans, int n, int t0,
+                           const __nv_bfloat16* q, cudaStream_t s);
+cudaError_t launch_score_prefill(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s);
+cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
+cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
+                                const __nv_bfloat16* q, int span_bound, cudaStream_t s);
+cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s);
+
+// prefill attention.  phase 0: local part over sink|local|cur, stores state (+ final output if `final`);
+// phase 1: continues from the stored state over the selected spans and writes the output.
+cudaError_t launch_attn_prefill(const DevCtx& c, const PrefillArgs& a, int phase, bool final, cudaStream_t s);
+cudaError_t launch_map_pass(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
+
+cudaError_t launch_decode_attn(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
+                               const __nv_bfloat16* q, __nv_bfloat16* out, int nsplit, cudaStream_t s);
+
+// ---- small device helpers --------------------------------------------------------------
+__device__ __forceinline__ void set_status(const DevCtx& c, int code, int detail) {
+  if (atomicCAS(&c.status[0], 0, code) == 0) c.status[1] = detail;
+}
+
+__device__ __forceinline__ long long shfl_xor_ll(long long v, int m) {
+  int lo = __shfl_xor_sync(0xffffffffu, (int)(v & 0xffffffffll), m);
+  int hi = __shfl_xor_sync(0xffffffffu, (int)(v >> 32), m);
+  return ((long long)hi << 32) | (unsigned int)lo;
+}
+__device__ __forceinline__ long long shfl_up_ll(long long v, int d) {
+  int lo = __shfl_up_sync(0xffffffffu, (int)(v & 0xffffffffll), d);
+  int hi = __shfl_up_sync(0xffffffffu, (int)(v >> 32), d);
+  return ((long long)hi << 32) | (unsigned int)lo;
+}
+__device__ __forceinline__ long long shfl_ll(long long v, int src) {
+  int lo = __shfl_sync(0xffffffffu, (int)(v & 0xffffffffll), src);
+  int hi = __shfl_sync(0xffffffffu, (int)(v >> 32), src);
+  return ((long long)hi << 32) | (unsigned int)lo;
+}
+
+// Warp-cooperative choice of the min(reps,len) tokens of [start,start+len) with the largest votes
+// (ties -> lower token index), returned ascending in toks[] (Eq. 6 / Sec. 3.3.1).  All lanes get the result.
+__device__ inline int select_reps(const long long* __restrict__ votes, int start, int len, int reps, int* toks) {
+  const int lane = threadIdx.x & 31;
+  int cnt = reps < len ? reps : len;
+  for (int r = 0; r < cnt; ++r) {
+    long long bv = (long long)0x8000000000000000ull;
+    int bi = 0x7fffffff;
+    for (int i = lane; i < len; i += 32) {
+      int tok = start + i;
+      bool used = false;
+      for (int q = 0; q < r; ++q) used |= (toks[q] == tok);
+      if (used) continue;
+      long long v = votes[tok];
+      if (v > bv || (v == bv && tok < bi)) {
+        bv = v;
+        bi = tok;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      long long ov = shfl_xor_ll(bv, o);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ov > bv || (ov == bv && oi < bi)) {
+        bv = ov;
+        bi = oi;
+      }
+    }
+    toks[r] = bi;
+  }
+  for (int a = 1; a < cnt; ++a) {  // insertion sort, ascending token
+    int x = toks[a], b = a - 1;
+    while (b >= 0 && toks[b] > x) {
+      toks[b + 1] = toks[b];
+      --b;
+    }
+    toks[b + 1] = x;
+  }
+  return cnt;
+}
+
+}  // namespace ltri

@@ -1,0 +1,679 @@
+// State kernels: cache append, eviction + span index build (Sec. 3.3.1, Eq. 6), span segmenter
+// (Eq. 4-5, App. "NMS Input Filtration"), query representatives, similarity scores (Eq. 7) and
+// top-k selection (Eq. 8).  All segmentation arithmetic is integer and order-independent.
+#include "common.cuh"
+
+namespace ltri {
+
+// ------------------------------------------------------------------------------------------
+__global__ void k_init(DevCtx c, int seq) {
+  const int s0 = seq < 0 ? 0 : seq, s1 = seq < 0 ? c.NS : seq + 1;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (int s = s0; s < s1; ++s) {
+    const size_t u0 = (size_t)s * c.NL;
+    for (size_t i = tid; i < (size_t)c.NL; i += stride) {
+      c.n_spans[u0 + i] = 0;
+      c.sel_tokens[u0 + i] = 0;
+    }
+    for (size_t i = tid; i < (size_t)c.NL * c.slots; i += stride) c.pend_cnt[u0 * c.slots + i] = 0;
+    for (size_t i = tid; i < (size_t)c.NL * c.Hkv * c.topk; i += stride) c.sel[u0 * c.Hkv * c.topk + i] = -1;
+    for (size_t i = tid; i < (size_t)c.NL * c.Hkv; i += stride) c.rng_cnt[u0 * c.Hkv + i] = 0;
+  }
+  if (seq < 0 && tid < 4) c.status[tid] = 0;
+  if (seq < 0)
+    for (size_t i = tid; i < (size_t)c.NL; i += stride) c.Jcnt[i] = 0;
+}
+
+cudaError_t launch_init(const DevCtx& c, int seq, cudaStream_t s) {
+  k_init<<<64, 256, 0, s>>>(c, seq);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// a0: copy the call's K/V rows into the cache slabs; 16 threads move one 256-byte row.
+__global__ void k_append_prefill(DevCtx c, PrefillArgs a) {
+  const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int c16 = gid & 15;
+  size_t row = gid >> 4;  // over [layer_count][n][Hkv]
+  const size_t nrows = (size_t)a.layer_count * a.n * c.Hkv;
+  if (row >= nrows) return;
+  const int g = row % c.Hkv;
+  const int r = (row / c.Hkv) % a.n;
+  const int l = row / ((size_t)c.Hkv * a.n);
+  const size_t unit = unit_of(c, a.seq, a.layer_begin + l);
+  const size_t dst = ((unit * c.Hkv + g) * c.Tpad + (a.t0 + r)) * kD + c16 * 8;
+  const size_t src = row * kD + c16 * 8;
+  *reinterpret_cast<uint4*>(c.Kc + dst) = *reinterpret_cast<const uint4*>(a.k + src);
+  *reinterpret_cast<uint4*>(c.Vc + dst) = *reinterpret_cast<const uint4*>(a.v + src);
+  if (g == 0 && c16 == 0) c.votes[unit * c.Tpad + a.t0 + r] = 0;
+}
+
+cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
+  const size_t threads = (size_t)a.layer_count * a.n * c.Hkv * 16;
+  k_append_prefill<<<(unsigned)((threads + 255) / 256), 256, 0, s>>>(c, a);
+  return cudaGetLastError();
+}
+
+__global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer_count,
+                                const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v) {
+  const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int c16 = gid & 15;
+  size_t row = gid >> 4;  // over [b.n][layer_count][Hkv]
+  if (row >= (size_t)b.n * layer_count * c.Hkv) return;
+  const int g = row % c.Hkv;
+  const int l = (row / c.Hkv) % layer_count;
+  const int bi = row / ((size_t)c.Hkv * layer_count);
+  const size_t unit = unit_of(c, b.seq[bi], layer_begin + l);
+  const size_t dst = ((unit * c.Hkv + g) * c.Tpad + b.pos[bi]) * kD + c16 * 8;
+  const size_t src = (((size_t)b.src[bi] * layer_count + l) * c.Hkv + g) * kD + c16 * 8;
+  *reinterpret_cast<uint4*>(c.Kc + dst) = *reinterpret_cast<const uint4*>(k + src);
+  *reinterpret_cast<uint4*>(c.Vc + dst) = *reinterpret_cast<const uint4*>(v + src);
+  if (g == 0 && c16 == 0) c.votes[unit * c.Tpad + b.pos[bi]] = 0;
+}
+
+cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int,
+                                 const __nv_bfloat16* k, const __nv_bfloat16* v, cudaStream_t s) {
+  const size_t threads = (size_t)b.n * layer_count * c.Hkv * 16;
+  k_append_decode<<<(unsigned)((threads + 255) / 256), 256, 0, s>>>(c, b, layer_begin, layer_count, k, v);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// a1: regions that left the window: every span gets its index vector, the bf16 sum of the keys of
+// its most voted token(s), and is appended to the span table.  One CTA per layer, one warp per span.
+__global__ void __launch_bounds__(256) k_evict_index(DevCtx c, EvictArgs a) {
+  const int layer = a.layer_begin + blockIdx.x;
+  const size_t unit = unit_of(c, a.seq, layer);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int base = c.n_spans[unit];
+  const long long* votes = c.votes + unit * c.Tpad;
+  int off = 0;
+  for (int si = 0; si < a.nslots; ++si) {
+    const size_t ps = (unit * c.slots + a.slot[si]) * c.Jmax;
+    const int cnt = c.pend_cnt[unit * c.slots + a.slot[si]];
+    for (int i = warp; i < cnt; i += nwarps) {
+      const int start = c.pend_start[ps + i], len = c.pend_len[ps + i];
+      const int dst = base + off + i;
+      if (dst >= c.cap) {
+        if (lane == 0) set_status(c, -2, dst);
+        continue;
+      }
+      if (lane == 0) {
+        c.span_start[unit * c.cap + dst] = start;
+        c.span_len[unit * c.cap + dst] = len;
+      }
+      int toks[kMaxReps];
+      const int nrep = select_reps(votes, start, len, c.reps, toks);
+      for (int g = 0; g < c.Hkv; ++g) {
+        const __nv_bfloat16* kslab = c.Kc + ((unit * c.Hkv + g) * c.Tpad) * kD;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int r = 0; r < nrep; ++r) {
+          const uint2 raw = *reinterpret_cast<const uint2*>(kslab + (size_t)toks[r] * kD + lane * 4);
+          const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+          const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+          acc[0] += __bfloat162float(p0.x);
+          acc[1] += __bfloat162float(p0.y);
+          acc[2] += __bfloat162float(p1.x);
+          acc[3] += __bfloat162float(p1.y);
+        }
+        __nv_bfloat162 o0 = __floats2bfloat162_rn(acc[0], acc[1]);
+        __nv_bfloat162 o1 = __floats2bfloat162_rn(acc[2], acc[3]);
+        uint2 w;
+        w.x = *reinterpret_cast<uint32_t*>(&o0);
+        w.y = *reinterpret_cast<uint32_t*>(&o1);
+        *reinterpret_cast<uint2*>(c.KR + ((unit * c.Hkv + g) * c.cap + dst) * kD + lane * 4) = w;
+      }
+    }
+    off += cnt;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) c.n_spans[unit] = min(base + off, c.cap);
+}
+
+cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_count, cudaStream_t s) {
+  k_evict_index<<<layer_count, 256, 0, s>>>(c, a);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// a3 segmenter, step 1: exact rank selection of theta (quantile mode) over the causal entries of Mq.
+// 4-pass MSB radix select on sign-flipped 32-bit keys; one CTA per layer.
+__global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin, int m, long long rank) {
+  const int layer = layer_begin + blockIdx.x;
+  const int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
+  __shared__ unsigned hist[256];
+  __shared__ unsigned s_prefix;
+  __shared__ long long s_rank;
+  if (threadIdx.x == 0) {
+    s_prefix = 0;
+    s_rank = rank;
+  }
+  const int total = m * m;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+    __syncthreads();
+    const unsigned prefix = s_prefix;
+    const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+    for (int base = 0; base < total; base += blockDim.x) {
+      const int idx = base + threadIdx.x;
+      bool valid = false;
+      unsigned bin = 0;
+      if (idx < total) {
+        const int i = idx / m, j = idx - i * m;
+        if (j <= i) {
+          const unsigned key = (unsigned)Mq[(size_t)i * c.chunk + j] ^ 0x80000000u;
+          if ((key & himask) == prefix) {
+            valid = true;
+            bin = (key >> shift) & 255u;
+          }
+        }
+      }
+      // warp-aggregated histogram update (most entries of a sparse map share one bin)
+      const unsigned act = __ballot_sync(0xffffffffu, valid);
+      if (valid) {
+        const unsigned peers = __match_any_sync(act, bin);
+        if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      long long r = s_rank;
+      unsigned b = 0;
+      for (; b < 256; ++b) {
+        if (r < (long long)hist[b]) break;
+        r -= hist[b];
+      }
+      if (b > 255) b = 255;
+      s_rank = r;
+      s_prefix = prefix | (b << shift);
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) c.thetaq[layer] = (long long)(int)(s_prefix ^ 0x80000000u);
+}
+
+__global__ void k_theta_set(DevCtx c, int layer_begin, long long thq) { c.thetaq[layer_begin + blockIdx.x] = thq; }
+
+// step 2: suffix sums along each row of D = Mq - theta ("sum the right elements", Fig. 2):
+// Rsuf[i][x] = sum_{j=x..i} D[i][j].  One warp per row, 32-wide shuffle scans from the diagonal leftwards.
+__global__ void __launch_bounds__(256) k_seg_rowscan(DevCtx c, int layer_begin, int m) {
+  const int layer = layer_begin + blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int i = blockIdx.x * 8 + warp;
+  if (blockIdx.x == 0)
+    for (int t = threadIdx.x; t < 2 * c.chunk; t += blockDim.x) c.best[(size_t)layer * 2 * c.chunk + t] = 0;
+  if (i >= m) return;
+  const long long thq = c.thetaq[layer];
+  const int* row = c.Mq + ((size_t)layer * c.chunk + i) * c.chunk;
+  long long* out = c.Rsuf + ((size_t)layer * c.chunk + i) * c.chunk;
+  long long carry = 0;
+  for (int hi = i; hi >= 0; hi -= 32) {
+    const int x = hi - lane;  // lane 0 is the rightmost element of this group
+    long long v = x >= 0 ? (long long)row[x] - thq : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const long long t = shfl_up_ll(v, o);
+      if (lane >= o) v += t;
+    }
+    v += carry;
+    if (x >= 0) out[x] = v;
+    carry = shfl_ll(v, 31);
+  }
+}
+
+// step 3: prefix sums down each column ("sum the upper elements"): S(x,y) = sum_{i=x..y} Rsuf[i][x], and the
+// best point of every anti-diagonal x+y=c (max S, ties -> shorter span), kept only when S > 0.
+// A CTA owns 32 columns; thread (cx, ry) scans rows [ry*R, ry*R+R) of its column, a shared-memory scan over ry
+// supplies the offsets, and a second pass emits S.  key = (S << 10) | (1023 - (y-x)).
+__global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin, int m) {
+  extern __shared__ long long sm[];
+  long long* part = sm;             // [32 ry][32 cx]
+  long long* sbest = sm + 32 * 32;  // [m + 32]
+  const int layer = layer_begin + blockIdx.y;
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int x0 = blockIdx.x * 32, x = x0 + cx;
+  const int R = (m + 31) / 32;
+  const long long* Rs = c.Rsuf + (size_t)layer * c.chunk * c.chunk;
+  for (int t = threadIdx.x; t < m + 32; t += blockDim.x) sbest[t] = 0;
+  const int ylo = ry * R, yhi = min(m, ylo + R);
+  long long acc = 0;
+  if (x < m)
+    for (int y = max(ylo, x); y < yhi; ++y) acc += Rs[(size_t)y * c.chunk + x];
+  part[ry * 32 + cx] = acc;
+  __syncthreads();
+  if (ry == 0) {  // exclusive scan over ry for column cx
+    long long run = 0;
+    for (int r = 0; r < 32; ++r) {
+      const long long t = part[r * 32 + cx];
+      part[r * 32 + cx] = run;
+      run += t;
+    }
+  }
+  __syncthreads();
+  if (x < m) {
+    long long S = part[ry * 32 + cx];
+    for (int y = max(ylo, x); y < yhi; ++y) {
+      S += Rs[(size_t)y * c.chunk + x];
+      if (S > 0) {
+        const long long key = (S << 10) | (long long)(1023 - (y - x));
+        atomicMax(&sbest[x + y - 2 * x0], key);
+      }
+    }
+  }
+  __syncthreads();
+  long long* gbest = c.best + (size_t)layer * 2 * c.chunk;
+  for (int t = threadIdx.x; t < m + 32; t += blockDim.x) {
+    const long long key = sbest[t];
+    const int cd = 2 * x0 + t;
+    if (key > 0 && cd <= 2 * m - 2) atomicMax(&gbest[cd], key);
+  }
+}
+
+// step 4: sort the <= 2m-1 candidates by (S desc, length asc, start asc), greedy non-maximum suppression with
+// IoU threshold 0 until max_spans are kept, gap fill, store the region's spans in its pending slot; then the
+// query representatives of every span (Sec. 3.4 step 2): u[g][j] = sum_{h in g} sum_{rep tokens} q_h[tok].
+struct NmsArgs {
+  int seq, layer_begin, m, reg_start, slot, max_spans;
+  int n, t0;                 // query tensor geometry (q == nullptr: skip the representatives)
+  const __nv_bfloat16* q;
+};
+
+__global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
+  __shared__ long long skey[2048];
+  __shared__ short scd[2048];
+  __shared__ int kx[kMaxTopK], ky[kMaxTopK];
+  __shared__ int s_kept;
+  __shared__ int out_start[2 * kMaxTopK + 1], out_len[2 * kMaxTopK + 1];
+  __shared__ int s_nout;
+  const int layer = a.layer_begin + blockIdx.x;
+  const size_t unit = unit_of(c, a.seq, layer);
+  const int m = a.m;
+  const int ncand = 2 * m - 1;
+  int npow = 1;
+  while (npow < ncand) npow <<= 1;
+  const long long* gbest = c.best + (size_t)layer * 2 * c.chunk;
+  for (int t = threadIdx.x; t < npow; t += blockDim.x) {
+    skey[t] = t < ncand ? gbest[t] : 0;
+    scd[t] = (short)t;
+  }
+  __syncthreads();
+  // bitonic sort, "a before b" iff key larger, or equal key and smaller anti-diagonal
+  for (int k = 2; k <= npow; k <<= 1)
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int t = threadIdx.x; t < npow; t += blockDim.x) {
+        const int p = t ^ j;
+        if (p > t) {
+          const long long ka = skey[t], kb = skey[p];
+          const short ca = scd[t], cb = scd[p];
+          const bool a_first = ka > kb || (ka == kb && ca < cb);
+          const bool up = (t & k) == 0;
+          if (up ? !a_first : a_first) {
+            skey[t] = kb;
+            skey[p] = ka;
+            scd[t] = cb;
+            scd[p] = ca;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  // greedy NMS by warp 0, 32 candidates per round
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    int kept = 0;
+    for (int base = 0; base < ncand && kept < a.max_spans; base += 32) {
+      const int idx = base + lane;
+      const long long key = idx < ncand ? skey[idx] : 0;
+      const int len = 1023 - (int)(key & 1023);
+      const int x = ((int)scd[idx < ncand ? idx : 0] - len) >> 1;
+      const int y = x + len;
+      bool alive = key > 0;
+      if (__ballot_sync(0xffffffffu, alive) == 0) break;  // sorted: nothing positive follows
+      for (int q = 0; q < kept; ++q) alive = alive && (y < kx[q] || x > ky[q]);
+      unsigned mask = __ballot_sync(0xffffffffu, alive);
+      while (mask && kept < a.max_spans) {
+        const int f = __ffs(mask) - 1;
+        const int fx = __shfl_sync(0xffffffffu, x, f), fy = __shfl_sync(0xffffffffu, y, f);
+        if (lane == 0) {
+          kx[kept] = fx;
+          ky[kept] = fy;
+        }
+        ++kept;
+        alive = alive && lane != f && (y < fx || x > fy);
+        mask = __ballot_sync(0xffffffffu, alive);
+      }
+      __syncwarp();
+    }
+    __syncwarp();
+    // order the kept spans by start (rank sort), then gap fill
+    int rank0 = 0, rank1 = 0;
+    const int x0 = lane < kept ? kx[lane] : 0x7fffffff;
+    const int x1 = lane + 32 < kept ? kx[lane + 32] : 0x7fffffff;
+    for (int q = 0; q < kept; ++q) {
+      rank0 += kx[q] < x0;
+      rank1 += kx[q] < x1;
+    }
+    const int y0 = lane < kept ? ky[lane] : 0, y1 = lane + 32 < kept ? ky[lane + 32] : 0;
+    __syncwarp();
+    if (lane < kept) kx[rank0] = x0;
+    if (lane + 32 < kept) kx[rank1] = x1;
+    __syncwarp();
+    if (lane < kept) ky[rank0] = y0;
+    if (lane + 32 < kept) ky[rank1] = y1;
+    __syncwarp();
+    if (lane == 0) {
+      int pos = 0, no = 0;
+      for (int q = 0; q < kept; ++q) {
+        if (kx[q] > pos) {
+          out_start[no] = pos;
+          out_len[no++] = kx[q] - pos;
+        }
+        out_start[no] = kx[q];
+        out_len[no++] = ky[q] - kx[q] + 1;
+        pos = ky[q] + 1;
+      }
+      if (pos < m) {
+        out_start[no] = pos;
+        out_len[no++] = m - pos;
+      }
+      s_nout = no;
+      s_kept = kept;
+    }
+  }
+  __syncthreads();
+  const int nout = s_nout;
+  const size_t ps = (unit * c.slots + a.slot) * c.Jmax;
+  if (nout > c.Jmax) {
+    if (threadIdx.x == 0) set_status(c, -5, nout);
+    return;
+  }
+  for (int t = threadIdx.x; t < nout; t += blockDim.x) {
+    c.pend_start[ps + t] = a.reg_start + out_start[t];
+    c.pend_len[ps + t] = out_len[t];
+  }
+  if (threadIdx.x == 0) {
+    c.pend_cnt[unit * c.slots + a.slot] = nout;
+    c.Jcnt[layer] = a.q ? nout : 0;
+  }
+  if (!a.q) return;
+  // query representatives: one warp per span
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const long long* votes = c.votes + unit * c.Tpad;
+  const __nv_bfloat16* q = a.q + (size_t)blockIdx.x * a.n * c.Hq * kD;
+  for (int j = warp; j < nout; j += nwarps) {
+    int toks[kMaxReps];
+    const int nrep = select_reps(votes, a.reg_start + out_start[j], out_len[j], c.reps, toks);
+    for (int g = 0; g < c.Hkv; ++g) {
+      float ug[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int hh = 0; hh < c.G; ++hh) {
+        const int h = g * c.G + hh;
+        float qr[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int r = 0; r < nrep; ++r) {
+          const uint2 raw =
+              *reinterpret_cast<const uint2*>(q + ((size_t)(toks[r] - a.t0) * c.Hq + h) * kD + lane * 4);
+          const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+          const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+          qr[0] += __bfloat162float(p0.x);
+          qr[1] += __bfloat162float(p0.y);
+          qr[2] += __bfloat162float(p1.x);
+          qr[3] += __bfloat162float(p1.y);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) ug[e] += qr[e];
+      }
+      *reinterpret_cast<float4*>(c.u + (((size_t)layer * c.Hkv + g) * c.Jmax + j) * kD + lane * 4) =
+          make_float4(ug[0], ug[1], ug[2], ug[3]);
+    }
+  }
+}
+
+cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_count, int m, int reg_start,
+                             int slot, int theta_mode, float theta, long long theta_q_abs, int max_spans, int n,
+                             int t0, const __nv_bfloat16* q, cudaStream_t s) {
+  if (theta_mode == 1) {
+    const long long N = (long long)m * (m + 1) / 2;
+    long long rank = (long long)floor((double)theta * (double)(N - 1));
+    if (rank < 0) rank = 0;
+    if (rank > N - 1) rank = N - 1;
+    k_theta_select<<<layer_count, 1024, 0, s>>>(c, layer_begin, m, rank);
+  } else {
+    k_theta_set<<<layer_count, 1, 0, s>>>(c, layer_begin, theta_q_abs);
+  }
+  k_seg_rowscan<<<dim3((m + 7) / 8, layer_count), 256, 0, s>>>(c, layer_begin, m);
+  const size_t smem = (size_t)(32 * 32 + m + 32) * sizeof(long long);
+  k_seg_colscan<<<dim3((m + 31) / 32, layer_count), 1024, smem, s>>>(c, layer_begin, m);
+  NmsArgs a{seq, layer_begin, m, reg_start, slot, max_spans, n, t0, q};
+  k_seg_nms<<<layer_count, 1024, 0, s>>>(c, a);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// a4 scores (Eq. 7 with summed representatives, max over the call's query spans):
+// score[g][s] = max_j u[g][j] . K^R[g][s].  One warp per span, 4 dims per lane.
+template <bool DECODE>
+__global__ void __launch_bounds__(256) k_score(DevCtx c, int seq, int layer_begin, DecBatch b, int layer_count,
+                                               const __nv_bfloat16* __restrict__ q) {
+  extern __shared__ float su[];  // [J][128]
+  int layer, sq, J;
+  const int g = blockIdx.y;
+  if (DECODE) {
+    const int bi = blockIdx.z / layer_count;
+    layer = layer_begin + blockIdx.z % layer_count;
+    sq = b.seq[bi];
+    J = 1;
+    if (threadIdx.x < kD) {
+      const __nv_bfloat16* qp =
+          q + (((size_t)b.src[bi] * layer_count + (layer - layer_begin)) * c.Hq + g * c.G) * kD + threadIdx.x;
+      float acc = 0.f;
+      for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
+      su[threadIdx.x] = acc;
+    }
+  } else {
+    layer = layer_begin + blockIdx.z;
+    sq = seq;
+    J = c.Jcnt[layer];
+    const float* up = c.u + ((size_t)layer * c.Hkv + g) * c.Jmax * kD;
+    for (int t = threadIdx.x; t < J * kD; t += blockDim.x) su[t] = up[t];
+  }
+  const size_t unit = unit_of(c, sq, layer);
+  if (blockIdx.x == 0 && g == 0 && threadIdx.x == 0) c.sel_tokens[unit] = 0;
+  __syncthreads();
+  const int N = c.n_spans[unit];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int s0 = blockIdx.x * 64;
+  const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + g) * (size_t)c.cap * kD;
+  float* sc = c.scores + (unit * c.Hkv + g) * (size_t)c.cap;
+  for (int s = s0 + warp; s < min(s0 + 64, N); s += 8) {
+    const uint2 raw = *reinterpret_cast<const uint2*>(KR + (size_t)s * kD + lane * 4);
+    const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+    const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+    const float k0 = __bfloat162float(p0.x), k1 = __bfloat162float(p0.y), k2 = __bfloat162float(p1.x),
+                k3 = __bfloat162float(p1.y);
+    float best = -INFINITY;
+    for (int j = 0; j < J; ++j) {
+      const float4 uv = *reinterpret_cast<const float4*>(su + j * kD + lane * 4);
+      float d = uv.x * k0;
+      d = fmaf(uv.y, k1, d);
+      d = fmaf(uv.z, k2, d);
+      d = fmaf(uv.w, k3, d);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+      best = fmaxf(best, d);
+    }
+    if (lane == 0) sc[s] = best;
+  }
+}
+
+cudaError_t launch_score_prefill(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s) {
+  DecBatch dummy;
+  dummy.n = 0;
+  const size_t smem = (size_t)c.Jmax * kD * sizeof(float);
+  if (smem > 48 * 1024) cudaFuncSetAttribute(k_score<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  k_score<false><<<dim3((span_bound + 63) / 64, c.Hkv, a.layer_count), 256, smem, s>>>(c, a.seq, a.layer_begin, dummy,
+                                                                                       a.layer_count, nullptr);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int,
+                                const __nv_bfloat16* q, int span_bound, cudaStream_t s) {
+  if (span_bound <= 0) span_bound = 1;
+  k_score<true><<<dim3((span_bound + 63) / 64, c.Hkv, b.n * layer_count), 256, kD * sizeof(float), s>>>(
+      c, 0, layer_begin, b, layer_count, q);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// a4 top-k (Eq. 8 with unit = span): the min(k, N_s) largest scores, ties -> lower span id.  4-pass radix select on
+// order-preserving keys, then an id-ordered pick of the threshold ties.  Writes the ascending id list and the token
+// ranges the attention kernels walk (adjacent spans merged).  One CTA per (unit, KV head).
+__device__ __forceinline__ unsigned order_key(float f) {
+  const unsigned u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+template <bool DECODE>
+__global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin, DecBatch b, int layer_count) {
+  __shared__ unsigned hist[256];
+  __shared__ unsigned s_prefix, s_need;
+  __shared__ int s_ids[kMaxTopK];
+  __shared__ int s_cnt;
+  __shared__ int s_scan[512];
+  const int g = blockIdx.x;
+  int layer, sq, pos = 0, loc_begin = 0;
+  if (DECODE) {
+    const int bi = blockIdx.y / layer_count;
+    layer = layer_begin + blockIdx.y % layer_count;
+    sq = b.seq[bi];
+    pos = b.pos[bi];
+    loc_begin = b.loc_begin[bi];
+  } else {
+    layer = layer_begin + blockIdx.y;
+    sq = seq;
+  }
+  const size_t unit = unit_of(c, sq, layer);
+  const int N = c.n_spans[unit];
+  const float* sc = c.scores + (unit * c.Hkv + g) * (size_t)c.cap;
+  const int K = min(c.topk, N);
+  const int tid = threadIdx.x, nt = blockDim.x;
+  if (tid == 0) s_cnt = 0;
+  __syncthreads();
+  if (K == N) {
+    for (int t = tid; t < K; t += nt) s_ids[t] = t;
+    if (tid == 0) s_cnt = K;
+  } else {
+    if (tid == 0) {
+      s_prefix = 0;
+      s_need = K;  // rank from the top, 1-based: find key T with #(key > T) < K <= #(key >= T)
+    }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      const unsigned prefix = s_prefix;
+      const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      for (int s = tid; s < N; s += nt) {
+        const unsigned key = order_key(sc[s]);
+        if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        unsigned need = s_need;
+        int bin = 255;
+        for (; bin >= 0; --bin) {
+          if (need <= hist[bin]) break;
+          need -= hist[bin];
+        }
+        if (bin < 0) bin = 0;
+        s_need = need;
+        s_prefix = prefix | ((unsigned)bin << shift);
+      }
+      __syncthreads();
+    }
+    const unsigned T = s_prefix;
+    const unsigned need_eq = s_need;  // how many of the == T elements are taken (lowest ids first)
+    // contiguous id partition so that ties are picked in id order
+    const int per = (N + nt - 1) / nt;
+    const int lo = tid * per, hi = min(N, lo + per);
+    int eq = 0;
+    for (int s = lo; s < hi; ++s) eq += order_key(sc[s]) == T;
+    s_scan[tid] = eq;
+    __syncthreads();
+    if (tid == 0) {
+      int run = 0;
+      for (int t = 0; t < nt; ++t) {
+        const int v = s_scan[t];
+        s_scan[t] = run;
+        run += v;
+      }
+    }
+    __syncthreads();
+    int eqrank = s_scan[tid];
+    for (int s = lo; s < hi; ++s) {
+      const unsigned key = order_key(sc[s]);
+      bool take = key > T;
+      if (key == T) {
+        take = (unsigned)eqrank < need_eq;
+        ++eqrank;
+      }
+      if (take) {
+        const int slot = atomicAdd(&s_cnt, 1);
+        if (slot < kMaxTopK) s_ids[slot] = s;
+      }
+    }
+  }
+  __syncthreads();
+  const int cnt = min(s_cnt, K);
+  // rank sort ascending
+  int myid = -1, rank = 0;
+  if (tid < cnt) {
+    myid = s_ids[tid];
+    for (int t = 0; t < cnt; ++t) rank += s_ids[t] < myid;
+  }
+  __syncthreads();
+  if (tid < cnt) s_ids[rank] = myid;
+  __syncthreads();
+  int* sel = c.sel + (unit * c.Hkv + g) * (size_t)c.topk;
+  for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
+  if (tid == 0) {
+    const size_t rb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
+    int* rs = c.rng_start + rb;
+    int* rl = c.rng_len + rb;
+    int nr = 0;
+    long long tokens = 0;
+    auto push = [&](int st, int ln) {
+      if (ln <= 0) return;
+      if (nr > 0 && rs[nr - 1] + rl[nr - 1] == st)
+        rl[nr - 1] += ln;
+      else {
+        rs[nr] = st;
+        rl[nr] = ln;
+        ++nr;
+      }
+    };
+    if (DECODE) push(0, min(c.Ls, pos + 1));
+    for (int t = 0; t < cnt; ++t) {
+      const int st = c.span_start[unit * c.cap + s_ids[t]], ln = c.span_len[unit * c.cap + s_ids[t]];
+      tokens += ln;
+      push(st, ln);
+    }
+    if (DECODE) push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
+    c.rng_cnt[unit * c.Hkv + g] = nr;
+    atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+  }
+}
+
+cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
+  DecBatch dummy;
+  dummy.n = 0;
+  k_topk<false><<<dim3(c.Hkv, a.layer_count), 512, 0, s>>>(c, a.seq, a.layer_begin, dummy, a.layer_count);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s) {
+  k_topk<true><<<dim3(c.Hkv, b.n * layer_count), 512, 0, s>>>(c, 0, layer_begin, b, layer_count);
+  return cudaGetLastError();
+}
+
+}  // namespace ltri

@@ -1,0 +1,546 @@
+// C ABI of the ltri library: host-side stream state, arena layout and the launch sequences of a prefill call
+// and a decode step.  Everything that computes runs in the kernels; this file only orders them.
+#include <cmath>
+#include <cstring>
+#include <deque>
+#include <new>
+#include <vector>
+
+#include "../../include/ltri.h"
+#include "common.cuh"
+
+using namespace ltri;
+
+namespace {
+
+struct Region {
+  int start, end, slot;
+};
+
+struct LayerState {
+  long long t = 0;  // tokens appended
+  int E = 0;        // end of the indexed prefix
+  bool decoding = false;
+  std::deque<Region> pending;
+  long long span_ub = 0;  // upper bound of the device-side span count
+  int last_m = 0;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+  char* base;
+  size_t off = 0;
+  template <typename T>
+  T* take(size_t count) {
+    off = align_up(off, 256);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+bool validate(const ltri_params* p) {
+  if (!p) return false;
+  if (p->n_layers < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->head_dim != kD) return false;
+  if (p->n_q_heads % p->n_kv_heads) return false;
+  const int G = p->n_q_heads / p->n_kv_heads;
+  if (!(G == 1 || G == 2 || G == 4 || G == 8)) return false;
+  if (p->max_seqs < 1 || p->max_tokens < 1 || p->max_tokens > (1ll << 30)) return false;
+  if (p->chunk < 16 || p->chunk > 1024 || p->chunk % 16) return false;
+  if (p->window < 1 || p->n_sink < 1 || p->n_sink > p->chunk) return false;
+  if (p->top_k < 1 || p->top_k > kMaxTopK) return false;
+  if (p->reps_per_span < 0 || p->reps_per_span > kMaxReps) return false;
+  if (p->max_spans_per_region < 0 || p->max_spans_per_region > kMaxTopK) return false;
+  if (p->theta_mode != 0 && p->theta_mode != 1) return false;
+  if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
+  if (!(p->softmax_scale >= 0.f)) return false;
+  return true;
+}
+
+// fills every pointer of `d` relative to `base` (nullptr: sizing only) and returns the bytes used
+size_t layout(const ltri_params& p, DevCtx& d, char* base) {
+  d.NL = p.n_layers;
+  d.Hq = p.n_q_heads;
+  d.Hkv = p.n_kv_heads;
+  d.G = d.Hq / d.Hkv;
+  d.NS = p.max_seqs;
+  d.Tmax = p.max_tokens;
+  d.Tpad = (long long)align_up((size_t)p.max_tokens, 128) + kTokPad;
+  d.chunk = p.chunk;
+  d.W = p.window;
+  d.Ls = p.n_sink;
+  d.topk = p.top_k;
+  d.reps = p.reps_per_span > 0 ? p.reps_per_span : 1;
+  d.C = p.max_spans_per_region > 0 ? p.max_spans_per_region : std::max(1, p.chunk / 32);
+  d.Jmax = 2 * d.C + 1;
+  d.slots = (p.window + p.chunk - 1) / p.chunk + 8;
+  d.cap = (int)std::min<long long>((long long)1 << 30, ((p.max_tokens + p.chunk - 1) / p.chunk + 8) * d.Jmax);
+  d.theta_mode = p.theta_mode;
+  d.theta = p.theta;
+  d.scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / std::sqrt((float)kD);
+  const size_t units = (size_t)d.NS * d.NL;
+  Carver cv{base};
+  d.Kc = cv.take<__nv_bfloat16>(units * d.Hkv * d.Tpad * kD);
+  d.Vc = cv.take<__nv_bfloat16>(units * d.Hkv * d.Tpad * kD);
+  d.votes = cv.take<long long>(units * d.Tpad);
+  d.span_start = cv.take<int>(units * d.cap);
+  d.span_len = cv.take<int>(units * d.cap);
+  d.n_spans = cv.take<int>(units);
+  d.KR = cv.take<__nv_bfloat16>(units * d.Hkv * d.cap * kD);
+  d.pend_start = cv.take<int>(units * (d.slots + 1) * d.Jmax);
+  d.pend_len = cv.take<int>(units * (d.slots + 1) * d.Jmax);
+  d.pend_cnt = cv.take<int>(units * (d.slots + 1));
+  d.sel = cv.take<int>(units * d.Hkv * d.topk);
+  d.sel_tokens = cv.take<long long>(units);
+  d.Mq = cv.take<int>((size_t)d.NL * d.chunk * d.chunk);
+  d.Rsuf = cv.take<long long>((size_t)d.NL * d.chunk * d.chunk);
+  d.best = cv.take<long long>((size_t)d.NL * 2 * d.chunk);
+  d.thetaq = cv.take<long long>(d.NL);
+  d.rowstat = cv.take<float2>((size_t)d.NL * d.chunk * d.Hq);
+  d.Oacc = cv.take<float>((size_t)d.NL * d.chunk * d.Hq * kD);
+  d.u = cv.take<float>((size_t)d.NL * d.Hkv * d.Jmax * kD);
+  d.Jcnt = cv.take<int>(d.NL);
+  d.scores = cv.take<float>(units * d.Hkv * d.cap);
+  d.rng_start = cv.take<int>(units * d.Hkv * (d.topk + 2));
+  d.rng_len = cv.take<int>(units * d.Hkv * (d.topk + 2));
+  d.rng_cnt = cv.take<int>(units * d.Hkv);
+  d.dec_part = cv.take<float>(units * d.Hq * kMaxDecSplit * (kD + 2));
+  d.status = cv.take<int>(4);
+  d.slots += 1;  // the extra slot is scratch for ltri_debug_segment_map
+  return align_up(cv.off, 256);
+}
+
+}  // namespace
+
+struct ltri_ctx {
+  ltri_params p;
+  DevCtx d;
+  std::vector<LayerState> st;  // [max_seqs][n_layers]
+  int last_cuda = 0;
+  int sm_count = 148;
+  LayerState& at(int seq, int layer) { return st[(size_t)seq * d.NL + layer]; }
+};
+
+namespace {
+
+int cuda_fail(ltri_ctx* ctx, cudaError_t e) {
+  if (e == cudaSuccess) return LTRI_OK;
+  ctx->last_cuda = (int)e;
+  return LTRI_ECUDA;
+}
+#define LTRI_CUDA(ctx, expr)                   \
+  do {                                         \
+    cudaError_t e__ = (expr);                  \
+    if (e__ != cudaSuccess) return cuda_fail(ctx, e__); \
+  } while (0)
+
+bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+size_t ltri_arena_bytes(const ltri_params* p) {
+  if (!validate(p)) return 0;
+  DevCtx d;
+  return layout(*p, d, nullptr);
+}
+
+int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
+  if (!out) return LTRI_EINVAL;
+  *out = nullptr;
+  if (!validate(p)) return LTRI_EINVAL;
+  if (!p->arena || (reinterpret_cast<uintptr_t>(p->arena) & 255)) return LTRI_EINVAL;
+  DevCtx d;
+  const size_t need = layout(*p, d, nullptr);
+  if (p->arena_bytes < need) return LTRI_ECAPACITY;
+  ltri_ctx* ctx = new (std::nothrow) ltri_ctx();
+  if (!ctx) return LTRI_ECAPACITY;
+  ctx->p = *p;
+  layout(*p, ctx->d, static_cast<char*>(p->arena));
+  ctx->st.resize((size_t)p->max_seqs * p->n_layers);
+  for (auto& s : ctx->st) s.E = p->n_sink;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) ctx->sm_count = sms;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = launch_init(ctx->d, -1, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return LTRI_ECUDA;
+  }
+  *out = ctx;
+  return LTRI_OK;
+}
+
+int ltri_destroy(ltri_ctx* ctx) {
+  if (!ctx) return LTRI_EINVAL;
+  delete ctx;
+  return LTRI_OK;
+}
+
+int ltri_reset_sequence(ltri_ctx* ctx, int seq, void* cuda_stream) {
+  if (!ctx || seq < 0 || seq >= ctx->d.NS) return LTRI_EINVAL;
+  for (int l = 0; l < ctx->d.NL; ++l) {
+    LayerState fresh;
+    fresh.E = ctx->d.Ls;
+    ctx->at(seq, l) = fresh;
+  }
+  LTRI_CUDA(ctx, launch_init(ctx->d, seq, static_cast<cudaStream_t>(cuda_stream)));
+  return LTRI_OK;
+}
+
+int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q,
+                       const void* k, const void* v, void* out, void* cuda_stream) {
+  if (!ctx) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  if (seq < 0 || seq >= d.NS || layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > d.NL)
+    return LTRI_EINVAL;
+  if (n_tokens < 1 || n_tokens > d.chunk) return LTRI_EINVAL;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return LTRI_EINVAL;
+  LayerState& s0 = ctx->at(seq, layer_begin);
+  for (int l = 0; l < layer_count; ++l) {
+    const LayerState& s = ctx->at(seq, layer_begin + l);
+    if (s.decoding) return LTRI_ESTATE;
+    if (s.t != s0.t || s.E != s0.E || s.pending.size() != s0.pending.size()) return LTRI_ESTATE;
+  }
+  if (s0.t + n_tokens > d.Tmax) return LTRI_ECAPACITY;
+  const int t0 = (int)s0.t;
+  // plan the evictions (host knows region boundaries; span counts live on the device)
+  std::vector<Region> ev;
+  int E = s0.E;
+  long long ub = s0.span_ub;
+  for (const Region& r : s0.pending) {
+    if (r.end <= t0 - d.W) {
+      ev.push_back(r);
+      E = r.end;
+      ub += std::min(d.Jmax, r.end - r.start);
+    } else
+      break;
+  }
+  if (ub > d.cap) return LTRI_ECAPACITY;
+  const int reg_start = std::max(d.Ls, t0);
+  const int m = std::max(0, t0 + n_tokens - reg_start);
+  const int user_slots = d.slots - 1;
+  if (m > 0 && (int)(s0.pending.size() - ev.size()) + 1 > user_slots) return LTRI_ECAPACITY;
+  int slot = -1;
+  if (m > 0) {
+    // first slot not used by a region that stays pending
+    std::vector<char> used(user_slots, 0);
+    for (size_t i = ev.size(); i < s0.pending.size(); ++i) used[s0.pending[i].slot] = 1;
+    for (int i = 0; i < user_slots; ++i)
+      if (!used[i]) {
+        slot = i;
+        break;
+      }
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  PrefillArgs a;
+  a.seq = seq;
+  a.layer_begin = layer_begin;
+  a.layer_count = layer_count;
+  a.n = n_tokens;
+  a.t0 = t0;
+  a.sink_end = std::min(d.Ls, t0);
+  a.loc_begin = std::min(E, t0);
+  a.reg_start = reg_start;
+  a.m = m;
+  a.slot = slot;
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.k = static_cast<const __nv_bfloat16*>(k);
+  a.v = static_cast<const __nv_bfloat16*>(v);
+  a.out = static_cast<__nv_bfloat16*>(out);
+
+  LTRI_CUDA(ctx, launch_append_prefill(d, a, st));
+  for (size_t i = 0; i < ev.size(); i += 8) {
+    EvictArgs ea;
+    ea.seq = seq;
+    ea.layer_begin = layer_begin;
+    ea.nslots = (int)std::min<size_t>(8, ev.size() - i);
+    for (int j = 0; j < ea.nslots; ++j) ea.slot[j] = ev[i + j].slot;
+    LTRI_CUDA(ctx, launch_evict_index(d, ea, layer_count, st));
+  }
+  const bool has_index = ub > 0;
+  LTRI_CUDA(ctx, launch_attn_prefill(d, a, 0, !has_index, st));
+  LTRI_CUDA(ctx, launch_map_pass(d, a, st));
+  if (m > 0) {
+    long long thq_abs = 0;
+    if (d.theta_mode == 0) thq_abs = (long long)std::nearbyint((double)d.theta * (double)d.Hq * (double)kQScale);
+    LTRI_CUDA(ctx, launch_segment(d, seq, layer_begin, layer_count, m, reg_start, slot, d.theta_mode, d.theta, thq_abs,
+                                  d.C, n_tokens, t0, a.q, st));
+  }
+  if (has_index) {
+    LTRI_CUDA(ctx, launch_score_prefill(d, a, (int)ub, st));
+    LTRI_CUDA(ctx, launch_topk_prefill(d, a, st));
+    LTRI_CUDA(ctx, launch_attn_prefill(d, a, 1, true, st));
+  }
+  // commit the host state
+  for (int l = 0; l < layer_count; ++l) {
+    LayerState& s = ctx->at(seq, layer_begin + l);
+    for (size_t i = 0; i < ev.size(); ++i) s.pending.pop_front();
+    s.E = E;
+    s.span_ub = ub;
+    s.t += n_tokens;
+    s.last_m = m;
+    if (m > 0) s.pending.push_back(Region{reg_start, t0 + n_tokens, slot});
+  }
+  return LTRI_OK;
+}
+
+int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int layer_begin, int layer_count,
+                     const void* q, const void* k, const void* v, void* out, void* cuda_stream) {
+  if (!ctx || !seq_ids) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  if (n_seqs < 1 || n_seqs > d.NS || layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > d.NL)
+    return LTRI_EINVAL;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return LTRI_EINVAL;
+  std::vector<char> seen(d.NS, 0);
+  long long ub = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    const int sq = seq_ids[i];
+    if (sq < 0 || sq >= d.NS || seen[sq]) return LTRI_EINVAL;
+    seen[sq] = 1;
+    const LayerState& s0 = ctx->at(sq, layer_begin);
+    if (s0.t < 1) return LTRI_ESTATE;
+    if (s0.t + 1 > d.Tmax) return LTRI_ECAPACITY;
+    for (int l = 0; l < layer_count; ++l) {
+      const LayerState& s = ctx->at(sq, layer_begin + l);
+      if (s.t != s0.t || s.E != s0.E) return LTRI_ESTATE;
+    }
+    ub = std::max(ub, s0.span_ub);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+  const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
+  const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
+  __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(out);
+  for (int i0 = 0; i0 < n_seqs; i0 += kDecBatch) {
+    DecBatch b;
+    b.n = std::min(kDecBatch, n_seqs - i0);
+    for (int i = 0; i < b.n; ++i) {
+      const LayerState& s = ctx->at(seq_ids[i0 + i], layer_begin);
+      b.seq[i] = seq_ids[i0 + i];
+      b.pos[i] = (int)s.t;
+      b.loc_begin[i] = s.E;
+      b.src[i] = i0 + i;
+    }
+    const int units = b.n * layer_count * d.Hkv;
+    int nsplit = (ctx->sm_count * 8 + units - 1) / units;
+    nsplit = std::max(1, std::min(nsplit, kMaxDecSplit));
+    LTRI_CUDA(ctx, launch_append_decode(d, b, layer_begin, layer_count, n_seqs, kb, vb, st));
+    LTRI_CUDA(ctx, launch_score_decode(d, b, layer_begin, layer_count, n_seqs, qb, (int)ub, st));
+    LTRI_CUDA(ctx, launch_topk_decode(d, b, layer_begin, layer_count, st));
+    LTRI_CUDA(ctx, launch_decode_attn(d, b, layer_begin, layer_count, n_seqs, qb, ob, nsplit, st));
+  }
+  for (int i = 0; i < n_seqs; ++i)
+    for (int l = 0; l < layer_count; ++l) {
+      LayerState& s = ctx->at(seq_ids[i], layer_begin + l);
+      s.t += 1;
+      s.decoding = true;
+    }
+  return LTRI_OK;
+}
+
+// ---- introspection ---------------------------------------------------------------------------
+static int copy_back(ltri_ctx* ctx, void* dst, const void* src, size_t bytes, cudaStream_t st) {
+  if (bytes == 0) return LTRI_OK;
+  LTRI_CUDA(ctx, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, st));
+  LTRI_CUDA(ctx, cudaStreamSynchronize(st));
+  return LTRI_OK;
+}
+
+int ltri_get_spans(ltri_ctx* ctx, int seq, int layer, int32_t* pairs, int cap, int* n_out, void* cuda_stream) {
+  if (!ctx || !n_out || seq < 0 || seq >= ctx->d.NS || layer < 0 || layer >= ctx->d.NL || cap < 0) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t unit = unit_of(d, seq, layer);
+  int n = 0;
+  int rc = copy_back(ctx, &n, d.n_spans + unit, sizeof(int), st);
+  if (rc) return rc;
+  *n_out = n;
+  const int take = std::min(n, cap);
+  if (take > 0 && pairs) {
+    std::vector<int> a(take), b(take);
+    rc = copy_back(ctx, a.data(), d.span_start + unit * d.cap, take * sizeof(int), st);
+    if (rc) return rc;
+    rc = copy_back(ctx, b.data(), d.span_len + unit * d.cap, take * sizeof(int), st);
+    if (rc) return rc;
+    for (int i = 0; i < take; ++i) {
+      pairs[2 * i] = a[i];
+      pairs[2 * i + 1] = b[i];
+    }
+  }
+  return LTRI_OK;
+}
+
+int ltri_get_pending_spans(ltri_ctx* ctx, int seq, int layer, int32_t* pairs, int cap, int* n_out, void* cuda_stream) {
+  if (!ctx || !n_out || seq < 0 || seq >= ctx->d.NS || layer < 0 || layer >= ctx->d.NL || cap < 0) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t unit = unit_of(d, seq, layer);
+  int total = 0;
+  for (const Region& r : ctx->at(seq, layer).pending) {
+    int cnt = 0;
+    int rc = copy_back(ctx, &cnt, d.pend_cnt + unit * d.slots + r.slot, sizeof(int), st);
+    if (rc) return rc;
+    cnt = std::max(0, std::min(cnt, d.Jmax));
+    std::vector<int> a(cnt), b(cnt);
+    rc = copy_back(ctx, a.data(), d.pend_start + (unit * d.slots + r.slot) * d.Jmax, cnt * sizeof(int), st);
+    if (rc) return rc;
+    rc = copy_back(ctx, b.data(), d.pend_len + (unit * d.slots + r.slot) * d.Jmax, cnt * sizeof(int), st);
+    if (rc) return rc;
+    for (int i = 0; i < cnt; ++i, ++total)
+      if (total < cap && pairs) {
+        pairs[2 * total] = a[i];
+        pairs[2 * total + 1] = b[i];
+      }
+  }
+  *n_out = total;
+  return LTRI_OK;
+}
+
+int ltri_get_selected(ltri_ctx* ctx, int seq, int layer, int32_t* ids, void* cuda_stream) {
+  if (!ctx || !ids || seq < 0 || seq >= ctx->d.NS || layer < 0 || layer >= ctx->d.NL) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  return copy_back(ctx, ids, d.sel + unit_of(d, seq, layer) * d.Hkv * d.topk, (size_t)d.Hkv * d.topk * sizeof(int),
+                   static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ltri_get_stats(ltri_ctx* ctx, int seq, int layer, ltri_stats* out, void* cuda_stream) {
+  if (!ctx || !out || seq < 0 || seq >= ctx->d.NS || layer < 0 || layer >= ctx->d.NL) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t unit = unit_of(d, seq, layer);
+  const LayerState& s = ctx->at(seq, layer);
+  std::memset(out, 0, sizeof(*out));
+  int n = 0;
+  long long rt = 0;
+  int rc = copy_back(ctx, &n, d.n_spans + unit, sizeof(int), st);
+  if (rc) return rc;
+  rc = copy_back(ctx, &rt, d.sel_tokens + unit, sizeof(long long), st);
+  if (rc) return rc;
+  out->tokens = s.t;
+  out->evicted_end = s.E;
+  out->n_spans = n;
+  out->n_pending_regions = (int)s.pending.size();
+  out->index_bytes = (int64_t)n * d.Hkv * kD * 2;
+  out->retrieved_tokens = rt;
+  if (!s.pending.empty() && !s.decoding) {
+    int cnt = 0;
+    rc = copy_back(ctx, &cnt, d.pend_cnt + unit * d.slots + s.pending.back().slot, sizeof(int), st);
+    if (rc) return rc;
+    out->last_call_spans = cnt;
+  }
+  return LTRI_OK;
+}
+
+int ltri_sync_status(ltri_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return LTRI_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int w[4] = {0, 0, 0, 0};
+  int rc = copy_back(ctx, w, ctx->d.status, sizeof(w), st);
+  if (rc) return rc;
+  if (w[0] != 0) {
+    LTRI_CUDA(ctx, cudaMemsetAsync(ctx->d.status, 0, sizeof(w), st));
+    LTRI_CUDA(ctx, cudaStreamSynchronize(st));
+    return (w[0] <= LTRI_EINVAL && w[0] >= LTRI_ETIMEOUT) ? w[0] : LTRI_EDEVICE;
+  }
+  return LTRI_OK;
+}
+
+int ltri_last_cuda_error(const ltri_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+const char* ltri_strerror(int code) {
+  switch (code) {
+    case LTRI_OK: return "ok";
+    case LTRI_EINVAL: return "invalid argument";
+    case LTRI_ECAPACITY: return "capacity exceeded";
+    case LTRI_ESTATE: return "call order violated";
+    case LTRI_ECUDA: return "CUDA runtime error";
+    case LTRI_EDEVICE: return "device-side check failed";
+    case LTRI_ETIMEOUT: return "device-side wait expired";
+  }
+  return "unknown error";
+}
+
+int ltri_span_capacity(const ltri_ctx* ctx) { return ctx ? ctx->d.cap : LTRI_EINVAL; }
+
+int ltri_debug_read(ltri_ctx* ctx, int what, int seq, int layer, void* dst, size_t cap_bytes, size_t* bytes_out,
+                    void* cuda_stream) {
+  if (!ctx || seq < 0 || seq >= ctx->d.NS || layer < 0 || layer >= ctx->d.NL) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  const size_t unit = unit_of(d, seq, layer);
+  const void* src = nullptr;
+  size_t bytes = 0;
+  switch (what) {
+    case LTRI_BUF_MAP:
+      src = d.Mq + (size_t)layer * d.chunk * d.chunk;
+      bytes = (size_t)d.chunk * d.chunk * sizeof(int);
+      break;
+    case LTRI_BUF_VOTES:
+      src = d.votes + unit * d.Tpad;
+      bytes = (size_t)d.Tmax * sizeof(long long);
+      break;
+    case LTRI_BUF_INDEX:
+      src = d.KR + unit * d.Hkv * (size_t)d.cap * kD;
+      bytes = (size_t)d.Hkv * d.cap * kD * 2;
+      break;
+    case LTRI_BUF_THETA:
+      src = d.thetaq + layer;
+      bytes = sizeof(long long);
+      break;
+    case LTRI_BUF_SCORES:
+      src = d.scores + unit * d.Hkv * (size_t)d.cap;
+      bytes = (size_t)d.Hkv * d.cap * sizeof(float);
+      break;
+    case LTRI_BUF_QREPS:
+      src = d.u + (size_t)layer * d.Hkv * d.Jmax * kD;
+      bytes = (size_t)d.Hkv * d.Jmax * kD * sizeof(float);
+      break;
+    case LTRI_BUF_ROWSTAT:
+      src = d.rowstat + (size_t)layer * d.chunk * d.Hq;
+      bytes = (size_t)d.chunk * d.Hq * sizeof(float2);
+      break;
+    default: return LTRI_EINVAL;
+  }
+  if (bytes_out) *bytes_out = bytes;
+  if (!dst) return LTRI_OK;
+  return copy_back(ctx, dst, src, std::min(bytes, cap_bytes), static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ltri_debug_segment_map(ltri_ctx* ctx, const int32_t* Mq, int m, int theta_mode, float theta, int64_t theta_q,
+                           int max_spans, int32_t* pairs, int cap, int* n_out, void* cuda_stream) {
+  if (!ctx || !Mq || !n_out || !pairs) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  if (m < 1 || m > d.chunk || theta_mode < 0 || theta_mode > 2 || max_spans < 1 || max_spans > d.C) return LTRI_EINVAL;
+  if (theta_mode == 1 && !(theta >= 0.f && theta <= 1.f)) return LTRI_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  LTRI_CUDA(ctx, cudaMemcpy2DAsync(d.Mq, (size_t)d.chunk * sizeof(int), Mq, (size_t)m * sizeof(int),
+                                   (size_t)m * sizeof(int), m, cudaMemcpyHostToDevice, st));
+  long long thq = theta_q;
+  if (theta_mode == 0) thq = (long long)std::nearbyint((double)theta * (double)d.Hq * (double)kQScale);
+  const int slot = d.slots - 1;
+  LTRI_CUDA(ctx, launch_segment(d, 0, 0, 1, m, 0, slot, theta_mode == 1 ? 1 : 0, theta, thq, max_spans, 0, 0, nullptr,
+                                st));
+  int cnt = 0;
+  int rc = copy_back(ctx, &cnt, d.pend_cnt + slot, sizeof(int), st);
+  if (rc) return rc;
+  *n_out = cnt;
+  cnt = std::max(0, std::min(std::min(cnt, cap), d.Jmax));
+  std::vector<int> a(cnt), b(cnt);
+  rc = copy_back(ctx, a.data(), d.pend_start + (size_t)slot * d.Jmax, cnt * sizeof(int), st);
+  if (rc) return rc;
+  rc = copy_back(ctx, b.data(), d.pend_len + (size_t)slot * d.Jmax, cnt * sizeof(int), st);
+  if (rc) return rc;
+  for (int i = 0; i < cnt; ++i) {
+    pairs[2 * i] = a[i];
+    pairs[2 * i + 1] = b[i];
+  }
+  return LTRI_OK;
+}
+
+}  // extern "C"

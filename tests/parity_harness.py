@@ -1,0 +1,235 @@
+"""GPU-vs-oracle parity harness used by the ``-m gpu`` tests and the smoke check.
+
+Drives the CUDA library (through the C ABI binding) and one CPU oracle per checked layer over
+the same seeded inputs, comparing after every call:
+
+* the Q20 region map and theta (floating point decides an integer: a few units of tolerance);
+* the segmenter, bit-exact, on the GPU's own map (oracle segmenter fed the GPU's integers);
+* the region's spans against the oracle's own run (bit-exact unless the oracle reports a
+  decisive relative gap below 1e-4, in which case the oracle adopts the GPU's pick);
+* votes, the span table and the index vectors; scores and the selected span sets (a pick may
+  differ only among candidates within 1e-4 relative of the cut; the oracle then adopts it);
+* attention outputs: max-abs <= 2e-2 and relative Frobenius error <= 1e-2.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import torch
+
+from oracle import ltri_oracle as orc
+from paper_2412_04757_b200 import binding, inputs
+
+MAX_ABS = 2e-2
+REL_FRO = 1e-2
+NEAR_TIE = 1e-4
+
+
+@dataclasses.dataclass
+class Report:
+    calls: int = 0
+    regions: int = 0
+    span_flips: int = 0
+    sel_checks: int = 0
+    sel_flips: int = 0
+    index_rows: int = 0
+    index_flips: int = 0
+    max_abs: float = 0.0
+    max_rel_fro: float = 0.0
+    max_map_diff: int = 0
+    max_theta_diff: int = 0
+    max_score_rel: float = 0.0
+
+
+def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
+    return binding.make_params(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_tokens, cfg.chunk, cfg.window,
+                               cfg.n_sink, cfg.top_k, head_dim=cfg.head_dim, max_seqs=max_seqs or cfg.n_seqs,
+                               reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
+                               theta_mode=cfg.theta_mode, theta=cfg.theta)
+
+
+def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
+    return orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
+                            cfg.max_tokens, reps_per_span=cfg.reps_per_span,
+                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta)
+
+
+def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str):
+    got = got_bf16.to(torch.float32).cpu().numpy().astype(np.float64)
+    ref = ref.astype(np.float64)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    ma = float(np.abs(got - ref).max())
+    rf = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30))
+    rep.max_abs = max(rep.max_abs, ma)
+    rep.max_rel_fro = max(rep.max_rel_fro, rf)
+    assert ma <= MAX_ABS, f"{what}: max-abs {ma:.4g} > {MAX_ABS}"
+    assert rf <= REL_FRO, f"{what}: relative Frobenius {rf:.4g} > {REL_FRO}"
+
+
+def check_selection(sel_gpu: np.ndarray, o: orc.OracleStream, rep: Report, what: str):
+    """sel_gpu [Hkv][k] ascending ids (-1 padded) against the oracle's scores; adopts tolerated picks."""
+    sel_o, _ = o.selected()
+    sc = o.scores()
+    adopt = False
+    for g in range(sel_gpu.shape[0]):
+        a = set(int(x) for x in sel_gpu[g] if x >= 0)
+        b = set(int(x) for x in sel_o[g] if x >= 0)
+        rep.sel_checks += 1
+        assert len(a) == len(b), f"{what}: KV head {g} selected {len(a)} spans, oracle {len(b)}"
+        if a == b:
+            continue
+        # the sets may differ only among spans whose oracle scores are within the near-tie band of the cut
+        cut = min(sc[g][i] for i in b)
+        band = NEAR_TIE * max(abs(cut), 1e-30)
+        for i in a ^ b:
+            assert abs(sc[g][i] - cut) <= band, (
+                f"{what}: KV head {g} span {i} score {sc[g][i]} vs cut {cut}: not a near tie")
+        rep.sel_flips += 1
+        adopt = True
+    if adopt:
+        ids = np.full_like(sel_o, -1)
+        for g in range(sel_gpu.shape[0]):
+            row = [int(x) for x in sel_gpu[g] if x >= 0]
+            ids[g, :len(row)] = row
+        o.set_selected(ids)
+
+
+class StreamPair:
+    """The library context plus oracles for the checked (seq, layer) pairs of one workload."""
+
+    def __init__(self, cfg: inputs.StreamConfig, layers, seqs=(0,), device="cuda:0", deep=True):
+        self.cfg, self.layers, self.seqs, self.deep = cfg, list(layers), list(seqs), deep
+        self.dev = torch.device(device)
+        self.lt = binding.Ltri(params_of(cfg), device=device)
+        self.orc = {(s, l): oracle_of(cfg) for s in self.seqs for l in self.layers}
+        self.rep = Report()
+        self.n_indexed = {(s, l): 0 for s in self.seqs for l in self.layers}
+
+    # ---- one prefill call -------------------------------------------------------------------
+    def prefill(self, seq, q, k, v, check_out=True):
+        """q [L][n][Hq][d], k, v [L][n][Hkv][d] bf16 on the CPU."""
+        cfg, lt, rep = self.cfg, self.lt, self.rep
+        L = cfg.n_layers
+        out = lt.ltri_prefill_chunk(seq, 0, L, q.to(self.dev), k.to(self.dev), v.to(self.dev))
+        torch.cuda.synchronize(self.dev)
+        assert lt.ltri_sync_status() == 0
+        rep.calls += 1
+        for layer in self.layers:
+            if (seq, layer) not in self.orc:
+                continue
+            o = self.orc[(seq, layer)]
+            what = f"seq {seq} layer {layer} call@{o.tokens}"
+            o.prefill_local(q[layer], k[layer], v[layer])
+            rs, m = o.region()
+            t1 = o.tokens
+            if m > 0:
+                rep.regions += 1
+                pend_g = lt.ltri_get_pending_spans(seq, layer)
+                newest_g = pend_g[pend_g[:, 0] >= rs]
+                spans_o = o.pending()[-1][2]
+                if self.deep:
+                    Mg = np.tril(lt.ltri_debug_read(binding.BUF_MAP, seq, layer)[:m, :m])
+                    Mo = o.map()
+                    md = int(np.abs(Mg.astype(np.int64) - Mo).max())
+                    rep.max_map_diff = max(rep.max_map_diff, md)
+                    assert md <= 4 + cfg.n_q_heads, f"{what}: region map differs by {md} Q20 units"
+                    thg = int(lt.ltri_debug_read(binding.BUF_THETA, seq, layer)[0])
+                    rep.max_theta_diff = max(rep.max_theta_diff, abs(thg - o.theta_q()))
+                    assert abs(thg - o.theta_q()) <= 4 + cfg.n_q_heads, f"{what}: theta {thg} vs {o.theta_q()}"
+                    if cfg.theta_mode == 1:
+                        assert thg == orc.theta_q(Mg, 1, cfg.theta, cfg.n_q_heads), f"{what}: theta rank select"
+                    # integer pipeline: bit-exact on identical integer input
+                    ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region)
+                    ref_spans[:, 0] += rs
+                    assert newest_g.tolist() == ref_spans.tolist(), f"{what}: segmenter differs on its own map"
+                if newest_g.tolist() != spans_o.tolist():
+                    assert o.seg_gap() < NEAR_TIE, (
+                        f"{what}: spans differ and the oracle's smallest decisive gap is {o.seg_gap():.3g}")
+                    rep.span_flips += 1
+                    o.set_newest_spans(newest_g)
+            if self.deep:
+                vg = lt.ltri_debug_read(binding.BUF_VOTES, seq, layer)[:t1].astype(np.float64)
+                vo = o.votes(0, t1).astype(np.float64)
+                lo = cfg.n_sink
+                dv = np.abs(vg[lo:] - vo[lo:])
+                assert np.all(dv <= 64 + 2e-5 * np.abs(vo[lo:])), f"{what}: votes differ by up to {dv.max()}"
+            self._check_index(seq, layer, o, k, what)
+            o.prefill_retrieve()
+            if len(o.spans()):
+                if self.deep and m > 0:
+                    J = len(o.pending()[-1][2])
+                    ug = lt.ltri_debug_read(binding.BUF_QREPS, seq, layer)[:, :J]
+                    assert np.allclose(ug, o.query_reps(), rtol=0, atol=1e-4), f"{what}: query representatives"
+                    ns = len(o.spans())
+                    sg = lt.ltri_debug_read(binding.BUF_SCORES, seq, layer)[:, :ns]
+                    so = o.scores()
+                    rel = float(np.abs(sg - so).max() / max(np.abs(so).max(), 1e-30))
+                    rep.max_score_rel = max(rep.max_score_rel, rel)
+                    assert rel <= 2e-5, f"{what}: scores differ by {rel:.3g} relative"
+                check_selection(lt.ltri_get_selected(seq, layer), o, rep, what)
+            if check_out:
+                check_output(out[layer], o.prefill_attend(), rep, what)
+        return out
+
+    def _check_index(self, seq, layer, o, k, what):
+        spans_o = o.spans()
+        done = self.n_indexed[(seq, layer)]
+        if len(spans_o) == done:
+            return
+        spans_g = self.lt.ltri_get_spans(seq, layer)
+        assert spans_g.tolist() == spans_o.tolist(), f"{what}: span tables differ"
+        idx_g = self.lt.ltri_debug_read(binding.BUF_INDEX, seq, layer)
+        idx_o = o.index()
+        for s in range(done, len(spans_o)):
+            self.rep.index_rows += 1
+            if np.array_equal(idx_g[:, s, :], idx_o[s]):
+                continue
+            # a different representative token is tolerated only as a near tie in the oracle's votes
+            st, ln = spans_o[s]
+            vo = o.votes(int(st), int(st + ln)).astype(np.float64)
+            top = np.sort(vo)[::-1]
+            assert self.cfg.reps_per_span < ln and (top[self.cfg.reps_per_span - 1] - top[self.cfg.reps_per_span]) <= \
+                NEAR_TIE * max(top[0], 1.0), f"{what}: index vector of span {s} differs"
+            self.rep.index_flips += 1
+        self.n_indexed[(seq, layer)] = len(spans_o)
+
+    # ---- one decode step ---------------------------------------------------------------------
+    def decode(self, seq_ids, q, k, v):
+        """q [n_seqs][L][Hq][d], k, v [n_seqs][L][Hkv][d] bf16 on the CPU."""
+        cfg, lt, rep = self.cfg, self.lt, self.rep
+        L = cfg.n_layers
+        out = lt.ltri_decode_step(seq_ids, 0, L, q.to(self.dev), k.to(self.dev), v.to(self.dev))
+        torch.cuda.synchronize(self.dev)
+        assert lt.ltri_sync_status() == 0
+        rep.calls += 1
+        for i, seq in enumerate(seq_ids):
+            for layer in self.layers:
+                if (seq, layer) not in self.orc:
+                    continue
+                o = self.orc[(seq, layer)]
+                what = f"seq {seq} layer {layer} decode@{o.tokens}"
+                o.decode_retrieve(q[i, layer], k[i, layer], v[i, layer])
+                if len(o.spans()):
+                    check_selection(lt.ltri_get_selected(seq, layer), o, rep, what)
+                check_output(out[i, layer], o.decode_attend(), rep, what)
+        return out
+
+
+def run_stream(cfg: inputs.StreamConfig, layers, max_calls=None, decode_steps=None, deep=True, device="cuda:0"):
+    """Stream the workload of `cfg` (sequence 0) through both sides; returns the Report."""
+    sp = StreamPair(cfg, layers, device=device, deep=deep)
+    st = inputs.SyntheticStream(cfg)
+    for ci, (t0, n) in enumerate(st.prefill_chunks()):
+        if max_calls is not None and ci >= max_calls:
+            break
+        q, k, v = st.tokens(t0, n)
+        sp.prefill(0, q, k, v)
+    steps = cfg.decode_steps if decode_steps is None else decode_steps
+    if max_calls is None:
+        for s in range(steps):
+            q, k, v = st.tokens(cfg.context + s, 1, kind=1)
+            sp.decode([0], q.permute(1, 0, 2, 3).contiguous(), k.permute(1, 0, 2, 3).contiguous(),
+                      v.permute(1, 0, 2, 3).contiguous())
+    sp.lt.close()
+    return sp.rep

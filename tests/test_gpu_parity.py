@@ -1,0 +1,166 @@
+"""GPU path (through the C ABI) against the CPU oracle on the same seeded inputs."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_04757_b200 import binding, inputs
+from tests import parity_harness as ph
+
+pytestmark = pytest.mark.gpu
+
+
+def small_cfg(**kw):
+    base = dict(name="small", n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=128, context=1536, chunk=128,
+                decode_steps=6, n_sink=32, window=384, top_k=4, max_spans_per_region=4, seg_min=16, seg_max=128,
+                seed=777)
+    base.update(kw)
+    return inputs.StreamConfig(**base)
+
+
+def test_cfg0_full_stream_and_decode():
+    cfg = inputs.config(0)
+    rep = ph.run_stream(cfg, layers=[0])
+    assert rep.regions == 8 and rep.calls == 8 + 16
+    assert rep.span_flips <= 1 and rep.sel_flips <= 2
+    print(rep)
+
+
+def test_two_layers_gqa4_ragged_tail():
+    # context not a multiple of the chunk: the last call is short; window not a multiple either
+    cfg = small_cfg(context=1500, window=300)
+    rep = ph.run_stream(cfg, layers=[0, 1])
+    assert rep.regions >= 20
+    print(rep)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (4, 2), (16, 2)])
+def test_group_sizes(Hq, Hkv):
+    cfg = small_cfg(n_layers=1, n_q_heads=Hq, n_kv_heads=Hkv, context=1024, decode_steps=3)
+    rep = ph.run_stream(cfg, layers=[0])
+    print(rep)
+
+
+def test_three_representatives_per_span_and_absolute_theta():
+    cfg = small_cfg(n_layers=1, reps_per_span=3, theta_mode=0, theta=0.02, context=1024, decode_steps=3)
+    rep = ph.run_stream(cfg, layers=[0])
+    print(rep)
+
+
+def test_top_k_covering_everything_equals_full_attention():
+    # with top_k >= number of spans the streamed output is plain causal attention (oracle O12)
+    cfg = small_cfg(n_layers=1, context=640, chunk=64, window=128, top_k=64, max_spans_per_region=2, decode_steps=2)
+    sp = ph.StreamPair(cfg, [0])
+    st = inputs.SyntheticStream(cfg)
+    outs, qs = [], []
+    for t0, n in st.prefill_chunks():
+        q, k, v = st.tokens(t0, n)
+        outs.append(sp.prefill(0, q, k, v)[0])
+        qs.append(q[0])
+    assert sp.lt.ltri_get_stats(0, 0).n_spans <= 64
+    o = sp.orc[(0, 0)]
+    pos = [70, 300, 639]
+    qall = torch.cat(qs)
+    ref = o.full_attention(pos, qall[pos])
+    got = torch.cat(outs)[pos].float().cpu().numpy()
+    assert np.abs(got - ref).max() <= ph.MAX_ABS
+    sp.lt.close()
+
+
+def test_irregular_call_sizes_and_single_token_calls():
+    cfg = small_cfg(n_layers=1, context=900, chunk=128, window=256)
+    sp = ph.StreamPair(cfg, [0])
+    st = inputs.SyntheticStream(cfg)
+    t0 = 0
+    for n in [128, 1, 37, 128, 128, 16, 128, 128, 5, 128, 73]:
+        q, k, v = st.tokens(t0, n)
+        sp.prefill(0, q, k, v)
+        t0 += n
+    s = sp.lt.ltri_get_stats(0, 0)
+    assert s.tokens == t0 and s.n_spans > 0
+    for step in range(3):
+        q, k, v = st.tokens(t0 + step, 1, kind=1)
+        sp.decode([0], q.permute(1, 0, 2, 3).contiguous(), k.permute(1, 0, 2, 3).contiguous(),
+                  v.permute(1, 0, 2, 3).contiguous())
+    sp.lt.close()
+    print(sp.rep)
+
+
+def test_batched_decode_independent_sequences():
+    cfg = small_cfg(n_layers=2, n_seqs=3, context=768, decode_steps=4)
+    sp = ph.StreamPair(cfg, layers=[0, 1], seqs=[0, 1, 2])
+    streams = [inputs.SyntheticStream(cfg, seq=s) for s in range(3)]
+    for s, st in enumerate(streams):
+        upto = cfg.context - 128 * s          # different lengths per sequence
+        for t0, n in st.prefill_chunks():
+            if t0 >= upto:
+                break
+            q, k, v = st.tokens(t0, n)
+            sp.prefill(s, q, k, v, check_out=(t0 + n >= upto))
+    lens = [cfg.context - 128 * s for s in range(3)]
+    for step in range(cfg.decode_steps):
+        qs, ks, vs = [], [], []
+        for s, st in enumerate(streams):
+            q, k, v = st.tokens(lens[s] + step, 1, kind=1)
+            qs.append(q[:, 0]); ks.append(k[:, 0]); vs.append(v[:, 0])
+        order = [2, 0, 1] if step % 2 else [0, 1, 2]
+        sp.decode(order, torch.stack([qs[i] for i in order]), torch.stack([ks[i] for i in order]),
+                  torch.stack([vs[i] for i in order]))
+    sp.lt.close()
+    print(sp.rep)
+
+
+def test_layer_ranges_are_independent_streams():
+    cfg = small_cfg(n_layers=2, context=512, decode_steps=0)
+    lt = binding.Ltri(ph.params_of(cfg))
+    st = inputs.SyntheticStream(cfg)
+    outs_all, outs_split = [], []
+    for t0, n in st.prefill_chunks():
+        q, k, v = (x.cuda() for x in st.tokens(t0, n))
+        outs_all.append(lt.ltri_prefill_chunk(0, 0, 2, q, k, v))
+    lt.ltri_reset_sequence(0)
+    for t0, n in st.prefill_chunks():
+        q, k, v = (x.cuda() for x in st.tokens(t0, n))
+        o0 = lt.ltri_prefill_chunk(0, 0, 1, q[:1].contiguous(), k[:1].contiguous(), v[:1].contiguous())
+        o1 = lt.ltri_prefill_chunk(0, 1, 1, q[1:].contiguous(), k[1:].contiguous(), v[1:].contiguous())
+        outs_split.append(torch.cat([o0, o1]))
+    torch.cuda.synchronize()
+    for a, b in zip(outs_all, outs_split):
+        assert torch.equal(a, b)
+    lt.close()
+
+
+def test_state_and_capacity_errors():
+    cfg = small_cfg(n_layers=2, context=256, decode_steps=2)
+    lt = binding.Ltri(ph.params_of(cfg))
+    st = inputs.SyntheticStream(cfg)
+    q, k, v = (x.cuda() for x in st.tokens(0, 128))
+    with pytest.raises(binding.LtriError) as e:
+        lt.ltri_decode_step([0], 0, 2, q[:, 0][None], k[:, 0][None], v[:, 0][None])   # nothing prefilled yet
+    assert e.value.code == binding.LTRI_ESTATE
+    lt.ltri_prefill_chunk(0, 0, 2, q, k, v)
+    with pytest.raises(binding.LtriError) as e:
+        lt.ltri_prefill_chunk(0, 1, 1, q[1:].contiguous(), k[1:].contiguous(), v[1:].contiguous())
+        lt.ltri_prefill_chunk(0, 0, 2, q, k, v)                                       # layers out of step
+    assert e.value.code == binding.LTRI_ESTATE
+    lt.ltri_reset_sequence(0)
+    lt.ltri_prefill_chunk(0, 0, 2, q, k, v)
+    lt.ltri_prefill_chunk(0, 0, 2, q, k, v)
+    with pytest.raises(binding.LtriError) as e:
+        lt.ltri_prefill_chunk(0, 0, 2, q, k, v)                                       # beyond max_tokens - decode room
+    assert e.value.code == binding.LTRI_ECAPACITY
+    qd, kd, vd = q[:, 0][None].contiguous(), k[:, 0][None].contiguous(), v[:, 0][None].contiguous()
+    lt.ltri_decode_step([0], 0, 2, qd, kd, vd)
+    with pytest.raises(binding.LtriError) as e:
+        lt.ltri_prefill_chunk(0, 0, 2, q[:, :1].contiguous(), k[:, :1].contiguous(), v[:, :1].contiguous())
+    assert e.value.code == binding.LTRI_ESTATE                                       # prefill after decode
+    with pytest.raises(binding.LtriError) as e:
+        lt.ltri_decode_step([0, 0], 0, 2, torch.cat([qd, qd]), torch.cat([kd, kd]), torch.cat([vd, vd]))
+    assert e.value.code == binding.LTRI_EINVAL                                       # duplicate / too many seqs
+    with pytest.raises(binding.LtriError) as e:
+        lt.ltri_prefill_chunk(0, 0, 3, q, k, v)
+    assert e.value.code == binding.LTRI_EINVAL
+    torch.cuda.synchronize()
+    assert lt.ltri_sync_status() == 0
+    lt.close()
