@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the streaming span-retrieval attention path on B200.
+
+A step is one `ltri_prefill_chunk` call: one chunk of the workload's stream through every
+layer (append, evict + index, local attention, local-map pass, segmentation, scoring +
+top-k, gather + retrieved attention).  The timed steps are the LAST K chunks of the
+context, so the reported prefill throughput is the one at full context length; the chunks
+before them are streamed untimed as set-up.  After the prefill measurement the workload's
+decode steps are timed the same way and reported under "decode".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ltri|reference]
+
+With N > 1 (launched by torchrun, one rank per GPU) every rank streams its own replica of
+the workload; nothing is exchanged (the path does not shard: replicas only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2412_04757_b200 import inputs  # noqa: E402
+
+METRIC = "streamed prefill tok/s at full context (decode tok/s and roofline fractions alongside)"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only)."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return rank, local, world
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x: float, world, device):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(x: float, world, device):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(cfg, steps, warmup):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: layer 0 of the first
+    prefill calls of the stream until the window is full, then `steps` timed calls.  Returns tok/s
+    extrapolated to all layers, the cores it ran on and a description of the sample."""
+    from oracle import ltri_oracle as orc  # test infrastructure: only this CPU-baseline leg touches it
+
+    one = inputs.StreamConfig(**{**cfg.__dict__, "n_layers": 1, "n_seqs": 1})
+    st = inputs.SyntheticStream(one)
+    fill = (cfg.window + cfg.chunk - 1) // cfg.chunk + 1
+    need = (fill + warmup + steps) * cfg.chunk
+    o = orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
+                         need + 8, reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
+                         theta_mode=cfg.theta_mode, theta=cfg.theta)
+    times = []
+    for ci in range(fill + warmup + steps):
+        q, k, v = st.tokens(ci * cfg.chunk, cfg.chunk)
+        t = time.perf_counter()
+        if ci < fill:
+            o.prefill_local(q[0], k[0], v[0])      # state only: fills the window and the index
+            o.prefill_retrieve()
+        else:
+            o.prefill_chunk(q[0], k[0], v[0])
+        dt = time.perf_counter() - t
+        if ci >= fill + warmup:
+            times.append(dt)
+    per_call_layer = sum(times) / len(times)
+    toks = cfg.chunk / (per_call_layer * cfg.n_layers)
+    cores = min(cfg.n_q_heads, os.cpu_count() or 1)
+    sample = (f"layer 0 of {cfg.name}: {steps} full prefill calls of {cfg.chunk} tokens with the {cfg.window}-token "
+              f"window full (after {fill} state-only calls), time x {cfg.n_layers} layers")
+    return toks, cores, sample, per_call_layer
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 4))
+    warm = min(args.warmup, 1)
+    toks, cores, sample, per = oracle_sample(cfg, steps, warm)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": toks, "unit": "tok/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": per * cfg.n_layers * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "chunk": cfg.chunk, "window": cfg.window, "top_k": cfg.top_k},
+        "cpu_baseline": {"value": toks, "unit": "tok/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": toks, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+def attn_local_flops(cfg, t0, n, E):
+    """Algorithmic flops of the local attention kernel for one call (all layers): QK^T + PV over
+    sink + local + causal current keys."""
+    keys = min(cfg.n_sink, t0) + (t0 - min(E, t0)) + (n + 1) / 2.0
+    return 4.0 * n * cfg.n_q_heads * cfg.head_dim * keys * cfg.n_layers
+
+
+def run_ltri(args, cfg):
+    from paper_2412_04757_b200 import binding, build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    rank, local, world = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    build.build()
+    peaks = measured_peaks()
+    L, n = cfg.n_layers, cfg.chunk
+    chunks = list(inputs.prefill_calls(cfg))
+    K, W = args.steps, args.warmup
+    if K + W > len(chunks):
+        raise SystemExit(f"steps+warmup = {K + W} exceeds the {len(chunks)} prefill calls of {cfg.name}")
+    first_timed = len(chunks) - K
+    first_warm = first_timed - W
+
+    st = inputs.SyntheticStream(cfg, seq=rank, device=dev)
+    p = binding.make_params(L, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_tokens, cfg.chunk, cfg.window, cfg.n_sink,
+                            cfg.top_k, head_dim=cfg.head_dim, max_seqs=1, reps_per_span=cfg.reps_per_span,
+                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta)
+
+    def stream_until(lt, upto, keep_from):
+        kept = []
+        for ci, (t0, cnt) in enumerate(chunks[:upto]):
+            q, k, v = st.tokens(t0, cnt)
+            if ci >= keep_from:
+                kept.append((q, k, v))
+            else:
+                lt.ltri_prefill_chunk(0, 0, L, q, k, v)
+        return kept
+
+    lt = binding.Ltri(p, device=dev)
+    # set-up: stream everything before the warm-up chunks, generate (and keep) warm-up + timed inputs
+    kept = stream_until(lt, len(chunks), first_warm)
+    outs = [torch.empty_like(kept[0][0]) for _ in range(2)]
+    dec_in = [tuple(x.permute(1, 0, 2, 3).contiguous() for x in st.tokens(cfg.context + s, 1, kind=1))
+              for s in range(cfg.decode_steps)]
+    torch.cuda.synchronize(dev)
+
+    # ---- device-resident timing ------------------------------------------------------------
+    for i in range(W):
+        lt.ltri_prefill_chunk(0, 0, L, *kept[i], out=outs[i & 1])
+    torch.cuda.synchronize(dev)
+    lt.ltri_profile_read()                      # clears counters
+    lt.ltri_profile_enable(True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = lt.ltri_launch_count()
+    barrier(world)
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K):
+        lt.ltri_prefill_chunk(0, 0, L, *kept[W + i], out=outs[i & 1])
+    e1.record()
+    torch.cuda.synchronize(dev)
+    barrier(world)
+    ms = e0.elapsed_time(e1)
+    launches = lt.ltri_launch_count() - launches0
+    prof = lt.ltri_profile_read()
+    lt.ltri_profile_enable(False)
+    assert lt.ltri_sync_status() == 0, "device-side status word reports an error"
+    stats = lt.ltri_get_stats(0, 0)
+    ms = max_over_ranks(ms, world, dev)
+    tokens = K * n
+    prefill_tps = sum_over_ranks(tokens / (ms * 1e-3), world, dev) if world > 1 else tokens / (ms * 1e-3)
+
+    # ---- decode (state is now at full context) ----------------------------------------------
+    dec = None
+    if cfg.decode_steps > 0:
+        dout = torch.empty_like(dec_in[0][0])
+        dw = min(3, cfg.decode_steps // 2)
+        for s in range(dw):
+            lt.ltri_decode_step([0], 0, L, *dec_in[s], out=dout)
+        torch.cuda.synchronize(dev)
+        lt.ltri_profile_read()
+        lt.ltri_profile_enable(True)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier(world)
+        d0.record()
+        for s in range(dw, cfg.decode_steps):
+            lt.ltri_decode_step([0], 0, L, *dec_in[s], out=dout)
+        d1.record()
+        torch.cuda.synchronize(dev)
+        dms = max_over_ranks(d0.elapsed_time(d1), world, dev)
+        dprof = lt.ltri_profile_read()
+        lt.ltri_profile_enable(False)
+        dsteps = cfg.decode_steps - dw
+        dst = lt.ltri_get_stats(0, 0)
+        ret_tok = dst.retrieved_tokens / cfg.n_kv_heads
+        keys = cfg.n_sink + ret_tok + (dst.tokens - dst.evicted_end)
+        # algorithmic bytes per step: index scan + K and V rows once per KV head
+        bytes_step = L * (cfg.n_kv_heads * dst.n_spans * cfg.head_dim * 2 + 2 * cfg.n_kv_heads * cfg.head_dim * 2 * keys)
+        k_ms = dprof["decode_retrieve"][0] + dprof["decode_attn"][0]
+        dec = {"value": world * dsteps / (dms * 1e-3), "unit": "tok/s", "steps": dsteps, "ms_per_step": dms / dsteps,
+               "keys_per_head": keys, "index_spans": dst.n_spans,
+               "roofline": {"bound": "hbm", "achieved": bytes_step * dsteps / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None,
+                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": (bytes_step * dsteps / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]) if k_ms > 0 else None,
+                            "traffic": None, "kernels": "decode score+top-k and split-KV attention+merge",
+                            "of": peaks["source"]},
+               "kernel_ms_per_step": {k: v[0] / dsteps for k, v in dprof.items() if v[1]}}
+    clocks = sampler.stop()
+
+    # ---- end-to-end: same steps with host buffers ---------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        lt.close()
+        del lt
+        torch.cuda.empty_cache()
+        lt = binding.Ltri(p, device=dev)
+        stream_until(lt, first_warm, len(chunks))
+        host = [tuple(x.cpu().pin_memory() for x in kept[i]) for i in range(W + K)]
+        hout = torch.empty(kept[0][0].shape, dtype=torch.bfloat16).pin_memory()
+        dq, dk, dv = (torch.empty_like(x) for x in kept[0])
+        h2d = sum(x.numel() * 2 for x in host[0])
+        d2h = hout.numel() * 2
+        del kept
+
+        def step(i):
+            dq.copy_(host[i][0], non_blocking=True)
+            dk.copy_(host[i][1], non_blocking=True)
+            dv.copy_(host[i][2], non_blocking=True)
+            lt.ltri_prefill_chunk(0, 0, L, dq, dk, dv, out=outs[0])
+            hout.copy_(outs[0], non_blocking=True)
+
+        for i in range(W):
+            step(i)
+        torch.cuda.synchronize(dev)
+        barrier(world)
+        t0 = time.perf_counter()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for i in range(K):
+            step(W + i)
+        g1.record()
+        torch.cuda.synchronize(dev)
+        wall = (time.perf_counter() - t0) * 1e3
+        ems = max_over_ranks(max(g0.elapsed_time(g1), wall), world, dev)
+        e2e = {"value": world * tokens / (ems * 1e-3), "unit": "tok/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ems / K}
+    lt.close()
+
+    if rank != 0:
+        return
+    # ---- roofline of the dominant kernel (local attention), live CUDA-event time -------------
+    flops = sum(attn_local_flops(cfg, t0, cnt, max(cfg.n_sink, t0 - cfg.window - (t0 % cfg.chunk)))
+                for (t0, cnt) in chunks[first_timed:])
+    a_ms, a_cnt = prof["attn_local"]
+    tf = flops / (a_ms * 1e-3) / 1e12 if a_ms > 0 else None
+    peak_tf = peaks["bf16_tflops_sustained"]
+    roof = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
+            "frac": tf / peak_tf if tf else None, "traffic": None, "kernel": "k_attn_prefill (local part)",
+            "launches": a_cnt, "ms_per_launch": a_ms / max(a_cnt, 1), "of": peaks["source"] + " (sustained)"}
+    cpu = None
+    if not args.no_cpu_baseline:
+        ctoks, cores, sample, _ = oracle_sample(cfg, 2, 0)
+        cpu = {"value": ctoks, "unit": "tok/s", "cores": cores, "kind": "oracle", "sample": sample}
+    line = {
+        "metric": METRIC, "value": prefill_tps, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
+                   "context": cfg.context, "chunk": cfg.chunk, "window": cfg.window, "sink": cfg.n_sink,
+                   "top_k": cfg.top_k, "timed_positions": [chunks[first_timed][0], cfg.context],
+                   "l2": "inputs of every step are distinct and larger than L2 (no flush needed)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "index_spans": stats.n_spans, "retrieved_tokens_per_kv_head": stats.retrieved_tokens / cfg.n_kv_heads},
+        "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "decode": dec, "roofline": roof, "cpu_baseline": cpu,
+        "kernel_ms_per_step": {k: v[0] / K for k, v in prof.items() if v[1]},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=32)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (2 = 128K needle, the headline)")
+    ap.add_argument("--impl", default="ltri", choices=["ltri", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = inputs.config(args.config)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ltri(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -133,6 +133,29 @@ int ltri_sync_status(ltri_ctx* ctx, void* cuda_stream);
 int ltri_last_cuda_error(const ltri_ctx* ctx);
 const char* ltri_strerror(int code);
 
+/* ---- measurement hooks ---- */
+
+/* Kernel classes reported by ltri_profile_read. */
+enum {
+  LTRI_K_APPEND = 0,   /* K/V cache append */
+  LTRI_K_EVICT,        /* eviction + span index build (Eq. 6) */
+  LTRI_K_ATTN_LOCAL,   /* prefill attention over sink | local | current */
+  LTRI_K_MAP,          /* local-map pass: votes + region map (Eq. 4, Eq. 6) */
+  LTRI_K_SEGMENT,      /* theta, cumulative sums, anti-diagonal filter, NMS, query representatives */
+  LTRI_K_SCORE_TOPK,   /* prefill similarity scores + top-k (Eq. 7-8) */
+  LTRI_K_ATTN_RET,     /* prefill attention over the retrieved spans + merge */
+  LTRI_K_DEC_RETRIEVE, /* decode scores + top-k */
+  LTRI_K_DEC_ATTN,     /* decode split-KV attention + merge */
+  LTRI_K_COUNT
+};
+/* Kernels launched by this context since it was created (host counter). */
+int64_t ltri_launch_count(const ltri_ctx* ctx);
+/* While enabled, every kernel class of a call is bracketed by CUDA events on the call's stream. */
+int ltri_profile_enable(ltri_ctx* ctx, int on);
+/* Synchronises the stream; writes, per class, the summed event time in ms (0 if profiling was off) and the
+ * kernels launched since the previous read: ms[LTRI_K_COUNT], launches[LTRI_K_COUNT] (HOST). */
+int ltri_profile_read(ltri_ctx* ctx, float* ms, int64_t* launches, void* cuda_stream);
+
 /* ---- debug / test entry points ---- */
 
 enum {

@@ -21,8 +21,10 @@ EXPORTS = [
     "ltri_arena_bytes", "ltri_create", "ltri_destroy", "ltri_reset_sequence", "ltri_prefill_chunk",
     "ltri_decode_step", "ltri_get_spans", "ltri_get_pending_spans", "ltri_get_selected", "ltri_get_stats",
     "ltri_sync_status", "ltri_last_cuda_error", "ltri_strerror", "ltri_debug_read", "ltri_span_capacity",
-    "ltri_debug_segment_map",
+    "ltri_debug_segment_map", "ltri_launch_count", "ltri_profile_enable", "ltri_profile_read",
 ]
+KERNEL_CLASSES = ["append", "evict_index", "attn_local", "map_pass", "segment", "score_topk", "attn_retrieved",
+                  "decode_retrieve", "decode_attn"]
 
 
 class LtriParams(C.Structure):
@@ -79,6 +81,10 @@ def load():
         L.ltri_debug_read.argtypes = [vp, ip, ip, ip, vp, C.c_size_t, C.POINTER(C.c_size_t), vp]
         L.ltri_span_capacity.argtypes = [vp]
         L.ltri_debug_segment_map.argtypes = [vp, vp, ip, ip, C.c_float, C.c_int64, ip, vp, ip, C.POINTER(ip), vp]
+        L.ltri_launch_count.restype = C.c_int64
+        L.ltri_launch_count.argtypes = [vp]
+        L.ltri_profile_enable.argtypes = [vp, ip]
+        L.ltri_profile_read.argtypes = [vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -202,6 +208,21 @@ class Ltri:
 
     def ltri_last_cuda_error(self) -> int:
         return int(self.lib.ltri_last_cuda_error(self._h))
+
+    def ltri_launch_count(self) -> int:
+        return int(self.lib.ltri_launch_count(self._h))
+
+    def ltri_profile_enable(self, on: bool):
+        _check(self.lib.ltri_profile_enable(self._h, 1 if on else 0), "ltri_profile_enable")
+
+    def ltri_profile_read(self, stream=None):
+        """{class name: (ms, launches)} since the previous read."""
+        n = len(KERNEL_CLASSES)
+        ms = np.zeros(n, dtype=np.float32)
+        cnt = np.zeros(n, dtype=np.int64)
+        _check(self.lib.ltri_profile_read(self._h, ms.ctypes.data_as(C.c_void_p), cnt.ctypes.data_as(C.c_void_p),
+                                          self._stream(stream)), "ltri_profile_read")
+        return {KERNEL_CLASSES[i]: (float(ms[i]), int(cnt[i])) for i in range(n)}
 
     def ltri_span_capacity(self) -> int:
         return int(self.lib.ltri_span_capacity(self._h))

@@ -119,6 +119,16 @@ struct ltri_ctx {
   std::vector<LayerState> st;  // [max_seqs][n_layers]
   int last_cuda = 0;
   int sm_count = 148;
+  long long launches = 0;  // kernels launched since creation
+  // optional per-kernel-class timing with CUDA events on the launching stream
+  bool profiling = false;
+  struct Timed {
+    cudaEvent_t a, b;
+    int cls;
+  };
+  std::vector<Timed> timed;      // recorded since the last read
+  std::vector<Timed> free_pool;  // reusable event pairs
+  long long cls_launches[LTRI_K_COUNT] = {0};
   LayerState& at(int seq, int layer) { return st[(size_t)seq * d.NL + layer]; }
 };
 
@@ -136,6 +146,32 @@ int cuda_fail(ltri_ctx* ctx, cudaError_t e) {
   } while (0)
 
 bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// Brackets one kernel group with events when profiling is on, and counts its kernels.
+struct Scope {
+  ltri_ctx* ctx;
+  cudaStream_t st;
+  ltri_ctx::Timed t;
+  bool on;
+  Scope(ltri_ctx* c, cudaStream_t s, int cls, int kernels) : ctx(c), st(s), on(false) {
+    ctx->launches += kernels;
+    ctx->cls_launches[cls] += kernels;
+    if (!ctx->profiling) return;
+    if (!ctx->free_pool.empty()) {
+      t = ctx->free_pool.back();
+      ctx->free_pool.pop_back();
+    } else if (cudaEventCreate(&t.a) != cudaSuccess || cudaEventCreate(&t.b) != cudaSuccess) {
+      return;
+    }
+    t.cls = cls;
+    on = cudaEventRecord(t.a, st) == cudaSuccess;
+  }
+  ~Scope() {
+    if (!on) return;
+    cudaEventRecord(t.b, st);
+    ctx->timed.push_back(t);
+  }
+};
 
 }  // namespace
 
@@ -179,6 +215,11 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
 
 int ltri_destroy(ltri_ctx* ctx) {
   if (!ctx) return LTRI_EINVAL;
+  for (auto* pool : {&ctx->timed, &ctx->free_pool})
+    for (auto& t : *pool) {
+      cudaEventDestroy(t.a);
+      cudaEventDestroy(t.b);
+    }
   delete ctx;
   return LTRI_OK;
 }
@@ -255,8 +296,12 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   a.v = static_cast<const __nv_bfloat16*>(v);
   a.out = static_cast<__nv_bfloat16*>(out);
 
-  LTRI_CUDA(ctx, launch_append_prefill(d, a, st));
+  {
+    Scope sc(ctx, st, LTRI_K_APPEND, 1);
+    LTRI_CUDA(ctx, launch_append_prefill(d, a, st));
+  }
   for (size_t i = 0; i < ev.size(); i += 8) {
+    Scope sc(ctx, st, LTRI_K_EVICT, 1);
     EvictArgs ea;
     ea.seq = seq;
     ea.layer_begin = layer_begin;
@@ -265,17 +310,28 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
     LTRI_CUDA(ctx, launch_evict_index(d, ea, layer_count, st));
   }
   const bool has_index = ub > 0;
-  LTRI_CUDA(ctx, launch_attn_prefill(d, a, 0, !has_index, st));
-  LTRI_CUDA(ctx, launch_map_pass(d, a, st));
+  {
+    Scope sc(ctx, st, LTRI_K_ATTN_LOCAL, 1);
+    LTRI_CUDA(ctx, launch_attn_prefill(d, a, 0, !has_index, st));
+  }
+  {
+    Scope sc(ctx, st, LTRI_K_MAP, (a.t0 - a.loc_begin > 0 && a.loc_begin >= d.Ls) ? 2 : 1);
+    LTRI_CUDA(ctx, launch_map_pass(d, a, st));
+  }
   if (m > 0) {
+    Scope sc(ctx, st, LTRI_K_SEGMENT, 4);
     long long thq_abs = 0;
     if (d.theta_mode == 0) thq_abs = (long long)std::nearbyint((double)d.theta * (double)d.Hq * (double)kQScale);
     LTRI_CUDA(ctx, launch_segment(d, seq, layer_begin, layer_count, m, reg_start, slot, d.theta_mode, d.theta, thq_abs,
                                   d.C, n_tokens, t0, a.q, st));
   }
   if (has_index) {
-    LTRI_CUDA(ctx, launch_score_prefill(d, a, (int)ub, st));
-    LTRI_CUDA(ctx, launch_topk_prefill(d, a, st));
+    {
+      Scope sc(ctx, st, LTRI_K_SCORE_TOPK, 2);
+      LTRI_CUDA(ctx, launch_score_prefill(d, a, (int)ub, st));
+      LTRI_CUDA(ctx, launch_topk_prefill(d, a, st));
+    }
+    Scope sc(ctx, st, LTRI_K_ATTN_RET, 1);
     LTRI_CUDA(ctx, launch_attn_prefill(d, a, 1, true, st));
   }
   // commit the host state
@@ -331,9 +387,16 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
     const int units = b.n * layer_count * d.Hkv;
     int nsplit = (ctx->sm_count * 8 + units - 1) / units;
     nsplit = std::max(1, std::min(nsplit, kMaxDecSplit));
-    LTRI_CUDA(ctx, launch_append_decode(d, b, layer_begin, layer_count, n_seqs, kb, vb, st));
-    LTRI_CUDA(ctx, launch_score_decode(d, b, layer_begin, layer_count, n_seqs, qb, (int)ub, st));
-    LTRI_CUDA(ctx, launch_topk_decode(d, b, layer_begin, layer_count, st));
+    {
+      Scope sc(ctx, st, LTRI_K_APPEND, 1);
+      LTRI_CUDA(ctx, launch_append_decode(d, b, layer_begin, layer_count, n_seqs, kb, vb, st));
+    }
+    {
+      Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 2);
+      LTRI_CUDA(ctx, launch_score_decode(d, b, layer_begin, layer_count, n_seqs, qb, (int)ub, st));
+      LTRI_CUDA(ctx, launch_topk_decode(d, b, layer_begin, layer_count, st));
+    }
+    Scope sc(ctx, st, LTRI_K_DEC_ATTN, 2);
     LTRI_CUDA(ctx, launch_decode_attn(d, b, layer_begin, layer_count, n_seqs, qb, ob, nsplit, st));
   }
   for (int i = 0; i < n_seqs; ++i)
@@ -453,6 +516,31 @@ int ltri_sync_status(ltri_ctx* ctx, void* cuda_stream) {
 }
 
 int ltri_last_cuda_error(const ltri_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int64_t ltri_launch_count(const ltri_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int ltri_profile_enable(ltri_ctx* ctx, int on) {
+  if (!ctx) return LTRI_EINVAL;
+  ctx->profiling = on != 0;
+  return LTRI_OK;
+}
+
+int ltri_profile_read(ltri_ctx* ctx, float* ms, int64_t* launches, void* cuda_stream) {
+  if (!ctx || !ms || !launches) return LTRI_EINVAL;
+  LTRI_CUDA(ctx, cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+  for (int i = 0; i < LTRI_K_COUNT; ++i) {
+    ms[i] = 0.f;
+    launches[i] = ctx->cls_launches[i];
+    ctx->cls_launches[i] = 0;
+  }
+  for (auto& t : ctx->timed) {
+    float e = 0.f;
+    if (cudaEventElapsedTime(&e, t.a, t.b) == cudaSuccess) ms[t.cls] += e;
+    ctx->free_pool.push_back(t);
+  }
+  ctx->timed.clear();
+  return LTRI_OK;
+}
 
 const char* ltri_strerror(int code) {
   switch (code) {

@@ -177,16 +177,21 @@ class SyntheticStream:
 
     def prefill_chunks(self):
         """Yield (t0, n) of the prefill calls."""
-        t0 = 0
-        while t0 < self.cfg.context:
-            n = min(self.cfg.chunk, self.cfg.context - t0)
-            yield t0, n
-            t0 += n
+        return prefill_calls(self.cfg)
 
     def needle_range(self):
         if self.needle_segment < 0:
             return None
         return int(self.bounds[self.needle_segment]), int(self.bounds[self.needle_segment + 1])
+
+
+def prefill_calls(cfg: StreamConfig):
+    """Yield (t0, n) of the prefill calls that stream `cfg.context` tokens in chunks."""
+    t0 = 0
+    while t0 < cfg.context:
+        n = min(cfg.chunk, cfg.context - t0)
+        yield t0, n
+        t0 += n
 
 
 def random_stream(seed: int, n_tokens: int, n_q_heads: int, n_kv_heads: int, head_dim: int, sharp: float = 1.0):
