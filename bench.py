@@ -374,10 +374,18 @@ def main():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (2 = 128K needle, the headline)")
     ap.add_argument("--impl", default="ltri", choices=["ltri", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling of small cases)")
+    ap.add_argument("--context", type=int, default=0, help="override the context length (profiling of small cases)")
+    ap.add_argument("--decode-steps", type=int, default=-1, help="override the number of decode steps")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = inputs.config(args.config)
+    if args.layers > 0 or args.context > 0 or args.decode_steps >= 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, n_layers=args.layers or cfg.n_layers, context=args.context or cfg.context,
+                                  decode_steps=cfg.decode_steps if args.decode_steps < 0 else args.decode_steps)
+        cfg.name += f"[layers={cfg.n_layers},context={cfg.context},decode={cfg.decode_steps}]"
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
