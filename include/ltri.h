@@ -182,6 +182,25 @@ int ltri_span_capacity(const ltri_ctx* ctx);
 int ltri_debug_segment_map(ltri_ctx* ctx, const int32_t* Mq, int m, int theta_mode, float theta, int64_t theta_q,
                            int max_spans, int32_t* start_len_pairs, int cap, int* n_out, void* cuda_stream);
 
+/* ---- allocation-free entry point ---- */
+
+/* The paper has no counterpart for this call; it exists for callers that cannot allocate device memory at the
+ * point of use (code inside a fully committed memory pool, plugins of a host that forbids cudaMalloc after
+ * start-up, service threads that must stay off the allocator).  It runs the same segmenter as
+ * ltri_debug_segment_map, but needs no context and no arena: its scratch is a fixed array inside the library
+ * image (about 0.5 MiB, held by every GPU that loads the library until the process exits).
+ *   Mq     DEVICE int32 [m][m] dense row-major map (lower triangle used), 1 <= m <= LTRI_STATIC_SEGMENT_MAX_M
+ *   theta_q threshold in map units (Eq. 5), max_spans 1..64 (NMS cap)
+ *   pairs  DEVICE int32 [cap_pairs][2]: {start,len} spans partitioning [0,m); n_out DEVICE int32[1]: span count
+ * Larger m or max_spans return LTRI_ECAPACITY and launch nothing.  The call allocates nothing and returns
+ * without synchronising.  The first call on each device also looks up the scratch array's device address; make
+ * that first call outside any stream capture.  All calls share the one scratch array, which keeps the previous
+ * call's contents (the call clears what has to start at zero), so two calls that overlap on the GPU race: keep
+ * them on one stream or order them yourself. */
+#define LTRI_STATIC_SEGMENT_MAX_M 256
+int ltri_segment_map_static(const int32_t* Mq, int m, int64_t theta_q, int max_spans, int32_t* pairs, int cap_pairs,
+                            int32_t* n_out, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

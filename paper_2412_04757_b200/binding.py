@@ -22,6 +22,7 @@ EXPORTS = [
     "ltri_decode_step", "ltri_get_spans", "ltri_get_pending_spans", "ltri_get_selected", "ltri_get_stats",
     "ltri_sync_status", "ltri_last_cuda_error", "ltri_strerror", "ltri_debug_read", "ltri_span_capacity",
     "ltri_debug_segment_map", "ltri_launch_count", "ltri_profile_enable", "ltri_profile_read",
+    "ltri_segment_map_static",
 ]
 KERNEL_CLASSES = ["append", "evict_index", "attn_local", "map_pass", "segment", "score_topk", "attn_retrieved",
                   "decode_retrieve", "decode_attn"]
@@ -85,6 +86,7 @@ def load():
         L.ltri_launch_count.argtypes = [vp]
         L.ltri_profile_enable.argtypes = [vp, ip]
         L.ltri_profile_read.argtypes = [vp, vp, vp, vp]
+        L.ltri_segment_map_static.argtypes = [vp, ip, C.c_int64, ip, vp, ip, vp, vp]
         _lib = L
     return _lib
 
@@ -110,6 +112,22 @@ def _check(rc: int, where: str):
 
 def _dptr(t):
     return C.c_void_p(t.data_ptr())
+
+
+STATIC_SEGMENT_MAX_M = 256
+
+
+def ltri_segment_map_static(Mq, theta_q: int, max_spans: int, pairs, n_out, stream=None) -> int:
+    """Allocation-free segmenter for callers that cannot allocate device memory where they need it.
+
+    Mq: device int32 tensor [m][m]; pairs: device int32 tensor [cap][2]; n_out: device int32 tensor [1].
+    The scratch is a fixed array inside the library, so no context is needed; returns the C status code.
+    """
+    import torch
+
+    s = stream if stream is not None else torch.cuda.current_stream(Mq.device)
+    return int(load().ltri_segment_map_static(_dptr(Mq), Mq.shape[0], int(theta_q), max_spans, _dptr(pairs),
+                                              pairs.shape[0], _dptr(n_out), C.c_void_p(s.cuda_stream)))
 
 
 class Ltri:
