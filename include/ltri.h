@@ -166,8 +166,9 @@ enum {
   LTRI_BUF_THETA = 4,    /* int64 [1]: theta of the last prefill call in Q20 head-sum units */
   LTRI_BUF_SCORES = 5,   /* float [n_kv_heads][span_capacity]: similarity scores of the last call (Eq. 7) */
   LTRI_BUF_QREPS = 6,    /* float [n_kv_heads][2*max_spans_per_region+1][head_dim]: summed query representatives */
-  LTRI_BUF_ROWSTAT = 7   /* float [chunk][n_q_heads][2]: row max (raw dot-product units) and row sum of the
-                            local softmax of the last prefill call */
+  LTRI_BUF_ROWSTAT = 7   /* float [chunk][n_q_heads][2]: reference maximum m (logits * scale * log2(e); may lag the true
+                            row maximum by up to 8) and the matching row sum of exp2(logit - m) of the local softmax
+                            of the last prefill call */
 };
 /* Copy an internal buffer of (seq, layer) to HOST memory `dst`; *bytes_out = full size.  Synchronises. */
 int ltri_debug_read(ltri_ctx* ctx, int what, int seq, int layer, void* dst, size_t cap_bytes, size_t* bytes_out,

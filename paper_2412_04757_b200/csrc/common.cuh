@@ -105,6 +105,12 @@ cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_beg
 // prefill attention.  phase 0: local part over sink|local|cur, stores state (+ final output if `final`);
 // phase 1: continues from the stored state over the selected spans and writes the output.
 cudaError_t launch_attn_prefill(const DevCtx& c, const PrefillArgs& a, int phase, bool final, cudaStream_t s);
+// tcgen05/TMEM/TMA version of launch_attn_prefill (same contract) and its availability check
+constexpr int kTcMapBytes = 5 * 128;  // host storage for a context's K/V tensor maps
+cudaError_t launch_attn_prefill_tc(const DevCtx& c, const PrefillArgs& a, int phase, bool final, const void* kv_maps,
+                                   cudaStream_t s);
+bool tc_attention_supported(const DevCtx& c);
+bool tc_encode_kv_maps(const DevCtx& c, void* out_bytes);
 cudaError_t launch_map_pass(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
 
 cudaError_t launch_decode_attn(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,

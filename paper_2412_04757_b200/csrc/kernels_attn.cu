@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_prefill(DevCtx c, PrefillArgs a
   if (phase == 1) {
     if (tk0 < a.n) {
       const float2 st = c.rowstat[((size_t)layer * c.chunk + tk0) * c.Hq + h0];
-      mraw[0] = st.x;
+      mraw[0] = st.x / c2;
       lsum[0] = (lane & 3) == 0 ? st.y : 0.f;
       const float* op = c.Oacc + (((size_t)layer * c.chunk + tk0) * c.Hq + h0) * kD + 2 * (lane & 3);
 #pragma unroll
@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_prefill(DevCtx c, PrefillArgs a
     }
     if (tk1 < a.n) {
       const float2 st = c.rowstat[((size_t)layer * c.chunk + tk1) * c.Hq + h1];
-      mraw[1] = st.x;
+      mraw[1] = st.x / c2;
       lsum[1] = (lane & 3) == 0 ? st.y : 0.f;
       const float* op = c.Oacc + (((size_t)layer * c.chunk + tk1) * c.Hq + h1) * kD + 2 * (lane & 3);
 #pragma unroll
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_prefill(DevCtx c, PrefillArgs a
     const int tk = r == 0 ? tk0 : tk1, h = r == 0 ? h0 : h1;
     if (tk >= a.n) continue;
     if (phase == 0) {
-      if ((lane & 3) == 0) c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(mraw[r], lsum[r]);
+      if ((lane & 3) == 0) c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(mraw[r] * c2, lsum[r]);
       if (!final_out) {
         float* op = c.Oacc + (((size_t)layer * c.chunk + tk) * c.Hq + h) * kD + 2 * (lane & 3);
 #pragma unroll
@@ -253,9 +253,9 @@ cudaError_t launch_attn_prefill(const DevCtx& c, const PrefillArgs& a, int phase
 
 // ------------------------------------------------------------------------------------------
 // Quantised probability of one logit given its row statistics (reading of Eq. 1-3 in Q20 fixed point):
-// Aq = rint(2^20 * exp(scale*(s - max)) / sum).
-__device__ __forceinline__ int quant_prob(float s, float mraw, float inv_l_q, float c2) {
-  return __float2int_rn(exp2f((s - mraw) * c2) * inv_l_q);
+// Aq = rint(2^20 * exp2(s*scale*log2e - m) / sum), (m, sum) being the row statistics the attention kernel stored.
+__device__ __forceinline__ int quant_prob(float s, float m_scaled, float inv_l_q, float c2) {
+  return __float2int_rn(exp2f(fmaf(s, c2, -m_scaled)) * inv_l_q);
 }
 
 // reduce the per-thread column sums of a 16x64 warp tile over the 8 row groups and add them to sh_cols[64]

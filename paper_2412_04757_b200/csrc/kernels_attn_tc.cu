@@ -1,0 +1,558 @@
+// Prefill attention on the 5th-generation tensor cores (tcgen05.mma, TMEM accumulators, TMA-fed shared memory).
+//
+// One CTA owns 256 query rows of one (layer, KV head): two 128-row tiles Q0/Q1, each row = (token, head of the
+// group), so one K/V tile serves the whole GQA group.  Keys arrive in 128-slot tiles assembled by TMA from pieces of
+// 8..128 rows, which lets a tile be packed from several short spans ("span-indirect" tiles): every range is padded
+// to a multiple of 8 rows only.  Roles (10 warps):
+//   warps 0-3 / 4-7 : softmax of S0 / S1, one thread per row (tcgen05.ld), P written back to TMEM as bf16
+//   warp 8          : TMA producer (Q once, K/V pieces through a 2-stage ring)
+//   warp 9          : MMA issuer: S = Q K^T (both operands in shared memory), O += P V (P from TMEM, V MN-major)
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P aliases the first 64 columns of its S.
+// The issue order QK0, QK1, {PV0_j, QK0_j+1, PV1_j, QK1_j+1} keeps the tensor pipe busy with one tile's MMAs while
+// the other tile's softmax runs.  The running max is updated lazily (only when it grows by more than 2^8), in which
+// case the softmax thread rescales its O row in TMEM; the in-order tensor pipe guarantees the row is quiescent then.
+// Every wait is bounded; on expiry the CTA sets LTRI_ETIMEOUT in the status word, drains and frees its TMEM.
+#include <cuda.h>
+
+#include <cstring>
+
+#include "common.cuh"
+#include "tc_util.cuh"
+
+namespace ltri {
+
+using namespace tc;
+
+constexpr float kLog2eT = 1.4426950408889634f;
+constexpr int kTcThreads = 320;
+constexpr int kNumBoxes = 5;  // box heights 8,16,32,64,128
+constexpr float kRescaleThreshold = 8.0f;
+
+struct TcMaps {
+  CUtensorMap q;             // [tokens][Hq][128] bf16, box {64, G, 256/G}
+  CUtensorMap kv[kNumBoxes]; // K slabs followed by V slabs: [rows][128] bf16, box {64, 8<<i}
+};
+static_assert(sizeof(CUtensorMap) * kNumBoxes <= kTcMapBytes, "kTcMapBytes too small");
+
+struct RangeList {
+  int n;
+  int start[kMaxTopK + 2];
+  int len[kMaxTopK + 2];
+};
+
+// Deterministic tile builder: every role walks the same range list and derives the same tiles.  All state lives in
+// registers (no dynamically indexed arrays); only the producer asks for the piece list.
+struct TileIter {
+  const RangeList* rg;
+  int ri = 0, off = 0;
+  int causal_ri;  // index of the causal (current-chunk) range, -1 if none
+  // description of the current tile
+  unsigned m0, m1, m2, m3;  // valid-slot mask
+  int causal_tok0;          // absolute token of slot 0 when the tile is causal, else -1
+  bool full;                // all 128 slots valid and no causal masking
+  __device__ __forceinline__ void set_bits(int lo, int cnt) {
+    const int hi = lo + cnt;
+    auto word = [&](int w) -> unsigned {
+      const int a = max(lo, 32 * w), b = min(hi, 32 * w + 32);
+      if (b <= a) return 0u;
+      const int n = b - a;
+      return (n == 32 ? 0xffffffffu : ((1u << n) - 1u)) << (a - 32 * w);
+    };
+    m0 |= word(0);
+    m1 |= word(1);
+    m2 |= word(2);
+    m3 |= word(3);
+  }
+  // Advances to the next tile.  f(slot, token, box_index) is called for every piece when PIECES is set.
+  template <bool PIECES, typename F>
+  __device__ __forceinline__ bool next(F&& f) {
+    m0 = m1 = m2 = m3 = 0u;
+    causal_tok0 = -1;
+    int slot = 0;
+    while (slot < 128 && ri < rg->n) {
+      const int rem = rg->len[ri] - off;
+      if (rem <= 0) {
+        ++ri;
+        off = 0;
+        continue;
+      }
+      const bool causal = ri == causal_ri;
+      if (causal && slot != 0 && causal_tok0 < 0) break;  // the causal range starts a fresh tile
+      const int need = (rem + 7) & ~7;
+      const int room = 128 - slot;
+      const int lim = need < room ? need : room;
+      int bi = 4;
+      while ((8 << bi) > lim) --bi;
+      const int h = 8 << bi;
+      const int nvalid = h < rem ? h : rem;
+      const int tok = rg->start[ri] + off;
+      if (causal && slot == 0) causal_tok0 = tok;
+      if (PIECES) f(slot, tok, bi);
+      set_bits(slot, nvalid);
+      off += nvalid;
+      slot += h;
+    }
+    full = causal_tok0 < 0 && (m0 & m1 & m2 & m3) == 0xffffffffu;
+    return slot > 0;
+  }
+  __device__ __forceinline__ bool next() {
+    return next<false>([](int, int, int) {});
+  }
+  __device__ __forceinline__ unsigned mask(int w) const { return w == 0 ? m0 : w == 1 ? m1 : w == 2 ? m2 : m3; }
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int G>
+__global__ void __launch_bounds__(kTcThreads, 1)
+    k_attn_tc(DevCtx c, PrefillArgs a, int phase, int final_out, const __grid_constant__ TcMaps maps,
+              long long v_row_offset) {
+  const CUtensorMap* kvmaps = maps.kv;
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[14];
+  __shared__ uint32_t s_tmem_base;
+  __shared__ int s_abort;
+  __shared__ RangeList rg;
+  constexpr int TOKB = 256 / G;  // tokens per CTA
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
+  const size_t unit = unit_of(c, a.seq, layer);
+  const int tok0 = blockIdx.x * TOKB;
+  const uint32_t sbase = (smem_addr(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = sbase;                 // 64 KB: [half d][256 rows][64]
+  const uint32_t sKV = sbase + 65536;        // 2 stages x (K 32 KB | V 32 KB), each [half d][128 slots][64]
+  // barrier indices
+  enum { B_QFULL = 0, B_KFULL = 1, B_VFULL = 3, B_KEMPTY = 5, B_VEMPTY = 7, B_SREADY = 9, B_PREADY = 11, B_ODONE = 13 };
+  auto bar = [&](int i) { return smem_addr(&bars[i]); };
+  volatile int* abortp = &s_abort;
+
+  if (tid == 0) {
+    s_abort = 0;
+    mbar_init(bar(B_QFULL), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(B_KFULL + s), 1);
+      mbar_init(bar(B_VFULL + s), 1);
+      mbar_init(bar(B_KEMPTY + s), 1);
+      mbar_init(bar(B_VEMPTY + s), 1);
+      mbar_init(bar(B_SREADY + s), 1);
+      mbar_init(bar(B_PREADY + s), 4);
+    }
+    mbar_init(bar(B_ODONE), 1);
+    fence_mbar_init();
+    const int last_tok = min(a.n, tok0 + TOKB) - 1;
+    if (phase == 0) {
+      rg.n = 3;
+      rg.start[0] = 0;
+      rg.len[0] = a.sink_end;
+      rg.start[1] = a.loc_begin;
+      rg.len[1] = a.t0 - a.loc_begin;
+      rg.start[2] = a.t0;
+      rg.len[2] = last_tok + 1;
+    } else {
+      const size_t rb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
+      const int nr = min(c.rng_cnt[unit * c.Hkv + g], c.topk + 2);
+      rg.n = nr;
+      for (int i = 0; i < nr; ++i) {
+        rg.start[i] = c.rng_start[rb + i];
+        rg.len[i] = c.rng_len[rb + i];
+      }
+    }
+  }
+  // stale shared memory must never hold non-finite bit patterns: unfilled key slots are multiplied by P = 0
+  for (uint32_t i = tid; i < 131072 / 16; i += kTcThreads)
+    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(sKV + i * 16), "r"(0) : "memory");
+  fence_async_smem();
+  if (warp == 8) tmem_alloc(smem_addr(&s_tmem_base), 512);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem = s_tmem_base;
+  const int causal_ri = phase == 0 ? 2 : -1;
+  const size_t slab_row0 = (unit * c.Hkv + g) * (size_t)c.Tpad;
+
+  if (warp == 8) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      prefetch_tmap(&maps.q);
+      mbar_expect_tx(bar(B_QFULL), 65536);
+      tma_load_3d(sQ, &maps.q, 0, g * G, l * a.n + tok0, bar(B_QFULL));
+      tma_load_3d(sQ + 32768, &maps.q, 64, g * G, l * a.n + tok0, bar(B_QFULL));
+      TileIter it;
+      it.rg = &rg;
+      it.causal_ri = causal_ri;
+      int j = 0;
+      bool ok = true;
+      int pslot[16], ptok[16], pbox[16];
+      while (ok) {
+        int np = 0;
+        if (!it.next<true>([&](int slot, int tok, int bi) {
+              pslot[np] = slot;
+              ptok[np] = tok;
+              pbox[np] = bi;
+              ++np;
+            }))
+          break;
+        const int st = j & 1;
+        if (j >= 2) ok = mbar_wait(bar(B_KEMPTY + st), ((j >> 1) - 1) & 1, abortp);
+        if (!ok) break;
+        uint32_t bytes = 0;
+        for (int p = 0; p < np; ++p) bytes += (uint32_t)(8 << pbox[p]) * 256u;
+        mbar_expect_tx(bar(B_KFULL + st), bytes);
+        const uint32_t sK = sKV + st * 65536, sV = sK + 32768;
+        for (int p = 0; p < np; ++p) {
+          const CUtensorMap* m = &kvmaps[pbox[p]];
+          const long long row = (long long)slab_row0 + ptok[p];
+          const uint32_t so = (uint32_t)pslot[p] * 128u;
+          tma_load_2d(sK + so, m, 0, (int)row, bar(B_KFULL + st));
+          tma_load_2d(sK + 16384 + so, m, 64, (int)row, bar(B_KFULL + st));
+        }
+        if (j >= 2) ok = mbar_wait(bar(B_VEMPTY + st), ((j >> 1) - 1) & 1, abortp);
+        if (!ok) break;
+        mbar_expect_tx(bar(B_VFULL + st), bytes);
+        for (int p = 0; p < np; ++p) {
+          const CUtensorMap* m = &kvmaps[pbox[p]];
+          const long long row = (long long)slab_row0 + ptok[p] + v_row_offset;
+          const uint32_t so = (uint32_t)pslot[p] * 128u;
+          tma_load_2d(sV + so, m, 0, (int)row, bar(B_VFULL + st));
+          tma_load_2d(sV + 16384 + so, m, 64, (int)row, bar(B_VFULL + st));
+        }
+        ++j;
+      }
+      // drain: every stage that was filled is released by the MMA warp; wait for the last ones so that no copy is
+      // in flight when the CTA exits
+      for (int back = 1; back <= 2 && back <= j; ++back) {
+        const int jj = j - back;
+        if (!mbar_wait(bar(B_VEMPTY + (jj & 1)), (jj >> 1) & 1, abortp)) break;
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      TileIter it;
+      it.rg = &rg;
+      it.causal_ri = causal_ri;
+      int T = 0;
+      while (it.next()) ++T;
+      constexpr uint32_t idesc_qk = make_idesc(128, 128, false);
+      constexpr uint32_t idesc_pv = make_idesc(128, 128, true);
+      bool ok = mbar_wait(bar(B_QFULL), 0, abortp);
+      auto issue_qk = [&](int q, int st) {
+        const uint32_t sK = sKV + st * 65536;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t half = ks >> 2, kin = (ks & 3) * 32;
+          const uint64_t ad = make_desc(sQ + half * 32768 + q * 16384 + kin, 16, 1024);
+          const uint64_t bd = make_desc(sK + half * 16384 + kin, 16, 1024);
+          mma_ss(tmem + q * 128, ad, bd, idesc_qk, ks > 0);
+        }
+        mma_commit(bar(B_SREADY + q));
+      };
+      auto issue_pv = [&](int q, int st, bool acc) {
+        const uint32_t sV = sKV + st * 65536 + 32768;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          // 16 keys per step: 2 KB down the V tile; N = 128 spans both 64-wide halves (LBO = 16 KB)
+          const uint64_t bd = make_desc(sV + ks * 2048, 16384, 1024);
+          mma_ts(tmem + 256 + q * 128, tmem + q * 128 + ks * 8, bd, idesc_pv, acc || ks > 0);
+        }
+      };
+      if (ok && T > 0) {
+        ok = mbar_wait(bar(B_KFULL + 0), 0, abortp);
+        if (ok) {
+          fence_after_sync();
+          issue_qk(0, 0);
+          issue_qk(1, 0);
+          mma_commit(bar(B_KEMPTY + 0));
+        }
+        for (int j = 0; ok && j < T; ++j) {
+          const int st = j & 1, nst = st ^ 1;
+          const bool acc = (j > 0) || (phase == 1);
+          ok = mbar_wait(bar(B_VFULL + st), (j >> 1) & 1, abortp);
+          if (!ok) break;
+          ok = mbar_wait(bar(B_PREADY + 0), j & 1, abortp);
+          if (!ok) break;
+          fence_after_sync();
+          issue_pv(0, st, acc);
+          if (j + 1 < T) {
+            ok = mbar_wait(bar(B_KFULL + nst), ((j + 1) >> 1) & 1, abortp);
+            if (!ok) break;
+            fence_after_sync();
+            issue_qk(0, nst);
+          }
+          ok = mbar_wait(bar(B_PREADY + 1), j & 1, abortp);
+          if (!ok) break;
+          fence_after_sync();
+          issue_pv(1, st, acc);
+          mma_commit(bar(B_VEMPTY + st));
+          if (j + 1 < T) {
+            issue_qk(1, nst);
+            mma_commit(bar(B_KEMPTY + nst));
+          }
+        }
+      }
+      mma_commit(bar(B_ODONE));
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue, one thread per row
+    const int q = warp >> 2;
+    const int r = (warp & 3) * 32 + lane;        // row inside the 128-row tile = TMEM lane
+    const int rr = q * 128 + r;                  // row inside the CTA
+    const int tk = tok0 + rr / G;                // call-relative token
+    const int h = g * G + rr % G;
+    const bool row_ok = tk < a.n;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_base + q * 128;
+    const uint32_t tO = tmem + lane_base + 256 + q * 128;
+    const float c2 = c.scale * kLog2eT;
+    float m_used = -INFINITY, lsum = 0.f;
+    if (phase == 1) {
+      uint32_t v[32];
+      const float* op = c.Oacc + (((size_t)layer * c.chunk + (row_ok ? tk : 0)) * c.Hq + h) * kD;
+      if (row_ok) {
+        const float2 stt = c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h];
+        m_used = stt.x;
+        lsum = stt.y;
+      }
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 f = row_ok ? *reinterpret_cast<const float4*>(op + ch * 32 + e) : make_float4(0, 0, 0, 0);
+          v[e] = __float_as_uint(f.x);
+          v[e + 1] = __float_as_uint(f.y);
+          v[e + 2] = __float_as_uint(f.z);
+          v[e + 3] = __float_as_uint(f.w);
+        }
+        tmem_st32(tO + ch * 32, v);
+      }
+      tmem_st_wait();
+    }
+    TileIter it;
+    it.rg = &rg;
+    it.causal_ri = causal_ri;
+    int j = 0;
+    bool ok = true;
+    const int row_abs = a.t0 + tk;
+    while (it.next()) {
+      ok = mbar_wait(bar(B_SREADY + q), j & 1, abortp);
+      if (!ok) break;
+      fence_after_sync();
+      // pass 1: row maximum over the valid slots
+      float mt = -INFINITY;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t v[32];
+        tmem_ld32(tS + ch * 32, v);
+        tmem_ld_wait();
+        if (it.full) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) mt = fmaxf(mt, __uint_as_float(v[e]));
+        } else {
+          const unsigned mk = it.mask(ch);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            bool okc = (mk >> e) & 1u;
+            if (it.causal_tok0 >= 0) okc = okc && (it.causal_tok0 + ch * 32 + e <= row_abs);
+            if (okc) mt = fmaxf(mt, __uint_as_float(v[e]));
+          }
+        }
+      }
+      mt *= c2;
+      // lazy running maximum: move it only when it grows by more than the threshold (or on first use)
+      float alpha = 1.f;
+      const bool grow = mt > m_used + kRescaleThreshold || (m_used == -INFINITY && mt > -INFINITY);
+      if (grow) {
+        alpha = ex2(m_used - mt);  // 0 when m_used = -inf
+        m_used = mt;
+        lsum *= alpha;
+      }
+      const bool have_o = (j > 0) || (phase == 1);
+      if (have_o && __any_sync(0xffffffffu, grow)) {
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(tO + ch * 32, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+          tmem_st32(tO + ch * 32, v);
+        }
+        tmem_st_wait();
+      }
+      // pass 2: probabilities, row sum, P (bf16) back into the first 64 columns of S
+      const float mneg = m_used == -INFINITY ? 0.f : -m_used;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t v[32];
+        tmem_ld32(tS + ch * 32, v);
+        tmem_ld_wait();
+        uint32_t pk[16];
+        if (it.full) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(v[e]), c2, mneg));
+            const float p1 = ex2(fmaf(__uint_as_float(v[e + 1]), c2, mneg));
+            lsum += p0 + p1;
+            pk[e >> 1] = pack2(p0, p1);
+          }
+        } else {
+          const unsigned mk = it.mask(ch);
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            bool ok0 = (mk >> e) & 1u, ok1 = (mk >> (e + 1)) & 1u;
+            if (it.causal_tok0 >= 0) {
+              ok0 = ok0 && (it.causal_tok0 + ch * 32 + e <= row_abs);
+              ok1 = ok1 && (it.causal_tok0 + ch * 32 + e + 1 <= row_abs);
+            }
+            const float p0 = ok0 ? ex2(fmaf(__uint_as_float(v[e]), c2, mneg)) : 0.f;
+            const float p1 = ok1 ? ex2(fmaf(__uint_as_float(v[e + 1]), c2, mneg)) : 0.f;
+            lsum += p0 + p1;
+            pk[e >> 1] = pack2(p0, p1);
+          }
+        }
+        tmem_st16(tS + ch * 16, pk);
+      }
+      tmem_st_wait();
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_PREADY + q));
+      ++j;
+    }
+    // epilogue
+    if (ok) ok = mbar_wait(bar(B_ODONE), 0, abortp);
+    if (ok) {
+      fence_after_sync();
+      if (phase == 0 && row_ok)
+        c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(m_used, lsum);
+      const float inv = 1.f / lsum;
+      const bool have_o = (j > 0) || (phase == 1);
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t v[32];
+        if (have_o) {
+          tmem_ld32(tO + ch * 32, v);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = 0u;
+        }
+        if (!row_ok) continue;
+        if (phase == 0 && !final_out) {
+          float* op = c.Oacc + (((size_t)layer * c.chunk + tk) * c.Hq + h) * kD + ch * 32;
+#pragma unroll
+          for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<uint4*>(op + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+        }
+        if (final_out) {
+          __nv_bfloat16* op = a.out + (((size_t)l * a.n + tk) * c.Hq + h) * kD + ch * 32;
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            uint4 w;
+            w.x = pack2(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv);
+            w.y = pack2(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
+            w.z = pack2(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
+            w.w = pack2(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
+            *reinterpret_cast<uint4*>(op + e) = w;
+          }
+        }
+      }
+    }
+  }
+  // ------------------------------------------------------------------ teardown
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  if (warp == 8) tmem_dealloc(tmem, 512);
+  if (tid == 0 && s_abort) set_status(c, -6, (int)(blockIdx.x + 1000 * blockIdx.y));
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeFn get_encode() {
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeFn>(p);
+  }
+  return fn;
+}
+
+// K/V tensor maps of a context (box heights 8..128); `out` receives kNumBoxes CUtensorMap objects (host memory).
+bool tc_encode_kv_maps(const DevCtx& c, void* out_bytes) {
+  EncodeFn enc = get_encode();
+  if (!enc) return false;
+  CUtensorMap* out = static_cast<CUtensorMap*>(out_bytes);
+  const cuuint64_t rows = (cuuint64_t)c.NS * c.NL * c.Hkv * (cuuint64_t)c.Tpad * 2;  // K slabs then V slabs
+  for (int i = 0; i < kNumBoxes; ++i) {
+    cuuint64_t dims[2] = {128, rows};
+    cuuint64_t strides[1] = {256};
+    cuuint32_t box[2] = {64, (cuuint32_t)(8 << i)};
+    cuuint32_t es[2] = {1, 1};
+    if (enc(&out[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c.Kc, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  return true;
+}
+
+bool tc_attention_supported(const DevCtx& c) {
+  // the V slabs must follow the K slabs directly (one tensor map covers both) and row indices must fit 31 bits
+  const size_t rows = (size_t)c.NS * c.NL * c.Hkv * (size_t)c.Tpad;
+  if (c.Vc != c.Kc + rows * kD) return false;
+  if (rows * 2 >= (1ull << 31)) return false;
+  return get_encode() != nullptr;
+}
+
+template <int G>
+static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out, const void* kv_maps,
+                               cudaStream_t s) {
+  TcMaps maps;
+  EncodeFn enc = get_encode();
+  if (!enc || !kv_maps) return cudaErrorNotSupported;
+  memcpy(maps.kv, kv_maps, sizeof(maps.kv));
+  {
+    cuuint64_t dims[3] = {128, (cuuint64_t)c.Hq, (cuuint64_t)a.layer_count * a.n};
+    cuuint64_t strides[2] = {256, (cuuint64_t)c.Hq * 256};
+    cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(256 / G)};
+    cuuint32_t es[3] = {1, 1, 1};
+    if (enc(&maps.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(a.q), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  constexpr int TOKB = 256 / G;
+  const int smem = 65536 + 131072 + 1024;
+  cudaFuncSetAttribute(k_attn_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const long long v_off = (long long)c.NS * c.NL * c.Hkv * c.Tpad;
+  k_attn_tc<G><<<dim3((a.n + TOKB - 1) / TOKB, c.Hkv, a.layer_count), kTcThreads, smem, s>>>(c, a, phase,
+                                                                                           final_out ? 1 : 0, maps, v_off);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn_prefill_tc(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out,
+                                   const void* kv_maps, cudaStream_t s) {
+  switch (c.G) {
+    case 1: return launch_tc_g<1>(c, a, phase, final_out, kv_maps, s);
+    case 2: return launch_tc_g<2>(c, a, phase, final_out, kv_maps, s);
+    case 4: return launch_tc_g<4>(c, a, phase, final_out, kv_maps, s);
+    case 8: return launch_tc_g<8>(c, a, phase, final_out, kv_maps, s);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace ltri

@@ -1,6 +1,7 @@
 // C ABI of the ltri library: host-side stream state, arena layout and the launch sequences of a prefill call
 // and a decode step.  Everything that computes runs in the kernels; this file only orders them.
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <deque>
 #include <new>
@@ -119,6 +120,8 @@ struct ltri_ctx {
   std::vector<LayerState> st;  // [max_seqs][n_layers]
   int last_cuda = 0;
   int sm_count = 148;
+  bool use_tc = false;     // tcgen05/TMEM/TMA attention kernels (default when available)
+  alignas(64) unsigned char kv_maps[kTcMapBytes];  // TMA descriptors of the K/V cache
   long long launches = 0;  // kernels launched since creation
   // optional per-kernel-class timing with CUDA events on the launching stream
   bool profiling = false;
@@ -203,7 +206,13 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) ctx->sm_count = sms;
   }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  cudaError_t e = launch_init(ctx->d, -1, s);
+  const char* impl = std::getenv("LTRI_ATTN_IMPL");  // "mma" selects the warp-MMA kernels (debugging aid)
+  ctx->use_tc = tc_attention_supported(ctx->d) && !(impl && std::strcmp(impl, "mma") == 0) &&
+                tc_encode_kv_maps(ctx->d, ctx->kv_maps);
+  // unfilled tile slots and over-fetched rows must hold finite values: start from an all-zero cache
+  const size_t kv_bytes = (size_t)p->max_seqs * p->n_layers * ctx->d.Hkv * (size_t)ctx->d.Tpad * kD * 2 * sizeof(__nv_bfloat16);
+  cudaError_t e = cudaMemsetAsync(ctx->d.Kc, 0, kv_bytes, s);
+  if (e == cudaSuccess) e = launch_init(ctx->d, -1, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) {
     delete ctx;
@@ -312,7 +321,8 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   const bool has_index = ub > 0;
   {
     Scope sc(ctx, st, LTRI_K_ATTN_LOCAL, 1);
-    LTRI_CUDA(ctx, launch_attn_prefill(d, a, 0, !has_index, st));
+    LTRI_CUDA(ctx, ctx->use_tc ? launch_attn_prefill_tc(d, a, 0, !has_index, ctx->kv_maps, st)
+                               : launch_attn_prefill(d, a, 0, !has_index, st));
   }
   {
     Scope sc(ctx, st, LTRI_K_MAP, (a.t0 - a.loc_begin > 0 && a.loc_begin >= d.Ls) ? 2 : 1);
@@ -332,7 +342,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
       LTRI_CUDA(ctx, launch_topk_prefill(d, a, st));
     }
     Scope sc(ctx, st, LTRI_K_ATTN_RET, 1);
-    LTRI_CUDA(ctx, launch_attn_prefill(d, a, 1, true, st));
+    LTRI_CUDA(ctx, ctx->use_tc ? launch_attn_prefill_tc(d, a, 1, true, ctx->kv_maps, st) : launch_attn_prefill(d, a, 1, true, st));
   }
   // commit the host state
   for (int l = 0; l < layer_count; ++l) {
