@@ -177,6 +177,8 @@ class Ltri:
             out = self.torch.empty_like(q)
         rc = self.lib.ltri_prefill_chunk(self._h, seq, layer_begin, layer_count, n, _dptr(q), _dptr(k), _dptr(v),
                                          _dptr(out), self._stream(stream))
+        if rc == LTRI_ECUDA:
+            raise LtriError(rc, f"ltri_prefill_chunk (cudaError {self.ltri_last_cuda_error()})")
         _check(rc, "ltri_prefill_chunk")
         return out
 

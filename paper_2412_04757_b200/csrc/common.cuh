@@ -42,7 +42,8 @@ struct DevCtx {
   long long* Rsuf;       // [NL][chunk][chunk]
   long long* best;       // [NL][2*chunk]
   long long* thetaq;     // [NL]
-  float2* rowstat;       // [NL][chunk][Hq]   (row max in raw dot units, row sum)
+  float2* rowstat;       // [NL][chunk][Hq]   (reference maximum m in scaled log2 units, row sum l)
+  float2* rowq;          // [NL][chunk][Hq]   (-m, 2^20 / l): the map pass turns a logit into a Q20 probability with these
   float* Oacc;           // [NL][chunk][Hq][128]  unnormalised accumulator of the local part
   float* u;              // [NL][Hkv][Jmax][128]  summed query representatives
   int* Jcnt;             // [NL]
@@ -111,6 +112,7 @@ cudaError_t launch_attn_prefill_tc(const DevCtx& c, const PrefillArgs& a, int ph
                                    cudaStream_t s);
 bool tc_attention_supported(const DevCtx& c);
 bool tc_encode_kv_maps(const DevCtx& c, void* out_bytes);
+cudaError_t launch_map_pass_tc(const DevCtx& c, const PrefillArgs& a, const void* kv_maps, cudaStream_t s);
 cudaError_t launch_map_pass(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
 
 cudaError_t launch_decode_attn(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,

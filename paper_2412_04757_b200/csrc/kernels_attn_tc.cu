@@ -345,26 +345,29 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       ok = mbar_wait(bar(B_SREADY + q), j & 1, abortp);
       if (!ok) break;
       fence_after_sync();
-      // pass 1: row maximum over the valid slots
-      float mt = -INFINITY;
-#pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(tS + ch * 32, v);
-        tmem_ld_wait();
-        if (it.full) {
+      // the whole S row in registers: four 32-column loads in flight, one wait
+      uint32_t v[4][32];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) mt = fmaxf(mt, __uint_as_float(v[e]));
-        } else {
+      for (int ch = 0; ch < 4; ++ch) tmem_ld32(tS + ch * 32, v[ch]);
+      tmem_ld_wait();
+      const bool masked = !it.full;
+      if (masked) {
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
           const unsigned mk = it.mask(ch);
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
             bool okc = (mk >> e) & 1u;
             if (it.causal_tok0 >= 0) okc = okc && (it.causal_tok0 + ch * 32 + e <= row_abs);
-            if (okc) mt = fmaxf(mt, __uint_as_float(v[e]));
+            if (!okc) v[ch][e] = 0xff800000u;  // -inf
           }
         }
       }
+      float mt = -INFINITY;
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch)
+#pragma unroll
+        for (int e = 0; e < 32; ++e) mt = fmaxf(mt, __uint_as_float(v[ch][e]));
       mt *= c2;
       // lazy running maximum: move it only when it grows by more than the threshold (or on first use)
       float alpha = 1.f;
@@ -377,49 +380,33 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       const bool have_o = (j > 0) || (phase == 1);
       if (have_o && __any_sync(0xffffffffu, grow)) {
 #pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(tO + ch * 32, v);
+        for (int ch = 0; ch < 8; ++ch) {
+          uint32_t w[16];
+          tmem_ld16(tO + ch * 16, w);
           tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
-          tmem_st32(tO + ch * 32, v);
+          for (int e = 0; e < 16; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * alpha);
+          tmem_st16(tO + ch * 16, w);
         }
         tmem_st_wait();
       }
-      // pass 2: probabilities, row sum, P (bf16) back into the first 64 columns of S
+      // probabilities, row sum, P (bf16) into the first 64 columns of S.  Masked entries are -inf -> exp2 gives 0.
       const float mneg = m_used == -INFINITY ? 0.f : -m_used;
-#pragma unroll 1
+      float ls0 = 0.f, ls1 = 0.f;
+#pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(tS + ch * 32, v);
-        tmem_ld_wait();
         uint32_t pk[16];
-        if (it.full) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float p0 = ex2(fmaf(__uint_as_float(v[e]), c2, mneg));
-            const float p1 = ex2(fmaf(__uint_as_float(v[e + 1]), c2, mneg));
-            lsum += p0 + p1;
-            pk[e >> 1] = pack2(p0, p1);
-          }
-        } else {
-          const unsigned mk = it.mask(ch);
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            bool ok0 = (mk >> e) & 1u, ok1 = (mk >> (e + 1)) & 1u;
-            if (it.causal_tok0 >= 0) {
-              ok0 = ok0 && (it.causal_tok0 + ch * 32 + e <= row_abs);
-              ok1 = ok1 && (it.causal_tok0 + ch * 32 + e + 1 <= row_abs);
-            }
-            const float p0 = ok0 ? ex2(fmaf(__uint_as_float(v[e]), c2, mneg)) : 0.f;
-            const float p1 = ok1 ? ex2(fmaf(__uint_as_float(v[e + 1]), c2, mneg)) : 0.f;
-            lsum += p0 + p1;
-            pk[e >> 1] = pack2(p0, p1);
-          }
+        for (int e = 0; e < 32; e += 2) {
+          const float p0 = ex2(fmaf(__uint_as_float(v[ch][e]), c2, mneg));
+          const float p1 = ex2(fmaf(__uint_as_float(v[ch][e + 1]), c2, mneg));
+          ls0 += p0;
+          ls1 += p1;
+          pk[e >> 1] = pack2(p0, p1);
         }
         tmem_st16(tS + ch * 16, pk);
       }
+      lsum += ls0 + ls1;
       tmem_st_wait();
       fence_before_sync();
       __syncwarp();
@@ -430,8 +417,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     if (ok) ok = mbar_wait(bar(B_ODONE), 0, abortp);
     if (ok) {
       fence_after_sync();
-      if (phase == 0 && row_ok)
+      if (phase == 0 && row_ok) {
         c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(m_used, lsum);
+        c.rowq[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(-m_used, kQScale / lsum);
+      }
       const float inv = 1.f / lsum;
       const bool have_o = (j > 0) || (phase == 1);
 #pragma unroll 1

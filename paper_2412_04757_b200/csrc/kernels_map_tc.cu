@@ -1,0 +1,262 @@
+// Local-map pass on tcgen05 tensor cores: with the row statistics of the local softmax known, recompute the logits of
+// local | current keys and turn them into Q20 fixed-point probabilities (reading of Eq. 1-3), accumulating the votes of
+// Eq. 6 (column sums over all rows and heads) and the head-summed region map of Eq. 4.
+//
+// The product is computed transposed, S^T = K Q^T: a CTA keeps one 128-key tile in shared memory and streams all query
+// rows of its KV group through it in 128-row blocks (row = (token, head)).  With keys on the TMEM lanes every epilogue
+// thread owns one key, so a column sum of the map is a thread-local sum and needs no shuffles; the G heads of a token
+// are adjacent columns, so their sum (Eq. 4) is thread-local too and goes to the region map with one integer reduction
+// per (token, key, KV head).  Roles: warps 0-7 epilogue (two warps per lane quarter, 64 columns each), warp 8 TMA
+// producer, warp 9 MMA issuer; two TMEM accumulators and two Q stages overlap the MMAs with the exp/round epilogue.
+#include <cuda.h>
+
+#include <cstring>
+
+#include "common.cuh"
+#include "tc_util.cuh"
+
+namespace ltri {
+
+using namespace tc;
+
+constexpr float kLog2eM = 1.4426950408889634f;
+constexpr int kMapThreads = 320;
+
+struct MapMaps {
+  CUtensorMap q;    // [tokens][Hq][128] bf16, box {64, G, 128/G}
+  CUtensorMap k128; // K slabs, box {64, 128}
+};
+
+__device__ __forceinline__ float ex2m(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// grid (key tiles, Hkv, layers).  Key tiles [0, n_local_tiles) cover [loc_begin, t0); the rest cover [t0, t0+n).
+template <int G>
+__global__ void __launch_bounds__(kMapThreads, 2)
+    k_map_tc(DevCtx c, PrefillArgs a, int n_local_tiles, const __grid_constant__ MapMaps maps) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[9];
+  __shared__ uint32_t s_tmem_base;
+  __shared__ int s_abort;
+  __shared__ float2 s_stats[2][128];
+  constexpr int TPB = 128 / G;  // tokens per query block
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
+  const size_t unit = unit_of(c, a.seq, layer);
+  const bool is_cur = (int)blockIdx.x >= n_local_tiles;
+  // first key of the tile (absolute) and the end of its range
+  const int key0 = is_cur ? a.t0 + ((int)blockIdx.x - n_local_tiles) * 128 : a.loc_begin + (int)blockIdx.x * 128;
+  const int key_end = is_cur ? a.t0 + a.n : a.t0;
+  const int nblocks = (a.n + TPB - 1) / TPB;
+  // causal tiles: query blocks whose tokens all precede the tile's first key see none of its keys
+  const int blk0 = is_cur ? (key0 - a.t0) / TPB : 0;
+
+  const uint32_t sbase = (smem_addr(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sK = sbase;            // 32 KB: [half d][128 keys][64]
+  const uint32_t sQ = sbase + 32768;    // 2 stages x 32 KB: [half d][128 rows][64]
+  enum { B_KFULL = 0, B_QFULL = 1, B_QEMPTY = 3, B_SFULL = 5, B_SEMPTY = 7 };
+  auto bar = [&](int i) { return smem_addr(&bars[i]); };
+  volatile int* abortp = &s_abort;
+  if (tid == 0) {
+    s_abort = 0;
+    mbar_init(bar(B_KFULL), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(B_QFULL + s), 1);
+      mbar_init(bar(B_QEMPTY + s), 1);
+      mbar_init(bar(B_SFULL + s), 1);
+      mbar_init(bar(B_SEMPTY + s), 8);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 8) tmem_alloc(smem_addr(&s_tmem_base), 256);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem = s_tmem_base;
+
+  if (warp == 8) {
+    if (lane == 0) {
+      const long long krow = (long long)(unit * c.Hkv + g) * c.Tpad + key0;
+      mbar_expect_tx(bar(B_KFULL), 32768);
+      tma_load_2d(sK, &maps.k128, 0, (int)krow, bar(B_KFULL));
+      tma_load_2d(sK + 16384, &maps.k128, 64, (int)krow, bar(B_KFULL));
+      bool ok = true;
+      int it = 0;
+      for (int blk = blk0; ok && blk < nblocks; ++blk, ++it) {
+        const int st = it & 1;
+        if (it >= 2) ok = mbar_wait(bar(B_QEMPTY + st), ((it >> 1) - 1) & 1, abortp);
+        if (!ok) break;
+        mbar_expect_tx(bar(B_QFULL + st), 32768);
+        tma_load_3d(sQ + st * 32768, &maps.q, 0, g * G, l * a.n + blk * TPB, bar(B_QFULL + st));
+        tma_load_3d(sQ + st * 32768 + 16384, &maps.q, 64, g * G, l * a.n + blk * TPB, bar(B_QFULL + st));
+      }
+      for (int back = 1; back <= 2 && back <= it; ++back) {  // no copy may be in flight at exit
+        const int ii = it - back;
+        if (!mbar_wait(bar(B_QEMPTY + (ii & 1)), (ii >> 1) & 1, abortp)) break;
+      }
+    }
+  } else if (warp == 9) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(128, 128, false);
+      bool ok = mbar_wait(bar(B_KFULL), 0, abortp);
+      int it = 0;
+      for (int blk = blk0; ok && blk < nblocks; ++blk, ++it) {
+        const int st = it & 1;
+        ok = mbar_wait(bar(B_QFULL + st), (it >> 1) & 1, abortp);
+        if (!ok) break;
+        if (it >= 2) ok = mbar_wait(bar(B_SEMPTY + st), ((it >> 1) - 1) & 1, abortp);
+        if (!ok) break;
+        fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t half = ks >> 2, kin = (ks & 3) * 32;
+          const uint64_t ad = make_desc(sK + half * 16384 + kin, 16, 1024);
+          const uint64_t bd = make_desc(sQ + st * 32768 + half * 16384 + kin, 16, 1024);
+          mma_ss(tmem + st * 128, ad, bd, idesc, ks > 0);
+        }
+        mma_commit(bar(B_SFULL + st));
+        mma_commit(bar(B_QEMPTY + st));
+      }
+    }
+  } else {
+    // epilogue: thread = key (TMEM lane), columns [64*chalf, +64) of every block
+    const int chalf = warp >> 2;
+    const int krel = (warp & 3) * 32 + lane;  // key inside the tile
+    const int key = key0 + krel;              // absolute key token
+    const bool key_ok = key < key_end && key >= c.Ls;
+    const int jrel = key - a.t0;              // call-relative (cur tiles only)
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const float c2 = c.scale * kLog2eM;
+    const float2* rq = c.rowq + (size_t)layer * c.chunk * c.Hq + g * G;
+    int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
+    const int roff = a.t0 - a.reg_start;      // region index = call-relative token + roff
+    // row statistics (-m, 2^20/l) of a block's 128 rows, staged in shared memory one block ahead
+    auto load_stats = [&](int blk) -> float2 {
+      const int tk = blk * TPB + tid / G;
+      return (tid < 128 && tk < a.n) ? __ldg(rq + (size_t)tk * c.Hq + tid % G) : make_float2(-INFINITY, 0.f);
+    };
+    if (tid < 128 && blk0 < nblocks) s_stats[0][tid] = load_stats(blk0);
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    long long total = 0;
+    bool ok = true;
+    int it = 0;
+    for (int blk = blk0; blk < nblocks; ++blk, ++it) {
+      const int st = it & 1;
+      const bool more = blk + 1 < nblocks;
+      float2 nxt = make_float2(-INFINITY, 0.f);
+      if (more) nxt = load_stats(blk + 1);
+      // after an expired wait every thread keeps walking the loop (without computing) so that the named barrier
+      // below is still reached by all 256 epilogue threads
+      ok = ok && mbar_wait(bar(B_SFULL + st), (it >> 1) & 1, abortp);
+      if (!ok) {
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        continue;
+      }
+      fence_after_sync();
+      uint32_t v[2][32];
+      tmem_ld32(tmem + lane_base + st * 128 + chalf * 64, v[0]);
+      tmem_ld32(tmem + lane_base + st * 128 + chalf * 64 + 32, v[1]);
+      tmem_ld_wait();
+      const int tokb = blk * TPB;                              // first token of the block (call-relative)
+      const bool diag = is_cur && tokb < (key0 - a.t0) + 128;  // some token of the block precedes some key
+      const float2* ss = &s_stats[st][chalf * 64];
+      int bsum = 0;
+#pragma unroll
+      for (int ch = 0; ch < 2; ++ch) {
+        int aq[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float2 sq = ss[ch * 32 + e];
+          // round to nearest even by adding 1.5 * 2^23: the integer sits in the mantissa
+          const float x = ex2m(fmaf(__uint_as_float(v[ch][e]), c2, sq.x)) * sq.y + 12582912.f;
+          aq[e] = __float_as_int(x) - 0x4B400000;
+        }
+        if (diag) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (tokb + (chalf * 64 + ch * 32 + e) / G < jrel) aq[e] = 0;
+        }
+        if (is_cur) {
+          // head sum per token (Eq. 4) -> region map; causality already zeroed the invalid entries
+#pragma unroll
+          for (int t = 0; t < 32 / G; ++t) {
+            int sv = 0;
+#pragma unroll
+            for (int hh = 0; hh < G; ++hh) sv += aq[t * G + hh];
+            bsum += sv;
+            const int tk = tokb + (chalf * 64 + ch * 32) / G + t;
+            if (key_ok && sv != 0 && tk < a.n) atomicAdd(&Mq[(size_t)(tk + roff) * c.chunk + (jrel + roff)], sv);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) bsum += aq[e];
+        }
+      }
+      total += bsum;
+      if (tid < 128 && more) s_stats[st ^ 1][tid] = nxt;
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_SEMPTY + st));
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+    }
+    if (ok && key_ok && total != 0)
+      atomicAdd((unsigned long long*)&c.votes[unit * c.Tpad + key], (unsigned long long)total);
+  }
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  if (warp == 8) tmem_dealloc(tmem, 256);
+  if (tid == 0 && s_abort) set_status(c, -6, 5000 + (int)blockIdx.x);
+}
+
+typedef CUresult (*EncodeFnM)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+template <int G>
+static cudaError_t launch_map_tc_g(const DevCtx& c, const PrefillArgs& a, const void* kv_maps, cudaStream_t s) {
+  static EncodeFnM enc = nullptr;
+  if (!enc) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return cudaErrorNotSupported;
+    enc = reinterpret_cast<EncodeFnM>(p);
+  }
+  MapMaps maps;
+  memcpy(&maps.k128, static_cast<const CUtensorMap*>(kv_maps) + 4, sizeof(CUtensorMap));  // the 128-row box
+  cuuint64_t dims[3] = {128, (cuuint64_t)c.Hq, (cuuint64_t)a.layer_count * a.n};
+  cuuint64_t strides[2] = {256, (cuuint64_t)c.Hq * 256};
+  cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(128 / G)};
+  cuuint32_t es[3] = {1, 1, 1};
+  if (enc(&maps.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(a.q), dims, strides, box, es,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  // the region map is accumulated with integer reductions: clear it first
+  cudaError_t e = cudaMemsetAsync(c.Mq + (size_t)a.layer_begin * c.chunk * c.chunk, 0,
+                                  (size_t)a.layer_count * c.chunk * c.chunk * sizeof(int), s);
+  if (e != cudaSuccess) return e;
+  const int nloc = (a.loc_begin >= c.Ls) ? (a.t0 - a.loc_begin + 127) / 128 : 0;
+  const int ncur = (a.n + 127) / 128;
+  const int smem = 32768 + 65536 + 1024;
+  cudaFuncSetAttribute(k_map_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  k_map_tc<G><<<dim3(nloc + ncur, c.Hkv, a.layer_count), kMapThreads, smem, s>>>(c, a, nloc, maps);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_map_pass_tc(const DevCtx& c, const PrefillArgs& a, const void* kv_maps, cudaStream_t s) {
+  switch (c.G) {
+    case 1: return launch_map_tc_g<1>(c, a, kv_maps, s);
+    case 2: return launch_map_tc_g<2>(c, a, kv_maps, s);
+    case 4: return launch_map_tc_g<4>(c, a, kv_maps, s);
+    case 8: return launch_map_tc_g<8>(c, a, kv_maps, s);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace ltri

@@ -1,6 +1,7 @@
 // C ABI of the ltri library: host-side stream state, arena layout and the launch sequences of a prefill call
 // and a decode step.  Everything that computes runs in the kernels; this file only orders them.
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <deque>
@@ -99,6 +100,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.best = cv.take<long long>((size_t)d.NL * 2 * d.chunk);
   d.thetaq = cv.take<long long>(d.NL);
   d.rowstat = cv.take<float2>((size_t)d.NL * d.chunk * d.Hq);
+  d.rowq = cv.take<float2>((size_t)d.NL * d.chunk * d.Hq);
   d.Oacc = cv.take<float>((size_t)d.NL * d.chunk * d.Hq * kD);
   d.u = cv.take<float>((size_t)d.NL * d.Hkv * d.Jmax * kD);
   d.Jcnt = cv.take<int>(d.NL);
@@ -142,10 +144,14 @@ int cuda_fail(ltri_ctx* ctx, cudaError_t e) {
   ctx->last_cuda = (int)e;
   return LTRI_ECUDA;
 }
-#define LTRI_CUDA(ctx, expr)                   \
-  do {                                         \
-    cudaError_t e__ = (expr);                  \
-    if (e__ != cudaSuccess) return cuda_fail(ctx, e__); \
+#define LTRI_CUDA(ctx, expr)                                                         \
+  do {                                                                               \
+    cudaError_t e__ = (expr);                                                        \
+    if (e__ != cudaSuccess) {                                                        \
+      if (std::getenv("LTRI_DEBUG"))                                                 \
+        fprintf(stderr, "ltri: %s failed at line %d: %s\n", #expr, __LINE__, cudaGetErrorString(e__)); \
+      return cuda_fail(ctx, e__);                                                    \
+    }                                                                                \
   } while (0)
 
 bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
@@ -326,7 +332,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   }
   {
     Scope sc(ctx, st, LTRI_K_MAP, (a.t0 - a.loc_begin > 0 && a.loc_begin >= d.Ls) ? 2 : 1);
-    LTRI_CUDA(ctx, launch_map_pass(d, a, st));
+    LTRI_CUDA(ctx, ctx->use_tc ? launch_map_pass_tc(d, a, ctx->kv_maps, st) : launch_map_pass(d, a, st));
   }
   if (m > 0) {
     Scope sc(ctx, st, LTRI_K_SEGMENT, 4);
