@@ -98,6 +98,8 @@ cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_
                            int theta_mode, float theta, long long theta_q_abs, int max_spans, int n, int t0,
                            const __nv_bfloat16* q, cudaStream_t s);
 cudaError_t launch_score_prefill(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s);
+// tensor-core version of launch_score_prefill (split-bf16 representatives)
+cudaError_t launch_score_prefill_mma(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s);
 cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
                                 const __nv_bfloat16* q, int span_bound, cudaStream_t s);

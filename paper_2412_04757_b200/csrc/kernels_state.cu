@@ -138,60 +138,112 @@ cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_co
 
 // ------------------------------------------------------------------------------------------
 // a3 segmenter, step 1: exact rank selection of theta (quantile mode) over the causal entries of Mq.
-// 4-pass MSB radix select on sign-flipped 32-bit keys; one CTA per layer.
+// A sparse map is mostly zeros, so zeros (and negatives, which only hand-built maps can contain) are counted first;
+// only when the rank falls among the positive entries does an MSB radix select run over them, 8 bits per pass from
+// the highest set bit of the maximum, with one private histogram per warp.  One CTA per layer.
 __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin, int m, long long rank) {
   const int layer = layer_begin + blockIdx.x;
   const int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
-  __shared__ unsigned hist[256];
-  __shared__ unsigned s_prefix;
+  __shared__ unsigned hist[32][256];
+  __shared__ unsigned tot[256];
+  __shared__ unsigned s_red[32][3];
+  __shared__ unsigned s_prefix, s_maxkey;
   __shared__ long long s_rank;
-  if (threadIdx.x == 0) {
-    s_prefix = 0;
-    s_rank = rank;
+  __shared__ int s_cls;  // 0: answer is 0, 1: among positives, -1: among negatives
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // class counts and maxima
+  unsigned nneg = 0, nzero = 0, maxpos = 0, maxneg = 0;
+  for (int i = warp; i < m; i += 32)
+    for (int j = lane; j <= i; j += 32) {
+      const int v = Mq[(size_t)i * c.chunk + j];
+      if (v > 0)
+        maxpos = max(maxpos, (unsigned)v);
+      else if (v == 0)
+        ++nzero;
+      else {
+        ++nneg;
+        maxneg = max(maxneg, (unsigned)v ^ 0x80000000u);
+      }
+    }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    nneg += __shfl_xor_sync(0xffffffffu, nneg, o);
+    nzero += __shfl_xor_sync(0xffffffffu, nzero, o);
+    maxpos = max(maxpos, __shfl_xor_sync(0xffffffffu, maxpos, o));
+    maxneg = max(maxneg, __shfl_xor_sync(0xffffffffu, maxneg, o));
   }
-  const int total = m * m;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+  if (lane == 0) {
+    s_red[warp][0] = nneg;
+    s_red[warp][1] = nzero;
+    s_red[warp][2] = maxpos;
+    tot[warp] = maxneg;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    long long cn = 0, cz = 0;
+    unsigned mp = 0, mn = 0;
+    for (int w = 0; w < 32; ++w) {
+      cn += s_red[w][0];
+      cz += s_red[w][1];
+      mp = max(mp, s_red[w][2]);
+      mn = max(mn, tot[w]);
+    }
+    if (rank < cn) {
+      s_cls = -1;
+      s_rank = rank;
+      s_maxkey = mn;
+    } else if (rank < cn + cz) {
+      s_cls = 0;
+    } else {
+      s_cls = 1;
+      s_rank = rank - cn - cz;
+      s_maxkey = mp;
+    }
+    s_prefix = 0;
+  }
+  __syncthreads();
+  const int cls = s_cls;
+  if (cls == 0) {
+    if (threadIdx.x == 0) c.thetaq[layer] = 0;
+    return;
+  }
+  int hi = 32 - __clz(s_maxkey | 1u);  // bits [0,hi) can be set
+  while (hi > 0) {
+    const int lo = max(0, hi - 8);
+    const unsigned dmask = (1u << (hi - lo)) - 1u;
+    for (int t = threadIdx.x; t < 32 * 256; t += blockDim.x) (&hist[0][0])[t] = 0;
     __syncthreads();
     const unsigned prefix = s_prefix;
-    const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-    for (int base = 0; base < total; base += blockDim.x) {
-      const int idx = base + threadIdx.x;
-      bool valid = false;
-      unsigned bin = 0;
-      if (idx < total) {
-        const int i = idx / m, j = idx - i * m;
-        if (j <= i) {
-          const unsigned key = (unsigned)Mq[(size_t)i * c.chunk + j] ^ 0x80000000u;
-          if ((key & himask) == prefix) {
-            valid = true;
-            bin = (key >> shift) & 255u;
-          }
-        }
+    for (int i = warp; i < m; i += 32)
+      for (int j = lane; j <= i; j += 32) {
+        const int v = Mq[(size_t)i * c.chunk + j];
+        const bool in_cls = cls > 0 ? v > 0 : v < 0;
+        const unsigned key = cls > 0 ? (unsigned)v : ((unsigned)v ^ 0x80000000u);
+        if (in_cls && (hi >= 32 || (key >> hi) == (prefix >> hi))) atomicAdd(&hist[warp][(key >> lo) & dmask], 1u);
       }
-      // warp-aggregated histogram update (most entries of a sparse map share one bin)
-      const unsigned act = __ballot_sync(0xffffffffu, valid);
-      if (valid) {
-        const unsigned peers = __match_any_sync(act, bin);
-        if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
-      }
+    __syncthreads();
+    if (threadIdx.x < 256) {
+      unsigned sum = 0;
+      for (int w = 0; w < 32; ++w) sum += hist[w][threadIdx.x];
+      tot[threadIdx.x] = sum;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
       long long r = s_rank;
       unsigned b = 0;
-      for (; b < 256; ++b) {
-        if (r < (long long)hist[b]) break;
-        r -= hist[b];
+      for (; b <= dmask; ++b) {
+        if (r < (long long)tot[b]) break;
+        r -= tot[b];
       }
-      if (b > 255) b = 255;
+      if (b > dmask) b = dmask;
       s_rank = r;
-      s_prefix = prefix | (b << shift);
+      s_prefix = prefix | (b << lo);
     }
     __syncthreads();
+    hi = lo;
   }
-  if (threadIdx.x == 0) c.thetaq[layer] = (long long)(int)(s_prefix ^ 0x80000000u);
+  if (threadIdx.x == 0)
+    c.thetaq[layer] = cls > 0 ? (long long)s_prefix : (long long)(int)(s_prefix ^ 0x80000000u);
 }
 
 __global__ void k_theta_set(DevCtx c, int layer_begin, long long thq) { c.thetaq[layer_begin + blockIdx.x] = thq; }
