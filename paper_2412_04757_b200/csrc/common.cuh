@@ -103,6 +103,10 @@ cudaError_t launch_score_prefill_mma(const DevCtx& c, const PrefillArgs& a, int 
 cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
                                 const __nv_bfloat16* q, int span_bound, cudaStream_t s);
+// decode scores + top-k + range list in one launch (span_bound <= dec_retrieve_fused_max_spans())
+cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count,
+                                      const __nv_bfloat16* q, int span_bound, cudaStream_t s);
+int dec_retrieve_fused_max_spans();
 cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s);
 
 // prefill attention.  phase 0: local part over sink|local|cur, stores state (+ final output if `final`);

@@ -2,6 +2,7 @@
 // token ranges [sink | selected spans | tokens since the last eviction].  Every K/V row is read once with 16-byte
 // loads and shared by the G query heads of its KV group; softmax reductions use warp shuffles.
 #include "common.cuh"
+#include "mma_util.cuh"
 
 namespace ltri {
 
@@ -18,15 +19,24 @@ __device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
   }
 }
 
-// grid (nsplit, Hkv, b.n*layer_count).  Partial results (m, l, O[128]) per (unit, head, split) go to dec_part.
+// grid (nsplit, Hkv, b.n*layer_count), 4 warps.  Each warp walks 16-token tiles of the CTA's slice of the virtual
+// token list (sink | selected spans | recent tokens): the tile's K and V rows (two contiguous 256-byte rows per
+// cp.async instruction, 16 bytes per lane) land in a warp-private, XOR-swizzled 3-stage ring; QK^T and PV run as
+// m16n8k16 tensor-core MMAs with the G query heads of the group in the first rows of the 16-row operand, so the
+// per-token ALU cost is a handful of instructions and the kernel stays bound by the K/V stream.
+// Partial results (m, l, O[128]) per (unit, head, split) go to dec_part.
+constexpr int kDTile = 16;
+constexpr int kDStages = 3;
+constexpr int kDWarpBytes = kDStages * 2 * kDTile * 256;  // K and V rows of every stage
+
 template <int G>
-__global__ void __launch_bounds__(kDecThreads) k_decode_attn(DevCtx c, DecBatch b, int layer_begin, int layer_count,
-                                                             const __nv_bfloat16* __restrict__ q, int nsplit) {
-  __shared__ int rs[kMaxTopK + 2], rl[kMaxTopK + 2], rp[kMaxTopK + 3];
-  __shared__ float sm_m[8][G], sm_l[8][G];
-  __shared__ float sm_o[8][G][kD];
-  const int tid = threadIdx.x;
-  const int hw = tid >> 4, hl = tid & 15;  // half-warp id (0..7), lane in half-warp
+__global__ void __launch_bounds__(kDecThreads, 2) k_decode_attn(DevCtx c, DecBatch b, int layer_begin, int layer_count,
+                                                                const __nv_bfloat16* __restrict__ q, int nsplit) {
+  extern __shared__ __align__(1024) unsigned char dsm[];
+  __shared__ int rs[kMaxTopK + 2], rp[kMaxTopK + 3];
+  __shared__ float sm_m[4][G], sm_l[4][G];
+  __shared__ float sm_o[4][G][kD];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int split = blockIdx.x, g = blockIdx.y;
   const int bi = blockIdx.z / layer_count, l = blockIdx.z % layer_count, layer = layer_begin + l;
   const size_t unit = unit_of(c, b.seq[bi], layer);
@@ -36,9 +46,8 @@ __global__ void __launch_bounds__(kDecThreads) k_decode_attn(DevCtx c, DecBatch 
     int run = 0;
     for (int i = 0; i < nr; ++i) {
       rs[i] = c.rng_start[rb + i];
-      rl[i] = c.rng_len[rb + i];
       rp[i] = run;
-      run += rl[i];
+      run += c.rng_len[rb + i];
     }
     rp[nr] = run;
   }
@@ -46,118 +55,135 @@ __global__ void __launch_bounds__(kDecThreads) k_decode_attn(DevCtx c, DecBatch 
   const int total = rp[nr];
   const int per = (total + nsplit - 1) / nsplit;
   const int v0 = split * per, v1 = min(total, v0 + per);
+  const int ntiles = v1 > v0 ? (v1 - v0 + kDTile - 1) / kDTile : 0;
 
-  // this lane's 8 dims of the G query heads, pre-scaled
-  float qf[G][8];
+  // query fragments: rows 0..G-1 of the 16-row A operand are the heads of the group, the rest are zero
+  const int r = lane >> 2, qd = lane & 3;
+  uint32_t qa[8][2];
+  {
+    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + (size_t)g * G + (r < G ? r : 0)) * kD;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][0] = r < G ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 2 * qd) : 0u;
+      qa[ks][1] = r < G ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + 2 * qd) : 0u;
+    }
+  }
+  const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD;
+  const __nv_bfloat16* Vslab = c.Vc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD;
+  const uint32_t wbase = smem_u32(dsm) + warp * kDWarpBytes;
   const float c2 = c.scale * kLog2eD;
-  const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + (size_t)g * G) * kD + hl * 8;
-#pragma unroll
-  for (int hh = 0; hh < G; ++hh) {
-    const uint4 raw = *reinterpret_cast<const uint4*>(qp + (size_t)hh * kD);
-    unpack8(raw, qf[hh]);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) qf[hh][e] *= c2;
-  }
-  const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD + hl * 8;
-  const __nv_bfloat16* Vslab = c.Vc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD + hl * 8;
 
-  float m[G], lsum[G], O[G][8];
-#pragma unroll
-  for (int hh = 0; hh < G; ++hh) {
-    m[hh] = -INFINITY;
-    lsum[hh] = 0.f;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) O[hh][e] = 0.f;
-  }
-  // range cursor of this half-warp
+  // this lane copies rows (lane>>4) + 2i of every tile, 16 bytes at chunk (lane&15)
   int ri = 0;
-  constexpr int U = 4;  // tokens in flight per half-warp
-  for (int base = v0; base < v1; base += 8 * U) {  // trip count is uniform over the CTA (shuffles inside)
-    const int vb = base + hw * U;
-    uint4 kraw[U], vraw[U];
-    bool ok[U];
+  const int ch = lane & 15;
+  auto issue = [&](int t, int stage) {
+    const uint32_t sk = wbase + stage * (2 * kDTile * 256), sv = sk + kDTile * 256;
+    const int vb = v0 + t * kDTile;
 #pragma unroll
-    for (int t = 0; t < U; ++t) {
-      const int v = vb + t;
-      ok[t] = v < v1;
-      int tok = 0;
-      if (ok[t]) {
+    for (int i = 0; i < kDTile / 2; ++i) {
+      const int row = 2 * i + (lane >> 4);
+      const int v = vb + row;
+      const bool okr = v < v1;
+      size_t tok = 0;
+      if (okr) {
         while (v >= rp[ri + 1]) ++ri;
-        tok = rs[ri] + (v - rp[ri]);
+        tok = (size_t)(rs[ri] + (v - rp[ri]));
       }
-      kraw[t] = ok[t] ? __ldg(reinterpret_cast<const uint4*>(Kslab + (size_t)tok * kD)) : make_uint4(0, 0, 0, 0);
-      vraw[t] = ok[t] ? __ldg(reinterpret_cast<const uint4*>(Vslab + (size_t)tok * kD)) : make_uint4(0, 0, 0, 0);
+      cp_async16(sk + tile_off(row, ch), Kslab + tok * kD + ch * 8, okr ? 16 : 0);
+      cp_async16(sv + tile_off(row, ch), Vslab + tok * kD + ch * 8, okr ? 16 : 0);
     }
-    float s[U][G];
+  };
+
+  float O[16][4];
 #pragma unroll
-    for (int t = 0; t < U; ++t) {
-      float kf[8];
-      unpack8(kraw[t], kf);
+  for (int i = 0; i < 16; ++i) O[i][0] = O[i][1] = O[i][2] = O[i][3] = 0.f;
+  float m = -INFINITY, lsum = 0.f;
+
+  // tiles of this warp: warp, warp + 4, ...
+  const int my_tiles = ntiles > warp ? (ntiles - warp + 3) / 4 : 0;
 #pragma unroll
-      for (int hh = 0; hh < G; ++hh) {
-        float d = 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) d = fmaf(qf[hh][e], kf[e], d);
-        s[t][hh] = d;
-      }
-    }
-#pragma unroll
-    for (int t = 0; t < U; ++t)
-#pragma unroll
-      for (int hh = 0; hh < G; ++hh) {
-        float d = s[t][hh];
-        d += __shfl_xor_sync(0xffffffffu, d, 1);
-        d += __shfl_xor_sync(0xffffffffu, d, 2);
-        d += __shfl_xor_sync(0xffffffffu, d, 4);
-        d += __shfl_xor_sync(0xffffffffu, d, 8);
-        s[t][hh] = ok[t] ? d : -INFINITY;
-      }
-#pragma unroll
-    for (int hh = 0; hh < G; ++hh) {
-      float mx = m[hh];
-#pragma unroll
-      for (int t = 0; t < U; ++t) mx = fmaxf(mx, s[t][hh]);
-      const float mu = mx == -INFINITY ? 0.f : mx;  // a half-warp may have seen no token yet
-      const float alpha = exp2f(m[hh] - mu);
-      m[hh] = mx;
-      lsum[hh] *= alpha;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) O[hh][e] *= alpha;
-#pragma unroll
-      for (int t = 0; t < U; ++t) s[t][hh] = exp2f(s[t][hh] - mu);
-    }
-#pragma unroll
-    for (int t = 0; t < U; ++t) {
-      float vf[8];
-      unpack8(vraw[t], vf);
-#pragma unroll
-      for (int hh = 0; hh < G; ++hh) {
-        const float p = s[t][hh];
-        lsum[hh] += p;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) O[hh][e] = fmaf(p, vf[e], O[hh][e]);
-      }
-    }
+  for (int s = 0; s < kDStages - 1; ++s) {
+    if (s < my_tiles) issue(warp + 4 * s, s);
+    cp_async_commit();
   }
-  // merge the 8 half-warps through shared memory
+  for (int it = 0; it < my_tiles; ++it) {
+    const int stage = it % kDStages;
+    if (it + kDStages - 1 < my_tiles) issue(warp + 4 * (it + kDStages - 1), (it + kDStages - 1) % kDStages);
+    cp_async_commit();
+    cp_async_wait<kDStages - 1>();
+    __syncwarp();
+    const uint32_t sk = wbase + stage * (2 * kDTile * 256), sv = sk + kDTile * 256;
+    const int vb = v0 + (warp + 4 * it) * kDTile;
+    float S[2][4];
 #pragma unroll
-  for (int hh = 0; hh < G; ++hh) {
-    if (hl == 0) {
-      sm_m[hw][hh] = m[hh];
-      sm_l[hw][hh] = lsum[hh];
+    for (int i = 0; i < 2; ++i) S[i][0] = S[i][1] = S[i][2] = S[i][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      uint32_t bf[4];
+      ldsm_x4(bf, sk + tile_off((lane & 7) + ((lane >> 4) << 3), ks * 2 + ((lane >> 3) & 1)));
+      const uint32_t a[4] = {qa[ks][0], 0u, qa[ks][1], 0u};
+      mma_bf16(S[0], a, bf[0], bf[1]);
+      mma_bf16(S[1], a, bf[2], bf[3]);
+    }
+    // row r of this lane: tokens nt*8 + 2*qd + e
+    float tmax = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        if (vb + nt * 8 + 2 * qd + e >= v1) S[nt][e] = -INFINITY;
+        tmax = fmaxf(tmax, S[nt][e]);
+      }
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+    const float mnew = fmaxf(m, tmax * c2);
+    const float mu = mnew == -INFINITY ? 0.f : mnew;
+    const float alpha = exp2f(m - mu);
+    m = mnew;
+    float p[2][2];
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) p[nt][e] = exp2f(fmaf(S[nt][e], c2, -mu));
+    lsum = lsum * alpha + (p[0][0] + p[0][1] + p[1][0] + p[1][1]);
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) {
+      O[nt][0] *= alpha;
+      O[nt][1] *= alpha;
+    }
+    const uint32_t pa[4] = {pack_bf16(p[0][0], p[0][1]), 0u, pack_bf16(p[1][0], p[1][1]), 0u};
+#pragma unroll
+    for (int dp = 0; dp < 8; ++dp) {
+      uint32_t bf[4];
+      ldsm_x4_t(bf, sv + tile_off((lane & 7) + (((lane >> 3) & 1) << 3), dp * 2 + (lane >> 4)));
+      mma_bf16(O[2 * dp], pa, bf[0], bf[1]);
+      mma_bf16(O[2 * dp + 1], pa, bf[2], bf[3]);
+    }
+    __syncwarp();
+  }
+  cp_async_wait<0>();
+  lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+  lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+  if (r < G) {
+    if (qd == 0) {
+      sm_m[warp][r] = m;
+      sm_l[warp][r] = lsum;
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) sm_o[hw][hh][hl * 8 + e] = O[hh][e];
+    for (int nt = 0; nt < 16; ++nt) {
+      sm_o[warp][r][nt * 8 + 2 * qd] = O[nt][0];
+      sm_o[warp][r][nt * 8 + 2 * qd + 1] = O[nt][1];
+    }
   }
   __syncthreads();
   for (int idx = tid; idx < G * kD; idx += kDecThreads) {
     const int hh = idx / kD, e = idx % kD;
     float mx = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) mx = fmaxf(mx, sm_m[w][hh]);
+    for (int w = 0; w < 4; ++w) mx = fmaxf(mx, sm_m[w][hh]);
     float lt = 0.f, ot = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) {
+    for (int w = 0; w < 4; ++w) {
       const float sc = sm_m[w][hh] == -INFINITY ? 0.f : exp2f(sm_m[w][hh] - mx);
       lt += sm_l[w][hh] * sc;
       ot += sm_o[w][hh][e] * sc;
@@ -193,8 +219,10 @@ __global__ void __launch_bounds__(kD) k_decode_merge(DevCtx c, DecBatch b, int l
 template <int G>
 static cudaError_t launch_dec_g(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count,
                                 const __nv_bfloat16* q, __nv_bfloat16* out, int nsplit, cudaStream_t s) {
-  k_decode_attn<G><<<dim3(nsplit, c.Hkv, b.n * layer_count), kDecThreads, 0, s>>>(c, b, layer_begin, layer_count, q,
-                                                                                 nsplit);
+  const int smem = 4 * kDWarpBytes;
+  cudaFuncSetAttribute(k_decode_attn<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  k_decode_attn<G><<<dim3(nsplit, c.Hkv, b.n * layer_count), kDecThreads, smem, s>>>(c, b, layer_begin, layer_count, q,
+                                                                                    nsplit);
   k_decode_merge<<<dim3(c.Hq, b.n * layer_count), kD, 0, s>>>(c, b, layer_begin, layer_count, out, nsplit);
   return cudaGetLastError();
 }

@@ -716,6 +716,191 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   }
 }
 
+// Decode retrieval in one launch: a CTA owns one (sequence, layer, KV head), streams that head's index once
+// (half-warp per 256-byte row, 16 bytes per lane, four rows in flight), keeps the scores in shared memory, selects the
+// top-k there (same radix select as k_topk) and writes the selection and the token ranges of the attention kernel.
+constexpr int kFusedMaxSpans = 12288;  // scores kept in shared memory (48 KB)
+
+__global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin, DecBatch b, int layer_count,
+                                                       const __nv_bfloat16* __restrict__ q) {
+  extern __shared__ float ssc[];  // [N]
+  __shared__ float su[kD];
+  __shared__ unsigned hist[256];
+  __shared__ unsigned s_prefix, s_need;
+  __shared__ int s_ids[kMaxTopK];
+  __shared__ int s_cnt;
+  __shared__ int s_scan[1024];
+  const int g = blockIdx.x;
+  const int bi = blockIdx.y / layer_count, l = blockIdx.y % layer_count, layer = layer_begin + l;
+  const int sq = b.seq[bi], pos = b.pos[bi], loc_begin = b.loc_begin[bi];
+  const size_t unit = unit_of(c, sq, layer);
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int N = min(c.n_spans[unit], kFusedMaxSpans);
+  if (tid < kD) {
+    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + g * c.G) * kD + tid;
+    float acc = 0.f;
+    for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
+    su[tid] = acc;
+  }
+  if (tid == 0) {
+    s_cnt = 0;
+    if (g == 0) c.sel_tokens[unit] = 0;
+  }
+  __syncthreads();
+  // ---- scores
+  {
+    const int hw = tid >> 4, hl = tid & 15;  // 64 half-warps
+    float uf[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
+    const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + g) * (size_t)c.cap * kD + hl * 8;
+    for (int base = 0; base < N; base += 64 * 4) {  // uniform trip count (shuffles inside)
+      uint4 raw[4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int s = base + t * 64 + hw;
+        raw[t] = s < N ? __ldg(reinterpret_cast<const uint4*>(KR + (size_t)s * kD)) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw[t]);
+        float d = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(p2[i]);
+          d = fmaf(uf[2 * i], f.x, d);
+          d = fmaf(uf[2 * i + 1], f.y, d);
+        }
+        d += __shfl_xor_sync(0xffffffffu, d, 1);
+        d += __shfl_xor_sync(0xffffffffu, d, 2);
+        d += __shfl_xor_sync(0xffffffffu, d, 4);
+        d += __shfl_xor_sync(0xffffffffu, d, 8);
+        const int s = base + t * 64 + hw;
+        if (hl == 0 && s < N) ssc[s] = d;
+      }
+    }
+  }
+  __syncthreads();
+  // ---- top-k over the shared-memory scores
+  const int K = min(c.topk, N);
+  if (K == N) {
+    for (int t = tid; t < K; t += nt) s_ids[t] = t;
+    if (tid == 0) s_cnt = K;
+  } else {
+    if (tid == 0) {
+      s_prefix = 0;
+      s_need = K;
+    }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      const unsigned prefix = s_prefix;
+      const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      for (int s = tid; s < N; s += nt) {
+        const unsigned key = order_key(ssc[s]);
+        if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        unsigned need = s_need;
+        int bin = 255;
+        for (; bin >= 0; --bin) {
+          if (need <= hist[bin]) break;
+          need -= hist[bin];
+        }
+        if (bin < 0) bin = 0;
+        s_need = need;
+        s_prefix = prefix | ((unsigned)bin << shift);
+      }
+      __syncthreads();
+    }
+    const unsigned T = s_prefix;
+    const unsigned need_eq = s_need;
+    const int per = (N + nt - 1) / nt;
+    const int lo = tid * per, hi = min(N, lo + per);
+    int eq = 0;
+    for (int s = lo; s < hi; ++s) eq += order_key(ssc[s]) == T;
+    s_scan[tid] = eq;
+    __syncthreads();
+    if (tid < 32) {  // exclusive scan of 1024 counts by one warp
+      int run = 0;
+      for (int blk = 0; blk < nt; blk += 32) {
+        const int v = s_scan[blk + tid];
+        int inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (tid >= o) inc += t;
+        }
+        s_scan[blk + tid] = run + inc - v;
+        run += __shfl_sync(0xffffffffu, inc, 31);
+      }
+    }
+    __syncthreads();
+    int eqrank = s_scan[tid];
+    for (int s = lo; s < hi; ++s) {
+      const unsigned key = order_key(ssc[s]);
+      bool take = key > T;
+      if (key == T) {
+        take = (unsigned)eqrank < need_eq;
+        ++eqrank;
+      }
+      if (take) {
+        const int slot = atomicAdd(&s_cnt, 1);
+        if (slot < kMaxTopK) s_ids[slot] = s;
+      }
+    }
+  }
+  __syncthreads();
+  const int cnt = min(s_cnt, K);
+  int myid = -1, rank = 0;
+  if (tid < cnt) {
+    myid = s_ids[tid];
+    for (int t = 0; t < cnt; ++t) rank += s_ids[t] < myid;
+  }
+  __syncthreads();
+  if (tid < cnt) s_ids[rank] = myid;
+  __syncthreads();
+  int* sel = c.sel + (unit * c.Hkv + g) * (size_t)c.topk;
+  for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
+  if (tid == 0) {
+    const size_t rbb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
+    int* rs = c.rng_start + rbb;
+    int* rl = c.rng_len + rbb;
+    int nr = 0;
+    long long tokens = 0;
+    auto push = [&](int st, int ln) {
+      if (ln <= 0) return;
+      if (nr > 0 && rs[nr - 1] + rl[nr - 1] == st)
+        rl[nr - 1] += ln;
+      else {
+        rs[nr] = st;
+        rl[nr] = ln;
+        ++nr;
+      }
+    };
+    push(0, min(c.Ls, pos + 1));
+    for (int t = 0; t < cnt; ++t) {
+      const int st = c.span_start[unit * c.cap + s_ids[t]], ln = c.span_len[unit * c.cap + s_ids[t]];
+      tokens += ln;
+      push(st, ln);
+    }
+    push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
+    c.rng_cnt[unit * c.Hkv + g] = nr;
+    atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+  }
+}
+
+cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count,
+                                      const __nv_bfloat16* q, int span_bound, cudaStream_t s) {
+  const int smem = (int)sizeof(float) * max(span_bound, 1);
+  if (smem > 48 * 1024) return cudaErrorInvalidValue;
+  k_dec_retrieve<<<dim3(c.Hkv, b.n * layer_count), 1024, smem, s>>>(c, layer_begin, b, layer_count, q);
+  return cudaGetLastError();
+}
+int dec_retrieve_fused_max_spans() { return kFusedMaxSpans; }
+
 cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
   DecBatch dummy;
   dummy.n = 0;

@@ -123,6 +123,7 @@ struct ltri_ctx {
   int last_cuda = 0;
   int sm_count = 148;
   bool use_tc = false;     // tcgen05/TMEM/TMA attention kernels (default when available)
+  int dec_fused = -1;      // decode retrieval in one launch: -1 auto, 0 never, 1 whenever the index fits
   alignas(64) unsigned char kv_maps[kTcMapBytes];  // TMA descriptors of the K/V cache
   long long launches = 0;  // kernels launched since creation
   // optional per-kernel-class timing with CUDA events on the launching stream
@@ -212,6 +213,7 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) ctx->sm_count = sms;
   }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (const char* f = std::getenv("LTRI_DEC_FUSED")) ctx->dec_fused = std::atoi(f) != 0 ? 1 : 0;  // testing aid
   const char* impl = std::getenv("LTRI_ATTN_IMPL");  // "mma" selects the warp-MMA kernels (debugging aid)
   ctx->use_tc = tc_attention_supported(ctx->d) && !(impl && std::strcmp(impl, "mma") == 0) &&
                 tc_encode_kv_maps(ctx->d, ctx->kv_maps);
@@ -407,7 +409,14 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
       Scope sc(ctx, st, LTRI_K_APPEND, 1);
       LTRI_CUDA(ctx, launch_append_decode(d, b, layer_begin, layer_count, n_seqs, kb, vb, st));
     }
-    {
+    // one CTA per (sequence, layer, KV head) keeps the scores in shared memory when the index is small enough and
+    // there are enough heads to fill the GPU; otherwise scores go through global memory in two launches
+    const bool fused = ub <= dec_retrieve_fused_max_spans() &&
+                       (ctx->dec_fused == 1 || (ctx->dec_fused < 0 && units >= ctx->sm_count));
+    if (fused) {
+      Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 1);
+      LTRI_CUDA(ctx, launch_dec_retrieve_fused(d, b, layer_begin, layer_count, qb, (int)ub, st));
+    } else {
       Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 2);
       LTRI_CUDA(ctx, launch_score_decode(d, b, layer_begin, layer_count, n_seqs, qb, (int)ub, st));
       LTRI_CUDA(ctx, launch_topk_decode(d, b, layer_begin, layer_count, st));

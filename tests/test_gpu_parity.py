@@ -111,6 +111,24 @@ def test_batched_decode_independent_sequences():
     print(sp.rep)
 
 
+@pytest.mark.parametrize("fused", ["0", "1"])
+def test_decode_retrieval_paths(fused, monkeypatch):
+    # decode retrieval has a one-launch path (scores in shared memory) and a two-launch path; check both
+    monkeypatch.setenv("LTRI_DEC_FUSED", fused)
+    cfg = small_cfg(n_layers=2, context=1280, decode_steps=5, top_k=6)
+    rep = ph.run_stream(cfg, layers=[0, 1], deep=False)
+    assert rep.sel_checks > 0
+    print(rep)
+
+
+def test_warp_mma_fallback_path(monkeypatch):
+    # the warp-MMA kernels remain selectable; they must match the oracle as well
+    monkeypatch.setenv("LTRI_ATTN_IMPL", "mma")
+    cfg = small_cfg(n_layers=1, context=768, decode_steps=2)
+    rep = ph.run_stream(cfg, layers=[0])
+    print(rep)
+
+
 def test_layer_ranges_are_independent_streams():
     cfg = small_cfg(n_layers=2, context=512, decode_steps=0)
     lt = binding.Ltri(ph.params_of(cfg))
