@@ -3,10 +3,10 @@
 // One CTA owns 256 query rows of one (layer, KV head): two 128-row tiles Q0/Q1, each row = (token, head of the
 // group), so one K/V tile serves the whole GQA group.  Keys arrive in 128-slot tiles assembled by TMA from pieces of
 // 8..128 rows, which lets a tile be packed from several short spans ("span-indirect" tiles): every range is padded
-// to a multiple of 8 rows only.  Roles (10 warps):
-//   warps 0-3 / 4-7 : softmax of S0 / S1, one thread per row (tcgen05.ld), P written back to TMEM as bf16
-//   warp 8          : TMA producer (Q once, K/V pieces through a 2-stage ring)
-//   warp 9          : MMA issuer: S = Q K^T (both operands in shared memory), O += P V (P from TMEM, V MN-major)
+// to a multiple of 8 rows only.  Roles (18 warps):
+//   warps 0-7 / 8-15 : softmax of S0 / S1, two threads per row (64 columns each), P written back to TMEM as bf16
+//   warp 16          : TMA producer (Q once, K/V pieces through a 2-stage ring)
+//   warp 17          : MMA issuer: S = Q K^T (both operands in shared memory), O += P V (P from TMEM, V MN-major)
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P aliases the first 64 columns of its S.
 // The issue order QK0, QK1, {PV0_j, QK0_j+1, PV1_j, QK1_j+1} keeps the tensor pipe busy with one tile's MMAs while
 // the other tile's softmax runs.  The running max is updated lazily (only when it grows by more than 2^8), in which
@@ -24,7 +24,7 @@ namespace ltri {
 using namespace tc;
 
 constexpr float kLog2eT = 1.4426950408889634f;
-constexpr int kTcThreads = 320;
+constexpr int kTcThreads = 576;  // 16 softmax warps + TMA producer + MMA issuer
 constexpr int kNumBoxes = 5;  // box heights 8,16,32,64,128
 constexpr float kRescaleThreshold = 8.0f;
 
@@ -106,6 +106,11 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -121,6 +126,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
   __shared__ RangeList rg;
+  __shared__ float s_max[2][2][128];  // per Q tile, per column half, per row: partial maxima / sums
   constexpr int TOKB = 256 / G;  // tokens per CTA
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
@@ -143,7 +149,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       mbar_init(bar(B_KEMPTY + s), 1);
       mbar_init(bar(B_VEMPTY + s), 1);
       mbar_init(bar(B_SREADY + s), 1);
-      mbar_init(bar(B_PREADY + s), 4);
+      mbar_init(bar(B_PREADY + s), 8);
     }
     mbar_init(bar(B_ODONE), 1);
     fence_mbar_init();
@@ -170,7 +176,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   for (uint32_t i = tid; i < 131072 / 16; i += kTcThreads)
     asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(sKV + i * 16), "r"(0) : "memory");
   fence_async_smem();
-  if (warp == 8) tmem_alloc(smem_addr(&s_tmem_base), 512);
+  if (warp == 16) tmem_alloc(smem_addr(&s_tmem_base), 512);
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
@@ -178,20 +184,24 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   const int causal_ri = phase == 0 ? 2 : -1;
   const size_t slab_row0 = (unit * c.Hkv + g) * (size_t)c.Tpad;
 
-  if (warp == 8) {
+  if (warp == 16) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      prefetch_tmap(&maps.q);
-      mbar_expect_tx(bar(B_QFULL), 65536);
-      tma_load_3d(sQ, &maps.q, 0, g * G, l * a.n + tok0, bar(B_QFULL));
-      tma_load_3d(sQ + 32768, &maps.q, 64, g * G, l * a.n + tok0, bar(B_QFULL));
+    // Every lane walks the tile list; lane 0 owns the barrier bookkeeping and lanes 0-3 issue the copies of
+    // (K low half, K high half, V low half, V high half) so that many small pieces do not serialise on one thread.
+    {
+      if (lane == 0) {
+        prefetch_tmap(&maps.q);
+        mbar_expect_tx(bar(B_QFULL), 65536);
+        tma_load_3d(sQ, &maps.q, 0, g * G, l * a.n + tok0, bar(B_QFULL));
+        tma_load_3d(sQ + 32768, &maps.q, 64, g * G, l * a.n + tok0, bar(B_QFULL));
+      }
       TileIter it;
       it.rg = &rg;
       it.causal_ri = causal_ri;
       int j = 0;
-      bool ok = true;
+      int ok = 1;
       int pslot[16], ptok[16], pbox[16];
-      while (ok) {
+      while (true) {
         int np = 0;
         if (!it.next<true>([&](int slot, int tok, int bi) {
               pslot[np] = slot;
@@ -201,39 +211,40 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             }))
           break;
         const int st = j & 1;
-        if (j >= 2) ok = mbar_wait(bar(B_KEMPTY + st), ((j >> 1) - 1) & 1, abortp);
-        if (!ok) break;
         uint32_t bytes = 0;
         for (int p = 0; p < np; ++p) bytes += (uint32_t)(8 << pbox[p]) * 256u;
-        mbar_expect_tx(bar(B_KFULL + st), bytes);
-        const uint32_t sK = sKV + st * 65536, sV = sK + 32768;
-        for (int p = 0; p < np; ++p) {
-          const CUtensorMap* m = &kvmaps[pbox[p]];
-          const long long row = (long long)slab_row0 + ptok[p];
-          const uint32_t so = (uint32_t)pslot[p] * 128u;
-          tma_load_2d(sK + so, m, 0, (int)row, bar(B_KFULL + st));
-          tma_load_2d(sK + 16384 + so, m, 64, (int)row, bar(B_KFULL + st));
+        if (lane == 0) {
+          if (j >= 2) ok = mbar_wait(bar(B_KEMPTY + st), ((j >> 1) - 1) & 1, abortp) ? 1 : 0;
+          if (ok) mbar_expect_tx(bar(B_KFULL + st), bytes);
         }
-        if (j >= 2) ok = mbar_wait(bar(B_VEMPTY + st), ((j >> 1) - 1) & 1, abortp);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
-        mbar_expect_tx(bar(B_VFULL + st), bytes);
-        for (int p = 0; p < np; ++p) {
-          const CUtensorMap* m = &kvmaps[pbox[p]];
-          const long long row = (long long)slab_row0 + ptok[p] + v_row_offset;
-          const uint32_t so = (uint32_t)pslot[p] * 128u;
-          tma_load_2d(sV + so, m, 0, (int)row, bar(B_VFULL + st));
-          tma_load_2d(sV + 16384 + so, m, 64, (int)row, bar(B_VFULL + st));
+        const uint32_t sK = sKV + st * 65536, sV = sK + 32768;
+        if (lane < 2)
+          for (int p = 0; p < np; ++p)
+            tma_load_2d(sK + lane * 16384 + (uint32_t)pslot[p] * 128u, &kvmaps[pbox[p]], lane * 64,
+                        (int)((long long)slab_row0 + ptok[p]), bar(B_KFULL + st));
+        if (lane == 0) {
+          if (j >= 2) ok = mbar_wait(bar(B_VEMPTY + st), ((j >> 1) - 1) & 1, abortp) ? 1 : 0;
+          if (ok) mbar_expect_tx(bar(B_VFULL + st), bytes);
         }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane == 2 || lane == 3)
+          for (int p = 0; p < np; ++p)
+            tma_load_2d(sV + (lane - 2) * 16384 + (uint32_t)pslot[p] * 128u, &kvmaps[pbox[p]], (lane - 2) * 64,
+                        (int)((long long)slab_row0 + ptok[p] + v_row_offset), bar(B_VFULL + st));
         ++j;
       }
-      // drain: every stage that was filled is released by the MMA warp; wait for the last ones so that no copy is
-      // in flight when the CTA exits
-      for (int back = 1; back <= 2 && back <= j; ++back) {
-        const int jj = j - back;
-        if (!mbar_wait(bar(B_VEMPTY + (jj & 1)), (jj >> 1) & 1, abortp)) break;
-      }
+      // drain: wait until the MMA warp has released the last stages so that no copy is in flight at exit
+      if (lane == 0)
+        for (int back = 1; back <= 2 && back <= j; ++back) {
+          const int jj = j - back;
+          if (!mbar_wait(bar(B_VEMPTY + (jj & 1)), (jj >> 1) & 1, abortp)) break;
+        }
+      __syncwarp();
     }
-  } else if (warp == 9) {
+  } else if (warp == 17) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       TileIter it;
@@ -244,25 +255,28 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       constexpr uint32_t idesc_qk = make_idesc(128, 128, false);
       constexpr uint32_t idesc_pv = make_idesc(128, 128, true);
       bool ok = mbar_wait(bar(B_QFULL), 0, abortp);
+      // descriptors differ only in their start-address field: build one per operand, then add constants
+      // (the address field holds bytes/16 and cannot carry out for any shared-memory offset)
+      const uint64_t dQ = make_desc(sQ, 16, 1024);
+      const uint64_t dK = make_desc(sKV, 16, 1024);
+      const uint64_t dV = make_desc(sKV + 32768, 16384, 1024);
       auto issue_qk = [&](int q, int st) {
-        const uint32_t sK = sKV + st * 65536;
+        const uint64_t da = dQ + (uint64_t)((q * 16384) >> 4);
+        const uint64_t db = dK + (uint64_t)((st * 65536) >> 4);
+        const uint32_t d = tmem + q * 128;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
           const uint32_t half = ks >> 2, kin = (ks & 3) * 32;
-          const uint64_t ad = make_desc(sQ + half * 32768 + q * 16384 + kin, 16, 1024);
-          const uint64_t bd = make_desc(sK + half * 16384 + kin, 16, 1024);
-          mma_ss(tmem + q * 128, ad, bd, idesc_qk, ks > 0);
+          mma_ss(d, da + ((half * 32768 + kin) >> 4), db + ((half * 16384 + kin) >> 4), idesc_qk, ks > 0);
         }
         mma_commit(bar(B_SREADY + q));
       };
       auto issue_pv = [&](int q, int st, bool acc) {
-        const uint32_t sV = sKV + st * 65536 + 32768;
+        // 16 keys per step: 2 KB down the V tile; N = 128 spans both 64-wide halves (LBO = 16 KB)
+        const uint64_t db = dV + (uint64_t)((st * 65536) >> 4);
+        const uint32_t d = tmem + 256 + q * 128, pa = tmem + q * 128;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          // 16 keys per step: 2 KB down the V tile; N = 128 spans both 64-wide halves (LBO = 16 KB)
-          const uint64_t bd = make_desc(sV + ks * 2048, 16384, 1024);
-          mma_ts(tmem + 256 + q * 128, tmem + q * 128 + ks * 8, bd, idesc_pv, acc || ks > 0);
-        }
+        for (int ks = 0; ks < 8; ++ks) mma_ts(d, pa + ks * 8, db + ((ks * 2048) >> 4), idesc_pv, acc || ks > 0);
       };
       if (ok && T > 0) {
         ok = mbar_wait(bar(B_KFULL + 0), 0, abortp);
@@ -301,28 +315,34 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       mma_commit(bar(B_ODONE));
     }
   } else {
-    // ------------------------------------------------------------------ softmax + epilogue, one thread per row
-    const int q = warp >> 2;
+    // ------------------------------------------------------------------ softmax + epilogue
+    // Two threads per row: warps 0-7 serve Q tile 0, warps 8-15 Q tile 1; inside a tile warps 0-3 take the columns
+    // [0,64) of S and O, warps 4-7 the columns [64,128).  The two halves of a row agree on the running maximum
+    // through shared memory and one named barrier per tile, after both have their S values in registers (so the
+    // P write-back, which aliases S, cannot clobber columns the other half still needs).
+    const int q = warp >> 3;
+    const int half = (warp >> 2) & 1;
     const int r = (warp & 3) * 32 + lane;        // row inside the 128-row tile = TMEM lane
     const int rr = q * 128 + r;                  // row inside the CTA
     const int tk = tok0 + rr / G;                // call-relative token
     const int h = g * G + rr % G;
     const bool row_ok = tk < a.n;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + lane_base + q * 128;
-    const uint32_t tO = tmem + lane_base + 256 + q * 128;
+    const uint32_t tS = tmem + lane_base + q * 128 + half * 64;   // this thread's 64 logits
+    const uint32_t tP = tmem + lane_base + q * 128 + half * 32;   // its 64 probabilities (bf16 pairs)
+    const uint32_t tO = tmem + lane_base + 256 + q * 128 + half * 64;
     const float c2 = c.scale * kLog2eT;
     float m_used = -INFINITY, lsum = 0.f;
     if (phase == 1) {
-      uint32_t v[32];
-      const float* op = c.Oacc + (((size_t)layer * c.chunk + (row_ok ? tk : 0)) * c.Hq + h) * kD;
+      const float* op = c.Oacc + (((size_t)layer * c.chunk + (row_ok ? tk : 0)) * c.Hq + h) * kD + half * 64;
       if (row_ok) {
         const float2 stt = c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h];
         m_used = stt.x;
-        lsum = stt.y;
+        lsum = half == 0 ? stt.y : 0.f;
       }
 #pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
+      for (int ch = 0; ch < 2; ++ch) {
+        uint32_t v[32];
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
           const float4 f = row_ok ? *reinterpret_cast<const float4*>(op + ch * 32 + e) : make_float4(0, 0, 0, 0);
@@ -342,33 +362,39 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     bool ok = true;
     const int row_abs = a.t0 + tk;
     while (it.next()) {
-      ok = mbar_wait(bar(B_SREADY + q), j & 1, abortp);
-      if (!ok) break;
+      // after an expired wait every thread keeps walking the loop (without computing) so that the named barrier
+      // is still reached by all 256 threads of the tile
+      ok = ok && mbar_wait(bar(B_SREADY + q), j & 1, abortp);
+      if (!ok) {
+        asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+        ++j;
+        continue;
+      }
       fence_after_sync();
-      // the whole S row in registers: four 32-column loads in flight, one wait
-      uint32_t v[4][32];
-#pragma unroll
-      for (int ch = 0; ch < 4; ++ch) tmem_ld32(tS + ch * 32, v[ch]);
+      uint32_t v[2][32];
+      tmem_ld32(tS, v[0]);
+      tmem_ld32(tS + 32, v[1]);
       tmem_ld_wait();
-      const bool masked = !it.full;
-      if (masked) {
+      if (!it.full) {
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          const unsigned mk = it.mask(ch);
+        for (int ch = 0; ch < 2; ++ch) {
+          const unsigned mk = it.mask(half * 2 + ch);
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
             bool okc = (mk >> e) & 1u;
-            if (it.causal_tok0 >= 0) okc = okc && (it.causal_tok0 + ch * 32 + e <= row_abs);
+            if (it.causal_tok0 >= 0) okc = okc && (it.causal_tok0 + half * 64 + ch * 32 + e <= row_abs);
             if (!okc) v[ch][e] = 0xff800000u;  // -inf
           }
         }
       }
       float mt = -INFINITY;
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch)
+      for (int ch = 0; ch < 2; ++ch)
 #pragma unroll
-        for (int e = 0; e < 32; ++e) mt = fmaxf(mt, __uint_as_float(v[ch][e]));
-      mt *= c2;
+        for (int e = 0; e < 32; e += 2) mt = max3(mt, __uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1]));
+      s_max[q][half][r] = mt;
+      asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+      mt = fmaxf(mt, s_max[q][half ^ 1][r]) * c2;
       // lazy running maximum: move it only when it grows by more than the threshold (or on first use)
       float alpha = 1.f;
       const bool grow = mt > m_used + kRescaleThreshold || (m_used == -INFINITY && mt > -INFINITY);
@@ -380,7 +406,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       const bool have_o = (j > 0) || (phase == 1);
       if (have_o && __any_sync(0xffffffffu, grow)) {
 #pragma unroll 1
-        for (int ch = 0; ch < 8; ++ch) {
+        for (int ch = 0; ch < 4; ++ch) {
           uint32_t w[16];
           tmem_ld16(tO + ch * 16, w);
           tmem_ld_wait();
@@ -390,41 +416,45 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         }
         tmem_st_wait();
       }
-      // probabilities, row sum, P (bf16) into the first 64 columns of S.  Masked entries are -inf -> exp2 gives 0.
+      // probabilities, row sum, P (bf16).  Masked entries are -inf -> exp2 gives 0.
       const float mneg = m_used == -INFINITY ? 0.f : -m_used;
-      float ls0 = 0.f, ls1 = 0.f;
+      const float2 c2v = make_float2(c2, c2), mnv = make_float2(mneg, mneg);
+      float2 ls = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
+      for (int ch = 0; ch < 2; ++ch) {
         uint32_t pk[16];
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
-          const float p0 = ex2(fmaf(__uint_as_float(v[ch][e]), c2, mneg));
-          const float p1 = ex2(fmaf(__uint_as_float(v[ch][e + 1]), c2, mneg));
-          ls0 += p0;
-          ls1 += p1;
-          pk[e >> 1] = pack2(p0, p1);
+          // packed fp32x2 arithmetic: one FFMA2 and one FADD2 per pair of logits
+          const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1])), c2v, mnv);
+          const float2 pp = make_float2(ex2(x.x), ex2(x.y));
+          ls = __fadd2_rn(ls, pp);
+          pk[e >> 1] = pack2(pp.x, pp.y);
         }
-        tmem_st16(tS + ch * 16, pk);
+        tmem_st16(tP + ch * 16, pk);
       }
-      lsum += ls0 + ls1;
+      lsum += ls.x + ls.y;
       tmem_st_wait();
       fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(B_PREADY + q));
       ++j;
     }
-    // epilogue
+    // epilogue: the two halves of a row exchange their partial sums, then each writes its 64 output columns
+    s_max[q][half][r] = lsum;
+    asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+    lsum += s_max[q][half ^ 1][r];
     if (ok) ok = mbar_wait(bar(B_ODONE), 0, abortp);
     if (ok) {
       fence_after_sync();
-      if (phase == 0 && row_ok) {
+      if (phase == 0 && row_ok && half == 0) {
         c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(m_used, lsum);
         c.rowq[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(-m_used, kQScale / lsum);
       }
       const float inv = 1.f / lsum;
       const bool have_o = (j > 0) || (phase == 1);
 #pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
+      for (int ch = 0; ch < 2; ++ch) {
         uint32_t v[32];
         if (have_o) {
           tmem_ld32(tO + ch * 32, v);
@@ -435,13 +465,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         }
         if (!row_ok) continue;
         if (phase == 0 && !final_out) {
-          float* op = c.Oacc + (((size_t)layer * c.chunk + tk) * c.Hq + h) * kD + ch * 32;
+          float* op = c.Oacc + (((size_t)layer * c.chunk + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
 #pragma unroll
           for (int e = 0; e < 32; e += 4)
             *reinterpret_cast<uint4*>(op + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
         }
         if (final_out) {
-          __nv_bfloat16* op = a.out + (((size_t)l * a.n + tk) * c.Hq + h) * kD + ch * 32;
+          __nv_bfloat16* op = a.out + (((size_t)l * a.n + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
             uint4 w;
@@ -459,7 +489,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
-  if (warp == 8) tmem_dealloc(tmem, 512);
+  if (warp == 16) tmem_dealloc(tmem, 512);
   if (tid == 0 && s_abort) set_status(c, -6, (int)(blockIdx.x + 1000 * blockIdx.y));
 }
 

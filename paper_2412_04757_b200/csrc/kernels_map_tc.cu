@@ -101,6 +101,7 @@ __global__ void __launch_bounds__(kMapThreads, 2)
   } else if (warp == 9) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(128, 128, false);
+      const uint64_t dK = make_desc(sK, 16, 1024), dQ = make_desc(sQ, 16, 1024);
       bool ok = mbar_wait(bar(B_KFULL), 0, abortp);
       int it = 0;
       for (int blk = blk0; ok && blk < nblocks; ++blk, ++it) {
@@ -110,12 +111,11 @@ __global__ void __launch_bounds__(kMapThreads, 2)
         if (it >= 2) ok = mbar_wait(bar(B_SEMPTY + st), ((it >> 1) - 1) & 1, abortp);
         if (!ok) break;
         fence_after_sync();
+        const uint64_t db = dQ + (uint64_t)((st * 32768) >> 4);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t half = ks >> 2, kin = (ks & 3) * 32;
-          const uint64_t ad = make_desc(sK + half * 16384 + kin, 16, 1024);
-          const uint64_t bd = make_desc(sQ + st * 32768 + half * 16384 + kin, 16, 1024);
-          mma_ss(tmem + st * 128, ad, bd, idesc, ks > 0);
+          const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
+          mma_ss(tmem + st * 128, dK + off, db + off, idesc, ks > 0);
         }
         mma_commit(bar(B_SFULL + st));
         mma_commit(bar(B_QEMPTY + st));

@@ -568,11 +568,64 @@ cudaError_t launch_score_prefill(const DevCtx& c, const PrefillArgs& a, int span
   return cudaGetLastError();
 }
 
+// decode scores, memory-bound index scan: one query representative per KV head (the summed query of the group).
+// Half-warp per 256-byte index row, 16 bytes per lane, four rows in flight; grid (span tiles of 256, Hkv, units).
+__global__ void __launch_bounds__(256) k_score_dec(DevCtx c, int layer_begin, DecBatch b, int layer_count,
+                                                   const __nv_bfloat16* __restrict__ q) {
+  __shared__ float su[kD];
+  const int g = blockIdx.y;
+  const int bi = blockIdx.z / layer_count, l = blockIdx.z % layer_count, layer = layer_begin + l;
+  const size_t unit = unit_of(c, b.seq[bi], layer);
+  const int tid = threadIdx.x;
+  const int N = c.n_spans[unit];
+  if (blockIdx.x == 0 && g == 0 && tid == 0) c.sel_tokens[unit] = 0;
+  const int s0 = blockIdx.x * 256;
+  if (s0 >= N) return;
+  if (tid < kD) {
+    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + g * c.G) * kD + tid;
+    float acc = 0.f;
+    for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
+    su[tid] = acc;
+  }
+  __syncthreads();
+  const int hw = tid >> 4, hl = tid & 15;  // 16 half-warps
+  float uf[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
+  const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + g) * (size_t)c.cap * kD + hl * 8;
+  float* sc = c.scores + (unit * c.Hkv + g) * (size_t)c.cap;
+#pragma unroll
+  for (int rep = 0; rep < 4; ++rep) {
+    uint4 raw[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const int s = s0 + rep * 64 + t * 16 + hw;
+      raw[t] = s < N ? __ldg(reinterpret_cast<const uint4*>(KR + (size_t)s * kD)) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw[t]);
+      float d = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(p2[i]);
+        d = fmaf(uf[2 * i], f.x, d);
+        d = fmaf(uf[2 * i + 1], f.y, d);
+      }
+      d += __shfl_xor_sync(0xffffffffu, d, 1);
+      d += __shfl_xor_sync(0xffffffffu, d, 2);
+      d += __shfl_xor_sync(0xffffffffu, d, 4);
+      d += __shfl_xor_sync(0xffffffffu, d, 8);
+      const int s = s0 + rep * 64 + t * 16 + hw;
+      if (hl == 0 && s < N) sc[s] = d;
+    }
+  }
+}
+
 cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int,
                                 const __nv_bfloat16* q, int span_bound, cudaStream_t s) {
   if (span_bound <= 0) span_bound = 1;
-  k_score<true><<<dim3((span_bound + 63) / 64, c.Hkv, b.n * layer_count), 256, kD * sizeof(float), s>>>(
-      c, 0, layer_begin, b, layer_count, q);
+  k_score_dec<<<dim3((span_bound + 255) / 256, c.Hkv, b.n * layer_count), 256, 0, s>>>(c, layer_begin, b, layer_count, q);
   return cudaGetLastError();
 }
 
