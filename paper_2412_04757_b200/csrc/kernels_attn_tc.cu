@@ -14,6 +14,7 @@
 // Every wait is bounded; on expiry the CTA sets LTRI_ETIMEOUT in the status word, drains and frees its TMEM.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -122,27 +123,37 @@ __global__ void __launch_bounds__(kTcThreads, 1)
               long long v_row_offset) {
   const CUtensorMap* kvmaps = maps.kv;
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[14];
+  // QFULL QFREE ODONE | KFULL[2] VFULL[2] KEMPTY[2] VEMPTY[2] | SREADY[2] PREADY[2] OFREE[2]
+  __shared__ __align__(8) unsigned long long bars[3 + 8 + 6];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ RangeList rg;
+  __shared__ RangeList rgs[3];        // key ranges of the work items in flight (roles may be up to two items apart)
+  __shared__ int s_quit[2];
+  __shared__ int s_items_ready;       // number of work items whose key ranges the producer has published
   __shared__ float s_max[2][2][128];  // per Q tile, per column half, per row: partial maxima / sums
-  constexpr int TOKB = 256 / G;  // tokens per CTA
+  constexpr int TOKB = 256 / G;  // tokens per work item
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
-  const size_t unit = unit_of(c, a.seq, layer);
-  const int tok0 = blockIdx.x * TOKB;
+  // persistent CTA: work items (token block, KV head, layer) are dealt round-robin
+  const int MB = (a.n + TOKB - 1) / TOKB;
+  const int nitems = MB * c.Hkv * a.layer_count;
   const uint32_t sbase = (smem_addr(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = sbase;                 // 64 KB: [half d][256 rows][64]
   const uint32_t sKV = sbase + 65536;        // 2 stages x (K 32 KB | V 32 KB), each [half d][128 slots][64]
-  // barrier indices
-  enum { B_QFULL = 0, B_KFULL = 1, B_VFULL = 3, B_KEMPTY = 5, B_VEMPTY = 7, B_SREADY = 9, B_PREADY = 11, B_ODONE = 13 };
+  enum {
+    B_QFULL = 0, B_QFREE = 1, B_ODONE = 2, B_KFULL = 3, B_VFULL = 5, B_KEMPTY = 7, B_VEMPTY = 9, B_SREADY = 11,
+    B_PREADY = 13, B_OFREE = 15
+  };
   auto bar = [&](int i) { return smem_addr(&bars[i]); };
   volatile int* abortp = &s_abort;
 
   if (tid == 0) {
     s_abort = 0;
+    s_quit[0] = s_quit[1] = 0;
+    s_items_ready = 0;
+    rgs[0].n = rgs[1].n = rgs[2].n = 0;
     mbar_init(bar(B_QFULL), 1);
+    mbar_init(bar(B_QFREE), 1);
+    mbar_init(bar(B_ODONE), 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(B_KFULL + s), 1);
       mbar_init(bar(B_VFULL + s), 1);
@@ -150,27 +161,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       mbar_init(bar(B_VEMPTY + s), 1);
       mbar_init(bar(B_SREADY + s), 1);
       mbar_init(bar(B_PREADY + s), 8);
+      mbar_init(bar(B_OFREE + s), 8);
     }
-    mbar_init(bar(B_ODONE), 1);
     fence_mbar_init();
-    const int last_tok = min(a.n, tok0 + TOKB) - 1;
-    if (phase == 0) {
-      rg.n = 3;
-      rg.start[0] = 0;
-      rg.len[0] = a.sink_end;
-      rg.start[1] = a.loc_begin;
-      rg.len[1] = a.t0 - a.loc_begin;
-      rg.start[2] = a.t0;
-      rg.len[2] = last_tok + 1;
-    } else {
-      const size_t rb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
-      const int nr = min(c.rng_cnt[unit * c.Hkv + g], c.topk + 2);
-      rg.n = nr;
-      for (int i = 0; i < nr; ++i) {
-        rg.start[i] = c.rng_start[rb + i];
-        rg.len[i] = c.rng_len[rb + i];
-      }
-    }
   }
   // stale shared memory must never hold non-finite bit patterns: unfilled key slots are multiplied by P = 0
   for (uint32_t i = tid; i < 131072 / 16; i += kTcThreads)
@@ -182,24 +175,71 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   fence_after_sync();
   const uint32_t tmem = s_tmem_base;
   const int causal_ri = phase == 0 ? 2 : -1;
-  const size_t slab_row0 = (unit * c.Hkv + g) * (size_t)c.Tpad;
+
+  // decode a work item
+  struct Item {
+    int mb, g, l, layer, tok0;
+    size_t unit, slab_row0;
+  };
+  auto decode = [&](int item) {
+    Item w;
+    w.mb = item % MB;
+    w.g = (item / MB) % c.Hkv;
+    w.l = item / (MB * c.Hkv);
+    w.layer = a.layer_begin + w.l;
+    w.tok0 = w.mb * TOKB;
+    w.unit = unit_of(c, a.seq, w.layer);
+    w.slab_row0 = (w.unit * c.Hkv + w.g) * (size_t)c.Tpad;
+    return w;
+  };
 
   if (warp == 16) {
     // ------------------------------------------------------------------ TMA producer
     // Every lane walks the tile list; lane 0 owns the barrier bookkeeping and lanes 0-3 issue the copies of
     // (K low half, K high half, V low half, V high half) so that many small pieces do not serialise on one thread.
-    {
+    int jt = 0, ok = 1;
+    if (lane == 0) prefetch_tmap(&maps.q);
+    for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
+      const Item w = decode(item);
+      RangeList& rg = rgs[wi % 3];
       if (lane == 0) {
-        prefetch_tmap(&maps.q);
-        mbar_expect_tx(bar(B_QFULL), 65536);
-        tma_load_3d(sQ, &maps.q, 0, g * G, l * a.n + tok0, bar(B_QFULL));
-        tma_load_3d(sQ + 32768, &maps.q, 64, g * G, l * a.n + tok0, bar(B_QFULL));
+        // the Q buffer is free once every QK^T product of the previous item has completed
+        if (wi > 0) ok = mbar_wait(bar(B_QFREE), (wi - 1) & 1, abortp) ? 1 : 0;
+        // the key ranges of this item (the other roles read them after they have seen its Q tile arrive)
+        const int last_tok = min(a.n, w.tok0 + TOKB) - 1;
+        if (phase == 0) {
+          rg.n = 3;
+          rg.start[0] = 0;
+          rg.len[0] = a.sink_end;
+          rg.start[1] = a.loc_begin;
+          rg.len[1] = a.t0 - a.loc_begin;
+          rg.start[2] = a.t0;
+          rg.len[2] = last_tok + 1;
+        } else {
+          const size_t rb = (w.unit * c.Hkv + w.g) * (size_t)(c.topk + 2);
+          const int nr = min(c.rng_cnt[w.unit * c.Hkv + w.g], c.topk + 2);
+          rg.n = nr;
+          for (int i = 0; i < nr; ++i) {
+            rg.start[i] = c.rng_start[rb + i];
+            rg.len[i] = c.rng_len[rb + i];
+          }
+        }
+        // publish the ranges with a monotonic counter: a softmax thread may look for item wi only after the Q tile
+        // of item wi+1 has arrived, so a parity barrier could not tell the two apart
+        __threadfence_block();
+        *reinterpret_cast<volatile int*>(&s_items_ready) = wi + 1;
+        if (ok) {
+          mbar_expect_tx(bar(B_QFULL), 65536);
+          tma_load_3d(sQ, &maps.q, 0, w.g * G, w.l * a.n + w.tok0, bar(B_QFULL));
+          tma_load_3d(sQ + 32768, &maps.q, 64, w.g * G, w.l * a.n + w.tok0, bar(B_QFULL));
+        }
       }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      __syncwarp();
       TileIter it;
       it.rg = &rg;
       it.causal_ri = causal_ri;
-      int j = 0;
-      int ok = 1;
       int pslot[16], ptok[16], pbox[16];
       while (true) {
         int np = 0;
@@ -210,11 +250,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
               ++np;
             }))
           break;
-        const int st = j & 1;
+        const int st = jt & 1;
+        const uint32_t par = ((jt >> 1) - 1) & 1;
         uint32_t bytes = 0;
         for (int p = 0; p < np; ++p) bytes += (uint32_t)(8 << pbox[p]) * 256u;
         if (lane == 0) {
-          if (j >= 2) ok = mbar_wait(bar(B_KEMPTY + st), ((j >> 1) - 1) & 1, abortp) ? 1 : 0;
+          if (jt >= 2) ok = mbar_wait(bar(B_KEMPTY + st), par, abortp) ? 1 : 0;
           if (ok) mbar_expect_tx(bar(B_KFULL + st), bytes);
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -223,9 +264,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (lane < 2)
           for (int p = 0; p < np; ++p)
             tma_load_2d(sK + lane * 16384 + (uint32_t)pslot[p] * 128u, &kvmaps[pbox[p]], lane * 64,
-                        (int)((long long)slab_row0 + ptok[p]), bar(B_KFULL + st));
+                        (int)((long long)w.slab_row0 + ptok[p]), bar(B_KFULL + st));
         if (lane == 0) {
-          if (j >= 2) ok = mbar_wait(bar(B_VEMPTY + st), ((j >> 1) - 1) & 1, abortp) ? 1 : 0;
+          if (jt >= 2) ok = mbar_wait(bar(B_VEMPTY + st), par, abortp) ? 1 : 0;
           if (ok) mbar_expect_tx(bar(B_VFULL + st), bytes);
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -233,28 +274,22 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (lane == 2 || lane == 3)
           for (int p = 0; p < np; ++p)
             tma_load_2d(sV + (lane - 2) * 16384 + (uint32_t)pslot[p] * 128u, &kvmaps[pbox[p]], (lane - 2) * 64,
-                        (int)((long long)slab_row0 + ptok[p] + v_row_offset), bar(B_VFULL + st));
-        ++j;
+                        (int)((long long)w.slab_row0 + ptok[p] + v_row_offset), bar(B_VFULL + st));
+        ++jt;
       }
-      // drain: wait until the MMA warp has released the last stages so that no copy is in flight at exit
-      if (lane == 0)
-        for (int back = 1; back <= 2 && back <= j; ++back) {
-          const int jj = j - back;
-          if (!mbar_wait(bar(B_VEMPTY + (jj & 1)), (jj >> 1) & 1, abortp)) break;
-        }
-      __syncwarp();
     }
+    // drain: wait until the MMA warp has released the last stages so that no copy is in flight at exit
+    if (lane == 0)
+      for (int back = 1; back <= 2 && back <= jt; ++back) {
+        const int jj = jt - back;
+        if (!mbar_wait(bar(B_VEMPTY + (jj & 1)), (jj >> 1) & 1, abortp)) break;
+      }
+    __syncwarp();
   } else if (warp == 17) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      TileIter it;
-      it.rg = &rg;
-      it.causal_ri = causal_ri;
-      int T = 0;
-      while (it.next()) ++T;
       constexpr uint32_t idesc_qk = make_idesc(128, 128, false);
       constexpr uint32_t idesc_pv = make_idesc(128, 128, true);
-      bool ok = mbar_wait(bar(B_QFULL), 0, abortp);
       // descriptors differ only in their start-address field: build one per operand, then add constants
       // (the address field holds bytes/16 and cannot carry out for any shared-memory offset)
       const uint64_t dQ = make_desc(sQ, 16, 1024);
@@ -278,30 +313,48 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) mma_ts(d, pa + ks * 8, db + ((ks * 2048) >> 4), idesc_pv, acc || ks > 0);
       };
-      if (ok && T > 0) {
-        ok = mbar_wait(bar(B_KFULL + 0), 0, abortp);
-        if (ok) {
+      int jt = 0;
+      bool ok = true;
+      for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
+        ok = mbar_wait(bar(B_QFULL), wi & 1, abortp);
+        if (!ok) break;
+        TileIter it;
+        it.rg = &rgs[wi % 3];
+        it.causal_ri = causal_ri;
+        int T = 0;
+        while (it.next()) ++T;
+        if (T > 0) {
+          ok = mbar_wait(bar(B_KFULL + (jt & 1)), (jt >> 1) & 1, abortp);
+          if (!ok) break;
           fence_after_sync();
-          issue_qk(0, 0);
-          issue_qk(1, 0);
-          mma_commit(bar(B_KEMPTY + 0));
+          issue_qk(0, jt & 1);
+          issue_qk(1, jt & 1);
+          mma_commit(bar(B_KEMPTY + (jt & 1)));
+          if (T == 1) mma_commit(bar(B_QFREE));
+        } else {
+          mma_commit(bar(B_QFREE));
         }
-        for (int j = 0; ok && j < T; ++j) {
-          const int st = j & 1, nst = st ^ 1;
+        for (int j = 0; ok && j < T; ++j, ++jt) {
+          const int st = jt & 1, nst = st ^ 1;
           const bool acc = (j > 0) || (phase == 1);
-          ok = mbar_wait(bar(B_VFULL + st), (j >> 1) & 1, abortp);
+          ok = mbar_wait(bar(B_VFULL + st), (jt >> 1) & 1, abortp);
           if (!ok) break;
-          ok = mbar_wait(bar(B_PREADY + 0), j & 1, abortp);
+          ok = mbar_wait(bar(B_PREADY + 0), jt & 1, abortp);
           if (!ok) break;
+          // the first P.V product of an item overwrites O: the previous item's epilogue must have read it
+          if (j == 0 && wi > 0) {
+            ok = mbar_wait(bar(B_OFREE + 0), (wi - 1) & 1, abortp) && mbar_wait(bar(B_OFREE + 1), (wi - 1) & 1, abortp);
+            if (!ok) break;
+          }
           fence_after_sync();
           issue_pv(0, st, acc);
           if (j + 1 < T) {
-            ok = mbar_wait(bar(B_KFULL + nst), ((j + 1) >> 1) & 1, abortp);
+            ok = mbar_wait(bar(B_KFULL + nst), ((jt + 1) >> 1) & 1, abortp);
             if (!ok) break;
             fence_after_sync();
             issue_qk(0, nst);
           }
-          ok = mbar_wait(bar(B_PREADY + 1), j & 1, abortp);
+          ok = mbar_wait(bar(B_PREADY + 1), jt & 1, abortp);
           if (!ok) break;
           fence_after_sync();
           issue_pv(1, st, acc);
@@ -309,10 +362,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           if (j + 1 < T) {
             issue_qk(1, nst);
             mma_commit(bar(B_KEMPTY + nst));
+            if (j + 2 == T) mma_commit(bar(B_QFREE));  // the last QK^T products of the item are in flight
           }
         }
+        if (!ok) break;
+        mma_commit(bar(B_ODONE));
       }
-      mma_commit(bar(B_ODONE));
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
@@ -323,129 +378,155 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     const int q = warp >> 3;
     const int half = (warp >> 2) & 1;
     const int r = (warp & 3) * 32 + lane;        // row inside the 128-row tile = TMEM lane
-    const int rr = q * 128 + r;                  // row inside the CTA
-    const int tk = tok0 + rr / G;                // call-relative token
-    const int h = g * G + rr % G;
-    const bool row_ok = tk < a.n;
+    const int rr = q * 128 + r;                  // row inside the work item
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_base + q * 128 + half * 64;   // this thread's 64 logits
     const uint32_t tP = tmem + lane_base + q * 128 + half * 32;   // its 64 probabilities (bf16 pairs)
     const uint32_t tO = tmem + lane_base + 256 + q * 128 + half * 64;
     const float c2 = c.scale * kLog2eT;
-    float m_used = -INFINITY, lsum = 0.f;
-    if (phase == 1) {
-      const float* op = c.Oacc + (((size_t)layer * c.chunk + (row_ok ? tk : 0)) * c.Hq + h) * kD + half * 64;
-      if (row_ok) {
-        const float2 stt = c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h];
-        m_used = stt.x;
-        lsum = half == 0 ? stt.y : 0.f;
-      }
-#pragma unroll 1
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t v[32];
-#pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-          const float4 f = row_ok ? *reinterpret_cast<const float4*>(op + ch * 32 + e) : make_float4(0, 0, 0, 0);
-          v[e] = __float_as_uint(f.x);
-          v[e + 1] = __float_as_uint(f.y);
-          v[e + 2] = __float_as_uint(f.z);
-          v[e + 3] = __float_as_uint(f.w);
-        }
-        tmem_st32(tO + ch * 32, v);
-      }
-      tmem_st_wait();
-    }
-    TileIter it;
-    it.rg = &rg;
-    it.causal_ri = causal_ri;
-    int j = 0;
+    int jt = 0;
     bool ok = true;
-    const int row_abs = a.t0 + tk;
-    while (it.next()) {
-      // after an expired wait every thread keeps walking the loop (without computing) so that the named barrier
-      // is still reached by all 256 threads of the tile
-      ok = ok && mbar_wait(bar(B_SREADY + q), j & 1, abortp);
-      if (!ok) {
-        asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
-        ++j;
-        continue;
-      }
-      fence_after_sync();
-      uint32_t v[2][32];
-      tmem_ld32(tS, v[0]);
-      tmem_ld32(tS + 32, v[1]);
-      tmem_ld_wait();
-      if (!it.full) {
-#pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          const unsigned mk = it.mask(half * 2 + ch);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            bool okc = (mk >> e) & 1u;
-            if (it.causal_tok0 >= 0) okc = okc && (it.causal_tok0 + half * 64 + ch * 32 + e <= row_abs);
-            if (!okc) v[ch][e] = 0xff800000u;  // -inf
+    for (int item = blockIdx.x, wi = 0; item < nitems; item += gridDim.x, ++wi) {
+      const Item w = decode(item);
+      const int tk = w.tok0 + rr / G;              // call-relative token
+      const int h = w.g * G + rr % G;
+      const bool row_ok = tk < a.n;
+      const int layer = w.layer;
+      if (ok) {
+        // wait (bounded) until the producer has published this item's key ranges
+        const long long t0c = clock64();
+        while (*reinterpret_cast<volatile int*>(&s_items_ready) <= wi) {
+          if (*abortp) {
+            ok = false;
+            break;
+          }
+          if (clock64() - t0c > kWaitLimitCycles) {
+            *abortp = 1;
+            ok = false;
+            break;
           }
         }
+        __threadfence_block();
       }
-      float mt = -INFINITY;
-#pragma unroll
-      for (int ch = 0; ch < 2; ++ch)
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) mt = max3(mt, __uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1]));
-      s_max[q][half][r] = mt;
-      asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
-      mt = fmaxf(mt, s_max[q][half ^ 1][r]) * c2;
-      // lazy running maximum: move it only when it grows by more than the threshold (or on first use)
-      float alpha = 1.f;
-      const bool grow = mt > m_used + kRescaleThreshold || (m_used == -INFINITY && mt > -INFINITY);
-      if (grow) {
-        alpha = ex2(m_used - mt);  // 0 when m_used = -inf
-        m_used = mt;
-        lsum *= alpha;
-      }
-      const bool have_o = (j > 0) || (phase == 1);
-      if (have_o && __any_sync(0xffffffffu, grow)) {
+      float m_used = -INFINITY, lsum = 0.f;
+      if (ok && phase == 1) {
+        // continue from the state the local pass stored: running max, row sum and the unnormalised O row
+        const float* op = c.Oacc + (((size_t)layer * c.chunk + (row_ok ? tk : 0)) * c.Hq + h) * kD + half * 64;
+        if (row_ok) {
+          const float2 stt = c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h];
+          m_used = stt.x;
+          lsum = half == 0 ? stt.y : 0.f;
+        }
 #pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t w[16];
-          tmem_ld16(tO + ch * 16, w);
-          tmem_ld_wait();
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t v[32];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * alpha);
-          tmem_st16(tO + ch * 16, w);
+          for (int e = 0; e < 32; e += 4) {
+            const float4 f = row_ok ? *reinterpret_cast<const float4*>(op + ch * 32 + e) : make_float4(0, 0, 0, 0);
+            v[e] = __float_as_uint(f.x);
+            v[e + 1] = __float_as_uint(f.y);
+            v[e + 2] = __float_as_uint(f.z);
+            v[e + 3] = __float_as_uint(f.w);
+          }
+          tmem_st32(tO + ch * 32, v);
         }
         tmem_st_wait();
       }
-      // probabilities, row sum, P (bf16).  Masked entries are -inf -> exp2 gives 0.
-      const float mneg = m_used == -INFINITY ? 0.f : -m_used;
-      const float2 c2v = make_float2(c2, c2), mnv = make_float2(mneg, mneg);
-      float2 ls = make_float2(0.f, 0.f);
-#pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          // packed fp32x2 arithmetic: one FFMA2 and one FADD2 per pair of logits
-          const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1])), c2v, mnv);
-          const float2 pp = make_float2(ex2(x.x), ex2(x.y));
-          ls = __fadd2_rn(ls, pp);
-          pk[e >> 1] = pack2(pp.x, pp.y);
+      TileIter it;
+      it.rg = &rgs[wi % 3];
+      it.causal_ri = causal_ri;
+      int j = 0;
+      const int row_abs = a.t0 + tk;
+      while (it.next()) {
+        // after an expired wait every thread keeps walking the item's tiles (without computing) so that the named
+        // barrier is still reached by all 256 threads of the tile
+        ok = ok && mbar_wait(bar(B_SREADY + q), jt & 1, abortp);
+        if (!ok) {
+          asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+          ++j;
+          ++jt;
+          continue;
         }
-        tmem_st16(tP + ch * 16, pk);
+        fence_after_sync();
+        uint32_t v[2][32];
+        tmem_ld32(tS, v[0]);
+        tmem_ld32(tS + 32, v[1]);
+        tmem_ld_wait();
+        if (!it.full) {
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) {
+            const unsigned mk = it.mask(half * 2 + ch);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              bool okc = (mk >> e) & 1u;
+              if (it.causal_tok0 >= 0) okc = okc && (it.causal_tok0 + half * 64 + ch * 32 + e <= row_abs);
+              if (!okc) v[ch][e] = 0xff800000u;  // -inf
+            }
+          }
+        }
+        float mt = -INFINITY;
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch)
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) mt = max3(mt, __uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1]));
+        s_max[q][half][r] = mt;
+        asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+        mt = fmaxf(mt, s_max[q][half ^ 1][r]) * c2;
+        // lazy running maximum: move it only when it grows by more than the threshold (or on first use)
+        float alpha = 1.f;
+        const bool grow = mt > m_used + kRescaleThreshold || (m_used == -INFINITY && mt > -INFINITY);
+        if (grow) {
+          alpha = ex2(m_used - mt);  // 0 when m_used = -inf
+          m_used = mt;
+          lsum *= alpha;
+        }
+        const bool have_o = (j > 0) || (phase == 1);
+        if (have_o && __any_sync(0xffffffffu, grow)) {
+#pragma unroll 1
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t wv[16];
+            tmem_ld16(tO + ch * 16, wv);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) wv[e] = __float_as_uint(__uint_as_float(wv[e]) * alpha);
+            tmem_st16(tO + ch * 16, wv);
+          }
+          tmem_st_wait();
+        }
+        // probabilities, row sum, P (bf16).  Masked entries are -inf -> exp2 gives 0.
+        const float mneg = m_used == -INFINITY ? 0.f : -m_used;
+        const float2 c2v = make_float2(c2, c2), mnv = make_float2(mneg, mneg);
+        float2 ls = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            // packed fp32x2 arithmetic: one FFMA2 and one FADD2 per pair of logits
+            const float2 x =
+                __ffma2_rn(make_float2(__uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1])), c2v, mnv);
+            const float2 pp = make_float2(ex2(x.x), ex2(x.y));
+            ls = __fadd2_rn(ls, pp);
+            pk[e >> 1] = pack2(pp.x, pp.y);
+          }
+          tmem_st16(tP + ch * 16, pk);
+        }
+        lsum += ls.x + ls.y;
+        tmem_st_wait();
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_PREADY + q));
+        ++j;
+        ++jt;
       }
-      lsum += ls.x + ls.y;
-      tmem_st_wait();
-      fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_PREADY + q));
-      ++j;
-    }
-    // epilogue: the two halves of a row exchange their partial sums, then each writes its 64 output columns
-    s_max[q][half][r] = lsum;
-    asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
-    lsum += s_max[q][half ^ 1][r];
-    if (ok) ok = mbar_wait(bar(B_ODONE), 0, abortp);
-    if (ok) {
+      // epilogue: the two halves of a row exchange their partial sums, then each writes its 64 output columns
+      s_max[q][half][r] = lsum;
+      asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+      lsum += s_max[q][half ^ 1][r];
+      if (ok) ok = mbar_wait(bar(B_ODONE), wi & 1, abortp);
+      if (!ok) s_quit[q] = 1;
+      asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");  // also: s_max is reused by the next item
+      if (s_quit[q]) break;  // collective decision: all 256 threads of the tile leave after the same item
       fence_after_sync();
       if (phase == 0 && row_ok && half == 0) {
         c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(m_used, lsum);
@@ -453,33 +534,39 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       }
       const float inv = 1.f / lsum;
       const bool have_o = (j > 0) || (phase == 1);
-#pragma unroll 1
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t v[32];
-        if (have_o) {
-          tmem_ld32(tO + ch * 32, v);
-          tmem_ld_wait();
-        } else {
+      uint32_t ov[2][32];
+      if (have_o) {
+        tmem_ld32(tO, ov[0]);
+        tmem_ld32(tO + 32, ov[1]);
+        tmem_ld_wait();
+      } else {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] = 0u;
-        }
-        if (!row_ok) continue;
-        if (phase == 0 && !final_out) {
-          float* op = c.Oacc + (((size_t)layer * c.chunk + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
+        for (int e = 0; e < 32; ++e) ov[0][e] = ov[1][e] = 0u;
+      }
+      // O is in registers: the next item's first P.V product may overwrite the accumulator
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_OFREE + q));
+      if (row_ok) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<uint4*>(op + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
-        }
-        if (final_out) {
-          __nv_bfloat16* op = a.out + (((size_t)l * a.n + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
+        for (int ch = 0; ch < 2; ++ch) {
+          if (phase == 0 && !final_out) {
+            float* op = c.Oacc + (((size_t)layer * c.chunk + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
 #pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 w;
-            w.x = pack2(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv);
-            w.y = pack2(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
-            w.z = pack2(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
-            w.w = pack2(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
-            *reinterpret_cast<uint4*>(op + e) = w;
+            for (int e = 0; e < 32; e += 4)
+              *reinterpret_cast<uint4*>(op + e) = make_uint4(ov[ch][e], ov[ch][e + 1], ov[ch][e + 2], ov[ch][e + 3]);
+          }
+          if (final_out) {
+            __nv_bfloat16* op = a.out + (((size_t)w.l * a.n + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
+#pragma unroll
+            for (int e = 0; e < 32; e += 8) {
+              uint4 wv;
+              wv.x = pack2(__uint_as_float(ov[ch][e]) * inv, __uint_as_float(ov[ch][e + 1]) * inv);
+              wv.y = pack2(__uint_as_float(ov[ch][e + 2]) * inv, __uint_as_float(ov[ch][e + 3]) * inv);
+              wv.z = pack2(__uint_as_float(ov[ch][e + 4]) * inv, __uint_as_float(ov[ch][e + 5]) * inv);
+              wv.w = pack2(__uint_as_float(ov[ch][e + 6]) * inv, __uint_as_float(ov[ch][e + 7]) * inv);
+              *reinterpret_cast<uint4*>(op + e) = wv;
+            }
           }
         }
       }
@@ -490,7 +577,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __syncthreads();
   fence_after_sync();
   if (warp == 16) tmem_dealloc(tmem, 512);
-  if (tid == 0 && s_abort) set_status(c, -6, (int)(blockIdx.x + 1000 * blockIdx.y));
+  if (tid == 0 && s_abort) set_status(c, -6, (int)blockIdx.x);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -558,8 +645,17 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase,
   const int smem = 65536 + 131072 + 1024;
   cudaFuncSetAttribute(k_attn_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   const long long v_off = (long long)c.NS * c.NL * c.Hkv * c.Tpad;
-  k_attn_tc<G><<<dim3((a.n + TOKB - 1) / TOKB, c.Hkv, a.layer_count), kTcThreads, smem, s>>>(c, a, phase,
-                                                                                           final_out ? 1 : 0, maps, v_off);
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    // testing aid: fewer CTAs make every CTA walk several work items even on small problems
+    if (const char* cap = getenv("LTRI_TC_MAX_CTAS")) sms = max(1, min(sms, atoi(cap)));
+  }
+  // persistent CTAs: one per SM (the kernel needs the whole TMEM and most of the shared memory of an SM)
+  const int nitems = ((a.n + TOKB - 1) / TOKB) * c.Hkv * a.layer_count;
+  k_attn_tc<G><<<min(nitems, sms), kTcThreads, smem, s>>>(c, a, phase, final_out ? 1 : 0, maps, v_off);
   return cudaGetLastError();
 }
 

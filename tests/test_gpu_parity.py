@@ -121,6 +121,16 @@ def test_decode_retrieval_paths(fused, monkeypatch):
     print(rep)
 
 
+def test_persistent_ctas_walk_several_work_items(monkeypatch):
+    # the tensor-core attention kernel is persistent (one CTA per SM); with the CTA count capped every CTA has to
+    # process several (token block, KV head, layer) items back to back, including one-tile items
+    monkeypatch.setenv("LTRI_TC_MAX_CTAS", "3")
+    cfg = small_cfg(n_layers=2, context=1024, decode_steps=0)
+    rep = ph.run_stream(cfg, layers=[0, 1], deep=False)
+    assert rep.calls == 8
+    print(rep)
+
+
 def test_warp_mma_fallback_path(monkeypatch):
     # the warp-MMA kernels remain selectable; they must match the oracle as well
     monkeypatch.setenv("LTRI_ATTN_IMPL", "mma")
