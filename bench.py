@@ -46,7 +46,8 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only)."""
+    """Samples SM clocks and throttle reasons while the timed region runs (read-only NVML queries every 20 ms;
+    falls back to `nvidia-smi -lms 200` when the NVML binding is missing)."""
 
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -56,8 +57,30 @@ class ClockSampler:
         self.index = index
         self.proc = None
         self.lines = []
+        self.samples = []       # (sm_mhz, reasons bitmask, power W)
+        self.stop_flag = False
+        self.nvml = None
+        self.thread = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = self.index
+            if vis:
+                try:
+                    phys = int(vis.split(",")[self.index])
+                except ValueError:
+                    phys = self.index
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.sm_max = pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
                                           "--format=csv,noheader,nounits", "-lms", "200"],
@@ -67,13 +90,43 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def _poll(self):
+        n = self.nvml
+        while not self.stop_flag:
+            try:
+                mhz = n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)
+                reasons = n.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                watts = n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0
+                self.samples.append((mhz, reasons, watts))
+            except Exception:
+                pass
+            time.sleep(0.02)
+
     def _read(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
-    def stop(self):
+    def mark(self):
+        """Index of the next sample (to restrict the summary to a window)."""
+        return len(self.samples)
+
+    def stop(self, lo=0, hi=None):
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+            n = self.nvml
+            win = self.samples[lo:hi] or self.samples
+            sm = [s[0] for s in win]
+            names = {"hw_slowdown": n.nvmlClocksEventReasonHwSlowdown,
+                     "hw_thermal_slowdown": n.nvmlClocksEventReasonHwThermalSlowdown,
+                     "sw_thermal_slowdown": n.nvmlClocksEventReasonSwThermalSlowdown,
+                     "sw_power_cap": n.nvmlClocksEventReasonSwPowerCap}
+            reasons = sorted(k for k, bit in names.items() if any(s[1] & bit for s in win))
+            return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": float(self.sm_max),
+                    "samples": len(sm), "power_w_max": max((s[2] for s in win), default=None), "reasons": reasons,
+                    "source": "nvml, 20 ms"}
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source available"]}
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -93,7 +146,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "source": "nvidia-smi -lms 200"}
 
 
 def dist_setup(n_gpus):
@@ -243,12 +296,14 @@ def run_ltri(args, cfg):
     launches0 = lt.ltri_launch_count()
     barrier(world)
     torch.cuda.synchronize(dev)
+    clk_lo = sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(K):
         lt.ltri_prefill_chunk(0, 0, L, *kept[W + i], out=outs[i & 1])
     e1.record()
     torch.cuda.synchronize(dev)
+    clk_hi = sampler.mark()
     barrier(world)
     ms = e0.elapsed_time(e1)
     launches = lt.ltri_launch_count() - launches0
@@ -295,7 +350,7 @@ def run_ltri(args, cfg):
                             "traffic": None, "kernels": "decode score+top-k and split-KV attention+merge",
                             "of": peaks["source"]},
                "kernel_ms_per_step": {k: v[0] / dsteps for k, v in dprof.items() if v[1]}}
-    clocks = sampler.stop()
+    clocks = sampler.stop(clk_lo, clk_hi)
 
     # ---- end-to-end: same steps with host buffers ---------------------------------------------
     e2e = None
@@ -345,7 +400,7 @@ def run_ltri(args, cfg):
     tf = flops / (a_ms * 1e-3) / 1e12 if a_ms > 0 else None
     peak_tf = peaks["bf16_tflops_sustained"]
     roof = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
-            "frac": tf / peak_tf if tf else None, "traffic": None, "kernel": "k_attn_prefill (local part)",
+            "frac": tf / peak_tf if tf else None, "traffic": None, "kernel": "k_attn_tc, local part (sink | local | current)",
             "launches": a_cnt, "ms_per_launch": a_ms / max(a_cnt, 1), "of": peaks["source"] + " (sustained)"}
     cpu = None
     if not args.no_cpu_baseline:

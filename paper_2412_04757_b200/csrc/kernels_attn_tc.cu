@@ -102,6 +102,19 @@ struct TileIter {
   __device__ __forceinline__ unsigned mask(int w) const { return w == 0 ? m0 : w == 1 ? m1 : w == 2 ? m2 : m3; }
 };
 
+// Number of tiles the iterator yields for a range list: every range is padded to 8 rows and the causal range starts
+// a fresh tile.
+__device__ __forceinline__ int count_tiles(const RangeList* rg, int causal_ri) {
+  int slots = 0;
+  for (int i = 0; i < rg->n; ++i) {
+    const int len = rg->len[i];
+    if (len <= 0) continue;
+    if (i == causal_ri) slots = (slots + 127) & ~127;
+    slots += (len + 7) & ~7;
+  }
+  return (slots + 127) >> 7;
+}
+
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -191,6 +204,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     w.unit = unit_of(c, a.seq, w.layer);
     w.slab_row0 = (w.unit * c.Hkv + w.g) * (size_t)c.Tpad;
     return w;
+  };
+
+  // unnormalised O state between the two phases: one 128 x 128 fp32 block per (layer, item, Q tile)
+  auto oacc_base = [&](const Item& w, int q) -> size_t {
+    return ((((size_t)w.layer * MB + w.mb) * c.Hkv + w.g) * 2 + q) * (size_t)(128 * kD);
   };
 
   if (warp == 16) {
@@ -318,11 +336,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
         ok = mbar_wait(bar(B_QFULL), wi & 1, abortp);
         if (!ok) break;
-        TileIter it;
-        it.rg = &rgs[wi % 3];
-        it.causal_ri = causal_ri;
-        int T = 0;
-        while (it.next()) ++T;
+        const int T = count_tiles(&rgs[wi % 3], causal_ri);
         if (T > 0) {
           ok = mbar_wait(bar(B_KFULL + (jt & 1)), (jt >> 1) & 1, abortp);
           if (!ok) break;
@@ -411,7 +425,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       float m_used = -INFINITY, lsum = 0.f;
       if (ok && phase == 1) {
         // continue from the state the local pass stored: running max, row sum and the unnormalised O row
-        const float* op = c.Oacc + (((size_t)layer * c.chunk + (row_ok ? tk : 0)) * c.Hq + h) * kD + half * 64;
+        const float* op = c.Oacc + oacc_base(w, q) + (size_t)(half * 16) * 512 + r * 4;
         if (row_ok) {
           const float2 stt = c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h];
           m_used = stt.x;
@@ -422,7 +436,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           uint32_t v[32];
 #pragma unroll
           for (int e = 0; e < 32; e += 4) {
-            const float4 f = row_ok ? *reinterpret_cast<const float4*>(op + ch * 32 + e) : make_float4(0, 0, 0, 0);
+            const float4 f = row_ok ? *reinterpret_cast<const float4*>(op + (size_t)(ch * 8 + (e >> 2)) * 512)
+                                    : make_float4(0, 0, 0, 0);
             v[e] = __float_as_uint(f.x);
             v[e + 1] = __float_as_uint(f.y);
             v[e + 2] = __float_as_uint(f.z);
@@ -453,15 +468,15 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         tmem_ld32(tS + 32, v[1]);
         tmem_ld_wait();
         if (!it.full) {
+          // valid-slot bits, and for the causal tile the last visible column of this row (keys are consecutive
+          // tokens from slot 0): column c is visible iff c <= lim
+          const int lim = it.causal_tok0 >= 0 ? row_abs - it.causal_tok0 - half * 64 : 127;
 #pragma unroll
           for (int ch = 0; ch < 2; ++ch) {
             const unsigned mk = it.mask(half * 2 + ch);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              bool okc = (mk >> e) & 1u;
-              if (it.causal_tok0 >= 0) okc = okc && (it.causal_tok0 + half * 64 + ch * 32 + e <= row_abs);
-              if (!okc) v[ch][e] = 0xff800000u;  // -inf
-            }
+            for (int e = 0; e < 32; ++e)
+              if (!((mk >> e) & 1u) || ch * 32 + e > lim) v[ch][e] = 0xff800000u;  // -inf
           }
         }
         float mt = -INFINITY;
@@ -551,10 +566,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
           if (phase == 0 && !final_out) {
-            float* op = c.Oacc + (((size_t)layer * c.chunk + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
+            // scratch layout [4-float column group][row][4]: the 32 rows of a warp write 512 contiguous bytes
+            float* op = c.Oacc + oacc_base(w, q) + (size_t)(half * 16 + ch * 8) * 512 + r * 4;
 #pragma unroll
             for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<uint4*>(op + e) = make_uint4(ov[ch][e], ov[ch][e + 1], ov[ch][e + 2], ov[ch][e + 3]);
+              *reinterpret_cast<uint4*>(op + (size_t)(e >> 2) * 512) =
+                  make_uint4(ov[ch][e], ov[ch][e + 1], ov[ch][e + 2], ov[ch][e + 3]);
           }
           if (final_out) {
             __nv_bfloat16* op = a.out + (((size_t)w.l * a.n + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
@@ -650,12 +667,13 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase,
     int dev = 0;
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-    // testing aid: fewer CTAs make every CTA walk several work items even on small problems
-    if (const char* cap = getenv("LTRI_TC_MAX_CTAS")) sms = max(1, min(sms, atoi(cap)));
   }
+  int ctas = sms;
+  // testing aid: fewer CTAs make every CTA walk several work items even on small problems
+  if (const char* cap = getenv("LTRI_TC_MAX_CTAS")) ctas = max(1, min(sms, atoi(cap)));
   // persistent CTAs: one per SM (the kernel needs the whole TMEM and most of the shared memory of an SM)
   const int nitems = ((a.n + TOKB - 1) / TOKB) * c.Hkv * a.layer_count;
-  k_attn_tc<G><<<min(nitems, sms), kTcThreads, smem, s>>>(c, a, phase, final_out ? 1 : 0, maps, v_off);
+  k_attn_tc<G><<<min(nitems, ctas), kTcThreads, smem, s>>>(c, a, phase, final_out ? 1 : 0, maps, v_off);
   return cudaGetLastError();
 }
 

@@ -101,7 +101,8 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.thetaq = cv.take<long long>(d.NL);
   d.rowstat = cv.take<float2>((size_t)d.NL * d.chunk * d.Hq);
   d.rowq = cv.take<float2>((size_t)d.NL * d.chunk * d.Hq);
-  d.Oacc = cv.take<float>((size_t)d.NL * d.chunk * d.Hq * kD);
+  // rows padded to whole 256-row work items of the tensor-core attention kernel
+  d.Oacc = cv.take<float>((size_t)d.NL * align_up((size_t)d.chunk * d.G, 256) * d.Hkv * kD);
   d.u = cv.take<float>((size_t)d.NL * d.Hkv * d.Jmax * kD);
   d.Jcnt = cv.take<int>(d.NL);
   d.scores = cv.take<float>(units * d.Hkv * d.cap);
