@@ -14,6 +14,8 @@ constexpr float kQScale = 1048576.0f;
 constexpr int kMaxReps = 8;
 constexpr int kMaxTopK = 64;
 constexpr int kMaxDecSplit = 32;
+constexpr float kMapMargin = 0.0078125f;          // safety margin (in log2 units) of the map pass's skip test
+constexpr float kMapScale = 0.4972997117f;         // 2^-(1 + kMapMargin)
 constexpr int kTokPad = 128;          // rows of slack after every K/V slab so tile over-reads stay inside it
 
 // Device-side view of one context.  Passed to kernels by value.
@@ -43,7 +45,8 @@ struct DevCtx {
   long long* best;       // [NL][2*chunk]
   long long* thetaq;     // [NL]
   float2* rowstat;       // [NL][chunk][Hq]   (reference maximum m in scaled log2 units, row sum l)
-  float2* rowq;          // [NL][chunk][Hq]   (-m, 2^20 / l): the map pass turns a logit into a Q20 probability with these
+  float* rowq;           // [NL][chunk][Hq]   -m - log2(l) + 21 + kMapMargin: offset that turns a scaled logit into
+                         //                   log2 of its Q20 probability (see kernels_map_tc.cu)
   float* Oacc;           // [NL][chunk][Hq][128]  unnormalised accumulator of the local part
   float* u;              // [NL][Hkv][Jmax][128]  summed query representatives
   int* Jcnt;             // [NL]

@@ -545,7 +545,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       fence_after_sync();
       if (phase == 0 && row_ok && half == 0) {
         c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(m_used, lsum);
-        c.rowq[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(-m_used, kQScale / lsum);
+        c.rowq[((size_t)layer * c.chunk + tk) * c.Hq + h] = -m_used - __log2f(lsum) + (21.0f + kMapMargin);
       }
       const float inv = 1.f / lsum;
       const bool have_o = (j > 0) || (phase == 1);

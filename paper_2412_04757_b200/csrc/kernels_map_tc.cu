@@ -21,12 +21,20 @@ using namespace tc;
 
 constexpr float kLog2eM = 1.4426950408889634f;
 constexpr int kMapThreads = 320;
+// The attention kernel stores per row off = -m - log2(l) + 21 + kMapMargin, so that x = logit*scale*log2e + off is
+// log2(p * 2^20) + 1 + margin and the Q20 value is rint(2^x * kMapScale); x < 0 means the value is below
+// 2^-(1+margin) < 0.5 and rounds to zero.
 
 struct MapMaps {
   CUtensorMap q;    // [tokens][Hq][128] bf16, box {64, G, 128/G}
   CUtensorMap k128; // K slabs, box {64, 128}
 };
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ float ex2m(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -41,7 +49,7 @@ __global__ void __launch_bounds__(kMapThreads, 2)
   __shared__ __align__(8) unsigned long long bars[9];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ float2 s_stats[2][128];
+  __shared__ __align__(16) float s_stats[2][128];
   constexpr int TPB = 128 / G;  // tokens per query block
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
@@ -130,13 +138,13 @@ __global__ void __launch_bounds__(kMapThreads, 2)
     const int jrel = key - a.t0;              // call-relative (cur tiles only)
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float c2 = c.scale * kLog2eM;
-    const float2* rq = c.rowq + (size_t)layer * c.chunk * c.Hq + g * G;
+    const float* rq = c.rowq + (size_t)layer * c.chunk * c.Hq + g * G;
     int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
     const int roff = a.t0 - a.reg_start;      // region index = call-relative token + roff
-    // row statistics (-m, 2^20/l) of a block's 128 rows, staged in shared memory one block ahead
-    auto load_stats = [&](int blk) -> float2 {
+    // per-row offsets (see kMapMargin) of a block's 128 rows, staged in shared memory one block ahead
+    auto load_stats = [&](int blk) -> float {
       const int tk = blk * TPB + tid / G;
-      return (tid < 128 && tk < a.n) ? __ldg(rq + (size_t)tk * c.Hq + tid % G) : make_float2(-INFINITY, 0.f);
+      return (tid < 128 && tk < a.n) ? __ldg(rq + (size_t)tk * c.Hq + tid % G) : -INFINITY;
     };
     if (tid < 128 && blk0 < nblocks) s_stats[0][tid] = load_stats(blk0);
     asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -146,7 +154,7 @@ __global__ void __launch_bounds__(kMapThreads, 2)
     for (int blk = blk0; blk < nblocks; ++blk, ++it) {
       const int st = it & 1;
       const bool more = blk + 1 < nblocks;
-      float2 nxt = make_float2(-INFINITY, 0.f);
+      float nxt = -INFINITY;
       if (more) nxt = load_stats(blk + 1);
       // after an expired wait every thread keeps walking the loop (without computing) so that the named barrier
       // below is still reached by all 256 epilogue threads
@@ -162,17 +170,42 @@ __global__ void __launch_bounds__(kMapThreads, 2)
       tmem_ld_wait();
       const int tokb = blk * TPB;                              // first token of the block (call-relative)
       const bool diag = is_cur && tokb < (key0 - a.t0) + 128;  // some token of the block precedes some key
-      const float2* ss = &s_stats[st][chalf * 64];
+      const float* ss = &s_stats[st][chalf * 64];
       int bsum = 0;
 #pragma unroll
       for (int ch = 0; ch < 2; ++ch) {
         int aq[32];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float2 sq = ss[ch * 32 + e];
-          // round to nearest even by adding 1.5 * 2^23: the integer sits in the mantissa
-          const float x = ex2m(fmaf(__uint_as_float(v[ch][e]), c2, sq.x)) * sq.y + 12582912.f;
-          aq[e] = __float_as_int(x) - 0x4B400000;
+        for (int e8 = 0; e8 < 32; e8 += 8) {
+          // x = log2 of (probability * 2^20) + 1 + margin.  An entry with x < 0 rounds to zero, so a group of eight
+          // columns whose x is negative on every lane of the warp needs no exponentials at all.
+          const float4 o0 = *reinterpret_cast<const float4*>(ss + ch * 32 + e8);
+          const float4 o1 = *reinterpret_cast<const float4*>(ss + ch * 32 + e8 + 4);
+          const float2 c2v = make_float2(c2, c2);
+          float2 x[4];
+          x[0] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8]), __uint_as_float(v[ch][e8 + 1])), c2v,
+                            make_float2(o0.x, o0.y));
+          x[1] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 2]), __uint_as_float(v[ch][e8 + 3])), c2v,
+                            make_float2(o0.z, o0.w));
+          x[2] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 4]), __uint_as_float(v[ch][e8 + 5])), c2v,
+                            make_float2(o1.x, o1.y));
+          x[3] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 6]), __uint_as_float(v[ch][e8 + 7])), c2v,
+                            make_float2(o1.z, o1.w));
+          const float xm = fmaxf(fmaxf(fmax3(x[0].x, x[0].y, x[1].x), fmax3(x[1].y, x[2].x, x[2].y)),
+                                 fmaxf(x[3].x, x[3].y));
+          if (__any_sync(0xffffffffu, xm >= 0.f)) {
+            const float2 sc = make_float2(kMapScale, kMapScale), mg = make_float2(12582912.f, 12582912.f);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              // round to nearest even by adding 1.5 * 2^23: the integer sits in the mantissa
+              const float2 y = __ffma2_rn(make_float2(ex2m(x[e].x), ex2m(x[e].y)), sc, mg);
+              aq[e8 + 2 * e] = __float_as_int(y.x) - 0x4B400000;
+              aq[e8 + 2 * e + 1] = __float_as_int(y.y) - 0x4B400000;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) aq[e8 + e] = 0;
+          }
         }
         if (diag) {
 #pragma unroll

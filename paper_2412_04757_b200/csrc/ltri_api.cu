@@ -100,7 +100,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.best = cv.take<long long>((size_t)d.NL * 2 * d.chunk);
   d.thetaq = cv.take<long long>(d.NL);
   d.rowstat = cv.take<float2>((size_t)d.NL * d.chunk * d.Hq);
-  d.rowq = cv.take<float2>((size_t)d.NL * d.chunk * d.Hq);
+  d.rowq = cv.take<float>((size_t)d.NL * d.chunk * d.Hq);
   // rows padded to whole 256-row work items of the tensor-core attention kernel
   d.Oacc = cv.take<float>((size_t)d.NL * align_up((size_t)d.chunk * d.G, 256) * d.Hkv * kD);
   d.u = cv.take<float>((size_t)d.NL * d.Hkv * d.Jmax * kD);
