@@ -20,7 +20,7 @@ namespace ltri {
 using namespace tc;
 
 constexpr float kLog2eM = 1.4426950408889634f;
-constexpr int kMapThreads = 320;
+constexpr int kMapThreads = 576;  // 16 epilogue warps + TMA producer + MMA issuer
 // The attention kernel stores per row off = -m - log2(l) + 21 + kMapMargin, so that x = logit*scale*log2e + off is
 // log2(p * 2^20) + 1 + margin and the Q20 value is rint(2^x * kMapScale); x < 0 means the value is below
 // 2^-(1+margin) < 0.5 and rounds to zero.
@@ -41,12 +41,18 @@ __device__ __forceinline__ float ex2m(float x) {
   return y;
 }
 
-// grid (key tiles, Hkv, layers).  Key tiles [0, n_local_tiles) cover [loc_begin, t0); the rest cover [t0, t0+n).
+// grid (key-tile groups, Hkv, layers).  A CTA keeps up to kMapKT 128-key tiles of one KV head in shared memory (all
+// from [loc_begin, t0) or all from the call's own tokens [t0, t0+n)) and streams the query blocks through them once,
+// so the query tensor is re-read kMapKT times less often than with one key tile per CTA.
+constexpr int kMapKT = 4;
+
 template <int G>
-__global__ void __launch_bounds__(kMapThreads, 2)
-    k_map_tc(DevCtx c, PrefillArgs a, int n_local_tiles, const __grid_constant__ MapMaps maps) {
+__global__ void __launch_bounds__(kMapThreads, 1)
+    k_map_tc(DevCtx c, PrefillArgs a, int n_local_groups, int n_local_tiles, int n_cur_tiles,
+             const __grid_constant__ MapMaps maps) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[9];
+  // KFULL | QFULL[2] QEMPTY[2] | SFULL[4] SEMPTY[4]
+  __shared__ __align__(8) unsigned long long bars[1 + 4 + 8];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
   __shared__ __align__(16) float s_stats[2][128];
@@ -54,18 +60,21 @@ __global__ void __launch_bounds__(kMapThreads, 2)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
   const size_t unit = unit_of(c, a.seq, layer);
-  const bool is_cur = (int)blockIdx.x >= n_local_tiles;
-  // first key of the tile (absolute) and the end of its range
-  const int key0 = is_cur ? a.t0 + ((int)blockIdx.x - n_local_tiles) * 128 : a.loc_begin + (int)blockIdx.x * 128;
+  const bool is_cur = (int)blockIdx.x >= n_local_groups;
+  const int tile0 = (is_cur ? (int)blockIdx.x - n_local_groups : (int)blockIdx.x) * kMapKT;
+  const int ntile = min(kMapKT, (is_cur ? n_cur_tiles : n_local_tiles) - tile0);
+  // first key (absolute) of key tile kt, the end of the range, and the first query block that sees the tile
+  const int kbase = is_cur ? a.t0 : a.loc_begin;
   const int key_end = is_cur ? a.t0 + a.n : a.t0;
+  auto key0_of = [&](int kt) { return kbase + (tile0 + kt) * 128; };
+  auto blk0_of = [&](int kt) { return is_cur ? ((tile0 + kt) * 128) / TPB : 0; };
   const int nblocks = (a.n + TPB - 1) / TPB;
-  // causal tiles: query blocks whose tokens all precede the tile's first key see none of its keys
-  const int blk0 = is_cur ? (key0 - a.t0) / TPB : 0;
+  const int bmin = blk0_of(0);
 
   const uint32_t sbase = (smem_addr(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sK = sbase;            // 32 KB: [half d][128 keys][64]
-  const uint32_t sQ = sbase + 32768;    // 2 stages x 32 KB: [half d][128 rows][64]
-  enum { B_KFULL = 0, B_QFULL = 1, B_QEMPTY = 3, B_SFULL = 5, B_SEMPTY = 7 };
+  const uint32_t sK = sbase;                      // kMapKT x 32 KB: [tile][half d][128 keys][64]
+  const uint32_t sQ = sbase + kMapKT * 32768;     // 2 stages x 32 KB: [half d][128 rows][64]
+  enum { B_KFULL = 0, B_QFULL = 1, B_QEMPTY = 3, B_SFULL = 5, B_SEMPTY = 9 };
   auto bar = [&](int i) { return smem_addr(&bars[i]); };
   volatile int* abortp = &s_abort;
   if (tid == 0) {
@@ -74,26 +83,30 @@ __global__ void __launch_bounds__(kMapThreads, 2)
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(B_QFULL + s), 1);
       mbar_init(bar(B_QEMPTY + s), 1);
+    }
+    for (int s = 0; s < 4; ++s) {
       mbar_init(bar(B_SFULL + s), 1);
-      mbar_init(bar(B_SEMPTY + s), 8);
+      mbar_init(bar(B_SEMPTY + s), 16);
     }
     fence_mbar_init();
   }
-  if (warp == 8) tmem_alloc(smem_addr(&s_tmem_base), 256);
+  if (warp == 16) tmem_alloc(smem_addr(&s_tmem_base), 512);
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem = s_tmem_base;
 
-  if (warp == 8) {
+  if (warp == 16) {
     if (lane == 0) {
-      const long long krow = (long long)(unit * c.Hkv + g) * c.Tpad + key0;
-      mbar_expect_tx(bar(B_KFULL), 32768);
-      tma_load_2d(sK, &maps.k128, 0, (int)krow, bar(B_KFULL));
-      tma_load_2d(sK + 16384, &maps.k128, 64, (int)krow, bar(B_KFULL));
+      mbar_expect_tx(bar(B_KFULL), (uint32_t)ntile * 32768u);
+      for (int kt = 0; kt < ntile; ++kt) {
+        const long long krow = (long long)(unit * c.Hkv + g) * c.Tpad + key0_of(kt);
+        tma_load_2d(sK + kt * 32768, &maps.k128, 0, (int)krow, bar(B_KFULL));
+        tma_load_2d(sK + kt * 32768 + 16384, &maps.k128, 64, (int)krow, bar(B_KFULL));
+      }
       bool ok = true;
       int it = 0;
-      for (int blk = blk0; ok && blk < nblocks; ++blk, ++it) {
+      for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
         const int st = it & 1;
         if (it >= 2) ok = mbar_wait(bar(B_QEMPTY + st), ((it >> 1) - 1) & 1, abortp);
         if (!ok) break;
@@ -106,36 +119,40 @@ __global__ void __launch_bounds__(kMapThreads, 2)
         if (!mbar_wait(bar(B_QEMPTY + (ii & 1)), (ii >> 1) & 1, abortp)) break;
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == 17) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(128, 128, false);
       const uint64_t dK = make_desc(sK, 16, 1024), dQ = make_desc(sQ, 16, 1024);
       bool ok = mbar_wait(bar(B_KFULL), 0, abortp);
-      int it = 0;
-      for (int blk = blk0; ok && blk < nblocks; ++blk, ++it) {
+      int it = 0, seq = 0;
+      for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
         const int st = it & 1;
         ok = mbar_wait(bar(B_QFULL + st), (it >> 1) & 1, abortp);
         if (!ok) break;
-        if (it >= 2) ok = mbar_wait(bar(B_SEMPTY + st), ((it >> 1) - 1) & 1, abortp);
-        if (!ok) break;
-        fence_after_sync();
         const uint64_t db = dQ + (uint64_t)((st * 32768) >> 4);
+        for (int kt = 0; ok && kt < ntile; ++kt) {
+          if (blk < blk0_of(kt)) continue;
+          const int buf = seq & 3;
+          if (seq >= 4) ok = mbar_wait(bar(B_SEMPTY + buf), ((seq >> 2) - 1) & 1, abortp);
+          if (!ok) break;
+          fence_after_sync();
+          const uint64_t da = dK + (uint64_t)((kt * 32768) >> 4);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
-          mma_ss(tmem + st * 128, dK + off, db + off, idesc, ks > 0);
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
+            mma_ss(tmem + buf * 128, da + off, db + off, idesc, ks > 0);
+          }
+          mma_commit(bar(B_SFULL + buf));
+          ++seq;
         }
-        mma_commit(bar(B_SFULL + st));
+        if (!ok) break;
         mma_commit(bar(B_QEMPTY + st));
       }
     }
   } else {
-    // epilogue: thread = key (TMEM lane), columns [64*chalf, +64) of every block
-    const int chalf = warp >> 2;
-    const int krel = (warp & 3) * 32 + lane;  // key inside the tile
-    const int key = key0 + krel;              // absolute key token
-    const bool key_ok = key < key_end && key >= c.Ls;
-    const int jrel = key - a.t0;              // call-relative (cur tiles only)
+    // epilogue: thread = key (TMEM lane), columns [32*cq, +32) of every block
+    const int cq = warp >> 2;
+    const int krel = (warp & 3) * 32 + lane;  // key inside its tile
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float c2 = c.scale * kLog2eM;
     const float* rq = c.rowq + (size_t)layer * c.chunk * c.Hq + g * G;
@@ -146,102 +163,117 @@ __global__ void __launch_bounds__(kMapThreads, 2)
       const int tk = blk * TPB + tid / G;
       return (tid < 128 && tk < a.n) ? __ldg(rq + (size_t)tk * c.Hq + tid % G) : -INFINITY;
     };
-    if (tid < 128 && blk0 < nblocks) s_stats[0][tid] = load_stats(blk0);
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    long long total = 0;
+    if (tid < 128 && bmin < nblocks) s_stats[0][tid] = load_stats(bmin);
+    asm volatile("bar.sync 1, 512;" ::: "memory");
+    long long total[kMapKT];
+#pragma unroll
+    for (int kt = 0; kt < kMapKT; ++kt) total[kt] = 0;
     bool ok = true;
-    int it = 0;
-    for (int blk = blk0; blk < nblocks; ++blk, ++it) {
+    int it = 0, seq = 0;
+    for (int blk = bmin; blk < nblocks; ++blk, ++it) {
       const int st = it & 1;
       const bool more = blk + 1 < nblocks;
       float nxt = -INFINITY;
       if (more) nxt = load_stats(blk + 1);
-      // after an expired wait every thread keeps walking the loop (without computing) so that the named barrier
-      // below is still reached by all 256 epilogue threads
-      ok = ok && mbar_wait(bar(B_SFULL + st), (it >> 1) & 1, abortp);
-      if (!ok) {
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        continue;
-      }
-      fence_after_sync();
-      uint32_t v[2][32];
-      tmem_ld32(tmem + lane_base + st * 128 + chalf * 64, v[0]);
-      tmem_ld32(tmem + lane_base + st * 128 + chalf * 64 + 32, v[1]);
-      tmem_ld_wait();
-      const int tokb = blk * TPB;                              // first token of the block (call-relative)
-      const bool diag = is_cur && tokb < (key0 - a.t0) + 128;  // some token of the block precedes some key
-      const float* ss = &s_stats[st][chalf * 64];
-      int bsum = 0;
+      const int tokb = blk * TPB;  // first token of the block (call-relative)
+      const float* ss = &s_stats[st][cq * 32];
 #pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        int aq[32];
+      for (int kt = 0; kt < kMapKT; ++kt) {
+        if (kt >= ntile || blk < blk0_of(kt)) continue;
+        const int buf = seq & 3;
+        // after an expired wait every thread keeps walking the steps (without computing) so that the named barrier
+        // below is still reached by all 512 epilogue threads
+        ok = ok && mbar_wait(bar(B_SFULL + buf), (seq >> 2) & 1, abortp);
+        ++seq;
+        if (!ok) continue;
+        fence_after_sync();
+        uint32_t v[1][32];
+        tmem_ld32(tmem + lane_base + buf * 128 + cq * 32, v[0]);
+        tmem_ld_wait();
+        // the accumulator is in registers: hand the TMEM buffer back
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_SEMPTY + buf));
+        const int key0 = key0_of(kt);
+        const int key = key0 + krel;
+        const bool key_ok = key < key_end && key >= c.Ls;
+        const int jrel = key - a.t0;  // call-relative (cur tiles only)
+        const bool diag = is_cur && tokb < (key0 - a.t0) + 128;  // some token of the block precedes some key
+        int bsum = 0;
 #pragma unroll
-        for (int e8 = 0; e8 < 32; e8 += 8) {
-          // x = log2 of (probability * 2^20) + 1 + margin.  An entry with x < 0 rounds to zero, so a group of eight
-          // columns whose x is negative on every lane of the warp needs no exponentials at all.
-          const float4 o0 = *reinterpret_cast<const float4*>(ss + ch * 32 + e8);
-          const float4 o1 = *reinterpret_cast<const float4*>(ss + ch * 32 + e8 + 4);
-          const float2 c2v = make_float2(c2, c2);
-          float2 x[4];
-          x[0] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8]), __uint_as_float(v[ch][e8 + 1])), c2v,
-                            make_float2(o0.x, o0.y));
-          x[1] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 2]), __uint_as_float(v[ch][e8 + 3])), c2v,
-                            make_float2(o0.z, o0.w));
-          x[2] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 4]), __uint_as_float(v[ch][e8 + 5])), c2v,
-                            make_float2(o1.x, o1.y));
-          x[3] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 6]), __uint_as_float(v[ch][e8 + 7])), c2v,
-                            make_float2(o1.z, o1.w));
-          const float xm = fmaxf(fmaxf(fmax3(x[0].x, x[0].y, x[1].x), fmax3(x[1].y, x[2].x, x[2].y)),
-                                 fmaxf(x[3].x, x[3].y));
-          if (__any_sync(0xffffffffu, xm >= 0.f)) {
-            const float2 sc = make_float2(kMapScale, kMapScale), mg = make_float2(12582912.f, 12582912.f);
+        for (int ch = 0; ch < 1; ++ch) {
+          int aq[32];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              // round to nearest even by adding 1.5 * 2^23: the integer sits in the mantissa
-              const float2 y = __ffma2_rn(make_float2(ex2m(x[e].x), ex2m(x[e].y)), sc, mg);
-              aq[e8 + 2 * e] = __float_as_int(y.x) - 0x4B400000;
-              aq[e8 + 2 * e + 1] = __float_as_int(y.y) - 0x4B400000;
+          for (int e8 = 0; e8 < 32; e8 += 8) {
+            // x = log2 of (probability * 2^20) + 1 + margin.  An entry with x < 0 rounds to zero, so a group of
+            // eight columns whose x is negative on every lane of the warp needs no exponentials at all.
+            const float4 o0 = *reinterpret_cast<const float4*>(ss + ch * 32 + e8);
+            const float4 o1 = *reinterpret_cast<const float4*>(ss + ch * 32 + e8 + 4);
+            const float2 c2v = make_float2(c2, c2);
+            float2 x[4];
+            x[0] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8]), __uint_as_float(v[ch][e8 + 1])), c2v,
+                              make_float2(o0.x, o0.y));
+            x[1] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 2]), __uint_as_float(v[ch][e8 + 3])), c2v,
+                              make_float2(o0.z, o0.w));
+            x[2] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 4]), __uint_as_float(v[ch][e8 + 5])), c2v,
+                              make_float2(o1.x, o1.y));
+            x[3] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 6]), __uint_as_float(v[ch][e8 + 7])), c2v,
+                              make_float2(o1.z, o1.w));
+            const float xm = fmaxf(fmaxf(fmax3(x[0].x, x[0].y, x[1].x), fmax3(x[1].y, x[2].x, x[2].y)),
+                                   fmaxf(x[3].x, x[3].y));
+            if (__any_sync(0xffffffffu, xm >= 0.f)) {
+              const float2 sc = make_float2(kMapScale, kMapScale), mg = make_float2(12582912.f, 12582912.f);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                // round to nearest even by adding 1.5 * 2^23: the integer sits in the mantissa
+                const float2 y = __ffma2_rn(make_float2(ex2m(x[e].x), ex2m(x[e].y)), sc, mg);
+                aq[e8 + 2 * e] = __float_as_int(y.x) - 0x4B400000;
+                aq[e8 + 2 * e + 1] = __float_as_int(y.y) - 0x4B400000;
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) aq[e8 + e] = 0;
+            }
+          }
+          if (diag) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (tokb + (cq * 32 + e) / G < jrel) aq[e] = 0;
+          }
+          if (is_cur) {
+            // head sum per token (Eq. 4) -> region map; causality already zeroed the invalid entries
+#pragma unroll
+            for (int t = 0; t < 32 / G; ++t) {
+              int sv = 0;
+#pragma unroll
+              for (int hh = 0; hh < G; ++hh) sv += aq[t * G + hh];
+              bsum += sv;
+              const int tk = tokb + (cq * 32) / G + t;
+              if (key_ok && sv != 0 && tk < a.n) atomicAdd(&Mq[(size_t)(tk + roff) * c.chunk + (jrel + roff)], sv);
             }
           } else {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) aq[e8 + e] = 0;
+            for (int e = 0; e < 32; ++e) bsum += aq[e];
           }
         }
-        if (diag) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (tokb + (chalf * 64 + ch * 32 + e) / G < jrel) aq[e] = 0;
-        }
-        if (is_cur) {
-          // head sum per token (Eq. 4) -> region map; causality already zeroed the invalid entries
-#pragma unroll
-          for (int t = 0; t < 32 / G; ++t) {
-            int sv = 0;
-#pragma unroll
-            for (int hh = 0; hh < G; ++hh) sv += aq[t * G + hh];
-            bsum += sv;
-            const int tk = tokb + (chalf * 64 + ch * 32) / G + t;
-            if (key_ok && sv != 0 && tk < a.n) atomicAdd(&Mq[(size_t)(tk + roff) * c.chunk + (jrel + roff)], sv);
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) bsum += aq[e];
-        }
+        total[kt] += bsum;
       }
-      total += bsum;
       if (tid < 128 && more) s_stats[st ^ 1][tid] = nxt;
-      fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_SEMPTY + st));
-      asm volatile("bar.sync 1, 256;" ::: "memory");
+      asm volatile("bar.sync 1, 512;" ::: "memory");
     }
-    if (ok && key_ok && total != 0)
-      atomicAdd((unsigned long long*)&c.votes[unit * c.Tpad + key], (unsigned long long)total);
+    if (ok) {
+#pragma unroll
+      for (int kt = 0; kt < kMapKT; ++kt) {
+        const int key = key0_of(kt) + krel;
+        if (kt < ntile && key < key_end && key >= c.Ls && total[kt] != 0)
+          atomicAdd((unsigned long long*)&c.votes[unit * c.Tpad + key], (unsigned long long)total[kt]);
+      }
+    }
   }
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
-  if (warp == 8) tmem_dealloc(tmem, 256);
+  if (warp == 16) tmem_dealloc(tmem, 512);
   if (tid == 0 && s_abort) set_status(c, -6, 5000 + (int)blockIdx.x);
 }
 
@@ -276,9 +308,10 @@ static cudaError_t launch_map_tc_g(const DevCtx& c, const PrefillArgs& a, const 
   if (e != cudaSuccess) return e;
   const int nloc = (a.loc_begin >= c.Ls) ? (a.t0 - a.loc_begin + 127) / 128 : 0;
   const int ncur = (a.n + 127) / 128;
-  const int smem = 32768 + 65536 + 1024;
+  const int gloc = (nloc + kMapKT - 1) / kMapKT, gcur = (ncur + kMapKT - 1) / kMapKT;
+  const int smem = kMapKT * 32768 + 65536 + 1024;
   cudaFuncSetAttribute(k_map_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  k_map_tc<G><<<dim3(nloc + ncur, c.Hkv, a.layer_count), kMapThreads, smem, s>>>(c, a, nloc, maps);
+  k_map_tc<G><<<dim3(gloc + gcur, c.Hkv, a.layer_count), kMapThreads, smem, s>>>(c, a, gloc, nloc, ncur, maps);
   return cudaGetLastError();
 }
 
