@@ -311,6 +311,59 @@ struct Stream {
     return idx;
   }
 
+  // ---- test hooks (no arithmetic of the method): let a test continue the stream from a given state --------------
+  // append tokens without any processing (O1 only)
+  int append_only(int cnt, const uint16_t* kb, const uint16_t* vb) {
+    if (cnt < 0 || (int64_t)t + cnt > p.max_tokens) return -2;
+    append(cnt, kb, vb);
+    return 0;
+  }
+  // replace the indexed prefix: evicted end, span table and (optionally) index vectors; pending regions are dropped
+  int load_state(int evicted_end, int nspans, const int* start_len, const uint16_t* kr) {
+    if (evicted_end < p.n_sink || evicted_end > t) return -1;
+    spans.clear();
+    int pos = p.n_sink;
+    for (int i = 0; i < nspans; ++i) {
+      if (start_len[2 * i] != pos || start_len[2 * i + 1] < 1) return -1;
+      spans.push_back(Span{start_len[2 * i], start_len[2 * i + 1]});
+      pos += start_len[2 * i + 1];
+    }
+    if (pos != evicted_end) return -1;
+    KR.assign((size_t)nspans * Hkv * d, 0);
+    if (kr) std::memcpy(KR.data(), kr, KR.size() * sizeof(uint16_t));
+    E = evicted_end;
+    pending.clear();
+    return 0;
+  }
+  // append a region that is still inside the window, with its spans (its votes start from zero)
+  int add_pending(int start, int end, int nspans, const int* start_len) {
+    if (start < E || end <= start || end > t) return -1;
+    if (!pending.empty() && pending.back().end != start) return -1;
+    if (pending.empty() && start != E) return -1;
+    Region r;
+    r.start = start;
+    r.end = end;
+    int pos = start;
+    for (int i = 0; i < nspans; ++i) {
+      if (start_len[2 * i] != pos || start_len[2 * i + 1] < 1) return -1;
+      r.spans.push_back(Span{start_len[2 * i], start_len[2 * i + 1]});
+      pos += start_len[2 * i + 1];
+    }
+    if (pos != end) return -1;
+    pending.push_back(r);
+    return 0;
+  }
+  // make the last `cnt` appended tokens the current call (sets t0, n, Q) without running the local pass
+  int begin_call(int cnt, const uint16_t* qb) {
+    if (cnt < 1 || cnt > t) return -1;
+    t0 = t - cnt;
+    n = cnt;
+    m = 0;
+    Q.resize((size_t)n * Hq * d);
+    for (size_t i = 0; i < Q.size(); ++i) Q[i] = bf16_to_f32(qb[i]);
+    return 0;
+  }
+
   // O2
   void evict(int t0_) {
     while (!pending.empty() && pending.front().end <= t0_ - p.window) {
@@ -588,6 +641,16 @@ int orc_decode_retrieve(void* h, const uint16_t* q, const uint16_t* k, const uin
 void orc_decode_attend(void* h, float* out) { ((Stream*)h)->decode_attend(out); }
 void orc_full_attention(void* h, int cnt, const int* pos, const uint16_t* q, float* out) {
   ((Stream*)h)->full_attention(cnt, pos, q, out);
+}
+
+// --- test hooks ---------------------------------------------------------------
+int orc_append_only(void* h, int n, const uint16_t* k, const uint16_t* v) { return ((Stream*)h)->append_only(n, k, v); }
+int orc_load_state(void* h, int evicted_end, int nspans, const int* start_len, const uint16_t* kr) {
+  return ((Stream*)h)->load_state(evicted_end, nspans, start_len, kr);
+}
+int orc_begin_call(void* h, int n, const uint16_t* q) { return ((Stream*)h)->begin_call(n, q); }
+int orc_add_pending(void* h, int start, int end, int nspans, const int* start_len) {
+  return ((Stream*)h)->add_pending(start, end, nspans, start_len);
 }
 
 // --- state access -----------------------------------------------------------

@@ -50,6 +50,10 @@ def lib():
         L.orc_prefill_local.argtypes = [vp, ip, vp, vp, vp]
         L.orc_prefill_retrieve.argtypes = [vp]
         L.orc_prefill_attend.argtypes = [vp, ip, ip, vp]
+        L.orc_append_only.argtypes = [vp, ip, vp, vp]
+        L.orc_load_state.argtypes = [vp, ip, ip, vp, vp]
+        L.orc_begin_call.argtypes = [vp, ip, vp]
+        L.orc_add_pending.argtypes = [vp, ip, ip, ip, vp]
         L.orc_decode_retrieve.argtypes = [vp, vp, vp, vp]
         L.orc_decode_attend.argtypes = [vp, vp]
         L.orc_full_attention.argtypes = [vp, ip, vp, vp, vp]
@@ -143,6 +147,29 @@ class OracleStream:
         self.prefill_local(q, k, v)
         self.prefill_retrieve()
         return self.prefill_attend()
+
+    # --- test hooks: continue a stream from a given state (no method arithmetic) --------
+    def append_only(self, k, v):
+        k, v = _u16(k), _u16(v)
+        if lib().orc_append_only(self._h, k.shape[0], _ptr(k), _ptr(v)):
+            raise RuntimeError("oracle append_only failed")
+
+    def load_state(self, evicted_end, spans, index=None):
+        sp = np.ascontiguousarray(np.asarray(spans, dtype=np.int32).reshape(-1, 2))
+        kr = None if index is None else np.ascontiguousarray(index, dtype=np.uint16)
+        if lib().orc_load_state(self._h, int(evicted_end), len(sp), _ptr(sp), None if kr is None else _ptr(kr)):
+            raise ValueError("inconsistent oracle state")
+
+    def add_pending(self, start, end, spans):
+        sp = np.ascontiguousarray(np.asarray(spans, dtype=np.int32).reshape(-1, 2))
+        if lib().orc_add_pending(self._h, int(start), int(end), len(sp), _ptr(sp)):
+            raise ValueError("inconsistent pending region")
+
+    def begin_call(self, q):
+        q = _u16(q)
+        if lib().orc_begin_call(self._h, q.shape[0], _ptr(q)):
+            raise ValueError("bad call")
+        self._n = q.shape[0]
 
     # --- decode ----------------------------------------------------------
     def decode_retrieve(self, q, k, v):

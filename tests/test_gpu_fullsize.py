@@ -1,0 +1,146 @@
+"""Parity at the benchmark's full size (128K tokens, 32 layers, the launch configuration bench.py times).
+
+The oracle cannot stream 128K x 32 layers, so outputs are sampled: for two layers the oracle is brought to the
+GPU's state at the start of a call (cache contents, span table, index, pending regions) and then computes that
+call itself -- local map, threshold, segmentation, query representatives, scores, top-k, attention rows -- which
+are compared with what the GPU produced for the same call.  A second check rebuilds the votes of one region over
+the nine calls it spends in the window and compares the index vectors it gets at eviction; a third continues into
+decode.  Every upstream quantity the oracle is seeded with is itself covered by one of these samples.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ltri_oracle as orc
+from paper_2412_04757_b200 import binding, inputs
+from tests import parity_harness as ph
+
+pytestmark = pytest.mark.gpu
+LAYERS = [3, 29]
+ROWS = [0, 1, 255, 256, 510, 511]
+
+
+def regions_from_table(spans, lo, hi, chunk):
+    """Split the span table rows covering [lo,hi) into chunk-aligned regions."""
+    out = []
+    for rs in range(lo, hi, chunk):
+        sp = spans[(spans[:, 0] >= rs) & (spans[:, 0] < rs + chunk)]
+        assert sp[0, 0] == rs and sp[-1, 0] + sp[-1, 1] == rs + chunk
+        out.append((rs, rs + chunk, sp))
+    return out
+
+
+def test_cfg2_sampled_calls_match_the_oracle():
+    cfg = inputs.config(2)
+    dev = torch.device("cuda:0")
+    st = inputs.SyntheticStream(cfg, device=dev)
+    lt = binding.Ltri(ph.params_of(cfg), device=dev)
+    L, n, W = cfg.n_layers, cfg.chunk, cfg.window
+    chunks = list(st.prefill_chunks())
+    K = {l: [] for l in LAYERS}
+    V = {l: [] for l in LAYERS}
+    Q = {l: {} for l in LAYERS}
+    probe_call = len(chunks) - 14          # region whose index vectors are rebuilt (evicted 9 calls later)
+    snap = {}
+    out_last = None
+    for ci, (t0, cnt) in enumerate(chunks):
+        q, k, v = st.tokens(t0, cnt)
+        out = lt.ltri_prefill_chunk(0, 0, L, q, k, v)
+        for l in LAYERS:
+            K[l].append(k[l].cpu())
+            V[l].append(v[l].cpu())
+            if ci >= probe_call:
+                Q[l][ci] = q[l].cpu()
+        if ci == len(chunks) - 1:
+            out_last = out
+    torch.cuda.synchronize()
+    assert lt.ltri_sync_status() == 0
+    t0_last = chunks[-1][0]
+    rep = ph.Report()
+    for l in LAYERS:
+        Kall, Vall = torch.cat(K[l]), torch.cat(V[l])
+        spans_g = lt.ltri_get_spans(0, l)
+        idx_g = lt.ltri_debug_read(binding.BUF_INDEX, 0, l)[:, :len(spans_g)].transpose(1, 0, 2).copy()
+        stats = lt.ltri_get_stats(0, l)
+        E = int(stats.evicted_end)
+        assert E == t0_last - W and spans_g[-1, 0] + spans_g[-1, 1] == E
+        pend_g = lt.ltri_get_pending_spans(0, l)
+        what = f"layer {l} last call"
+        # ---- the last prefill call, recomputed by the oracle from the GPU's state at its start -------------
+        o = ph.oracle_of(cfg)
+        o.append_only(Kall[:t0_last], Vall[:t0_last])
+        o.load_state(E, spans_g, idx_g)
+        for (rs, re, sp) in regions_from_table(pend_g, E, t0_last, n):
+            o.add_pending(rs, re, sp)
+        o.prefill_local(Q[l][len(chunks) - 1], Kall[t0_last:], Vall[t0_last:])
+        rs, m = o.region()
+        Mg = np.tril(lt.ltri_debug_read(binding.BUF_MAP, 0, l)[:m, :m])
+        assert np.abs(Mg.astype(np.int64) - o.map()).max() <= 4 + cfg.n_q_heads, f"{what}: region map"
+        thg = int(lt.ltri_debug_read(binding.BUF_THETA, 0, l)[0])
+        assert abs(thg - o.theta_q()) <= 4 + cfg.n_q_heads
+        newest_g = pend_g[pend_g[:, 0] >= rs]
+        ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region)
+        ref_spans[:, 0] += rs
+        assert newest_g.tolist() == ref_spans.tolist(), f"{what}: segmenter on its own map"
+        if newest_g.tolist() != o.pending()[-1][2].tolist():
+            assert o.seg_gap() < ph.NEAR_TIE, f"{what}: spans differ without a near tie"
+            o.set_newest_spans(newest_g)
+            rep.span_flips += 1
+        o.prefill_retrieve()
+        ns = len(spans_g)
+        sg = lt.ltri_debug_read(binding.BUF_SCORES, 0, l)[:, :ns]
+        so = o.scores()
+        assert np.abs(sg - so).max() / np.abs(so).max() <= 2e-5, f"{what}: scores"
+        ph.check_selection(lt.ltri_get_selected(0, l), o, rep, what)
+        for r in ROWS:
+            ref = o.prefill_attend(r, r + 1)
+            ph.check_output(out_last[l, r:r + 1], ref, rep, f"{what} row {r}")
+        snap[l] = o
+        # ---- index vectors of one region: its votes over the nine calls it spends in the window ------------
+        c0 = probe_call
+        t0c = chunks[c0][0]
+        Ec = t0c - W
+        o2 = ph.oracle_of(cfg)
+        o2.append_only(Kall[:t0c], Vall[:t0c])
+        keep = spans_g[:, 0] + spans_g[:, 1] <= Ec
+        o2.load_state(Ec, spans_g[keep], idx_g[keep])
+        for (rs2, re2, sp2) in regions_from_table(np.concatenate([spans_g, pend_g]), Ec, t0c, n):
+            o2.add_pending(rs2, re2, sp2)
+        for ci in range(c0, c0 + W // n + 2):
+            tt = chunks[ci][0]
+            o2.prefill_local(Q[l][ci], Kall[tt:tt + n], Vall[tt:tt + n])
+            if ci == c0:
+                reg_g = spans_g[(spans_g[:, 0] >= t0c) & (spans_g[:, 0] < t0c + n)]
+                if o2.pending()[-1][2].tolist() != reg_g.tolist():
+                    assert o2.seg_gap() < ph.NEAR_TIE, f"layer {l}: probe region spans differ without a near tie"
+                    o2.set_newest_spans(reg_g)
+            if o2.evicted_end >= t0c + n:
+                break
+        assert o2.evicted_end >= t0c + n, "probe region was not evicted"
+        sp2, idx2 = o2.spans(), o2.index()
+        sel_rows = np.where((sp2[:, 0] >= t0c) & (sp2[:, 0] < t0c + n))[0]
+        assert len(sel_rows) > 0
+        for s in sel_rows:
+            gs = np.where(spans_g[:, 0] == sp2[s, 0])[0][0]
+            assert spans_g[gs, 1] == sp2[s, 1]
+            rep.index_rows += 1
+            if not np.array_equal(idx_g[gs], idx2[s]):
+                vo = np.sort(o2.votes(int(sp2[s, 0]), int(sp2[s, 0] + sp2[s, 1])).astype(np.float64))[::-1]
+                assert len(vo) > 1 and (vo[0] - vo[1]) <= ph.NEAR_TIE * max(vo[0], 1.0), \
+                    f"layer {l}: index vector of span {gs} differs"
+                rep.index_flips += 1
+    # ---- decode continues from the same state --------------------------------------------------------------
+    for s in range(3):
+        q, k, v = st.tokens(cfg.context + s, 1, kind=1)
+        qd, kd, vd = (x.permute(1, 0, 2, 3).contiguous() for x in (q, k, v))
+        out = lt.ltri_decode_step([0], 0, L, qd, kd, vd)
+        torch.cuda.synchronize()
+        for l in LAYERS:
+            o = snap[l]
+            o.decode_retrieve(qd[0, l].cpu(), kd[0, l].cpu(), vd[0, l].cpu())
+            ph.check_selection(lt.ltri_get_selected(0, l), o, rep, f"layer {l} decode {s}")
+            ph.check_output(out[0, l], o.decode_attend(), rep, f"layer {l} decode {s}")
+    assert lt.ltri_sync_status() == 0
+    assert rep.span_flips <= 1 and rep.sel_flips <= 4 and rep.index_flips <= 2
+    print(rep)
+    lt.close()

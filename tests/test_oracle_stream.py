@@ -235,6 +235,33 @@ def test_retrieval_finds_the_planted_segment():
     assert tot > 0 and hits / tot > 0.7
 
 
+def test_continuing_from_a_loaded_state_reproduces_the_stream():
+    # the state hooks (used by the full-size GPU checks) must not change what the oracle computes
+    Hq, Hkv, d, chunk, W, Ls, T = 4, 2, 16, 16, 32, 4, 160
+    q, k, v = inputs.random_stream(21, T, Hq, Hkv, d, sharp=2.0)
+    a = make(Hq, Hkv, d, chunk, W, Ls, 3, T, max_spans_per_region=3)
+    outs, states = [], []
+    for t0 in range(0, T, chunk):
+        states.append((a.evicted_end, a.spans().copy(), a.index().copy(), a.pending()))
+        outs.append(a.prefill_chunk(q[t0:t0 + chunk], k[t0:t0 + chunk], v[t0:t0 + chunk]))
+    for c in (5, 8):
+        t0 = c * chunk
+        b = make(Hq, Hkv, d, chunk, W, Ls, 3, T, max_spans_per_region=3)
+        b.append_only(k[:t0], v[:t0])
+        # state at the START of call c is the state after eviction: take it from the original after the call
+        E_after, spans_after, idx_after = states[c + 1][0], states[c + 1][1], states[c + 1][2]
+        b.load_state(E_after, spans_after, idx_after)
+        for (rs, re, sp) in states[c + 1][3][:-1]:          # regions still pending, without call c's own region
+            b.add_pending(rs, re, sp)
+        got = b.prefill_chunk(q[t0:t0 + chunk], k[t0:t0 + chunk], v[t0:t0 + chunk])
+        assert np.array_equal(got, outs[c])
+        assert b.pending()[-1][2].tolist() == a_pending_of(states, c)
+
+
+def a_pending_of(states, c):
+    return states[c + 1][3][-1][2].tolist()
+
+
 def test_state_errors():
     q, k, v = inputs.random_stream(9, 40, 4, 2, 16)
     o = make(T=40)
