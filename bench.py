@@ -257,37 +257,49 @@ def run_ltri(args, cfg):
     L, n = cfg.n_layers, cfg.chunk
     chunks = list(inputs.prefill_calls(cfg))
     K, W = args.steps, args.warmup
-    if K + W > len(chunks):
-        raise SystemExit(f"steps+warmup = {K + W} exceeds the {len(chunks)} prefill calls of {cfg.name}")
+    if K + W > len(chunks):   # tiny workloads: fewer calls exist than were asked for
+        W = min(W, max(0, len(chunks) // 2 - 1))
+        K = len(chunks) - W
     first_timed = len(chunks) - K
     first_warm = first_timed - W
 
-    st = inputs.SyntheticStream(cfg, seq=rank, device=dev)
+    NSEQ = cfg.n_seqs
+    streams = [inputs.SyntheticStream(cfg, seq=rank * NSEQ + s, device=dev) for s in range(NSEQ)]
+    st = streams[-1]        # the timed prefill steps run on the last sequence; the others are streamed as set-up
+    SQ = NSEQ - 1
     p = binding.make_params(L, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_tokens, cfg.chunk, cfg.window, cfg.n_sink,
-                            cfg.top_k, head_dim=cfg.head_dim, max_seqs=1, reps_per_span=cfg.reps_per_span,
+                            cfg.top_k, head_dim=cfg.head_dim, max_seqs=NSEQ, reps_per_span=cfg.reps_per_span,
                             max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta)
 
     def stream_until(lt, upto, keep_from):
+        for s in range(NSEQ - 1):
+            for (t0, cnt) in chunks:
+                q, k, v = streams[s].tokens(t0, cnt)
+                lt.ltri_prefill_chunk(s, 0, L, q, k, v)
         kept = []
         for ci, (t0, cnt) in enumerate(chunks[:upto]):
             q, k, v = st.tokens(t0, cnt)
             if ci >= keep_from:
                 kept.append((q, k, v))
             else:
-                lt.ltri_prefill_chunk(0, 0, L, q, k, v)
+                lt.ltri_prefill_chunk(SQ, 0, L, q, k, v)
         return kept
 
     lt = binding.Ltri(p, device=dev)
     # set-up: stream everything before the warm-up chunks, generate (and keep) warm-up + timed inputs
     kept = stream_until(lt, len(chunks), first_warm)
     outs = [torch.empty_like(kept[0][0]) for _ in range(2)]
-    dec_in = [tuple(x.permute(1, 0, 2, 3).contiguous() for x in st.tokens(cfg.context + s, 1, kind=1))
-              for s in range(cfg.decode_steps)]
+    def decode_inputs(step):
+        parts = [sx.tokens(cfg.context + step, 1, kind=1) for sx in streams]
+        return tuple(torch.cat([pp[i].permute(1, 0, 2, 3) for pp in parts]).contiguous() for i in range(3))
+
+    dec_in = [decode_inputs(s) for s in range(cfg.decode_steps)]
+    seq_ids = list(range(NSEQ))
     torch.cuda.synchronize(dev)
 
     # ---- device-resident timing ------------------------------------------------------------
     for i in range(W):
-        lt.ltri_prefill_chunk(0, 0, L, *kept[i], out=outs[i & 1])
+        lt.ltri_prefill_chunk(SQ, 0, L, *kept[i], out=outs[i & 1])
     torch.cuda.synchronize(dev)
     lt.ltri_profile_read()                      # clears counters
     lt.ltri_profile_enable(True)
@@ -300,7 +312,7 @@ def run_ltri(args, cfg):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(K):
-        lt.ltri_prefill_chunk(0, 0, L, *kept[W + i], out=outs[i & 1])
+        lt.ltri_prefill_chunk(SQ, 0, L, *kept[W + i], out=outs[i & 1])
     e1.record()
     torch.cuda.synchronize(dev)
     clk_hi = sampler.mark()
@@ -310,7 +322,7 @@ def run_ltri(args, cfg):
     prof = lt.ltri_profile_read()
     lt.ltri_profile_enable(False)
     assert lt.ltri_sync_status() == 0, "device-side status word reports an error"
-    stats = lt.ltri_get_stats(0, 0)
+    stats = lt.ltri_get_stats(SQ, 0)
     ms = max_over_ranks(ms, world, dev)
     tokens = K * n
     prefill_tps = sum_over_ranks(tokens / (ms * 1e-3), world, dev) if world > 1 else tokens / (ms * 1e-3)
@@ -321,7 +333,7 @@ def run_ltri(args, cfg):
         dout = torch.empty_like(dec_in[0][0])
         dw = min(3, cfg.decode_steps // 2)
         for s in range(dw):
-            lt.ltri_decode_step([0], 0, L, *dec_in[s], out=dout)
+            lt.ltri_decode_step(seq_ids, 0, L, *dec_in[s], out=dout)
         torch.cuda.synchronize(dev)
         lt.ltri_profile_read()
         lt.ltri_profile_enable(True)
@@ -329,20 +341,22 @@ def run_ltri(args, cfg):
         barrier(world)
         d0.record()
         for s in range(dw, cfg.decode_steps):
-            lt.ltri_decode_step([0], 0, L, *dec_in[s], out=dout)
+            lt.ltri_decode_step(seq_ids, 0, L, *dec_in[s], out=dout)
         d1.record()
         torch.cuda.synchronize(dev)
         dms = max_over_ranks(d0.elapsed_time(d1), world, dev)
         dprof = lt.ltri_profile_read()
         lt.ltri_profile_enable(False)
         dsteps = cfg.decode_steps - dw
-        dst = lt.ltri_get_stats(0, 0)
+        dst = lt.ltri_get_stats(SQ, 0)
         ret_tok = dst.retrieved_tokens / cfg.n_kv_heads
         keys = cfg.n_sink + ret_tok + (dst.tokens - dst.evicted_end)
         # algorithmic bytes per step: index scan + K and V rows once per KV head
-        bytes_step = L * (cfg.n_kv_heads * dst.n_spans * cfg.head_dim * 2 + 2 * cfg.n_kv_heads * cfg.head_dim * 2 * keys)
+        bytes_step = NSEQ * L * (cfg.n_kv_heads * dst.n_spans * cfg.head_dim * 2 +
+                                 2 * cfg.n_kv_heads * cfg.head_dim * 2 * keys)
         k_ms = dprof["decode_retrieve"][0] + dprof["decode_attn"][0]
-        dec = {"value": world * dsteps / (dms * 1e-3), "unit": "tok/s", "steps": dsteps, "ms_per_step": dms / dsteps,
+        dec = {"value": world * NSEQ * dsteps / (dms * 1e-3), "unit": "tok/s", "steps": dsteps, "sequences": NSEQ,
+               "ms_per_step": dms / dsteps,
                "keys_per_head": keys, "index_spans": dst.n_spans,
                "roofline": {"bound": "hbm", "achieved": bytes_step * dsteps / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -371,7 +385,7 @@ def run_ltri(args, cfg):
             dq.copy_(host[i][0], non_blocking=True)
             dk.copy_(host[i][1], non_blocking=True)
             dv.copy_(host[i][2], non_blocking=True)
-            lt.ltri_prefill_chunk(0, 0, L, dq, dk, dv, out=outs[0])
+            lt.ltri_prefill_chunk(SQ, 0, L, dq, dk, dv, out=outs[0])
             hout.copy_(outs[0], non_blocking=True)
 
         for i in range(W):
@@ -414,7 +428,7 @@ def run_ltri(args, cfg):
                    "context": cfg.context, "chunk": cfg.chunk, "window": cfg.window, "sink": cfg.n_sink,
                    "top_k": cfg.top_k, "timed_positions": [chunks[first_timed][0], cfg.context],
                    "l2": "inputs of every step are distinct and larger than L2 (no flush needed)",
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "parallelism": "replicas only" if world > 1 else "single GPU", "sequences": NSEQ,
                    "index_spans": stats.n_spans, "retrieved_tokens_per_kv_head": stats.retrieved_tokens / cfg.n_kv_heads},
         "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "decode": dec, "roofline": roof, "cpu_baseline": cpu,
         "kernel_ms_per_step": {k: v[0] / K for k, v in prof.items() if v[1]},

@@ -77,9 +77,10 @@ __global__ void __launch_bounds__(128) k_score_mma(DevCtx c, int seq, int layer_
       float S[8][4];
 #pragma unroll
       for (int i = 0; i < 8; ++i) S[i][0] = S[i][1] = S[i][2] = S[i][3] = 0.f;
+      const int npairs = min(4, (J - jb * 64 + 15) >> 4);  // only the column tiles that hold query spans
 #pragma unroll 1
       for (int t = 2; t >= 0; --t)  // smallest term first
-        warp_qk_16x64(S, sA + stage * 16384, warp * 16, sU + (jb * 3 + t) * 16384, lane);
+        warp_qk_16xN(S, sA + stage * 16384, warp * 16, sU + (jb * 3 + t) * 16384, lane, npairs);
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
@@ -109,7 +110,9 @@ cudaError_t launch_score_prefill_mma(const DevCtx& c, const PrefillArgs& a, int 
   const int smem = njb_max * 3 * 16384 + 2 * 16384;
   cudaFuncSetAttribute(k_score_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   const int tiles = (span_bound + 63) / 64;
-  const int gx = max(1, (tiles + 3) / 4);
+  // enough tiles per CTA to amortise the split of the representatives, enough CTAs to fill the GPU
+  const int per_cta = tiles >= 512 ? 32 : 16;
+  const int gx = max(1, (tiles + per_cta - 1) / per_cta);
   k_score_mma<<<dim3(gx, c.Hkv, a.layer_count), 128, smem, s>>>(c, a.seq, a.layer_begin);
   return cudaGetLastError();
 }

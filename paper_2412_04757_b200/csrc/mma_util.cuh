@@ -69,4 +69,23 @@ __device__ __forceinline__ void warp_qk_16x64(float (&S)[8][4], uint32_t a_tile,
   }
 }
 
+// Same as warp_qk_16x64 but only the first `npairs` pairs of 8-column tiles (16 columns each) are computed.
+__device__ __forceinline__ void warp_qk_16xN(float (&S)[8][4], uint32_t a_tile, int a_row0, uint32_t b_tile, int lane,
+                                             int npairs) {
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    uint32_t a[4];
+    ldsm_x4(a, a_tile + tile_off(a_row0 + (lane & 15), ks * 2 + (lane >> 4)));
+#pragma unroll
+    for (int np = 0; np < 4; ++np) {
+      if (np < npairs) {
+        uint32_t b[4];
+        ldsm_x4(b, b_tile + tile_off(np * 16 + (lane & 7) + ((lane >> 4) << 3), ks * 2 + ((lane >> 3) & 1)));
+        mma_bf16(S[2 * np], a, b[0], b[1]);
+        mma_bf16(S[2 * np + 1], a, b[2], b[3]);
+      }
+    }
+  }
+}
+
 }  // namespace ltri
