@@ -138,93 +138,136 @@ cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_co
 
 // ------------------------------------------------------------------------------------------
 // a3 segmenter, step 1: exact rank selection of theta (quantile mode) over the causal entries of Mq.
-// A sparse map is mostly zeros, so zeros (and negatives, which only hand-built maps can contain) are counted first;
-// only when the rank falls among the positive entries does an MSB radix select run over them, 8 bits per pass from
-// the highest set bit of the maximum, with one private histogram per warp.  One CTA per layer.
+// Pass 1 counts negatives (only hand-built maps have any) and zeros (a sparse map is mostly zeros) and builds a
+// log-scale histogram of the positive entries: bin = (position of the leading one, next four bits), which is monotone
+// in the value and spreads a heavy-tailed map over many bins.  If the rank falls among the positives, the remaining
+// low bits of the selected bin are resolved by MSB radix passes of 9 bits.  One private histogram per warp, four loads
+// in flight per lane, one CTA per layer.
+constexpr int kThetaBits = 9;
+constexpr int kThetaBins = 1 << kThetaBits;
+
+// visits the causal entries of the m x m map: f(value) for every (i, j <= i); a warp owns rows warp, warp+32, ...
+template <typename F>
+__device__ __forceinline__ void for_each_causal(const int* __restrict__ Mq, int ld, int m, F&& f) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  for (int i = warp; i < m; i += nwarps) {
+    const int* row = Mq + (size_t)i * ld;
+    for (int j0 = 0; j0 <= i; j0 += 128) {
+      int v[4];
+      bool ok[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = j0 + u * 32 + lane;
+        ok[u] = j <= i;
+        v[u] = ok[u] ? row[j] : 0;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (ok[u]) f(v[u]);
+    }
+  }
+}
+
+// monotone log-scale bin of a positive value: 16 bins per power of two
+__device__ __forceinline__ unsigned log_bin(unsigned v) {
+  const int e = 31 - __clz(v);
+  const unsigned frac = e >= 4 ? (v >> (e - 4)) & 15u : (v << (4 - e)) & 15u;
+  return ((unsigned)e << 4) | frac;
+}
+
 __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin, int m, long long rank) {
+  extern __shared__ unsigned hist[];  // [32 warps][kThetaBins]
   const int layer = layer_begin + blockIdx.x;
   const int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
-  __shared__ unsigned hist[32][256];
-  __shared__ unsigned tot[256];
-  __shared__ unsigned s_red[32][3];
-  __shared__ unsigned s_prefix, s_maxkey;
+  __shared__ unsigned tot[kThetaBins];
+  __shared__ unsigned s_red[32][2];
+  __shared__ unsigned s_prefix, s_lo_bits;
   __shared__ long long s_rank;
-  __shared__ int s_cls;  // 0: answer is 0, 1: among positives, -1: among negatives
+  __shared__ int s_cls;  // 0: answer found, 1: among positives (bin chosen), -1: among negatives
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // class counts and maxima
-  unsigned nneg = 0, nzero = 0, maxpos = 0, maxneg = 0;
-  for (int i = warp; i < m; i += 32)
-    for (int j = lane; j <= i; j += 32) {
-      const int v = Mq[(size_t)i * c.chunk + j];
-      if (v > 0)
-        maxpos = max(maxpos, (unsigned)v);
-      else if (v == 0)
-        ++nzero;
-      else {
-        ++nneg;
-        maxneg = max(maxneg, (unsigned)v ^ 0x80000000u);
-      }
-    }
+  unsigned* myhist = hist + warp * kThetaBins;
+  for (int t = threadIdx.x; t < 32 * kThetaBins; t += blockDim.x) hist[t] = 0;
+  __syncthreads();
+  unsigned nneg = 0, nzero = 0;
+  for_each_causal(Mq, c.chunk, m, [&](int v) {
+    if (v > 0)
+      atomicAdd(&myhist[log_bin((unsigned)v)], 1u);
+    else if (v == 0)
+      ++nzero;
+    else
+      ++nneg;
+  });
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     nneg += __shfl_xor_sync(0xffffffffu, nneg, o);
     nzero += __shfl_xor_sync(0xffffffffu, nzero, o);
-    maxpos = max(maxpos, __shfl_xor_sync(0xffffffffu, maxpos, o));
-    maxneg = max(maxneg, __shfl_xor_sync(0xffffffffu, maxneg, o));
   }
   if (lane == 0) {
     s_red[warp][0] = nneg;
     s_red[warp][1] = nzero;
-    s_red[warp][2] = maxpos;
-    tot[warp] = maxneg;
+  }
+  __syncthreads();
+  if (threadIdx.x < kThetaBins) {
+    unsigned sum = 0;
+    for (int w = 0; w < 32; ++w) sum += hist[w * kThetaBins + threadIdx.x];
+    tot[threadIdx.x] = sum;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     long long cn = 0, cz = 0;
-    unsigned mp = 0, mn = 0;
     for (int w = 0; w < 32; ++w) {
       cn += s_red[w][0];
       cz += s_red[w][1];
-      mp = max(mp, s_red[w][2]);
-      mn = max(mn, tot[w]);
     }
     if (rank < cn) {
       s_cls = -1;
       s_rank = rank;
-      s_maxkey = mn;
     } else if (rank < cn + cz) {
       s_cls = 0;
+      c.thetaq[layer] = 0;
     } else {
-      s_cls = 1;
-      s_rank = rank - cn - cz;
-      s_maxkey = mp;
+      long long r = rank - cn - cz;
+      unsigned b = 0;
+      for (; b < kThetaBins - 1; ++b) {
+        if (r < (long long)tot[b]) break;
+        r -= tot[b];
+      }
+      const int e = (int)(b >> 4);
+      const unsigned frac = b & 15u;
+      s_rank = r;
+      if (e <= 4) {  // the bin holds a single value
+        s_cls = 0;
+        c.thetaq[layer] = (long long)((1u << e) | (frac >> (4 - e)));
+      } else {
+        s_cls = 1;
+        s_prefix = (1u << e) | (frac << (e - 4));  // leading one and the next four bits
+        s_lo_bits = (unsigned)(e - 4);             // bits still unknown
+      }
     }
-    s_prefix = 0;
   }
   __syncthreads();
   const int cls = s_cls;
-  if (cls == 0) {
-    if (threadIdx.x == 0) c.thetaq[layer] = 0;
-    return;
-  }
-  int hi = 32 - __clz(s_maxkey | 1u);  // bits [0,hi) can be set
+  if (cls == 0) return;
+  // remaining bits: [0, hi).  Negatives: plain MSB radix over the sign-flipped key.
+  int hi = cls > 0 ? (int)s_lo_bits : 31;
+  const int top = hi;  // entries take part when their bits above `top` equal the prefix's
+  if (cls < 0 && threadIdx.x == 0) s_prefix = 0;
+  __syncthreads();
   while (hi > 0) {
-    const int lo = max(0, hi - 8);
+    const int lo = max(0, hi - kThetaBits);
     const unsigned dmask = (1u << (hi - lo)) - 1u;
-    for (int t = threadIdx.x; t < 32 * 256; t += blockDim.x) (&hist[0][0])[t] = 0;
+    for (int t = threadIdx.x; t < 32 * kThetaBins; t += blockDim.x) hist[t] = 0;
     __syncthreads();
     const unsigned prefix = s_prefix;
-    for (int i = warp; i < m; i += 32)
-      for (int j = lane; j <= i; j += 32) {
-        const int v = Mq[(size_t)i * c.chunk + j];
-        const bool in_cls = cls > 0 ? v > 0 : v < 0;
-        const unsigned key = cls > 0 ? (unsigned)v : ((unsigned)v ^ 0x80000000u);
-        if (in_cls && (hi >= 32 || (key >> hi) == (prefix >> hi))) atomicAdd(&hist[warp][(key >> lo) & dmask], 1u);
-      }
+    for_each_causal(Mq, c.chunk, m, [&](int v) {
+      const bool in_cls = cls > 0 ? v > 0 : v < 0;
+      const unsigned key = cls > 0 ? (unsigned)v : ((unsigned)v ^ 0x80000000u);
+      if (in_cls && (key >> hi) == (prefix >> hi)) atomicAdd(&myhist[(key >> lo) & dmask], 1u);
+    });
     __syncthreads();
-    if (threadIdx.x < 256) {
+    if (threadIdx.x < kThetaBins) {
       unsigned sum = 0;
-      for (int w = 0; w < 32; ++w) sum += hist[w][threadIdx.x];
+      for (int w = 0; w < 32; ++w) sum += hist[w * kThetaBins + threadIdx.x];
       tot[threadIdx.x] = sum;
     }
     __syncthreads();
@@ -242,6 +285,7 @@ __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin
     __syncthreads();
     hi = lo;
   }
+  (void)top;
   if (threadIdx.x == 0)
     c.thetaq[layer] = cls > 0 ? (long long)s_prefix : (long long)(int)(s_prefix ^ 0x80000000u);
 }
@@ -489,7 +533,9 @@ cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_
     long long rank = (long long)floor((double)theta * (double)(N - 1));
     if (rank < 0) rank = 0;
     if (rank > N - 1) rank = N - 1;
-    k_theta_select<<<layer_count, 1024, 0, s>>>(c, layer_begin, m, rank);
+    const int hsmem = 32 * kThetaBins * (int)sizeof(unsigned);
+    cudaFuncSetAttribute(k_theta_select, cudaFuncAttributeMaxDynamicSharedMemorySize, hsmem);
+    k_theta_select<<<layer_count, 1024, hsmem, s>>>(c, layer_begin, m, rank);
   } else {
     k_theta_set<<<layer_count, 1, 0, s>>>(c, layer_begin, theta_q_abs);
   }
