@@ -8,6 +8,8 @@
 
 namespace ltri {
 
+constexpr int kScoreStages = 4;
+
 // grid (tile groups, Hkv, layers), 128 threads (4 warps x 16 spans)
 __global__ void __launch_bounds__(128) k_score_mma(DevCtx c, int seq, int layer_begin) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -21,7 +23,7 @@ __global__ void __launch_bounds__(128) k_score_mma(DevCtx c, int seq, int layer_
   if ((int)blockIdx.x >= ntiles) return;
   const int njb = (J + 63) / 64;                      // blocks of 64 query spans
   const uint32_t sU = smem_u32(smem);                 // [njb][3 terms][64 rows][128] bf16 = njb * 48 KB
-  const uint32_t sA = sU + njb * 3 * 16384;           // 2 stages x 16 KB of index rows
+  const uint32_t sA = sU + njb * 3 * 16384;           // kScoreStages x 16 KB of index rows
   // split the representatives
   const float* up = c.u + ((size_t)layer * c.Hkv + g) * c.Jmax * kD;
   for (int i = tid; i < njb * 64 * 16; i += 128) {
@@ -59,18 +61,20 @@ __global__ void __launch_bounds__(128) k_score_mma(DevCtx c, int seq, int layer_
   auto issue = [&](int stage, int tile) {
     load_tile_async(sA + stage * 16384, KR + (size_t)tile * 64 * kD, kD, 64, min(64, N - tile * 64), tid, 128);
   };
-  int tile = blockIdx.x;
-  issue(0, tile);
-  cp_async_commit();
-  int stage = 0;
-  for (; tile < ntiles; tile += gridDim.x, stage ^= 1) {
-    const int nxt = tile + gridDim.x;
-    if (nxt < ntiles) issue(stage ^ 1, nxt);
+  // kScoreStages-deep cp.async ring over this CTA's tiles blockIdx.x, blockIdx.x + gridDim.x, ...
+  const int my_tiles = (ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+#pragma unroll
+  for (int s = 0; s < kScoreStages - 1; ++s) {
+    if (s < my_tiles) issue(s, blockIdx.x + s * gridDim.x);
     cp_async_commit();
-    if (nxt < ntiles)
-      cp_async_wait<1>();
-    else
-      cp_async_wait<0>();
+  }
+  for (int it = 0; it < my_tiles; ++it) {
+    const int stage = it % kScoreStages;
+    const int tile = blockIdx.x + it * gridDim.x;
+    if (it + kScoreStages - 1 < my_tiles)
+      issue((it + kScoreStages - 1) % kScoreStages, blockIdx.x + (it + kScoreStages - 1) * gridDim.x);
+    cp_async_commit();
+    cp_async_wait<kScoreStages - 1>();
     __syncthreads();
     float best0 = -INFINITY, best1 = -INFINITY;
     for (int jb = 0; jb < njb; ++jb) {
@@ -107,7 +111,7 @@ __global__ void __launch_bounds__(128) k_score_mma(DevCtx c, int seq, int layer_
 
 cudaError_t launch_score_prefill_mma(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s) {
   const int njb_max = (c.Jmax + 63) / 64;
-  const int smem = njb_max * 3 * 16384 + 2 * 16384;
+  const int smem = njb_max * 3 * 16384 + kScoreStages * 16384;
   cudaFuncSetAttribute(k_score_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   const int tiles = (span_bound + 63) / 64;
   // enough tiles per CTA to amortise the split of the representatives, enough CTAs to fill the GPU
