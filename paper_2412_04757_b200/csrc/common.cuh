@@ -116,12 +116,16 @@ cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_beg
 // phase 1: continues from the stored state over the selected spans and writes the output.
 cudaError_t launch_attn_prefill(const DevCtx& c, const PrefillArgs& a, int phase, bool final, cudaStream_t s);
 // tcgen05/TMEM/TMA version of launch_attn_prefill (same contract) and its availability check
-constexpr int kTcMapBytes = 5 * 128;  // host storage for a context's K/V tensor maps
+constexpr int kTcMapBytes = 6 * 128;  // host storage for a context's tensor maps: five K/V box heights + the index
 cudaError_t launch_attn_prefill_tc(const DevCtx& c, const PrefillArgs& a, int phase, bool final, const void* kv_maps,
                                    cudaStream_t s);
 bool tc_attention_supported(const DevCtx& c);
 bool tc_encode_kv_maps(const DevCtx& c, void* out_bytes);
 cudaError_t launch_map_pass_tc(const DevCtx& c, const PrefillArgs& a, const void* kv_maps, cudaStream_t s);
+// tcgen05 version of the prefill scores; returns cudaErrorNotSupported when the query-span count does not fit
+cudaError_t launch_score_prefill_tc(const DevCtx& c, const PrefillArgs& a, int span_bound, const void* kv_maps,
+                                    cudaStream_t s);
+bool score_tc_supported(const DevCtx& c);
 cudaError_t launch_map_pass(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
 
 cudaError_t launch_decode_attn(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,

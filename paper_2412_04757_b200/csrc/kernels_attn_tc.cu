@@ -33,7 +33,7 @@ struct TcMaps {
   CUtensorMap q;             // [tokens][Hq][128] bf16, box {64, G, 256/G}
   CUtensorMap kv[kNumBoxes]; // K slabs followed by V slabs: [rows][128] bf16, box {64, 8<<i}
 };
-static_assert(sizeof(CUtensorMap) * kNumBoxes <= kTcMapBytes, "kTcMapBytes too small");
+static_assert(sizeof(CUtensorMap) * (kNumBoxes + 1) <= kTcMapBytes, "kTcMapBytes too small");
 
 struct RangeList {
   int n;
@@ -627,6 +627,17 @@ bool tc_encode_kv_maps(const DevCtx& c, void* out_bytes) {
     cuuint32_t es[2] = {1, 1};
     if (enc(&out[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c.Kc, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  // sixth map: the span index K^R, [rows][128] bf16 in 128-row boxes
+  {
+    cuuint64_t dims[2] = {128, (cuuint64_t)c.NS * c.NL * c.Hkv * (cuuint64_t)c.cap};
+    cuuint64_t strides[1] = {256};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t es[2] = {1, 1};
+    if (enc(&out[kNumBoxes], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c.KR, dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
   }

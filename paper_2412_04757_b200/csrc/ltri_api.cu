@@ -347,7 +347,12 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   if (has_index) {
     {
       Scope sc(ctx, st, LTRI_K_SCORE_TOPK, 2);
-      LTRI_CUDA(ctx, ctx->use_tc ? launch_score_prefill_mma(d, a, (int)ub, st) : launch_score_prefill(d, a, (int)ub, st));
+      if (ctx->use_tc && score_tc_supported(d))
+        LTRI_CUDA(ctx, launch_score_prefill_tc(d, a, (int)ub, ctx->kv_maps, st));
+      else if (ctx->use_tc)
+        LTRI_CUDA(ctx, launch_score_prefill_mma(d, a, (int)ub, st));
+      else
+        LTRI_CUDA(ctx, launch_score_prefill(d, a, (int)ub, st));
       LTRI_CUDA(ctx, launch_topk_prefill(d, a, st));
     }
     Scope sc(ctx, st, LTRI_K_ATTN_RET, 1);
