@@ -49,6 +49,10 @@ struct DevCtx {
                          //                   log2 of its Q20 probability (see kernels_map_tc.cu)
   float* Oacc;           // [NL][chunk][Hq][128]  unnormalised accumulator of the local part
   float* u;              // [NL][Hkv][Jmax][128]  summed query representatives
+  __nv_bfloat16* Kg;     // [NL][Hkv][Rcap][128]  keys of the spans selected for the call in flight, packed
+  __nv_bfloat16* Vg;     //                       (directly behind Kg) their values
+  int* gcnt;             // [NL][Hkv]             packed rows (retrieved tokens) per KV head
+  long long Rcap;        // row capacity of a packed slab: top_k spans of at most `chunk` tokens, rounded up
   int* Jcnt;             // [NL]
   // per-(seq,layer) scratch
   float* scores;         // [NS*NL][Hkv][cap]
@@ -116,7 +120,8 @@ cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_beg
 // phase 1: continues from the stored state over the selected spans and writes the output.
 cudaError_t launch_attn_prefill(const DevCtx& c, const PrefillArgs& a, int phase, bool final, cudaStream_t s);
 // tcgen05/TMEM/TMA version of launch_attn_prefill (same contract) and its availability check
-constexpr int kTcMapBytes = 6 * 128;  // host storage for a context's tensor maps: five K/V box heights + the index
+// host storage for a context's tensor maps: five box heights of the K/V cache, the index, five of the packed slabs
+constexpr int kTcMapBytes = 11 * 128;
 cudaError_t launch_attn_prefill_tc(const DevCtx& c, const PrefillArgs& a, int phase, bool final, const void* kv_maps,
                                    cudaStream_t s);
 bool tc_attention_supported(const DevCtx& c);

@@ -33,7 +33,7 @@ struct TcMaps {
   CUtensorMap q;             // [tokens][Hq][128] bf16, box {64, G, 256/G}
   CUtensorMap kv[kNumBoxes]; // K slabs followed by V slabs: [rows][128] bf16, box {64, 8<<i}
 };
-static_assert(sizeof(CUtensorMap) * (kNumBoxes + 1) <= kTcMapBytes, "kTcMapBytes too small");
+static_assert(sizeof(CUtensorMap) * (2 * kNumBoxes + 1) <= kTcMapBytes, "kTcMapBytes too small");
 
 struct RangeList {
   int n;
@@ -202,7 +202,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     w.layer = a.layer_begin + w.l;
     w.tok0 = w.mb * TOKB;
     w.unit = unit_of(c, a.seq, w.layer);
-    w.slab_row0 = (w.unit * c.Hkv + w.g) * (size_t)c.Tpad;
+    // phase 0 reads the K/V cache of the (sequence, layer, KV head); phase 1 the packed slab of the selected spans
+    w.slab_row0 = phase == 0 ? (w.unit * c.Hkv + w.g) * (size_t)c.Tpad
+                             : ((size_t)w.layer * c.Hkv + w.g) * (size_t)c.Rcap;
     return w;
   };
 
@@ -234,13 +236,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           rg.start[2] = a.t0;
           rg.len[2] = last_tok + 1;
         } else {
-          const size_t rb = (w.unit * c.Hkv + w.g) * (size_t)(c.topk + 2);
-          const int nr = min(c.rng_cnt[w.unit * c.Hkv + w.g], c.topk + 2);
-          rg.n = nr;
-          for (int i = 0; i < nr; ++i) {
-            rg.start[i] = c.rng_start[rb + i];
-            rg.len[i] = c.rng_len[rb + i];
-          }
+          rg.n = 1;
+          rg.start[0] = 0;
+          rg.len[0] = c.gcnt[(size_t)w.layer * c.Hkv + w.g];
         }
         // publish the ranges with a monotonic counter: a softmax thread may look for item wi only after the Q tile
         // of item wi+1 has arrived, so a parity barrier could not tell the two apart
@@ -630,6 +628,17 @@ bool tc_encode_kv_maps(const DevCtx& c, void* out_bytes) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
   }
+  // maps 6..10: the packed slabs of the selected spans (K slabs then V slabs), same box heights
+  for (int i = 0; i < kNumBoxes; ++i) {
+    cuuint64_t dims[2] = {128, (cuuint64_t)c.NL * c.Hkv * (cuuint64_t)c.Rcap * 2};
+    cuuint64_t strides[1] = {256};
+    cuuint32_t box[2] = {64, (cuuint32_t)(8 << i)};
+    cuuint32_t es[2] = {1, 1};
+    if (enc(&out[kNumBoxes + 1 + i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c.Kg, dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
   // sixth map: the span index K^R, [rows][128] bf16 in 128-row boxes
   {
     cuuint64_t dims[2] = {128, (cuuint64_t)c.NS * c.NL * c.Hkv * (cuuint64_t)c.cap};
@@ -649,6 +658,8 @@ bool tc_attention_supported(const DevCtx& c) {
   const size_t rows = (size_t)c.NS * c.NL * c.Hkv * (size_t)c.Tpad;
   if (c.Vc != c.Kc + rows * kD) return false;
   if (rows * 2 >= (1ull << 31)) return false;
+  const size_t grows = (size_t)c.NL * c.Hkv * (size_t)c.Rcap;
+  if (c.Vg != c.Kg + grows * kD || grows * 2 >= (1ull << 31)) return false;
   return get_encode() != nullptr;
 }
 
@@ -658,7 +669,7 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase,
   TcMaps maps;
   EncodeFn enc = get_encode();
   if (!enc || !kv_maps) return cudaErrorNotSupported;
-  memcpy(maps.kv, kv_maps, sizeof(maps.kv));
+  memcpy(maps.kv, static_cast<const CUtensorMap*>(kv_maps) + (phase == 0 ? 0 : kNumBoxes + 1), sizeof(maps.kv));
   {
     cuuint64_t dims[3] = {128, (cuuint64_t)c.Hq, (cuuint64_t)a.layer_count * a.n};
     cuuint64_t strides[2] = {256, (cuuint64_t)c.Hq * 256};
@@ -672,7 +683,7 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase,
   constexpr int TOKB = 256 / G;
   const int smem = 65536 + 131072 + 1024;
   cudaFuncSetAttribute(k_attn_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  const long long v_off = (long long)c.NS * c.NL * c.Hkv * c.Tpad;
+  const long long v_off = phase == 0 ? (long long)c.NS * c.NL * c.Hkv * c.Tpad : (long long)c.NL * c.Hkv * c.Rcap;
   static int sms = 0;
   if (sms == 0) {
     int dev = 0;

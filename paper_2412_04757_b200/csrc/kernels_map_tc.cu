@@ -2,12 +2,13 @@
 // local | current keys and turn them into Q20 fixed-point probabilities (reading of Eq. 1-3), accumulating the votes of
 // Eq. 6 (column sums over all rows and heads) and the head-summed region map of Eq. 4.
 //
-// The product is computed transposed, S^T = K Q^T: a CTA keeps one 128-key tile in shared memory and streams all query
-// rows of its KV group through it in 128-row blocks (row = (token, head)).  With keys on the TMEM lanes every epilogue
-// thread owns one key, so a column sum of the map is a thread-local sum and needs no shuffles; the G heads of a token
-// are adjacent columns, so their sum (Eq. 4) is thread-local too and goes to the region map with one integer reduction
-// per (token, key, KV head).  Roles: warps 0-7 epilogue (two warps per lane quarter, 64 columns each), warp 8 TMA
-// producer, warp 9 MMA issuer; two TMEM accumulators and two Q stages overlap the MMAs with the exp/round epilogue.
+// The product is computed transposed, S^T = K Q^T: a CTA keeps up to four 128-key tiles in shared memory and streams
+// all query rows of its KV group through them in 128-row blocks (row = (token, head)).  With keys on the TMEM lanes
+// every epilogue thread owns one key, so a column sum of the map is a thread-local sum and needs no shuffles; the G
+// heads of a token are adjacent columns, so their sum (Eq. 4) is thread-local too and goes to the region map with one
+// integer reduction per (token, key, KV head).  Roles: warps 0-15 epilogue (four warps per lane quarter, 32 columns
+// each), warp 16 TMA producer, warp 17 MMA issuer; four TMEM accumulators and two Q stages overlap the MMAs with the
+// exp/round epilogue, which is bound by the special-function unit (one ex2 per map entry).
 #include <cuda.h>
 
 #include <cstring>
@@ -55,7 +56,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
   __shared__ __align__(8) unsigned long long bars[1 + 4 + 8];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ __align__(16) float s_stats[2][128];
+  __shared__ __align__(16) float s_stats[16][2][32];  // per epilogue warp: offsets of its 32 columns, two blocks
   constexpr int TPB = 128 / G;  // tokens per query block
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
@@ -158,108 +159,135 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     const float* rq = c.rowq + (size_t)layer * c.chunk * c.Hq + g * G;
     int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
     const int roff = a.t0 - a.reg_start;      // region index = call-relative token + roff
-    // per-row offsets (see kMapMargin) of a block's 128 rows, staged in shared memory one block ahead
+    // per-row offsets (see kMapMargin) of the warp's 32 columns, staged per warp in shared memory one block ahead:
+    // lane e fetches the offset of column e, every lane then reads all 32 back as broadcast vector loads
     auto load_stats = [&](int blk) -> float {
-      const int tk = blk * TPB + tid / G;
-      return (tid < 128 && tk < a.n) ? __ldg(rq + (size_t)tk * c.Hq + tid % G) : -INFINITY;
+      const int col = cq * 32 + lane;
+      const int tk = blk * TPB + col / G;
+      return tk < a.n ? __ldg(rq + (size_t)tk * c.Hq + col % G) : -INFINITY;
     };
-    if (tid < 128 && bmin < nblocks) s_stats[0][tid] = load_stats(bmin);
-    asm volatile("bar.sync 1, 512;" ::: "memory");
+    float* my_stats = &s_stats[warp][0][0];
+    if (bmin < nblocks) my_stats[lane] = load_stats(bmin);
+    __syncwarp();
     long long total[kMapKT];
 #pragma unroll
     for (int kt = 0; kt < kMapKT; ++kt) total[kt] = 0;
     bool ok = true;
     int it = 0, seq = 0;
-    for (int blk = bmin; blk < nblocks; ++blk, ++it) {
+    const float2 c2v = make_float2(c2, c2);
+    const float2 sc = make_float2(kMapScale, kMapScale), mg = make_float2(12582912.f, 12582912.f);
+    for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
       const int st = it & 1;
       const bool more = blk + 1 < nblocks;
       float nxt = -INFINITY;
       if (more) nxt = load_stats(blk + 1);
       const int tokb = blk * TPB;  // first token of the block (call-relative)
-      const float* ss = &s_stats[st][cq * 32];
+      const float* ss = my_stats + st * 32;
 #pragma unroll
       for (int kt = 0; kt < kMapKT; ++kt) {
         if (kt >= ntile || blk < blk0_of(kt)) continue;
         const int buf = seq & 3;
-        // after an expired wait every thread keeps walking the steps (without computing) so that the named barrier
-        // below is still reached by all 512 epilogue threads
         ok = ok && mbar_wait(bar(B_SFULL + buf), (seq >> 2) & 1, abortp);
         ++seq;
-        if (!ok) continue;
+        if (!ok) break;
         fence_after_sync();
-        uint32_t v[1][32];
-        tmem_ld32(tmem + lane_base + buf * 128 + cq * 32, v[0]);
+        uint32_t v[32];
+        tmem_ld32(tmem + lane_base + buf * 128 + cq * 32, v);
         tmem_ld_wait();
         // the accumulator is in registers: hand the TMEM buffer back
         fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(B_SEMPTY + buf));
+        // x = log2 of (probability * 2^20) + 1 + margin; the Q20 value is rint(2^x * kMapScale), rounded to nearest
+        // even by adding 1.5 * 2^23: the integer sits in the mantissa.
+        if (!is_cur) {
+          // keys before the call: every row sees them, only the column sum (votes) is wanted.  The mantissa
+          // integers are summed as raw bit patterns (modulo 2^32) and the bias is taken off once per group.
+          // (No test for all-zero groups here: with thousands of visible keys a whole 8 x 32 group of entries
+          // below half a Q20 unit is rare, and the test costs more than the exponentials it saves.)
+          uint32_t bsum = 0;
+#pragma unroll
+          for (int e8 = 0; e8 < 32; e8 += 8) {
+            const float4 o0 = *reinterpret_cast<const float4*>(ss + e8);
+            const float4 o1 = *reinterpret_cast<const float4*>(ss + e8 + 4);
+            float2 x[4];
+            x[0] = __ffma2_rn(make_float2(__uint_as_float(v[e8]), __uint_as_float(v[e8 + 1])), c2v,
+                              make_float2(o0.x, o0.y));
+            x[1] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 2]), __uint_as_float(v[e8 + 3])), c2v,
+                              make_float2(o0.z, o0.w));
+            x[2] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 4]), __uint_as_float(v[e8 + 5])), c2v,
+                              make_float2(o1.x, o1.y));
+            x[3] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 6]), __uint_as_float(v[e8 + 7])), c2v,
+                              make_float2(o1.z, o1.w));
+            {
+              uint32_t part = 0u - 8u * 0x4B400000u;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float2 y = __ffma2_rn(make_float2(ex2m(x[e].x), ex2m(x[e].y)), sc, mg);
+                part += __float_as_uint(y.x) + __float_as_uint(y.y);
+              }
+              bsum += part;
+            }
+          }
+          total[kt] += (long long)bsum;
+          continue;
+        }
         const int key0 = key0_of(kt);
         const int key = key0 + krel;
         const bool key_ok = key < key_end && key >= c.Ls;
-        const int jrel = key - a.t0;  // call-relative (cur tiles only)
-        const bool diag = is_cur && tokb < (key0 - a.t0) + 128;  // some token of the block precedes some key
+        const int jrel = key - a.t0;  // call-relative
+        const bool diag = tokb < (key0 - a.t0) + 128;  // some token of the block precedes some key
         int bsum = 0;
+        int aq[32];
 #pragma unroll
-        for (int ch = 0; ch < 1; ++ch) {
-          int aq[32];
+        for (int e8 = 0; e8 < 32; e8 += 8) {
+          const float4 o0 = *reinterpret_cast<const float4*>(ss + e8);
+          const float4 o1 = *reinterpret_cast<const float4*>(ss + e8 + 4);
+          float2 x[4];
+          x[0] = __ffma2_rn(make_float2(__uint_as_float(v[e8]), __uint_as_float(v[e8 + 1])), c2v,
+                            make_float2(o0.x, o0.y));
+          x[1] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 2]), __uint_as_float(v[e8 + 3])), c2v,
+                            make_float2(o0.z, o0.w));
+          x[2] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 4]), __uint_as_float(v[e8 + 5])), c2v,
+                            make_float2(o1.x, o1.y));
+          x[3] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 6]), __uint_as_float(v[e8 + 7])), c2v,
+                            make_float2(o1.z, o1.w));
+          // an entry with x < 0 rounds to zero: a group of eight columns whose x is negative on every lane of the
+          // warp (common under the causal diagonal) needs no exponentials at all
+          const float xm = fmaxf(fmaxf(fmax3(x[0].x, x[0].y, x[1].x), fmax3(x[1].y, x[2].x, x[2].y)),
+                                 fmaxf(x[3].x, x[3].y));
+          if (__any_sync(0xffffffffu, xm >= 0.f)) {
 #pragma unroll
-          for (int e8 = 0; e8 < 32; e8 += 8) {
-            // x = log2 of (probability * 2^20) + 1 + margin.  An entry with x < 0 rounds to zero, so a group of
-            // eight columns whose x is negative on every lane of the warp needs no exponentials at all.
-            const float4 o0 = *reinterpret_cast<const float4*>(ss + ch * 32 + e8);
-            const float4 o1 = *reinterpret_cast<const float4*>(ss + ch * 32 + e8 + 4);
-            const float2 c2v = make_float2(c2, c2);
-            float2 x[4];
-            x[0] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8]), __uint_as_float(v[ch][e8 + 1])), c2v,
-                              make_float2(o0.x, o0.y));
-            x[1] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 2]), __uint_as_float(v[ch][e8 + 3])), c2v,
-                              make_float2(o0.z, o0.w));
-            x[2] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 4]), __uint_as_float(v[ch][e8 + 5])), c2v,
-                              make_float2(o1.x, o1.y));
-            x[3] = __ffma2_rn(make_float2(__uint_as_float(v[ch][e8 + 6]), __uint_as_float(v[ch][e8 + 7])), c2v,
-                              make_float2(o1.z, o1.w));
-            const float xm = fmaxf(fmaxf(fmax3(x[0].x, x[0].y, x[1].x), fmax3(x[1].y, x[2].x, x[2].y)),
-                                   fmaxf(x[3].x, x[3].y));
-            if (__any_sync(0xffffffffu, xm >= 0.f)) {
-              const float2 sc = make_float2(kMapScale, kMapScale), mg = make_float2(12582912.f, 12582912.f);
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                // round to nearest even by adding 1.5 * 2^23: the integer sits in the mantissa
-                const float2 y = __ffma2_rn(make_float2(ex2m(x[e].x), ex2m(x[e].y)), sc, mg);
-                aq[e8 + 2 * e] = __float_as_int(y.x) - 0x4B400000;
-                aq[e8 + 2 * e + 1] = __float_as_int(y.y) - 0x4B400000;
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 8; ++e) aq[e8 + e] = 0;
-            }
-          }
-          if (diag) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (tokb + (cq * 32 + e) / G < jrel) aq[e] = 0;
-          }
-          if (is_cur) {
-            // head sum per token (Eq. 4) -> region map; causality already zeroed the invalid entries
-#pragma unroll
-            for (int t = 0; t < 32 / G; ++t) {
-              int sv = 0;
-#pragma unroll
-              for (int hh = 0; hh < G; ++hh) sv += aq[t * G + hh];
-              bsum += sv;
-              const int tk = tokb + (cq * 32) / G + t;
-              if (key_ok && sv != 0 && tk < a.n) atomicAdd(&Mq[(size_t)(tk + roff) * c.chunk + (jrel + roff)], sv);
+            for (int e = 0; e < 4; ++e) {
+              const float2 y = __ffma2_rn(make_float2(ex2m(x[e].x), ex2m(x[e].y)), sc, mg);
+              aq[e8 + 2 * e] = __float_as_int(y.x) - 0x4B400000;
+              aq[e8 + 2 * e + 1] = __float_as_int(y.y) - 0x4B400000;
             }
           } else {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) bsum += aq[e];
+            for (int e = 0; e < 8; ++e) aq[e8 + e] = 0;
           }
+        }
+        if (diag) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (tokb + (cq * 32 + e) / G < jrel) aq[e] = 0;
+        }
+        // head sum per token (Eq. 4) -> region map; causality already zeroed the invalid entries
+#pragma unroll
+        for (int t = 0; t < 32 / G; ++t) {
+          int sv = 0;
+#pragma unroll
+          for (int hh = 0; hh < G; ++hh) sv += aq[t * G + hh];
+          bsum += sv;
+          const int tk = tokb + (cq * 32) / G + t;
+          if (key_ok && sv != 0 && tk < a.n) atomicAdd(&Mq[(size_t)(tk + roff) * c.chunk + (jrel + roff)], sv);
         }
         total[kt] += bsum;
       }
-      if (tid < 128 && more) s_stats[st ^ 1][tid] = nxt;
-      asm volatile("bar.sync 1, 512;" ::: "memory");
+      __syncwarp();
+      if (more) my_stats[(st ^ 1) * 32 + lane] = nxt;
+      __syncwarp();
     }
     if (ok) {
 #pragma unroll

@@ -691,6 +691,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   __shared__ int s_ids[kMaxTopK];
   __shared__ int s_cnt;
   __shared__ int s_scan[512];
+  __shared__ int s_rs[kMaxTopK + 2], s_pre[kMaxTopK + 3], s_nr;  // merged ranges and their packed-row prefix
   const int g = blockIdx.x;
   int layer, sq, pos = 0, loc_begin = 0;
   if (DECODE) {
@@ -812,6 +813,57 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     if (DECODE) push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
     c.rng_cnt[unit * c.Hkv + g] = nr;
     atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+    if (!DECODE) {
+      int run = 0;
+      for (int i = 0; i < nr; ++i) {
+        s_rs[i] = rs[i];
+        s_pre[i] = run;
+        run += rl[i];
+      }
+      s_pre[nr] = run;
+      s_nr = nr;
+      c.gcnt[(size_t)layer * c.Hkv + g] = run;
+    }
+  }
+  if (!DECODE) {
+    // a5 gather: pack the K and V rows of the selected spans into one contiguous slab per (layer, KV head), so the
+    // attention kernel that continues over them reads whole 128-row tiles.  16 threads per 256-byte row, four rows
+    // of K and of V in flight per thread; the rows up to the next multiple of 8 are zero-filled.
+    __syncthreads();
+    const int nr = s_nr, R = s_pre[nr], Rz = (R + 7) & ~7;
+    const size_t slab = (unit * c.Hkv + g) * (size_t)c.Tpad;
+    const uint4* Ksrc = reinterpret_cast<const uint4*>(c.Kc + slab * kD);
+    const uint4* Vsrc = reinterpret_cast<const uint4*>(c.Vc + slab * kD);
+    const size_t gslab = ((size_t)layer * c.Hkv + g) * (size_t)c.Rcap;
+    uint4* Kdst = reinterpret_cast<uint4*>(c.Kg + gslab * kD);
+    uint4* Vdst = reinterpret_cast<uint4*>(c.Vg + gslab * kD);
+    const int ch = tid & 15, rpp = nt >> 4;  // 16-byte chunk of the row, rows per pass
+    for (int r0 = tid >> 4; r0 < Rz; r0 += 4 * rpp) {
+      uint4 kv[4], vv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int r = r0 + i * rpp;
+        kv[i] = vv[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (r < R) {
+          int lo = 0, hi = nr - 1;  // last range whose first packed row is <= r
+          while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (s_pre[mid] <= r) lo = mid; else hi = mid - 1;
+          }
+          const size_t tok = (size_t)(s_rs[lo] + (r - s_pre[lo]));
+          kv[i] = __ldg(Ksrc + tok * 16 + ch);
+          vv[i] = __ldg(Vsrc + tok * 16 + ch);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int r = r0 + i * rpp;
+        if (r < Rz) {
+          Kdst[(size_t)r * 16 + ch] = kv[i];
+          Vdst[(size_t)r * 16 + ch] = vv[i];
+        }
+      }
+    }
   }
 }
 

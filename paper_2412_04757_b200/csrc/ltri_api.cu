@@ -105,6 +105,10 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.Oacc = cv.take<float>((size_t)d.NL * align_up((size_t)d.chunk * d.G, 256) * d.Hkv * kD);
   d.u = cv.take<float>((size_t)d.NL * d.Hkv * d.Jmax * kD);
   d.Jcnt = cv.take<int>(d.NL);
+  d.Rcap = (long long)align_up((size_t)d.topk * d.chunk, 128) + kTokPad;
+  d.Kg = cv.take<__nv_bfloat16>((size_t)d.NL * d.Hkv * d.Rcap * kD);
+  d.Vg = cv.take<__nv_bfloat16>((size_t)d.NL * d.Hkv * d.Rcap * kD);
+  d.gcnt = cv.take<int>((size_t)d.NL * d.Hkv);
   d.scores = cv.take<float>(units * d.Hkv * d.cap);
   d.rng_start = cv.take<int>(units * d.Hkv * (d.topk + 2));
   d.rng_len = cv.take<int>(units * d.Hkv * (d.topk + 2));
