@@ -137,6 +137,66 @@ cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_co
 }
 
 // ------------------------------------------------------------------------------------------
+// Warp-parallel walks over a shared-memory histogram (all 32 lanes of one warp call them).
+// pick_from_top: the largest bin b with  sum(hist[b+1..nb-1]) < need <= sum(hist[b..nb-1]);  `need` becomes the rank
+// inside that bin.  pick_from_bottom: the smallest bin b with  rank < sum(hist[0..b]);  `rank` becomes the rank inside
+// the bin.  Both clamp to the last bin they look at when the counts do not reach the target.  nb is a multiple of 32.
+__device__ __forceinline__ int pick_from_top(const unsigned* hist, int nb, unsigned& need) {
+  const int lane = threadIdx.x & 31, per = nb >> 5;
+  const int b1 = nb - lane * per;  // lane 0 owns the top `per` bins
+  unsigned mine = 0;
+  for (int i = 1; i <= per; ++i) mine += hist[b1 - i];
+  unsigned incl = mine;  // counts of this lane's bins and of all higher ones
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  const unsigned hit = __ballot_sync(0xffffffffu, incl >= need);
+  const int src = hit ? __ffs(hit) - 1 : 31;
+  int bin = 0;
+  unsigned left = 0;
+  if (lane == src) {
+    left = need - (incl - mine);
+    bin = b1 - 1;
+    for (; bin > b1 - per; --bin) {
+      if (left <= hist[bin]) break;
+      left -= hist[bin];
+    }
+    if (!hit && left > hist[bin]) left = hist[bin];
+  }
+  need = __shfl_sync(0xffffffffu, left, src);
+  return __shfl_sync(0xffffffffu, bin, src);
+}
+
+__device__ __forceinline__ unsigned pick_from_bottom(const unsigned* hist, int nb, long long& rank) {
+  const int lane = threadIdx.x & 31, per = nb >> 5;
+  const int b0 = lane * per;
+  long long mine = 0;
+  for (int i = 0; i < per; ++i) mine += hist[b0 + i];
+  long long incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long t = shfl_up_ll(incl, o);
+    if (lane >= o) incl += t;
+  }
+  const unsigned hit = __ballot_sync(0xffffffffu, rank < incl);
+  const int src = hit ? __ffs(hit) - 1 : 31;
+  unsigned bin = 0;
+  long long left = 0;
+  if (lane == src) {
+    left = rank - (incl - mine);
+    bin = (unsigned)b0;
+    for (; bin < (unsigned)(b0 + per - 1); ++bin) {
+      if (left < (long long)hist[bin]) break;
+      left -= hist[bin];
+    }
+  }
+  rank = shfl_ll(left, src);
+  return __shfl_sync(0xffffffffu, bin, src);
+}
+
+// ------------------------------------------------------------------------------------------
 // a3 segmenter, step 1: exact rank selection of theta (quantile mode) over the causal entries of Mq.
 // Pass 1 counts negatives (only hand-built maps have any) and zeros (a sparse map is mostly zeros) and builds a
 // log-scale histogram of the positive entries: bin = (position of the leading one, next four bits), which is monotone
@@ -213,35 +273,37 @@ __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin
     tot[threadIdx.x] = sum;
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (threadIdx.x < 32) {
     long long cn = 0, cz = 0;
     for (int w = 0; w < 32; ++w) {
       cn += s_red[w][0];
       cz += s_red[w][1];
     }
     if (rank < cn) {
-      s_cls = -1;
-      s_rank = rank;
+      if (lane == 0) {
+        s_cls = -1;
+        s_rank = rank;
+      }
     } else if (rank < cn + cz) {
-      s_cls = 0;
-      c.thetaq[layer] = 0;
+      if (lane == 0) {
+        s_cls = 0;
+        c.thetaq[layer] = 0;
+      }
     } else {
       long long r = rank - cn - cz;
-      unsigned b = 0;
-      for (; b < kThetaBins - 1; ++b) {
-        if (r < (long long)tot[b]) break;
-        r -= tot[b];
-      }
+      const unsigned b = pick_from_bottom(tot, kThetaBins, r);
       const int e = (int)(b >> 4);
       const unsigned frac = b & 15u;
-      s_rank = r;
-      if (e <= 4) {  // the bin holds a single value
-        s_cls = 0;
-        c.thetaq[layer] = (long long)((1u << e) | (frac >> (4 - e)));
-      } else {
-        s_cls = 1;
-        s_prefix = (1u << e) | (frac << (e - 4));  // leading one and the next four bits
-        s_lo_bits = (unsigned)(e - 4);             // bits still unknown
+      if (lane == 0) {
+        s_rank = r;
+        if (e <= 4) {  // the bin holds a single value
+          s_cls = 0;
+          c.thetaq[layer] = (long long)((1u << e) | (frac >> (4 - e)));
+        } else {
+          s_cls = 1;
+          s_prefix = (1u << e) | (frac << (e - 4));  // leading one and the next four bits
+          s_lo_bits = (unsigned)(e - 4);             // bits still unknown
+        }
       }
     }
   }
@@ -271,16 +333,14 @@ __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin
       tot[threadIdx.x] = sum;
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x < 32) {
       long long r = s_rank;
-      unsigned b = 0;
-      for (; b <= dmask; ++b) {
-        if (r < (long long)tot[b]) break;
-        r -= tot[b];
-      }
+      unsigned b = pick_from_bottom(tot, kThetaBins, r);  // bins above dmask are empty
       if (b > dmask) b = dmask;
-      s_rank = r;
-      s_prefix = prefix | (b << lo);
+      if (threadIdx.x == 0) {
+        s_rank = r;
+        s_prefix = prefix | (b << lo);
+      }
     }
     __syncthreads();
     hi = lo;
@@ -730,16 +790,13 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
         if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (tid == 0) {
+      if (tid < 32) {
         unsigned need = s_need;
-        int bin = 255;
-        for (; bin >= 0; --bin) {
-          if (need <= hist[bin]) break;
-          need -= hist[bin];
+        const int bin = pick_from_top(hist, 256, need);
+        if (tid == 0) {
+          s_need = need;
+          s_prefix = prefix | ((unsigned)bin << shift);
         }
-        if (bin < 0) bin = 0;
-        s_need = need;
-        s_prefix = prefix | ((unsigned)bin << shift);
       }
       __syncthreads();
     }
@@ -953,16 +1010,13 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
         if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (tid == 0) {
+      if (tid < 32) {
         unsigned need = s_need;
-        int bin = 255;
-        for (; bin >= 0; --bin) {
-          if (need <= hist[bin]) break;
-          need -= hist[bin];
+        const int bin = pick_from_top(hist, 256, need);
+        if (tid == 0) {
+          s_need = need;
+          s_prefix = prefix | ((unsigned)bin << shift);
         }
-        if (bin < 0) bin = 0;
-        s_need = need;
-        s_prefix = prefix | ((unsigned)bin << shift);
       }
       __syncthreads();
     }

@@ -129,6 +129,7 @@ struct ltri_ctx {
   int sm_count = 148;
   bool use_tc = false;     // tcgen05/TMEM/TMA attention kernels (default when available)
   int dec_fused = -1;      // decode retrieval in one launch: -1 auto, 0 never, 1 whenever the index fits
+  int dec_split = 0;       // split count of the decode attention: 0 auto (testing aid)
   alignas(64) unsigned char kv_maps[kTcMapBytes];  // TMA descriptors of the K/V cache
   long long launches = 0;  // kernels launched since creation
   // optional per-kernel-class timing with CUDA events on the launching stream
@@ -219,6 +220,7 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
   }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (const char* f = std::getenv("LTRI_DEC_FUSED")) ctx->dec_fused = std::atoi(f) != 0 ? 1 : 0;  // testing aid
+  if (const char* f = std::getenv("LTRI_DEC_SPLIT")) ctx->dec_split = std::max(0, std::atoi(f));    // testing aid
   const char* impl = std::getenv("LTRI_ATTN_IMPL");  // "mma" selects the warp-MMA kernels (debugging aid)
   ctx->use_tc = tc_attention_supported(ctx->d) && !(impl && std::strcmp(impl, "mma") == 0) &&
                 tc_encode_kv_maps(ctx->d, ctx->kv_maps);
@@ -413,8 +415,27 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
       b.src[i] = i0 + i;
     }
     const int units = b.n * layer_count * d.Hkv;
-    int nsplit = (ctx->sm_count * 8 + units - 1) / units;
-    nsplit = std::max(1, std::min(nsplit, kMaxDecSplit));
+    // split count of the decode attention: two CTAs fit an SM, so the grid runs in waves of 2 x SMs CTAs.  Among
+    // the split counts that leave a CTA at least ~512 tokens (of the tokens known on the host: sink + everything
+    // since the last eviction) take the one whose last wave is fullest; ties go to fewer, longer slices.
+    int nsplit = 1;
+    {
+      const LayerState& s0 = ctx->at(seq_ids[i0], layer_begin);
+      const long long known = d.Ls + (s0.t + 1 - s0.E);
+      const int wave = 2 * ctx->sm_count;
+      const int max_split = (int)std::max<long long>(1, std::min<long long>(kMaxDecSplit, known / 512));
+      double best = -1.0;
+      for (int ns = 1; ns <= max_split; ++ns) {
+        const long long ctas = (long long)units * ns;
+        const long long waves = (ctas + wave - 1) / wave;
+        const double eff = (double)ctas / (double)(waves * wave);
+        if (eff > best + 1e-9) {
+          best = eff;
+          nsplit = ns;
+        }
+      }
+      if (ctx->dec_split > 0) nsplit = std::min(ctx->dec_split, kMaxDecSplit);
+    }
     {
       Scope sc(ctx, st, LTRI_K_APPEND, 1);
       LTRI_CUDA(ctx, launch_append_decode(d, b, layer_begin, layer_count, n_seqs, kb, vb, st));
