@@ -41,6 +41,15 @@ struct RangeList {
   int len[kMaxTopK + 2];
 };
 
+// What the softmax threads need to know about a tile: which of its 128 key slots hold keys, and for the causal
+// (current-chunk) tile the absolute token of slot 0 (-1 otherwise).
+struct __align__(16) TileDesc {
+  unsigned m0, m1, m2, m3;
+  int causal_tok0;
+  int full;  // all 128 slots valid and no causal masking
+  int pad0, pad1;
+};
+
 // Deterministic tile builder: every role walks the same range list and derives the same tiles.  All state lives in
 // registers (no dynamically indexed arrays); only the producer asks for the piece list.
 struct TileIter {
@@ -140,7 +149,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __shared__ __align__(8) unsigned long long bars[3 + 8 + 6];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ RangeList rgs[3];        // key ranges of the work items in flight (roles may be up to two items apart)
+  __shared__ RangeList rg;            // key ranges of the work item the producer is walking
+  __shared__ int s_item_tiles[3];     // tile count of the work items in flight (roles may be up to two items apart)
+  __shared__ TileDesc s_td[8];        // per-tile masks, written by the producer, read by the softmax threads
   __shared__ int s_quit[2];
   __shared__ int s_items_ready;       // number of work items whose key ranges the producer has published
   __shared__ float s_max[2][2][128];  // per Q tile, per column half, per row: partial maxima / sums
@@ -163,7 +174,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     s_abort = 0;
     s_quit[0] = s_quit[1] = 0;
     s_items_ready = 0;
-    rgs[0].n = rgs[1].n = rgs[2].n = 0;
+    rg.n = 0;
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QFREE), 1);
     mbar_init(bar(B_ODONE), 1);
@@ -221,7 +232,6 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     if (lane == 0) prefetch_tmap(&maps.q);
     for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
       const Item w = decode(item);
-      RangeList& rg = rgs[wi % 3];
       if (lane == 0) {
         // the Q buffer is free once every QK^T product of the previous item has completed
         if (wi > 0) ok = mbar_wait(bar(B_QFREE), (wi - 1) & 1, abortp) ? 1 : 0;
@@ -240,8 +250,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           rg.start[0] = 0;
           rg.len[0] = c.gcnt[(size_t)w.layer * c.Hkv + w.g];
         }
-        // publish the ranges with a monotonic counter: a softmax thread may look for item wi only after the Q tile
-        // of item wi+1 has arrived, so a parity barrier could not tell the two apart
+        // publish the item's tile count with a monotonic counter: a softmax thread may look for item wi only after
+        // the Q tile of item wi+1 has arrived, so a parity barrier could not tell the two apart
+        s_item_tiles[wi % 3] = count_tiles(&rg, causal_ri);
         __threadfence_block();
         *reinterpret_cast<volatile int*>(&s_items_ready) = wi + 1;
         if (ok) {
@@ -272,7 +283,18 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         for (int p = 0; p < np; ++p) bytes += (uint32_t)(8 << pbox[p]) * 256u;
         if (lane == 0) {
           if (jt >= 2) ok = mbar_wait(bar(B_KEMPTY + st), par, abortp) ? 1 : 0;
-          if (ok) mbar_expect_tx(bar(B_KFULL + st), bytes);
+          if (ok) {
+            // the tile's masks travel to the softmax threads through the barrier chain KFULL -> SREADY; slot jt & 7
+            // was last read for tile jt - 8, whose softmax ended before K stage jt - 2 was released
+            TileDesc& td = s_td[jt & 7];
+            td.m0 = it.m0;
+            td.m1 = it.m1;
+            td.m2 = it.m2;
+            td.m3 = it.m3;
+            td.causal_tok0 = it.causal_tok0;
+            td.full = it.full ? 1 : 0;
+            mbar_expect_tx(bar(B_KFULL + st), bytes);
+          }
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
@@ -334,7 +356,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
         ok = mbar_wait(bar(B_QFULL), wi & 1, abortp);
         if (!ok) break;
-        const int T = count_tiles(&rgs[wi % 3], causal_ri);
+        const int T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
         if (T > 0) {
           ok = mbar_wait(bar(B_KFULL + (jt & 1)), (jt >> 1) & 1, abortp);
           if (!ok) break;
@@ -420,6 +442,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         }
         __threadfence_block();
       }
+      // collective decision per Q tile: either all 256 threads walk the item's tiles or all leave here, so the named
+      // barriers below always see every thread
+      if (!ok) s_quit[q] = 1;
+      asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+      if (s_quit[q]) break;
+      const int T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
       float m_used = -INFINITY, lsum = 0.f;
       if (ok && phase == 1) {
         // continue from the state the local pass stored: running max, row sum and the unnormalised O row
@@ -445,12 +473,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         }
         tmem_st_wait();
       }
-      TileIter it;
-      it.rg = &rgs[wi % 3];
-      it.causal_ri = causal_ri;
       int j = 0;
       const int row_abs = a.t0 + tk;
-      while (it.next()) {
+      while (j < T) {
         // after an expired wait every thread keeps walking the item's tiles (without computing) so that the named
         // barrier is still reached by all 256 threads of the tile
         ok = ok && mbar_wait(bar(B_SREADY + q), jt & 1, abortp);
@@ -465,13 +490,16 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         tmem_ld32(tS, v[0]);
         tmem_ld32(tS + 32, v[1]);
         tmem_ld_wait();
-        if (!it.full) {
+        const TileDesc& td = s_td[jt & 7];
+        if (!td.full) {
           // valid-slot bits, and for the causal tile the last visible column of this row (keys are consecutive
           // tokens from slot 0): column c is visible iff c <= lim
-          const int lim = it.causal_tok0 >= 0 ? row_abs - it.causal_tok0 - half * 64 : 127;
+          const int ctok = td.causal_tok0;
+          const int lim = ctok >= 0 ? row_abs - ctok - half * 64 : 127;
+          const uint2 mks = *reinterpret_cast<const uint2*>(&td.m0 + half * 2);
 #pragma unroll
           for (int ch = 0; ch < 2; ++ch) {
-            const unsigned mk = it.mask(half * 2 + ch);
+            const unsigned mk = ch == 0 ? mks.x : mks.y;
 #pragma unroll
             for (int e = 0; e < 32; ++e)
               if (!((mk >> e) & 1u) || ch * 32 + e > lim) v[ch][e] = 0xff800000u;  // -inf
