@@ -1,6 +1,8 @@
 // State kernels: cache append, eviction + span index build (Sec. 3.3.1, Eq. 6), span segmenter
 // (Eq. 4-5, App. "NMS Input Filtration"), query representatives, similarity scores (Eq. 7) and
 // top-k selection (Eq. 8).  All segmentation arithmetic is integer and order-independent.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace ltri {
@@ -202,28 +204,36 @@ __device__ __forceinline__ unsigned pick_from_bottom(const unsigned* hist, int n
 // log-scale histogram of the positive entries: bin = (position of the leading one, next four bits), which is monotone
 // in the value and spreads a heavy-tailed map over many bins.  If the rank falls among the positives, the remaining
 // low bits of the selected bin are resolved by MSB radix passes of 9 bits.  One private histogram per warp, four loads
-// in flight per lane, one CTA per layer.
+// in flight per lane; a thread-block cluster of eight CTAs shares a layer: each counts its share of the rows, then
+// every CTA adds up the eight histograms through distributed shared memory and takes the same decision.
 constexpr int kThetaBits = 9;
 constexpr int kThetaBins = 1 << kThetaBits;
 
-// visits the causal entries of the m x m map: f(value) for every (i, j <= i); a warp owns rows warp, warp+32, ...
+// visits the causal entries of the m x m map: f(value) for every (i, j <= i).  The rows are dealt to the warps of the
+// `nparts` CTAs that share a map in pairs (i, m-1-i), so every warp sees about the same number of entries.
 template <typename F>
-__device__ __forceinline__ void for_each_causal(const int* __restrict__ Mq, int ld, int m, F&& f) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-  for (int i = warp; i < m; i += nwarps) {
-    const int* row = Mq + (size_t)i * ld;
-    for (int j0 = 0; j0 <= i; j0 += 128) {
-      int v[4];
-      bool ok[4];
+__device__ __forceinline__ void for_each_causal(const int* __restrict__ Mq, int ld, int m, int part, int nparts, F&& f) {
+  const int lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int gw = part * nwarps + (threadIdx.x >> 5), step = nparts * nwarps;
+  for (int idx = gw; 2 * idx < m; idx += step) {
+#pragma unroll 1
+    for (int side = 0; side < 2; ++side) {
+      const int i = side == 0 ? idx : m - 1 - idx;
+      if (side == 1 && i == idx) break;
+      const int* row = Mq + (size_t)i * ld;
+      for (int j0 = 0; j0 <= i; j0 += 128) {
+        int v[4];
+        bool ok[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int j = j0 + u * 32 + lane;
-        ok[u] = j <= i;
-        v[u] = ok[u] ? row[j] : 0;
+        for (int u = 0; u < 4; ++u) {
+          const int j = j0 + u * 32 + lane;
+          ok[u] = j <= i;
+          v[u] = ok[u] ? row[j] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (ok[u]) f(v[u]);
       }
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (ok[u]) f(v[u]);
     }
   }
 }
@@ -235,21 +245,66 @@ __device__ __forceinline__ unsigned log_bin(unsigned v) {
   return ((unsigned)e << 4) | frac;
 }
 
-__global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin, int m, long long rank) {
-  extern __shared__ unsigned hist[];  // [32 warps][kThetaBins]
-  const int layer = layer_begin + blockIdx.x;
+constexpr int kThetaCluster = 8;   // CTAs (one thread-block cluster) per layer
+constexpr int kThetaThreads = 512;
+
+__global__ void __cluster_dims__(kThetaCluster, 1, 1) __launch_bounds__(kThetaThreads)
+    k_theta_select(DevCtx c, int layer_begin, int m, long long rank) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ unsigned hist[];  // [warps][kThetaBins]
+  constexpr int NW = kThetaThreads / 32;
+  const int layer = layer_begin + blockIdx.x / kThetaCluster;
+  const int part = (int)cluster.block_rank();
   const int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
-  __shared__ unsigned tot[kThetaBins];
-  __shared__ unsigned s_red[32][2];
+  __shared__ unsigned loc[kThetaBins + 2];  // this CTA's histogram, then its counts of negatives and zeros
+  __shared__ unsigned tot[kThetaBins];      // the cluster's histogram (every CTA builds its own copy)
+  __shared__ unsigned s_red[NW][2];
   __shared__ unsigned s_prefix, s_lo_bits;
-  __shared__ long long s_rank;
+  __shared__ long long s_rank, s_cn, s_cz;
   __shared__ int s_cls;  // 0: answer found, 1: among positives (bin chosen), -1: among negatives
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   unsigned* myhist = hist + warp * kThetaBins;
-  for (int t = threadIdx.x; t < 32 * kThetaBins; t += blockDim.x) hist[t] = 0;
+  // sums the per-warp histograms into loc, then the cluster's loc arrays into tot.  The second cluster barrier keeps
+  // every CTA's loc intact until all have read it (and keeps a CTA from exiting while it can still be read).
+  auto combine = [&](bool with_counts) {
+    __syncthreads();
+    if (threadIdx.x < kThetaBins) {
+      unsigned sum = 0;
+      for (int w = 0; w < NW; ++w) sum += hist[w * kThetaBins + threadIdx.x];
+      loc[threadIdx.x] = sum;
+    }
+    if (with_counts && threadIdx.x == 0) {
+      unsigned cn = 0, cz = 0;
+      for (int w = 0; w < NW; ++w) {
+        cn += s_red[w][0];
+        cz += s_red[w][1];
+      }
+      loc[kThetaBins] = cn;
+      loc[kThetaBins + 1] = cz;
+    }
+    cluster.sync();
+    if (threadIdx.x < kThetaBins) {
+      unsigned sum = 0;
+      for (int r = 0; r < kThetaCluster; ++r) sum += cluster.map_shared_rank(loc, r)[threadIdx.x];
+      tot[threadIdx.x] = sum;
+    }
+    if (with_counts && threadIdx.x == 0) {
+      long long cn = 0, cz = 0;
+      for (int r = 0; r < kThetaCluster; ++r) {
+        const unsigned* rl = cluster.map_shared_rank(loc, r);
+        cn += rl[kThetaBins];
+        cz += rl[kThetaBins + 1];
+      }
+      s_cn = cn;
+      s_cz = cz;
+    }
+    cluster.sync();
+  };
+  for (int t = threadIdx.x; t < NW * kThetaBins; t += blockDim.x) hist[t] = 0;
   __syncthreads();
   unsigned nneg = 0, nzero = 0;
-  for_each_causal(Mq, c.chunk, m, [&](int v) {
+  for_each_causal(Mq, c.chunk, m, part, kThetaCluster, [&](int v) {
     if (v > 0)
       atomicAdd(&myhist[log_bin((unsigned)v)], 1u);
     else if (v == 0)
@@ -266,19 +321,9 @@ __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin
     s_red[warp][0] = nneg;
     s_red[warp][1] = nzero;
   }
-  __syncthreads();
-  if (threadIdx.x < kThetaBins) {
-    unsigned sum = 0;
-    for (int w = 0; w < 32; ++w) sum += hist[w * kThetaBins + threadIdx.x];
-    tot[threadIdx.x] = sum;
-  }
-  __syncthreads();
+  combine(true);
   if (threadIdx.x < 32) {
-    long long cn = 0, cz = 0;
-    for (int w = 0; w < 32; ++w) {
-      cn += s_red[w][0];
-      cz += s_red[w][1];
-    }
+    const long long cn = s_cn, cz = s_cz;
     if (rank < cn) {
       if (lane == 0) {
         s_cls = -1;
@@ -287,7 +332,7 @@ __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin
     } else if (rank < cn + cz) {
       if (lane == 0) {
         s_cls = 0;
-        c.thetaq[layer] = 0;
+        if (part == 0) c.thetaq[layer] = 0;
       }
     } else {
       long long r = rank - cn - cz;
@@ -298,7 +343,7 @@ __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin
         s_rank = r;
         if (e <= 4) {  // the bin holds a single value
           s_cls = 0;
-          c.thetaq[layer] = (long long)((1u << e) | (frac >> (4 - e)));
+          if (part == 0) c.thetaq[layer] = (long long)((1u << e) | (frac >> (4 - e)));
         } else {
           s_cls = 1;
           s_prefix = (1u << e) | (frac << (e - 4));  // leading one and the next four bits
@@ -309,30 +354,23 @@ __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin
   }
   __syncthreads();
   const int cls = s_cls;
-  if (cls == 0) return;
+  if (cls == 0) return;  // the same decision in every CTA of the cluster
   // remaining bits: [0, hi).  Negatives: plain MSB radix over the sign-flipped key.
   int hi = cls > 0 ? (int)s_lo_bits : 31;
-  const int top = hi;  // entries take part when their bits above `top` equal the prefix's
   if (cls < 0 && threadIdx.x == 0) s_prefix = 0;
   __syncthreads();
   while (hi > 0) {
     const int lo = max(0, hi - kThetaBits);
     const unsigned dmask = (1u << (hi - lo)) - 1u;
-    for (int t = threadIdx.x; t < 32 * kThetaBins; t += blockDim.x) hist[t] = 0;
+    for (int t = threadIdx.x; t < NW * kThetaBins; t += blockDim.x) hist[t] = 0;
     __syncthreads();
     const unsigned prefix = s_prefix;
-    for_each_causal(Mq, c.chunk, m, [&](int v) {
+    for_each_causal(Mq, c.chunk, m, part, kThetaCluster, [&](int v) {
       const bool in_cls = cls > 0 ? v > 0 : v < 0;
       const unsigned key = cls > 0 ? (unsigned)v : ((unsigned)v ^ 0x80000000u);
       if (in_cls && (key >> hi) == (prefix >> hi)) atomicAdd(&myhist[(key >> lo) & dmask], 1u);
     });
-    __syncthreads();
-    if (threadIdx.x < kThetaBins) {
-      unsigned sum = 0;
-      for (int w = 0; w < 32; ++w) sum += hist[w * kThetaBins + threadIdx.x];
-      tot[threadIdx.x] = sum;
-    }
-    __syncthreads();
+    combine(false);
     if (threadIdx.x < 32) {
       long long r = s_rank;
       unsigned b = pick_from_bottom(tot, kThetaBins, r);  // bins above dmask are empty
@@ -345,8 +383,7 @@ __global__ void __launch_bounds__(1024) k_theta_select(DevCtx c, int layer_begin
     __syncthreads();
     hi = lo;
   }
-  (void)top;
-  if (threadIdx.x == 0)
+  if (threadIdx.x == 0 && part == 0)
     c.thetaq[layer] = cls > 0 ? (long long)s_prefix : (long long)(int)(s_prefix ^ 0x80000000u);
 }
 
@@ -593,9 +630,8 @@ cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_
     long long rank = (long long)floor((double)theta * (double)(N - 1));
     if (rank < 0) rank = 0;
     if (rank > N - 1) rank = N - 1;
-    const int hsmem = 32 * kThetaBins * (int)sizeof(unsigned);
-    cudaFuncSetAttribute(k_theta_select, cudaFuncAttributeMaxDynamicSharedMemorySize, hsmem);
-    k_theta_select<<<layer_count, 1024, hsmem, s>>>(c, layer_begin, m, rank);
+    const int hsmem = (kThetaThreads / 32) * kThetaBins * (int)sizeof(unsigned);
+    k_theta_select<<<layer_count * kThetaCluster, kThetaThreads, hsmem, s>>>(c, layer_begin, m, rank);
   } else {
     k_theta_set<<<layer_count, 1, 0, s>>>(c, layer_begin, theta_q_abs);
   }
