@@ -37,7 +37,7 @@ enum {
   LTRI_ECAPACITY = -2, /* tokens, sequences, spans or arena size exceeded */
   LTRI_ESTATE = -3,    /* call order violated (e.g. prefill after decode, layers out of step) */
   LTRI_ECUDA = -4,     /* a CUDA runtime call failed; see ltri_last_cuda_error */
-  LTRI_EDEVICE = -5,   /* a device-side bounds check failed */
+  LTRI_EDEVICE = -5,   /* a device-side bounds or numeric-range check failed */
   LTRI_ETIMEOUT = -6   /* a bounded device-side wait expired */
 };
 

@@ -154,7 +154,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __shared__ TileDesc s_td[8];        // per-tile masks, written by the producer, read by the softmax threads
   __shared__ int s_quit[2];
   __shared__ int s_items_ready;       // number of work items whose key ranges the producer has published
-  __shared__ float s_max[2][2][128];  // per Q tile, per column half, per row: partial maxima / sums
+  __shared__ float s_max[2][2][2][128];  // per tile parity, Q tile, column half, row: partial maxima
+  __shared__ float s_sum[2][2][128];     // per Q tile, column half, row: partial row sums (end of an item)
   constexpr int TOKB = 256 / G;  // tokens per work item
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // persistent CTA: work items (token block, KV head, layer) are dealt round-robin
@@ -475,12 +476,15 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       }
       int j = 0;
       const int row_abs = a.t0 + tk;
+      bool need_ref = true;   // no reference maximum yet: the first tile exchanges the halves' maxima
+      float mprev = -INFINITY;
       while (j < T) {
         // after an expired wait every thread keeps walking the item's tiles (without computing) so that the named
         // barrier is still reached by all 256 threads of the tile
         ok = ok && mbar_wait(bar(B_SREADY + q), jt & 1, abortp);
         if (!ok) {
-          asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+          if (need_ref) asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+          need_ref = false;
           ++j;
           ++jt;
           continue;
@@ -505,14 +509,34 @@ __global__ void __launch_bounds__(kTcThreads, 1)
               if (!((mk >> e) & 1u) || ch * 32 + e > lim) v[ch][e] = 0xff800000u;  // -inf
           }
         }
-        float mt = -INFINITY;
+        // maximum of this thread's 64 logits (four independent chains)
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch)
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) mt = max3(mt, __uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1]));
-        s_max[q][half][r] = mt;
-        asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
-        mt = fmaxf(mt, s_max[q][half ^ 1][r]) * c2;
+          for (int e = 0; e < 32; e += 8) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              mx[u] = max3(mx[u], __uint_as_float(v[ch][e + 2 * u]), __uint_as_float(v[ch][e + 2 * u + 1]));
+          }
+        const float mloc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        // The two threads of a row must scale by the same reference.  On an item's first tile (no reference yet)
+        // they exchange their maxima through shared memory and a named barrier.  On later tiles the reference moves
+        // one tile late: it is the maximum over the previous tiles, whose partner half is already visible (the
+        // partner stored it before its PREADY arrival of the previous tile, which precedes this tile's SREADY), so
+        // no barrier sits between the logits and the exponentials.  A tile that exceeds the reference is harmless
+        // (the exponent is merely positive) unless it does so by more than 2^100, which raises the status word.
+        s_max[jt & 1][q][half][r] = mloc;
+        float mt;
+        if (need_ref) {
+          asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+          mt = fmaxf(mloc, s_max[jt & 1][q][half ^ 1][r]) * c2;
+        } else {
+          mt = fmaxf(mprev, s_max[(jt & 1) ^ 1][q][half ^ 1][r]) * c2;
+          if (mloc * c2 > m_used + 100.f && m_used > -INFINITY) set_status(c, -5, 7000 + (int)blockIdx.x);
+        }
+        need_ref = false;
+        mprev = mloc;
         // lazy running maximum: move it only when it grows by more than the threshold (or on first use)
         float alpha = 1.f;
         const bool grow = mt > m_used + kRescaleThreshold || (m_used == -INFINITY && mt > -INFINITY);
@@ -561,12 +585,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         ++jt;
       }
       // epilogue: the two halves of a row exchange their partial sums, then each writes its 64 output columns
-      s_max[q][half][r] = lsum;
+      s_sum[q][half][r] = lsum;
       asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
-      lsum += s_max[q][half ^ 1][r];
+      lsum += s_sum[q][half ^ 1][r];
       if (ok) ok = mbar_wait(bar(B_ODONE), wi & 1, abortp);
       if (!ok) s_quit[q] = 1;
-      asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");  // also: s_max is reused by the next item
+      asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");  // also: s_sum is reused by the next item
       if (s_quit[q]) break;  // collective decision: all 256 threads of the tile leave after the same item
       fence_after_sync();
       if (phase == 0 && row_ok && half == 0) {

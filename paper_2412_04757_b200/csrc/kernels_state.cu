@@ -591,34 +591,64 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
     c.Jcnt[layer] = a.q ? nout : 0;
   }
   if (!a.q) return;
-  // query representatives: one warp per span
+  // query representatives.  First one warp per span picks the representative tokens, then one warp per
+  // (span, KV head) sums their query rows with all loads of the head group in flight at once.
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   const long long* votes = c.votes + unit * c.Tpad;
   const __nv_bfloat16* q = a.q + (size_t)blockIdx.x * a.n * c.Hq * kD;
+  int* rep_tok = reinterpret_cast<int*>(skey);          // [Jmax][kMaxReps], the sort buffer is free now
+  int* rep_cnt = rep_tok + (2 * kMaxTopK + 1) * kMaxReps;
+  __syncthreads();
   for (int j = warp; j < nout; j += nwarps) {
     int toks[kMaxReps];
     const int nrep = select_reps(votes, a.reg_start + out_start[j], out_len[j], c.reps, toks);
-    for (int g = 0; g < c.Hkv; ++g) {
-      float ug[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int hh = 0; hh < c.G; ++hh) {
-        const int h = g * c.G + hh;
-        float qr[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int r = 0; r < nrep; ++r) {
-          const uint2 raw =
-              *reinterpret_cast<const uint2*>(q + ((size_t)(toks[r] - a.t0) * c.Hq + h) * kD + lane * 4);
-          const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
-          const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
-          qr[0] += __bfloat162float(p0.x);
-          qr[1] += __bfloat162float(p0.y);
-          qr[2] += __bfloat162float(p1.x);
-          qr[3] += __bfloat162float(p1.y);
-        }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) ug[e] += qr[e];
-      }
-      *reinterpret_cast<float4*>(c.u + (((size_t)layer * c.Hkv + g) * c.Jmax + j) * kD + lane * 4) =
-          make_float4(ug[0], ug[1], ug[2], ug[3]);
+    if (lane == 0) {
+      rep_cnt[j] = nrep;
+      for (int r = 0; r < nrep; ++r) rep_tok[j * kMaxReps + r] = toks[r];
     }
+  }
+  __syncthreads();
+  for (int task = warp; task < nout * c.Hkv; task += nwarps) {
+    const int j = task / c.Hkv, g = task % c.Hkv;
+    const int nrep = rep_cnt[j];
+    // per head: sum over the representative tokens (ascending), then the heads of the group in ascending order
+    float qr[8][4];
+#pragma unroll
+    for (int hh = 0; hh < 8; ++hh) qr[hh][0] = qr[hh][1] = qr[hh][2] = qr[hh][3] = 0.f;
+    auto add_row = [](float (&acc)[4], const uint2& w) {
+      const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&w.x);
+      const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&w.y);
+      acc[0] += __bfloat162float(p0.x);
+      acc[1] += __bfloat162float(p0.y);
+      acc[2] += __bfloat162float(p1.x);
+      acc[3] += __bfloat162float(p1.y);
+    };
+    const __nv_bfloat16* qg = q + (size_t)g * c.G * kD + lane * 4;
+    for (int r = 0; r < nrep; ++r) {
+      const __nv_bfloat16* row = qg + (size_t)(rep_tok[j * kMaxReps + r] - a.t0) * c.Hq * kD;
+      uint2 raw[8];
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh)
+        raw[hh] = hh < c.G ? *reinterpret_cast<const uint2*>(row + (size_t)hh * kD) : make_uint2(0u, 0u);
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh) add_row(qr[hh], raw[hh]);
+    }
+    float ug[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int hh = 0; hh < 8; ++hh)
+      if (hh < c.G) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) ug[e] += qr[hh][e];
+      }
+    for (int hh = 8; hh < c.G; ++hh) {  // groups wider than eight heads
+      float w[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int r = 0; r < nrep; ++r)
+        add_row(w, *reinterpret_cast<const uint2*>(qg + ((size_t)(rep_tok[j * kMaxReps + r] - a.t0) * c.Hq + hh) * kD));
+#pragma unroll
+      for (int e = 0; e < 4; ++e) ug[e] += w[e];
+    }
+    *reinterpret_cast<float4*>(c.u + (((size_t)layer * c.Hkv + g) * c.Jmax + j) * kD + lane * 4) =
+        make_float4(ug[0], ug[1], ug[2], ug[3]);
   }
 }
 
