@@ -7,7 +7,8 @@
 //   warps 0-7 / 8-15 : softmax of S0 / S1, two threads per row (64 columns each), P written back to TMEM as bf16
 //   warp 16          : TMA producer (Q once, K/V pieces through a 2-stage ring)
 //   warp 17          : MMA issuer: S = Q K^T (both operands in shared memory), O += P V (P from TMEM, V MN-major)
-// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P aliases the first 64 columns of its S.
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P (bf16) aliases columns [0,32) and [64,96) of
+// its S: every softmax thread overwrites only logit columns it has already read.
 // The issue order QK0, QK1, {PV0_j, QK0_j+1, PV1_j, QK1_j+1} keeps the tensor pipe busy with one tile's MMAs while
 // the other tile's softmax runs.  The running max is updated lazily (only when it grows by more than 2^8), in which
 // case the softmax thread rescales its O row in TMEM; the in-order tensor pipe guarantees the row is quiescent then.
@@ -145,8 +146,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
               long long v_row_offset) {
   const CUtensorMap* kvmaps = maps.kv;
   extern __shared__ unsigned char smem_raw[];
-  // QFULL QFREE ODONE | KFULL[2] VFULL[2] KEMPTY[2] VEMPTY[2] | SREADY[2] PREADY[2] OFREE[2]
-  __shared__ __align__(8) unsigned long long bars[3 + 8 + 6];
+  // QFULL QFREE ODONE | KFULL[2] VFULL[2] KEMPTY[2] VEMPTY[2] | SREADY[2] PREADY[2][2] OFREE[2]
+  __shared__ __align__(8) unsigned long long bars[3 + 8 + 8];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
   __shared__ RangeList rg;            // key ranges of the work item the producer is walking
@@ -166,7 +167,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   const uint32_t sKV = sbase + 65536;        // 2 stages x (K 32 KB | V 32 KB), each [half d][128 slots][64]
   enum {
     B_QFULL = 0, B_QFREE = 1, B_ODONE = 2, B_KFULL = 3, B_VFULL = 5, B_KEMPTY = 7, B_VEMPTY = 9, B_SREADY = 11,
-    B_PREADY = 13, B_OFREE = 15
+    B_PREADY = 13,  // + 2 * part + q: the two 32-column chunks of a thread's probabilities are handed over separately
+    B_OFREE = 17
   };
   auto bar = [&](int i) { return smem_addr(&bars[i]); };
   volatile int* abortp = &s_abort;
@@ -186,6 +188,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       mbar_init(bar(B_VEMPTY + s), 1);
       mbar_init(bar(B_SREADY + s), 1);
       mbar_init(bar(B_PREADY + s), 8);
+      mbar_init(bar(B_PREADY + 2 + s), 8);
       mbar_init(bar(B_OFREE + s), 8);
     }
     fence_mbar_init();
@@ -345,12 +348,17 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         }
         mma_commit(bar(B_SREADY + q));
       };
-      auto issue_pv = [&](int q, int st, bool acc) {
-        // 16 keys per step: 2 KB down the V tile; N = 128 spans both 64-wide halves (LBO = 16 KB)
+      auto issue_pv = [&](int q, int st, bool acc, int part) {
+        // 16 keys per step: 2 KB down the V tile; N = 128 spans both 64-wide halves (LBO = 16 KB).  Part 0 takes the
+        // key steps whose probabilities the softmax threads write first (keys [0,32) and [64,96)), part 1 the rest.
         const uint64_t db = dV + (uint64_t)((st * 65536) >> 4);
         const uint32_t d = tmem + 256 + q * 128, pa = tmem + q * 128;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) mma_ts(d, pa + ks * 8, db + ((ks * 2048) >> 4), idesc_pv, acc || ks > 0);
+        for (int i = 0; i < 4; ++i) {
+          const int ks = (i & 1) + 2 * part + 4 * (i >> 1);
+          // P of keys [64h, 64h+64) sits in the first 32 columns of column half h of the S buffer
+          mma_ts(d, pa + ks * 8 + (ks >> 2) * 32, db + ((ks * 2048) >> 4), idesc_pv, acc || part > 0 || i > 0);
+        }
       };
       int jt = 0;
       bool ok = true;
@@ -382,7 +390,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             if (!ok) break;
           }
           fence_after_sync();
-          issue_pv(0, st, acc);
+          issue_pv(0, st, acc, 0);
+          ok = mbar_wait(bar(B_PREADY + 2), jt & 1, abortp);
+          if (!ok) break;
+          fence_after_sync();
+          issue_pv(0, st, acc, 1);
           if (j + 1 < T) {
             ok = mbar_wait(bar(B_KFULL + nst), ((jt + 1) >> 1) & 1, abortp);
             if (!ok) break;
@@ -392,7 +404,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           ok = mbar_wait(bar(B_PREADY + 1), jt & 1, abortp);
           if (!ok) break;
           fence_after_sync();
-          issue_pv(1, st, acc);
+          issue_pv(1, st, acc, 0);
+          ok = mbar_wait(bar(B_PREADY + 3), jt & 1, abortp);
+          if (!ok) break;
+          fence_after_sync();
+          issue_pv(1, st, acc, 1);
           mma_commit(bar(B_VEMPTY + st));
           if (j + 1 < T) {
             issue_qk(1, nst);
@@ -407,16 +423,15 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
     // Two threads per row: warps 0-7 serve Q tile 0, warps 8-15 Q tile 1; inside a tile warps 0-3 take the columns
-    // [0,64) of S and O, warps 4-7 the columns [64,128).  The two halves of a row agree on the running maximum
-    // through shared memory and one named barrier per tile, after both have their S values in registers (so the
-    // P write-back, which aliases S, cannot clobber columns the other half still needs).
+    // [0,64) of S and O, warps 4-7 the columns [64,128).  A thread writes its probabilities over its own logit
+    // columns only, so the halves need no ordering between the loads of one and the stores of the other.
     const int q = warp >> 3;
     const int half = (warp >> 2) & 1;
     const int r = (warp & 3) * 32 + lane;        // row inside the 128-row tile = TMEM lane
     const int rr = q * 128 + r;                  // row inside the work item
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_base + q * 128 + half * 64;   // this thread's 64 logits
-    const uint32_t tP = tmem + lane_base + q * 128 + half * 32;   // its 64 probabilities (bf16 pairs)
+    const uint32_t tP = tS;  // its 64 probabilities (bf16 pairs) overwrite the first 32 of its own logit columns
     const uint32_t tO = tmem + lane_base + 256 + q * 128 + half * 64;
     const float c2 = c.scale * kLog2eT;
     int jt = 0;
@@ -575,12 +590,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             pk[e >> 1] = pack2(pp.x, pp.y);
           }
           tmem_st16(tP + ch * 16, pk);
+          // hand this chunk over: the P.V product starts on it while the other chunk's exponentials run
+          tmem_st_wait();
+          fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(B_PREADY + 2 * ch + q));
         }
         lsum += ls.x + ls.y;
-        tmem_st_wait();
-        fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(B_PREADY + q));
         ++j;
         ++jt;
       }
