@@ -21,16 +21,17 @@ __device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
 
 // grid (nsplit, Hkv, b.n*layer_count), 4 warps.  Each warp walks 16-token tiles of the CTA's slice of the virtual
 // token list (sink | selected spans | recent tokens): the tile's K and V rows (two contiguous 256-byte rows per
-// cp.async instruction, 16 bytes per lane) land in a warp-private, XOR-swizzled 3-stage ring; QK^T and PV run as
+// cp.async instruction, 16 bytes per lane) land in a warp-private, XOR-swizzled 2-stage ring; QK^T and PV run as
 // m16n8k16 tensor-core MMAs with the G query heads of the group in the first rows of the 16-row operand, so the
 // per-token ALU cost is a handful of instructions and the kernel stays bound by the K/V stream.
 // Partial results (m, l, O[128]) per (unit, head, split) go to dec_part.
 constexpr int kDTile = 16;
-constexpr int kDStages = 3;
+constexpr int kDStages = 2;     // two stages of 8 KB per warp: three CTAs (12 warps) fit an SM, which hides more latency
+constexpr int kDecCtasPerSm = 3;  // than a deeper ring at two CTAs per SM
 constexpr int kDWarpBytes = kDStages * 2 * kDTile * 256;  // K and V rows of every stage
 
 template <int G>
-__global__ void __launch_bounds__(kDecThreads, 2) k_decode_attn(DevCtx c, DecBatch b, int layer_begin, int layer_count,
+__global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevCtx c, DecBatch b, int layer_begin, int layer_count,
                                                                 const __nv_bfloat16* __restrict__ q, int nsplit) {
   extern __shared__ __align__(1024) unsigned char dsm[];
   __shared__ int rs[kMaxTopK + 2], rp[kMaxTopK + 3];

@@ -817,7 +817,8 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   __shared__ int s_ids[kMaxTopK];
   __shared__ int s_cnt;
   __shared__ int s_scan[512];
-  __shared__ int s_rs[kMaxTopK + 2], s_pre[kMaxTopK + 3], s_nr;  // merged ranges and their packed-row prefix
+  __shared__ int s_rs[kMaxTopK + 2], s_rl[kMaxTopK + 2], s_pre[kMaxTopK + 3], s_nr;  // merged ranges, packed-row prefix
+  __shared__ int s_sst[kMaxTopK], s_sln[kMaxTopK];  // extents of the selected spans
   const int g = blockIdx.x;
   int layer, sq, pos = 0, loc_begin = 0;
   if (DECODE) {
@@ -911,48 +912,55 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   __syncthreads();
   int* sel = c.sel + (unit * c.Hkv + g) * (size_t)c.topk;
   for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
+  // token ranges of the attention kernels: the spans' extents are fetched in parallel, merged (adjacent spans become
+  // one range) by one thread in shared memory and written out in parallel
+  if (tid < cnt) {
+    s_sst[tid] = c.span_start[unit * c.cap + s_ids[tid]];
+    s_sln[tid] = c.span_len[unit * c.cap + s_ids[tid]];
+  }
+  __syncthreads();
   if (tid == 0) {
-    const size_t rb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
-    int* rs = c.rng_start + rb;
-    int* rl = c.rng_len + rb;
     int nr = 0;
     long long tokens = 0;
     auto push = [&](int st, int ln) {
       if (ln <= 0) return;
-      if (nr > 0 && rs[nr - 1] + rl[nr - 1] == st)
-        rl[nr - 1] += ln;
+      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] == st)
+        s_rl[nr - 1] += ln;
       else {
-        rs[nr] = st;
-        rl[nr] = ln;
+        s_rs[nr] = st;
+        s_rl[nr] = ln;
         ++nr;
       }
     };
     if (DECODE) push(0, min(c.Ls, pos + 1));
     for (int t = 0; t < cnt; ++t) {
-      const int st = c.span_start[unit * c.cap + s_ids[t]], ln = c.span_len[unit * c.cap + s_ids[t]];
-      tokens += ln;
-      push(st, ln);
+      tokens += s_sln[t];
+      push(s_sst[t], s_sln[t]);
     }
     if (DECODE) push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
+    int run = 0;
+    for (int i = 0; i < nr; ++i) {
+      s_pre[i] = run;
+      run += s_rl[i];
+    }
+    s_pre[nr] = run;
+    s_nr = nr;
     c.rng_cnt[unit * c.Hkv + g] = nr;
     atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
-    if (!DECODE) {
-      int run = 0;
-      for (int i = 0; i < nr; ++i) {
-        s_rs[i] = rs[i];
-        s_pre[i] = run;
-        run += rl[i];
-      }
-      s_pre[nr] = run;
-      s_nr = nr;
-      c.gcnt[(size_t)layer * c.Hkv + g] = run;
+    if (!DECODE) c.gcnt[(size_t)layer * c.Hkv + g] = run;
+  }
+  __syncthreads();
+  {
+    const size_t rb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
+    for (int t = tid; t < s_nr; t += nt) {
+      c.rng_start[rb + t] = s_rs[t];
+      c.rng_len[rb + t] = s_rl[t];
     }
   }
   if (!DECODE) {
     // a5 gather: pack the K and V rows of the selected spans into one contiguous slab per (layer, KV head), so the
     // attention kernel that continues over them reads whole 128-row tiles.  16 threads per 256-byte row, four rows
     // of K and of V in flight per thread; the rows up to the next multiple of 8 are zero-filled.
-    __syncthreads();
     const int nr = s_nr, R = s_pre[nr], Rz = (R + 7) & ~7;
     const size_t slab = (unit * c.Hkv + g) * (size_t)c.Tpad;
     const uint4* Ksrc = reinterpret_cast<const uint4*>(c.Kc + slab * kD);
@@ -1004,6 +1012,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   __shared__ int s_ids[kMaxTopK];
   __shared__ int s_cnt;
   __shared__ int s_scan[1024];
+  __shared__ int s_rs[kMaxTopK + 2], s_rl[kMaxTopK + 2], s_nr, s_sst[kMaxTopK], s_sln[kMaxTopK];
   const int g = blockIdx.x;
   const int bi = blockIdx.y / layer_count, l = blockIdx.y % layer_count, layer = layer_begin + l;
   const int sq = b.seq[bi], pos = b.pos[bi], loc_begin = b.loc_begin[bi];
@@ -1028,16 +1037,21 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
 #pragma unroll
     for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
     const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + g) * (size_t)c.cap * kD + hl * 8;
-    for (int base = 0; base < N; base += 64 * 4) {  // uniform trip count (shuffles inside)
-      uint4 raw[4];
+    // software pipeline: the next four rows are in flight while the current four are reduced
+    auto fetch = [&](int base, uint4 (&raw)[4]) {
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const int s = base + t * 64 + hw;
         raw[t] = s < N ? __ldg(reinterpret_cast<const uint4*>(KR + (size_t)s * kD)) : make_uint4(0, 0, 0, 0);
       }
+    };
+    uint4 cur[4], nxt[4];
+    fetch(0, cur);
+    for (int base = 0; base < N; base += 64 * 4) {  // uniform trip count (shuffles inside)
+      fetch(base + 64 * 4, nxt);                    // past the end: zeros, no loads
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
-        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw[t]);
+        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&cur[t]);
         float d = 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -1052,6 +1066,8 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
         const int s = base + t * 64 + hw;
         if (hl == 0 && s < N) ssc[s] = d;
       }
+#pragma unroll
+      for (int t = 0; t < 4; ++t) cur[t] = nxt[t];
     }
   }
   __syncthreads();
@@ -1135,31 +1151,39 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   __syncthreads();
   int* sel = c.sel + (unit * c.Hkv + g) * (size_t)c.topk;
   for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
+  if (tid < cnt) {
+    s_sst[tid] = c.span_start[unit * c.cap + s_ids[tid]];
+    s_sln[tid] = c.span_len[unit * c.cap + s_ids[tid]];
+  }
+  __syncthreads();
   if (tid == 0) {
-    const size_t rbb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
-    int* rs = c.rng_start + rbb;
-    int* rl = c.rng_len + rbb;
     int nr = 0;
     long long tokens = 0;
     auto push = [&](int st, int ln) {
       if (ln <= 0) return;
-      if (nr > 0 && rs[nr - 1] + rl[nr - 1] == st)
-        rl[nr - 1] += ln;
+      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] == st)
+        s_rl[nr - 1] += ln;
       else {
-        rs[nr] = st;
-        rl[nr] = ln;
+        s_rs[nr] = st;
+        s_rl[nr] = ln;
         ++nr;
       }
     };
     push(0, min(c.Ls, pos + 1));
     for (int t = 0; t < cnt; ++t) {
-      const int st = c.span_start[unit * c.cap + s_ids[t]], ln = c.span_len[unit * c.cap + s_ids[t]];
-      tokens += ln;
-      push(st, ln);
+      tokens += s_sln[t];
+      push(s_sst[t], s_sln[t]);
     }
     push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
+    s_nr = nr;
     c.rng_cnt[unit * c.Hkv + g] = nr;
     atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+  }
+  __syncthreads();
+  const size_t rbb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
+  for (int t = tid; t < s_nr; t += nt) {
+    c.rng_start[rbb + t] = s_rs[t];
+    c.rng_len[rbb + t] = s_rl[t];
   }
 }
 

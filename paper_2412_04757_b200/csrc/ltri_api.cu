@@ -415,14 +415,14 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
       b.src[i] = i0 + i;
     }
     const int units = b.n * layer_count * d.Hkv;
-    // split count of the decode attention: two CTAs fit an SM, so the grid runs in waves of 2 x SMs CTAs.  Among
+    // split count of the decode attention: three CTAs fit an SM, so the grid runs in waves of 3 x SMs CTAs.  Among
     // the split counts that leave a CTA at least ~512 tokens (of the tokens known on the host: sink + everything
     // since the last eviction) take the one whose last wave is fullest; ties go to fewer, longer slices.
     int nsplit = 1;
     {
       const LayerState& s0 = ctx->at(seq_ids[i0], layer_begin);
       const long long known = d.Ls + (s0.t + 1 - s0.E);
-      const int wave = 2 * ctx->sm_count;
+      const int wave = 3 * ctx->sm_count;
       const int max_split = (int)std::max<long long>(1, std::min<long long>(kMaxDecSplit, known / 512));
       double best = -1.0;
       for (int ns = 1; ns <= max_split; ++ns) {
