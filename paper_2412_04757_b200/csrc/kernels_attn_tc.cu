@@ -295,8 +295,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             td.m1 = it.m1;
             td.m2 = it.m2;
             td.m3 = it.m3;
-            td.causal_tok0 = it.causal_tok0;
-            td.full = it.full ? 1 : 0;
+            // a tile of the current chunk that ends at or before the item's first token is visible to every row
+            const bool all_slots = (it.m0 & it.m1 & it.m2 & it.m3) == 0xffffffffu;
+            const bool below = it.causal_tok0 >= 0 && all_slots && it.causal_tok0 + 127 <= a.t0 + w.tok0;
+            td.causal_tok0 = below ? -1 : it.causal_tok0;
+            td.full = (it.full || below) ? 1 : 0;
             mbar_expect_tx(bar(B_KFULL + st), bytes);
           }
         }
