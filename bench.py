@@ -237,6 +237,16 @@ def run_reference(args, cfg):
 
 
 # ------------------------------------------------------------------------------------------------
+# DRAM traffic measured by Nsight Compute on small cases of the same kernels (summaries under profiles/), expressed per
+# unit so that it can be scaled to the launch this run times; traffic grows in proportion to these units.
+#  * local attention (k_attn_tc phase 0), Llama-3-8B geometry, chunk 512, window 4096 full, sink 64:
+#    101.85 MB for a 4-layer launch (profiles/k_attn_tc_cfg2_4layers_16k.md) -> bytes per layer of a launch
+ATTN_LOCAL_DRAM_BYTES_PER_LAYER = {(32, 8, 512, 4096, 64): 101.85e6 / 4}
+#  * decode retrieval + attention: 239.4 MB measured against 237.8 MB of algorithmic bytes for an 8-layer step at 64K
+#    (profiles/decode_kernels_cfg2_8layers_64k.md): every byte is read once, nothing is re-read
+DECODE_DRAM_PER_ALGORITHMIC_BYTE = 239.4 / 237.8
+
+
 def attn_local_flops(cfg, t0, n, E):
     """Algorithmic flops of the local attention kernel for one call (all layers): QK^T + PV over
     sink + local + causal current keys."""
@@ -386,7 +396,9 @@ def run_ltri(args, cfg):
                "roofline": {"bound": "hbm", "achieved": bytes_step * dsteps / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s",
                             "frac": (bytes_step * dsteps / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]) if k_ms > 0 else None,
-                            "traffic": None, "kernels": "decode score+top-k and split-KV attention+merge",
+                            "traffic": bytes_step * DECODE_DRAM_PER_ALGORITHMIC_BYTE,
+                            "traffic_note": "bytes per step, scaled from an ncu capture of an 8-layer 64K case",
+                            "kernels": "decode score+top-k and split-KV attention+merge",
                             "of": peaks["source"]},
                "kernel_ms_per_step": {k: v[0] / dsteps for k, v in dprof.items() if v[1]}}
         if recall is not None:
@@ -476,8 +488,13 @@ def run_ltri(args, cfg):
     a_ms, a_cnt = prof["attn_local"]
     tf = flops / (a_ms * 1e-3) / 1e12 if a_ms > 0 else None
     peak_tf = peaks["bf16_tflops_sustained"]
+    per_layer = ATTN_LOCAL_DRAM_BYTES_PER_LAYER.get((cfg.n_q_heads, cfg.n_kv_heads, cfg.chunk, cfg.window, cfg.n_sink))
+    window_full = chunks[first_timed][0] >= cfg.window + cfg.chunk
+    traffic = per_layer * L if per_layer and window_full else None
     roof = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
-            "frac": tf / peak_tf if tf else None, "traffic": None, "kernel": "k_attn_tc, local part (sink | local | current)",
+            "frac": tf / peak_tf if tf else None, "traffic": traffic,
+            "traffic_note": "DRAM bytes per launch, ncu capture of a 4-layer case of the same geometry x layers / 4",
+            "kernel": "k_attn_tc, local part (sink | local | current)",
             "launches": a_cnt, "ms_per_launch": a_ms / max(a_cnt, 1), "of": peaks["source"] + " (sustained)"}
     cpu = None
     if not args.no_cpu_baseline:
