@@ -1,6 +1,7 @@
-"""Parity at the benchmark's full size (128K tokens, 32 layers, the launch configuration bench.py times).
+"""Parity at the benchmark's full sizes (configs 1-4 as bench.py runs them: 32K and 128K x 32 layers, 1M x 8 layers,
+16 sequences x 128K x 4 layers).
 
-The oracle cannot stream 128K x 32 layers, so outputs are sampled: for two layers the oracle is brought to the
+The oracle cannot stream these, so outputs are sampled: for two layers the oracle is brought to the
 GPU's state at the start of a call (cache contents, span table, index, pending regions) and then computes that
 call itself -- local map, threshold, segmentation, query representatives, scores, top-k, attention rows -- which
 are compared with what the GPU produced for the same call.  A second check rebuilds the votes of one region over
@@ -16,8 +17,6 @@ from paper_2412_04757_b200 import binding, inputs
 from tests import parity_harness as ph
 
 pytestmark = pytest.mark.gpu
-LAYERS = [3, 29]
-ROWS = [0, 1, 255, 256, 510, 511]
 
 
 def regions_from_table(spans, lo, hi, chunk):
@@ -30,12 +29,24 @@ def regions_from_table(spans, lo, hi, chunk):
     return out
 
 
-def test_cfg2_sampled_calls_match_the_oracle():
-    cfg = inputs.config(2)
+# (config, sampled layers, sampled sequence): the 1M-token config keeps one layer on the host (4 GB of K/V)
+CASES = [(1, [0, 31], 0), (2, [3, 29], 0), (3, [5], 0), (4, [2], 11)]
+
+
+@pytest.mark.parametrize("cfg_idx,LAYERS,SEQ", CASES, ids=[f"cfg{c[0]}" for c in CASES])
+def test_sampled_calls_match_the_oracle(cfg_idx, LAYERS, SEQ):
+    cfg = inputs.config(cfg_idx)
     dev = torch.device("cuda:0")
-    st = inputs.SyntheticStream(cfg, device=dev)
     lt = binding.Ltri(ph.params_of(cfg), device=dev)
     L, n, W = cfg.n_layers, cfg.chunk, cfg.window
+    ROWS = [0, 1, n // 2 - 1, n // 2, n - 2, n - 1]
+    # the other sequences of a batched config are streamed first (they only have to be there for the decode batch)
+    others = [s for s in range(cfg.n_seqs) if s != SEQ]
+    for s in others:
+        so = inputs.SyntheticStream(cfg, seq=s, device=dev)
+        for (t0, cnt) in so.prefill_chunks():
+            lt.ltri_prefill_chunk(s, 0, L, *so.tokens(t0, cnt))
+    st = inputs.SyntheticStream(cfg, seq=SEQ, device=dev)
     chunks = list(st.prefill_chunks())
     K = {l: [] for l in LAYERS}
     V = {l: [] for l in LAYERS}
@@ -45,7 +56,7 @@ def test_cfg2_sampled_calls_match_the_oracle():
     out_last = None
     for ci, (t0, cnt) in enumerate(chunks):
         q, k, v = st.tokens(t0, cnt)
-        out = lt.ltri_prefill_chunk(0, 0, L, q, k, v)
+        out = lt.ltri_prefill_chunk(SEQ, 0, L, q, k, v)
         for l in LAYERS:
             K[l].append(k[l].cpu())
             V[l].append(v[l].cpu())
@@ -59,12 +70,12 @@ def test_cfg2_sampled_calls_match_the_oracle():
     rep = ph.Report()
     for l in LAYERS:
         Kall, Vall = torch.cat(K[l]), torch.cat(V[l])
-        spans_g = lt.ltri_get_spans(0, l)
-        idx_g = lt.ltri_debug_read(binding.BUF_INDEX, 0, l)[:, :len(spans_g)].transpose(1, 0, 2).copy()
-        stats = lt.ltri_get_stats(0, l)
+        spans_g = lt.ltri_get_spans(SEQ, l)
+        idx_g = lt.ltri_debug_read(binding.BUF_INDEX, SEQ, l)[:, :len(spans_g)].transpose(1, 0, 2).copy()
+        stats = lt.ltri_get_stats(SEQ, l)
         E = int(stats.evicted_end)
         assert E == t0_last - W and spans_g[-1, 0] + spans_g[-1, 1] == E
-        pend_g = lt.ltri_get_pending_spans(0, l)
+        pend_g = lt.ltri_get_pending_spans(SEQ, l)
         what = f"layer {l} last call"
         # ---- the last prefill call, recomputed by the oracle from the GPU's state at its start -------------
         o = ph.oracle_of(cfg)
@@ -74,9 +85,9 @@ def test_cfg2_sampled_calls_match_the_oracle():
             o.add_pending(rs, re, sp)
         o.prefill_local(Q[l][len(chunks) - 1], Kall[t0_last:], Vall[t0_last:])
         rs, m = o.region()
-        Mg = np.tril(lt.ltri_debug_read(binding.BUF_MAP, 0, l)[:m, :m])
+        Mg = np.tril(lt.ltri_debug_read(binding.BUF_MAP, SEQ, l)[:m, :m])
         assert np.abs(Mg.astype(np.int64) - o.map()).max() <= 4 + cfg.n_q_heads, f"{what}: region map"
-        thg = int(lt.ltri_debug_read(binding.BUF_THETA, 0, l)[0])
+        thg = int(lt.ltri_debug_read(binding.BUF_THETA, SEQ, l)[0])
         assert abs(thg - o.theta_q()) <= 4 + cfg.n_q_heads
         newest_g = pend_g[pend_g[:, 0] >= rs]
         ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region)
@@ -88,10 +99,10 @@ def test_cfg2_sampled_calls_match_the_oracle():
             rep.span_flips += 1
         o.prefill_retrieve()
         ns = len(spans_g)
-        sg = lt.ltri_debug_read(binding.BUF_SCORES, 0, l)[:, :ns]
+        sg = lt.ltri_debug_read(binding.BUF_SCORES, SEQ, l)[:, :ns]
         so = o.scores()
         assert np.abs(sg - so).max() / np.abs(so).max() <= 2e-5, f"{what}: scores"
-        ph.check_selection(lt.ltri_get_selected(0, l), o, rep, what)
+        ph.check_selection(lt.ltri_get_selected(SEQ, l), o, rep, what)
         for r in ROWS:
             ref = o.prefill_attend(r, r + 1)
             ph.check_output(out_last[l, r:r + 1], ref, rep, f"{what} row {r}")
@@ -129,17 +140,24 @@ def test_cfg2_sampled_calls_match_the_oracle():
                 assert len(vo) > 1 and (vo[0] - vo[1]) <= ph.NEAR_TIE * max(vo[0], 1.0), \
                     f"layer {l}: index vector of span {gs} differs"
                 rep.index_flips += 1
-    # ---- decode continues from the same state --------------------------------------------------------------
+    # ---- decode continues from the same state (all sequences of the config in one batch) --------------------
+    if cfg.decode_steps < 3:
+        lt.close()
+        return
+    streams = {s: inputs.SyntheticStream(cfg, seq=s, device=dev) for s in others}
+    streams[SEQ] = st
+    ids = list(range(cfg.n_seqs))
+    pos = ids.index(SEQ)
     for s in range(3):
-        q, k, v = st.tokens(cfg.context + s, 1, kind=1)
-        qd, kd, vd = (x.permute(1, 0, 2, 3).contiguous() for x in (q, k, v))
-        out = lt.ltri_decode_step([0], 0, L, qd, kd, vd)
+        parts = [streams[i].tokens(cfg.context + s, 1, kind=1) for i in ids]
+        qd, kd, vd = (torch.cat([pp[j].permute(1, 0, 2, 3) for pp in parts]).contiguous() for j in range(3))
+        out = lt.ltri_decode_step(ids, 0, L, qd, kd, vd)
         torch.cuda.synchronize()
         for l in LAYERS:
             o = snap[l]
-            o.decode_retrieve(qd[0, l].cpu(), kd[0, l].cpu(), vd[0, l].cpu())
-            ph.check_selection(lt.ltri_get_selected(0, l), o, rep, f"layer {l} decode {s}")
-            ph.check_output(out[0, l], o.decode_attend(), rep, f"layer {l} decode {s}")
+            o.decode_retrieve(qd[pos, l].cpu(), kd[pos, l].cpu(), vd[pos, l].cpu())
+            ph.check_selection(lt.ltri_get_selected(SEQ, l), o, rep, f"layer {l} decode {s}")
+            ph.check_output(out[pos, l], o.decode_attend(), rep, f"layer {l} decode {s}")
     assert lt.ltri_sync_status() == 0
     assert rep.span_flips <= 1 and rep.sel_flips <= 4 and rep.index_flips <= 2
     print(rep)
