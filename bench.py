@@ -197,7 +197,8 @@ def oracle_sample(cfg, steps, warmup):
     need = (fill + warmup + steps) * cfg.chunk
     o = orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
                          need + 8, reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
-                         theta_mode=cfg.theta_mode, theta=cfg.theta)
+                         theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind,
+                         min_reps=cfg.min_reps, max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda)
     times = []
     for ci in range(fill + warmup + steps):
         q, k, v = st.tokens(ci * cfg.chunk, cfg.chunk)
@@ -303,7 +304,9 @@ def run_ltri(args, cfg):
     SQ = NSEQ - 1
     p = binding.make_params(L, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_tokens, cfg.chunk, cfg.window, cfg.n_sink,
                             cfg.top_k, head_dim=cfg.head_dim, max_seqs=NSEQ, reps_per_span=cfg.reps_per_span,
-                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta)
+                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
+                            rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
+                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda)
 
     def stream_until(lt, upto, keep_from):
         for s in range(NSEQ - 1):
@@ -527,6 +530,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling of small cases)")
     ap.add_argument("--context", type=int, default=0, help="override the context length (profiling of small cases)")
     ap.add_argument("--decode-steps", type=int, default=-1, help="override the number of decode steps")
+    ap.add_argument("--dynamic-reps", action="store_true",
+                    help="dynamic span index vectors (rep_mode 1, both neighbours, lambda 2, 1..4 per span)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -536,6 +541,10 @@ def main():
         cfg = dataclasses.replace(cfg, n_layers=args.layers or cfg.n_layers, context=args.context or cfg.context,
                                   decode_steps=cfg.decode_steps if args.decode_steps < 0 else args.decode_steps)
         cfg.name += f"[layers={cfg.n_layers},context={cfg.context},decode={cfg.decode_steps}]"
+    if args.dynamic_reps:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, rep_mode=1, ratio_kind=2, rep_lambda=2.0, min_reps=1, max_reps=4)
+        cfg.name += "[dynamic-reps]"
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -59,6 +59,16 @@ typedef struct {
   float theta;                                       /* mode 1 default 0.90 */
   float softmax_scale;                               /* 0 -> 1/sqrt(head_dim) */
   uint32_t flags;                                    /* LTRI_FLAG_* */
+  /* Dynamic span index vectors (Sec. 3.3.2, Eq. r_v).  rep_mode 0: every span keeps reps_per_span representatives.
+   * rep_mode 1: a span of L tokens keeps round(L * exp(-rep_lambda * (1 - r_a))) of them, clamped to
+   * [min_reps, max_reps] and to L, where r_a = T / (T + neighbours) on the call's head-summed Q20 region map: T is
+   * the mass of the span's own triangle; the neighbours are the mass its rows give to earlier tokens of the region
+   * (ratio_kind 0, "row"), the mass later rows of the region give to its columns (1, "column"), or both (2).  The
+   * same count is used for the query side while the region is current and for the key side when it is indexed. */
+  int32_t rep_mode;                                  /* 0 static, 1 dynamic */
+  int32_t ratio_kind;                                /* 0 row, 1 column, 2 both */
+  int32_t min_reps, max_reps;                        /* 1 <= min_reps <= max_reps <= 8 (rep_mode 1 only) */
+  float rep_lambda;                                  /* >= 0 (rep_mode 1 only) */
   void* arena;                                       /* caller-owned device memory, 256-byte aligned */
   size_t arena_bytes;                                /* >= ltri_arena_bytes(params) */
 } ltri_params;
@@ -166,6 +176,8 @@ enum {
   LTRI_BUF_THETA = 4,    /* int64 [1]: theta of the last prefill call in Q20 head-sum units */
   LTRI_BUF_SCORES = 5,   /* float [n_kv_heads][span_capacity]: similarity scores of the last call (Eq. 7) */
   LTRI_BUF_QREPS = 6,    /* float [n_kv_heads][2*max_spans_per_region+1][head_dim]: summed query representatives */
+  LTRI_BUF_NREPS = 8,    /* int32 [2*max_spans_per_region+1]: representative counts of the spans of the last prefill
+                            call's region (Sec. 3.3.2) */
   LTRI_BUF_ROWSTAT = 7   /* float [chunk][n_q_heads][2]: reference maximum m (logits * scale * log2(e); may lag the true
                             row maximum by up to 8) and the matching row sum of exp2(logit - m) of the local softmax
                             of the last prefill call */

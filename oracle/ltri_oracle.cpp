@@ -67,6 +67,7 @@ inline uint16_t f32_to_bf16_rne(float f) {
 
 struct Span {
   int start, len;
+  int nrep = 0;  // number of representative tokens (0: not decided yet -> static count)
 };
 
 struct Region {
@@ -82,6 +83,10 @@ struct Params {
   float theta;
   float softmax_scale;
   int64_t max_tokens;
+  // dynamic span index vectors (Sec. 3.3.2): rep_mode 0 = static count reps_per_span, 1 = count from the area ratio
+  int32_t rep_mode, ratio_kind;  // ratio_kind 0: row neighbours, 1: column neighbours, 2: both
+  int32_t min_reps, max_reps;
+  float rep_lambda;
 };
 
 // ---------------------------------------------------------------------------
@@ -101,6 +106,32 @@ int64_t theta_q(const int32_t* Mq, int m, int ld, int mode, float theta, int Hq)
   if (rank > N - 1) rank = N - 1;
   std::nth_element(vals.begin(), vals.begin() + rank, vals.end());
   return vals[(size_t)rank];
+}
+
+// Sec. 3.3.2 (dynamic span index vectors), written out from its definition on the raw region map:
+// T = mass of the span's own triangle, R = mass its rows give to earlier tokens of the region ("row neighbours"),
+// C = mass later rows of the region give to its columns ("column neighbours").  r_a = T / (T + neighbours) for the
+// chosen kind (1 when there is no mass at all), r_v = 1 / e^(lambda (1 - r_a)) (Eq. r_v), and the span keeps
+// round(len * r_v) representatives, clamped to [min_reps, max_reps] and to the span length.  All sums are integers;
+// the ratio, the exponential and the rounding (to nearest even) are taken in double precision.
+int dynamic_rep_count(const int32_t* Mq, int m, int ld, int x, int y, int kind, double lambda, int min_reps,
+                      int max_reps) {
+  int64_t T = 0, R = 0, Cn = 0;
+  for (int i = x; i <= y; ++i) {
+    for (int j = 0; j < x; ++j) R += Mq[(size_t)i * ld + j];
+    for (int j = x; j <= i; ++j) T += Mq[(size_t)i * ld + j];
+  }
+  for (int i = y + 1; i < m; ++i)
+    for (int j = x; j <= y; ++j) Cn += Mq[(size_t)i * ld + j];
+  const int64_t nb = kind == 0 ? R : kind == 1 ? Cn : R + Cn;
+  const double ra = (T + nb) > 0 ? (double)T / (double)(T + nb) : 1.0;
+  const double rv = 1.0 / std::exp(lambda * (1.0 - ra));
+  const int len = y - x + 1;
+  int cnt = (int)std::nearbyint((double)len * rv);
+  cnt = std::max(cnt, min_reps);
+  cnt = std::min(cnt, max_reps);
+  cnt = std::min(cnt, len);
+  return std::max(cnt, 1);
 }
 
 // Eq. 4-5 by the two cumulative sums of Fig. 2: S(x,y) = sum_{x<=j<=i<=y} (Mq[i][j]-theta).
@@ -300,9 +331,21 @@ struct Stream {
     t += cnt;
   }
 
+  int rep_stride() const { return p.rep_mode == 1 ? std::max(p.max_reps, 1) : p.reps_per_span; }
+  // representative counts of the spans of the newest region (the region map of the current call is still there)
+  void decide_rep_counts(Region& reg) const {
+    for (Span& s : reg.spans) {
+      if (p.rep_mode == 1)
+        s.nrep = dynamic_rep_count(Mq.data(), m, m, s.start - reg_start, s.start - reg_start + s.len - 1, p.ratio_kind,
+                                   (double)p.rep_lambda, p.min_reps, p.max_reps);
+      else
+        s.nrep = std::min(p.reps_per_span, s.len);
+    }
+  }
+
   // tokens of [lo,hi) with the largest votes, ties -> lower index; returned ascending.
-  std::vector<int> rep_tokens(int lo, int len) const {
-    int cnt = std::min(p.reps_per_span, len);
+  std::vector<int> rep_tokens(int lo, int len, int nrep) const {
+    int cnt = std::min(nrep > 0 ? nrep : p.reps_per_span, len);
     std::vector<int> idx(len);
     for (int i = 0; i < len; ++i) idx[i] = lo + i;
     std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) { return votes[a] > votes[b]; });
@@ -369,7 +412,7 @@ struct Stream {
     while (!pending.empty() && pending.front().end <= t0_ - p.window) {
       Region& r = pending.front();
       for (const Span& s : r.spans) {
-        std::vector<int> reps = rep_tokens(s.start, s.len);
+        std::vector<int> reps = rep_tokens(s.start, s.len, s.nrep);
         size_t base = KR.size();
         KR.resize(base + (size_t)Hkv * d);
         for (int g = 0; g < Hkv; ++g)
@@ -467,6 +510,7 @@ struct Stream {
       segment_map(Mq.data(), m, m, thq, p.max_spans_per_region, sp, &seg_gap);
       for (Span& s : sp) s.start += reg_start;
       reg.spans = sp;
+      decide_rep_counts(reg);
       pending.push_back(reg);
     } else {
       thq = 0;
@@ -484,10 +528,10 @@ struct Stream {
       const Region& reg = pending.back();
       J = (int)reg.spans.size();
       u.assign((size_t)Hkv * J * d, 0.f);
-      qrep_tok.assign((size_t)J * p.reps_per_span, -1);
+      qrep_tok.assign((size_t)J * rep_stride(), -1);
       for (int j = 0; j < J; ++j) {
-        std::vector<int> reps = rep_tokens(reg.spans[j].start, reg.spans[j].len);
-        for (size_t r = 0; r < reps.size(); ++r) qrep_tok[(size_t)j * p.reps_per_span + r] = reps[r];
+        std::vector<int> reps = rep_tokens(reg.spans[j].start, reg.spans[j].len, reg.spans[j].nrep);
+        for (size_t r = 0; r < reps.size(); ++r) qrep_tok[(size_t)j * rep_stride() + r] = reps[r];
         for (int g = 0; g < Hkv; ++g)
           for (int e = 0; e < d; ++e) {
             float ug = 0.f;
@@ -626,6 +670,10 @@ void* orc_create(const Params* p) {
   if (!p || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads) return nullptr;
   if (p->head_dim < 1 || p->chunk < 1 || p->window < 1 || p->n_sink < 1 || p->top_k < 1) return nullptr;
   if (p->reps_per_span < 1 || p->max_spans_per_region < 1 || p->max_tokens < 1) return nullptr;
+  if (p->rep_mode != 0 && p->rep_mode != 1) return nullptr;
+  if (p->rep_mode == 1 && (p->ratio_kind < 0 || p->ratio_kind > 2 || p->min_reps < 1 || p->max_reps < p->min_reps ||
+                           !(p->rep_lambda >= 0.f)))
+    return nullptr;
   return new Stream(*p);
 }
 void orc_destroy(void* h) { delete (Stream*)h; }
@@ -696,7 +744,31 @@ int orc_set_newest_spans(void* h, const int* start_len, int cnt) {
   if (pos != reg.end) return -1;
   reg.spans.clear();
   for (int i = 0; i < cnt; ++i) reg.spans.push_back(Span{start_len[2 * i], start_len[2 * i + 1]});
+  if (s->m > 0 && reg.start == s->reg_start) s->decide_rep_counts(reg);
   return 0;
+}
+// representative counts of the newest pending region's spans
+int orc_get_newest_rep_counts(void* h, int* out, int cap) {
+  Stream* s = (Stream*)h;
+  if (s->pending.empty()) return 0;
+  const Region& reg = s->pending.back();
+  int c = (int)reg.spans.size();
+  for (int i = 0; i < c && i < cap; ++i) out[i] = reg.spans[i].nrep > 0 ? reg.spans[i].nrep : std::min(s->p.reps_per_span, reg.spans[i].len);
+  return c;
+}
+// overwrite the representative counts of the newest region's spans (re-synchronisation after a tolerated rounding flip)
+int orc_set_newest_rep_counts(void* h, const int* counts, int cnt) {
+  Stream* s = (Stream*)h;
+  if (s->pending.empty() || (int)s->pending.back().spans.size() != cnt) return -1;
+  for (int i = 0; i < cnt; ++i) {
+    if (counts[i] < 1 || counts[i] > s->pending.back().spans[i].len) return -1;
+    s->pending.back().spans[i].nrep = counts[i];
+  }
+  return 0;
+}
+int orc_rep_stride(void* h) { return ((Stream*)h)->rep_stride(); }
+int orc_dynamic_rep_count(const int32_t* Mq, int m, int x, int y, int kind, double lambda, int min_reps, int max_reps) {
+  return dynamic_rep_count(Mq, m, m, x, y, kind, lambda, min_reps, max_reps);
 }
 void orc_get_votes(void* h, int lo, int hi, int64_t* out) {
   Stream* s = (Stream*)h;

@@ -33,6 +33,8 @@ class _Params(C.Structure):
         ("reps_per_span", C.c_int32), ("max_spans_per_region", C.c_int32),
         ("theta_mode", C.c_int32), ("theta", C.c_float), ("softmax_scale", C.c_float),
         ("max_tokens", C.c_int64),
+        ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
+        ("rep_lambda", C.c_float),
     ]
 
 
@@ -80,6 +82,14 @@ def lib():
         L.orc_ta_scores.argtypes = [vp, ip, i64, vp]
         L.orc_segment_map.argtypes = [vp, ip, i64, ip, vp, ip, vp]
         L.orc_top_k.argtypes = [vp, ip, ip, vp, vp]
+        L.orc_get_newest_rep_counts.argtypes = [vp, vp, ip]
+        L.orc_get_newest_rep_counts.restype = ip
+        L.orc_set_newest_rep_counts.argtypes = [vp, vp, ip]
+        L.orc_set_newest_rep_counts.restype = ip
+        L.orc_rep_stride.argtypes = [vp]
+        L.orc_rep_stride.restype = ip
+        L.orc_dynamic_rep_count.argtypes = [vp, ip, ip, ip, ip, C.c_double, ip, ip]
+        L.orc_dynamic_rep_count.restype = ip
         L.orc_f32_to_bf16.argtypes = [C.c_float]
         L.orc_f32_to_bf16.restype = C.c_uint16
         _lib = L
@@ -105,14 +115,16 @@ class OracleStream:
     """The oracle for one (sequence, layer) stream."""
 
     def __init__(self, n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, max_tokens,
-                 reps_per_span=1, max_spans_per_region=None, theta_mode=1, theta=0.90, softmax_scale=0.0):
+                 reps_per_span=1, max_spans_per_region=None, theta_mode=1, theta=0.90, softmax_scale=0.0,
+                 rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0):
         if max_spans_per_region is None:
             max_spans_per_region = max(1, chunk // 32)
         self.Hq, self.Hkv, self.d = n_q_heads, n_kv_heads, head_dim
         self.top_k, self.reps = top_k, reps_per_span
         self.chunk, self.window, self.n_sink = chunk, window, n_sink
         self._p = _Params(n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, reps_per_span,
-                          max_spans_per_region, theta_mode, theta, softmax_scale, max_tokens)
+                          max_spans_per_region, theta_mode, theta, softmax_scale, max_tokens,
+                          rep_mode, ratio_kind, min_reps, max_reps, rep_lambda)
         self._h = lib().orc_create(C.byref(self._p))
         if not self._h:
             raise ValueError("bad oracle parameters")
@@ -265,10 +277,21 @@ class OracleStream:
 
     def query_rep_tokens(self) -> np.ndarray:
         J = lib().orc_num_query_reps(self._h)
-        a = np.full((J, self.reps), -1, dtype=np.int32)
+        a = np.full((J, lib().orc_rep_stride(self._h)), -1, dtype=np.int32)
         if J and lib().orc_region_len(self._h) > 0:
             lib().orc_get_query_rep_tokens(self._h, _ptr(a))
         return a
+
+    def newest_rep_counts(self) -> np.ndarray:
+        """Representative counts of the newest pending region's spans (Sec. 3.3.2 when rep_mode = 1)."""
+        a = np.zeros(4096, dtype=np.int32)
+        n = lib().orc_get_newest_rep_counts(self._h, _ptr(a), len(a))
+        return a[:n].copy()
+
+    def set_newest_rep_counts(self, counts):
+        a = np.ascontiguousarray(np.asarray(counts, dtype=np.int32))
+        if lib().orc_set_newest_rep_counts(self._h, _ptr(a), len(a)):
+            raise ValueError("representative counts do not fit the newest region")
 
     def scores(self) -> np.ndarray:
         n = lib().orc_num_spans(self._h)
@@ -289,6 +312,12 @@ class OracleStream:
 
 
 # --- stateless pieces ---------------------------------------------------------
+def dynamic_rep_count(Mq: np.ndarray, x: int, y: int, kind: int, lam: float, min_reps: int, max_reps: int) -> int:
+    """Representative count of the span [x, y] of a region map (Sec. 3.3.2, Eq. r_v)."""
+    Mq = np.ascontiguousarray(Mq, dtype=np.int32)
+    return int(lib().orc_dynamic_rep_count(_ptr(Mq), Mq.shape[0], x, y, kind, float(lam), min_reps, max_reps))
+
+
 def theta_q(Mq: np.ndarray, mode: int, theta: float, n_q_heads: int) -> int:
     Mq = np.ascontiguousarray(Mq, dtype=np.int32)
     return int(lib().orc_theta_q(_ptr(Mq), Mq.shape[0], mode, theta, n_q_heads))

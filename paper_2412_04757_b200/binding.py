@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libltri.so")
 
 LTRI_OK, LTRI_EINVAL, LTRI_ECAPACITY, LTRI_ESTATE, LTRI_ECUDA, LTRI_EDEVICE, LTRI_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
-BUF_MAP, BUF_VOTES, BUF_INDEX, BUF_THETA, BUF_SCORES, BUF_QREPS, BUF_ROWSTAT = 1, 2, 3, 4, 5, 6, 7
+BUF_MAP, BUF_VOTES, BUF_INDEX, BUF_THETA, BUF_SCORES, BUF_QREPS, BUF_ROWSTAT, BUF_NREPS = 1, 2, 3, 4, 5, 6, 7, 8
 
 EXPORTS = [
     "ltri_arena_bytes", "ltri_create", "ltri_destroy", "ltri_reset_sequence", "ltri_prefill_chunk",
@@ -35,6 +35,8 @@ class LtriParams(C.Structure):
         ("chunk", C.c_int32), ("window", C.c_int32), ("n_sink", C.c_int32), ("top_k", C.c_int32),
         ("reps_per_span", C.c_int32), ("max_spans_per_region", C.c_int32),
         ("theta_mode", C.c_int32), ("theta", C.c_float), ("softmax_scale", C.c_float), ("flags", C.c_uint32),
+        ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
+        ("rep_lambda", C.c_float),
         ("arena", C.c_void_p), ("arena_bytes", C.c_size_t),
     ]
 
@@ -96,9 +98,11 @@ def strerror(code: int) -> str:
 
 
 def make_params(n_layers, n_q_heads, n_kv_heads, max_tokens, chunk, window, n_sink, top_k, head_dim=128, max_seqs=1,
-                reps_per_span=1, max_spans_per_region=0, theta_mode=1, theta=0.90, softmax_scale=0.0) -> LtriParams:
+                reps_per_span=1, max_spans_per_region=0, theta_mode=1, theta=0.90, softmax_scale=0.0,
+                rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0) -> LtriParams:
     return LtriParams(n_layers, n_q_heads, n_kv_heads, head_dim, max_seqs, max_tokens, chunk, window, n_sink, top_k,
-                      reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, 0, None, 0)
+                      reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, 0,
+                      rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, None, 0)
 
 
 def ltri_arena_bytes(params: LtriParams) -> int:
@@ -269,6 +273,8 @@ class Ltri:
             return raw.view(np.float32).reshape(p.n_kv_heads, cap)
         if what == BUF_QREPS:
             return raw.view(np.float32).reshape(p.n_kv_heads, 2 * C_ + 1, p.head_dim)
+        if what == BUF_NREPS:
+            return raw.view(np.int32)
         if what == BUF_ROWSTAT:
             return raw.view(np.float32).reshape(p.chunk, p.n_q_heads, 2)
         return raw

@@ -26,6 +26,8 @@ struct DevCtx {
   int chunk, W, Ls, topk, reps, C, Jmax, cap, slots;
   int theta_mode;
   float theta, scale;
+  int rep_mode, ratio_kind, min_reps, max_reps;  // dynamic span index vectors (Sec. 3.3.2); rep_mode 0: static count
+  float rep_lambda;
   // persistent state
   __nv_bfloat16* Kc;     // [NS][NL][Hkv][Tpad][128]
   __nv_bfloat16* Vc;
@@ -37,6 +39,7 @@ struct DevCtx {
   int* pend_start;       // [NS][NL][slots][Jmax]
   int* pend_len;
   int* pend_cnt;         // [NS][NL][slots]
+  int* pend_nrep;        // [NS][NL][slots][Jmax]  representative count of every pending span
   int* sel;              // [NS][NL][Hkv][topk]  ascending ids, -1 padded
   long long* sel_tokens; // [NS][NL]  retrieved tokens of the last call, summed over KV heads
   // per-layer scratch of the prefill call in flight
@@ -54,6 +57,7 @@ struct DevCtx {
   int* gcnt;             // [NL][Hkv]             packed rows (retrieved tokens) per KV head
   long long Rcap;        // row capacity of a packed slab: top_k spans of at most `chunk` tokens, rounded up
   int* Jcnt;             // [NL]
+  int* nrep_last;        // [NL][Jmax]  representative counts of the spans of the call in flight
   // per-(seq,layer) scratch
   float* scores;         // [NS*NL][Hkv][cap]
   int* rng_start;        // [NS*NL][Hkv][topk+2]

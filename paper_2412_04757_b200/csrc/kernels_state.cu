@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(256) k_evict_index(DevCtx c, EvictArgs a) {
         c.span_len[unit * c.cap + dst] = len;
       }
       int toks[kMaxReps];
-      const int nrep = select_reps(votes, start, len, c.reps, toks);
+      const int nrep = select_reps(votes, start, len, c.rep_mode == 1 ? c.pend_nrep[ps + i] : c.reps, toks);
       for (int g = 0; g < c.Hkv; ++g) {
         const __nv_bfloat16* kslab = c.Kc + ((unit * c.Hkv + g) * c.Tpad) * kD;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -590,7 +590,6 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
     c.pend_cnt[unit * c.slots + a.slot] = nout;
     c.Jcnt[layer] = a.q ? nout : 0;
   }
-  if (!a.q) return;
   // query representatives.  First one warp per span picks the representative tokens, then one warp per
   // (span, KV head) sums their query rows with all loads of the head group in flight at once.
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
@@ -599,9 +598,49 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   int* rep_tok = reinterpret_cast<int*>(skey);          // [Jmax][kMaxReps], the sort buffer is free now
   int* rep_cnt = rep_tok + (2 * kMaxTopK + 1) * kMaxReps;
   __syncthreads();
+  // representative count of every span: static, or from the area ratio of Sec. 3.3.2 on the raw region map.  The
+  // row-suffix table holds sums of (Mq - theta), so a raw sum over w entries is the table value + theta * w.
+  int* nrep_of = rep_cnt + (2 * kMaxTopK + 1);
+  for (int j = warp; j < nout; j += nwarps) {
+    int cnt = min(c.reps, out_len[j]);
+    if (c.rep_mode == 1) {
+      const long long* Rs = c.Rsuf + (size_t)layer * c.chunk * c.chunk;
+      const long long th = c.thetaq[layer];
+      const int x = out_start[j], y = x + out_len[j] - 1;
+      long long T = 0, TR = 0, Cn = 0;
+      for (int i = x + lane; i <= y; i += 32) {
+        T += Rs[(size_t)i * c.chunk + x] + th * (i - x + 1);
+        TR += Rs[(size_t)i * c.chunk] + th * (i + 1);
+      }
+      for (int i = y + 1 + lane; i < m; i += 32)
+        Cn += Rs[(size_t)i * c.chunk + x] - Rs[(size_t)i * c.chunk + y + 1] + th * (y - x + 1);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        T += shfl_xor_ll(T, o);
+        TR += shfl_xor_ll(TR, o);
+        Cn += shfl_xor_ll(Cn, o);
+      }
+      const long long R = TR - T;
+      const long long nb = c.ratio_kind == 0 ? R : c.ratio_kind == 1 ? Cn : R + Cn;
+      const double ra = (T + nb) > 0 ? (double)T / (double)(T + nb) : 1.0;
+      const double rv = 1.0 / exp((double)c.rep_lambda * (1.0 - ra));
+      cnt = (int)rint((double)out_len[j] * rv);  // to nearest even
+      cnt = max(cnt, c.min_reps);
+      cnt = min(cnt, c.max_reps);
+      cnt = min(cnt, out_len[j]);
+      cnt = max(cnt, 1);
+    }
+    if (lane == 0) {
+      nrep_of[j] = cnt;
+      if (c.pend_nrep) c.pend_nrep[ps + j] = cnt;  // (absent in the scratch-only context of the static entry)
+      if (c.nrep_last) c.nrep_last[(size_t)layer * c.Jmax + j] = cnt;
+    }
+  }
+  __syncthreads();
+  if (!a.q) return;
   for (int j = warp; j < nout; j += nwarps) {
     int toks[kMaxReps];
-    const int nrep = select_reps(votes, a.reg_start + out_start[j], out_len[j], c.reps, toks);
+    const int nrep = select_reps(votes, a.reg_start + out_start[j], out_len[j], nrep_of[j], toks);
     if (lane == 0) {
       rep_cnt[j] = nrep;
       for (int r = 0; r < nrep; ++r) rep_tok[j * kMaxReps + r] = toks[r];

@@ -57,6 +57,12 @@ bool validate(const ltri_params* p) {
   if (p->theta_mode != 0 && p->theta_mode != 1) return false;
   if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
   if (!(p->softmax_scale >= 0.f)) return false;
+  if (p->rep_mode != 0 && p->rep_mode != 1) return false;
+  if (p->rep_mode == 1) {
+    if (p->ratio_kind < 0 || p->ratio_kind > 2) return false;
+    if (p->min_reps < 1 || p->max_reps < p->min_reps || p->max_reps > kMaxReps) return false;
+    if (!(p->rep_lambda >= 0.f)) return false;
+  }
   return true;
 }
 
@@ -80,6 +86,11 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.cap = (int)std::min<long long>((long long)1 << 30, ((p.max_tokens + p.chunk - 1) / p.chunk + 8) * d.Jmax);
   d.theta_mode = p.theta_mode;
   d.theta = p.theta;
+  d.rep_mode = p.rep_mode;
+  d.ratio_kind = p.ratio_kind;
+  d.min_reps = p.min_reps;
+  d.max_reps = p.max_reps;
+  d.rep_lambda = p.rep_lambda;
   d.scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / std::sqrt((float)kD);
   const size_t units = (size_t)d.NS * d.NL;
   Carver cv{base};
@@ -93,6 +104,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.pend_start = cv.take<int>(units * (d.slots + 1) * d.Jmax);
   d.pend_len = cv.take<int>(units * (d.slots + 1) * d.Jmax);
   d.pend_cnt = cv.take<int>(units * (d.slots + 1));
+  d.pend_nrep = cv.take<int>(units * (d.slots + 1) * d.Jmax);
   d.sel = cv.take<int>(units * d.Hkv * d.topk);
   d.sel_tokens = cv.take<long long>(units);
   d.Mq = cv.take<int>((size_t)d.NL * d.chunk * d.chunk);
@@ -105,6 +117,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.Oacc = cv.take<float>((size_t)d.NL * align_up((size_t)d.chunk * d.G, 256) * d.Hkv * kD);
   d.u = cv.take<float>((size_t)d.NL * d.Hkv * d.Jmax * kD);
   d.Jcnt = cv.take<int>(d.NL);
+  d.nrep_last = cv.take<int>((size_t)d.NL * d.Jmax);
   d.Rcap = (long long)align_up((size_t)d.topk * d.chunk, 128) + kTokPad;
   d.Kg = cv.take<__nv_bfloat16>((size_t)d.NL * d.Hkv * d.Rcap * kD);
   d.Vg = cv.take<__nv_bfloat16>((size_t)d.NL * d.Hkv * d.Rcap * kD);
@@ -644,6 +657,10 @@ int ltri_debug_read(ltri_ctx* ctx, int what, int seq, int layer, void* dst, size
     case LTRI_BUF_QREPS:
       src = d.u + (size_t)layer * d.Hkv * d.Jmax * kD;
       bytes = (size_t)d.Hkv * d.Jmax * kD * sizeof(float);
+      break;
+    case LTRI_BUF_NREPS:
+      src = d.nrep_last + (size_t)layer * d.Jmax;
+      bytes = (size_t)d.Jmax * sizeof(int);
       break;
     case LTRI_BUF_ROWSTAT:
       src = d.rowstat + (size_t)layer * d.chunk * d.Hq;

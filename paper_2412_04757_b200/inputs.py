@@ -60,6 +60,11 @@ class StreamConfig:
     theta_mode: int = 1
     theta: float = 0.90
     seed: int = 2412047570
+    rep_mode: int = 0      # 1: dynamic representative counts (Sec. 3.3.2)
+    ratio_kind: int = 2
+    min_reps: int = 1
+    max_reps: int = 4
+    rep_lambda: float = 2.0
 
     @property
     def max_tokens(self) -> int:

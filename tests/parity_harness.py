@@ -40,19 +40,25 @@ class Report:
     max_map_diff: int = 0
     max_theta_diff: int = 0
     max_score_rel: float = 0.0
+    rep_counts: int = 0
+    rep_count_flips: int = 0
 
 
 def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
     return binding.make_params(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_tokens, cfg.chunk, cfg.window,
                                cfg.n_sink, cfg.top_k, head_dim=cfg.head_dim, max_seqs=max_seqs or cfg.n_seqs,
                                reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
-                               theta_mode=cfg.theta_mode, theta=cfg.theta)
+                               theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode,
+                               ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps, max_reps=cfg.max_reps,
+                               rep_lambda=cfg.rep_lambda)
 
 
 def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
     return orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
                             cfg.max_tokens, reps_per_span=cfg.reps_per_span,
-                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta)
+                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
+                            rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
+                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda)
 
 
 def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str):
@@ -105,6 +111,7 @@ class StreamPair:
         self.orc = {(s, l): oracle_of(cfg) for s in self.seqs for l in self.layers}
         self.rep = Report()
         self.n_indexed = {(s, l): 0 for s in self.seqs for l in self.layers}
+        self.count_of = {}   # (seq, layer, span start) -> representative count decided when its region was current
 
     # ---- one prefill call -------------------------------------------------------------------
     def prefill(self, seq, q, k, v, check_out=True):
@@ -148,6 +155,24 @@ class StreamPair:
                         f"{what}: spans differ and the oracle's smallest decisive gap is {o.seg_gap():.3g}")
                     rep.span_flips += 1
                     o.set_newest_spans(newest_g)
+                # representative counts of the region's spans (Sec. 3.3.2 when rep_mode = 1)
+                J = len(newest_g)
+                ng = lt.ltri_debug_read(binding.BUF_NREPS, seq, layer)[:J]
+                no = o.newest_rep_counts()
+                rep.rep_counts += J
+                if cfg.rep_mode == 1 and self.deep:
+                    # integer sums, one division, one exponential, one rounding: the same on the GPU's own map
+                    ref = [orc.dynamic_rep_count(Mg, int(st - rs), int(st - rs + ln - 1), cfg.ratio_kind, cfg.rep_lambda,
+                                                 cfg.min_reps, cfg.max_reps) for st, ln in newest_g]
+                    assert ng.tolist() == ref, f"{what}: representative counts differ on the GPU's own map"
+                if ng.tolist() != no.tolist():
+                    # the two maps differ by a few Q20 units: a count may flip by one where len * r_v is near .5
+                    assert cfg.rep_mode == 1 and int(np.abs(ng - no).max()) <= 1, (
+                        f"{what}: representative counts {ng.tolist()} vs {no.tolist()}")
+                    rep.rep_count_flips += int((ng != no).sum())
+                    o.set_newest_rep_counts(ng)
+                for (st, ln), c in zip(newest_g, ng):
+                    self.count_of[(seq, layer, int(st))] = int(c)
             if self.deep:
                 vg = lt.ltri_debug_read(binding.BUF_VOTES, seq, layer)[:t1].astype(np.float64)
                 vo = o.votes(0, t1).astype(np.float64)
@@ -189,7 +214,8 @@ class StreamPair:
             st, ln = spans_o[s]
             vo = o.votes(int(st), int(st + ln)).astype(np.float64)
             top = np.sort(vo)[::-1]
-            assert self.cfg.reps_per_span < ln and (top[self.cfg.reps_per_span - 1] - top[self.cfg.reps_per_span]) <= \
+            cnt = self.count_of.get((seq, layer, int(st)), self.cfg.reps_per_span)
+            assert cnt < ln and (top[cnt - 1] - top[cnt]) <= \
                 NEAR_TIE * max(top[0], 1.0), f"{what}: index vector of span {s} differs"
             self.rep.index_flips += 1
         self.n_indexed[(seq, layer)] = len(spans_o)

@@ -48,6 +48,17 @@ def test_three_representatives_per_span_and_absolute_theta():
     print(rep)
 
 
+@pytest.mark.parametrize("kind,lam,lo,hi", [(0, 1.0, 1, 4), (1, 2.0, 1, 8), (2, 0.7, 2, 6)])
+def test_dynamic_representative_counts(kind, lam, lo, hi):
+    # Sec. 3.3.2: the number of index vectors of a span follows its area ratio; checked per region against the oracle
+    # (counts, then the query representatives, index vectors, scores, selections and outputs that depend on them)
+    cfg = small_cfg(n_layers=2, context=1280, decode_steps=3, rep_mode=1, ratio_kind=kind, rep_lambda=lam,
+                    min_reps=lo, max_reps=hi)
+    rep = ph.run_stream(cfg, layers=[0, 1])
+    assert rep.rep_counts > 50 and rep.rep_count_flips <= 2
+    print(rep)
+
+
 def test_top_k_covering_everything_equals_full_attention():
     # with top_k >= number of spans the streamed output is plain causal attention (oracle O12)
     cfg = small_cfg(n_layers=1, context=640, chunk=64, window=128, top_k=64, max_spans_per_region=2, decode_steps=2)
