@@ -306,7 +306,8 @@ def run_ltri(args, cfg):
                             cfg.top_k, head_dim=cfg.head_dim, max_seqs=NSEQ, reps_per_span=cfg.reps_per_span,
                             max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
-                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda)
+                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
+                            flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0)
 
     def stream_until(lt, upto, keep_from):
         for s in range(NSEQ - 1):
@@ -532,6 +533,8 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=-1, help="override the number of decode steps")
     ap.add_argument("--dynamic-reps", action="store_true",
                     help="dynamic span index vectors (rep_mode 1, both neighbours, lambda 2, 1..4 per span)")
+    ap.add_argument("--persist-decode", action="store_true",
+                    help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -545,6 +548,10 @@ def main():
         import dataclasses
         cfg = dataclasses.replace(cfg, rep_mode=1, ratio_kind=2, rep_lambda=2.0, min_reps=1, max_reps=4)
         cfg.name += "[dynamic-reps]"
+    if args.persist_decode:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, persist_decode=True)
+        cfg.name += "[persist-decode]"
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -73,7 +73,12 @@ typedef struct {
   size_t arena_bytes;                                /* >= ltri_arena_bytes(params) */
 } ltri_params;
 
-enum { LTRI_FLAG_NONE = 0 };
+enum {
+  LTRI_FLAG_NONE = 0,
+  /* Persistent mechanism (Sec. 3.5): the spans selected by the last prefill call of a sequence stay in the attention
+   * of every decode step, next to the spans the step retrieves itself. */
+  LTRI_FLAG_PERSIST_DECODE = 1
+};
 
 typedef struct {
   int64_t tokens;          /* tokens appended so far (prefill + decode) */

@@ -87,6 +87,8 @@ struct Params {
   int32_t rep_mode, ratio_kind;  // ratio_kind 0: row neighbours, 1: column neighbours, 2: both
   int32_t min_reps, max_reps;
   float rep_lambda;
+  // persistent mechanism (Sec. 3.5): decode keeps the spans selected by the last prefill call
+  int32_t persist_decode;
 };
 
 // ---------------------------------------------------------------------------
@@ -298,6 +300,7 @@ struct Stream {
   int J = 0;
   std::vector<float> score;  // [Hkv][Ns]
   std::vector<int> sel;      // [Hkv][top_k]
+  std::vector<int> persist;  // [Hkv][top_k] selection of the last prefill call, kept through decode (Sec. 3.5)
   std::vector<double> cut_gap;  // [Hkv]
   std::vector<int> qrep_tok;    // [J][reps] absolute tokens, -1 padded
 
@@ -575,10 +578,19 @@ struct Stream {
   std::vector<std::pair<int, int>> key_ranges(int g, int sink_end, int loc_begin, int loc_end) const {
     std::vector<std::pair<int, int>> ranges;
     ranges.push_back({0, sink_end});
+    // the spans selected now (rank order) and, in a decode step under the persistent mechanism, those the last
+    // prefill call selected that are not among them; every span once
+    std::vector<int> ids;
     for (int i = 0; i < p.top_k; ++i) {
       int s = sel[(size_t)g * p.top_k + i];
-      if (s >= 0) ranges.push_back({spans[s].start, spans[s].start + spans[s].len});
+      if (s >= 0) ids.push_back(s);
     }
+    if (decoding && p.persist_decode && !persist.empty())
+      for (int i = 0; i < p.top_k; ++i) {
+        int s = persist[(size_t)g * p.top_k + i];
+        if (s >= 0 && std::find(ids.begin(), ids.end(), s) == ids.end()) ids.push_back(s);
+      }
+    for (int s : ids) ranges.push_back({spans[s].start, spans[s].start + spans[s].len});
     ranges.push_back({loc_begin, loc_end});
     return ranges;
   }
@@ -615,6 +627,7 @@ struct Stream {
   // O11: retrieval part of a decode step.
   int decode_retrieve(const uint16_t* qb, const uint16_t* kb, const uint16_t* vb) {
     if ((int64_t)t + 1 > p.max_tokens) return -2;
+    if (!decoding && p.persist_decode) persist = sel;  // what the last prefill call retrieved (may be empty)
     decoding = true;
     t0 = t;
     n = 1;
@@ -800,6 +813,11 @@ void orc_get_selected(void* h, int* ids, double* gaps) {  // [Hkv][top_k], [Hkv]
   Stream* s = (Stream*)h;
   std::memcpy(ids, s->sel.data(), s->sel.size() * sizeof(int));
   if (gaps) std::memcpy(gaps, s->cut_gap.data(), s->cut_gap.size() * sizeof(double));
+}
+// [Hkv][top_k] span ids kept through decode by the persistent mechanism (-1 padded; all -1 before the first decode step)
+void orc_get_persistent(void* h, int* ids) {
+  Stream* s = (Stream*)h;
+  for (size_t i = 0; i < s->sel.size(); ++i) ids[i] = i < s->persist.size() ? s->persist[i] : -1;
 }
 void orc_set_selected(void* h, const int* ids) {
   Stream* s = (Stream*)h;

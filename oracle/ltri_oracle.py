@@ -34,7 +34,7 @@ class _Params(C.Structure):
         ("theta_mode", C.c_int32), ("theta", C.c_float), ("softmax_scale", C.c_float),
         ("max_tokens", C.c_int64),
         ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
-        ("rep_lambda", C.c_float),
+        ("rep_lambda", C.c_float), ("persist_decode", C.c_int32),
     ]
 
 
@@ -84,6 +84,7 @@ def lib():
         L.orc_top_k.argtypes = [vp, ip, ip, vp, vp]
         L.orc_get_newest_rep_counts.argtypes = [vp, vp, ip]
         L.orc_get_newest_rep_counts.restype = ip
+        L.orc_get_persistent.argtypes = [vp, vp]
         L.orc_set_newest_rep_counts.argtypes = [vp, vp, ip]
         L.orc_set_newest_rep_counts.restype = ip
         L.orc_rep_stride.argtypes = [vp]
@@ -116,7 +117,7 @@ class OracleStream:
 
     def __init__(self, n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, max_tokens,
                  reps_per_span=1, max_spans_per_region=None, theta_mode=1, theta=0.90, softmax_scale=0.0,
-                 rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0):
+                 rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, persist_decode=0):
         if max_spans_per_region is None:
             max_spans_per_region = max(1, chunk // 32)
         self.Hq, self.Hkv, self.d = n_q_heads, n_kv_heads, head_dim
@@ -124,7 +125,7 @@ class OracleStream:
         self.chunk, self.window, self.n_sink = chunk, window, n_sink
         self._p = _Params(n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, reps_per_span,
                           max_spans_per_region, theta_mode, theta, softmax_scale, max_tokens,
-                          rep_mode, ratio_kind, min_reps, max_reps, rep_lambda)
+                          rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, persist_decode)
         self._h = lib().orc_create(C.byref(self._p))
         if not self._h:
             raise ValueError("bad oracle parameters")
@@ -305,6 +306,12 @@ class OracleStream:
         gaps = np.zeros(self.Hkv, dtype=np.float64)
         lib().orc_get_selected(self._h, _ptr(ids), _ptr(gaps))
         return ids, gaps
+
+    def persistent(self) -> np.ndarray:
+        """Span ids [Hkv][top_k] kept through decode by the persistent mechanism (-1 padded)."""
+        ids = np.zeros((self.Hkv, self.top_k), dtype=np.int32)
+        lib().orc_get_persistent(self._h, _ptr(ids))
+        return ids
 
     def set_selected(self, ids):
         a = np.ascontiguousarray(np.asarray(ids, dtype=np.int32).reshape(self.Hkv, self.top_k))

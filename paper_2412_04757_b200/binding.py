@@ -15,6 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libltri.so")
 
 LTRI_OK, LTRI_EINVAL, LTRI_ECAPACITY, LTRI_ESTATE, LTRI_ECUDA, LTRI_EDEVICE, LTRI_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+FLAG_PERSIST_DECODE = 1
 BUF_MAP, BUF_VOTES, BUF_INDEX, BUF_THETA, BUF_SCORES, BUF_QREPS, BUF_ROWSTAT, BUF_NREPS = 1, 2, 3, 4, 5, 6, 7, 8
 
 EXPORTS = [
@@ -99,9 +100,9 @@ def strerror(code: int) -> str:
 
 def make_params(n_layers, n_q_heads, n_kv_heads, max_tokens, chunk, window, n_sink, top_k, head_dim=128, max_seqs=1,
                 reps_per_span=1, max_spans_per_region=0, theta_mode=1, theta=0.90, softmax_scale=0.0,
-                rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0) -> LtriParams:
+                rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, flags=0) -> LtriParams:
     return LtriParams(n_layers, n_q_heads, n_kv_heads, head_dim, max_seqs, max_tokens, chunk, window, n_sink, top_k,
-                      reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, 0,
+                      reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, flags,
                       rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, None, 0)
 
 

@@ -14,6 +14,7 @@ constexpr float kQScale = 1048576.0f;
 constexpr int kMaxReps = 8;
 constexpr int kMaxTopK = 64;
 constexpr int kMaxDecSplit = 32;
+constexpr int kMaxRanges = 2 * kMaxTopK + 2;  // sink + local + the spans of this step's and of the persistent selection
 constexpr float kMapMargin = 0.0078125f;          // safety margin (in log2 units) of the map pass's skip test
 constexpr float kMapScale = 0.4972997117f;         // 2^-(1 + kMapMargin)
 constexpr int kTokPad = 128;          // rows of slack after every K/V slab so tile over-reads stay inside it
@@ -24,6 +25,8 @@ struct DevCtx {
   long long Tpad;        // row capacity of a per-(seq,layer,kv-head) K/V slab (max_tokens + slack)
   long long Tmax;
   int chunk, W, Ls, topk, reps, C, Jmax, cap, slots;
+  int rcap;              // token ranges kept per (seq, layer, KV head): 2 * top_k + 2
+  int persist;           // decode keeps the spans selected by the last prefill call (Sec. 3.5, persistent mechanism)
   int theta_mode;
   float theta, scale;
   int rep_mode, ratio_kind, min_reps, max_reps;  // dynamic span index vectors (Sec. 3.3.2); rep_mode 0: static count
@@ -41,6 +44,7 @@ struct DevCtx {
   int* pend_cnt;         // [NS][NL][slots]
   int* pend_nrep;        // [NS][NL][slots][Jmax]  representative count of every pending span
   int* sel;              // [NS][NL][Hkv][topk]  ascending ids, -1 padded
+  int* persist_sel;      // [NS][NL][Hkv][topk]  selection of the last prefill call, kept through decode
   long long* sel_tokens; // [NS][NL]  retrieved tokens of the last call, summed over KV heads
   // per-layer scratch of the prefill call in flight
   int* Mq;               // [NL][chunk][chunk]
@@ -60,7 +64,7 @@ struct DevCtx {
   int* nrep_last;        // [NL][Jmax]  representative counts of the spans of the call in flight
   // per-(seq,layer) scratch
   float* scores;         // [NS*NL][Hkv][cap]
-  int* rng_start;        // [NS*NL][Hkv][topk+2]
+  int* rng_start;        // [NS*NL][Hkv][rcap]
   int* rng_len;
   int* rng_cnt;          // [NS*NL][Hkv]
   float* dec_part;       // [NS*NL][Hq][kMaxDecSplit][128+2]

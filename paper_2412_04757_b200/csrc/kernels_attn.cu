@@ -41,8 +41,8 @@ __global__ void __launch_bounds__(256, 1) k_attn_prefill(DevCtx c, PrefillArgs a
       rg.start[2] = a.t0;
       rg.len[2] = last_tok + 1;  // causal range: keys up to the tile's last token
     } else {
-      const size_t rb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
-      const int nr = min(c.rng_cnt[unit * c.Hkv + g], c.topk + 2);
+      const size_t rb = (unit * c.Hkv + g) * (size_t)c.rcap;
+      const int nr = min(c.rng_cnt[unit * c.Hkv + g], kMaxTopK + 2);
       rg.n = nr;
       for (int i = 0; i < nr; ++i) {
         rg.start[i] = c.rng_start[rb + i];

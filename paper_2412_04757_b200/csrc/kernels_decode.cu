@@ -34,15 +34,15 @@ template <int G>
 __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevCtx c, DecBatch b, int layer_begin, int layer_count,
                                                                 const __nv_bfloat16* __restrict__ q, int nsplit) {
   extern __shared__ __align__(1024) unsigned char dsm[];
-  __shared__ int rs[kMaxTopK + 2], rp[kMaxTopK + 3];
+  __shared__ int rs[kMaxRanges], rp[kMaxRanges + 1];
   __shared__ float sm_m[4][G], sm_l[4][G];
   __shared__ float sm_o[4][G][kD];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int split = blockIdx.x, g = blockIdx.y;
   const int bi = blockIdx.z / layer_count, l = blockIdx.z % layer_count, layer = layer_begin + l;
   const size_t unit = unit_of(c, b.seq[bi], layer);
-  const size_t rb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
-  const int nr = min(c.rng_cnt[unit * c.Hkv + g], c.topk + 2);
+  const size_t rb = (unit * c.Hkv + g) * (size_t)c.rcap;
+  const int nr = min(c.rng_cnt[unit * c.Hkv + g], c.rcap);
   if (tid == 0) {
     int run = 0;
     for (int i = 0; i < nr; ++i) {

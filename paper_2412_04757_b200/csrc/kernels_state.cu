@@ -19,7 +19,10 @@ __global__ void k_init(DevCtx c, int seq) {
       c.sel_tokens[u0 + i] = 0;
     }
     for (size_t i = tid; i < (size_t)c.NL * c.slots; i += stride) c.pend_cnt[u0 * c.slots + i] = 0;
-    for (size_t i = tid; i < (size_t)c.NL * c.Hkv * c.topk; i += stride) c.sel[u0 * c.Hkv * c.topk + i] = -1;
+    for (size_t i = tid; i < (size_t)c.NL * c.Hkv * c.topk; i += stride) {
+      c.sel[u0 * c.Hkv * c.topk + i] = -1;
+      c.persist_sel[u0 * c.Hkv * c.topk + i] = -1;
+    }
     for (size_t i = tid; i < (size_t)c.NL * c.Hkv; i += stride) c.rng_cnt[u0 * c.Hkv + i] = 0;
   }
   if (seq < 0 && tid < 4) c.status[tid] = 0;
@@ -844,6 +847,35 @@ cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_be
 // a4 top-k (Eq. 8 with unit = span): the min(k, N_s) largest scores, ties -> lower span id.  4-pass radix select on
 // order-preserving keys, then an id-ordered pick of the threshold ties.  Writes the ascending id list and the token
 // ranges the attention kernels walk (adjacent spans merged).  One CTA per (unit, KV head).
+// Union of this step's selection (s_ids[0..cnt), ascending) with the selection the last prefill call left in
+// persist_sel (ascending, -1 padded): the persistent mechanism of Sec. 3.5.  Writes the ascending, duplicate-free id
+// list to s_all and returns its length.  Called by every thread of the CTA; s_tmp has room for kMaxTopK ints.
+__device__ __forceinline__ int union_with_persistent(const DevCtx& c, size_t unit, int g, const int* s_ids, int cnt,
+                                                     int* s_tmp, int* s_all, int* s_nall) {
+  const int tid = threadIdx.x;
+  if (tid < c.topk) s_tmp[tid] = c.persist ? c.persist_sel[(unit * c.Hkv + g) * (size_t)c.topk + tid] : -1;
+  __syncthreads();
+  if (tid == 0) {
+    int a = 0, b = 0, n = 0;
+    while (b < c.topk && s_tmp[b] < 0) ++b;  // (-1 padding sits at the end, but tolerate it anywhere)
+    while (a < cnt || b < c.topk) {
+      const int va = a < cnt ? s_ids[a] : 0x7fffffff;
+      const int vb = b < c.topk && s_tmp[b] >= 0 ? s_tmp[b] : 0x7fffffff;
+      if (va == 0x7fffffff && vb == 0x7fffffff) break;
+      const int v = va < vb ? va : vb;
+      s_all[n++] = v;
+      if (va == v) ++a;
+      if (vb == v) {
+        ++b;
+        while (b < c.topk && s_tmp[b] < 0) ++b;
+      }
+    }
+    *s_nall = n;
+  }
+  __syncthreads();
+  return *s_nall;
+}
+
 __device__ __forceinline__ unsigned order_key(float f) {
   const unsigned u = __float_as_uint(f);
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
@@ -856,8 +888,9 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   __shared__ int s_ids[kMaxTopK];
   __shared__ int s_cnt;
   __shared__ int s_scan[512];
-  __shared__ int s_rs[kMaxTopK + 2], s_rl[kMaxTopK + 2], s_pre[kMaxTopK + 3], s_nr;  // merged ranges, packed-row prefix
-  __shared__ int s_sst[kMaxTopK], s_sln[kMaxTopK];  // extents of the selected spans
+  __shared__ int s_rs[kMaxRanges], s_rl[kMaxRanges], s_pre[kMaxRanges + 1], s_nr;  // merged ranges, packed-row prefix
+  __shared__ int s_sst[2 * kMaxTopK], s_sln[2 * kMaxTopK];  // extents of the selected spans
+  __shared__ int s_all[2 * kMaxTopK], s_nall;            // decode: this step's selection united with the persistent one
   const int g = blockIdx.x;
   int layer, sq, pos = 0, loc_begin = 0;
   if (DECODE) {
@@ -953,9 +986,15 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
   // token ranges of the attention kernels: the spans' extents are fetched in parallel, merged (adjacent spans become
   // one range) by one thread in shared memory and written out in parallel
-  if (tid < cnt) {
-    s_sst[tid] = c.span_start[unit * c.cap + s_ids[tid]];
-    s_sln[tid] = c.span_len[unit * c.cap + s_ids[tid]];
+  const int* ids_all = s_ids;
+  int nall = cnt;
+  if (DECODE && c.persist) {
+    nall = union_with_persistent(c, unit, g, s_ids, cnt, s_scan, s_all, &s_nall);
+    ids_all = s_all;
+  }
+  if (tid < nall) {
+    s_sst[tid] = c.span_start[unit * c.cap + ids_all[tid]];
+    s_sln[tid] = c.span_len[unit * c.cap + ids_all[tid]];
   }
   __syncthreads();
   if (tid == 0) {
@@ -972,7 +1011,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
       }
     };
     if (DECODE) push(0, min(c.Ls, pos + 1));
-    for (int t = 0; t < cnt; ++t) {
+    for (int t = 0; t < nall; ++t) {
       tokens += s_sln[t];
       push(s_sst[t], s_sln[t]);
     }
@@ -990,7 +1029,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   }
   __syncthreads();
   {
-    const size_t rb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
+    const size_t rb = (unit * c.Hkv + g) * (size_t)c.rcap;
     for (int t = tid; t < s_nr; t += nt) {
       c.rng_start[rb + t] = s_rs[t];
       c.rng_len[rb + t] = s_rl[t];
@@ -1051,7 +1090,8 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   __shared__ int s_ids[kMaxTopK];
   __shared__ int s_cnt;
   __shared__ int s_scan[1024];
-  __shared__ int s_rs[kMaxTopK + 2], s_rl[kMaxTopK + 2], s_nr, s_sst[kMaxTopK], s_sln[kMaxTopK];
+  __shared__ int s_rs[kMaxRanges], s_rl[kMaxRanges], s_nr, s_sst[2 * kMaxTopK], s_sln[2 * kMaxTopK];
+  __shared__ int s_all[2 * kMaxTopK], s_nall;
   const int g = blockIdx.x;
   const int bi = blockIdx.y / layer_count, l = blockIdx.y % layer_count, layer = layer_begin + l;
   const int sq = b.seq[bi], pos = b.pos[bi], loc_begin = b.loc_begin[bi];
@@ -1190,9 +1230,15 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   __syncthreads();
   int* sel = c.sel + (unit * c.Hkv + g) * (size_t)c.topk;
   for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
-  if (tid < cnt) {
-    s_sst[tid] = c.span_start[unit * c.cap + s_ids[tid]];
-    s_sln[tid] = c.span_len[unit * c.cap + s_ids[tid]];
+  const int* ids_all = s_ids;
+  int nall = cnt;
+  if (c.persist) {
+    nall = union_with_persistent(c, unit, g, s_ids, cnt, s_scan, s_all, &s_nall);
+    ids_all = s_all;
+  }
+  if (tid < nall) {
+    s_sst[tid] = c.span_start[unit * c.cap + ids_all[tid]];
+    s_sln[tid] = c.span_len[unit * c.cap + ids_all[tid]];
   }
   __syncthreads();
   if (tid == 0) {
@@ -1209,7 +1255,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
       }
     };
     push(0, min(c.Ls, pos + 1));
-    for (int t = 0; t < cnt; ++t) {
+    for (int t = 0; t < nall; ++t) {
       tokens += s_sln[t];
       push(s_sst[t], s_sln[t]);
     }
@@ -1219,7 +1265,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
   }
   __syncthreads();
-  const size_t rbb = (unit * c.Hkv + g) * (size_t)(c.topk + 2);
+  const size_t rbb = (unit * c.Hkv + g) * (size_t)c.rcap;
   for (int t = tid; t < s_nr; t += nt) {
     c.rng_start[rbb + t] = s_rs[t];
     c.rng_len[rbb + t] = s_rl[t];

@@ -57,6 +57,7 @@ bool validate(const ltri_params* p) {
   if (p->theta_mode != 0 && p->theta_mode != 1) return false;
   if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
   if (!(p->softmax_scale >= 0.f)) return false;
+  if (p->flags & ~(uint32_t)LTRI_FLAG_PERSIST_DECODE) return false;
   if (p->rep_mode != 0 && p->rep_mode != 1) return false;
   if (p->rep_mode == 1) {
     if (p->ratio_kind < 0 || p->ratio_kind > 2) return false;
@@ -79,6 +80,8 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.W = p.window;
   d.Ls = p.n_sink;
   d.topk = p.top_k;
+  d.rcap = 2 * p.top_k + 2;
+  d.persist = (p.flags & LTRI_FLAG_PERSIST_DECODE) ? 1 : 0;
   d.reps = p.reps_per_span > 0 ? p.reps_per_span : 1;
   d.C = p.max_spans_per_region > 0 ? p.max_spans_per_region : std::max(1, p.chunk / 32);
   d.Jmax = 2 * d.C + 1;
@@ -106,6 +109,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.pend_cnt = cv.take<int>(units * (d.slots + 1));
   d.pend_nrep = cv.take<int>(units * (d.slots + 1) * d.Jmax);
   d.sel = cv.take<int>(units * d.Hkv * d.topk);
+  d.persist_sel = cv.take<int>(units * d.Hkv * d.topk);
   d.sel_tokens = cv.take<long long>(units);
   d.Mq = cv.take<int>((size_t)d.NL * d.chunk * d.chunk);
   d.Rsuf = cv.take<long long>((size_t)d.NL * d.chunk * d.chunk);
@@ -123,8 +127,8 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.Vg = cv.take<__nv_bfloat16>((size_t)d.NL * d.Hkv * d.Rcap * kD);
   d.gcnt = cv.take<int>((size_t)d.NL * d.Hkv);
   d.scores = cv.take<float>(units * d.Hkv * d.cap);
-  d.rng_start = cv.take<int>(units * d.Hkv * (d.topk + 2));
-  d.rng_len = cv.take<int>(units * d.Hkv * (d.topk + 2));
+  d.rng_start = cv.take<int>(units * d.Hkv * d.rcap);
+  d.rng_len = cv.take<int>(units * d.Hkv * d.rcap);
   d.rng_cnt = cv.take<int>(units * d.Hkv);
   d.dec_part = cv.take<float>(units * d.Hq * kMaxDecSplit * (kD + 2));
   d.status = cv.take<int>(4);
@@ -417,6 +421,19 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
   const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
   const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
   __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(out);
+  // persistent mechanism: before a sequence's first decode step overwrites the selection of its last prefill call,
+  // that selection is set aside; every decode step then attends over it as well
+  if (d.persist) {
+    for (int i = 0; i < n_seqs; ++i) {
+      const int sq = seq_ids[i];
+      for (int l = 0; l < layer_count; ++l) {
+        if (ctx->at(sq, layer_begin + l).decoding) continue;
+        const size_t off = unit_of(d, sq, layer_begin + l) * d.Hkv * (size_t)d.topk;
+        LTRI_CUDA(ctx, cudaMemcpyAsync(d.persist_sel + off, d.sel + off, (size_t)d.Hkv * d.topk * sizeof(int),
+                                       cudaMemcpyDeviceToDevice, st));
+      }
+    }
+  }
   for (int i0 = 0; i0 < n_seqs; i0 += kDecBatch) {
     DecBatch b;
     b.n = std::min(kDecBatch, n_seqs - i0);

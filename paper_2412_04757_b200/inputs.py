@@ -65,6 +65,7 @@ class StreamConfig:
     min_reps: int = 1
     max_reps: int = 4
     rep_lambda: float = 2.0
+    persist_decode: bool = False   # decode keeps the spans selected by the last prefill call (Sec. 3.5)
 
     @property
     def max_tokens(self) -> int:

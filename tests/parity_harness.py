@@ -50,7 +50,7 @@ def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
                                reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
                                theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode,
                                ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps, max_reps=cfg.max_reps,
-                               rep_lambda=cfg.rep_lambda)
+                               rep_lambda=cfg.rep_lambda, flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0)
 
 
 def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
@@ -58,7 +58,7 @@ def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
                             cfg.max_tokens, reps_per_span=cfg.reps_per_span,
                             max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
-                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda)
+                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda, persist_decode=int(cfg.persist_decode))
 
 
 def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str):
@@ -238,6 +238,17 @@ class StreamPair:
                 o.decode_retrieve(q[i, layer], k[i, layer], v[i, layer])
                 if len(o.spans()):
                     check_selection(lt.ltri_get_selected(seq, layer), o, rep, what)
+                    # tokens the step attends over besides sink and local: this step's spans united, under the
+                    # persistent mechanism, with those of the last prefill call (every span once)
+                    sel_o, _ = o.selected()
+                    pers = o.persistent() if cfg.persist_decode else np.full_like(sel_o, -1)
+                    sp = o.spans()
+                    want = 0
+                    for g in range(sel_o.shape[0]):
+                        ids = set(int(x) for x in sel_o[g] if x >= 0) | set(int(x) for x in pers[g] if x >= 0)
+                        want += sum(int(sp[j, 1]) for j in ids)
+                    got = int(lt.ltri_get_stats(seq, layer).retrieved_tokens)
+                    assert got == want, f"{what}: attends over {got} retrieved tokens, oracle {want}"
                 check_output(out[i, layer], o.decode_attend(), rep, what)
         return out
 

@@ -59,6 +59,16 @@ def test_dynamic_representative_counts(kind, lam, lo, hi):
     print(rep)
 
 
+@pytest.mark.parametrize("fused", ["0", "1"])
+def test_persistent_mechanism_in_decode(fused, monkeypatch):
+    # Sec. 3.5: the spans the last prefill call retrieved stay in the attention of every decode step (both
+    # decode retrieval paths); the harness checks the united token count exactly and the outputs
+    monkeypatch.setenv("LTRI_DEC_FUSED", fused)
+    cfg = small_cfg(n_layers=2, context=1280, decode_steps=8, persist_decode=True)
+    rep = ph.run_stream(cfg, layers=[0, 1])
+    print(rep)
+
+
 def test_top_k_covering_everything_equals_full_attention():
     # with top_k >= number of spans the streamed output is plain causal attention (oracle O12)
     cfg = small_cfg(n_layers=1, context=640, chunk=64, window=128, top_k=64, max_spans_per_region=2, decode_steps=2)
