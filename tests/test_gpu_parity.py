@@ -69,6 +69,18 @@ def test_persistent_mechanism_in_decode(fused, monkeypatch):
     print(rep)
 
 
+def test_maximum_sizes():
+    # the largest chunk (1024), top-k (64), spans per region (64 -> room for 129 query spans, more than the tcgen05
+    # score kernel takes, so the scores run on the warp-MMA kernel), representatives per span (8) and group size
+    # (8 query heads on one KV head) the library accepts; an absolute threshold keeps the planted segments apart
+    cfg = small_cfg(n_layers=1, n_q_heads=8, n_kv_heads=1, context=5 * 1024 + 200, chunk=1024, window=1024, n_sink=1024,
+                    top_k=64, max_spans_per_region=64, reps_per_span=8, decode_steps=2, seg_min=4, seg_max=24,
+                    theta_mode=0, theta=0.01)
+    rep = ph.run_stream(cfg, layers=[0])
+    assert rep.regions == 5
+    print(rep)
+
+
 def test_top_k_covering_everything_equals_full_attention():
     # with top_k >= number of spans the streamed output is plain causal attention (oracle O12)
     cfg = small_cfg(n_layers=1, context=640, chunk=64, window=128, top_k=64, max_spans_per_region=2, decode_steps=2)
