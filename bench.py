@@ -532,7 +532,8 @@ def main():
     ap.add_argument("--context", type=int, default=0, help="override the context length (profiling of small cases)")
     ap.add_argument("--decode-steps", type=int, default=-1, help="override the number of decode steps")
     ap.add_argument("--dynamic-reps", action="store_true",
-                    help="dynamic span index vectors (rep_mode 1, both neighbours, lambda 2, 1..4 per span)")
+                    help="dynamic span index vectors (rep_mode 1; row ratio and lambda 3 as in the paper's "
+                         "implementation details, 1..4 per span)")
     ap.add_argument("--persist-decode", action="store_true",
                     help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -546,7 +547,7 @@ def main():
         cfg.name += f"[layers={cfg.n_layers},context={cfg.context},decode={cfg.decode_steps}]"
     if args.dynamic_reps:
         import dataclasses
-        cfg = dataclasses.replace(cfg, rep_mode=1, ratio_kind=2, rep_lambda=2.0, min_reps=1, max_reps=4)
+        cfg = dataclasses.replace(cfg, rep_mode=1, ratio_kind=0, rep_lambda=3.0, min_reps=1, max_reps=4)
         cfg.name += "[dynamic-reps]"
     if args.persist_decode:
         import dataclasses
