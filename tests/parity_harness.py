@@ -204,6 +204,9 @@ class StreamPair:
             return
         spans_g = self.lt.ltri_get_spans(seq, layer)
         assert spans_g.tolist() == spans_o.tolist(), f"{what}: span tables differ"
+        stats = self.lt.ltri_get_stats(seq, layer)
+        assert stats.n_spans == len(spans_o) and stats.evicted_end == o.evicted_end
+        assert stats.index_bytes == len(spans_o) * self.cfg.n_kv_heads * self.cfg.head_dim * 2, f"{what}: index size"
         idx_g = self.lt.ltri_debug_read(binding.BUF_INDEX, seq, layer)
         idx_o = o.index()
         for s in range(done, len(spans_o)):
