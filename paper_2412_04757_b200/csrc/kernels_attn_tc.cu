@@ -476,20 +476,21 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           m_used = stt.x;
           lsum = half == 0 ? stt.y : 0.f;
         }
-#pragma unroll 1
-        for (int ch = 0; ch < 2; ++ch) {
-          uint32_t v[32];
+        // all sixteen 16-byte loads of the row half in flight at once, then two TMEM stores
+        uint32_t v[2][32];
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch)
 #pragma unroll
           for (int e = 0; e < 32; e += 4) {
             const float4 f = row_ok ? *reinterpret_cast<const float4*>(op + (size_t)(ch * 8 + (e >> 2)) * 512)
                                     : make_float4(0, 0, 0, 0);
-            v[e] = __float_as_uint(f.x);
-            v[e + 1] = __float_as_uint(f.y);
-            v[e + 2] = __float_as_uint(f.z);
-            v[e + 3] = __float_as_uint(f.w);
+            v[ch][e] = __float_as_uint(f.x);
+            v[ch][e + 1] = __float_as_uint(f.y);
+            v[ch][e + 2] = __float_as_uint(f.z);
+            v[ch][e + 3] = __float_as_uint(f.w);
           }
-          tmem_st32(tO + ch * 32, v);
-        }
+        tmem_st32(tO, v[0]);
+        tmem_st32(tO + 32, v[1]);
         tmem_st_wait();
       }
       int j = 0;

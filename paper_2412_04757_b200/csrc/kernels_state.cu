@@ -86,8 +86,8 @@ cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_b
 
 // ------------------------------------------------------------------------------------------
 // a1: regions that left the window: every span gets its index vector, the bf16 sum of the keys of
-// its most voted token(s), and is appended to the span table.  One CTA per layer, one warp per span.
-__global__ void __launch_bounds__(256) k_evict_index(DevCtx c, EvictArgs a) {
+// its most voted token(s), and is appended to the span table.  One CTA per layer, one warp per span (32 warps).
+__global__ void __launch_bounds__(1024) k_evict_index(DevCtx c, EvictArgs a) {
   const int layer = a.layer_begin + blockIdx.x;
   const size_t unit = unit_of(c, a.seq, layer);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(256) k_evict_index(DevCtx c, EvictArgs a) {
 }
 
 cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_count, cudaStream_t s) {
-  k_evict_index<<<layer_count, 256, 0, s>>>(c, a);
+  k_evict_index<<<layer_count, 1024, 0, s>>>(c, a);  // a warp per span: one round for a region of up to 32 spans
   return cudaGetLastError();
 }
 
