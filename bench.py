@@ -415,73 +415,46 @@ def run_ltri(args, cfg):
         lt.close()
         del lt
         torch.cuda.empty_cache()
-        lt = binding.Ltri(p, device=dev)
+        p_host = binding.LtriParams.from_buffer_copy(p)
+        p_host.flags |= binding.FLAG_HOST_STAGING
+        lt = binding.Ltri(p_host, device=dev)
         stream_until(lt, first_warm, len(chunks))
         host = [tuple(x.cpu().pin_memory() for x in kept[i]) for i in range(W + K)]
         h2d = sum(x.numel() * 2 for x in host[0])
         shape = kept[0][0].shape
         del kept
-        # A user streaming from host memory overlaps the copies with the kernels: the layers of a call are
-        # independent, so each call is issued as layer groups -- group g's inputs go up on a copy stream while
-        # group g-1 computes and group g-2's outputs come down on a third stream.  Two buffer sets alternate
-        # between steps; events order every reuse.
-        ngrp = min(4, L)
-        bounds = [L * g // ngrp for g in range(ngrp + 1)]
-        s_up, s_run, s_down = (torch.cuda.Stream(dev) for _ in range(3))
-        dbuf = [tuple(torch.empty_like(x, device=dev) for x in host[0]) for _ in range(2)]
-        dout = [torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        # The library's host-buffer entry: q, k, v in pinned host memory, output back to pinned host memory.  It
+        # carries a call out in layer groups (the layers are independent): a group's inputs go up on a copy stream
+        # while the previous group computes and the one before sends its output down; two staging sets alternate
+        # between calls.
         hout = [torch.empty(shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
         d2h = hout[0].numel() * 2
-        ev_up = [[torch.cuda.Event() for _ in range(ngrp)] for _ in range(2)]
-        ev_run = [[torch.cuda.Event() for _ in range(ngrp)] for _ in range(2)]
-        ev_down = [[torch.cuda.Event() for _ in range(ngrp)] for _ in range(2)]
-        used = [False, False]
 
         def step(i):
-            b = i & 1
-            for g in range(ngrp):
-                lo, hi = bounds[g], bounds[g + 1]
-                with torch.cuda.stream(s_up):
-                    if used[b]:
-                        s_up.wait_event(ev_run[b][g])         # the kernels of two steps ago have read this slice
-                    for src, dst in zip(host[i], dbuf[b]):
-                        dst[lo:hi].copy_(src[lo:hi], non_blocking=True)
-                    ev_up[b][g].record(s_up)
-                with torch.cuda.stream(s_run):
-                    s_run.wait_event(ev_up[b][g])
-                    if used[b]:
-                        s_run.wait_event(ev_down[b][g])       # its old output has reached the host
-                    lt.ltri_prefill_chunk(SQ, lo, hi - lo, dbuf[b][0][lo:hi], dbuf[b][1][lo:hi], dbuf[b][2][lo:hi],
-                                          out=dout[b][lo:hi], stream=s_run)
-                    ev_run[b][g].record(s_run)
-                with torch.cuda.stream(s_down):
-                    s_down.wait_event(ev_run[b][g])
-                    hout[b][lo:hi].copy_(dout[b][lo:hi], non_blocking=True)
-                    ev_down[b][g].record(s_down)
-            used[b] = True
-
-        def drain():
-            for s in (s_up, s_run, s_down):
-                s.synchronize()
+            lt.ltri_prefill_chunk_host(SQ, 0, L, host[i][0], host[i][1], host[i][2], hout[i & 1])
 
         torch.cuda.synchronize(dev)
         for i in range(W):
             step(i)
-        drain()
+        lt.ltri_host_outputs_ready()
+        torch.cuda.synchronize(dev)
         barrier(world)
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.perf_counter()
-        g0.record(s_up)                           # the copy stream is idle here and starts every step
+        g0.record()
         for i in range(K):
             step(W + i)
-        g1.record(s_down)                         # behind the last output copy, which is behind everything else
-        drain()                                   # every output of every timed step is in host memory
+        lt.ltri_host_outputs_ready()                  # the stream now waits for the last output copy
+        g1.record()
+        torch.cuda.synchronize(dev)                   # every output of every timed step is in host memory
         wall = (time.perf_counter() - t0) * 1e3
         ems = max_over_ranks(max(g0.elapsed_time(g1), wall), world, dev)
+        ngrp = min(4, L)
         assert lt.ltri_sync_status() == 0, "device-side status word reports an error"
         e2e = {"value": world * tokens / (ems * 1e-3), "unit": "tok/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ems / K, "layer_groups": ngrp,
-               "timing": "max of device events (first copy -> last output copy) and the host clock, streams drained"}
+               "api": "ltri_prefill_chunk_host",
+               "timing": "max of device events (first call -> last output copy done) and the host clock"}
     lt.close()
 
     if rank != 0:

@@ -77,7 +77,9 @@ enum {
   LTRI_FLAG_NONE = 0,
   /* Persistent mechanism (Sec. 3.5): the spans selected by the last prefill call of a sequence stay in the attention
    * of every decode step, next to the spans the step retrieves itself. */
-  LTRI_FLAG_PERSIST_DECODE = 1
+  LTRI_FLAG_PERSIST_DECODE = 1,
+  /* Reserve two staging sets in the arena (q, k, v and out of one full call each) for ltri_prefill_chunk_host. */
+  LTRI_FLAG_HOST_STAGING = 2
 };
 
 typedef struct {
@@ -120,6 +122,21 @@ int ltri_reset_sequence(ltri_ctx* ctx, int seq, void* cuda_stream);
  * all be at the same position. */
 int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q,
                        const void* k, const void* v, void* out, void* cuda_stream);
+
+/* ltri_prefill_chunk for a caller whose tensors live in HOST memory (pinned memory for the copies to overlap): same
+ * shapes and meaning, but q_host, k_host, v_host and out_host are host pointers.  The context must have been created
+ * with LTRI_FLAG_HOST_STAGING.  The layers of a call are independent, so the call is carried out in up to four layer
+ * groups: a group's inputs go up on an internal copy stream while the previous group computes on `cuda_stream` and the
+ * group before that sends its output down on a second internal stream; two staging sets alternate between calls, so
+ * the copies of one call also overlap the kernels of its neighbours.  The host inputs must stay valid, and out_host
+ * must not be read, until the work is done: make a stream wait for it with ltri_host_outputs_ready (or synchronise
+ * the device).  On an error return the sequence may be left with some layers advanced; reset it.
+ * The streamed-context setting of Sec. 3.4 with the context memory on the host side. */
+int ltri_prefill_chunk_host(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q_host,
+                            const void* k_host, const void* v_host, void* out_host, void* cuda_stream);
+
+/* Make `cuda_stream` wait until every output of earlier ltri_prefill_chunk_host calls has reached host memory. */
+int ltri_host_outputs_ready(ltri_ctx* ctx, void* cuda_stream);
 
 /* One decode step (the block becomes a single token, Sec. 3.5) for `n_seqs` sequences.
  *   seq_ids  HOST array [n_seqs] of distinct sequence slots

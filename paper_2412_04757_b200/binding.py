@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libltri.so")
 
 LTRI_OK, LTRI_EINVAL, LTRI_ECAPACITY, LTRI_ESTATE, LTRI_ECUDA, LTRI_EDEVICE, LTRI_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 FLAG_PERSIST_DECODE = 1
+FLAG_HOST_STAGING = 2
 BUF_MAP, BUF_VOTES, BUF_INDEX, BUF_THETA, BUF_SCORES, BUF_QREPS, BUF_ROWSTAT, BUF_NREPS = 1, 2, 3, 4, 5, 6, 7, 8
 
 EXPORTS = [
@@ -23,7 +24,7 @@ EXPORTS = [
     "ltri_decode_step", "ltri_get_spans", "ltri_get_pending_spans", "ltri_get_selected", "ltri_get_stats",
     "ltri_sync_status", "ltri_last_cuda_error", "ltri_strerror", "ltri_debug_read", "ltri_span_capacity",
     "ltri_debug_segment_map", "ltri_launch_count", "ltri_profile_enable", "ltri_profile_read",
-    "ltri_segment_map_static",
+    "ltri_segment_map_static", "ltri_prefill_chunk_host", "ltri_host_outputs_ready",
 ]
 KERNEL_CLASSES = ["append", "evict_index", "attn_local", "map_pass", "segment", "score_topk", "attn_retrieved",
                   "decode_retrieve", "decode_attn"]
@@ -74,6 +75,8 @@ def load():
         L.ltri_reset_sequence.argtypes = [vp, ip, vp]
         L.ltri_prefill_chunk.argtypes = [vp, ip, ip, ip, ip, vp, vp, vp, vp, vp]
         L.ltri_decode_step.argtypes = [vp, vp, ip, ip, ip, vp, vp, vp, vp, vp]
+        L.ltri_prefill_chunk_host.argtypes = [vp, ip, ip, ip, ip, vp, vp, vp, vp, vp]
+        L.ltri_host_outputs_ready.argtypes = [vp, vp]
         L.ltri_get_spans.argtypes = [vp, ip, ip, vp, ip, C.POINTER(ip), vp]
         L.ltri_get_pending_spans.argtypes = [vp, ip, ip, vp, ip, C.POINTER(ip), vp]
         L.ltri_get_selected.argtypes = [vp, ip, ip, vp, vp]
@@ -186,6 +189,23 @@ class Ltri:
             raise LtriError(rc, f"ltri_prefill_chunk (cudaError {self.ltri_last_cuda_error()})")
         _check(rc, "ltri_prefill_chunk")
         return out
+
+    def ltri_prefill_chunk_host(self, seq, layer_begin, layer_count, q, k, v, out, stream=None):
+        """Same as ltri_prefill_chunk with q, k, v, out in (pinned) host memory.  Returns out, which is complete
+        only after ltri_host_outputs_ready(stream) + a synchronisation of that stream."""
+        for t in (q, k, v, out):
+            if t.device.type != "cpu" or not t.is_contiguous() or t.dtype != self.torch.bfloat16:
+                raise ValueError("host entry takes contiguous bf16 CPU tensors")
+        rc = self.lib.ltri_prefill_chunk_host(self._h, seq, layer_begin, layer_count, q.shape[1], C.c_void_p(q.data_ptr()),
+                                              C.c_void_p(k.data_ptr()), C.c_void_p(v.data_ptr()),
+                                              C.c_void_p(out.data_ptr()), self._stream(stream))
+        if rc == LTRI_ECUDA:
+            raise LtriError(rc, f"ltri_prefill_chunk_host (cudaError {self.ltri_last_cuda_error()})")
+        _check(rc, "ltri_prefill_chunk_host")
+        return out
+
+    def ltri_host_outputs_ready(self, stream=None):
+        _check(self.lib.ltri_host_outputs_ready(self._h, self._stream(stream)), "ltri_host_outputs_ready")
 
     def ltri_decode_step(self, seq_ids, layer_begin, layer_count, q, k, v, out=None, stream=None):
         """q [n_seqs][layers][Hq][d], k, v [n_seqs][layers][Hkv][d].  Returns out."""

@@ -57,7 +57,7 @@ bool validate(const ltri_params* p) {
   if (p->theta_mode != 0 && p->theta_mode != 1) return false;
   if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
   if (!(p->softmax_scale >= 0.f)) return false;
-  if (p->flags & ~(uint32_t)LTRI_FLAG_PERSIST_DECODE) return false;
+  if (p->flags & ~(uint32_t)(LTRI_FLAG_PERSIST_DECODE | LTRI_FLAG_HOST_STAGING)) return false;
   if (p->rep_mode != 0 && p->rep_mode != 1) return false;
   if (p->rep_mode == 1) {
     if (p->ratio_kind < 0 || p->ratio_kind > 2) return false;
@@ -67,8 +67,14 @@ bool validate(const ltri_params* p) {
   return true;
 }
 
+// bytes of one staging set of the host-buffer entry: q, k, v and out of a full call
+size_t stage_set_bytes(const ltri_params& p) {
+  const size_t rows = (size_t)p.n_layers * p.chunk;
+  return align_up(rows * p.n_q_heads * kD * 2, 256) * 2 + align_up(rows * p.n_kv_heads * kD * 2, 256) * 2;
+}
+
 // fills every pointer of `d` relative to `base` (nullptr: sizing only) and returns the bytes used
-size_t layout(const ltri_params& p, DevCtx& d, char* base) {
+size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nullptr) {
   d.NL = p.n_layers;
   d.Hq = p.n_q_heads;
   d.Hkv = p.n_kv_heads;
@@ -133,6 +139,13 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base) {
   d.dec_part = cv.take<float>(units * d.Hq * kMaxDecSplit * (kD + 2));
   d.status = cv.take<int>(4);
   d.slots += 1;  // the extra slot is scratch for ltri_debug_segment_map
+  if (p.flags & LTRI_FLAG_HOST_STAGING) {
+    const size_t set_bytes = stage_set_bytes(p);
+    for (int s = 0; s < 2; ++s) {
+      char* ptr = cv.take<char>(set_bytes);
+      if (stage_out) stage_out[s] = ptr;
+    }
+  }
   return align_up(cv.off, 256);
 }
 
@@ -147,6 +160,14 @@ struct ltri_ctx {
   bool use_tc = false;     // tcgen05/TMEM/TMA attention kernels (default when available)
   int dec_fused = -1;      // decode retrieval in one launch: -1 auto, 0 never, 1 whenever the index fits
   int dec_split = 0;       // split count of the decode attention: 0 auto (testing aid)
+  // host-buffer entry (LTRI_FLAG_HOST_STAGING): two staging sets in the arena, a copy-up and a copy-down stream, and
+  // events that order every reuse of a set's layer-group slices
+  static constexpr int kHostGroups = 4;
+  char* stage[2] = {nullptr, nullptr};   // per set: q | k | v | out of one call, [NL][chunk][H][128] bf16 each
+  cudaStream_t s_up = nullptr, s_down = nullptr;
+  cudaEvent_t ev_up[2][kHostGroups] = {}, ev_run[2][kHostGroups] = {}, ev_down[2][kHostGroups] = {};
+  bool set_used[2] = {false, false};
+  long long host_calls = 0;
   alignas(64) unsigned char kv_maps[kTcMapBytes];  // TMA descriptors of the K/V cache
   long long launches = 0;  // kernels launched since creation
   // optional per-kernel-class timing with CUDA events on the launching stream
@@ -227,7 +248,20 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
   ltri_ctx* ctx = new (std::nothrow) ltri_ctx();
   if (!ctx) return LTRI_ECAPACITY;
   ctx->p = *p;
-  layout(*p, ctx->d, static_cast<char*>(p->arena));
+  layout(*p, ctx->d, static_cast<char*>(p->arena), ctx->stage);
+  if (p->flags & LTRI_FLAG_HOST_STAGING) {
+    bool ok = cudaStreamCreateWithFlags(&ctx->s_up, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&ctx->s_down, cudaStreamNonBlocking) == cudaSuccess;
+    for (int s = 0; s < 2 && ok; ++s)
+      for (int g = 0; g < ltri_ctx::kHostGroups && ok; ++g)
+        ok = cudaEventCreateWithFlags(&ctx->ev_up[s][g], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&ctx->ev_run[s][g], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&ctx->ev_down[s][g], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      ltri_destroy(ctx);
+      return LTRI_ECUDA;
+    }
+  }
   ctx->st.resize((size_t)p->max_seqs * p->n_layers);
   for (auto& s : ctx->st) s.E = p->n_sink;
   int dev = 0;
@@ -256,6 +290,20 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
 
 int ltri_destroy(ltri_ctx* ctx) {
   if (!ctx) return LTRI_EINVAL;
+  if (ctx->s_up) {  // copies of the host-buffer entry may still be in flight
+    cudaStreamSynchronize(ctx->s_up);
+    cudaStreamDestroy(ctx->s_up);
+  }
+  if (ctx->s_down) {
+    cudaStreamSynchronize(ctx->s_down);
+    cudaStreamDestroy(ctx->s_down);
+  }
+  for (int s = 0; s < 2; ++s)
+    for (int g = 0; g < ltri_ctx::kHostGroups; ++g) {
+      if (ctx->ev_up[s][g]) cudaEventDestroy(ctx->ev_up[s][g]);
+      if (ctx->ev_run[s][g]) cudaEventDestroy(ctx->ev_run[s][g]);
+      if (ctx->ev_down[s][g]) cudaEventDestroy(ctx->ev_down[s][g]);
+    }
   for (auto* pool : {&ctx->timed, &ctx->free_pool})
     for (auto& t : *pool) {
       cudaEventDestroy(t.a);
@@ -391,6 +439,64 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
     s.last_m = m;
     if (m > 0) s.pending.push_back(Region{reg_start, t0 + n_tokens, slot});
   }
+  return LTRI_OK;
+}
+
+int ltri_prefill_chunk_host(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q_host,
+                            const void* k_host, const void* v_host, void* out_host, void* cuda_stream) {
+  if (!ctx) return LTRI_EINVAL;
+  if (!ctx->stage[0]) return LTRI_ESTATE;  // created without LTRI_FLAG_HOST_STAGING
+  const DevCtx& d = ctx->d;
+  if (seq < 0 || seq >= d.NS || layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > d.NL)
+    return LTRI_EINVAL;
+  if (n_tokens < 1 || n_tokens > d.chunk || !q_host || !k_host || !v_host || !out_host) return LTRI_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int set = (int)(ctx->host_calls & 1);
+  const size_t rows = (size_t)d.NL * d.chunk;
+  const size_t qb = align_up(rows * d.Hq * kD * 2, 256), kb = align_up(rows * d.Hkv * kD * 2, 256);
+  char* sq = ctx->stage[set];
+  char* sk = sq + qb;
+  char* sv = sk + kb;
+  char* so = sv + kb;
+  const int ng = std::min((int)ltri_ctx::kHostGroups, layer_count);
+  const size_t qrow = (size_t)n_tokens * d.Hq * kD * 2, krow = (size_t)n_tokens * d.Hkv * kD * 2;  // bytes per layer
+  for (int g = 0; g < ng; ++g) {
+    const int lo = layer_count * g / ng, hi = layer_count * (g + 1) / ng;  // layers of the group, call-relative
+    const size_t qo = lo * qrow, ko = lo * krow, qn = (hi - lo) * qrow, kn = (hi - lo) * krow;
+    // up: the kernels that read this slice two calls ago are done
+    if (ctx->set_used[set]) LTRI_CUDA(ctx, cudaStreamWaitEvent(ctx->s_up, ctx->ev_run[set][g], 0));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(sq + qo, static_cast<const char*>(q_host) + qo, qn, cudaMemcpyHostToDevice, ctx->s_up));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(sk + ko, static_cast<const char*>(k_host) + ko, kn, cudaMemcpyHostToDevice, ctx->s_up));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(sv + ko, static_cast<const char*>(v_host) + ko, kn, cudaMemcpyHostToDevice, ctx->s_up));
+    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_up[set][g], ctx->s_up));
+    // run: inputs are up, and the output slice written two calls ago has gone down
+    LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_up[set][g], 0));
+    if (ctx->set_used[set]) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down[set][g], 0));
+    const int rc = ltri_prefill_chunk(ctx, seq, layer_begin + lo, hi - lo, n_tokens, sq + qo, sk + ko, sv + ko, so + qo, st);
+    if (rc != LTRI_OK) return rc;
+    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_run[set][g], st));
+    // down
+    LTRI_CUDA(ctx, cudaStreamWaitEvent(ctx->s_down, ctx->ev_run[set][g], 0));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(static_cast<char*>(out_host) + qo, so + qo, qn, cudaMemcpyDeviceToHost, ctx->s_down));
+    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_down[set][g], ctx->s_down));
+  }
+  // groups beyond ng keep their old events; make them harmless for the next use of this set
+  for (int g = ng; g < ltri_ctx::kHostGroups; ++g) {
+    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_run[set][g], st));
+    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_down[set][g], ctx->s_down));
+  }
+  ctx->set_used[set] = true;
+  ctx->host_calls += 1;
+  return LTRI_OK;
+}
+
+int ltri_host_outputs_ready(ltri_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return LTRI_EINVAL;
+  if (!ctx->stage[0]) return LTRI_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  for (int s = 0; s < 2; ++s)
+    if (ctx->set_used[s])
+      for (int g = 0; g < ltri_ctx::kHostGroups; ++g) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down[s][g], 0));
   return LTRI_OK;
 }
 

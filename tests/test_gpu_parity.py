@@ -225,3 +225,37 @@ def test_state_and_capacity_errors():
     torch.cuda.synchronize()
     assert lt.ltri_sync_status() == 0
     lt.close()
+
+
+def test_host_buffer_entry_matches_the_device_entry():
+    # the same stream once through ltri_prefill_chunk (device tensors) and once through ltri_prefill_chunk_host
+    # (pinned host tensors, layer groups pipelined over internal copy streams): identical outputs and state
+    cfg = small_cfg(n_layers=6, context=1152, decode_steps=0)
+    dev = torch.device("cuda:0")
+    st = inputs.SyntheticStream(cfg)
+    lt_d = binding.Ltri(ph.params_of(cfg), device=dev)
+    p = ph.params_of(cfg)
+    p.flags |= binding.FLAG_HOST_STAGING
+    lt_h = binding.Ltri(p, device=dev)
+    outs_h = []
+    for t0, n in st.prefill_chunks():
+        q, k, v = st.tokens(t0, n)
+        ref = lt_d.ltri_prefill_chunk(0, 0, cfg.n_layers, q.to(dev), k.to(dev), v.to(dev))
+        hq, hk, hv = (x.contiguous().pin_memory() for x in (q, k, v))
+        ho = torch.empty_like(hq).pin_memory()
+        lt_h.ltri_prefill_chunk_host(0, 0, cfg.n_layers, hq, hk, hv, ho)
+        outs_h.append((ref, ho, (hq, hk, hv)))       # keep the host inputs alive until the work is done
+    lt_h.ltri_host_outputs_ready()
+    torch.cuda.synchronize(dev)
+    assert lt_d.ltri_sync_status() == 0 and lt_h.ltri_sync_status() == 0
+    for ref, ho, _ in outs_h:
+        assert torch.equal(ref.cpu(), ho)
+    for layer in range(cfg.n_layers):
+        assert lt_d.ltri_get_spans(0, layer).tolist() == lt_h.ltri_get_spans(0, layer).tolist()
+        assert np.array_equal(lt_d.ltri_get_selected(0, layer), lt_h.ltri_get_selected(0, layer))
+    # a context created without the staging flag refuses the host entry
+    q, k, v = st.tokens(0, cfg.chunk)
+    with pytest.raises(binding.LtriError):
+        lt_d.ltri_prefill_chunk_host(0, 0, cfg.n_layers, q.contiguous(), k.contiguous(), v.contiguous(), torch.empty_like(q))
+    lt_d.close()
+    lt_h.close()
