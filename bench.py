@@ -509,6 +509,9 @@ def main():
                          "implementation details, 1..4 per span)")
     ap.add_argument("--persist-decode", action="store_true",
                     help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
+    ap.add_argument("--p-self", type=float, default=-1.0,
+                    help="generator: probability that a prefill token targets its own segment (default 0.5; 0 = the "
+                         "literal 'earlier segment' reading)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -522,6 +525,10 @@ def main():
         import dataclasses
         cfg = dataclasses.replace(cfg, rep_mode=1, ratio_kind=0, rep_lambda=3.0, min_reps=1, max_reps=4)
         cfg.name += "[dynamic-reps]"
+    if args.p_self >= 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, p_self=args.p_self)
+        cfg.name += f"[p_self={args.p_self:g}]"
     if args.persist_decode:
         import dataclasses
         cfg = dataclasses.replace(cfg, persist_decode=True)
