@@ -74,7 +74,10 @@ __global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer
   const size_t src = (((size_t)b.src[bi] * layer_count + l) * c.Hkv + g) * kD + c16 * 8;
   *reinterpret_cast<uint4*>(c.Kc + dst) = *reinterpret_cast<const uint4*>(k + src);
   *reinterpret_cast<uint4*>(c.Vc + dst) = *reinterpret_cast<const uint4*>(v + src);
-  if (g == 0 && c16 == 0) c.votes[unit * c.Tpad + b.pos[bi]] = 0;
+  if (g == 0 && c16 == 0) {
+    c.votes[unit * c.Tpad + b.pos[bi]] = 0;
+    c.sel_tokens[unit] = 0;  // the retrieval kernels of this step add the tokens they select
+  }
 }
 
 cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int,
@@ -1104,10 +1107,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
     su[tid] = acc;
   }
-  if (tid == 0) {
-    s_cnt = 0;
-    if (g == 0) c.sel_tokens[unit] = 0;
-  }
+  if (tid == 0) s_cnt = 0;
   __syncthreads();
   // ---- scores
   {
@@ -1272,14 +1272,242 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   }
 }
 
+// Decode retrieval in one launch for an index too large for one CTA's shared memory (up to 98K spans, the 1M-token
+// workload): a thread-block cluster of eight CTAs owns one (sequence, layer, KV head).  Each
+// CTA streams its eighth of that head's index once (half-warp per 256-byte row, 16 bytes per lane, four rows in
+// flight, the next four prefetched) and keeps its scores in shared memory; the cluster then selects the top-k with
+// the radix select of k_topk, every CTA counting its own scores and all of them adding the eight histograms up
+// through distributed shared memory; the selected ids meet in the first CTA, which writes the selection and the
+// token ranges of the attention kernel.
+constexpr int kRetCluster = 8;
+constexpr int kRetThreads = 512;
+constexpr int kRetSliceMax = 12288;  // scores a CTA keeps in shared memory (48 KB)
+
+__global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThreads)
+    k_dec_retrieve_cl(DevCtx c, int layer_begin, DecBatch b, int layer_count, const __nv_bfloat16* __restrict__ q) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ float ssc[];  // this CTA's slice of the scores
+  __shared__ float su[kD];
+  __shared__ unsigned hist[256];  // this CTA's histogram (read by the whole cluster)
+  __shared__ unsigned tot[256];   // the cluster's histogram (every CTA builds its own copy)
+  __shared__ unsigned s_prefix, s_need;
+  __shared__ int s_eq, s_take;    // this CTA's count of scores equal to the threshold / of selected scores
+  __shared__ int s_ids[kMaxTopK]; // first CTA: all selected ids, ascending
+  __shared__ int s_loc[kMaxTopK]; // this CTA's selected ids
+  __shared__ int s_cnt;
+  __shared__ int s_scan[kRetThreads];
+  __shared__ int s_rs[kMaxRanges], s_rl[kMaxRanges], s_nr, s_sst[2 * kMaxTopK], s_sln[2 * kMaxTopK];
+  __shared__ int s_all[2 * kMaxTopK], s_nall;
+  const int rank = (int)cluster.block_rank();
+  const int g = blockIdx.x / kRetCluster;
+  const int bi = blockIdx.y / layer_count, l = blockIdx.y % layer_count, layer = layer_begin + l;
+  const int sq = b.seq[bi], pos = b.pos[bi], loc_begin = b.loc_begin[bi];
+  const size_t unit = unit_of(c, sq, layer);
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int N = min(c.n_spans[unit], kRetCluster * kRetSliceMax);
+  const int per = (N + kRetCluster - 1) / kRetCluster;
+  const int lo = min(N, rank * per), hi = min(N, lo + per), nloc = hi - lo;  // this CTA's spans [lo, hi)
+  if (tid < kD) {
+    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + g * c.G) * kD + tid;
+    float acc = 0.f;
+    for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
+    su[tid] = acc;
+  }
+  if (tid == 0) s_cnt = 0;
+  __syncthreads();
+  // ---- scores of the slice
+  {
+    constexpr int HW = kRetThreads / 16;  // half-warps
+    const int hw = tid >> 4, hl = tid & 15;
+    float uf[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
+    const __nv_bfloat16* KR = c.KR + ((unit * c.Hkv + g) * (size_t)c.cap + lo) * kD + hl * 8;
+    auto fetch = [&](int base, uint4 (&raw)[4]) {
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int s = base + t * HW + hw;
+        raw[t] = s < nloc ? __ldg(reinterpret_cast<const uint4*>(KR + (size_t)s * kD)) : make_uint4(0, 0, 0, 0);
+      }
+    };
+    uint4 cur[4], nxt[4];
+    fetch(0, cur);
+    for (int base = 0; base < nloc; base += HW * 4) {  // uniform trip count (shuffles inside)
+      fetch(base + HW * 4, nxt);                       // past the end: zeros, no loads
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&cur[t]);
+        float d = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(p2[i]);
+          d = fmaf(uf[2 * i], f.x, d);
+          d = fmaf(uf[2 * i + 1], f.y, d);
+        }
+        d += __shfl_xor_sync(0xffffffffu, d, 1);
+        d += __shfl_xor_sync(0xffffffffu, d, 2);
+        d += __shfl_xor_sync(0xffffffffu, d, 4);
+        d += __shfl_xor_sync(0xffffffffu, d, 8);
+        const int s = base + t * HW + hw;
+        if (hl == 0 && s < nloc) ssc[s] = d;
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t) cur[t] = nxt[t];
+    }
+  }
+  __syncthreads();
+  // ---- top-k over the cluster's scores
+  const int K = min(c.topk, N);
+  if (tid == 0) s_take = 0;
+  __syncthreads();
+  if (K == N) {
+    for (int t = tid; t < nloc; t += nt) s_loc[t] = lo + t;  // (N <= top_k <= 64)
+    if (tid == 0) s_take = nloc;
+  } else {
+    if (tid == 0) {
+      s_prefix = 0;
+      s_need = K;  // rank from the top, 1-based: find key T with #(key > T) < K <= #(key >= T)
+    }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      const unsigned prefix = s_prefix;
+      const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      for (int s = tid; s < nloc; s += nt) {
+        const unsigned key = order_key(ssc[s]);
+        if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
+      cluster.sync();
+      if (tid < 256) {
+        unsigned sum = 0;
+        for (int r = 0; r < kRetCluster; ++r) sum += cluster.map_shared_rank(hist, r)[tid];
+        tot[tid] = sum;
+      }
+      cluster.sync();  // every CTA has read every histogram: they may be reset
+      if (tid < 32) {
+        unsigned need = s_need;
+        const int bin = pick_from_top(tot, 256, need);
+        if (tid == 0) {
+          s_need = need;
+          s_prefix = prefix | ((unsigned)bin << shift);
+        }
+      }
+      __syncthreads();
+    }
+    const unsigned T = s_prefix;
+    const unsigned need_eq = s_need;  // how many of the == T elements are taken (lowest ids first, cluster-wide)
+    // contiguous id partition so that ties are picked in id order: inside the CTA by thread, across CTAs by rank
+    const int pt = (nloc + nt - 1) / nt;
+    const int tlo = min(nloc, tid * pt), thi = min(nloc, tlo + pt);
+    int eq = 0;
+    for (int s = tlo; s < thi; ++s) eq += order_key(ssc[s]) == T;
+    s_scan[tid] = eq;
+    __syncthreads();
+    if (tid == 0) {
+      int run = 0;
+      for (int t = 0; t < nt; ++t) {
+        const int v = s_scan[t];
+        s_scan[t] = run;
+        run += v;
+      }
+      s_eq = run;
+    }
+    cluster.sync();
+    int eqrank = s_scan[tid];
+    for (int r = 0; r < rank; ++r) eqrank += *cluster.map_shared_rank(&s_eq, r);
+    for (int s = tlo; s < thi; ++s) {
+      const unsigned key = order_key(ssc[s]);
+      bool take = key > T;
+      if (key == T) {
+        take = (unsigned)eqrank < need_eq;
+        ++eqrank;
+      }
+      if (take) {
+        const int slot = atomicAdd(&s_take, 1);
+        if (slot < kMaxTopK) s_loc[slot] = lo + s;
+      }
+    }
+  }
+  __syncthreads();
+  // this CTA's ids in ascending order (rank sort), then into the first CTA's list behind those of the lower ranks
+  const int ntake = min(s_take, kMaxTopK);
+  int myid = -1, myrank = 0;
+  if (tid < ntake) {
+    myid = s_loc[tid];
+    for (int t = 0; t < ntake; ++t) myrank += s_loc[t] < myid;
+  }
+  cluster.sync();  // every CTA's s_take is final
+  int offset = 0, total = 0;
+  for (int r = 0; r < kRetCluster; ++r) {
+    const int v = min(*cluster.map_shared_rank(&s_take, r), kMaxTopK);
+    if (r < rank) offset += v;
+    total += v;
+  }
+  if (tid < ntake && offset + myrank < kMaxTopK) cluster.map_shared_rank(s_ids, 0)[offset + myrank] = myid;
+  cluster.sync();  // the list is complete; the other CTAs' shared memory is not read after this point
+  if (rank != 0) return;
+  const int cnt = min(total, K);
+  int* sel = c.sel + (unit * c.Hkv + g) * (size_t)c.topk;
+  for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
+  const int* ids_all = s_ids;
+  int nall = cnt;
+  if (c.persist) {
+    nall = union_with_persistent(c, unit, g, s_ids, cnt, s_scan, s_all, &s_nall);
+    ids_all = s_all;
+  }
+  if (tid < nall) {
+    s_sst[tid] = c.span_start[unit * c.cap + ids_all[tid]];
+    s_sln[tid] = c.span_len[unit * c.cap + ids_all[tid]];
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int nr = 0;
+    long long tokens = 0;
+    auto push = [&](int st, int ln) {
+      if (ln <= 0) return;
+      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] == st)
+        s_rl[nr - 1] += ln;
+      else {
+        s_rs[nr] = st;
+        s_rl[nr] = ln;
+        ++nr;
+      }
+    };
+    push(0, min(c.Ls, pos + 1));
+    for (int t = 0; t < nall; ++t) {
+      tokens += s_sln[t];
+      push(s_sst[t], s_sln[t]);
+    }
+    push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
+    s_nr = nr;
+    c.rng_cnt[unit * c.Hkv + g] = nr;
+    atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+  }
+  __syncthreads();
+  const size_t rbb = (unit * c.Hkv + g) * (size_t)c.rcap;
+  for (int t = tid; t < s_nr; t += nt) {
+    c.rng_start[rbb + t] = s_rs[t];
+    c.rng_len[rbb + t] = s_rl[t];
+  }
+}
+
 cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count,
-                                      const __nv_bfloat16* q, int span_bound, cudaStream_t s) {
-  const int smem = (int)sizeof(float) * max(span_bound, 1);
-  if (smem > 48 * 1024) return cudaErrorInvalidValue;
-  k_dec_retrieve<<<dim3(c.Hkv, b.n * layer_count), 1024, smem, s>>>(c, layer_begin, b, layer_count, q);
+                                      const __nv_bfloat16* q, int span_bound, bool force_cluster, cudaStream_t s) {
+  span_bound = max(span_bound, 1);
+  if (span_bound <= kFusedMaxSpans && !force_cluster) {  // one CTA per head: no cluster barriers
+    k_dec_retrieve<<<dim3(c.Hkv, b.n * layer_count), 1024, (int)sizeof(float) * span_bound, s>>>(c, layer_begin, b,
+                                                                                                 layer_count, q);
+    return cudaGetLastError();
+  }
+  const int per = (span_bound + kRetCluster - 1) / kRetCluster;
+  if (per > kRetSliceMax) return cudaErrorInvalidValue;
+  k_dec_retrieve_cl<<<dim3(c.Hkv * kRetCluster, b.n * layer_count), kRetThreads, (int)sizeof(float) * per, s>>>(
+      c, layer_begin, b, layer_count, q);
   return cudaGetLastError();
 }
-int dec_retrieve_fused_max_spans() { return kFusedMaxSpans; }
+int dec_retrieve_fused_max_spans() { return kRetCluster * kRetSliceMax; }
 
 cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
   DecBatch dummy;

@@ -158,7 +158,7 @@ struct ltri_ctx {
   int last_cuda = 0;
   int sm_count = 148;
   bool use_tc = false;     // tcgen05/TMEM/TMA attention kernels (default when available)
-  int dec_fused = -1;      // decode retrieval in one launch: -1 auto, 0 never, 1 whenever the index fits
+  int dec_fused = -1;      // decode retrieval in one launch: -1 auto, 0 never, 1 whenever the index fits, 2 cluster kernel
   int dec_split = 0;       // split count of the decode attention: 0 auto (testing aid)
   // host-buffer entry (LTRI_FLAG_HOST_STAGING): two staging sets in the arena, a copy-up and a copy-down stream, and
   // events that order every reuse of a set's layer-group slices
@@ -270,7 +270,8 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) ctx->sm_count = sms;
   }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  if (const char* f = std::getenv("LTRI_DEC_FUSED")) ctx->dec_fused = std::atoi(f) != 0 ? 1 : 0;  // testing aid
+  // testing aid: 0 two launches, 1 one launch, 2 one launch with the cluster kernel whatever the index size
+  if (const char* f = std::getenv("LTRI_DEC_FUSED")) ctx->dec_fused = std::max(0, std::min(2, std::atoi(f)));
   if (const char* f = std::getenv("LTRI_DEC_SPLIT")) ctx->dec_split = std::max(0, std::atoi(f));    // testing aid
   const char* impl = std::getenv("LTRI_ATTN_IMPL");  // "mma" selects the warp-MMA kernels (debugging aid)
   ctx->use_tc = tc_attention_supported(ctx->d) && !(impl && std::strcmp(impl, "mma") == 0) &&
@@ -576,13 +577,15 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
       Scope sc(ctx, st, LTRI_K_APPEND, 1);
       LTRI_CUDA(ctx, launch_append_decode(d, b, layer_begin, layer_count, n_seqs, kb, vb, st));
     }
-    // one CTA per (sequence, layer, KV head) keeps the scores in shared memory when the index is small enough and
-    // there are enough heads to fill the GPU; otherwise scores go through global memory in two launches
+    // retrieval in one launch with the scores in shared memory: one CTA per (sequence, layer, KV head) when there are
+    // enough heads to fill the GPU and the index fits one CTA (12K spans), a cluster of eight CTAs per head for a larger
+    // index (up to 98K spans); otherwise the scores go through global memory in two launches
+    const bool one_cta = ub <= 12288;
     const bool fused = ub <= dec_retrieve_fused_max_spans() &&
-                       (ctx->dec_fused == 1 || (ctx->dec_fused < 0 && units >= ctx->sm_count));
+                       (ctx->dec_fused >= 1 || (ctx->dec_fused < 0 && (!one_cta || units >= ctx->sm_count)));
     if (fused) {
       Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 1);
-      LTRI_CUDA(ctx, launch_dec_retrieve_fused(d, b, layer_begin, layer_count, qb, (int)ub, st));
+      LTRI_CUDA(ctx, launch_dec_retrieve_fused(d, b, layer_begin, layer_count, qb, (int)ub, ctx->dec_fused == 2, st));
     } else {
       Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 2);
       LTRI_CUDA(ctx, launch_score_decode(d, b, layer_begin, layer_count, n_seqs, qb, (int)ub, st));

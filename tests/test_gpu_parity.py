@@ -59,7 +59,7 @@ def test_dynamic_representative_counts(kind, lam, lo, hi):
     print(rep)
 
 
-@pytest.mark.parametrize("fused", ["0", "1"])
+@pytest.mark.parametrize("fused", ["0", "1", "2"])
 def test_persistent_mechanism_in_decode(fused, monkeypatch):
     # Sec. 3.5: the spans the last prefill call retrieved stay in the attention of every decode step (both
     # decode retrieval paths); the harness checks the united token count exactly and the outputs
@@ -144,7 +144,7 @@ def test_batched_decode_independent_sequences():
     print(sp.rep)
 
 
-@pytest.mark.parametrize("fused", ["0", "1"])
+@pytest.mark.parametrize("fused", ["0", "1", "2"])
 def test_decode_retrieval_paths(fused, monkeypatch):
     # decode retrieval has a one-launch path (scores in shared memory) and a two-launch path; check both
     monkeypatch.setenv("LTRI_DEC_FUSED", fused)
