@@ -198,7 +198,8 @@ def oracle_sample(cfg, steps, warmup):
     o = orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
                          need + 8, reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
                          theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind,
-                         min_reps=cfg.min_reps, max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda)
+                         min_reps=cfg.min_reps, max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
+                         unit_tokens=cfg.unit_tokens, persist_decode=int(cfg.persist_decode))
     times = []
     for ci in range(fill + warmup + steps):
         q, k, v = st.tokens(ci * cfg.chunk, cfg.chunk)
@@ -270,8 +271,12 @@ def needle_recall(lt, st, seq, cfg):
         sel = lt.ltri_get_selected(seq, layer)
         for g in range(cfg.n_kv_heads):
             ids = sel[g][sel[g] >= 0]
-            lo = np.maximum(spans[ids, 0], a)
-            hi = np.minimum(spans[ids, 0] + spans[ids, 1], b)
+            if cfg.unit_tokens > 0:   # the ids are unit numbers: tokens [id * U, (id + 1) * U)
+                lo = np.maximum(ids * cfg.unit_tokens, a)
+                hi = np.minimum((ids + 1) * cfg.unit_tokens, b)
+            else:
+                lo = np.maximum(spans[ids, 0], a)
+                hi = np.minimum(spans[ids, 0] + spans[ids, 1], b)
             c = float(np.clip(hi - lo, 0, None).sum()) / (b - a)
             cover += c
             full += c >= 1.0
@@ -307,7 +312,8 @@ def run_ltri(args, cfg):
                             max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
                             max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
-                            flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0)
+                            flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0,
+                            unit_tokens=cfg.unit_tokens)
 
     def stream_until(lt, upto, keep_from):
         for s in range(NSEQ - 1):
@@ -507,6 +513,8 @@ def main():
     ap.add_argument("--dynamic-reps", action="store_true",
                     help="dynamic span index vectors (rep_mode 1; row ratio and lambda 3 as in the paper's "
                          "implementation details, 1..4 per span)")
+    ap.add_argument("--unit-tokens", type=int, default=0,
+                    help="retrieval granularity: fixed units of this many tokens instead of spans (the paper's 128)")
     ap.add_argument("--persist-decode", action="store_true",
                     help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
     ap.add_argument("--p-self", type=float, default=-1.0,
@@ -529,6 +537,10 @@ def main():
         import dataclasses
         cfg = dataclasses.replace(cfg, p_self=args.p_self)
         cfg.name += f"[p_self={args.p_self:g}]"
+    if args.unit_tokens > 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, unit_tokens=args.unit_tokens)
+        cfg.name += f"[unit={args.unit_tokens}]"
     if args.persist_decode:
         import dataclasses
         cfg = dataclasses.replace(cfg, persist_decode=True)

@@ -69,6 +69,12 @@ typedef struct {
   int32_t ratio_kind;                                /* 0 row, 1 column, 2 both */
   int32_t min_reps, max_reps;                        /* 1 <= min_reps <= max_reps <= 8 (rep_mode 1 only) */
   float rep_lambda;                                  /* >= 0 (rep_mode 1 only) */
+  int32_t unit_tokens;                               /* retrieval granularity.  0: the k best spans are fetched.
+                                                        U (multiple of 8, 8..chunk): Eq. 8 as printed -- the tokens are
+                                                        cut into fixed units of U on the absolute token grid, a unit's
+                                                        score is the maximum over the spans it meets, the k best units
+                                                        are fetched whole (clipped to the indexed range) and
+                                                        ltri_get_selected reports unit numbers (token / U) */
   void* arena;                                       /* caller-owned device memory, 256-byte aligned */
   size_t arena_bytes;                                /* >= ltri_arena_bytes(params) */
 } ltri_params;

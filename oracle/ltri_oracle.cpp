@@ -89,6 +89,9 @@ struct Params {
   float rep_lambda;
   // persistent mechanism (Sec. 3.5): decode keeps the spans selected by the last prefill call
   int32_t persist_decode;
+  // retrieval granularity (Eq. 8 as printed): 0 = the span; U > 0 = fixed units of U tokens on the absolute token
+  // grid, scored by the maximum over the spans they meet and fetched whole (clipped to the indexed range)
+  int32_t unit_tokens;
 };
 
 // ---------------------------------------------------------------------------
@@ -299,6 +302,7 @@ struct Stream {
   std::vector<float> u;  // [Hkv][J][d]
   int J = 0;
   std::vector<float> score;  // [Hkv][Ns]
+  std::vector<float> unit_score;  // [Hkv][units] (unit mode)
   std::vector<int> sel;      // [Hkv][top_k]
   std::vector<int> persist;  // [Hkv][top_k] selection of the last prefill call, kept through decode (Sec. 3.5)
   std::vector<double> cut_gap;  // [Hkv]
@@ -334,6 +338,11 @@ struct Stream {
     t += cnt;
   }
 
+  // units (of unit_tokens tokens on the absolute grid) that meet the indexed range [n_sink, E)
+  int unit_count() const {
+    if (p.unit_tokens <= 0 || E <= p.n_sink) return 0;
+    return (E + p.unit_tokens - 1) / p.unit_tokens - p.n_sink / p.unit_tokens;
+  }
   int rep_stride() const { return p.rep_mode == 1 ? std::max(p.max_reps, 1) : p.reps_per_span; }
   // representative counts of the spans of the newest region (the region map of the current call is still there)
   void decide_rep_counts(Region& reg) const {
@@ -554,6 +563,7 @@ struct Stream {
   void score_and_select() {
     int Ns = (int)spans.size();
     score.assign((size_t)Hkv * Ns, -INFINITY);
+    if (p.unit_tokens > 0) unit_score.assign((size_t)Hkv * unit_count(), -INFINITY);
     for (int g = 0; g < Hkv; ++g) {
       for (int s = 0; s < Ns; ++s) {
         float best = -INFINITY;
@@ -566,7 +576,18 @@ struct Stream {
         }
         score[(size_t)g * Ns + s] = best;
       }
-      if (J > 0)
+      if (J > 0 && p.unit_tokens > 0) {
+        // Eq. 8: the score of a unit is the maximum over its spans; the top-k units are fetched
+        const int U = p.unit_tokens, u0 = p.n_sink / U, nu = unit_count();
+        float* us = &unit_score[(size_t)g * nu];
+        for (int u = 0; u < nu; ++u) us[u] = -INFINITY;
+        for (int s = 0; s < Ns; ++s)
+          for (int u = spans[s].start / U; u <= (spans[s].start + spans[s].len - 1) / U; ++u)
+            us[u - u0] = std::max(us[u - u0], score[(size_t)g * Ns + s]);
+        top_k(us, nu, p.top_k, &sel[(size_t)g * p.top_k], &cut_gap[g]);
+        for (int i = 0; i < p.top_k; ++i)
+          if (sel[(size_t)g * p.top_k + i] >= 0) sel[(size_t)g * p.top_k + i] += u0;  // absolute unit ids
+      } else if (J > 0)
         top_k(&score[(size_t)g * Ns], Ns, p.top_k, &sel[(size_t)g * p.top_k], &cut_gap[g]);
       else {
         for (int i = 0; i < p.top_k; ++i) sel[(size_t)g * p.top_k + i] = -1;
@@ -590,7 +611,12 @@ struct Stream {
         int s = persist[(size_t)g * p.top_k + i];
         if (s >= 0 && std::find(ids.begin(), ids.end(), s) == ids.end()) ids.push_back(s);
       }
-    for (int s : ids) ranges.push_back({spans[s].start, spans[s].start + spans[s].len});
+    for (int s : ids) {
+      if (p.unit_tokens > 0)  // the unit's tokens inside the indexed range [n_sink, E)
+        ranges.push_back({std::max(s * p.unit_tokens, p.n_sink), std::min((s + 1) * p.unit_tokens, E)});
+      else
+        ranges.push_back({spans[s].start, spans[s].start + spans[s].len});
+    }
     ranges.push_back({loc_begin, loc_end});
     return ranges;
   }
@@ -683,6 +709,7 @@ void* orc_create(const Params* p) {
   if (!p || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads) return nullptr;
   if (p->head_dim < 1 || p->chunk < 1 || p->window < 1 || p->n_sink < 1 || p->top_k < 1) return nullptr;
   if (p->reps_per_span < 1 || p->max_spans_per_region < 1 || p->max_tokens < 1) return nullptr;
+  if (p->unit_tokens < 0) return nullptr;
   if (p->rep_mode != 0 && p->rep_mode != 1) return nullptr;
   if (p->rep_mode == 1 && (p->ratio_kind < 0 || p->ratio_kind > 2 || p->min_reps < 1 || p->max_reps < p->min_reps ||
                            !(p->rep_lambda >= 0.f)))
@@ -778,6 +805,11 @@ int orc_set_newest_rep_counts(void* h, const int* counts, int cnt) {
     s->pending.back().spans[i].nrep = counts[i];
   }
   return 0;
+}
+int orc_num_units(void* h) { return ((Stream*)h)->unit_count(); }
+void orc_get_unit_scores(void* h, float* out) {  // [Hkv][units]
+  Stream* s = (Stream*)h;
+  std::memcpy(out, s->unit_score.data(), s->unit_score.size() * sizeof(float));
 }
 int orc_rep_stride(void* h) { return ((Stream*)h)->rep_stride(); }
 int orc_dynamic_rep_count(const int32_t* Mq, int m, int x, int y, int kind, double lambda, int min_reps, int max_reps) {

@@ -34,7 +34,7 @@ class _Params(C.Structure):
         ("theta_mode", C.c_int32), ("theta", C.c_float), ("softmax_scale", C.c_float),
         ("max_tokens", C.c_int64),
         ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
-        ("rep_lambda", C.c_float), ("persist_decode", C.c_int32),
+        ("rep_lambda", C.c_float), ("persist_decode", C.c_int32), ("unit_tokens", C.c_int32),
     ]
 
 
@@ -85,6 +85,9 @@ def lib():
         L.orc_get_newest_rep_counts.argtypes = [vp, vp, ip]
         L.orc_get_newest_rep_counts.restype = ip
         L.orc_get_persistent.argtypes = [vp, vp]
+        L.orc_num_units.argtypes = [vp]
+        L.orc_num_units.restype = ip
+        L.orc_get_unit_scores.argtypes = [vp, vp]
         L.orc_set_newest_rep_counts.argtypes = [vp, vp, ip]
         L.orc_set_newest_rep_counts.restype = ip
         L.orc_rep_stride.argtypes = [vp]
@@ -117,7 +120,8 @@ class OracleStream:
 
     def __init__(self, n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, max_tokens,
                  reps_per_span=1, max_spans_per_region=None, theta_mode=1, theta=0.90, softmax_scale=0.0,
-                 rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, persist_decode=0):
+                 rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, persist_decode=0,
+                 unit_tokens=0):
         if max_spans_per_region is None:
             max_spans_per_region = max(1, chunk // 32)
         self.Hq, self.Hkv, self.d = n_q_heads, n_kv_heads, head_dim
@@ -125,7 +129,8 @@ class OracleStream:
         self.chunk, self.window, self.n_sink = chunk, window, n_sink
         self._p = _Params(n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, reps_per_span,
                           max_spans_per_region, theta_mode, theta, softmax_scale, max_tokens,
-                          rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, persist_decode)
+                          rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, persist_decode, unit_tokens)
+        self.unit_tokens = unit_tokens
         self._h = lib().orc_create(C.byref(self._p))
         if not self._h:
             raise ValueError("bad oracle parameters")
@@ -306,6 +311,15 @@ class OracleStream:
         gaps = np.zeros(self.Hkv, dtype=np.float64)
         lib().orc_get_selected(self._h, _ptr(ids), _ptr(gaps))
         return ids, gaps
+
+    def unit_scores(self) -> np.ndarray:
+        """Unit mode: score of every unit that meets the indexed range, [Hkv][units]; unit i is the absolute unit
+        n_sink // unit_tokens + i (Eq. 8: the maximum over the unit's spans)."""
+        n = lib().orc_num_units(self._h)
+        a = np.zeros((self.Hkv, n), dtype=np.float32)
+        if n:
+            lib().orc_get_unit_scores(self._h, _ptr(a))
+        return a
 
     def persistent(self) -> np.ndarray:
         """Span ids [Hkv][top_k] kept through decode by the persistent mechanism (-1 padded)."""

@@ -907,10 +907,30 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     sq = seq;
   }
   const size_t unit = unit_of(c, sq, layer);
-  const int N = c.n_spans[unit];
+  const int nspans = c.n_spans[unit];
   const float* sc = c.scores + (unit * c.Hkv + g) * (size_t)c.cap;
-  const int K = min(c.topk, N);
   const int tid = threadIdx.x, nt = blockDim.x;
+  // What is ranked: the spans themselves, or (Eq. 8 as printed) fixed units of c.unit tokens on the absolute token
+  // grid, each scored by the maximum over the spans it meets.  N = number of candidates, KEY(i) = order key of
+  // candidate i.
+  extern __shared__ unsigned ukey[];  // unit mode: order key of every unit that meets the indexed range [Ls, E)
+  const int U = c.unit;
+  int N = nspans, u0 = 0, Eend = 0;
+  if (U > 0) {
+    Eend = nspans > 0 ? c.span_start[unit * c.cap + nspans - 1] + c.span_len[unit * c.cap + nspans - 1] : c.Ls;
+    u0 = c.Ls / U;
+    N = Eend > c.Ls ? (Eend + U - 1) / U - u0 : 0;
+    for (int i = tid; i < N; i += nt) ukey[i] = 0u;  // below the key of every real score
+    __syncthreads();
+    for (int s = tid; s < nspans; s += nt) {
+      const int st = c.span_start[unit * c.cap + s], ln = c.span_len[unit * c.cap + s];
+      const unsigned key = order_key(sc[s]);
+      for (int u = st / U; u <= (st + ln - 1) / U; ++u) atomicMax(&ukey[u - u0], key);
+    }
+    __syncthreads();
+  }
+  auto KEY = [&](int i) -> unsigned { return U > 0 ? ukey[i] : order_key(sc[i]); };
+  const int K = min(c.topk, N);
   if (tid == 0) s_cnt = 0;
   __syncthreads();
   if (K == N) {
@@ -928,7 +948,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
       const unsigned prefix = s_prefix;
       const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
       for (int s = tid; s < N; s += nt) {
-        const unsigned key = order_key(sc[s]);
+        const unsigned key = KEY(s);
         if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
       }
       __syncthreads();
@@ -948,7 +968,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     const int per = (N + nt - 1) / nt;
     const int lo = tid * per, hi = min(N, lo + per);
     int eq = 0;
-    for (int s = lo; s < hi; ++s) eq += order_key(sc[s]) == T;
+    for (int s = lo; s < hi; ++s) eq += KEY(s) == T;
     s_scan[tid] = eq;
     __syncthreads();
     if (tid == 0) {
@@ -962,7 +982,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     __syncthreads();
     int eqrank = s_scan[tid];
     for (int s = lo; s < hi; ++s) {
-      const unsigned key = order_key(sc[s]);
+      const unsigned key = KEY(s);
       bool take = key > T;
       if (key == T) {
         take = (unsigned)eqrank < need_eq;
@@ -985,6 +1005,8 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   __syncthreads();
   if (tid < cnt) s_ids[rank] = myid;
   __syncthreads();
+  if (U > 0 && tid < cnt) s_ids[tid] += u0;  // absolute unit ids
+  __syncthreads();
   int* sel = c.sel + (unit * c.Hkv + g) * (size_t)c.topk;
   for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
   // token ranges of the attention kernels: the spans' extents are fetched in parallel, merged (adjacent spans become
@@ -996,8 +1018,14 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     ids_all = s_all;
   }
   if (tid < nall) {
-    s_sst[tid] = c.span_start[unit * c.cap + ids_all[tid]];
-    s_sln[tid] = c.span_len[unit * c.cap + ids_all[tid]];
+    if (U > 0) {  // the unit's tokens inside the indexed range
+      const int st = max(ids_all[tid] * U, c.Ls);
+      s_sst[tid] = st;
+      s_sln[tid] = min((ids_all[tid] + 1) * U, Eend) - st;
+    } else {
+      s_sst[tid] = c.span_start[unit * c.cap + ids_all[tid]];
+      s_sln[tid] = c.span_len[unit * c.cap + ids_all[tid]];
+    }
   }
   __syncthreads();
   if (tid == 0) {
@@ -1509,15 +1537,21 @@ cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int la
 }
 int dec_retrieve_fused_max_spans() { return kRetCluster * kRetSliceMax; }
 
+// dynamic shared memory of k_topk: one order key per unit in unit mode (at most 12K units: 48 KB), nothing otherwise
+static int topk_unit_smem(const DevCtx& c) {
+  return c.unit > 0 ? (int)sizeof(unsigned) * (int)(c.Tmax / c.unit + 2) : 0;
+}
+
 cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
   DecBatch dummy;
   dummy.n = 0;
-  k_topk<false><<<dim3(c.Hkv, a.layer_count), 512, 0, s>>>(c, a.seq, a.layer_begin, dummy, a.layer_count);
+  k_topk<false><<<dim3(c.Hkv, a.layer_count), 512, topk_unit_smem(c), s>>>(c, a.seq, a.layer_begin, dummy,
+                                                                           a.layer_count);
   return cudaGetLastError();
 }
 
 cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s) {
-  k_topk<true><<<dim3(c.Hkv, b.n * layer_count), 512, 0, s>>>(c, 0, layer_begin, b, layer_count);
+  k_topk<true><<<dim3(c.Hkv, b.n * layer_count), 512, topk_unit_smem(c), s>>>(c, 0, layer_begin, b, layer_count);
   return cudaGetLastError();
 }
 

@@ -58,6 +58,10 @@ bool validate(const ltri_params* p) {
   if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
   if (!(p->softmax_scale >= 0.f)) return false;
   if (p->flags & ~(uint32_t)(LTRI_FLAG_PERSIST_DECODE | LTRI_FLAG_HOST_STAGING)) return false;
+  if (p->unit_tokens != 0) {
+    if (p->unit_tokens < 8 || p->unit_tokens > p->chunk || p->unit_tokens % 8) return false;
+    if (p->max_tokens / p->unit_tokens + 2 > 12288) return false;  // unit keys of the top-k kernel: 48 KB of shared memory
+  }
   if (p->rep_mode != 0 && p->rep_mode != 1) return false;
   if (p->rep_mode == 1) {
     if (p->ratio_kind < 0 || p->ratio_kind > 2) return false;
@@ -95,6 +99,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.cap = (int)std::min<long long>((long long)1 << 30, ((p.max_tokens + p.chunk - 1) / p.chunk + 8) * d.Jmax);
   d.theta_mode = p.theta_mode;
   d.theta = p.theta;
+  d.unit = p.unit_tokens;
   d.rep_mode = p.rep_mode;
   d.ratio_kind = p.ratio_kind;
   d.min_reps = p.min_reps;
@@ -581,7 +586,8 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
     // enough heads to fill the GPU and the index fits one CTA (12K spans), a cluster of eight CTAs per head for a larger
     // index (up to 98K spans); otherwise the scores go through global memory in two launches
     const bool one_cta = ub <= 12288;
-    const bool fused = ub <= dec_retrieve_fused_max_spans() &&
+    // (unit-granular retrieval ranks units, which only the two-launch path does)
+    const bool fused = d.unit == 0 && ub <= dec_retrieve_fused_max_spans() &&
                        (ctx->dec_fused >= 1 || (ctx->dec_fused < 0 && (!one_cta || units >= ctx->sm_count)));
     if (fused) {
       Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 1);

@@ -65,6 +65,7 @@ class StreamConfig:
     min_reps: int = 1
     max_reps: int = 4
     rep_lambda: float = 2.0
+    unit_tokens: int = 0           # retrieval granularity: 0 = spans, U = fixed units of U tokens (Eq. 8 as printed)
     persist_decode: bool = False   # decode keeps the spans selected by the last prefill call (Sec. 3.5)
 
     @property

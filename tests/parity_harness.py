@@ -50,7 +50,8 @@ def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
                                reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
                                theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode,
                                ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps, max_reps=cfg.max_reps,
-                               rep_lambda=cfg.rep_lambda, flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0)
+                               rep_lambda=cfg.rep_lambda, flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0,
+                               unit_tokens=cfg.unit_tokens)
 
 
 def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
@@ -58,7 +59,8 @@ def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
                             cfg.max_tokens, reps_per_span=cfg.reps_per_span,
                             max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
-                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda, persist_decode=int(cfg.persist_decode))
+                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda, persist_decode=int(cfg.persist_decode),
+                            unit_tokens=cfg.unit_tokens)
 
 
 def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str):
@@ -76,7 +78,13 @@ def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str
 def check_selection(sel_gpu: np.ndarray, o: orc.OracleStream, rep: Report, what: str):
     """sel_gpu [Hkv][k] ascending ids (-1 padded) against the oracle's scores; adopts tolerated picks."""
     sel_o, _ = o.selected()
-    sc = o.scores()
+    if o.unit_tokens > 0:
+        # unit mode: the ids are absolute unit numbers, the scores those of the units that meet the indexed range
+        us = o.unit_scores()
+        u0 = o.n_sink // o.unit_tokens
+        sc = [{u0 + i: us[g][i] for i in range(us.shape[1])} for g in range(us.shape[0])]
+    else:
+        sc = o.scores()
     adopt = False
     for g in range(sel_gpu.shape[0]):
         a = set(int(x) for x in sel_gpu[g] if x >= 0)
@@ -246,10 +254,14 @@ class StreamPair:
                     sel_o, _ = o.selected()
                     pers = o.persistent() if cfg.persist_decode else np.full_like(sel_o, -1)
                     sp = o.spans()
+                    U, E = cfg.unit_tokens, o.evicted_end
                     want = 0
                     for g in range(sel_o.shape[0]):
                         ids = set(int(x) for x in sel_o[g] if x >= 0) | set(int(x) for x in pers[g] if x >= 0)
-                        want += sum(int(sp[j, 1]) for j in ids)
+                        if U > 0:
+                            want += sum(min((j + 1) * U, E) - max(j * U, cfg.n_sink) for j in ids)
+                        else:
+                            want += sum(int(sp[j, 1]) for j in ids)
                     got = int(lt.ltri_get_stats(seq, layer).retrieved_tokens)
                     assert got == want, f"{what}: attends over {got} retrieved tokens, oracle {want}"
                 check_output(out[i, layer], o.decode_attend(), rep, what)

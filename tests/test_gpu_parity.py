@@ -81,6 +81,16 @@ def test_maximum_sizes():
     print(rep)
 
 
+@pytest.mark.parametrize("U,persist", [(64, False), (128, False), (40, True)])
+def test_unit_granular_retrieval(U, persist):
+    # Eq. 8 as printed: fixed units of U tokens ranked by the maximum over their spans and fetched whole; unit
+    # selections, the token count of every decode step and the outputs are checked against the oracle
+    cfg = small_cfg(n_layers=2, context=1536, decode_steps=4, unit_tokens=U, persist_decode=persist, top_k=3)
+    rep = ph.run_stream(cfg, layers=[0, 1])
+    assert rep.sel_checks > 20
+    print(rep)
+
+
 def test_top_k_covering_everything_equals_full_attention():
     # with top_k >= number of spans the streamed output is plain causal attention (oracle O12)
     cfg = small_cfg(n_layers=1, context=640, chunk=64, window=128, top_k=64, max_spans_per_region=2, decode_steps=2)
