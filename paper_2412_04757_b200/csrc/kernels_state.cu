@@ -483,7 +483,6 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   __shared__ long long skey[2048];
   __shared__ short scd[2048];
   __shared__ int kx[kMaxTopK], ky[kMaxTopK];
-  __shared__ int s_kept;
   __shared__ int out_start[2 * kMaxTopK + 1], out_len[2 * kMaxTopK + 1];
   __shared__ int s_nout;
   const int layer = a.layer_begin + blockIdx.x;
@@ -578,7 +577,6 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
         out_len[no++] = m - pos;
       }
       s_nout = no;
-      s_kept = kept;
     }
   }
   __syncthreads();
@@ -1323,7 +1321,6 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
   __shared__ int s_eq, s_take;    // this CTA's count of scores equal to the threshold / of selected scores
   __shared__ int s_ids[kMaxTopK]; // first CTA: all selected ids, ascending
   __shared__ int s_loc[kMaxTopK]; // this CTA's selected ids
-  __shared__ int s_cnt;
   __shared__ int s_scan[kRetThreads];
   __shared__ int s_rs[kMaxRanges], s_rl[kMaxRanges], s_nr, s_sst[2 * kMaxTopK], s_sln[2 * kMaxTopK];
   __shared__ int s_all[2 * kMaxTopK], s_nall;
@@ -1342,7 +1339,6 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
     for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
     su[tid] = acc;
   }
-  if (tid == 0) s_cnt = 0;
   __syncthreads();
   // ---- scores of the slice
   {
