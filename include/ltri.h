@@ -75,6 +75,10 @@ typedef struct {
                                                         score is the maximum over the spans it meets, the k best units
                                                         are fetched whole (clipped to the indexed range) and
                                                         ltri_get_selected reports unit numbers (token / U) */
+  int32_t nms_iou_milli;                             /* NMS IoU threshold phi in thousandths, 0..999 (App. "NMS Input
+                                                        Filtration", boxes = squares on the diagonal).  0: kept spans
+                                                        never overlap and the spans partition the region; > 0: kept
+                                                        spans may overlap, the gaps are the runs none of them covers */
   void* arena;                                       /* caller-owned device memory, 256-byte aligned */
   size_t arena_bytes;                                /* >= ltri_arena_bytes(params) */
 } ltri_params;

@@ -92,6 +92,8 @@ struct Params {
   // retrieval granularity (Eq. 8 as printed): 0 = the span; U > 0 = fixed units of U tokens on the absolute token
   // grid, scored by the maximum over the spans they meet and fetched whole (clipped to the indexed range)
   int32_t unit_tokens;
+  // NMS IoU threshold phi in thousandths (0: spans never overlap)
+  int32_t nms_iou_milli;
 };
 
 // ---------------------------------------------------------------------------
@@ -174,13 +176,16 @@ inline double rel_gap(int64_t a, int64_t b) {
   return std::fabs(da - db) / den;
 }
 
-// O6: anti-diagonal filter, sort, greedy disjoint NMS (IoU threshold 0), gap fill.
+// O6: anti-diagonal filter, sort, greedy NMS, gap fill.  A candidate is suppressed when its IoU with a kept one
+// exceeds phi = phi_milli / 1000, the boxes being the squares (x, x, y+1, y+1) on the diagonal: two spans that share
+// `inter` tokens have IoU = inter^2 / (L1^2 + L2^2 - inter^2).  phi = 0: any overlap suppresses and the spans
+// partition the region; phi > 0: kept spans may overlap, and the gaps are the runs no kept span covers.
 // `min_gap` (optional) receives the smallest relative gap between two quantities whose
 // comparison decided something: best vs runner-up on an anti-diagonal that produced a
 // candidate; the best point's triangle mass vs its theta*area (the sign test S>0) on every
 // anti-diagonal; and neighbours in the sorted candidate list up to the last one the
 // greedy pass looked at.
-void segment_map(const int32_t* Mq, int m, int ld, int64_t thq, int C, std::vector<Span>& out,
+void segment_map(const int32_t* Mq, int m, int ld, int64_t thq, int C, int phi_milli, std::vector<Span>& out,
                  double* min_gap) {
   out.clear();
   double gap = 1.0;
@@ -235,21 +240,25 @@ void segment_map(const int32_t* Mq, int m, int ld, int64_t thq, int C, std::vect
     examined = ci + 1;
     const Cand& c = cands[ci];
     bool ok = true;
-    for (const Cand& k : kept)
-      if (!(c.y < k.x || c.x > k.y)) {
+    for (const Cand& k : kept) {
+      const int64_t inter = std::min(c.y, k.y) - std::max(c.x, k.x) + 1;
+      if (inter <= 0) continue;
+      const int64_t l1 = c.y - c.x + 1, l2 = k.y - k.x + 1, i2 = inter * inter;
+      if (i2 * 1000 > (int64_t)phi_milli * (l1 * l1 + l2 * l2 - i2)) {
         ok = false;
         break;
       }
+    }
     if (ok) kept.push_back(c);
   }
   for (size_t ci = 0; ci + 1 < cands.size() && ci < examined; ++ci)
     gap = std::min(gap, rel_gap(cands[ci].S, cands[ci + 1].S));
-  std::sort(kept.begin(), kept.end(), [](const Cand& a, const Cand& b) { return a.x < b.x; });
-  int pos = 0;
+  std::sort(kept.begin(), kept.end(), [](const Cand& a, const Cand& b) { return a.x != b.x ? a.x < b.x : a.y < b.y; });
+  int pos = 0;  // first token no span emitted so far covers
   for (const Cand& k : kept) {
     if (k.x > pos) out.push_back(Span{pos, k.x - pos});
     out.push_back(Span{k.x, k.y - k.x + 1});
-    pos = k.y + 1;
+    pos = std::max(pos, k.y + 1);
   }
   if (pos < m) out.push_back(Span{pos, m - pos});
   if (min_gap) *min_gap = gap;
@@ -519,7 +528,7 @@ struct Stream {
     if (m > 0) {
       thq = theta_q(Mq.data(), m, m, p.theta_mode, p.theta, Hq);
       std::vector<Span> sp;
-      segment_map(Mq.data(), m, m, thq, p.max_spans_per_region, sp, &seg_gap);
+      segment_map(Mq.data(), m, m, thq, p.max_spans_per_region, p.nms_iou_milli, sp, &seg_gap);
       for (Span& s : sp) s.start += reg_start;
       reg.spans = sp;
       decide_rep_counts(reg);
@@ -611,6 +620,19 @@ struct Stream {
         int s = persist[(size_t)g * p.top_k + i];
         if (s >= 0 && std::find(ids.begin(), ids.end(), s) == ids.end()) ids.push_back(s);
       }
+    if (p.nms_iou_milli > 0 && p.unit_tokens == 0) {
+      // selected spans may overlap: every token once (ranges in position order, overlaps merged)
+      std::sort(ids.begin(), ids.end());
+      for (int s : ids) {
+        const int a = spans[s].start, b = spans[s].start + spans[s].len;
+        if (ranges.size() > 1 && a <= ranges.back().second)
+          ranges.back().second = std::max(ranges.back().second, b);
+        else
+          ranges.push_back({a, b});
+      }
+      ranges.push_back({loc_begin, loc_end});
+      return ranges;
+    }
     for (int s : ids) {
       if (p.unit_tokens > 0)  // the unit's tokens inside the indexed range [n_sink, E)
         ranges.push_back({std::max(s * p.unit_tokens, p.n_sink), std::min((s + 1) * p.unit_tokens, E)});
@@ -709,7 +731,7 @@ void* orc_create(const Params* p) {
   if (!p || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads) return nullptr;
   if (p->head_dim < 1 || p->chunk < 1 || p->window < 1 || p->n_sink < 1 || p->top_k < 1) return nullptr;
   if (p->reps_per_span < 1 || p->max_spans_per_region < 1 || p->max_tokens < 1) return nullptr;
-  if (p->unit_tokens < 0) return nullptr;
+  if (p->unit_tokens < 0 || p->nms_iou_milli < 0 || p->nms_iou_milli >= 1000) return nullptr;
   if (p->rep_mode != 0 && p->rep_mode != 1) return nullptr;
   if (p->rep_mode == 1 && (p->ratio_kind < 0 || p->ratio_kind > 2 || p->min_reps < 1 || p->max_reps < p->min_reps ||
                            !(p->rep_lambda >= 0.f)))
@@ -776,10 +798,12 @@ int orc_set_newest_spans(void* h, const int* start_len, int cnt) {
   Stream* s = (Stream*)h;
   if (s->pending.empty()) return -1;
   Region& reg = s->pending.back();
-  int pos = reg.start;
+  int pos = reg.start;  // first token not covered yet: the spans come sorted by start and leave no hole
   for (int i = 0; i < cnt; ++i) {
-    if (start_len[2 * i] != pos || start_len[2 * i + 1] < 1) return -1;
-    pos += start_len[2 * i + 1];
+    const int st = start_len[2 * i], ln = start_len[2 * i + 1];
+    if (ln < 1 || st > pos || st < reg.start || (s->p.nms_iou_milli == 0 && st != pos)) return -1;
+    if (i > 0 && st < start_len[2 * i - 2]) return -1;
+    pos = std::max(pos, st + ln);
   }
   if (pos != reg.end) return -1;
   reg.spans.clear();
@@ -865,9 +889,9 @@ void orc_ta_scores(const int32_t* Mq, int m, int64_t thq, int64_t* S) {  // S[x*
   ta_scores(Mq, m, m, thq, s);
   std::memcpy(S, s.data(), s.size() * sizeof(int64_t));
 }
-int orc_segment_map(const int32_t* Mq, int m, int64_t thq, int C, int* start_len, int cap, double* gap) {
+int orc_segment_map(const int32_t* Mq, int m, int64_t thq, int C, int phi_milli, int* start_len, int cap, double* gap) {
   std::vector<Span> sp;
-  segment_map(Mq, m, m, thq, C, sp, gap);
+  segment_map(Mq, m, m, thq, C, phi_milli, sp, gap);
   for (size_t i = 0; i < sp.size() && (int)i < cap; ++i) {
     start_len[2 * i] = sp[i].start;
     start_len[2 * i + 1] = sp[i].len;

@@ -38,7 +38,7 @@ class LtriParams(C.Structure):
         ("reps_per_span", C.c_int32), ("max_spans_per_region", C.c_int32),
         ("theta_mode", C.c_int32), ("theta", C.c_float), ("softmax_scale", C.c_float), ("flags", C.c_uint32),
         ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
-        ("rep_lambda", C.c_float), ("unit_tokens", C.c_int32),
+        ("rep_lambda", C.c_float), ("unit_tokens", C.c_int32), ("nms_iou_milli", C.c_int32),
         ("arena", C.c_void_p), ("arena_bytes", C.c_size_t),
     ]
 
@@ -103,10 +103,10 @@ def strerror(code: int) -> str:
 
 def make_params(n_layers, n_q_heads, n_kv_heads, max_tokens, chunk, window, n_sink, top_k, head_dim=128, max_seqs=1,
                 reps_per_span=1, max_spans_per_region=0, theta_mode=1, theta=0.90, softmax_scale=0.0,
-                rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, flags=0, unit_tokens=0) -> LtriParams:
+                rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, flags=0, unit_tokens=0, nms_iou_milli=0) -> LtriParams:
     return LtriParams(n_layers, n_q_heads, n_kv_heads, head_dim, max_seqs, max_tokens, chunk, window, n_sink, top_k,
                       reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, flags,
-                      rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, unit_tokens, None, 0)
+                      rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, unit_tokens, nms_iou_milli, None, 0)
 
 
 def ltri_arena_bytes(params: LtriParams) -> int:

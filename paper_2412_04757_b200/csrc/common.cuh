@@ -26,6 +26,7 @@ struct DevCtx {
   long long Tmax;
   int chunk, W, Ls, topk, reps, C, Jmax, cap, slots;
   int rcap;              // token ranges kept per (seq, layer, KV head): 2 * top_k + 2
+  int phi_milli;         // NMS IoU threshold in thousandths (0: spans never overlap)
   int unit;              // retrieval granularity: 0 = span, U > 0 = units of U tokens (Eq. 8 as printed)
   int persist;           // decode keeps the spans selected by the last prefill call (Sec. 3.5, persistent mechanism)
   int theta_mode;

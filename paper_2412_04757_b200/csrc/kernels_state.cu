@@ -473,6 +473,16 @@ __global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin,
 // step 4: sort the <= 2m-1 candidates by (S desc, length asc, start asc), greedy non-maximum suppression with
 // IoU threshold 0 until max_spans are kept, gap fill, store the region's spans in its pending slot; then the
 // query representatives of every span (Sec. 3.4 step 2): u[g][j] = sum_{h in g} sum_{rep tokens} q_h[tok].
+// NMS on the squares (x, x, y+1, y+1): a candidate is suppressed by a kept span when their IoU exceeds phi_milli/1000;
+// two spans that share `inter` tokens have IoU = inter^2 / (L1^2 + L2^2 - inter^2).  Integer arithmetic; phi = 0
+// means any overlap suppresses.
+__device__ __forceinline__ bool nms_suppressed(int x, int y, int kx, int ky, int phi_milli) {
+  const long long inter = (long long)min(y, ky) - max(x, kx) + 1;
+  if (inter <= 0) return false;
+  const long long l1 = y - x + 1, l2 = ky - kx + 1, i2 = inter * inter;
+  return i2 * 1000 > (long long)phi_milli * (l1 * l1 + l2 * l2 - i2);
+}
+
 struct NmsArgs {
   int seq, layer_begin, m, reg_start, slot, max_spans;
   int n, t0;                 // query tensor geometry (q == nullptr: skip the representatives)
@@ -488,6 +498,7 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   const int layer = a.layer_begin + blockIdx.x;
   const size_t unit = unit_of(c, a.seq, layer);
   const int m = a.m;
+  const int phi_milli = c.phi_milli;
   const int ncand = 2 * m - 1;
   int npow = 1;
   while (npow < ncand) npow <<= 1;
@@ -529,7 +540,7 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
       const int y = x + len;
       bool alive = key > 0;
       if (__ballot_sync(0xffffffffu, alive) == 0) break;  // sorted: nothing positive follows
-      for (int q = 0; q < kept; ++q) alive = alive && (y < kx[q] || x > ky[q]);
+      for (int q = 0; q < kept; ++q) alive = alive && !nms_suppressed(x, y, kx[q], ky[q], phi_milli);
       unsigned mask = __ballot_sync(0xffffffffu, alive);
       while (mask && kept < a.max_spans) {
         const int f = __ffs(mask) - 1;
@@ -539,7 +550,7 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
           ky[kept] = fy;
         }
         ++kept;
-        alive = alive && lane != f && (y < fx || x > fy);
+        alive = alive && lane != f && !nms_suppressed(x, y, fx, fy, phi_milli);
         mask = __ballot_sync(0xffffffffu, alive);
       }
       __syncwarp();
@@ -549,11 +560,11 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
     int rank0 = 0, rank1 = 0;
     const int x0 = lane < kept ? kx[lane] : 0x7fffffff;
     const int x1 = lane + 32 < kept ? kx[lane + 32] : 0x7fffffff;
-    for (int q = 0; q < kept; ++q) {
-      rank0 += kx[q] < x0;
-      rank1 += kx[q] < x1;
-    }
     const int y0 = lane < kept ? ky[lane] : 0, y1 = lane + 32 < kept ? ky[lane + 32] : 0;
+    for (int q = 0; q < kept; ++q) {  // with phi > 0 two kept spans may share their start: then the shorter first
+      rank0 += kx[q] < x0 || (kx[q] == x0 && ky[q] < y0);
+      rank1 += kx[q] < x1 || (kx[q] == x1 && ky[q] < y1);
+    }
     __syncwarp();
     if (lane < kept) kx[rank0] = x0;
     if (lane + 32 < kept) kx[rank1] = x1;
@@ -570,7 +581,7 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
         }
         out_start[no] = kx[q];
         out_len[no++] = ky[q] - kx[q] + 1;
-        pos = ky[q] + 1;
+        pos = max(pos, ky[q] + 1);  // kept spans may overlap when phi > 0
       }
       if (pos < m) {
         out_start[no] = pos;
@@ -883,7 +894,8 @@ __device__ __forceinline__ unsigned order_key(float f) {
 }
 
 template <bool DECODE>
-__global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin, DecBatch b, int layer_count) {
+__global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin, DecBatch b, int layer_count,
+                                              int evicted_end) {
   __shared__ unsigned hist[256];
   __shared__ unsigned s_prefix, s_need;
   __shared__ int s_ids[kMaxTopK];
@@ -915,7 +927,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   const int U = c.unit;
   int N = nspans, u0 = 0, Eend = 0;
   if (U > 0) {
-    Eend = nspans > 0 ? c.span_start[unit * c.cap + nspans - 1] + c.span_len[unit * c.cap + nspans - 1] : c.Ls;
+    Eend = nspans > 0 ? (DECODE ? loc_begin : evicted_end) : c.Ls;  // end of the indexed range
     u0 = c.Ls / U;
     N = Eend > c.Ls ? (Eend + U - 1) / U - u0 : 0;
     for (int i = tid; i < N; i += nt) ukey[i] = 0u;  // below the key of every real score
@@ -1031,8 +1043,8 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     long long tokens = 0;
     auto push = [&](int st, int ln) {
       if (ln <= 0) return;
-      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] == st)
-        s_rl[nr - 1] += ln;
+      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] >= st)  // adjacent, or (NMS with phi > 0) overlapping: one range
+        s_rl[nr - 1] = max(s_rl[nr - 1], st + ln - s_rs[nr - 1]);
       else {
         s_rs[nr] = st;
         s_rl[nr] = ln;
@@ -1272,8 +1284,8 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     long long tokens = 0;
     auto push = [&](int st, int ln) {
       if (ln <= 0) return;
-      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] == st)
-        s_rl[nr - 1] += ln;
+      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] >= st)  // adjacent, or (NMS with phi > 0) overlapping: one range
+        s_rl[nr - 1] = max(s_rl[nr - 1], st + ln - s_rs[nr - 1]);
       else {
         s_rs[nr] = st;
         s_rl[nr] = ln;
@@ -1491,8 +1503,8 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
     long long tokens = 0;
     auto push = [&](int st, int ln) {
       if (ln <= 0) return;
-      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] == st)
-        s_rl[nr - 1] += ln;
+      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] >= st)  // adjacent, or (NMS with phi > 0) overlapping: one range
+        s_rl[nr - 1] = max(s_rl[nr - 1], st + ln - s_rs[nr - 1]);
       else {
         s_rs[nr] = st;
         s_rl[nr] = ln;
@@ -1542,12 +1554,12 @@ cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStrea
   DecBatch dummy;
   dummy.n = 0;
   k_topk<false><<<dim3(c.Hkv, a.layer_count), 512, topk_unit_smem(c), s>>>(c, a.seq, a.layer_begin, dummy,
-                                                                           a.layer_count);
+                                                                           a.layer_count, a.loc_begin);
   return cudaGetLastError();
 }
 
 cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s) {
-  k_topk<true><<<dim3(c.Hkv, b.n * layer_count), 512, topk_unit_smem(c), s>>>(c, 0, layer_begin, b, layer_count);
+  k_topk<true><<<dim3(c.Hkv, b.n * layer_count), 512, topk_unit_smem(c), s>>>(c, 0, layer_begin, b, layer_count, 0);
   return cudaGetLastError();
 }
 

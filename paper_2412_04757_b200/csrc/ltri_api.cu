@@ -58,6 +58,7 @@ bool validate(const ltri_params* p) {
   if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
   if (!(p->softmax_scale >= 0.f)) return false;
   if (p->flags & ~(uint32_t)(LTRI_FLAG_PERSIST_DECODE | LTRI_FLAG_HOST_STAGING)) return false;
+  if (p->nms_iou_milli < 0 || p->nms_iou_milli > 999) return false;
   if (p->unit_tokens != 0) {
     if (p->unit_tokens < 8 || p->unit_tokens > p->chunk || p->unit_tokens % 8) return false;
     if (p->max_tokens / p->unit_tokens + 2 > 12288) return false;  // unit keys of the top-k kernel: 48 KB of shared memory
@@ -100,6 +101,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.theta_mode = p.theta_mode;
   d.theta = p.theta;
   d.unit = p.unit_tokens;
+  d.phi_milli = p.nms_iou_milli;
   d.rep_mode = p.rep_mode;
   d.ratio_kind = p.ratio_kind;
   d.min_reps = p.min_reps;

@@ -65,6 +65,7 @@ class StreamConfig:
     min_reps: int = 1
     max_reps: int = 4
     rep_lambda: float = 2.0
+    nms_iou_milli: int = 0         # NMS IoU threshold in thousandths (0: spans never overlap)
     unit_tokens: int = 0           # retrieval granularity: 0 = spans, U = fixed units of U tokens (Eq. 8 as printed)
     persist_decode: bool = False   # decode keeps the spans selected by the last prefill call (Sec. 3.5)
 

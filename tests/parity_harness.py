@@ -51,7 +51,7 @@ def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
                                theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode,
                                ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps, max_reps=cfg.max_reps,
                                rep_lambda=cfg.rep_lambda, flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0,
-                               unit_tokens=cfg.unit_tokens)
+                               unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli)
 
 
 def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
@@ -60,7 +60,7 @@ def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
                             max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
                             max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda, persist_decode=int(cfg.persist_decode),
-                            unit_tokens=cfg.unit_tokens)
+                            unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli)
 
 
 def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str):
@@ -155,7 +155,7 @@ class StreamPair:
                     if cfg.theta_mode == 1:
                         assert thg == orc.theta_q(Mg, 1, cfg.theta, cfg.n_q_heads), f"{what}: theta rank select"
                     # integer pipeline: bit-exact on identical integer input
-                    ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region)
+                    ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region, cfg.nms_iou_milli)
                     ref_spans[:, 0] += rs
                     assert newest_g.tolist() == ref_spans.tolist(), f"{what}: segmenter differs on its own map"
                 if newest_g.tolist() != spans_o.tolist():

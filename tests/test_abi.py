@@ -31,8 +31,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_struct_sizes_match_header(lib):
-    # the C struct has 21 int32/float fields, one int64, a pointer and a size_t with natural alignment
-    assert ctypes.sizeof(binding.LtriParams) == 112
+    # the C struct has 23 int32/float fields, one int64, a pointer and a size_t with natural alignment
+    assert ctypes.sizeof(binding.LtriParams) == 120
     assert ctypes.sizeof(binding.LtriStats) == 48
 
 
@@ -49,7 +49,7 @@ def test_arena_sizing_is_host_only_and_monotone(lib):
     dict(n_sink=0), dict(n_sink=512), dict(window=0), dict(reps_per_span=9), dict(theta=1.5), dict(theta_mode=3),
     dict(max_tokens=0), dict(max_seqs=0), dict(n_kv_heads=3), dict(rep_mode=2), dict(rep_mode=1, max_reps=9),
     dict(rep_mode=1, min_reps=0), dict(rep_mode=1, min_reps=3, max_reps=2), dict(rep_mode=1, ratio_kind=3),
-    dict(rep_mode=1, rep_lambda=-1.0),
+    dict(rep_mode=1, rep_lambda=-1.0), dict(unit_tokens=12), dict(unit_tokens=512), dict(nms_iou_milli=1000),
 ])
 def test_bad_parameters_are_rejected_on_the_host(lib, kw):
     base = dict(n_layers=1, n_q_heads=8, n_kv_heads=2, max_tokens=1024, chunk=256, window=512, n_sink=64, top_k=4)

@@ -91,6 +91,16 @@ def test_unit_granular_retrieval(U, persist):
     print(rep)
 
 
+@pytest.mark.parametrize("phi_milli,U", [(300, 0), (500, 0), (300, 64)])
+def test_overlapping_spans_from_nms_with_iou_threshold(phi_milli, U):
+    # NMS with an IoU threshold above zero: spans overlap, selected overlapping spans are attended once per token
+    cfg = small_cfg(n_layers=2, context=1536, decode_steps=4, nms_iou_milli=phi_milli, unit_tokens=U, top_k=6,
+                    max_spans_per_region=8)
+    rep = ph.run_stream(cfg, layers=[0, 1])
+    assert rep.sel_checks > 20
+    print(rep)
+
+
 def test_top_k_covering_everything_equals_full_attention():
     # with top_k >= number of spans the streamed output is plain causal attention (oracle O12)
     cfg = small_cfg(n_layers=1, context=640, chunk=64, window=128, top_k=64, max_spans_per_region=2, decode_steps=2)

@@ -85,3 +85,23 @@ def test_bad_arguments(lt):
         lt.ltri_debug_segment_map(np.zeros((1024, 1024), dtype=np.int32), theta_mode=2)   # m > chunk
     with pytest.raises(binding.LtriError):
         lt.ltri_debug_segment_map(Mq, theta_mode=2, max_spans=64)                       # > context's C
+
+
+@pytest.mark.parametrize("phi_milli", [100, 300, 600])
+def test_nms_with_iou_threshold_matches_oracle_exactly(phi_milli):
+    # kept spans may overlap once the IoU threshold is above zero; integer rule, so bit-exact on the same map
+    p = binding.make_params(1, 8, 2, 4096, 512, 1024, 64, 4, max_spans_per_region=16, nms_iou_milli=phi_milli)
+    lt = binding.Ltri(p)
+    rng = np.random.default_rng(900 + phi_milli)
+    overlaps = 0
+    for m in (17, 64, 200, 512):
+        for _ in range(3):
+            Mq = np.tril(rng.integers(0, 2**20, size=(m, m))).astype(np.int32)
+            thq = int(np.quantile(Mq[np.tril_indices(m)], 0.85))
+            for C in (3, 16):
+                ref, _ = orc.segment_map(Mq, thq, C, phi_milli)
+                got = lt.ltri_debug_segment_map(Mq, theta_mode=2, theta_q=thq, max_spans=C)
+                assert got.tolist() == ref.tolist()
+                overlaps += sum(a[0] + a[1] > b[0] for a, b in zip(ref, ref[1:]))
+    assert overlaps > 0 or phi_milli < 300      # (a low threshold rarely lets two of these random spans overlap)
+    lt.close()

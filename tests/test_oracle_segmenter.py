@@ -150,8 +150,9 @@ def test_gap_fill_partitions_region_and_respects_cap():
             assert len(spans) <= 2 * C + 1
 
 
+@pytest.mark.parametrize("phi_milli", [0, 100, 300])
 @pytest.mark.parametrize("seed", range(6))
-def test_greedy_nms_matches_torchvision(seed):
+def test_greedy_nms_matches_torchvision(seed, phi_milli):
     tv = pytest.importorskip("torchvision")
     rng = np.random.default_rng(100 + seed)
     m = int(rng.integers(8, 40))
@@ -170,18 +171,20 @@ def test_greedy_nms_matches_torchvision(seed):
         pytest.skip("non-distinct scores; library tie order is unspecified")
     C = 5
     boxes = torch.tensor([[x, x, y + 1, y + 1] for x, y in cands], dtype=torch.float64).reshape(-1, 4)
-    keep = tv.ops.nms(boxes, torch.tensor([float(s) for s in scores], dtype=torch.float64), 0.0)[:C]
+    keep = tv.ops.nms(boxes, torch.tensor([float(s) for s in scores], dtype=torch.float64), phi_milli / 1000.0)[:C]
     kept = sorted(cands[i] for i in keep.tolist())
     expect, pos = [], 0
     for x, y in kept:
         if x > pos:
             expect.append([pos, x - pos])
         expect.append([x, y - x + 1])
-        pos = y + 1
+        pos = max(pos, y + 1)          # with phi > 0 kept spans may overlap
     if pos < m:
         expect.append([pos, m - pos])
-    spans, _ = orc.segment_map(Mq, thq, C)
+    spans, _ = orc.segment_map(Mq, thq, C, phi_milli)
     assert spans.tolist() == expect
+    if phi_milli == 0:                  # a partition
+        assert all(a[0] + a[1] == b[0] for a, b in zip(expect, expect[1:]))
 
 
 def test_anti_diagonal_tie_prefers_shorter_span():

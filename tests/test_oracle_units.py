@@ -88,3 +88,24 @@ def test_covering_every_unit_equals_full_attention():
         q, k, v = st.tokens(cfg.context + s, 1, kind=1)
         out = o.decode_step(q[0, 0], k[0, 0], v[0, 0])
         assert np.abs(out - o.full_attention([cfg.context + s], q[0])[0]).max() < 5e-6
+
+
+@pytest.mark.parametrize("U", [0, 64])
+def test_overlapping_spans_are_attended_once_per_token(U):
+    # NMS with an IoU threshold above zero keeps overlapping spans; selecting all of them must still give plain
+    # causal attention (every token once), span-granular and unit-granular
+    cfg = inputs.StreamConfig("o", 1, 4, 2, 128, 1000, 128, 2, 16, 256, 64, 8, 16, 64, seed=43)
+    st = inputs.SyntheticStream(cfg)
+    o = orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, 64,
+                         cfg.max_tokens, max_spans_per_region=8, nms_iou_milli=500, unit_tokens=U)
+    for t0, n in st.prefill_chunks():
+        q, k, v = st.tokens(t0, n)
+        out = o.prefill_chunk(q[0], k[0], v[0])
+        assert np.abs(out - o.full_attention(list(range(t0, t0 + n)), q[0])).max() < 5e-6
+    sp = o.spans()
+    assert sum(a[0] + a[1] > b[0] for a, b in zip(sp, sp[1:])) > 3      # the spans really overlap
+    assert sp[0][0] == cfg.n_sink and max(a[0] + a[1] for a in sp) == o.evicted_end
+    for s in range(cfg.decode_steps):
+        q, k, v = st.tokens(cfg.context + s, 1, kind=1)
+        out = o.decode_step(q[0, 0], k[0, 0], v[0, 0])
+        assert np.abs(out - o.full_attention([cfg.context + s], q[0])[0]).max() < 5e-6
