@@ -413,7 +413,8 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
                                : launch_attn_prefill(d, a, 0, !has_index, st));
   }
   {
-    Scope sc(ctx, st, LTRI_K_MAP, (a.t0 - a.loc_begin > 0 && a.loc_begin >= d.Ls) ? 2 : 1);
+    // (the tensor-core pass is one kernel; the warp-MMA fallback has one for the local keys and one for the call's own)
+    Scope sc(ctx, st, LTRI_K_MAP, ctx->use_tc ? 1 : ((a.t0 - a.loc_begin > 0 && a.loc_begin >= d.Ls) ? 2 : 1));
     LTRI_CUDA(ctx, ctx->use_tc ? launch_map_pass_tc(d, a, ctx->kv_maps, st) : launch_map_pass(d, a, st));
   }
   if (m > 0) {
