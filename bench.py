@@ -199,7 +199,8 @@ def oracle_sample(cfg, steps, warmup):
                          need + 8, reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
                          theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind,
                          min_reps=cfg.min_reps, max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
-                         unit_tokens=cfg.unit_tokens, persist_decode=int(cfg.persist_decode))
+                         unit_tokens=cfg.unit_tokens, persist_decode=int(cfg.persist_decode),
+                         nms_iou_milli=cfg.nms_iou_milli)
     times = []
     for ci in range(fill + warmup + steps):
         q, k, v = st.tokens(ci * cfg.chunk, cfg.chunk)
@@ -313,7 +314,7 @@ def run_ltri(args, cfg):
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
                             max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
                             flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0,
-                            unit_tokens=cfg.unit_tokens)
+                            unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli)
 
     def stream_until(lt, upto, keep_from):
         for s in range(NSEQ - 1):
@@ -515,6 +516,8 @@ def main():
                          "implementation details, 1..4 per span)")
     ap.add_argument("--unit-tokens", type=int, default=0,
                     help="retrieval granularity: fixed units of this many tokens instead of spans (the paper's 128)")
+    ap.add_argument("--nms-iou", type=float, default=0.0,
+                    help="IoU threshold of the segmenter's NMS (0: spans never overlap; the paper lists 0.1 / 0.01)")
     ap.add_argument("--persist-decode", action="store_true",
                     help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
     ap.add_argument("--p-self", type=float, default=-1.0,
@@ -541,6 +544,10 @@ def main():
         import dataclasses
         cfg = dataclasses.replace(cfg, unit_tokens=args.unit_tokens)
         cfg.name += f"[unit={args.unit_tokens}]"
+    if args.nms_iou > 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, nms_iou_milli=int(round(args.nms_iou * 1000)))
+        cfg.name += f"[nms-iou={args.nms_iou:g}]"
     if args.persist_decode:
         import dataclasses
         cfg = dataclasses.replace(cfg, persist_decode=True)
