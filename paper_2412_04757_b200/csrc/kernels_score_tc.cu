@@ -185,7 +185,7 @@ cudaError_t launch_score_prefill_tc(const DevCtx& c, const PrefillArgs& a, int s
   const int smem = kScStages * 32768 + 3 * 2 * kScMaxN * 128 + 1024;
   cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   const int tiles = (span_bound + 127) / 128;
-  const int per_cta = tiles >= 48 ? 16 : 8;
+  const int per_cta = tiles >= 256 ? 32 : (tiles >= 48 ? 16 : 8);  // amortise the split of the representatives
   const int gx = (tiles + per_cta - 1) / per_cta;
   k_score_tc<<<dim3(gx > 0 ? gx : 1, c.Hkv, a.layer_count), kScThreads, smem, s>>>(c, a.seq, a.layer_begin, per_cta, kr);
   return cudaGetLastError();
