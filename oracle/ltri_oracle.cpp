@@ -24,6 +24,12 @@
 //                                                             block becomes a single token)
 //   O12 full causal attention (reference for the pin
 //       "top-k covers every span => method == full attention")
+// Optional modes (off by default):
+//   O7'  dynamic number of representatives per span            Sec. 3.3.2, Eq. r_v
+//   O6'  NMS with an IoU threshold above zero                  App. "NMS Input Filtration"
+//   O9'  retrieval in fixed token units, unit score = max      Eq. 8 as printed
+//        over the unit's spans
+//   O11' decode keeps the last prefill call's selection        Sec. 3.5 "Persistent Mechanism"
 //
 // Parity status: O3/O10/O12 are pinned by softmax invariants and by the full-attention
 // equivalence; O6 is pinned by brute force, by hand-built block maps and by a library
@@ -31,7 +37,11 @@
 // of passages the paper leaves open, checked by brute force and hand-built cases but by
 // nothing the paper prints): the quantile convention of theta, the Q20 rounding of the
 // map, gap filling, the vote-based choice of representative tokens and its tie rule,
-// the max over query spans of summed representatives, and the decode rules.
+// the max over query spans of summed representatives, the decode rules, and (optional
+// modes) the definition of the area ratio r_a behind Eq. r_v, which the paper gives only
+// as a figure.  Pinned among the optional modes: the shape of Eq. r_v and its clamps, the
+// IoU NMS against a library NMS, the unit scores and the tokens a unit-granular step
+// attends over, the union semantics of the persistent mechanism.
 //
 // Build: g++ -O2 -std=c++17 -shared -fPIC -pthread ltri_oracle.cpp -o libltri_oracle.so
 
