@@ -104,6 +104,14 @@ struct Params {
   int32_t unit_tokens;
   // NMS IoU threshold phi in thousandths (0: spans never overlap)
   int32_t nms_iou_milli;
+  // retrieval head of this layer (Sec. 3.5): -1 = none, the layer locates evidence with all its heads; h >= 0 = the
+  // local map, the votes, the query representatives and the scores come from head h alone, and its one selection
+  // serves every KV head of the layer.  head_weight is that head's score, its voting weight.
+  int32_t ret_head;
+  float head_weight;
+  // collaborative voting (Sec. 3.5): rank the units by the summed weights of the ballots (own top-k of this and of the
+  // preceding layers that have a retrieval head) before their own scores; needs unit_tokens > 0
+  int32_t collab_vote;
 };
 
 // ---------------------------------------------------------------------------
@@ -324,6 +332,15 @@ struct Stream {
   std::vector<float> unit_score;  // [Hkv][units] (unit mode)
   std::vector<int> sel;      // [Hkv][top_k]
   std::vector<int> persist;  // [Hkv][top_k] selection of the last prefill call, kept through decode (Sec. 3.5)
+  // collaborative voting: ballots of the preceding layers for the current call (set by the caller in layer order),
+  // this layer's own ballot (its top-k by its own scores, absolute unit ids, -1 padded) and the tallies of the units
+  struct Ballot {
+    float w;
+    std::vector<int> ids;
+  };
+  std::vector<Ballot> ballots;
+  std::vector<int> own_ballot;
+  std::vector<float> tally;  // [units]
   std::vector<double> cut_gap;  // [Hkv]
   std::vector<int> qrep_tok;    // [J][reps] absolute tokens, -1 padded
 
@@ -507,6 +524,7 @@ struct Stream {
       int g = h / G;
       Mh[h].assign((size_t)m * m, 0);
       vh[h].assign((size_t)(t0 + n - vbase), 0);
+      if (p.ret_head >= 0 && h != p.ret_head) return;  // the layer's retrieval head alone draws the map and votes
       std::vector<float> pbuf;
       std::vector<std::pair<int, int>> ranges(3);
       for (int r = 0; r < n; ++r) {
@@ -536,7 +554,7 @@ struct Stream {
     reg.start = reg_start;
     reg.end = t0 + n;
     if (m > 0) {
-      thq = theta_q(Mq.data(), m, m, p.theta_mode, p.theta, Hq);
+      thq = theta_q(Mq.data(), m, m, p.theta_mode, p.theta, p.ret_head >= 0 ? 1 : Hq);
       std::vector<Span> sp;
       segment_map(Mq.data(), m, m, thq, p.max_spans_per_region, p.nms_iou_milli, sp, &seg_gap);
       for (Span& s : sp) s.start += reg_start;
@@ -565,8 +583,10 @@ struct Stream {
         for (size_t r = 0; r < reps.size(); ++r) qrep_tok[(size_t)j * rep_stride() + r] = reps[r];
         for (int g = 0; g < Hkv; ++g)
           for (int e = 0; e < d; ++e) {
+            // the heads whose queries locate the evidence for KV head g: its own group, or the layer's retrieval head
+            const int h_lo = p.ret_head >= 0 ? p.ret_head : g * G, h_hi = p.ret_head >= 0 ? p.ret_head + 1 : (g + 1) * G;
             float ug = 0.f;
-            for (int h = g * G; h < (g + 1) * G; ++h) {
+            for (int h = h_lo; h < h_hi; ++h) {
               float qr = 0.f;
               for (int tok : reps) qr += Q[((size_t)(tok - t0) * Hq + h) * d + e];
               ug += qr;
@@ -578,17 +598,21 @@ struct Stream {
     score_and_select();
   }
 
-  // O8 + O9 with the representatives in `u` ([Hkv][J][d]).
+  // O8 + O9 with the representatives in `u` ([Hkv][J][d]).  A layer with a retrieval head scores against the index
+  // of that head's KV head, so every row of its scores and of its selection is the same.
   void score_and_select() {
     int Ns = (int)spans.size();
     score.assign((size_t)Hkv * Ns, -INFINITY);
     if (p.unit_tokens > 0) unit_score.assign((size_t)Hkv * unit_count(), -INFINITY);
+    own_ballot.assign(p.top_k, -1);
+    tally.clear();
     for (int g = 0; g < Hkv; ++g) {
+      const int gk = p.ret_head >= 0 ? p.ret_head / G : g;  // KV head whose index vectors are scored
       for (int s = 0; s < Ns; ++s) {
         float best = -INFINITY;
         for (int j = 0; j < J; ++j) {
           const float* uj = &u[((size_t)g * J + j) * d];
-          const uint16_t* kr = &KR[((size_t)s * Hkv + g) * d];
+          const uint16_t* kr = &KR[((size_t)s * Hkv + gk) * d];
           float acc = 0.f;
           for (int e = 0; e < d; ++e) acc += uj[e] * bf16_to_f32(kr[e]);
           best = std::max(best, acc);
@@ -603,14 +627,53 @@ struct Stream {
         for (int s = 0; s < Ns; ++s)
           for (int u = spans[s].start / U; u <= (spans[s].start + spans[s].len - 1) / U; ++u)
             us[u - u0] = std::max(us[u - u0], score[(size_t)g * Ns + s]);
-        top_k(us, nu, p.top_k, &sel[(size_t)g * p.top_k], &cut_gap[g]);
+        int* sg = &sel[(size_t)g * p.top_k];
+        top_k(us, nu, p.top_k, sg, &cut_gap[g]);
         for (int i = 0; i < p.top_k; ++i)
-          if (sel[(size_t)g * p.top_k + i] >= 0) sel[(size_t)g * p.top_k + i] += u0;  // absolute unit ids
+          if (sg[i] >= 0) sg[i] += u0;  // absolute unit ids
       } else if (J > 0)
         top_k(&score[(size_t)g * Ns], Ns, p.top_k, &sel[(size_t)g * p.top_k], &cut_gap[g]);
       else {
         for (int i = 0; i < p.top_k; ++i) sel[(size_t)g * p.top_k + i] = -1;
         cut_gap[g] = 1.0;
+      }
+    }
+    if (p.collab_vote && J > 0 && p.unit_tokens > 0) {
+      // the layer's ballot: its top-k by its own scores (every row is the same under a retrieval head); layers
+      // without a retrieval head cast none
+      if (p.ret_head >= 0) own_ballot.assign(sel.begin(), sel.begin() + p.top_k);
+      vote_select();
+    }
+  }
+
+  // Sec. 3.5, collaborative voting.  A ballot counts with its layer's retrieval-head score.  Tally of a unit = sum of
+  // the weights of the ballots that name it, preceding layers first (ascending), then this layer's own.  The units
+  // are ranked by tally, then own score, then lower id, and the first top_k are fetched.
+  void vote_select() {
+    const int U = p.unit_tokens, u0 = p.n_sink / U, nu = unit_count();
+    tally.assign(nu, 0.f);
+    for (const Ballot& b : ballots)
+      for (int id : b.ids)
+        if (id >= u0 && id - u0 < nu) tally[id - u0] += b.w;
+    if (p.ret_head >= 0)
+      for (int id : own_ballot)
+        if (id >= u0 && id - u0 < nu) tally[id - u0] += p.head_weight;
+    for (int g = 0; g < Hkv; ++g) {
+      const float* us = &unit_score[(size_t)g * nu];
+      int* sg = &sel[(size_t)g * p.top_k];
+      std::vector<int> order(nu);
+      for (int i = 0; i < nu; ++i) order[i] = i;
+      std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+        if (tally[a] != tally[b]) return tally[a] > tally[b];
+        return us[a] > us[b];
+      });
+      const int kk = std::min(p.top_k, nu);
+      for (int i = 0; i < p.top_k; ++i) sg[i] = i < kk ? order[i] + u0 : -1;
+      cut_gap[g] = 1.0;
+      if (kk < nu && kk > 0 && tally[order[kk - 1]] == tally[order[kk]]) {
+        double a = us[order[kk - 1]], b = us[order[kk]];
+        double den = std::max(std::fabs(a), std::fabs(b));
+        cut_gap[g] = den == 0.0 ? 0.0 : std::fabs(a - b) / den;
       }
     }
   }
@@ -697,8 +760,9 @@ struct Stream {
     u.assign((size_t)Hkv * d, 0.f);
     for (int g = 0; g < Hkv; ++g)
       for (int e = 0; e < d; ++e) {
+        const int h_lo = p.ret_head >= 0 ? p.ret_head : g * G, h_hi = p.ret_head >= 0 ? p.ret_head + 1 : (g + 1) * G;
         float ug = 0.f;
-        for (int h = g * G; h < (g + 1) * G; ++h) ug += Q[(size_t)h * d + e];
+        for (int h = h_lo; h < h_hi; ++h) ug += Q[(size_t)h * d + e];
         u[(size_t)g * d + e] = ug;
       }
     score_and_select();
@@ -742,6 +806,8 @@ void* orc_create(const Params* p) {
   if (p->head_dim < 1 || p->chunk < 1 || p->window < 1 || p->n_sink < 1 || p->top_k < 1) return nullptr;
   if (p->reps_per_span < 1 || p->max_spans_per_region < 1 || p->max_tokens < 1) return nullptr;
   if (p->unit_tokens < 0 || p->nms_iou_milli < 0 || p->nms_iou_milli >= 1000) return nullptr;
+  if (p->ret_head < -1 || p->ret_head >= p->n_q_heads || !(p->head_weight >= 0.f)) return nullptr;
+  if (p->collab_vote && p->unit_tokens <= 0) return nullptr;
   if (p->rep_mode != 0 && p->rep_mode != 1) return nullptr;
   if (p->rep_mode == 1 && (p->ratio_kind < 0 || p->ratio_kind > 2 || p->min_reps < 1 || p->max_reps < p->min_reps ||
                            !(p->rep_lambda >= 0.f)))
@@ -841,6 +907,33 @@ int orc_set_newest_rep_counts(void* h, const int* counts, int cnt) {
   return 0;
 }
 int orc_num_units(void* h) { return ((Stream*)h)->unit_count(); }
+// collaborative voting: the ballots of the preceding layers for the next retrieval (ascending layer order);
+// ids [n][top_k] absolute unit ids, -1 padded
+void orc_set_ballots(void* h, int n, const float* w, const int* ids) {
+  Stream* s = (Stream*)h;
+  s->ballots.clear();
+  for (int i = 0; i < n; ++i) {
+    Stream::Ballot b;
+    b.w = w[i];
+    for (int j = 0; j < s->p.top_k; ++j)
+      if (ids[(size_t)i * s->p.top_k + j] >= 0) b.ids.push_back(ids[(size_t)i * s->p.top_k + j]);
+    s->ballots.push_back(b);
+  }
+}
+// this layer's own ballot of the last retrieval ([top_k], -1 padded; all -1 for a layer without a retrieval head)
+void orc_get_ballot(void* h, int* ids) {
+  Stream* s = (Stream*)h;
+  for (int i = 0; i < s->p.top_k; ++i) ids[i] = i < (int)s->own_ballot.size() ? s->own_ballot[i] : -1;
+}
+void orc_set_ballot(void* h, const int* ids) {  // test hook: adopt a tolerated pick and count the votes again
+  Stream* s = (Stream*)h;
+  s->own_ballot.assign(ids, ids + s->p.top_k);
+  if (s->p.collab_vote && s->J > 0 && s->p.unit_tokens > 0 && s->unit_count() > 0) s->vote_select();
+}
+void orc_get_tally(void* h, float* out) {  // [units]
+  Stream* s = (Stream*)h;
+  std::memcpy(out, s->tally.data(), s->tally.size() * sizeof(float));
+}
 void orc_get_unit_scores(void* h, float* out) {  // [Hkv][units]
   Stream* s = (Stream*)h;
   std::memcpy(out, s->unit_score.data(), s->unit_score.size() * sizeof(float));

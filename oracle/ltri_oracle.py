@@ -35,6 +35,7 @@ class _Params(C.Structure):
         ("max_tokens", C.c_int64),
         ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
         ("rep_lambda", C.c_float), ("persist_decode", C.c_int32), ("unit_tokens", C.c_int32), ("nms_iou_milli", C.c_int32),
+        ("ret_head", C.c_int32), ("head_weight", C.c_float), ("collab_vote", C.c_int32),
     ]
 
 
@@ -88,6 +89,10 @@ def lib():
         L.orc_num_units.argtypes = [vp]
         L.orc_num_units.restype = ip
         L.orc_get_unit_scores.argtypes = [vp, vp]
+        L.orc_set_ballots.argtypes = [vp, ip, vp, vp]
+        L.orc_get_ballot.argtypes = [vp, vp]
+        L.orc_set_ballot.argtypes = [vp, vp]
+        L.orc_get_tally.argtypes = [vp, vp]
         L.orc_set_newest_rep_counts.argtypes = [vp, vp, ip]
         L.orc_set_newest_rep_counts.restype = ip
         L.orc_rep_stride.argtypes = [vp]
@@ -121,7 +126,7 @@ class OracleStream:
     def __init__(self, n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, max_tokens,
                  reps_per_span=1, max_spans_per_region=None, theta_mode=1, theta=0.90, softmax_scale=0.0,
                  rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, persist_decode=0,
-                 unit_tokens=0, nms_iou_milli=0):
+                 unit_tokens=0, nms_iou_milli=0, ret_head=-1, head_weight=0.0, collab_vote=0):
         if max_spans_per_region is None:
             max_spans_per_region = max(1, chunk // 32)
         self.Hq, self.Hkv, self.d = n_q_heads, n_kv_heads, head_dim
@@ -129,8 +134,10 @@ class OracleStream:
         self.chunk, self.window, self.n_sink = chunk, window, n_sink
         self._p = _Params(n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, reps_per_span,
                           max_spans_per_region, theta_mode, theta, softmax_scale, max_tokens,
-                          rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, persist_decode, unit_tokens, nms_iou_milli)
+                          rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, persist_decode, unit_tokens, nms_iou_milli,
+                          ret_head, head_weight, collab_vote)
         self.unit_tokens = unit_tokens
+        self.ret_head, self.head_weight = ret_head, head_weight
         self._h = lib().orc_create(C.byref(self._p))
         if not self._h:
             raise ValueError("bad oracle parameters")
@@ -322,6 +329,34 @@ class OracleStream:
         a = np.zeros((self.Hkv, n), dtype=np.float32)
         if n:
             lib().orc_get_unit_scores(self._h, _ptr(a))
+        return a
+
+    # --- collaborative voting (Sec. 3.5) ----------------------------------------------
+    def set_ballots(self, ballots):
+        """Ballots of the preceding layers for the next retrieval, in ascending layer order: a list of
+        (weight, unit ids [top_k], -1 padded)."""
+        w = np.ascontiguousarray([b[0] for b in ballots], dtype=np.float32)
+        ids = np.full((max(len(ballots), 1), self.top_k), -1, dtype=np.int32)
+        for i, b in enumerate(ballots):
+            ids[i] = np.asarray(b[1], dtype=np.int32)
+        lib().orc_set_ballots(self._h, len(ballots), _ptr(w) if len(ballots) else None, _ptr(ids))
+
+    def ballot(self) -> np.ndarray:
+        """This layer's own ballot of the last retrieval: absolute unit ids [top_k], -1 padded (all -1 for a layer
+        without a retrieval head)."""
+        ids = np.zeros(self.top_k, dtype=np.int32)
+        lib().orc_get_ballot(self._h, _ptr(ids))
+        return ids
+
+    def set_ballot(self, ids):
+        a = np.ascontiguousarray(np.asarray(ids, dtype=np.int32).reshape(self.top_k))
+        lib().orc_set_ballot(self._h, _ptr(a))
+
+    def tally(self) -> np.ndarray:
+        """Summed ballot weights of every unit that meets the indexed range, [units]."""
+        a = np.zeros(lib().orc_num_units(self._h), dtype=np.float32)
+        if a.size:
+            lib().orc_get_tally(self._h, _ptr(a))
         return a
 
     def persistent(self) -> np.ndarray:
