@@ -200,7 +200,10 @@ def oracle_sample(cfg, steps, warmup):
                          theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind,
                          min_reps=cfg.min_reps, max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
                          unit_tokens=cfg.unit_tokens, persist_decode=int(cfg.persist_decode),
-                         nms_iou_milli=cfg.nms_iou_milli)
+                         nms_iou_milli=cfg.nms_iou_milli,
+                         ret_head=cfg.retrieval_head[0] if cfg.retrieval_head else -1,
+                         head_weight=cfg.retrieval_head_score[0] if cfg.retrieval_head_score else 1.0,
+                         collab_vote=int(cfg.collab_vote))
     times = []
     for ci in range(fill + warmup + steps):
         q, k, v = st.tokens(ci * cfg.chunk, cfg.chunk)
@@ -313,8 +316,10 @@ def run_ltri(args, cfg):
                             max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
                             max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
-                            flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0,
-                            unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli)
+                            flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
+                                  (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0),
+                            unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
+                            retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score)
 
     def stream_until(lt, upto, keep_from):
         for s in range(NSEQ - 1):
@@ -520,6 +525,11 @@ def main():
                     help="IoU threshold of the segmenter's NMS (0: spans never overlap; the paper lists 0.1 / 0.01)")
     ap.add_argument("--persist-decode", action="store_true",
                     help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
+    ap.add_argument("--retrieval-heads", action="store_true",
+                    help="give 14 of every 32 layers a retrieval head (a made-up table: which heads these are belongs "
+                         "to a trained model); such a layer locates evidence with that head alone")
+    ap.add_argument("--collab-vote", action="store_true",
+                    help="collaborative voting over the layers' ballots (needs --retrieval-heads and --unit-tokens)")
     ap.add_argument("--p-self", type=float, default=-1.0,
                     help="generator: probability that a prefill token targets its own segment (default 0.5; 0 = the "
                          "literal 'earlier segment' reading)")
@@ -552,6 +562,16 @@ def main():
         import dataclasses
         cfg = dataclasses.replace(cfg, persist_decode=True)
         cfg.name += "[persist-decode]"
+    if args.retrieval_heads:
+        import dataclasses
+        has = [(l * 7) % 16 < 7 for l in range(cfg.n_layers)]
+        cfg = dataclasses.replace(
+            cfg, retrieval_head=tuple((l * 5 + 3) % cfg.n_q_heads if has[l] else -1 for l in range(cfg.n_layers)),
+            retrieval_head_score=tuple(0.1 + 0.4 * ((l * 37) % 17) / 16 if has[l] else 0.0 for l in range(cfg.n_layers)),
+            collab_vote=args.collab_vote)
+        cfg.name += "[retrieval-heads" + (",vote]" if args.collab_vote else "]")
+    elif args.collab_vote:
+        ap.error("--collab-vote needs --retrieval-heads and --unit-tokens")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -79,6 +79,16 @@ typedef struct {
                                                         Filtration", boxes = squares on the diagonal).  0: kept spans
                                                         never overlap and the spans partition the region; > 0: kept
                                                         spans may overlap, the gaps are the runs none of them covers */
+  /* Retrieval heads (Sec. 3.5).  HOST arrays of n_layers entries, read at ltri_create and not kept; NULL: no layer
+   * has one.  retrieval_head[l] = -1: layer l locates evidence with all its heads (the default path).
+   * retrieval_head[l] = h in [0, n_q_heads): layer l uses head h alone -- the local map of Eq. 1-4, the threshold
+   * (mode 0: theta in that head's probability units), the votes of Eq. 6, the query representatives and the scores
+   * of Eq. 7 (against the index of h's KV head) come from h, and the one selection serves every KV head of the layer.
+   * retrieval_head_score[l] >= 0 is the head's score, its weight under LTRI_FLAG_COLLAB_VOTE (ignored where
+   * retrieval_head[l] < 0; NULL: every weight 1).  Which heads these are is a property of the model; the caller
+   * supplies them. */
+  const int32_t* retrieval_head;
+  const float* retrieval_head_score;
   void* arena;                                       /* caller-owned device memory, 256-byte aligned */
   size_t arena_bytes;                                /* >= ltri_arena_bytes(params) */
 } ltri_params;
@@ -89,7 +99,14 @@ enum {
    * of every decode step, next to the spans the step retrieves itself. */
   LTRI_FLAG_PERSIST_DECODE = 1,
   /* Reserve two staging sets in the arena (q, k, v and out of one full call each) for ltri_prefill_chunk_host. */
-  LTRI_FLAG_HOST_STAGING = 2
+  LTRI_FLAG_HOST_STAGING = 2,
+  /* Collaborative voting (Sec. 3.5); needs unit_tokens > 0 (unit numbers mean the same tokens in every layer) and
+   * retrieval_head.  Every layer with a retrieval head casts a ballot: its k best units by its own scores, weighted
+   * by retrieval_head_score.  Layer K ranks its units by tally -- the summed weights of the ballots of layers 0..K
+   * (fp32, ascending layer order) that name the unit -- then by its own score, then by lower unit number, and fetches
+   * the first k.  The layers of a chunk (or decode step) must be submitted in ascending order, each layer of a
+   * sequence exactly once, so that the ballots a layer reads are those of the same chunk. */
+  LTRI_FLAG_COLLAB_VOTE = 4
 };
 
 typedef struct {
@@ -210,6 +227,8 @@ enum {
   LTRI_BUF_QREPS = 6,    /* float [n_kv_heads][2*max_spans_per_region+1][head_dim]: summed query representatives */
   LTRI_BUF_NREPS = 8,    /* int32 [2*max_spans_per_region+1]: representative counts of the spans of the last prefill
                             call's region (Sec. 3.3.2) */
+  LTRI_BUF_BALLOT = 9,   /* int32 [top_k]: the layer's own ballot under LTRI_FLAG_COLLAB_VOTE (ascending unit numbers,
+                            -1 padded; all -1 for a layer without a retrieval head) */
   LTRI_BUF_ROWSTAT = 7   /* float [chunk][n_q_heads][2]: reference maximum m (logits * scale * log2(e); may lag the true
                             row maximum by up to 8) and the matching row sum of exp2(logit - m) of the local softmax
                             of the last prefill call */

@@ -17,7 +17,9 @@ LIB_PATH = os.path.join(_HERE, "libltri.so")
 LTRI_OK, LTRI_EINVAL, LTRI_ECAPACITY, LTRI_ESTATE, LTRI_ECUDA, LTRI_EDEVICE, LTRI_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 FLAG_PERSIST_DECODE = 1
 FLAG_HOST_STAGING = 2
+FLAG_COLLAB_VOTE = 4
 BUF_MAP, BUF_VOTES, BUF_INDEX, BUF_THETA, BUF_SCORES, BUF_QREPS, BUF_ROWSTAT, BUF_NREPS = 1, 2, 3, 4, 5, 6, 7, 8
+BUF_BALLOT = 9
 
 EXPORTS = [
     "ltri_arena_bytes", "ltri_create", "ltri_destroy", "ltri_reset_sequence", "ltri_prefill_chunk",
@@ -39,6 +41,7 @@ class LtriParams(C.Structure):
         ("theta_mode", C.c_int32), ("theta", C.c_float), ("softmax_scale", C.c_float), ("flags", C.c_uint32),
         ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
         ("rep_lambda", C.c_float), ("unit_tokens", C.c_int32), ("nms_iou_milli", C.c_int32),
+        ("retrieval_head", C.POINTER(C.c_int32)), ("retrieval_head_score", C.POINTER(C.c_float)),
         ("arena", C.c_void_p), ("arena_bytes", C.c_size_t),
     ]
 
@@ -103,10 +106,24 @@ def strerror(code: int) -> str:
 
 def make_params(n_layers, n_q_heads, n_kv_heads, max_tokens, chunk, window, n_sink, top_k, head_dim=128, max_seqs=1,
                 reps_per_span=1, max_spans_per_region=0, theta_mode=1, theta=0.90, softmax_scale=0.0,
-                rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, flags=0, unit_tokens=0, nms_iou_milli=0) -> LtriParams:
-    return LtriParams(n_layers, n_q_heads, n_kv_heads, head_dim, max_seqs, max_tokens, chunk, window, n_sink, top_k,
-                      reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, flags,
-                      rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, unit_tokens, nms_iou_milli, None, 0)
+                rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, flags=0, unit_tokens=0, nms_iou_milli=0,
+                retrieval_head=None, retrieval_head_score=None) -> LtriParams:
+    """retrieval_head / retrieval_head_score: per-layer sequences (head or -1; weight), marshalled into host arrays
+    that live as long as the returned struct."""
+    p = LtriParams(n_layers, n_q_heads, n_kv_heads, head_dim, max_seqs, max_tokens, chunk, window, n_sink, top_k,
+                   reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, flags,
+                   rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, unit_tokens, nms_iou_milli, None, None, None, 0)
+    if retrieval_head is not None:
+        if len(retrieval_head) != n_layers:
+            raise ValueError("retrieval_head needs one entry per layer")
+        p._rh = (C.c_int32 * n_layers)(*[int(h) for h in retrieval_head])
+        p.retrieval_head = C.cast(p._rh, C.POINTER(C.c_int32))
+        if retrieval_head_score is not None:
+            if len(retrieval_head_score) != n_layers:
+                raise ValueError("retrieval_head_score needs one entry per layer")
+            p._rw = (C.c_float * n_layers)(*[float(w) for w in retrieval_head_score])
+            p.retrieval_head_score = C.cast(p._rw, C.POINTER(C.c_float))
+    return p
 
 
 def ltri_arena_bytes(params: LtriParams) -> int:
@@ -155,6 +172,7 @@ class Ltri:
         self.arena = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
         base = (self.arena.data_ptr() + 255) // 256 * 256
         self.params = LtriParams.from_buffer_copy(params)
+        self._params_src = params   # owns the host arrays the copy points to
         self.params.arena = base
         self.params.arena_bytes = nbytes
         self.arena_bytes = nbytes
@@ -294,7 +312,7 @@ class Ltri:
             return raw.view(np.float32).reshape(p.n_kv_heads, cap)
         if what == BUF_QREPS:
             return raw.view(np.float32).reshape(p.n_kv_heads, 2 * C_ + 1, p.head_dim)
-        if what == BUF_NREPS:
+        if what in (BUF_NREPS, BUF_BALLOT):
             return raw.view(np.int32)
         if what == BUF_ROWSTAT:
             return raw.view(np.float32).reshape(p.chunk, p.n_q_heads, 2)

@@ -47,6 +47,11 @@ struct DevCtx {
   int* pend_nrep;        // [NS][NL][slots][Jmax]  representative count of every pending span
   int* sel;              // [NS][NL][Hkv][topk]  ascending ids, -1 padded
   int* persist_sel;      // [NS][NL][Hkv][topk]  selection of the last prefill call, kept through decode
+  // retrieval heads and collaborative voting (Sec. 3.5)
+  int vote;              // rank units by the tally of the layers' ballots before their own scores
+  const int* ret_head;   // [NL]  retrieval head of the layer, -1 none; nullptr: no layer has one
+  const float* head_w;   // [NL]  its score = the weight of the layer's ballot
+  int* ballot;           // [NS][NL][topk]  own top-k units of a layer with a retrieval head (ascending, -1 padded)
   long long* sel_tokens; // [NS][NL]  retrieved tokens of the last call, summed over KV heads
   // per-layer scratch of the prefill call in flight
   int* Mq;               // [NL][chunk][chunk]
@@ -74,6 +79,11 @@ struct DevCtx {
 };
 
 __host__ __device__ inline size_t unit_of(const DevCtx& c, int seq, int layer) { return (size_t)seq * c.NL + layer; }
+
+#ifdef __CUDACC__
+// Retrieval head of a layer (Sec. 3.5): -1 when the layer locates evidence with all its heads.
+__device__ __forceinline__ int ret_head_of(const DevCtx& c, int layer) { return c.ret_head ? c.ret_head[layer] : -1; }
+#endif
 
 // Decode batch descriptor (passed by value; at most 64 sequences per launch).
 constexpr int kDecBatch = 64;

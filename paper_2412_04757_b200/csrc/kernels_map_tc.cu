@@ -61,6 +61,10 @@ __global__ void __launch_bounds__(kMapThreads, 1)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
   const size_t unit = unit_of(c, a.seq, layer);
+  // a layer with a retrieval head (Sec. 3.5) draws its map and votes from that head alone: the other KV heads have
+  // nothing to add, and in the head's own group the other heads' columns are switched off through their offsets
+  const int rh = ret_head_of(c, layer);
+  if (rh >= 0 && g != rh / G) return;
   const bool is_cur = (int)blockIdx.x >= n_local_groups;
   const int tile0 = (is_cur ? (int)blockIdx.x - n_local_groups : (int)blockIdx.x) * kMapKT;
   const int ntile = min(kMapKT, (is_cur ? n_cur_tiles : n_local_tiles) - tile0);
@@ -164,7 +168,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     auto load_stats = [&](int blk) -> float {
       const int col = cq * 32 + lane;
       const int tk = blk * TPB + col / G;
-      return tk < a.n ? __ldg(rq + (size_t)tk * c.Hq + col % G) : -INFINITY;
+      return tk < a.n && (rh < 0 || g * G + col % G == rh) ? __ldg(rq + (size_t)tk * c.Hq + col % G) : -INFINITY;
     };
     float* my_stats = &s_stats[warp][0][0];
     if (bmin < nblocks) my_stats[lane] = load_stats(bmin);

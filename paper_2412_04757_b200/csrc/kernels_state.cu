@@ -24,6 +24,7 @@ __global__ void k_init(DevCtx c, int seq) {
       c.persist_sel[u0 * c.Hkv * c.topk + i] = -1;
     }
     for (size_t i = tid; i < (size_t)c.NL * c.Hkv; i += stride) c.rng_cnt[u0 * c.Hkv + i] = 0;
+    for (size_t i = tid; i < (size_t)c.NL * c.topk; i += stride) c.ballot[u0 * c.topk + i] = -1;
   }
   if (seq < 0 && tid < 4) c.status[tid] = 0;
   if (seq < 0)
@@ -393,7 +394,11 @@ __global__ void __cluster_dims__(kThetaCluster, 1, 1) __launch_bounds__(kThetaTh
     c.thetaq[layer] = cls > 0 ? (long long)s_prefix : (long long)(int)(s_prefix ^ 0x80000000u);
 }
 
-__global__ void k_theta_set(DevCtx c, int layer_begin, long long thq) { c.thetaq[layer_begin + blockIdx.x] = thq; }
+// absolute threshold: thq in units of the map summed over all heads, thq1 in units of a single (retrieval) head's map
+__global__ void k_theta_set(DevCtx c, int layer_begin, long long thq, long long thq1) {
+  const int layer = layer_begin + blockIdx.x;
+  c.thetaq[layer] = ret_head_of(c, layer) >= 0 ? thq1 : thq;
+}
 
 // step 2: suffix sums along each row of D = Mq - theta ("sum the right elements", Fig. 2):
 // Rsuf[i][x] = sum_{j=x..i} D[i][j].  One warp per row, 32-wide shuffle scans from the diagonal leftwards.
@@ -678,12 +683,15 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
       acc[3] += __bfloat162float(p1.y);
     };
     const __nv_bfloat16* qg = q + (size_t)g * c.G * kD + lane * 4;
+    // a layer with a retrieval head (Sec. 3.5) has one representative per span, that head's: the other heads add zero
+    const int rh = ret_head_of(c, layer);
+    auto counts = [&](int hh) { return hh < c.G && (rh < 0 || g * c.G + hh == rh); };
     for (int r = 0; r < nrep; ++r) {
       const __nv_bfloat16* row = qg + (size_t)(rep_tok[j * kMaxReps + r] - a.t0) * c.Hq * kD;
       uint2 raw[8];
 #pragma unroll
       for (int hh = 0; hh < 8; ++hh)
-        raw[hh] = hh < c.G ? *reinterpret_cast<const uint2*>(row + (size_t)hh * kD) : make_uint2(0u, 0u);
+        raw[hh] = counts(hh) ? *reinterpret_cast<const uint2*>(row + (size_t)hh * kD) : make_uint2(0u, 0u);
 #pragma unroll
       for (int hh = 0; hh < 8; ++hh) add_row(qr[hh], raw[hh]);
     }
@@ -695,6 +703,7 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
         for (int e = 0; e < 4; ++e) ug[e] += qr[hh][e];
       }
     for (int hh = 8; hh < c.G; ++hh) {  // groups wider than eight heads
+      if (!counts(hh)) continue;
       float w[4] = {0.f, 0.f, 0.f, 0.f};
       for (int r = 0; r < nrep; ++r)
         add_row(w, *reinterpret_cast<const uint2*>(qg + ((size_t)(rep_tok[j * kMaxReps + r] - a.t0) * c.Hq + hh) * kD));
@@ -717,7 +726,8 @@ cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_
     const int hsmem = (kThetaThreads / 32) * kThetaBins * (int)sizeof(unsigned);
     k_theta_select<<<layer_count * kThetaCluster, kThetaThreads, hsmem, s>>>(c, layer_begin, m, rank);
   } else {
-    k_theta_set<<<layer_count, 1, 0, s>>>(c, layer_begin, theta_q_abs);
+    k_theta_set<<<layer_count, 1, 0, s>>>(c, layer_begin, theta_q_abs,
+                                          (long long)nearbyint((double)theta * (double)kQScale));
   }
   k_seg_rowscan<<<dim3((m + 7) / 8, layer_count), 256, 0, s>>>(c, layer_begin, m);
   const size_t smem = (size_t)(32 * 32 + m + 32) * sizeof(long long);
@@ -804,13 +814,16 @@ __global__ void __launch_bounds__(256) k_score_dec(DevCtx c, int layer_begin, De
   const size_t unit = unit_of(c, b.seq[bi], layer);
   const int tid = threadIdx.x;
   const int N = c.n_spans[unit];
+  // a layer with a retrieval head (Sec. 3.5) scores that head's query against the index of its KV head, for every g
+  const int rh = ret_head_of(c, layer), gk = rh >= 0 ? rh / c.G : g;
   if (blockIdx.x == 0 && g == 0 && tid == 0) c.sel_tokens[unit] = 0;
   const int s0 = blockIdx.x * 256;
   if (s0 >= N) return;
   if (tid < kD) {
-    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + g * c.G) * kD + tid;
+    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + gk * c.G) * kD + tid;
     float acc = 0.f;
-    for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
+    for (int hh = 0; hh < c.G; ++hh)
+      if (rh < 0 || gk * c.G + hh == rh) acc += __bfloat162float(qp[(size_t)hh * kD]);
     su[tid] = acc;
   }
   __syncthreads();
@@ -818,7 +831,7 @@ __global__ void __launch_bounds__(256) k_score_dec(DevCtx c, int layer_begin, De
   float uf[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
-  const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + g) * (size_t)c.cap * kD + hl * 8;
+  const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + gk) * (size_t)c.cap * kD + hl * 8;
   float* sc = c.scores + (unit * c.Hkv + g) * (size_t)c.cap;
 #pragma unroll
   for (int rep = 0; rep < 4; ++rep) {
@@ -893,11 +906,84 @@ __device__ __forceinline__ unsigned order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Radix select of the K largest keys among KEY(0..N) (ties: lower index first), one 8-bit digit per pass from the top.
+// Writes the chosen indices, unordered, to s_ids and their number to *s_cnt (which the caller has zeroed).  Called by
+// every thread of the CTA; K < N.
+template <typename KT, typename KeyF>
+__device__ __forceinline__ void radix_select_top(KeyF&& KEY, int N, int K, unsigned* hist, KT* s_prefix,
+                                                 unsigned* s_need, int* s_scan, int* s_cnt, int* s_ids) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  constexpr int kPasses = (int)sizeof(KT);
+  if (tid == 0) {
+    *s_prefix = 0;
+    *s_need = K;  // rank from the top, 1-based: find key T with #(key > T) < K <= #(key >= T)
+  }
+  for (int pass = 0; pass < kPasses; ++pass) {
+    const int shift = 8 * (kPasses - 1 - pass);
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    const KT prefix = *s_prefix;
+    const KT himask = pass == 0 ? (KT)0 : (KT)(~(KT)0 << (shift + 8));
+    for (int s = tid; s < N; s += nt) {
+      const KT key = KEY(s);
+      if ((key & himask) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 32) {
+      unsigned need = *s_need;
+      const int bin = pick_from_top(hist, 256, need);
+      if (tid == 0) {
+        *s_need = need;
+        *s_prefix = prefix | ((KT)bin << shift);
+      }
+    }
+    __syncthreads();
+  }
+  const KT T = *s_prefix;
+  const unsigned need_eq = *s_need;  // how many of the == T elements are taken (lowest ids first)
+  // contiguous id partition so that ties are picked in id order
+  const int per = (N + nt - 1) / nt;
+  const int lo = tid * per, hi = min(N, lo + per);
+  int eq = 0;
+  for (int s = lo; s < hi; ++s) eq += KEY(s) == T;
+  s_scan[tid] = eq;
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int t = 0; t < nt; ++t) {
+      const int v = s_scan[t];
+      s_scan[t] = run;
+      run += v;
+    }
+  }
+  __syncthreads();
+  int eqrank = s_scan[tid];
+  for (int s = lo; s < hi; ++s) {
+    const KT key = KEY(s);
+    bool take = key > T;
+    if (key == T) {
+      take = (unsigned)eqrank < need_eq;
+      ++eqrank;
+    }
+    if (take) {
+      const int slot = atomicAdd(s_cnt, 1);
+      if (slot < kMaxTopK) s_ids[slot] = s;
+    }
+  }
+}
+
+// What a launch of k_topk does.  kTopkSelect: the selection, the token ranges and (prefill) the gather.  The other
+// two are the collaborative voting of Sec. 3.5: kTopkBallot only records the own top-k units of every layer that has a
+// retrieval head; kTopkVote then ranks a layer's units by the tally of the ballots of the layers up to it before
+// their own scores and goes on like kTopkSelect.
+enum { kTopkSelect = 0, kTopkBallot = 1, kTopkVote = 2 };
+
 template <bool DECODE>
 __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin, DecBatch b, int layer_count,
-                                              int evicted_end) {
+                                              int evicted_end, int mode) {
   __shared__ unsigned hist[256];
   __shared__ unsigned s_prefix, s_need;
+  __shared__ unsigned long long s_prefix64;
   __shared__ int s_ids[kMaxTopK];
   __shared__ int s_cnt;
   __shared__ int s_scan[512];
@@ -916,9 +1002,12 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     layer = layer_begin + blockIdx.y;
     sq = seq;
   }
+  // a layer with a retrieval head (Sec. 3.5) has one selection, made from the scores of that head's KV head
+  const int rh = ret_head_of(c, layer);
+  if (mode == kTopkBallot && (rh < 0 || g != 0)) return;
   const size_t unit = unit_of(c, sq, layer);
   const int nspans = c.n_spans[unit];
-  const float* sc = c.scores + (unit * c.Hkv + g) * (size_t)c.cap;
+  const float* sc = c.scores + (unit * c.Hkv + (rh >= 0 ? rh / c.G : g)) * (size_t)c.cap;
   const int tid = threadIdx.x, nt = blockDim.x;
   // What is ranked: the spans themselves, or (Eq. 8 as printed) fixed units of c.unit tokens on the absolute token
   // grid, each scored by the maximum over the spans it meets.  N = number of candidates, KEY(i) = order key of
@@ -939,70 +1028,35 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     }
     __syncthreads();
   }
+  // voting: tally of every unit = summed weights of the ballots that name it, layers in ascending order (fp32)
+  float* utally = reinterpret_cast<float*>(ukey + ((N + 3) & ~3));
+  if (mode == kTopkVote) {
+    for (int i = tid; i < N; i += nt) utally[i] = 0.f;
+    __syncthreads();
+    for (int l = 0; l <= layer; ++l) {
+      if (ret_head_of(c, l) < 0) continue;
+      const float w = c.head_w[l];
+      if (tid < c.topk) {
+        const int id = c.ballot[unit_of(c, sq, l) * c.topk + tid];  // distinct within a ballot
+        if (id >= u0 && id - u0 < N) utally[id - u0] += w;
+      }
+      __syncthreads();
+    }
+  }
   auto KEY = [&](int i) -> unsigned { return U > 0 ? ukey[i] : order_key(sc[i]); };
+  auto KEY64 = [&](int i) -> unsigned long long {
+    return ((unsigned long long)order_key(utally[i]) << 32) | ukey[i];
+  };
   const int K = min(c.topk, N);
   if (tid == 0) s_cnt = 0;
   __syncthreads();
   if (K == N) {
     for (int t = tid; t < K; t += nt) s_ids[t] = t;
     if (tid == 0) s_cnt = K;
+  } else if (mode == kTopkVote) {
+    radix_select_top<unsigned long long>(KEY64, N, K, hist, &s_prefix64, &s_need, s_scan, &s_cnt, s_ids);
   } else {
-    if (tid == 0) {
-      s_prefix = 0;
-      s_need = K;  // rank from the top, 1-based: find key T with #(key > T) < K <= #(key >= T)
-    }
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      if (tid < 256) hist[tid] = 0;
-      __syncthreads();
-      const unsigned prefix = s_prefix;
-      const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-      for (int s = tid; s < N; s += nt) {
-        const unsigned key = KEY(s);
-        if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-      }
-      __syncthreads();
-      if (tid < 32) {
-        unsigned need = s_need;
-        const int bin = pick_from_top(hist, 256, need);
-        if (tid == 0) {
-          s_need = need;
-          s_prefix = prefix | ((unsigned)bin << shift);
-        }
-      }
-      __syncthreads();
-    }
-    const unsigned T = s_prefix;
-    const unsigned need_eq = s_need;  // how many of the == T elements are taken (lowest ids first)
-    // contiguous id partition so that ties are picked in id order
-    const int per = (N + nt - 1) / nt;
-    const int lo = tid * per, hi = min(N, lo + per);
-    int eq = 0;
-    for (int s = lo; s < hi; ++s) eq += KEY(s) == T;
-    s_scan[tid] = eq;
-    __syncthreads();
-    if (tid == 0) {
-      int run = 0;
-      for (int t = 0; t < nt; ++t) {
-        const int v = s_scan[t];
-        s_scan[t] = run;
-        run += v;
-      }
-    }
-    __syncthreads();
-    int eqrank = s_scan[tid];
-    for (int s = lo; s < hi; ++s) {
-      const unsigned key = KEY(s);
-      bool take = key > T;
-      if (key == T) {
-        take = (unsigned)eqrank < need_eq;
-        ++eqrank;
-      }
-      if (take) {
-        const int slot = atomicAdd(&s_cnt, 1);
-        if (slot < kMaxTopK) s_ids[slot] = s;
-      }
-    }
+    radix_select_top<unsigned>(KEY, N, K, hist, &s_prefix, &s_need, s_scan, &s_cnt, s_ids);
   }
   __syncthreads();
   const int cnt = min(s_cnt, K);
@@ -1017,6 +1071,10 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   __syncthreads();
   if (U > 0 && tid < cnt) s_ids[tid] += u0;  // absolute unit ids
   __syncthreads();
+  if (mode == kTopkBallot) {
+    for (int t = tid; t < c.topk; t += nt) c.ballot[unit * c.topk + t] = t < cnt ? s_ids[t] : -1;
+    return;
+  }
   int* sel = c.sel + (unit * c.Hkv + g) * (size_t)c.topk;
   for (int t = tid; t < c.topk; t += nt) sel[t] = t < cnt ? s_ids[t] : -1;
   // token ranges of the attention kernels: the spans' extents are fetched in parallel, merged (adjacent spans become
@@ -1139,10 +1197,12 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   const size_t unit = unit_of(c, sq, layer);
   const int tid = threadIdx.x, nt = blockDim.x;
   const int N = min(c.n_spans[unit], kFusedMaxSpans);
+  const int rh = ret_head_of(c, layer), gk = rh >= 0 ? rh / c.G : g;  // retrieval head of the layer (Sec. 3.5)
   if (tid < kD) {
-    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + g * c.G) * kD + tid;
+    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + gk * c.G) * kD + tid;
     float acc = 0.f;
-    for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
+    for (int hh = 0; hh < c.G; ++hh)
+      if (rh < 0 || gk * c.G + hh == rh) acc += __bfloat162float(qp[(size_t)hh * kD]);
     su[tid] = acc;
   }
   if (tid == 0) s_cnt = 0;
@@ -1153,7 +1213,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     float uf[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
-    const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + g) * (size_t)c.cap * kD + hl * 8;
+    const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + gk) * (size_t)c.cap * kD + hl * 8;
     // software pipeline: the next four rows are in flight while the current four are reduced
     auto fetch = [&](int base, uint4 (&raw)[4]) {
 #pragma unroll
@@ -1345,10 +1405,12 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
   const int N = min(c.n_spans[unit], kRetCluster * kRetSliceMax);
   const int per = (N + kRetCluster - 1) / kRetCluster;
   const int lo = min(N, rank * per), hi = min(N, lo + per), nloc = hi - lo;  // this CTA's spans [lo, hi)
+  const int rh = ret_head_of(c, layer), gk = rh >= 0 ? rh / c.G : g;  // retrieval head of the layer (Sec. 3.5)
   if (tid < kD) {
-    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + g * c.G) * kD + tid;
+    const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + gk * c.G) * kD + tid;
     float acc = 0.f;
-    for (int hh = 0; hh < c.G; ++hh) acc += __bfloat162float(qp[(size_t)hh * kD]);
+    for (int hh = 0; hh < c.G; ++hh)
+      if (rh < 0 || gk * c.G + hh == rh) acc += __bfloat162float(qp[(size_t)hh * kD]);
     su[tid] = acc;
   }
   __syncthreads();
@@ -1359,7 +1421,7 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
     float uf[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
-    const __nv_bfloat16* KR = c.KR + ((unit * c.Hkv + g) * (size_t)c.cap + lo) * kD + hl * 8;
+    const __nv_bfloat16* KR = c.KR + ((unit * c.Hkv + gk) * (size_t)c.cap + lo) * kD + hl * 8;
     auto fetch = [&](int base, uint4 (&raw)[4]) {
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
@@ -1545,22 +1607,40 @@ cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int la
 }
 int dec_retrieve_fused_max_spans() { return kRetCluster * kRetSliceMax; }
 
-// dynamic shared memory of k_topk: one order key per unit in unit mode (at most 12K units: 48 KB), nothing otherwise
+// dynamic shared memory of k_topk: one order key per unit in unit mode (at most 12K units: 48 KB), nothing otherwise;
+// under collaborative voting a tally per unit behind the keys
 static int topk_unit_smem(const DevCtx& c) {
-  return c.unit > 0 ? (int)sizeof(unsigned) * (int)(c.Tmax / c.unit + 2) : 0;
+  if (c.unit <= 0) return 0;
+  const int n = (int)(c.Tmax / c.unit + 2);
+  return (int)sizeof(unsigned) * (c.vote ? 2 * n + 4 : n);
+}
+
+// Top-k of the call.  Under collaborative voting (Sec. 3.5) two launches: the ballots of the layers with a retrieval
+// head, then the vote (a layer reads the ballots of the layers up to its own, also those of earlier calls for the same
+// chunk or step).
+template <bool DECODE>
+static cudaError_t launch_topk(const DevCtx& c, int seq, int layer_begin, const DecBatch& b, int layer_count, int gy,
+                               int evicted_end, cudaStream_t s) {
+  const int smem = topk_unit_smem(c);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k_topk<DECODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+  }
+  if (c.vote)
+    k_topk<DECODE><<<dim3(c.Hkv, gy), 512, smem, s>>>(c, seq, layer_begin, b, layer_count, evicted_end, kTopkBallot);
+  k_topk<DECODE><<<dim3(c.Hkv, gy), 512, smem, s>>>(c, seq, layer_begin, b, layer_count, evicted_end,
+                                                   c.vote ? kTopkVote : kTopkSelect);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
   DecBatch dummy;
   dummy.n = 0;
-  k_topk<false><<<dim3(c.Hkv, a.layer_count), 512, topk_unit_smem(c), s>>>(c, a.seq, a.layer_begin, dummy,
-                                                                           a.layer_count, a.loc_begin);
-  return cudaGetLastError();
+  return launch_topk<false>(c, a.seq, a.layer_begin, dummy, a.layer_count, a.layer_count, a.loc_begin, s);
 }
 
 cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s) {
-  k_topk<true><<<dim3(c.Hkv, b.n * layer_count), 512, topk_unit_smem(c), s>>>(c, 0, layer_begin, b, layer_count, 0);
-  return cudaGetLastError();
+  return launch_topk<true>(c, 0, layer_begin, b, layer_count, b.n * layer_count, 0, s);
 }
 
 }  // namespace ltri

@@ -57,7 +57,14 @@ bool validate(const ltri_params* p) {
   if (p->theta_mode != 0 && p->theta_mode != 1) return false;
   if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
   if (!(p->softmax_scale >= 0.f)) return false;
-  if (p->flags & ~(uint32_t)(LTRI_FLAG_PERSIST_DECODE | LTRI_FLAG_HOST_STAGING)) return false;
+  if (p->flags & ~(uint32_t)(LTRI_FLAG_PERSIST_DECODE | LTRI_FLAG_HOST_STAGING | LTRI_FLAG_COLLAB_VOTE)) return false;
+  if ((p->flags & LTRI_FLAG_COLLAB_VOTE) && (p->unit_tokens == 0 || !p->retrieval_head)) return false;
+  if (p->retrieval_head)
+    for (int l = 0; l < p->n_layers; ++l) {
+      if (p->retrieval_head[l] < -1 || p->retrieval_head[l] >= p->n_q_heads) return false;
+      if (p->retrieval_head_score && !(p->retrieval_head_score[l] >= 0.f && p->retrieval_head_score[l] < 1e30f))
+        return false;
+    }
   if (p->nms_iou_milli < 0 || p->nms_iou_milli > 999) return false;
   if (p->unit_tokens != 0) {
     if (p->unit_tokens < 8 || p->unit_tokens > p->chunk || p->unit_tokens % 8) return false;
@@ -93,6 +100,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.topk = p.top_k;
   d.rcap = 2 * p.top_k + 2;
   d.persist = (p.flags & LTRI_FLAG_PERSIST_DECODE) ? 1 : 0;
+  d.vote = (p.flags & LTRI_FLAG_COLLAB_VOTE) ? 1 : 0;
   d.reps = p.reps_per_span > 0 ? p.reps_per_span : 1;
   d.C = p.max_spans_per_region > 0 ? p.max_spans_per_region : std::max(1, p.chunk / 32);
   d.Jmax = 2 * d.C + 1;
@@ -124,6 +132,14 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.sel = cv.take<int>(units * d.Hkv * d.topk);
   d.persist_sel = cv.take<int>(units * d.Hkv * d.topk);
   d.sel_tokens = cv.take<long long>(units);
+  {
+    // (carved whether or not a layer has a retrieval head, so that the arena size does not depend on host arrays)
+    int* rh = cv.take<int>(d.NL);
+    float* hw = cv.take<float>(d.NL);
+    d.ret_head = p.retrieval_head ? rh : nullptr;
+    d.head_w = p.retrieval_head ? hw : nullptr;
+    d.ballot = cv.take<int>(units * d.topk);
+  }
   d.Mq = cv.take<int>((size_t)d.NL * d.chunk * d.chunk);
   d.Rsuf = cv.take<long long>((size_t)d.NL * d.chunk * d.chunk);
   d.best = cv.take<long long>((size_t)d.NL * 2 * d.chunk);
@@ -162,6 +178,8 @@ struct ltri_ctx {
   ltri_params p;
   DevCtx d;
   std::vector<LayerState> st;  // [max_seqs][n_layers]
+  std::vector<int> ret_head;   // [n_layers] copy of the caller's retrieval heads (empty: none)
+  std::vector<float> head_w;
   int last_cuda = 0;
   int sm_count = 148;
   bool use_tc = false;     // tcgen05/TMEM/TMA attention kernels (default when available)
@@ -256,6 +274,13 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
   if (!ctx) return LTRI_ECAPACITY;
   ctx->p = *p;
   layout(*p, ctx->d, static_cast<char*>(p->arena), ctx->stage);
+  if (p->retrieval_head) {  // the caller's arrays are read now and not kept
+    ctx->ret_head.assign(p->retrieval_head, p->retrieval_head + p->n_layers);
+    ctx->head_w.assign((size_t)p->n_layers, 1.0f);
+    if (p->retrieval_head_score) ctx->head_w.assign(p->retrieval_head_score, p->retrieval_head_score + p->n_layers);
+  }
+  ctx->p.retrieval_head = nullptr;
+  ctx->p.retrieval_head_score = nullptr;
   if (p->flags & LTRI_FLAG_HOST_STAGING) {
     bool ok = cudaStreamCreateWithFlags(&ctx->s_up, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&ctx->s_down, cudaStreamNonBlocking) == cudaSuccess;
@@ -285,7 +310,18 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
                 tc_encode_kv_maps(ctx->d, ctx->kv_maps);
   // unfilled tile slots and over-fetched rows must hold finite values: start from an all-zero cache
   const size_t kv_bytes = (size_t)p->max_seqs * p->n_layers * ctx->d.Hkv * (size_t)ctx->d.Tpad * kD * 2 * sizeof(__nv_bfloat16);
+  if (!ctx->ret_head.empty() && !ctx->use_tc) {  // retrieval heads are built into the tensor-core map pass only
+    ltri_destroy(ctx);
+    return LTRI_EINVAL;
+  }
   cudaError_t e = cudaMemsetAsync(ctx->d.Kc, 0, kv_bytes, s);
+  if (e == cudaSuccess && !ctx->ret_head.empty()) {
+    e = cudaMemcpyAsync(const_cast<int*>(ctx->d.ret_head), ctx->ret_head.data(), ctx->ret_head.size() * sizeof(int),
+                        cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(const_cast<float*>(ctx->d.head_w), ctx->head_w.data(), ctx->head_w.size() * sizeof(float),
+                          cudaMemcpyHostToDevice, s);
+  }
   if (e == cudaSuccess) e = launch_init(ctx->d, -1, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) {
@@ -426,7 +462,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   }
   if (has_index) {
     {
-      Scope sc(ctx, st, LTRI_K_SCORE_TOPK, 2);
+      Scope sc(ctx, st, LTRI_K_SCORE_TOPK, d.vote ? 3 : 2);
       if (ctx->use_tc && score_tc_supported(d))
         LTRI_CUDA(ctx, launch_score_prefill_tc(d, a, (int)ub, ctx->kv_maps, st));
       else if (ctx->use_tc)
@@ -596,7 +632,7 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
       Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 1);
       LTRI_CUDA(ctx, launch_dec_retrieve_fused(d, b, layer_begin, layer_count, qb, (int)ub, ctx->dec_fused == 2, st));
     } else {
-      Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 2);
+      Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, d.vote ? 3 : 2);
       LTRI_CUDA(ctx, launch_score_decode(d, b, layer_begin, layer_count, n_seqs, qb, (int)ub, st));
       LTRI_CUDA(ctx, launch_topk_decode(d, b, layer_begin, layer_count, st));
     }
@@ -796,6 +832,10 @@ int ltri_debug_read(ltri_ctx* ctx, int what, int seq, int layer, void* dst, size
     case LTRI_BUF_NREPS:
       src = d.nrep_last + (size_t)layer * d.Jmax;
       bytes = (size_t)d.Jmax * sizeof(int);
+      break;
+    case LTRI_BUF_BALLOT:
+      src = d.ballot + unit_of(d, seq, layer) * d.topk;
+      bytes = (size_t)d.topk * sizeof(int);
       break;
     case LTRI_BUF_ROWSTAT:
       src = d.rowstat + (size_t)layer * d.chunk * d.Hq;

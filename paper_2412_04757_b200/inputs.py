@@ -68,6 +68,9 @@ class StreamConfig:
     nms_iou_milli: int = 0         # NMS IoU threshold in thousandths (0: spans never overlap)
     unit_tokens: int = 0           # retrieval granularity: 0 = spans, U = fixed units of U tokens (Eq. 8 as printed)
     persist_decode: bool = False   # decode keeps the spans selected by the last prefill call (Sec. 3.5)
+    retrieval_head: tuple = None   # per layer: retrieval head or -1 (Sec. 3.5); None: no layer has one
+    retrieval_head_score: tuple = None   # per layer: the head's score, its voting weight
+    collab_vote: bool = False      # collaborative voting over the layers' ballots (Sec. 3.5; needs unit_tokens)
 
     @property
     def max_tokens(self) -> int:

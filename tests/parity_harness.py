@@ -42,6 +42,7 @@ class Report:
     max_score_rel: float = 0.0
     rep_counts: int = 0
     rep_count_flips: int = 0
+    vote_changes: int = 0   # selections that the ballots of other layers changed (collaborative voting)
 
 
 def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
@@ -50,17 +51,30 @@ def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
                                reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
                                theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode,
                                ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps, max_reps=cfg.max_reps,
-                               rep_lambda=cfg.rep_lambda, flags=binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0,
-                               unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli)
+                               rep_lambda=cfg.rep_lambda,
+                               flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
+                                     (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0),
+                               unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
+                               retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score)
 
 
-def oracle_of(cfg: inputs.StreamConfig) -> orc.OracleStream:
+def ret_head_of(cfg: inputs.StreamConfig, layer: int):
+    """(retrieval head or -1, its weight) of a layer."""
+    if cfg.retrieval_head is None:
+        return -1, 0.0
+    w = 1.0 if cfg.retrieval_head_score is None else float(cfg.retrieval_head_score[layer])
+    return int(cfg.retrieval_head[layer]), w
+
+
+def oracle_of(cfg: inputs.StreamConfig, layer: int = 0) -> orc.OracleStream:
+    rh, w = ret_head_of(cfg, layer)
     return orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
                             cfg.max_tokens, reps_per_span=cfg.reps_per_span,
                             max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
                             max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda, persist_decode=int(cfg.persist_decode),
-                            unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli)
+                            unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli, ret_head=rh, head_weight=w,
+                            collab_vote=int(cfg.collab_vote))
 
 
 def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str):
@@ -75,9 +89,14 @@ def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str
     assert rf <= REL_FRO, f"{what}: relative Frobenius {rf:.4g} > {REL_FRO}"
 
 
-def check_selection(sel_gpu: np.ndarray, o: orc.OracleStream, rep: Report, what: str):
-    """sel_gpu [Hkv][k] ascending ids (-1 padded) against the oracle's scores; adopts tolerated picks."""
+def check_selection(sel_gpu: np.ndarray, o: orc.OracleStream, rep: Report, what: str, voted=False):
+    """sel_gpu [Hkv][k] ascending ids (-1 padded) against the oracle's scores; adopts tolerated picks.
+
+    voted: the units were ranked by the tally of the layers' ballots first (Sec. 3.5, collaborative voting); a pick
+    may then differ only among units with the tally of the last unit the oracle took.
+    """
     sel_o, _ = o.selected()
+    tally = o.tally() if voted else None
     if o.unit_tokens > 0:
         # unit mode: the ids are absolute unit numbers, the scores those of the units that meet the indexed range
         us = o.unit_scores()
@@ -94,7 +113,14 @@ def check_selection(sel_gpu: np.ndarray, o: orc.OracleStream, rep: Report, what:
         if a == b:
             continue
         # the sets may differ only among spans whose oracle scores are within the near-tie band of the cut
-        cut = min(sc[g][i] for i in b)
+        if voted:
+            u0 = o.n_sink // o.unit_tokens
+            last = [int(x) for x in sel_o[g] if x >= 0][-1]        # the oracle lists its picks in rank order
+            cut = sc[g][last]
+            for i in a ^ b:
+                assert tally[i - u0] == tally[last - u0], f"{what}: KV head {g} unit {i}: tally differs from the cut's"
+        else:
+            cut = min(sc[g][i] for i in b)
         band = NEAR_TIE * max(abs(cut), 1e-30)
         for i in a ^ b:
             assert abs(sc[g][i] - cut) <= band, (
@@ -116,7 +142,9 @@ class StreamPair:
         self.cfg, self.layers, self.seqs, self.deep = cfg, list(layers), list(seqs), deep
         self.dev = torch.device(device)
         self.lt = binding.Ltri(params_of(cfg), device=device)
-        self.orc = {(s, l): oracle_of(cfg) for s in self.seqs for l in self.layers}
+        self.orc = {(s, l): oracle_of(cfg, l) for s in self.seqs for l in self.layers}
+        if cfg.collab_vote:   # a layer needs the ballots of every layer before it
+            assert self.layers == list(range(cfg.n_layers)), "collaborative voting: check every layer"
         self.rep = Report()
         self.n_indexed = {(s, l): 0 for s in self.seqs for l in self.layers}
         self.count_of = {}   # (seq, layer, span start) -> representative count decided when its region was current
@@ -130,11 +158,16 @@ class StreamPair:
         torch.cuda.synchronize(self.dev)
         assert lt.ltri_sync_status() == 0
         rep.calls += 1
+        ballots = []   # collaborative voting: (weight, units) of the layers handled so far
         for layer in self.layers:
             if (seq, layer) not in self.orc:
                 continue
             o = self.orc[(seq, layer)]
             what = f"seq {seq} layer {layer} call@{o.tokens}"
+            rh, _ = ret_head_of(cfg, layer)
+            gk = slice(None) if rh < 0 else slice(rh // (cfg.n_q_heads // cfg.n_kv_heads),
+                                                  rh // (cfg.n_q_heads // cfg.n_kv_heads) + 1)
+            nh = cfg.n_q_heads if rh < 0 else 1    # heads summed into the layer's map
             o.prefill_local(q[layer], k[layer], v[layer])
             rs, m = o.region()
             t1 = o.tokens
@@ -148,10 +181,10 @@ class StreamPair:
                     Mo = o.map()
                     md = int(np.abs(Mg.astype(np.int64) - Mo).max())
                     rep.max_map_diff = max(rep.max_map_diff, md)
-                    assert md <= 4 + cfg.n_q_heads, f"{what}: region map differs by {md} Q20 units"
+                    assert md <= 4 + nh, f"{what}: region map differs by {md} Q20 units"
                     thg = int(lt.ltri_debug_read(binding.BUF_THETA, seq, layer)[0])
                     rep.max_theta_diff = max(rep.max_theta_diff, abs(thg - o.theta_q()))
-                    assert abs(thg - o.theta_q()) <= 4 + cfg.n_q_heads, f"{what}: theta {thg} vs {o.theta_q()}"
+                    assert abs(thg - o.theta_q()) <= 4 + nh, f"{what}: theta {thg} vs {o.theta_q()}"
                     if cfg.theta_mode == 1:
                         assert thg == orc.theta_q(Mg, 1, cfg.theta, cfg.n_q_heads), f"{what}: theta rank select"
                     # integer pipeline: bit-exact on identical integer input
@@ -188,22 +221,57 @@ class StreamPair:
                 dv = np.abs(vg[lo:] - vo[lo:])
                 assert np.all(dv <= 64 + 2e-5 * np.abs(vo[lo:])), f"{what}: votes differ by up to {dv.max()}"
             self._check_index(seq, layer, o, k, what)
+            if cfg.collab_vote:
+                o.set_ballots(ballots)
             o.prefill_retrieve()
             if len(o.spans()):
                 if self.deep and m > 0:
+                    # (under a retrieval head only the rows of its KV head mean anything on the GPU side)
                     J = len(o.pending()[-1][2])
                     ug = lt.ltri_debug_read(binding.BUF_QREPS, seq, layer)[:, :J]
-                    assert np.allclose(ug, o.query_reps(), rtol=0, atol=1e-4), f"{what}: query representatives"
+                    assert np.allclose(ug[gk], o.query_reps()[gk], rtol=0, atol=1e-4), f"{what}: query representatives"
                     ns = len(o.spans())
                     sg = lt.ltri_debug_read(binding.BUF_SCORES, seq, layer)[:, :ns]
                     so = o.scores()
-                    rel = float(np.abs(sg - so).max() / max(np.abs(so).max(), 1e-30))
+                    rel = float(np.abs(sg[gk] - so[gk]).max() / max(np.abs(so[gk]).max(), 1e-30))
                     rep.max_score_rel = max(rep.max_score_rel, rel)
                     assert rel <= 2e-5, f"{what}: scores differ by {rel:.3g} relative"
-                check_selection(lt.ltri_get_selected(seq, layer), o, rep, what)
+                if cfg.collab_vote:
+                    self._vote(seq, layer, o, ballots, what)
+                    self._count_vote_changes(o)
+                check_selection(lt.ltri_get_selected(seq, layer), o, rep, what, voted=cfg.collab_vote)
             if check_out:
                 check_output(out[layer], o.prefill_attend(), rep, what)
         return out
+
+    def _vote(self, seq, layer, o, ballots, what):
+        """Collaborative voting (Sec. 3.5): compare the layer's own ballot, let the oracle adopt a tolerated pick and
+        count again, and add the ballot to those the later layers read."""
+        cfg, rep = self.cfg, self.rep
+        rh, w = ret_head_of(cfg, layer)
+        bg = self.lt.ltri_debug_read(binding.BUF_BALLOT, seq, layer)
+        bo = o.ballot()
+        if rh < 0:
+            assert (bg < 0).all() and (bo < 0).all(), f"{what}: a layer without a retrieval head cast a ballot"
+            return
+        a, b = set(int(x) for x in bg if x >= 0), set(int(x) for x in bo if x >= 0)
+        assert len(a) == len(b), f"{what}: ballot of {len(a)} units, oracle {len(b)}"
+        if a != b:
+            us = o.unit_scores()[0]
+            u0 = cfg.n_sink // cfg.unit_tokens
+            cut = min(us[i - u0] for i in b)
+            for i in a ^ b:
+                assert abs(us[i - u0] - cut) <= NEAR_TIE * max(abs(cut), 1e-30), f"{what}: ballot unit {i}: no near tie"
+            rep.sel_flips += 1
+            o.set_ballot(bg)
+        ballots.append((w, o.ballot()))
+
+    def _count_vote_changes(self, o):
+        us, sel = o.unit_scores(), o.selected()[0]
+        u0 = self.cfg.n_sink // self.cfg.unit_tokens
+        for g in range(us.shape[0]):
+            own = set((np.argsort(-us[g], kind="stable")[:self.cfg.top_k] + u0).tolist())
+            self.rep.vote_changes += own != set(int(x) for x in sel[g] if x >= 0)
 
     def _check_index(self, seq, layer, o, k, what):
         spans_o = o.spans()
@@ -241,14 +309,20 @@ class StreamPair:
         assert lt.ltri_sync_status() == 0
         rep.calls += 1
         for i, seq in enumerate(seq_ids):
+            ballots = []
             for layer in self.layers:
                 if (seq, layer) not in self.orc:
                     continue
                 o = self.orc[(seq, layer)]
                 what = f"seq {seq} layer {layer} decode@{o.tokens}"
+                if cfg.collab_vote:
+                    o.set_ballots(ballots)
                 o.decode_retrieve(q[i, layer], k[i, layer], v[i, layer])
                 if len(o.spans()):
-                    check_selection(lt.ltri_get_selected(seq, layer), o, rep, what)
+                    if cfg.collab_vote:
+                        self._vote(seq, layer, o, ballots, what)
+                        self._count_vote_changes(o)
+                    check_selection(lt.ltri_get_selected(seq, layer), o, rep, what, voted=cfg.collab_vote)
                     # tokens the step attends over besides sink and local: this step's spans united, under the
                     # persistent mechanism, with those of the last prefill call (every span once)
                     sel_o, _ = o.selected()

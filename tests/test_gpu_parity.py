@@ -101,6 +101,55 @@ def test_overlapping_spans_from_nms_with_iou_threshold(phi_milli, U):
     print(rep)
 
 
+@pytest.mark.parametrize("fused,theta_mode", [("0", 1), ("1", 0), ("2", 1)])
+def test_retrieval_heads(fused, theta_mode, monkeypatch):
+    # Sec. 3.5: a layer with a retrieval head draws its map, threshold, votes, query representatives and scores from
+    # that head alone and fetches one selection for all its KV heads; layers without one keep the default path.  All
+    # decode retrieval paths, span-granular retrieval.
+    monkeypatch.setenv("LTRI_DEC_FUSED", fused)
+    cfg = small_cfg(n_layers=3, context=1408, decode_steps=5, retrieval_head=(5, -1, 2),
+                    theta_mode=theta_mode, theta=0.90 if theta_mode else 0.004)
+    rep = ph.run_stream(cfg, layers=[0, 1, 2])
+    assert rep.sel_checks > 30
+    print(rep)
+
+
+@pytest.mark.parametrize("U,persist,heads,weights", [
+    (64, False, (1, -1, 6, 3), (0.5, 0.0, 0.25, 0.25)),
+    (32, True, (-1, 4, 4, -1), (0.0, 0.3, 0.3, 0.0)),
+    (128, False, (0, 7, 2, 5), None),
+])
+def test_collaborative_voting(U, persist, heads, weights):
+    # Sec. 3.5: every layer with a retrieval head casts its own top-k units as a ballot weighted by the head's score;
+    # a layer ranks its units by the tally of the ballots up to its own, then by its own scores.  Ballots, tallied
+    # selections, decode token counts and outputs are checked layer by layer.
+    cfg = small_cfg(n_layers=4, context=1536, decode_steps=4, unit_tokens=U, persist_decode=persist, top_k=3,
+                    retrieval_head=heads, retrieval_head_score=weights, collab_vote=True)
+    rep = ph.run_stream(cfg, layers=[0, 1, 2, 3])
+    assert rep.sel_checks > 40 and rep.vote_changes > 5   # the other layers' ballots did change selections
+    print(rep)
+
+
+def test_voting_layer_by_layer_calls_match_one_call():
+    # a real model submits one layer at a time: the ballots of the earlier layers of the same chunk are read from the
+    # context's state and the selections must equal those of the all-layers call
+    cfg = small_cfg(n_layers=3, context=1024, decode_steps=0, unit_tokens=64, top_k=3, retrieval_head=(2, 5, -1),
+                    retrieval_head_score=(0.4, 0.6, 0.0), collab_vote=True)
+    st = inputs.SyntheticStream(cfg)
+    a, b = binding.Ltri(ph.params_of(cfg)), binding.Ltri(ph.params_of(cfg))
+    for t0, n in st.prefill_chunks():
+        q, k, v = (x.cuda() for x in st.tokens(t0, n))
+        oa = a.ltri_prefill_chunk(0, 0, 3, q, k, v)
+        for l in range(3):
+            ob = b.ltri_prefill_chunk(0, l, 1, q[l:l + 1].contiguous(), k[l:l + 1].contiguous(), v[l:l + 1].contiguous())
+            assert torch.equal(oa[l], ob[0])
+            assert np.array_equal(a.ltri_get_selected(0, l), b.ltri_get_selected(0, l))
+    assert a.ltri_sync_status() == 0 and b.ltri_sync_status() == 0
+    assert (a.ltri_get_selected(0, 2) >= 0).any()
+    a.close()
+    b.close()
+
+
 def test_top_k_covering_everything_equals_full_attention():
     # with top_k >= number of spans the streamed output is plain causal attention (oracle O12)
     cfg = small_cfg(n_layers=1, context=640, chunk=64, window=128, top_k=64, max_spans_per_region=2, decode_steps=2)
