@@ -30,6 +30,10 @@
 //   O9'  retrieval in fixed token units, unit score = max      Eq. 8 as printed
 //        over the unit's spans
 //   O11' decode keeps the last prefill call's selection        Sec. 3.5 "Persistent Mechanism"
+//   O3'  a layer locates evidence with its retrieval head      Sec. 3.5 "Retrieval Heads"
+//        alone (map, theta, votes, representatives, scores)
+//   O9'' units ranked by the weighted ballots of the layers    Sec. 3.5 "Collaborative Voting"
+//        up to this one, then by the layer's own scores
 //
 // Parity status: O3/O10/O12 are pinned by softmax invariants and by the full-attention
 // equivalence; O6 is pinned by brute force, by hand-built block maps and by a library
@@ -41,7 +45,10 @@
 // modes) the definition of the area ratio r_a behind Eq. r_v, which the paper gives only
 // as a figure.  Pinned among the optional modes: the shape of Eq. r_v and its clamps, the
 // IoU NMS against a library NMS, the unit scores and the tokens a unit-granular step
-// attends over, the union semantics of the persistent mechanism.
+// attends over, the union semantics of the persistent mechanism, the retrieval-head layer
+// against the one-head model of that head, the vote ranking against a restated sort.
+// "parity unpinned" there too: what a ballot is and how tallies and own scores combine,
+// which the paper describes in one sentence.
 //
 // Build: g++ -O2 -std=c++17 -shared -fPIC -pthread ltri_oracle.cpp -o libltri_oracle.so
 
