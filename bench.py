@@ -197,10 +197,11 @@ def oracle_sample(cfg, steps, warmup):
     need = (fill + warmup + steps) * cfg.chunk
     o = orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
                          need + 8, reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
-                         theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind,
-                         min_reps=cfg.min_reps, max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
+                         theta_mode=cfg.theta_mode, theta=cfg.layer_theta[0] if cfg.layer_theta else cfg.theta,
+                         rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps, max_reps=cfg.max_reps,
+                         rep_lambda=cfg.layer_rep_lambda[0] if cfg.layer_rep_lambda else cfg.rep_lambda,
                          unit_tokens=cfg.unit_tokens, persist_decode=int(cfg.persist_decode),
-                         nms_iou_milli=cfg.nms_iou_milli,
+                         nms_iou_milli=cfg.layer_nms_iou_milli[0] if cfg.layer_nms_iou_milli else cfg.nms_iou_milli,
                          ret_head=cfg.retrieval_head[0] if cfg.retrieval_head else -1,
                          head_weight=cfg.retrieval_head_score[0] if cfg.retrieval_head_score else 1.0,
                          collab_vote=int(cfg.collab_vote))
@@ -319,7 +320,9 @@ def run_ltri(args, cfg):
                             flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
                                   (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0),
                             unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
-                            retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score)
+                            retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score,
+                            layer_theta=cfg.layer_theta, layer_nms_iou_milli=cfg.layer_nms_iou_milli,
+                            layer_rep_lambda=cfg.layer_rep_lambda)
 
     def stream_until(lt, upto, keep_from):
         for s in range(NSEQ - 1):
@@ -525,6 +528,10 @@ def main():
                     help="IoU threshold of the segmenter's NMS (0: spans never overlap; the paper lists 0.1 / 0.01)")
     ap.add_argument("--persist-decode", action="store_true",
                     help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
+    ap.add_argument("--layer-tables", action="store_true",
+                    help="per-layer theta (quantile levels spread over 0.88..0.95), phi (0.1 / 0.01 alternating) and "
+                         "lambda (20 for the first four layers, 3 after them, as in the paper's implementation "
+                         "details); the theta and phi values are made up within the paper's ranges")
     ap.add_argument("--retrieval-heads", action="store_true",
                     help="give 14 of every 32 layers a retrieval head (a made-up table: which heads these are belongs "
                          "to a trained model); such a layer locates evidence with that head alone")
@@ -562,6 +569,14 @@ def main():
         import dataclasses
         cfg = dataclasses.replace(cfg, persist_decode=True)
         cfg.name += "[persist-decode]"
+    if args.layer_tables:
+        import dataclasses
+        L = cfg.n_layers
+        cfg = dataclasses.replace(
+            cfg, layer_theta=tuple(0.88 + 0.07 * ((l * 13) % 8) / 7 for l in range(L)),
+            layer_nms_iou_milli=tuple(100 if l % 2 == 0 else 10 for l in range(L)),
+            layer_rep_lambda=tuple(20.0 if l < 4 else 3.0 for l in range(L)))
+        cfg.name += "[layer-tables]"
     if args.retrieval_heads:
         import dataclasses
         has = [(l * 7) % 16 < 7 for l in range(cfg.n_layers)]

@@ -89,6 +89,12 @@ typedef struct {
    * supplies them. */
   const int32_t* retrieval_head;
   const float* retrieval_head_score;
+  /* Per-layer tables (App. "Experimental Details": theta and phi are searched per layer, lambda is larger for the
+   * first layers).  HOST arrays of n_layers entries, read at ltri_create and not kept; NULL: the scalar above holds
+   * for every layer.  Same meaning and range as theta, nms_iou_milli and rep_lambda. */
+  const float* layer_theta;
+  const int32_t* layer_nms_iou_milli;
+  const float* layer_rep_lambda;
   void* arena;                                       /* caller-owned device memory, 256-byte aligned */
   size_t arena_bytes;                                /* >= ltri_arena_bytes(params) */
 } ltri_params;

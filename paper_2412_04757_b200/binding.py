@@ -42,6 +42,8 @@ class LtriParams(C.Structure):
         ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
         ("rep_lambda", C.c_float), ("unit_tokens", C.c_int32), ("nms_iou_milli", C.c_int32),
         ("retrieval_head", C.POINTER(C.c_int32)), ("retrieval_head_score", C.POINTER(C.c_float)),
+        ("layer_theta", C.POINTER(C.c_float)), ("layer_nms_iou_milli", C.POINTER(C.c_int32)),
+        ("layer_rep_lambda", C.POINTER(C.c_float)),
         ("arena", C.c_void_p), ("arena_bytes", C.c_size_t),
     ]
 
@@ -107,12 +109,14 @@ def strerror(code: int) -> str:
 def make_params(n_layers, n_q_heads, n_kv_heads, max_tokens, chunk, window, n_sink, top_k, head_dim=128, max_seqs=1,
                 reps_per_span=1, max_spans_per_region=0, theta_mode=1, theta=0.90, softmax_scale=0.0,
                 rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, flags=0, unit_tokens=0, nms_iou_milli=0,
-                retrieval_head=None, retrieval_head_score=None) -> LtriParams:
-    """retrieval_head / retrieval_head_score: per-layer sequences (head or -1; weight), marshalled into host arrays
-    that live as long as the returned struct."""
+                retrieval_head=None, retrieval_head_score=None, layer_theta=None, layer_nms_iou_milli=None,
+                layer_rep_lambda=None) -> LtriParams:
+    """retrieval_head / retrieval_head_score (head or -1; weight) and layer_theta / layer_nms_iou_milli /
+    layer_rep_lambda: per-layer sequences, marshalled into host arrays that live as long as the returned struct."""
     p = LtriParams(n_layers, n_q_heads, n_kv_heads, head_dim, max_seqs, max_tokens, chunk, window, n_sink, top_k,
                    reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, flags,
-                   rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, unit_tokens, nms_iou_milli, None, None, None, 0)
+                   rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, unit_tokens, nms_iou_milli, None, None, None, None,
+                   None, None, 0)
     if retrieval_head is not None:
         if len(retrieval_head) != n_layers:
             raise ValueError("retrieval_head needs one entry per layer")
@@ -123,6 +127,15 @@ def make_params(n_layers, n_q_heads, n_kv_heads, max_tokens, chunk, window, n_si
                 raise ValueError("retrieval_head_score needs one entry per layer")
             p._rw = (C.c_float * n_layers)(*[float(w) for w in retrieval_head_score])
             p.retrieval_head_score = C.cast(p._rw, C.POINTER(C.c_float))
+    p._tables = []
+    for name, vals, ct in (("layer_theta", layer_theta, C.c_float), ("layer_nms_iou_milli", layer_nms_iou_milli, C.c_int32),
+                           ("layer_rep_lambda", layer_rep_lambda, C.c_float)):
+        if vals is not None:
+            if len(vals) != n_layers:
+                raise ValueError(f"{name} needs one entry per layer")
+            arr = (ct * n_layers)(*[ct(v).value for v in vals])
+            p._tables.append(arr)
+            setattr(p, name, C.cast(arr, C.POINTER(ct)))
     return p
 
 

@@ -52,6 +52,10 @@ struct DevCtx {
   const int* ret_head;   // [NL]  retrieval head of the layer, -1 none; nullptr: no layer has one
   const float* head_w;   // [NL]  its score = the weight of the layer's ballot
   int* ballot;           // [NS][NL][topk]  own top-k units of a layer with a retrieval head (ascending, -1 padded)
+  // per-layer tables of the paper's configuration appendix (nullptr: the scalar holds for every layer)
+  const float* theta_l;  // [NL]  theta
+  const int* phi_l;      // [NL]  NMS IoU threshold in thousandths
+  const float* lambda_l; // [NL]  lambda of Eq. r_v
   long long* sel_tokens; // [NS][NL]  retrieved tokens of the last call, summed over KV heads
   // per-layer scratch of the prefill call in flight
   int* Mq;               // [NL][chunk][chunk]
@@ -123,7 +127,7 @@ cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_co
 // and, when q != nullptr, the summed query representatives of every span.  theta_mode 0/2: theta_q_abs is used.
 cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_count, int m, int reg_start, int slot,
                            int theta_mode, float theta, long long theta_q_abs, int max_spans, int n, int t0,
-                           const __nv_bfloat16* q, cudaStream_t s);
+                           const __nv_bfloat16* q, cudaStream_t s, bool tables = false);
 cudaError_t launch_score_prefill(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s);
 // tensor-core version of launch_score_prefill (split-bf16 representatives)
 cudaError_t launch_score_prefill_mma(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s);

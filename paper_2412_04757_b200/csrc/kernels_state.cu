@@ -256,13 +256,18 @@ constexpr int kThetaCluster = 8;   // CTAs (one thread-block cluster) per layer
 constexpr int kThetaThreads = 512;
 
 __global__ void __cluster_dims__(kThetaCluster, 1, 1) __launch_bounds__(kThetaThreads)
-    k_theta_select(DevCtx c, int layer_begin, int m, long long rank) {
+    k_theta_select(DevCtx c, int layer_begin, int m, long long rank, int tables) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ unsigned hist[];  // [warps][kThetaBins]
   constexpr int NW = kThetaThreads / 32;
   const int layer = layer_begin + blockIdx.x / kThetaCluster;
   const int part = (int)cluster.block_rank();
+  if (tables && c.theta_l) {  // the layer's own quantile level: the same double arithmetic as on the host
+    const long long N = (long long)m * (m + 1) / 2;
+    rank = (long long)floor((double)c.theta_l[layer] * (double)(N - 1));
+    rank = rank < 0 ? 0 : (rank > N - 1 ? N - 1 : rank);
+  }
   const int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
   __shared__ unsigned loc[kThetaBins + 2];  // this CTA's histogram, then its counts of negatives and zeros
   __shared__ unsigned tot[kThetaBins];      // the cluster's histogram (every CTA builds its own copy)
@@ -394,10 +399,14 @@ __global__ void __cluster_dims__(kThetaCluster, 1, 1) __launch_bounds__(kThetaTh
     c.thetaq[layer] = cls > 0 ? (long long)s_prefix : (long long)(int)(s_prefix ^ 0x80000000u);
 }
 
-// absolute threshold: thq in units of the map summed over all heads, thq1 in units of a single (retrieval) head's map
-__global__ void k_theta_set(DevCtx c, int layer_begin, long long thq, long long thq1) {
+// absolute threshold: thq in units of the map summed over all heads, thq1 in units of a single (retrieval) head's map;
+// with per-layer tables the layer's own theta, scaled here
+__global__ void k_theta_set(DevCtx c, int layer_begin, long long thq, long long thq1, int tables) {
   const int layer = layer_begin + blockIdx.x;
-  c.thetaq[layer] = ret_head_of(c, layer) >= 0 ? thq1 : thq;
+  const bool one = ret_head_of(c, layer) >= 0;
+  long long t = one ? thq1 : thq;
+  if (tables && c.theta_l) t = (long long)rint((double)c.theta_l[layer] * (one ? 1.0 : (double)c.Hq) * (double)kQScale);
+  c.thetaq[layer] = t;
 }
 
 // step 2: suffix sums along each row of D = Mq - theta ("sum the right elements", Fig. 2):
@@ -492,6 +501,7 @@ struct NmsArgs {
   int seq, layer_begin, m, reg_start, slot, max_spans;
   int n, t0;                 // query tensor geometry (q == nullptr: skip the representatives)
   const __nv_bfloat16* q;
+  int tables;                // use the context's per-layer phi and lambda tables where it has them
 };
 
 __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
@@ -503,7 +513,8 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   const int layer = a.layer_begin + blockIdx.x;
   const size_t unit = unit_of(c, a.seq, layer);
   const int m = a.m;
-  const int phi_milli = c.phi_milli;
+  const int phi_milli = a.tables && c.phi_l ? c.phi_l[layer] : c.phi_milli;
+  const float rep_lambda = a.tables && c.lambda_l ? c.lambda_l[layer] : c.rep_lambda;
   const int ncand = 2 * m - 1;
   int npow = 1;
   while (npow < ncand) npow <<= 1;
@@ -643,7 +654,7 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
       const long long R = TR - T;
       const long long nb = c.ratio_kind == 0 ? R : c.ratio_kind == 1 ? Cn : R + Cn;
       const double ra = (T + nb) > 0 ? (double)T / (double)(T + nb) : 1.0;
-      const double rv = 1.0 / exp((double)c.rep_lambda * (1.0 - ra));
+      const double rv = 1.0 / exp((double)rep_lambda * (1.0 - ra));
       cnt = (int)rint((double)out_len[j] * rv);  // to nearest even
       cnt = max(cnt, c.min_reps);
       cnt = min(cnt, c.max_reps);
@@ -717,22 +728,22 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
 
 cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_count, int m, int reg_start,
                              int slot, int theta_mode, float theta, long long theta_q_abs, int max_spans, int n,
-                             int t0, const __nv_bfloat16* q, cudaStream_t s) {
+                             int t0, const __nv_bfloat16* q, cudaStream_t s, bool tables) {
   if (theta_mode == 1) {
     const long long N = (long long)m * (m + 1) / 2;
     long long rank = (long long)floor((double)theta * (double)(N - 1));
     if (rank < 0) rank = 0;
     if (rank > N - 1) rank = N - 1;
     const int hsmem = (kThetaThreads / 32) * kThetaBins * (int)sizeof(unsigned);
-    k_theta_select<<<layer_count * kThetaCluster, kThetaThreads, hsmem, s>>>(c, layer_begin, m, rank);
+    k_theta_select<<<layer_count * kThetaCluster, kThetaThreads, hsmem, s>>>(c, layer_begin, m, rank, tables);
   } else {
     k_theta_set<<<layer_count, 1, 0, s>>>(c, layer_begin, theta_q_abs,
-                                          (long long)nearbyint((double)theta * (double)kQScale));
+                                          (long long)nearbyint((double)theta * (double)kQScale), tables);
   }
   k_seg_rowscan<<<dim3((m + 7) / 8, layer_count), 256, 0, s>>>(c, layer_begin, m);
   const size_t smem = (size_t)(32 * 32 + m + 32) * sizeof(long long);
   k_seg_colscan<<<dim3((m + 31) / 32, layer_count), 1024, smem, s>>>(c, layer_begin, m);
-  NmsArgs a{seq, layer_begin, m, reg_start, slot, max_spans, n, t0, q};
+  NmsArgs a{seq, layer_begin, m, reg_start, slot, max_spans, n, t0, q, tables ? 1 : 0};
   k_seg_nms<<<layer_count, 1024, 0, s>>>(c, a);
   return cudaGetLastError();
 }

@@ -70,6 +70,11 @@ bool validate(const ltri_params* p) {
     if (p->unit_tokens < 8 || p->unit_tokens > p->chunk || p->unit_tokens % 8) return false;
     if (p->max_tokens / p->unit_tokens + 2 > 12288) return false;  // unit keys of the top-k kernel: 48 KB of shared memory
   }
+  for (int l = 0; l < p->n_layers; ++l) {
+    if (p->layer_theta && (!(p->layer_theta[l] >= 0.f) || (p->theta_mode == 1 && p->layer_theta[l] > 1.f))) return false;
+    if (p->layer_nms_iou_milli && (p->layer_nms_iou_milli[l] < 0 || p->layer_nms_iou_milli[l] > 999)) return false;
+    if (p->layer_rep_lambda && !(p->layer_rep_lambda[l] >= 0.f)) return false;
+  }
   if (p->rep_mode != 0 && p->rep_mode != 1) return false;
   if (p->rep_mode == 1) {
     if (p->ratio_kind < 0 || p->ratio_kind > 2) return false;
@@ -139,6 +144,12 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
     d.ret_head = p.retrieval_head ? rh : nullptr;
     d.head_w = p.retrieval_head ? hw : nullptr;
     d.ballot = cv.take<int>(units * d.topk);
+    float* th = cv.take<float>(d.NL);
+    int* ph = cv.take<int>(d.NL);
+    float* la = cv.take<float>(d.NL);
+    d.theta_l = p.layer_theta ? th : nullptr;
+    d.phi_l = p.layer_nms_iou_milli ? ph : nullptr;
+    d.lambda_l = p.layer_rep_lambda ? la : nullptr;
   }
   d.Mq = cv.take<int>((size_t)d.NL * d.chunk * d.chunk);
   d.Rsuf = cv.take<long long>((size_t)d.NL * d.chunk * d.chunk);
@@ -281,6 +292,9 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
   }
   ctx->p.retrieval_head = nullptr;
   ctx->p.retrieval_head_score = nullptr;
+  ctx->p.layer_theta = nullptr;
+  ctx->p.layer_nms_iou_milli = nullptr;
+  ctx->p.layer_rep_lambda = nullptr;
   if (p->flags & LTRI_FLAG_HOST_STAGING) {
     bool ok = cudaStreamCreateWithFlags(&ctx->s_up, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&ctx->s_down, cudaStreamNonBlocking) == cudaSuccess;
@@ -322,6 +336,13 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
       e = cudaMemcpyAsync(const_cast<float*>(ctx->d.head_w), ctx->head_w.data(), ctx->head_w.size() * sizeof(float),
                           cudaMemcpyHostToDevice, s);
   }
+  // per-layer tables: copied from the caller's arrays (the stream is synchronised below, before this call returns)
+  auto up = [&](const void* dst, const void* src, size_t bytes) {
+    if (e == cudaSuccess && dst && src) e = cudaMemcpyAsync(const_cast<void*>(dst), src, bytes, cudaMemcpyHostToDevice, s);
+  };
+  up(ctx->d.theta_l, p->layer_theta, (size_t)p->n_layers * sizeof(float));
+  up(ctx->d.phi_l, p->layer_nms_iou_milli, (size_t)p->n_layers * sizeof(int));
+  up(ctx->d.lambda_l, p->layer_rep_lambda, (size_t)p->n_layers * sizeof(float));
   if (e == cudaSuccess) e = launch_init(ctx->d, -1, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) {
@@ -458,7 +479,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
     long long thq_abs = 0;
     if (d.theta_mode == 0) thq_abs = (long long)std::nearbyint((double)d.theta * (double)d.Hq * (double)kQScale);
     LTRI_CUDA(ctx, launch_segment(d, seq, layer_begin, layer_count, m, reg_start, slot, d.theta_mode, d.theta, thq_abs,
-                                  d.C, n_tokens, t0, a.q, st));
+                                  d.C, n_tokens, t0, a.q, st, /*tables=*/true));
   }
   if (has_index) {
     {

@@ -55,7 +55,9 @@ def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
                                flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
                                      (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0),
                                unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
-                               retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score)
+                               retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score,
+                               layer_theta=cfg.layer_theta, layer_nms_iou_milli=cfg.layer_nms_iou_milli,
+                               layer_rep_lambda=cfg.layer_rep_lambda)
 
 
 def ret_head_of(cfg: inputs.StreamConfig, layer: int):
@@ -66,14 +68,22 @@ def ret_head_of(cfg: inputs.StreamConfig, layer: int):
     return int(cfg.retrieval_head[layer]), w
 
 
+def layer_values(cfg: inputs.StreamConfig, layer: int):
+    """(theta, nms_iou_milli, rep_lambda) of a layer: its table entry, else the scalar."""
+    return (float(np.float32(cfg.layer_theta[layer])) if cfg.layer_theta else cfg.theta,
+            int(cfg.layer_nms_iou_milli[layer]) if cfg.layer_nms_iou_milli else cfg.nms_iou_milli,
+            float(np.float32(cfg.layer_rep_lambda[layer])) if cfg.layer_rep_lambda else cfg.rep_lambda)
+
+
 def oracle_of(cfg: inputs.StreamConfig, layer: int = 0) -> orc.OracleStream:
     rh, w = ret_head_of(cfg, layer)
+    theta, phi, lam = layer_values(cfg, layer)
     return orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
                             cfg.max_tokens, reps_per_span=cfg.reps_per_span,
-                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
+                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=theta,
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
-                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda, persist_decode=int(cfg.persist_decode),
-                            unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli, ret_head=rh, head_weight=w,
+                            max_reps=cfg.max_reps, rep_lambda=lam, persist_decode=int(cfg.persist_decode),
+                            unit_tokens=cfg.unit_tokens, nms_iou_milli=phi, ret_head=rh, head_weight=w,
                             collab_vote=int(cfg.collab_vote))
 
 
@@ -168,6 +178,7 @@ class StreamPair:
             gk = slice(None) if rh < 0 else slice(rh // (cfg.n_q_heads // cfg.n_kv_heads),
                                                   rh // (cfg.n_q_heads // cfg.n_kv_heads) + 1)
             nh = cfg.n_q_heads if rh < 0 else 1    # heads summed into the layer's map
+            theta_l, phi_l, lambda_l = layer_values(cfg, layer)
             o.prefill_local(q[layer], k[layer], v[layer])
             rs, m = o.region()
             t1 = o.tokens
@@ -186,9 +197,9 @@ class StreamPair:
                     rep.max_theta_diff = max(rep.max_theta_diff, abs(thg - o.theta_q()))
                     assert abs(thg - o.theta_q()) <= 4 + nh, f"{what}: theta {thg} vs {o.theta_q()}"
                     if cfg.theta_mode == 1:
-                        assert thg == orc.theta_q(Mg, 1, cfg.theta, cfg.n_q_heads), f"{what}: theta rank select"
+                        assert thg == orc.theta_q(Mg, 1, theta_l, cfg.n_q_heads), f"{what}: theta rank select"
                     # integer pipeline: bit-exact on identical integer input
-                    ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region, cfg.nms_iou_milli)
+                    ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region, phi_l)
                     ref_spans[:, 0] += rs
                     assert newest_g.tolist() == ref_spans.tolist(), f"{what}: segmenter differs on its own map"
                 if newest_g.tolist() != spans_o.tolist():
@@ -203,7 +214,7 @@ class StreamPair:
                 rep.rep_counts += J
                 if cfg.rep_mode == 1 and self.deep:
                     # integer sums, one division, one exponential, one rounding: the same on the GPU's own map
-                    ref = [orc.dynamic_rep_count(Mg, int(st - rs), int(st - rs + ln - 1), cfg.ratio_kind, cfg.rep_lambda,
+                    ref = [orc.dynamic_rep_count(Mg, int(st - rs), int(st - rs + ln - 1), cfg.ratio_kind, lambda_l,
                                                  cfg.min_reps, cfg.max_reps) for st, ln in newest_g]
                     assert ng.tolist() == ref, f"{what}: representative counts differ on the GPU's own map"
                 if ng.tolist() != no.tolist():

@@ -130,6 +130,18 @@ def test_collaborative_voting(U, persist, heads, weights):
     print(rep)
 
 
+@pytest.mark.parametrize("theta_mode,thetas", [(1, (0.88, 0.93, 0.95)), (0, (0.003, 0.006, 0.0045))])
+def test_per_layer_theta_phi_lambda_tables(theta_mode, thetas):
+    # the paper's configuration gives theta and phi per layer and a larger lambda to the first layers: every layer of
+    # the call must use its own entry (oracle streams are built with the layer's values)
+    cfg = small_cfg(n_layers=3, context=1408, decode_steps=3, theta_mode=theta_mode, layer_theta=thetas,
+                    layer_nms_iou_milli=(0, 100, 10), layer_rep_lambda=(20.0, 3.0, 0.5), rep_mode=1, ratio_kind=0,
+                    min_reps=1, max_reps=4, retrieval_head=(-1, 3, -1))
+    rep = ph.run_stream(cfg, layers=[0, 1, 2])
+    assert rep.regions >= 30 and rep.rep_counts > 50
+    print(rep)
+
+
 def test_voting_layer_by_layer_calls_match_one_call():
     # a real model submits one layer at a time: the ballots of the earlier layers of the same chunk are read from the
     # context's state and the selections must equal those of the all-layers call
