@@ -111,6 +111,8 @@ struct Params {
   int32_t unit_tokens;
   // NMS IoU threshold phi in thousandths (0: spans never overlap)
   int32_t nms_iou_milli;
+  // 1: every unit of unit_tokens tokens is segmented on its own, max_spans_per_region spans kept per unit
+  int32_t segment_per_unit;
   // retrieval head of this layer (Sec. 3.5): -1 = none, the layer locates evidence with all its heads; h >= 0 = the
   // local map, the votes, the query representatives and the scores come from head h alone, and its one selection
   // serves every KV head of the layer.  head_weight is that head's score, its voting weight.
@@ -286,6 +288,30 @@ void segment_map(const int32_t* Mq, int m, int ld, int64_t thq, int C, int phi_m
     pos = std::max(pos, k.y + 1);
   }
   if (pos < m) out.push_back(Span{pos, m - pos});
+  if (min_gap) *min_gap = gap;
+}
+
+// O6 per memory unit (Sec. 3.3 "each block ... divided into spans"): the region starts at absolute token `origin`;
+// the tokens are cut into units of `unit` tokens on the absolute grid and every unit's part of the region is segmented
+// on its own -- its own triangle of the map, its own candidates, NMS and cap C, its own gap fill -- with the region's
+// one threshold.  unit <= 0: the region is one piece.
+void segment_region(const int32_t* Mq, int m, int ld, int64_t thq, int C, int phi_milli, int unit, int origin,
+                    std::vector<Span>& out, double* min_gap) {
+  if (unit <= 0) {
+    segment_map(Mq, m, ld, thq, C, phi_milli, out, min_gap);
+    return;
+  }
+  out.clear();
+  double gap = 1.0;
+  for (int a = 0; a < m;) {
+    const int b = std::min(m, ((origin + a) / unit + 1) * unit - origin);  // end of the unit that holds token a
+    std::vector<Span> part;
+    double g = 1.0;
+    segment_map(Mq + (size_t)a * ld + a, b - a, ld, thq, C, phi_milli, part, &g);
+    for (const Span& sp : part) out.push_back(Span{sp.start + a, sp.len});
+    gap = std::min(gap, g);
+    a = b;
+  }
   if (min_gap) *min_gap = gap;
 }
 
@@ -563,7 +589,8 @@ struct Stream {
     if (m > 0) {
       thq = theta_q(Mq.data(), m, m, p.theta_mode, p.theta, p.ret_head >= 0 ? 1 : Hq);
       std::vector<Span> sp;
-      segment_map(Mq.data(), m, m, thq, p.max_spans_per_region, p.nms_iou_milli, sp, &seg_gap);
+      segment_region(Mq.data(), m, m, thq, p.max_spans_per_region, p.nms_iou_milli,
+                     p.segment_per_unit ? p.unit_tokens : 0, reg_start, sp, &seg_gap);
       for (Span& s : sp) s.start += reg_start;
       reg.spans = sp;
       decide_rep_counts(reg);
@@ -815,6 +842,7 @@ void* orc_create(const Params* p) {
   if (p->unit_tokens < 0 || p->nms_iou_milli < 0 || p->nms_iou_milli >= 1000) return nullptr;
   if (p->ret_head < -1 || p->ret_head >= p->n_q_heads || !(p->head_weight >= 0.f)) return nullptr;
   if (p->collab_vote && p->unit_tokens <= 0) return nullptr;
+  if (p->segment_per_unit && p->unit_tokens <= 0) return nullptr;
   if (p->rep_mode != 0 && p->rep_mode != 1) return nullptr;
   if (p->rep_mode == 1 && (p->ratio_kind < 0 || p->ratio_kind > 2 || p->min_reps < 1 || p->max_reps < p->min_reps ||
                            !(p->rep_lambda >= 0.f)))
@@ -999,9 +1027,10 @@ void orc_ta_scores(const int32_t* Mq, int m, int64_t thq, int64_t* S) {  // S[x*
   ta_scores(Mq, m, m, thq, s);
   std::memcpy(S, s.data(), s.size() * sizeof(int64_t));
 }
-int orc_segment_map(const int32_t* Mq, int m, int64_t thq, int C, int phi_milli, int* start_len, int cap, double* gap) {
+int orc_segment_map(const int32_t* Mq, int m, int64_t thq, int C, int phi_milli, int unit, int origin, int* start_len,
+                    int cap, double* gap) {
   std::vector<Span> sp;
-  segment_map(Mq, m, m, thq, C, phi_milli, sp, gap);
+  segment_region(Mq, m, m, thq, C, phi_milli, unit, origin, sp, gap);
   for (size_t i = 0; i < sp.size() && (int)i < cap; ++i) {
     start_len[2 * i] = sp[i].start;
     start_len[2 * i + 1] = sp[i].len;

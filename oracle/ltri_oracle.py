@@ -35,7 +35,7 @@ class _Params(C.Structure):
         ("max_tokens", C.c_int64),
         ("rep_mode", C.c_int32), ("ratio_kind", C.c_int32), ("min_reps", C.c_int32), ("max_reps", C.c_int32),
         ("rep_lambda", C.c_float), ("persist_decode", C.c_int32), ("unit_tokens", C.c_int32), ("nms_iou_milli", C.c_int32),
-        ("ret_head", C.c_int32), ("head_weight", C.c_float), ("collab_vote", C.c_int32),
+        ("segment_per_unit", C.c_int32), ("ret_head", C.c_int32), ("head_weight", C.c_float), ("collab_vote", C.c_int32),
     ]
 
 
@@ -81,7 +81,7 @@ def lib():
         L.orc_theta_q.argtypes = [vp, ip, ip, C.c_float, ip]
         L.orc_theta_q.restype = i64
         L.orc_ta_scores.argtypes = [vp, ip, i64, vp]
-        L.orc_segment_map.argtypes = [vp, ip, i64, ip, ip, vp, ip, vp]
+        L.orc_segment_map.argtypes = [vp, ip, i64, ip, ip, ip, ip, vp, ip, vp]
         L.orc_top_k.argtypes = [vp, ip, ip, vp, vp]
         L.orc_get_newest_rep_counts.argtypes = [vp, vp, ip]
         L.orc_get_newest_rep_counts.restype = ip
@@ -126,7 +126,8 @@ class OracleStream:
     def __init__(self, n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, max_tokens,
                  reps_per_span=1, max_spans_per_region=None, theta_mode=1, theta=0.90, softmax_scale=0.0,
                  rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, persist_decode=0,
-                 unit_tokens=0, nms_iou_milli=0, ret_head=-1, head_weight=0.0, collab_vote=0):
+                 unit_tokens=0, nms_iou_milli=0, ret_head=-1, head_weight=0.0, collab_vote=0,
+                 segment_per_unit=0):
         if max_spans_per_region is None:
             max_spans_per_region = max(1, chunk // 32)
         self.Hq, self.Hkv, self.d = n_q_heads, n_kv_heads, head_dim
@@ -135,7 +136,7 @@ class OracleStream:
         self._p = _Params(n_q_heads, n_kv_heads, head_dim, chunk, window, n_sink, top_k, reps_per_span,
                           max_spans_per_region, theta_mode, theta, softmax_scale, max_tokens,
                           rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, persist_decode, unit_tokens, nms_iou_milli,
-                          ret_head, head_weight, collab_vote)
+                          segment_per_unit, ret_head, head_weight, collab_vote)
         self.unit_tokens = unit_tokens
         self.ret_head, self.head_weight = ret_head, head_weight
         self._h = lib().orc_create(C.byref(self._p))
@@ -391,13 +392,17 @@ def ta_scores(Mq: np.ndarray, thq: int) -> np.ndarray:
     return S
 
 
-def segment_map(Mq: np.ndarray, thq: int, max_spans: int, phi_milli: int = 0):
-    """Spans [[start,len],...] covering [0,m) (a partition when phi = 0) and the smallest decisive relative gap."""
+def segment_map(Mq: np.ndarray, thq: int, max_spans: int, phi_milli: int = 0, unit: int = 0, origin: int = 0):
+    """Spans [[start,len],...] covering [0,m) (a partition when phi = 0) and the smallest decisive relative gap.
+
+    unit > 0: the region starts at absolute token `origin` and every unit of `unit` tokens (absolute grid) is
+    segmented on its own, `max_spans` kept per unit."""
     Mq = np.ascontiguousarray(Mq, dtype=np.int32)
     m = Mq.shape[0]
     out = np.zeros((2 * m + 1, 2), dtype=np.int32)
     gap = C.c_double(1.0)
-    c = lib().orc_segment_map(_ptr(Mq), m, int(thq), max_spans, int(phi_milli), _ptr(out), len(out), C.byref(gap))
+    c = lib().orc_segment_map(_ptr(Mq), m, int(thq), max_spans, int(phi_milli), int(unit), int(origin), _ptr(out),
+                              len(out), C.byref(gap))
     return out[:c].copy(), gap.value
 
 

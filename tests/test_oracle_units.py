@@ -109,3 +109,74 @@ def test_overlapping_spans_are_attended_once_per_token(U):
         q, k, v = st.tokens(cfg.context + s, 1, kind=1)
         out = o.decode_step(q[0, 0], k[0, 0], v[0, 0])
         assert np.abs(out - o.full_attention([cfg.context + s], q[0])[0]).max() < 5e-6
+
+
+# ---- segmentation per memory unit (Sec. 3.3: every unit is divided into spans on its own) ---------------------------
+def block_map(m, blocks, inside=4000, outside=0):
+    M = np.full((m, m), outside, dtype=np.int32)
+    for a, b in blocks:
+        M[a:b + 1, a:b + 1] = inside
+    return np.tril(M)
+
+
+@pytest.mark.parametrize("origin", [0, 64, 100, 37])
+def test_per_unit_segmentation_of_block_maps_cuts_blocks_at_unit_boundaries(origin):
+    # blocks of strong mutual attention; the expected spans are the blocks cut at the unit boundaries (closed form)
+    U, m = 64, 200
+    blocks = [(0, 29), (30, 79), (80, 139), (140, 199)]
+    M = block_map(m, blocks)
+    spans, _ = orc.segment_map(M, 2000, 8, 0, unit=U, origin=origin)   # inside +2000, outside -2000 per entry
+    cuts = sorted({0, m} | {a for a, _ in blocks} | {u * U - origin for u in range(1, 8) if 0 < u * U - origin < m})
+    want = [[a, b - a] for a, b in zip(cuts[:-1], cuts[1:])]
+    assert spans.tolist() == want
+    # one piece: the plain segmenter returns the blocks themselves
+    plain, _ = orc.segment_map(M, 2000, 8, 0)
+    assert plain.tolist() == [[a, b - a + 1] for a, b in blocks]
+
+
+def test_per_unit_segmentation_properties_on_random_maps():
+    r = np.random.default_rng(3)
+    for trial in range(20):
+        m, U, C = int(r.integers(40, 160)), int(r.choice([16, 32, 48])), int(r.integers(1, 5))
+        origin = int(r.integers(0, 200))
+        M = np.tril(r.integers(0, 3000, size=(m, m)).astype(np.int32))
+        for a in range(0, m, 11):     # some structure
+            M[a:a + 9, a:a + 9] += 5000
+        M = np.tril(M)
+        th = int(np.quantile(M[np.tril_indices(m)], 0.8))
+        spans, _ = orc.segment_map(M, th, C, 0, unit=U, origin=origin)
+        # a partition of the region whose spans never cross a unit boundary; at most 2C+1 spans per unit; a unit
+        # that lies wholly inside the region is segmented exactly like a region made of that unit alone
+        assert spans[0, 0] == 0 and (spans[1:, 0] == spans[:-1, 0] + spans[:-1, 1]).all()
+        assert spans[-1, 0] + spans[-1, 1] == m
+        per_unit = {}
+        for s0, ln in spans:
+            assert (origin + s0) // U == (origin + s0 + ln - 1) // U
+            per_unit.setdefault((origin + s0) // U, []).append([int(s0), int(ln)])
+        for u, sp in per_unit.items():
+            assert len(sp) <= 2 * C + 1
+            a, b = max(u * U - origin, 0), min((u + 1) * U - origin, m)
+            alone, _ = orc.segment_map(M[a:b, a:b], th, C, 0)
+            assert [[s0 - a, ln] for s0, ln in sp] == alone.tolist()
+    # a region inside one unit is one piece
+    M = np.tril(r.integers(0, 3000, size=(30, 30)).astype(np.int32))
+    assert orc.segment_map(M, 1500, 3, 0, unit=64, origin=70)[0].tolist() == orc.segment_map(M, 1500, 3, 0)[0].tolist()
+
+
+def test_per_unit_stream_spans_stay_inside_units_and_cover_the_context():
+    cfg = inputs.StreamConfig("pu", 1, 4, 2, 128, 1100, 200, 0, 24, 256, 4, 2, 16, 64, seed=43)
+    st = inputs.SyntheticStream(cfg)
+    U = 64
+    o = orc.OracleStream(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.chunk, cfg.window, cfg.n_sink, cfg.top_k,
+                         cfg.max_tokens, max_spans_per_region=2, unit_tokens=U, segment_per_unit=1)
+    for t0, n in st.prefill_chunks():
+        q, k, v = st.tokens(t0, n)
+        o.prefill_chunk(q[0], k[0], v[0])
+    sp = o.spans()
+    assert len(sp) > 10 and sp[0, 0] == cfg.n_sink and (sp[1:, 0] == sp[:-1, 0] + sp[:-1, 1]).all()
+    assert ((sp[:, 0] // U) == ((sp[:, 0] + sp[:, 1] - 1) // U)).all()
+    # (calls of 200 tokens: a unit that straddles two calls is segmented in two parts, each with its own cap)
+    counts = np.bincount(sp[:, 0] // U)
+    assert counts.max() <= 2 * (2 * 2 + 1)
+    with pytest.raises(ValueError):
+        orc.OracleStream(4, 2, 128, 128, 256, 16, 4, 1024, segment_per_unit=1)     # needs unit_tokens
