@@ -204,7 +204,7 @@ def oracle_sample(cfg, steps, warmup):
                          nms_iou_milli=cfg.layer_nms_iou_milli[0] if cfg.layer_nms_iou_milli else cfg.nms_iou_milli,
                          ret_head=cfg.retrieval_head[0] if cfg.retrieval_head else -1,
                          head_weight=cfg.retrieval_head_score[0] if cfg.retrieval_head_score else 1.0,
-                         collab_vote=int(cfg.collab_vote))
+                         collab_vote=int(cfg.collab_vote), segment_per_unit=int(cfg.segment_per_unit))
     times = []
     for ci in range(fill + warmup + steps):
         q, k, v = st.tokens(ci * cfg.chunk, cfg.chunk)
@@ -318,7 +318,8 @@ def run_ltri(args, cfg):
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
                             max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
                             flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
-                                  (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0),
+                                  (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0) |
+                                  (binding.FLAG_SEGMENT_PER_UNIT if cfg.segment_per_unit else 0),
                             unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
                             retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score,
                             layer_theta=cfg.layer_theta, layer_nms_iou_milli=cfg.layer_nms_iou_milli,
@@ -528,6 +529,9 @@ def main():
                     help="IoU threshold of the segmenter's NMS (0: spans never overlap; the paper lists 0.1 / 0.01)")
     ap.add_argument("--persist-decode", action="store_true",
                     help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
+    ap.add_argument("--segment-per-unit", action="store_true",
+                    help="segment every memory unit on its own, four spans kept per unit (the paper's 'Span' column); "
+                         "needs --unit-tokens")
     ap.add_argument("--layer-tables", action="store_true",
                     help="per-layer theta (quantile levels spread over 0.88..0.95), phi (0.1 / 0.01 alternating) and "
                          "lambda (20 for the first four layers, 3 after them, as in the paper's implementation "
@@ -569,6 +573,12 @@ def main():
         import dataclasses
         cfg = dataclasses.replace(cfg, persist_decode=True)
         cfg.name += "[persist-decode]"
+    if args.segment_per_unit:
+        import dataclasses
+        if args.unit_tokens <= 0:
+            ap.error("--segment-per-unit needs --unit-tokens")
+        cfg = dataclasses.replace(cfg, segment_per_unit=True, max_spans_per_region=4)
+        cfg.name += "[segment-per-unit]"
     if args.layer_tables:
         import dataclasses
         L = cfg.n_layers

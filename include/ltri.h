@@ -112,7 +112,13 @@ enum {
    * (fp32, ascending layer order) that name the unit -- then by its own score, then by lower unit number, and fetches
    * the first k.  The layers of a chunk (or decode step) must be submitted in ascending order, each layer of a
    * sequence exactly once, so that the ballots a layer reads are those of the same chunk. */
-  LTRI_FLAG_COLLAB_VOTE = 4
+  LTRI_FLAG_COLLAB_VOTE = 4,
+  /* Segmentation per memory unit (Sec. 3.3: every block is divided into spans); needs unit_tokens > 0.  The part of a
+   * call's region inside each unit of unit_tokens tokens (absolute grid) is segmented on its own: only intervals
+   * inside one unit are candidates, NMS keeps max_spans_per_region spans PER UNIT (0 -> unit_tokens/32), uncovered
+   * runs are cut at the unit boundaries; theta is still that of the whole region.  Spans never cross a unit boundary.
+   * max_spans_per_region * (units a call can touch = (chunk + unit_tokens - 2) / unit_tokens + 1) must be <= 64. */
+  LTRI_FLAG_SEGMENT_PER_UNIT = 8
 };
 
 typedef struct {
@@ -230,7 +236,8 @@ enum {
   LTRI_BUF_INDEX = 3,    /* bf16  [n_kv_heads][span_capacity][head_dim]: the span index K^R */
   LTRI_BUF_THETA = 4,    /* int64 [1]: theta of the last prefill call in Q20 head-sum units */
   LTRI_BUF_SCORES = 5,   /* float [n_kv_heads][span_capacity]: similarity scores of the last call (Eq. 7) */
-  LTRI_BUF_QREPS = 6,    /* float [n_kv_heads][2*max_spans_per_region+1][head_dim]: summed query representatives */
+  LTRI_BUF_QREPS = 6,    /* float [n_kv_heads][J][head_dim]: summed query representatives; J = 2*max_spans_per_region+1
+                            (times the units a call can touch under LTRI_FLAG_SEGMENT_PER_UNIT) */
   LTRI_BUF_NREPS = 8,    /* int32 [2*max_spans_per_region+1]: representative counts of the spans of the last prefill
                             call's region (Sec. 3.3.2) */
   LTRI_BUF_BALLOT = 9,   /* int32 [top_k]: the layer's own ballot under LTRI_FLAG_COLLAB_VOTE (ascending unit numbers,

@@ -18,6 +18,7 @@ LTRI_OK, LTRI_EINVAL, LTRI_ECAPACITY, LTRI_ESTATE, LTRI_ECUDA, LTRI_EDEVICE, LTR
 FLAG_PERSIST_DECODE = 1
 FLAG_HOST_STAGING = 2
 FLAG_COLLAB_VOTE = 4
+FLAG_SEGMENT_PER_UNIT = 8
 BUF_MAP, BUF_VOTES, BUF_INDEX, BUF_THETA, BUF_SCORES, BUF_QREPS, BUF_ROWSTAT, BUF_NREPS = 1, 2, 3, 4, 5, 6, 7, 8
 BUF_BALLOT = 9
 
@@ -324,7 +325,7 @@ class Ltri:
         if what == BUF_SCORES:
             return raw.view(np.float32).reshape(p.n_kv_heads, cap)
         if what == BUF_QREPS:
-            return raw.view(np.float32).reshape(p.n_kv_heads, 2 * C_ + 1, p.head_dim)
+            return raw.view(np.float32).reshape(p.n_kv_heads, -1, p.head_dim)
         if what in (BUF_NREPS, BUF_BALLOT):
             return raw.view(np.int32)
         if what == BUF_ROWSTAT:

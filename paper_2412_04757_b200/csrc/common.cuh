@@ -28,6 +28,7 @@ struct DevCtx {
   int rcap;              // token ranges kept per (seq, layer, KV head): 2 * top_k + 2
   int phi_milli;         // NMS IoU threshold in thousandths (0: spans never overlap)
   int unit;              // retrieval granularity: 0 = span, U > 0 = units of U tokens (Eq. 8 as printed)
+  int seg_unit;          // > 0: every unit of this many tokens is segmented on its own (C spans kept per unit)
   int persist;           // decode keeps the spans selected by the last prefill call (Sec. 3.5, persistent mechanism)
   int theta_mode;
   float theta, scale;
@@ -127,7 +128,7 @@ cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_co
 // and, when q != nullptr, the summed query representatives of every span.  theta_mode 0/2: theta_q_abs is used.
 cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_count, int m, int reg_start, int slot,
                            int theta_mode, float theta, long long theta_q_abs, int max_spans, int n, int t0,
-                           const __nv_bfloat16* q, cudaStream_t s, bool tables = false);
+                           const __nv_bfloat16* q, cudaStream_t s, bool tables = false, int seg_unit = 0);
 cudaError_t launch_score_prefill(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s);
 // tensor-core version of launch_score_prefill (split-bf16 representatives)
 cudaError_t launch_score_prefill_mma(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s);

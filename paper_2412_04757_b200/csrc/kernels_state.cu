@@ -440,7 +440,9 @@ __global__ void __launch_bounds__(256) k_seg_rowscan(DevCtx c, int layer_begin, 
 // best point of every anti-diagonal x+y=c (max S, ties -> shorter span), kept only when S > 0.
 // A CTA owns 32 columns; thread (cx, ry) scans rows [ry*R, ry*R+R) of its column, a shared-memory scan over ry
 // supplies the offsets, and a second pass emits S.  key = (S << 10) | (1023 - (y-x)).
-__global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin, int m) {
+// seg_unit > 0 (segmentation per memory unit): only intervals inside one unit of seg_unit tokens on the absolute grid
+// are candidates; `origin` is the absolute position of the region's first token.
+__global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin, int m, int seg_unit, int origin) {
   extern __shared__ long long sm[];
   long long* part = sm;             // [32 ry][32 cx]
   long long* sbest = sm + 32 * 32;  // [m + 32]
@@ -467,9 +469,11 @@ __global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin,
   __syncthreads();
   if (x < m) {
     long long S = part[ry * 32 + cx];
+    // last token of the unit that holds x (region-relative)
+    const int ymax = seg_unit > 0 ? ((origin + x) / seg_unit + 1) * seg_unit - origin - 1 : m;
     for (int y = max(ylo, x); y < yhi; ++y) {
       S += Rs[(size_t)y * c.chunk + x];
-      if (S > 0) {
+      if (S > 0 && y <= ymax) {
         const long long key = (S << 10) | (long long)(1023 - (y - x));
         atomicMax(&sbest[x + y - 2 * x0], key);
       }
@@ -502,6 +506,7 @@ struct NmsArgs {
   int n, t0;                 // query tensor geometry (q == nullptr: skip the representatives)
   const __nv_bfloat16* q;
   int tables;                // use the context's per-layer phi and lambda tables where it has them
+  int seg_unit;              // > 0: every unit of this many tokens (absolute grid) keeps max_spans spans of its own
 };
 
 __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
@@ -510,9 +515,13 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   __shared__ int kx[kMaxTopK], ky[kMaxTopK];
   __shared__ int out_start[2 * kMaxTopK + 1], out_len[2 * kMaxTopK + 1];
   __shared__ int s_nout;
+  __shared__ int s_ucnt[kMaxTopK + 2];  // segmentation per unit: spans kept in every unit the region touches
   const int layer = a.layer_begin + blockIdx.x;
   const size_t unit = unit_of(c, a.seq, layer);
   const int m = a.m;
+  const int SU = a.seg_unit;
+  auto unit_idx = [&](int x) { return (a.reg_start + x) / SU - a.reg_start / SU; };
+  const int cap_total = SU > 0 ? kMaxTopK : a.max_spans;
   const int phi_milli = a.tables && c.phi_l ? c.phi_l[layer] : c.phi_milli;
   const float rep_lambda = a.tables && c.lambda_l ? c.lambda_l[layer] : c.rep_lambda;
   const int ncand = 2 * m - 1;
@@ -548,7 +557,9 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   if (threadIdx.x < 32) {
     const int lane = threadIdx.x;
     int kept = 0;
-    for (int base = 0; base < ncand && kept < a.max_spans; base += 32) {
+    for (int t = lane; t < kMaxTopK + 2; t += 32) s_ucnt[t] = 0;
+    __syncwarp();
+    for (int base = 0; base < ncand && kept < cap_total; base += 32) {
       const int idx = base + lane;
       const long long key = idx < ncand ? skey[idx] : 0;
       const int len = 1023 - (int)(key & 1023);
@@ -557,16 +568,20 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
       bool alive = key > 0;
       if (__ballot_sync(0xffffffffu, alive) == 0) break;  // sorted: nothing positive follows
       for (int q = 0; q < kept; ++q) alive = alive && !nms_suppressed(x, y, kx[q], ky[q], phi_milli);
+      if (SU > 0) alive = alive && s_ucnt[unit_idx(x)] < a.max_spans;  // the candidate's unit still has room
       unsigned mask = __ballot_sync(0xffffffffu, alive);
-      while (mask && kept < a.max_spans) {
+      while (mask && kept < cap_total) {
         const int f = __ffs(mask) - 1;
         const int fx = __shfl_sync(0xffffffffu, x, f), fy = __shfl_sync(0xffffffffu, y, f);
         if (lane == 0) {
           kx[kept] = fx;
           ky[kept] = fy;
+          if (SU > 0) ++s_ucnt[unit_idx(fx)];
         }
         ++kept;
+        __syncwarp();
         alive = alive && lane != f && !nms_suppressed(x, y, fx, fy, phi_milli);
+        if (SU > 0) alive = alive && s_ucnt[unit_idx(x)] < a.max_spans;
         mask = __ballot_sync(0xffffffffu, alive);
       }
       __syncwarp();
@@ -590,19 +605,24 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
     __syncwarp();
     if (lane == 0) {
       int pos = 0, no = 0;
-      for (int q = 0; q < kept; ++q) {
-        if (kx[q] > pos) {
-          out_start[no] = pos;
-          out_len[no++] = kx[q] - pos;
+      // an uncovered run [g0, g1) becomes a span; under segmentation per unit it is cut at the unit boundaries
+      auto emit_gap = [&](int g0, int g1) {
+        while (g0 < g1 && no < 2 * kMaxTopK + 1) {
+          const int e = SU > 0 ? min(g1, ((a.reg_start + g0) / SU + 1) * SU - a.reg_start) : g1;
+          out_start[no] = g0;
+          out_len[no++] = e - g0;
+          g0 = e;
         }
-        out_start[no] = kx[q];
-        out_len[no++] = ky[q] - kx[q] + 1;
+      };
+      for (int q = 0; q < kept; ++q) {
+        if (kx[q] > pos) emit_gap(pos, kx[q]);
+        if (no < 2 * kMaxTopK + 1) {
+          out_start[no] = kx[q];
+          out_len[no++] = ky[q] - kx[q] + 1;
+        }
         pos = max(pos, ky[q] + 1);  // kept spans may overlap when phi > 0
       }
-      if (pos < m) {
-        out_start[no] = pos;
-        out_len[no++] = m - pos;
-      }
+      if (pos < m) emit_gap(pos, m);
       s_nout = no;
     }
   }
@@ -728,7 +748,7 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
 
 cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_count, int m, int reg_start,
                              int slot, int theta_mode, float theta, long long theta_q_abs, int max_spans, int n,
-                             int t0, const __nv_bfloat16* q, cudaStream_t s, bool tables) {
+                             int t0, const __nv_bfloat16* q, cudaStream_t s, bool tables, int seg_unit) {
   if (theta_mode == 1) {
     const long long N = (long long)m * (m + 1) / 2;
     long long rank = (long long)floor((double)theta * (double)(N - 1));
@@ -742,8 +762,8 @@ cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_
   }
   k_seg_rowscan<<<dim3((m + 7) / 8, layer_count), 256, 0, s>>>(c, layer_begin, m);
   const size_t smem = (size_t)(32 * 32 + m + 32) * sizeof(long long);
-  k_seg_colscan<<<dim3((m + 31) / 32, layer_count), 1024, smem, s>>>(c, layer_begin, m);
-  NmsArgs a{seq, layer_begin, m, reg_start, slot, max_spans, n, t0, q, tables ? 1 : 0};
+  k_seg_colscan<<<dim3((m + 31) / 32, layer_count), 1024, smem, s>>>(c, layer_begin, m, seg_unit, reg_start);
+  NmsArgs a{seq, layer_begin, m, reg_start, slot, max_spans, n, t0, q, tables ? 1 : 0, seg_unit};
   k_seg_nms<<<layer_count, 1024, 0, s>>>(c, a);
   return cudaGetLastError();
 }

@@ -57,8 +57,17 @@ bool validate(const ltri_params* p) {
   if (p->theta_mode != 0 && p->theta_mode != 1) return false;
   if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
   if (!(p->softmax_scale >= 0.f)) return false;
-  if (p->flags & ~(uint32_t)(LTRI_FLAG_PERSIST_DECODE | LTRI_FLAG_HOST_STAGING | LTRI_FLAG_COLLAB_VOTE)) return false;
+  if (p->flags & ~(uint32_t)(LTRI_FLAG_PERSIST_DECODE | LTRI_FLAG_HOST_STAGING | LTRI_FLAG_COLLAB_VOTE |
+                              LTRI_FLAG_SEGMENT_PER_UNIT))
+    return false;
   if ((p->flags & LTRI_FLAG_COLLAB_VOTE) && (p->unit_tokens == 0 || !p->retrieval_head)) return false;
+  if (p->flags & LTRI_FLAG_SEGMENT_PER_UNIT) {
+    // a call of up to `chunk` tokens touches at most this many units; their kept spans share the segmenter's arrays
+    if (p->unit_tokens == 0) return false;
+    const int nun = (p->chunk + p->unit_tokens - 2) / p->unit_tokens + 1;
+    const int cu = p->max_spans_per_region > 0 ? p->max_spans_per_region : std::max(1, p->unit_tokens / 32);
+    if (cu * nun > kMaxTopK) return false;
+  }
   if (p->retrieval_head)
     for (int l = 0; l < p->n_layers; ++l) {
       if (p->retrieval_head[l] < -1 || p->retrieval_head[l] >= p->n_q_heads) return false;
@@ -107,8 +116,11 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.persist = (p.flags & LTRI_FLAG_PERSIST_DECODE) ? 1 : 0;
   d.vote = (p.flags & LTRI_FLAG_COLLAB_VOTE) ? 1 : 0;
   d.reps = p.reps_per_span > 0 ? p.reps_per_span : 1;
-  d.C = p.max_spans_per_region > 0 ? p.max_spans_per_region : std::max(1, p.chunk / 32);
+  d.seg_unit = (p.flags & LTRI_FLAG_SEGMENT_PER_UNIT) ? p.unit_tokens : 0;
+  d.C = p.max_spans_per_region > 0 ? p.max_spans_per_region
+                                   : std::max(1, (d.seg_unit > 0 ? p.unit_tokens : p.chunk) / 32);
   d.Jmax = 2 * d.C + 1;
+  if (d.seg_unit > 0) d.Jmax *= (p.chunk + p.unit_tokens - 2) / p.unit_tokens + 1;  // every unit a call can touch
   d.slots = (p.window + p.chunk - 1) / p.chunk + 8;
   d.cap = (int)std::min<long long>((long long)1 << 30, ((p.max_tokens + p.chunk - 1) / p.chunk + 8) * d.Jmax);
   d.theta_mode = p.theta_mode;
@@ -479,7 +491,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
     long long thq_abs = 0;
     if (d.theta_mode == 0) thq_abs = (long long)std::nearbyint((double)d.theta * (double)d.Hq * (double)kQScale);
     LTRI_CUDA(ctx, launch_segment(d, seq, layer_begin, layer_count, m, reg_start, slot, d.theta_mode, d.theta, thq_abs,
-                                  d.C, n_tokens, t0, a.q, st, /*tables=*/true));
+                                  d.C, n_tokens, t0, a.q, st, /*tables=*/true, d.seg_unit));
   }
   if (has_index) {
     {

@@ -71,6 +71,7 @@ class StreamConfig:
     retrieval_head: tuple = None   # per layer: retrieval head or -1 (Sec. 3.5); None: no layer has one
     retrieval_head_score: tuple = None   # per layer: the head's score, its voting weight
     collab_vote: bool = False      # collaborative voting over the layers' ballots (Sec. 3.5; needs unit_tokens)
+    segment_per_unit: bool = False # every unit of unit_tokens tokens is segmented on its own (Sec. 3.3)
     layer_theta: tuple = None          # per-layer tables (None: the scalar holds for every layer)
     layer_nms_iou_milli: tuple = None
     layer_rep_lambda: tuple = None

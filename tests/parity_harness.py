@@ -53,7 +53,8 @@ def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
                                ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps, max_reps=cfg.max_reps,
                                rep_lambda=cfg.rep_lambda,
                                flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
-                                     (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0),
+                                     (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0) |
+                                     (binding.FLAG_SEGMENT_PER_UNIT if cfg.segment_per_unit else 0),
                                unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
                                retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score,
                                layer_theta=cfg.layer_theta, layer_nms_iou_milli=cfg.layer_nms_iou_milli,
@@ -84,7 +85,7 @@ def oracle_of(cfg: inputs.StreamConfig, layer: int = 0) -> orc.OracleStream:
                             rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
                             max_reps=cfg.max_reps, rep_lambda=lam, persist_decode=int(cfg.persist_decode),
                             unit_tokens=cfg.unit_tokens, nms_iou_milli=phi, ret_head=rh, head_weight=w,
-                            collab_vote=int(cfg.collab_vote))
+                            collab_vote=int(cfg.collab_vote), segment_per_unit=int(cfg.segment_per_unit))
 
 
 def check_output(got_bf16: torch.Tensor, ref: np.ndarray, rep: Report, what: str):
@@ -199,7 +200,8 @@ class StreamPair:
                     if cfg.theta_mode == 1:
                         assert thg == orc.theta_q(Mg, 1, theta_l, cfg.n_q_heads), f"{what}: theta rank select"
                     # integer pipeline: bit-exact on identical integer input
-                    ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region, phi_l)
+                    ref_spans, _ = orc.segment_map(Mg, thg, cfg.max_spans_per_region, phi_l,
+                                                   unit=cfg.unit_tokens if cfg.segment_per_unit else 0, origin=rs)
                     ref_spans[:, 0] += rs
                     assert newest_g.tolist() == ref_spans.tolist(), f"{what}: segmenter differs on its own map"
                 if newest_g.tolist() != spans_o.tolist():

@@ -52,7 +52,7 @@ def test_arena_sizing_is_host_only_and_monotone(lib):
     dict(rep_mode=1, rep_lambda=-1.0), dict(unit_tokens=12), dict(unit_tokens=512), dict(nms_iou_milli=1000),
     dict(retrieval_head=[8]), dict(retrieval_head=[-2]), dict(retrieval_head=[1], retrieval_head_score=[-0.5]),
     dict(flags=4, unit_tokens=64), dict(flags=4, retrieval_head=[1]),
-    dict(layer_theta=[1.5]), dict(layer_nms_iou_milli=[1000]), dict(layer_rep_lambda=[-1.0]),
+    dict(flags=8), dict(flags=8, unit_tokens=16, max_spans_per_region=4), dict(layer_theta=[1.5]), dict(layer_nms_iou_milli=[1000]), dict(layer_rep_lambda=[-1.0]),
 ])
 def test_bad_parameters_are_rejected_on_the_host(lib, kw):
     base = dict(n_layers=1, n_q_heads=8, n_kv_heads=2, max_tokens=1024, chunk=256, window=512, n_sink=64, top_k=4)

@@ -142,6 +142,18 @@ def test_per_layer_theta_phi_lambda_tables(theta_mode, thetas):
     print(rep)
 
 
+@pytest.mark.parametrize("U,C,chunk,phi", [(64, 3, 128, 0), (32, 2, 128, 0), (48, 2, 96, 0), (64, 3, 128, 300)])
+def test_segmentation_per_memory_unit(U, C, chunk, phi):
+    # Sec. 3.3: every memory unit is divided into spans on its own -- candidates inside one unit, C spans kept per
+    # unit, gaps cut at the unit boundaries; units on the absolute grid (the first region starts at the sink's end,
+    # U = 48 does not divide the calls).  The segmenter is compared bit for bit on the GPU's own map.
+    cfg = small_cfg(n_layers=2, context=1536 if chunk == 128 else 1152, chunk=chunk, decode_steps=3, unit_tokens=U,
+                    max_spans_per_region=C, segment_per_unit=True, top_k=3, nms_iou_milli=phi)
+    rep = ph.run_stream(cfg, layers=[0, 1])
+    assert rep.regions >= 20
+    print(rep)
+
+
 def test_voting_layer_by_layer_calls_match_one_call():
     # a real model submits one layer at a time: the ballots of the earlier layers of the same chunk are read from the
     # context's state and the selections must equal those of the all-layers call
