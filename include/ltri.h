@@ -95,6 +95,18 @@ typedef struct {
   const float* layer_theta;
   const int32_t* layer_nms_iou_milli;
   const float* layer_rep_lambda;
+  /* Context memory on the host (Sec. 3.4: evicted tokens live in CPU memory behind a cache of memory units on the
+   * GPU; used with LTRI_FLAG_HOST_KV, which needs unit_tokens > 0).
+   * host_kv: caller-owned HOST memory, page-locked and mapped for the device (cudaHostAlloc / cudaHostRegister /
+   * a pinned torch tensor), 256-byte aligned, ltri_host_kv_bytes(params) bytes: the K rows of every (sequence, layer,
+   * KV head) slab, then the V rows.  cache_units: memory units of unit_tokens tokens kept in device memory per
+   * (sequence, layer, KV head), top_k..128 (2 * top_k with LTRI_FLAG_PERSIST_DECODE); score_decay in [0, 1]: at every
+   * retrieval the usage score of a cached unit becomes score_decay * score (+ 1 if the retrieval names it), and a
+   * unit that has to make room is the one with the lowest score (lowest slot among equals). */
+  void* host_kv;
+  size_t host_kv_bytes;
+  int32_t cache_units;
+  float score_decay;
   void* arena;                                       /* caller-owned device memory, 256-byte aligned */
   size_t arena_bytes;                                /* >= ltri_arena_bytes(params) */
 } ltri_params;
@@ -118,7 +130,16 @@ enum {
    * inside one unit are candidates, NMS keeps max_spans_per_region spans PER UNIT (0 -> unit_tokens/32), uncovered
    * runs are cut at the unit boundaries; theta is still that of the whole region.  Spans never cross a unit boundary.
    * max_spans_per_region * (units a call can touch = (chunk + unit_tokens - 2) / unit_tokens + 1) must be <= 64. */
-  LTRI_FLAG_SEGMENT_PER_UNIT = 8
+  LTRI_FLAG_SEGMENT_PER_UNIT = 8,
+  /* Host-memory pager for retrieved tokens (Sec. 3.4, "Implementation Details": GPU cache size, score decay).  When a
+   * region leaves the window its K/V rows are also copied to host_kv (on an internal stream, overlapping the call's
+   * attention).  The retrieved units of a prefill call are then no longer read from the device-resident K/V slabs:
+   * a unit found in the (sequence, layer, KV head)'s unit cache is read from there; a missing one is pulled from
+   * host_kv over the bus by the top-k kernel itself, into the slot of the unit with the lowest usage score.  Results
+   * are bit-identical to the default path.  In this version the device slabs still hold every token (sink and local
+   * window are read from them, and so are the retrieved units of decode steps), so the flag exercises the data path of
+   * the pager but does not yet shrink the device footprint. */
+  LTRI_FLAG_HOST_KV = 16
 };
 
 typedef struct {
@@ -135,6 +156,9 @@ typedef struct {
 /* Bytes of device memory the arena must provide for these parameters (host only; the
  * `arena` and `arena_bytes` fields are ignored).  Returns 0 if the parameters are invalid. */
 size_t ltri_arena_bytes(const ltri_params* p);
+
+/* Bytes of host memory that host_kv must provide under LTRI_FLAG_HOST_KV (0 if the parameters are invalid). */
+size_t ltri_host_kv_bytes(const ltri_params* p);
 
 /* Create a context over the caller's arena and initialise its device state on
  * `cuda_stream` (synchronises that stream once).  Streaming attention with parameters
@@ -240,6 +264,9 @@ enum {
                             (times the units a call can touch under LTRI_FLAG_SEGMENT_PER_UNIT) */
   LTRI_BUF_NREPS = 8,    /* int32 [2*max_spans_per_region+1]: representative counts of the spans of the last prefill
                             call's region (Sec. 3.3.2) */
+  LTRI_BUF_CACHE_TAGS = 10,   /* int32 [n_kv_heads][cache_units]: unit held by every slot of the unit cache, -1 empty */
+  LTRI_BUF_CACHE_SCORES = 11, /* float [n_kv_heads][cache_units]: usage scores of the slots */
+  LTRI_BUF_CACHE_STATS = 12,  /* int64 [2]: units found in the cache / pulled from the host so far (all KV heads) */
   LTRI_BUF_BALLOT = 9,   /* int32 [top_k]: the layer's own ballot under LTRI_FLAG_COLLAB_VOTE (ascending unit numbers,
                             -1 padded; all -1 for a layer without a retrieval head) */
   LTRI_BUF_ROWSTAT = 7   /* float [chunk][n_q_heads][2]: reference maximum m (logits * scale * log2(e); may lag the true

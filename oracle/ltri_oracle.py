@@ -416,3 +416,43 @@ def top_k(score: np.ndarray, k: int):
 
 def f32_to_bf16(x: float) -> int:
     return int(lib().orc_f32_to_bf16(C.c_float(x)))
+
+
+class UnitCachePolicy:
+    """Which memory units a device-side cache of `capacity` units holds (Sec. 3.4; "GPU cache size" and "score decay
+    coefficient" of the implementation details), as this build reads it: at every retrieval the usage score of every
+    slot is multiplied by `decay`; a unit the retrieval names that is in the cache gains 1; a named unit that is not
+    takes the slot with the lowest score among the slots not named by this retrieval (lowest slot among equals) and
+    starts at 1.  Scores are fp32, one rounding per operation.  Results of attention never depend on it.
+    """
+
+    def __init__(self, capacity: int, decay: float):
+        self.decay = np.float32(decay)
+        self.tags = np.full(capacity, -1, dtype=np.int32)
+        self.scores = np.zeros(capacity, dtype=np.float32)
+        self.hits = 0
+        self.misses = 0
+
+    def access(self, units):
+        """One retrieval naming `units` (distinct, ascending).  Returns the units that had to be fetched."""
+        self.scores = (self.scores * self.decay).astype(np.float32)
+        named = np.zeros(len(self.tags), dtype=bool)
+        missing = []
+        for u in units:
+            where = np.nonzero(self.tags == u)[0]
+            if len(where):
+                named[where[0]] = True
+                self.scores[where[0]] = np.float32(self.scores[where[0]] + np.float32(1.0))
+                self.hits += 1
+            else:
+                missing.append(int(u))
+        for u in missing:
+            free = np.nonzero(~named)[0]
+            if len(free) == 0:
+                raise ValueError("more units named at once than the cache holds")
+            victim = free[np.argmin(self.scores[free])]      # the first minimum: lowest slot among equals
+            self.tags[victim] = u
+            self.scores[victim] = np.float32(1.0)
+            named[victim] = True
+            self.misses += 1
+        return missing

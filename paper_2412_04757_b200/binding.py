@@ -19,15 +19,17 @@ FLAG_PERSIST_DECODE = 1
 FLAG_HOST_STAGING = 2
 FLAG_COLLAB_VOTE = 4
 FLAG_SEGMENT_PER_UNIT = 8
+FLAG_HOST_KV = 16
 BUF_MAP, BUF_VOTES, BUF_INDEX, BUF_THETA, BUF_SCORES, BUF_QREPS, BUF_ROWSTAT, BUF_NREPS = 1, 2, 3, 4, 5, 6, 7, 8
 BUF_BALLOT = 9
+BUF_CACHE_TAGS, BUF_CACHE_SCORES, BUF_CACHE_STATS = 10, 11, 12
 
 EXPORTS = [
     "ltri_arena_bytes", "ltri_create", "ltri_destroy", "ltri_reset_sequence", "ltri_prefill_chunk",
     "ltri_decode_step", "ltri_get_spans", "ltri_get_pending_spans", "ltri_get_selected", "ltri_get_stats",
     "ltri_sync_status", "ltri_last_cuda_error", "ltri_strerror", "ltri_debug_read", "ltri_span_capacity",
     "ltri_debug_segment_map", "ltri_launch_count", "ltri_profile_enable", "ltri_profile_read",
-    "ltri_segment_map_static", "ltri_prefill_chunk_host", "ltri_host_outputs_ready",
+    "ltri_segment_map_static", "ltri_prefill_chunk_host", "ltri_host_outputs_ready", "ltri_host_kv_bytes",
 ]
 KERNEL_CLASSES = ["append", "evict_index", "attn_local", "map_pass", "segment", "score_topk", "attn_retrieved",
                   "decode_retrieve", "decode_attn"]
@@ -45,6 +47,7 @@ class LtriParams(C.Structure):
         ("retrieval_head", C.POINTER(C.c_int32)), ("retrieval_head_score", C.POINTER(C.c_float)),
         ("layer_theta", C.POINTER(C.c_float)), ("layer_nms_iou_milli", C.POINTER(C.c_int32)),
         ("layer_rep_lambda", C.POINTER(C.c_float)),
+        ("host_kv", C.c_void_p), ("host_kv_bytes", C.c_size_t), ("cache_units", C.c_int32), ("score_decay", C.c_float),
         ("arena", C.c_void_p), ("arena_bytes", C.c_size_t),
     ]
 
@@ -76,6 +79,8 @@ def load():
         vp, ip = C.c_void_p, C.c_int
         L.ltri_arena_bytes.restype = C.c_size_t
         L.ltri_arena_bytes.argtypes = [C.POINTER(LtriParams)]
+        L.ltri_host_kv_bytes.restype = C.c_size_t
+        L.ltri_host_kv_bytes.argtypes = [C.POINTER(LtriParams)]
         L.ltri_create.argtypes = [C.POINTER(LtriParams), vp, C.POINTER(vp)]
         L.ltri_destroy.argtypes = [vp]
         L.ltri_reset_sequence.argtypes = [vp, ip, vp]
@@ -111,13 +116,13 @@ def make_params(n_layers, n_q_heads, n_kv_heads, max_tokens, chunk, window, n_si
                 reps_per_span=1, max_spans_per_region=0, theta_mode=1, theta=0.90, softmax_scale=0.0,
                 rep_mode=0, ratio_kind=2, min_reps=1, max_reps=4, rep_lambda=2.0, flags=0, unit_tokens=0, nms_iou_milli=0,
                 retrieval_head=None, retrieval_head_score=None, layer_theta=None, layer_nms_iou_milli=None,
-                layer_rep_lambda=None) -> LtriParams:
+                layer_rep_lambda=None, cache_units=0, score_decay=0.1) -> LtriParams:
     """retrieval_head / retrieval_head_score (head or -1; weight) and layer_theta / layer_nms_iou_milli /
     layer_rep_lambda: per-layer sequences, marshalled into host arrays that live as long as the returned struct."""
     p = LtriParams(n_layers, n_q_heads, n_kv_heads, head_dim, max_seqs, max_tokens, chunk, window, n_sink, top_k,
                    reps_per_span, max_spans_per_region, theta_mode, theta, softmax_scale, flags,
                    rep_mode, ratio_kind, min_reps, max_reps, rep_lambda, unit_tokens, nms_iou_milli, None, None, None, None,
-                   None, None, 0)
+                   None, None, 0, cache_units, score_decay, None, 0)
     if retrieval_head is not None:
         if len(retrieval_head) != n_layers:
             raise ValueError("retrieval_head needs one entry per layer")
@@ -142,6 +147,10 @@ def make_params(n_layers, n_q_heads, n_kv_heads, max_tokens, chunk, window, n_si
 
 def ltri_arena_bytes(params: LtriParams) -> int:
     return int(load().ltri_arena_bytes(C.byref(params)))
+
+
+def ltri_host_kv_bytes(params: LtriParams) -> int:
+    return int(load().ltri_host_kv_bytes(C.byref(params)))
 
 
 def _check(rc: int, where: str):
@@ -189,6 +198,12 @@ class Ltri:
         self._params_src = params   # owns the host arrays the copy points to
         self.params.arena = base
         self.params.arena_bytes = nbytes
+        if params.flags & FLAG_HOST_KV and not params.host_kv:
+            # the host mirror of the pager: pinned (page-locked, device-mapped) memory from torch
+            hb = ltri_host_kv_bytes(params)
+            self.host_kv = torch.empty(hb + 256, dtype=torch.uint8, pin_memory=True)
+            self.params.host_kv = (self.host_kv.data_ptr() + 255) // 256 * 256
+            self.params.host_kv_bytes = hb
         self.arena_bytes = nbytes
         self._h = C.c_void_p()
         with torch.cuda.device(self.device):
@@ -328,6 +343,12 @@ class Ltri:
             return raw.view(np.float32).reshape(p.n_kv_heads, -1, p.head_dim)
         if what in (BUF_NREPS, BUF_BALLOT):
             return raw.view(np.int32)
+        if what == BUF_CACHE_TAGS:
+            return raw.view(np.int32).reshape(p.n_kv_heads, -1)
+        if what == BUF_CACHE_SCORES:
+            return raw.view(np.float32).reshape(p.n_kv_heads, -1)
+        if what == BUF_CACHE_STATS:
+            return raw.view(np.int64)
         if what == BUF_ROWSTAT:
             return raw.view(np.float32).reshape(p.chunk, p.n_q_heads, 2)
         return raw

@@ -53,6 +53,17 @@ struct DevCtx {
   const int* ret_head;   // [NL]  retrieval head of the layer, -1 none; nullptr: no layer has one
   const float* head_w;   // [NL]  its score = the weight of the layer's ballot
   int* ballot;           // [NS][NL][topk]  own top-k units of a layer with a retrieval head (ascending, -1 padded)
+  // host-memory pager (Sec. 3.4): evicted rows mirrored in mapped host memory, unit cache in device memory
+  int host_kv;                  // 1: retrieved units of prefill calls come from the unit cache / the host mirror
+  int cache_units;              // slots per (seq, layer, KV head)
+  float score_decay;
+  const __nv_bfloat16* hostK;   // [NS][NL][Hkv][Tpad][128] in mapped host memory (device-visible address)
+  const __nv_bfloat16* hostV;
+  __nv_bfloat16* Kcache;        // [NS][NL][Hkv][cache_units][unit][128]
+  __nv_bfloat16* Vcache;
+  int* ctag;                    // [NS][NL][Hkv][cache_units]  unit held by the slot, -1 empty
+  float* cscore;                // [NS][NL][Hkv][cache_units]  usage score
+  unsigned long long* cstat;    // [NS][NL][2]  hits, misses
   // per-layer tables of the paper's configuration appendix (nullptr: the scalar holds for every layer)
   const float* theta_l;  // [NL]  theta
   const int* phi_l;      // [NL]  NMS IoU threshold in thousandths

@@ -25,6 +25,14 @@ __global__ void k_init(DevCtx c, int seq) {
     }
     for (size_t i = tid; i < (size_t)c.NL * c.Hkv; i += stride) c.rng_cnt[u0 * c.Hkv + i] = 0;
     for (size_t i = tid; i < (size_t)c.NL * c.topk; i += stride) c.ballot[u0 * c.topk + i] = -1;
+    if (c.host_kv) {  // empty unit caches
+      const size_t nslot = (size_t)c.NL * c.Hkv * c.cache_units;
+      for (size_t i = tid; i < nslot; i += stride) {
+        c.ctag[u0 * c.Hkv * c.cache_units + i] = -1;
+        c.cscore[u0 * c.Hkv * c.cache_units + i] = 0.f;
+      }
+      for (size_t i = tid; i < (size_t)c.NL * 2; i += stride) c.cstat[u0 * 2 + i] = 0ull;
+    }
   }
   if (seq < 0 && tid < 4) c.status[tid] = 0;
   if (seq < 0)
@@ -1165,7 +1173,112 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
       c.rng_len[rb + t] = s_rl[t];
     }
   }
-  if (!DECODE) {
+  if (!DECODE && c.host_kv) {
+    // Host-memory pager (Sec. 3.4).  The selected units are looked up in this (sequence, layer, KV head)'s unit
+    // cache; every slot's usage score decays, a unit named now gains 1; a missing unit takes the slot with the
+    // lowest score among the slots not named now (lowest slot among equals) and its rows are pulled from the host
+    // mirror.  Only whole units are cached: the unit the indexed range ends in, while it is still growing, is read
+    // from the mirror every time.  s_src[t]: slot of selected unit t, -1 = straight from the host.
+    __shared__ int s_tag[128], s_src[2 * kMaxTopK], s_fill[2 * kMaxTopK];
+    __shared__ float s_sco[128];
+    __shared__ unsigned char s_named[128];
+    const int CU = c.cache_units;
+    const size_t cb = (unit * c.Hkv + g) * (size_t)CU;
+    if (tid < CU) {
+      s_tag[tid] = c.ctag[cb + tid];
+      s_sco[tid] = __fmul_rn(c.cscore[cb + tid], c.score_decay);
+      s_named[tid] = 0;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long hits = 0, misses = 0;
+      for (int t = 0; t < nall; ++t) {  // first the units that are there, so that none of them is pushed out
+        const int id = ids_all[t];
+        s_src[t] = -1;
+        s_fill[t] = 0;
+        if ((id + 1) * U > Eend) continue;  // still growing: not cached
+        for (int sl = 0; sl < CU; ++sl)
+          if (s_tag[sl] == id) {
+            s_src[t] = sl;
+            s_named[sl] = 1;
+            s_sco[sl] = __fadd_rn(s_sco[sl], 1.f);
+            ++hits;
+            break;
+          }
+      }
+      for (int t = 0; t < nall; ++t) {
+        const int id = ids_all[t];
+        if ((id + 1) * U > Eend || s_src[t] >= 0) continue;
+        int victim = -1;
+        for (int sl = 0; sl < CU; ++sl)
+          if (!s_named[sl] && (victim < 0 || s_sco[sl] < s_sco[victim])) victim = sl;
+        if (victim < 0) continue;  // (cannot happen: cache_units >= the units one retrieval names)
+        s_tag[victim] = id;
+        s_sco[victim] = 1.f;
+        s_named[victim] = 1;
+        s_src[t] = victim;
+        s_fill[t] = 1;
+        ++misses;
+      }
+      atomicAdd(&c.cstat[unit * 2], hits);
+      atomicAdd(&c.cstat[unit * 2 + 1], misses);
+    }
+    __syncthreads();
+    if (tid < CU) {
+      c.ctag[cb + tid] = s_tag[tid];
+      c.cscore[cb + tid] = s_sco[tid];
+    }
+    // pull the missing units: the unit's valid rows [s_sst, s_sst + s_sln) go to the same row offsets of its slot
+    const size_t hslab = (unit * c.Hkv + g) * (size_t)c.Tpad;
+    for (int t = 0; t < nall; ++t) {
+      if (!s_fill[t]) continue;
+      const int st = s_sst[t], ln = s_sln[t];
+      const size_t drow = (cb + s_src[t]) * (size_t)U + (st - ids_all[t] * U);
+      const uint4* hk = reinterpret_cast<const uint4*>(c.hostK + (hslab + st) * kD);
+      const uint4* hv = reinterpret_cast<const uint4*>(c.hostV + (hslab + st) * kD);
+      uint4* dk = reinterpret_cast<uint4*>(c.Kcache + drow * kD);
+      uint4* dv = reinterpret_cast<uint4*>(c.Vcache + drow * kD);
+      for (int i = tid; i < ln * 16; i += nt) {
+        dk[i] = hk[i];
+        dv[i] = hv[i];
+      }
+    }
+    __syncthreads();  // the gather below reads what this CTA just wrote
+    // a5 gather, from the unit cache (or the host mirror) instead of the device slabs
+    const int nr = s_nr, R = s_pre[nr], Rz = (R + 7) & ~7;
+    const size_t gslab = ((size_t)layer * c.Hkv + g) * (size_t)c.Rcap;
+    uint4* Kdst = reinterpret_cast<uint4*>(c.Kg + gslab * kD);
+    uint4* Vdst = reinterpret_cast<uint4*>(c.Vg + gslab * kD);
+    const int ch = tid & 15, rpp = nt >> 4;
+    for (int r = tid >> 4; r < Rz; r += rpp) {
+      uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
+      if (r < R) {
+        int lo = 0, hi = nr - 1;  // last range whose first packed row is <= r
+        while (lo < hi) {
+          const int mid = (lo + hi + 1) >> 1;
+          if (s_pre[mid] <= r) lo = mid; else hi = mid - 1;
+        }
+        const int tok = s_rs[lo] + (r - s_pre[lo]);
+        const int uid = tok / U;
+        int a0 = 0, a1 = nall - 1;  // the selected unit (ascending ids) that holds the token
+        while (a0 < a1) {
+          const int mid = (a0 + a1) >> 1;
+          if (ids_all[mid] < uid) a0 = mid + 1; else a1 = mid;
+        }
+        const int sl = s_src[a0];
+        if (sl >= 0) {
+          const size_t row = (cb + sl) * (size_t)U + (tok - uid * U);
+          kv = *(reinterpret_cast<const uint4*>(c.Kcache + row * kD) + ch);
+          vv = *(reinterpret_cast<const uint4*>(c.Vcache + row * kD) + ch);
+        } else {
+          kv = *(reinterpret_cast<const uint4*>(c.hostK + (hslab + tok) * kD) + ch);
+          vv = *(reinterpret_cast<const uint4*>(c.hostV + (hslab + tok) * kD) + ch);
+        }
+      }
+      Kdst[(size_t)r * 16 + ch] = kv;
+      Vdst[(size_t)r * 16 + ch] = vv;
+    }
+  } else if (!DECODE) {
     // a5 gather: pack the K and V rows of the selected spans into one contiguous slab per (layer, KV head), so the
     // attention kernel that continues over them reads whole 128-row tiles.  16 threads per 256-byte row, four rows
     // of K and of V in flight per thread; the rows up to the next multiple of 8 are zero-filled.

@@ -58,9 +58,15 @@ bool validate(const ltri_params* p) {
   if (!(p->theta >= 0.f) || (p->theta_mode == 1 && p->theta > 1.f)) return false;
   if (!(p->softmax_scale >= 0.f)) return false;
   if (p->flags & ~(uint32_t)(LTRI_FLAG_PERSIST_DECODE | LTRI_FLAG_HOST_STAGING | LTRI_FLAG_COLLAB_VOTE |
-                              LTRI_FLAG_SEGMENT_PER_UNIT))
+                              LTRI_FLAG_SEGMENT_PER_UNIT | LTRI_FLAG_HOST_KV))
     return false;
   if ((p->flags & LTRI_FLAG_COLLAB_VOTE) && (p->unit_tokens == 0 || !p->retrieval_head)) return false;
+  if (p->flags & LTRI_FLAG_HOST_KV) {
+    if (p->unit_tokens == 0) return false;
+    const int need = p->top_k * ((p->flags & LTRI_FLAG_PERSIST_DECODE) ? 2 : 1);
+    if (p->cache_units < need || p->cache_units > 128) return false;
+    if (!(p->score_decay >= 0.f && p->score_decay <= 1.f)) return false;
+  }
   if (p->flags & LTRI_FLAG_SEGMENT_PER_UNIT) {
     // a call of up to `chunk` tokens touches at most this many units; their kept spans share the segmenter's arrays
     if (p->unit_tokens == 0) return false;
@@ -135,8 +141,17 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / std::sqrt((float)kD);
   const size_t units = (size_t)d.NS * d.NL;
   Carver cv{base};
+  d.host_kv = (p.flags & LTRI_FLAG_HOST_KV) ? 1 : 0;
+  d.cache_units = d.host_kv ? p.cache_units : 0;
+  d.score_decay = p.score_decay;
+  const size_t cache_rows = d.host_kv ? units * d.Hkv * (size_t)d.cache_units * p.unit_tokens : 0;
   d.Kc = cv.take<__nv_bfloat16>(units * d.Hkv * d.Tpad * kD);
   d.Vc = cv.take<__nv_bfloat16>(units * d.Hkv * d.Tpad * kD);
+  d.Kcache = cv.take<__nv_bfloat16>(cache_rows * kD);
+  d.Vcache = cv.take<__nv_bfloat16>(cache_rows * kD);
+  d.ctag = cv.take<int>(d.host_kv ? units * d.Hkv * d.cache_units : 0);
+  d.cscore = cv.take<float>(d.host_kv ? units * d.Hkv * d.cache_units : 0);
+  d.cstat = cv.take<unsigned long long>(d.host_kv ? units * 2 : 0);
   d.votes = cv.take<long long>(units * d.Tpad);
   d.span_start = cv.take<int>(units * d.cap);
   d.span_len = cv.take<int>(units * d.cap);
@@ -213,6 +228,10 @@ struct ltri_ctx {
   static constexpr int kHostGroups = 4;
   char* stage[2] = {nullptr, nullptr};   // per set: q | k | v | out of one call, [NL][chunk][H][128] bf16 each
   cudaStream_t s_up = nullptr, s_down = nullptr;
+  // host-memory pager: evicted rows are mirrored to the host on their own stream
+  cudaStream_t s_spill = nullptr;
+  cudaEvent_t ev_pre = nullptr, ev_spill = nullptr;
+  char* host_kv = nullptr;   // the caller's mirror (host address)
   cudaEvent_t ev_up[2][kHostGroups] = {}, ev_run[2][kHostGroups] = {}, ev_down[2][kHostGroups] = {};
   bool set_used[2] = {false, false};
   long long host_calls = 0;
@@ -279,6 +298,13 @@ struct Scope {
 
 extern "C" {
 
+size_t ltri_host_kv_bytes(const ltri_params* p) {
+  if (!validate(p) || !(p->flags & LTRI_FLAG_HOST_KV)) return 0;
+  DevCtx d;
+  layout(*p, d, nullptr);
+  return (size_t)d.NS * d.NL * d.Hkv * (size_t)d.Tpad * kD * sizeof(__nv_bfloat16) * 2;
+}
+
 size_t ltri_arena_bytes(const ltri_params* p) {
   if (!validate(p)) return 0;
   DevCtx d;
@@ -293,10 +319,40 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
   DevCtx d;
   const size_t need = layout(*p, d, nullptr);
   if (p->arena_bytes < need) return LTRI_ECAPACITY;
+  const __nv_bfloat16* host_dev = nullptr;
+  if (p->flags & LTRI_FLAG_HOST_KV) {
+    // the mirror must be page-locked host memory that kernels can read; checked here, on the host, so that a wrong
+    // pointer is an error code and never a device fault
+    if (!p->host_kv || (reinterpret_cast<uintptr_t>(p->host_kv) & 255)) return LTRI_EINVAL;
+    if (p->host_kv_bytes < ltri_host_kv_bytes(p)) return LTRI_ECAPACITY;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, p->host_kv) != cudaSuccess || attr.type != cudaMemoryTypeHost) {
+      cudaGetLastError();
+      return LTRI_EINVAL;
+    }
+    void* dp = nullptr;
+    if (cudaHostGetDevicePointer(&dp, p->host_kv, 0) != cudaSuccess || !dp) {
+      cudaGetLastError();
+      return LTRI_EINVAL;
+    }
+    host_dev = static_cast<const __nv_bfloat16*>(dp);
+  }
   ltri_ctx* ctx = new (std::nothrow) ltri_ctx();
   if (!ctx) return LTRI_ECAPACITY;
   ctx->p = *p;
   layout(*p, ctx->d, static_cast<char*>(p->arena), ctx->stage);
+  if (host_dev) {
+    const size_t half = (size_t)ctx->d.NS * ctx->d.NL * ctx->d.Hkv * (size_t)ctx->d.Tpad * kD;
+    ctx->d.hostK = host_dev;
+    ctx->d.hostV = host_dev + half;
+    ctx->host_kv = static_cast<char*>(p->host_kv);
+    if (cudaStreamCreateWithFlags(&ctx->s_spill, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_pre, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_spill, cudaEventDisableTiming) != cudaSuccess) {
+      ltri_destroy(ctx);
+      return LTRI_ECUDA;
+    }
+  }
   if (p->retrieval_head) {  // the caller's arrays are read now and not kept
     ctx->ret_head.assign(p->retrieval_head, p->retrieval_head + p->n_layers);
     ctx->head_w.assign((size_t)p->n_layers, 1.0f);
@@ -341,6 +397,11 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
     return LTRI_EINVAL;
   }
   cudaError_t e = cudaMemsetAsync(ctx->d.Kc, 0, kv_bytes, s);
+  if (e == cudaSuccess && ctx->d.host_kv)  // (the two unit caches are adjacent)
+    e = cudaMemsetAsync(ctx->d.Kcache, 0,
+                        (size_t)ctx->d.NS * ctx->d.NL * ctx->d.Hkv * ctx->d.cache_units * (size_t)ctx->d.unit * kD * 2 *
+                            sizeof(__nv_bfloat16),
+                        s);
   if (e == cudaSuccess && !ctx->ret_head.empty()) {
     e = cudaMemcpyAsync(const_cast<int*>(ctx->d.ret_head), ctx->ret_head.data(), ctx->ret_head.size() * sizeof(int),
                         cudaMemcpyHostToDevice, s);
@@ -375,6 +436,12 @@ int ltri_destroy(ltri_ctx* ctx) {
     cudaStreamSynchronize(ctx->s_down);
     cudaStreamDestroy(ctx->s_down);
   }
+  if (ctx->s_spill) {  // copies into the caller's host mirror may still be in flight
+    cudaStreamSynchronize(ctx->s_spill);
+    cudaStreamDestroy(ctx->s_spill);
+  }
+  if (ctx->ev_pre) cudaEventDestroy(ctx->ev_pre);
+  if (ctx->ev_spill) cudaEventDestroy(ctx->ev_spill);
   for (int s = 0; s < 2; ++s)
     for (int g = 0; g < ltri_ctx::kHostGroups; ++g) {
       if (ctx->ev_up[s][g]) cudaEventDestroy(ctx->ev_up[s][g]);
@@ -475,6 +542,25 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
     for (int j = 0; j < ea.nslots; ++j) ea.slot[j] = ev[i + j].slot;
     LTRI_CUDA(ctx, launch_evict_index(d, ea, layer_count, st));
   }
+  if (d.host_kv && !ev.empty()) {
+    // mirror the rows that just left the window to the host: one strided copy for K and one for V per region (the
+    // slabs of consecutive (layer, KV head) pairs are Tpad rows apart on both sides), on the spill stream, behind
+    // everything submitted before this call (the rows were appended by earlier calls); the top-k kernel, which may
+    // pull them back, waits for the copies
+    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_pre, st));
+    LTRI_CUDA(ctx, cudaStreamWaitEvent(ctx->s_spill, ctx->ev_pre, 0));
+    const size_t half = (size_t)d.NS * d.NL * d.Hkv * (size_t)d.Tpad * kD * sizeof(__nv_bfloat16);
+    const size_t pitch = (size_t)d.Tpad * kD * sizeof(__nv_bfloat16);
+    for (const Region& r : ev) {
+      const size_t off = ((unit_of(d, seq, layer_begin) * d.Hkv) * (size_t)d.Tpad + r.start) * kD * sizeof(__nv_bfloat16);
+      const size_t width = (size_t)(r.end - r.start) * kD * sizeof(__nv_bfloat16);
+      LTRI_CUDA(ctx, cudaMemcpy2DAsync(ctx->host_kv + off, pitch, reinterpret_cast<const char*>(d.Kc) + off, pitch, width,
+                                       (size_t)layer_count * d.Hkv, cudaMemcpyDeviceToHost, ctx->s_spill));
+      LTRI_CUDA(ctx, cudaMemcpy2DAsync(ctx->host_kv + half + off, pitch, reinterpret_cast<const char*>(d.Vc) + off, pitch,
+                                       width, (size_t)layer_count * d.Hkv, cudaMemcpyDeviceToHost, ctx->s_spill));
+    }
+    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_spill, ctx->s_spill));
+  }
   const bool has_index = ub > 0;
   {
     Scope sc(ctx, st, LTRI_K_ATTN_LOCAL, 1);
@@ -502,6 +588,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
         LTRI_CUDA(ctx, launch_score_prefill_mma(d, a, (int)ub, st));
       else
         LTRI_CUDA(ctx, launch_score_prefill(d, a, (int)ub, st));
+      if (d.host_kv && !ev.empty()) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_spill, 0));
       LTRI_CUDA(ctx, launch_topk_prefill(d, a, st));
     }
     Scope sc(ctx, st, LTRI_K_ATTN_RET, 1);
@@ -865,6 +952,21 @@ int ltri_debug_read(ltri_ctx* ctx, int what, int seq, int layer, void* dst, size
     case LTRI_BUF_NREPS:
       src = d.nrep_last + (size_t)layer * d.Jmax;
       bytes = (size_t)d.Jmax * sizeof(int);
+      break;
+    case LTRI_BUF_CACHE_TAGS:
+      if (!d.host_kv) return LTRI_ESTATE;
+      src = d.ctag + unit_of(d, seq, layer) * d.Hkv * d.cache_units;
+      bytes = (size_t)d.Hkv * d.cache_units * sizeof(int);
+      break;
+    case LTRI_BUF_CACHE_SCORES:
+      if (!d.host_kv) return LTRI_ESTATE;
+      src = d.cscore + unit_of(d, seq, layer) * d.Hkv * d.cache_units;
+      bytes = (size_t)d.Hkv * d.cache_units * sizeof(float);
+      break;
+    case LTRI_BUF_CACHE_STATS:
+      if (!d.host_kv) return LTRI_ESTATE;
+      src = d.cstat + unit_of(d, seq, layer) * 2;
+      bytes = 2 * sizeof(unsigned long long);
       break;
     case LTRI_BUF_BALLOT:
       src = d.ballot + unit_of(d, seq, layer) * d.topk;

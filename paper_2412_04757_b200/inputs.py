@@ -72,6 +72,9 @@ class StreamConfig:
     retrieval_head_score: tuple = None   # per layer: the head's score, its voting weight
     collab_vote: bool = False      # collaborative voting over the layers' ballots (Sec. 3.5; needs unit_tokens)
     segment_per_unit: bool = False # every unit of unit_tokens tokens is segmented on its own (Sec. 3.3)
+    host_kv: bool = False          # host-memory pager for retrieved units (Sec. 3.4), with a unit cache of
+    cache_units: int = 0           # this many units per (seq, layer, KV head) and
+    score_decay: float = 0.1       # this decay of the usage scores
     layer_theta: tuple = None          # per-layer tables (None: the scalar holds for every layer)
     layer_nms_iou_milli: tuple = None
     layer_rep_lambda: tuple = None

@@ -43,6 +43,8 @@ class Report:
     rep_counts: int = 0
     rep_count_flips: int = 0
     vote_changes: int = 0   # selections that the ballots of other layers changed (collaborative voting)
+    cache_hits: int = 0     # host-memory pager: units found in / fetched into the unit caches (last checked layer)
+    cache_misses: int = 0
 
 
 def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
@@ -54,7 +56,9 @@ def params_of(cfg: inputs.StreamConfig, max_seqs=None) -> binding.LtriParams:
                                rep_lambda=cfg.rep_lambda,
                                flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
                                      (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0) |
-                                     (binding.FLAG_SEGMENT_PER_UNIT if cfg.segment_per_unit else 0),
+                                     (binding.FLAG_SEGMENT_PER_UNIT if cfg.segment_per_unit else 0) |
+                                     (binding.FLAG_HOST_KV if cfg.host_kv else 0),
+                               cache_units=cfg.cache_units, score_decay=cfg.score_decay,
                                unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
                                retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score,
                                layer_theta=cfg.layer_theta, layer_nms_iou_milli=cfg.layer_nms_iou_milli,
@@ -159,6 +163,9 @@ class StreamPair:
         self.rep = Report()
         self.n_indexed = {(s, l): 0 for s in self.seqs for l in self.layers}
         self.count_of = {}   # (seq, layer, span start) -> representative count decided when its region was current
+        # host-memory pager: the oracle's model of every (seq, layer, KV head) unit cache
+        self.cache = {(s, l, g): orc.UnitCachePolicy(cfg.cache_units, cfg.score_decay)
+                      for s in self.seqs for l in self.layers for g in range(cfg.n_kv_heads)} if cfg.host_kv else {}
 
     # ---- one prefill call -------------------------------------------------------------------
     def prefill(self, seq, q, k, v, check_out=True):
@@ -253,9 +260,31 @@ class StreamPair:
                     self._vote(seq, layer, o, ballots, what)
                     self._count_vote_changes(o)
                 check_selection(lt.ltri_get_selected(seq, layer), o, rep, what, voted=cfg.collab_vote)
+                if cfg.host_kv:
+                    self._check_cache(seq, layer, o, what)
             if check_out:
                 check_output(out[layer], o.prefill_attend(), rep, what)
         return out
+
+    def _check_cache(self, seq, layer, o, what):
+        """Host-memory pager: the unit cache of every KV head holds what the policy model says after this retrieval
+        (fed with the units the call fetched; the unit the indexed range ends in is cached only once it is whole)."""
+        cfg, lt = self.cfg, self.lt
+        U, E = cfg.unit_tokens, o.evicted_end
+        sel = o.selected()[0]          # equal to the GPU's as a set (adopted where a near tie flipped a pick)
+        tags = lt.ltri_debug_read(binding.BUF_CACHE_TAGS, seq, layer)
+        scores = lt.ltri_debug_read(binding.BUF_CACHE_SCORES, seq, layer)
+        hits = misses = 0
+        for g in range(cfg.n_kv_heads):
+            pol = self.cache[(seq, layer, g)]
+            pol.access(sorted(int(u) for u in sel[g] if u >= 0 and (u + 1) * U <= E))
+            assert tags[g].tolist() == pol.tags.tolist(), f"{what}: unit cache of KV head {g} holds other units"
+            assert np.array_equal(scores[g], pol.scores), f"{what}: usage scores of KV head {g}"
+            hits += pol.hits
+            misses += pol.misses
+        st = lt.ltri_debug_read(binding.BUF_CACHE_STATS, seq, layer)
+        assert (int(st[0]), int(st[1])) == (hits, misses), f"{what}: cache hits/misses {st.tolist()} vs {(hits, misses)}"
+        self.rep.cache_hits, self.rep.cache_misses = hits, misses
 
     def _vote(self, seq, layer, o, ballots, what):
         """Collaborative voting (Sec. 3.5): compare the layer's own ballot, let the oracle adopt a tolerated pick and

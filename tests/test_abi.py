@@ -31,8 +31,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_struct_sizes_match_header(lib):
-    # the C struct has 23 int32/float fields, one int64, six pointers and a size_t with natural alignment
-    assert ctypes.sizeof(binding.LtriParams) == 160
+    # the C struct has 25 int32/float fields, one int64, seven pointers and two size_t with natural alignment
+    assert ctypes.sizeof(binding.LtriParams) == 184
     assert ctypes.sizeof(binding.LtriStats) == 48
 
 
@@ -52,7 +52,10 @@ def test_arena_sizing_is_host_only_and_monotone(lib):
     dict(rep_mode=1, rep_lambda=-1.0), dict(unit_tokens=12), dict(unit_tokens=512), dict(nms_iou_milli=1000),
     dict(retrieval_head=[8]), dict(retrieval_head=[-2]), dict(retrieval_head=[1], retrieval_head_score=[-0.5]),
     dict(flags=4, unit_tokens=64), dict(flags=4, retrieval_head=[1]),
-    dict(flags=8), dict(flags=8, unit_tokens=16, max_spans_per_region=4), dict(layer_theta=[1.5]), dict(layer_nms_iou_milli=[1000]), dict(layer_rep_lambda=[-1.0]),
+    dict(flags=8), dict(flags=8, unit_tokens=16, max_spans_per_region=4), dict(layer_theta=[1.5]),
+    dict(flags=16, cache_units=8), dict(flags=16, unit_tokens=64, cache_units=3),
+    dict(flags=16, unit_tokens=64, cache_units=129), dict(flags=16, unit_tokens=64, cache_units=8, score_decay=1.5),
+    dict(flags=17, unit_tokens=64, cache_units=7), dict(layer_nms_iou_milli=[1000]), dict(layer_rep_lambda=[-1.0]),
 ])
 def test_bad_parameters_are_rejected_on_the_host(lib, kw):
     base = dict(n_layers=1, n_q_heads=8, n_kv_heads=2, max_tokens=1024, chunk=256, window=512, n_sink=64, top_k=4)

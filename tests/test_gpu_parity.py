@@ -154,6 +154,48 @@ def test_segmentation_per_memory_unit(U, C, chunk, phi):
     print(rep)
 
 
+@pytest.mark.parametrize("cache_units,decay,extra", [
+    (4, 0.1, {}), (9, 0.5, dict(segment_per_unit=True, max_spans_per_region=3)),
+    (6, 1.0, dict(retrieval_head=(2, -1), retrieval_head_score=(0.5, 0.0), collab_vote=True)),
+])
+def test_host_memory_pager(cache_units, decay, extra):
+    # Sec. 3.4: evicted rows are mirrored in host memory, the retrieved units of a prefill call come from a unit
+    # cache in device memory or, when missing, over the bus from the mirror.  The harness checks the usual parity and,
+    # after every call, the cache's tags, usage scores and hit/miss counters against the policy model.
+    cfg = small_cfg(n_layers=2, context=2048, decode_steps=2, unit_tokens=64, top_k=4, host_kv=True,
+                    cache_units=cache_units, score_decay=decay, **extra)
+    rep = ph.run_stream(cfg, layers=[0, 1])
+    assert rep.cache_misses > 10 and rep.cache_hits > 10
+    print(rep)
+
+
+def test_host_memory_pager_is_bit_identical_to_the_resident_path():
+    # the same stream through a paged and a resident context: every output bit and every selection equal, also
+    # with irregular call sizes (units that are still growing bypass the cache) and after a sequence reset
+    cfg = small_cfg(n_layers=2, context=1800, decode_steps=0, unit_tokens=48, top_k=5)
+    paged = dataclasses.replace(cfg, host_kv=True, cache_units=7, score_decay=0.1)
+    st = inputs.SyntheticStream(cfg)
+    a, b = binding.Ltri(ph.params_of(cfg)), binding.Ltri(ph.params_of(paged))
+    sizes = [128, 100, 128, 7, 128, 128, 61, 128, 128, 128, 128, 128, 96, 128, 128]
+    for rnd in range(2):
+        t0 = 0
+        for n in sizes:
+            q, k, v = (x.cuda() for x in st.tokens(t0, n))
+            oa = a.ltri_prefill_chunk(0, 0, 2, q, k, v)
+            ob = b.ltri_prefill_chunk(0, 0, 2, q, k, v)
+            assert torch.equal(oa, ob), f"round {rnd} call at {t0}"
+            for l in range(2):
+                assert np.array_equal(a.ltri_get_selected(0, l), b.ltri_get_selected(0, l))
+            t0 += n
+        assert b.ltri_debug_read(binding.BUF_CACHE_STATS, 0, 1)[1] > 0
+        a.ltri_reset_sequence(0)
+        b.ltri_reset_sequence(0)
+        assert (b.ltri_debug_read(binding.BUF_CACHE_TAGS, 0, 0) == -1).all()
+    assert a.ltri_sync_status() == 0 and b.ltri_sync_status() == 0
+    a.close()
+    b.close()
+
+
 def test_voting_layer_by_layer_calls_match_one_call():
     # a real model submits one layer at a time: the ballots of the earlier layers of the same chunk are read from the
     # context's state and the selections must equal those of the all-layers call
