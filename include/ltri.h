@@ -133,12 +133,13 @@ enum {
   LTRI_FLAG_SEGMENT_PER_UNIT = 8,
   /* Host-memory pager for retrieved tokens (Sec. 3.4, "Implementation Details": GPU cache size, score decay).  When a
    * region leaves the window its K/V rows are also copied to host_kv (on an internal stream, overlapping the call's
-   * attention).  The retrieved units of a prefill call are then no longer read from the device-resident K/V slabs:
-   * a unit found in the (sequence, layer, KV head)'s unit cache is read from there; a missing one is pulled from
-   * host_kv over the bus by the top-k kernel itself, into the slot of the unit with the lowest usage score.  Results
-   * are bit-identical to the default path.  In this version the device slabs still hold every token (sink and local
-   * window are read from them, and so are the retrieved units of decode steps), so the flag exercises the data path of
-   * the pager but does not yet shrink the device footprint. */
+   * attention).  Retrieved units are then no longer read from the device-resident K/V slabs: a unit found in the
+   * (sequence, layer, KV head)'s unit cache is read from there; a missing one is pulled from host_kv over the bus by
+   * the top-k kernel itself, into the slot of the unit with the lowest usage score.  Prefill calls pack the units'
+   * rows from the cache slots (the unit the indexed range ends in, while still growing, straight from the mirror);
+   * decode steps attend over the cache slots in place.  Results are bit-identical to the default path.  In this
+   * version the device slabs still hold every token (sink and local window are read from them at absolute
+   * positions), so the flag exercises the whole data path of the pager but does not yet shrink the device footprint. */
   LTRI_FLAG_HOST_KV = 16
 };
 

@@ -35,6 +35,7 @@ __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevC
                                                                 const __nv_bfloat16* __restrict__ q, int nsplit) {
   extern __shared__ __align__(1024) unsigned char dsm[];
   __shared__ int rs[kMaxRanges], rp[kMaxRanges + 1];
+  __shared__ long long rko[kMaxRanges], rvo[kMaxRanges];  // host-memory pager: first K / V row of every range
   __shared__ float sm_m[4][G], sm_l[4][G];
   __shared__ float sm_o[4][G][kD];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -47,6 +48,10 @@ __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevC
     int run = 0;
     for (int i = 0; i < nr; ++i) {
       rs[i] = c.rng_start[rb + i];
+      if (c.host_kv) {
+        rko[i] = c.rng_koff[rb + i];
+        rvo[i] = c.rng_voff[rb + i];
+      }
       rp[i] = run;
       run += c.rng_len[rb + i];
     }
@@ -90,8 +95,14 @@ __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevC
         while (v >= rp[ri + 1]) ++ri;
         tok = (size_t)(rs[ri] + (v - rp[ri]));
       }
-      cp_async16(sk + tile_off(row, ch), Kslab + tok * kD + ch * 8, okr ? 16 : 0);
-      cp_async16(sv + tile_off(row, ch), Vslab + tok * kD + ch * 8, okr ? 16 : 0);
+      const __nv_bfloat16* kp = Kslab + tok * kD;
+      const __nv_bfloat16* vp = Vslab + tok * kD;
+      if (c.host_kv && okr) {  // the range may live in the unit cache: its rows are addressed from the slab bases
+        kp = c.Kc + (size_t)(rko[ri] + (v - rp[ri])) * kD;
+        vp = c.Vc + (size_t)(rvo[ri] + (v - rp[ri])) * kD;
+      }
+      cp_async16(sk + tile_off(row, ch), kp + ch * 8, okr ? 16 : 0);
+      cp_async16(sv + tile_off(row, ch), vp + ch * 8, okr ? 16 : 0);
     }
   };
 

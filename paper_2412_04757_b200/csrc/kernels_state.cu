@@ -1029,6 +1029,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   __shared__ int s_rs[kMaxRanges], s_rl[kMaxRanges], s_pre[kMaxRanges + 1], s_nr;  // merged ranges, packed-row prefix
   __shared__ int s_sst[2 * kMaxTopK], s_sln[2 * kMaxTopK];  // extents of the selected spans
   __shared__ int s_all[2 * kMaxTopK], s_nall;            // decode: this step's selection united with the persistent one
+  __shared__ long long s_ko[kMaxRanges], s_vo[kMaxRanges];  // pager, decode: first K / V row of every range
   const int g = blockIdx.x;
   int layer, sq, pos = 0, loc_begin = 0;
   if (DECODE) {
@@ -1135,53 +1136,16 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     }
   }
   __syncthreads();
-  if (tid == 0) {
-    int nr = 0;
-    long long tokens = 0;
-    auto push = [&](int st, int ln) {
-      if (ln <= 0) return;
-      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] >= st)  // adjacent, or (NMS with phi > 0) overlapping: one range
-        s_rl[nr - 1] = max(s_rl[nr - 1], st + ln - s_rs[nr - 1]);
-      else {
-        s_rs[nr] = st;
-        s_rl[nr] = ln;
-        ++nr;
-      }
-    };
-    if (DECODE) push(0, min(c.Ls, pos + 1));
-    for (int t = 0; t < nall; ++t) {
-      tokens += s_sln[t];
-      push(s_sst[t], s_sln[t]);
-    }
-    if (DECODE) push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
-    int run = 0;
-    for (int i = 0; i < nr; ++i) {
-      s_pre[i] = run;
-      run += s_rl[i];
-    }
-    s_pre[nr] = run;
-    s_nr = nr;
-    c.rng_cnt[unit * c.Hkv + g] = nr;
-    atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
-    if (!DECODE) c.gcnt[(size_t)layer * c.Hkv + g] = run;
-  }
-  __syncthreads();
-  {
-    const size_t rb = (unit * c.Hkv + g) * (size_t)c.rcap;
-    for (int t = tid; t < s_nr; t += nt) {
-      c.rng_start[rb + t] = s_rs[t];
-      c.rng_len[rb + t] = s_rl[t];
-    }
-  }
-  if (!DECODE && c.host_kv) {
-    // Host-memory pager (Sec. 3.4).  The selected units are looked up in this (sequence, layer, KV head)'s unit
-    // cache; every slot's usage score decays, a unit named now gains 1; a missing unit takes the slot with the
-    // lowest score among the slots not named now (lowest slot among equals) and its rows are pulled from the host
-    // mirror.  Only whole units are cached: the unit the indexed range ends in, while it is still growing, is read
-    // from the mirror every time.  s_src[t]: slot of selected unit t, -1 = straight from the host.
-    __shared__ int s_tag[128], s_src[2 * kMaxTopK], s_fill[2 * kMaxTopK];
-    __shared__ float s_sco[128];
-    __shared__ unsigned char s_named[128];
+  // Host-memory pager (Sec. 3.4).  The units named by this retrieval are looked up in this (sequence, layer, KV
+  // head)'s unit cache; every slot's usage score decays, a unit named now gains 1; a missing unit takes the slot with
+  // the lowest score among the slots not named now (lowest slot among equals) and its rows are pulled from the host
+  // mirror.  A prefill call caches only whole units: the unit the indexed range ends in, while it is still growing,
+  // is read from the mirror every time.  (During decode the indexed range no longer grows, so that unit is cached
+  // like the others.)  s_src[t]: slot of named unit t, -1 = straight from the host.
+  __shared__ int s_tag[128], s_src[2 * kMaxTopK], s_fill[2 * kMaxTopK];
+  __shared__ float s_sco[128];
+  __shared__ unsigned char s_named[128];
+  if (c.host_kv) {
     const int CU = c.cache_units;
     const size_t cb = (unit * c.Hkv + g) * (size_t)CU;
     if (tid < CU) {
@@ -1192,11 +1156,12 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     __syncthreads();
     if (tid == 0) {
       unsigned long long hits = 0, misses = 0;
+      auto growing = [&](int id) { return !DECODE && (id + 1) * U > Eend; };
       for (int t = 0; t < nall; ++t) {  // first the units that are there, so that none of them is pushed out
         const int id = ids_all[t];
         s_src[t] = -1;
         s_fill[t] = 0;
-        if ((id + 1) * U > Eend) continue;  // still growing: not cached
+        if (growing(id)) continue;
         for (int sl = 0; sl < CU; ++sl)
           if (s_tag[sl] == id) {
             s_src[t] = sl;
@@ -1208,7 +1173,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
       }
       for (int t = 0; t < nall; ++t) {
         const int id = ids_all[t];
-        if ((id + 1) * U > Eend || s_src[t] >= 0) continue;
+        if (growing(id) || s_src[t] >= 0) continue;
         int victim = -1;
         for (int sl = 0; sl < CU; ++sl)
           if (!s_named[sl] && (victim < 0 || s_sco[sl] < s_sco[victim])) victim = sl;
@@ -1243,7 +1208,68 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
         dv[i] = hv[i];
       }
     }
-    __syncthreads();  // the gather below reads what this CTA just wrote
+    __syncthreads();  // later reads of the slots by this CTA (the prefill gather) see the rows
+  }
+  if (tid == 0) {
+    int nr = 0;
+    long long tokens = 0;
+    // under the pager a decode step reads every named unit from its cache slot, so the units stay ranges of their own
+    // and every range carries the row it starts at, relative to the K slabs / the V slabs (s_ko, s_vo)
+    const bool paged = DECODE && c.host_kv;
+    const long long slab_row = (long long)((unit * c.Hkv + g) * (size_t)c.Tpad);
+    auto push = [&](int st, int ln, int slot) {
+      if (ln <= 0) return;
+      if (!paged && nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] >= st)  // adjacent, or (NMS with phi > 0) overlapping
+        s_rl[nr - 1] = max(s_rl[nr - 1], st + ln - s_rs[nr - 1]);
+      else {
+        s_rs[nr] = st;
+        s_rl[nr] = ln;
+        if (paged) {
+          if (slot >= 0) {
+            const long long crow =
+                (long long)(((unit * c.Hkv + g) * (size_t)c.cache_units + slot) * (size_t)U) + (st - (st / U) * U);
+            s_ko[nr] = (long long)((c.Kcache - c.Kc) / kD) + crow;
+            s_vo[nr] = (long long)((c.Vcache - c.Vc) / kD) + crow;
+          } else {
+            s_ko[nr] = s_vo[nr] = slab_row + st;
+          }
+        }
+        ++nr;
+      }
+    };
+    if (DECODE) push(0, min(c.Ls, pos + 1), -1);
+    for (int t = 0; t < nall; ++t) {
+      tokens += s_sln[t];
+      push(s_sst[t], s_sln[t], paged ? s_src[t] : -1);
+    }
+    if (DECODE) push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1), -1);
+    int run = 0;
+    for (int i = 0; i < nr; ++i) {
+      s_pre[i] = run;
+      run += s_rl[i];
+    }
+    s_pre[nr] = run;
+    s_nr = nr;
+    c.rng_cnt[unit * c.Hkv + g] = nr;
+    atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+    if (!DECODE) c.gcnt[(size_t)layer * c.Hkv + g] = run;
+  }
+  __syncthreads();
+  {
+    const size_t rb = (unit * c.Hkv + g) * (size_t)c.rcap;
+    for (int t = tid; t < s_nr; t += nt) {
+      c.rng_start[rb + t] = s_rs[t];
+      c.rng_len[rb + t] = s_rl[t];
+      if (DECODE && c.host_kv) {
+        c.rng_koff[rb + t] = s_ko[t];
+        c.rng_voff[rb + t] = s_vo[t];
+      }
+    }
+  }
+  if (!DECODE && c.host_kv) {
+    const int CU = c.cache_units;
+    const size_t cb = (unit * c.Hkv + g) * (size_t)CU;
+    const size_t hslab = (unit * c.Hkv + g) * (size_t)c.Tpad;
     // a5 gather, from the unit cache (or the host mirror) instead of the device slabs
     const int nr = s_nr, R = s_pre[nr], Rz = (R + 7) & ~7;
     const size_t gslab = ((size_t)layer * c.Hkv + g) * (size_t)c.Rcap;

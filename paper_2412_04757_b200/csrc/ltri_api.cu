@@ -152,6 +152,8 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.ctag = cv.take<int>(d.host_kv ? units * d.Hkv * d.cache_units : 0);
   d.cscore = cv.take<float>(d.host_kv ? units * d.Hkv * d.cache_units : 0);
   d.cstat = cv.take<unsigned long long>(d.host_kv ? units * 2 : 0);
+  d.rng_koff = cv.take<long long>(d.host_kv ? units * d.Hkv * d.rcap : 0);
+  d.rng_voff = cv.take<long long>(d.host_kv ? units * d.Hkv * d.rcap : 0);
   d.votes = cv.take<long long>(units * d.Tpad);
   d.span_start = cv.take<int>(units * d.cap);
   d.span_len = cv.take<int>(units * d.cap);

@@ -266,18 +266,21 @@ class StreamPair:
                 check_output(out[layer], o.prefill_attend(), rep, what)
         return out
 
-    def _check_cache(self, seq, layer, o, what):
-        """Host-memory pager: the unit cache of every KV head holds what the policy model says after this retrieval
-        (fed with the units the call fetched; the unit the indexed range ends in is cached only once it is whole)."""
+    def _check_cache(self, seq, layer, o, what, decode=False):
+        """Host-memory pager: the unit cache of every KV head holds what the policy model says after this retrieval,
+        fed with the units the call attends over.  Prefill: the unit the indexed range ends in is cached only once it
+        is whole.  Decode: the range no longer grows, every named unit is cached, the persistent ones included."""
         cfg, lt = self.cfg, self.lt
         U, E = cfg.unit_tokens, o.evicted_end
         sel = o.selected()[0]          # equal to the GPU's as a set (adopted where a near tie flipped a pick)
+        pers = o.persistent() if decode and cfg.persist_decode else np.full_like(sel, -1)
         tags = lt.ltri_debug_read(binding.BUF_CACHE_TAGS, seq, layer)
         scores = lt.ltri_debug_read(binding.BUF_CACHE_SCORES, seq, layer)
         hits = misses = 0
         for g in range(cfg.n_kv_heads):
             pol = self.cache[(seq, layer, g)]
-            pol.access(sorted(int(u) for u in sel[g] if u >= 0 and (u + 1) * U <= E))
+            named = set(int(u) for u in sel[g] if u >= 0) | set(int(u) for u in pers[g] if u >= 0)
+            pol.access(sorted(u for u in named if decode or (u + 1) * U <= E))
             assert tags[g].tolist() == pol.tags.tolist(), f"{what}: unit cache of KV head {g} holds other units"
             assert np.array_equal(scores[g], pol.scores), f"{what}: usage scores of KV head {g}"
             hits += pol.hits
@@ -365,6 +368,8 @@ class StreamPair:
                         self._vote(seq, layer, o, ballots, what)
                         self._count_vote_changes(o)
                     check_selection(lt.ltri_get_selected(seq, layer), o, rep, what, voted=cfg.collab_vote)
+                    if cfg.host_kv:
+                        self._check_cache(seq, layer, o, what, decode=True)
                     # tokens the step attends over besides sink and local: this step's spans united, under the
                     # persistent mechanism, with those of the last prefill call (every span once)
                     sel_o, _ = o.selected()

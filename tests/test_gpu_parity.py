@@ -155,15 +155,19 @@ def test_segmentation_per_memory_unit(U, C, chunk, phi):
 
 
 @pytest.mark.parametrize("cache_units,decay,extra", [
-    (4, 0.1, {}), (9, 0.5, dict(segment_per_unit=True, max_spans_per_region=3)),
+    (4, 0.1, dict(unit_tokens=48, window=256)), (9, 0.5, dict(segment_per_unit=True, max_spans_per_region=3, persist_decode=True)),
     (6, 1.0, dict(retrieval_head=(2, -1), retrieval_head_score=(0.5, 0.0), collab_vote=True)),
 ])
 def test_host_memory_pager(cache_units, decay, extra):
     # Sec. 3.4: evicted rows are mirrored in host memory, the retrieved units of a prefill call come from a unit
-    # cache in device memory or, when missing, over the bus from the mirror.  The harness checks the usual parity and,
-    # after every call, the cache's tags, usage scores and hit/miss counters against the policy model.
-    cfg = small_cfg(n_layers=2, context=2048, decode_steps=2, unit_tokens=64, top_k=4, host_kv=True,
-                    cache_units=cache_units, score_decay=decay, **extra)
+    # cache in device memory or, when missing, over the bus from the mirror; decode steps read their units from the
+    # cache slots as well (with the persistent mechanism: both sets).  The harness checks the usual parity and, after
+    # every call and step, the cache's tags, usage scores and hit/miss counters against the policy model.  The context
+    # length leaves the last unit of the indexed range partial.
+    kw = dict(n_layers=2, context=2048 - 40, decode_steps=6, unit_tokens=64, top_k=4, host_kv=True,
+              cache_units=cache_units, score_decay=decay)
+    kw.update(extra)    # (units of 48 tokens with a window of 256: the indexed range ends inside a unit during decode)
+    cfg = small_cfg(**kw)
     rep = ph.run_stream(cfg, layers=[0, 1])
     assert rep.cache_misses > 10 and rep.cache_hits > 10
     print(rep)
@@ -172,7 +176,7 @@ def test_host_memory_pager(cache_units, decay, extra):
 def test_host_memory_pager_is_bit_identical_to_the_resident_path():
     # the same stream through a paged and a resident context: every output bit and every selection equal, also
     # with irregular call sizes (units that are still growing bypass the cache) and after a sequence reset
-    cfg = small_cfg(n_layers=2, context=1800, decode_steps=0, unit_tokens=48, top_k=5)
+    cfg = small_cfg(n_layers=2, context=1800, decode_steps=4, unit_tokens=48, top_k=5)
     paged = dataclasses.replace(cfg, host_kv=True, cache_units=7, score_decay=0.1)
     st = inputs.SyntheticStream(cfg)
     a, b = binding.Ltri(ph.params_of(cfg)), binding.Ltri(ph.params_of(paged))
@@ -188,6 +192,9 @@ def test_host_memory_pager_is_bit_identical_to_the_resident_path():
                 assert np.array_equal(a.ltri_get_selected(0, l), b.ltri_get_selected(0, l))
             t0 += n
         assert b.ltri_debug_read(binding.BUF_CACHE_STATS, 0, 1)[1] > 0
+        for step in range(3):      # decode steps read their units from the cache slots
+            q, k, v = (x.permute(1, 0, 2, 3).contiguous().cuda() for x in st.tokens(t0 + step, 1, kind=1))
+            assert torch.equal(a.ltri_decode_step([0], 0, 2, q, k, v), b.ltri_decode_step([0], 0, 2, q, k, v))
         a.ltri_reset_sequence(0)
         b.ltri_reset_sequence(0)
         assert (b.ltri_debug_read(binding.BUF_CACHE_TAGS, 0, 0) == -1).all()
