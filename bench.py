@@ -319,7 +319,9 @@ def run_ltri(args, cfg):
                             max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
                             flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
                                   (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0) |
-                                  (binding.FLAG_SEGMENT_PER_UNIT if cfg.segment_per_unit else 0),
+                                  (binding.FLAG_SEGMENT_PER_UNIT if cfg.segment_per_unit else 0) |
+                                  (binding.FLAG_HOST_KV if cfg.host_kv else 0),
+                            cache_units=cfg.cache_units, score_decay=cfg.score_decay,
                             unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
                             retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score,
                             layer_theta=cfg.layer_theta, layer_nms_iou_milli=cfg.layer_nms_iou_milli,
@@ -377,6 +379,16 @@ def run_ltri(args, cfg):
     lt.ltri_profile_enable(False)
     assert lt.ltri_sync_status() == 0, "device-side status word reports an error"
     stats = lt.ltri_get_stats(SQ, 0)
+    pager = None
+    if cfg.host_kv:
+        # unit-cache traffic of all layers since the stream began (prefill calls only so far)
+        hm = sum(lt.ltri_debug_read(binding.BUF_CACHE_STATS, SQ, l) for l in range(L))
+        unit_bytes = cfg.unit_tokens * cfg.head_dim * 2 * 2     # K and V rows of one unit
+        pager = {"cache_units": cfg.cache_units, "score_decay": cfg.score_decay, "unit_hits": int(hm[0]),
+                 "unit_misses": int(hm[1]), "hit_rate": float(hm[0] / max(1, hm[0] + hm[1])),
+                 "host_to_device_bytes_per_call": float(hm[1]) * unit_bytes / max(1, len(chunks)),
+                 "device_to_host_bytes_per_call": float(L * cfg.n_kv_heads * cfg.chunk * cfg.head_dim * 2 * 2),
+                 "note": "prefill calls of the whole stream; the mirror gets every evicted row once"}
     recall = {"final_chunk": needle_recall(lt, st, SQ, cfg)} if cfg.needle and rank == 0 else None
     ms = max_over_ranks(ms, world, dev)
     tokens = K * n
@@ -504,7 +516,7 @@ def run_ltri(args, cfg):
                    "parallelism": "replicas only" if world > 1 else "single GPU", "sequences": NSEQ,
                    "index_spans": stats.n_spans, "retrieved_tokens_per_kv_head": stats.retrieved_tokens / cfg.n_kv_heads},
         "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "decode": dec, "roofline": roof, "cpu_baseline": cpu,
-        "needle_recall": recall,
+        "needle_recall": recall, "pager": pager,
         "kernel_ms_per_step": {k: v[0] / K for k, v in prof.items() if v[1]},
     }
     print(json.dumps(line))
@@ -529,6 +541,10 @@ def main():
                     help="IoU threshold of the segmenter's NMS (0: spans never overlap; the paper lists 0.1 / 0.01)")
     ap.add_argument("--persist-decode", action="store_true",
                     help="decode keeps the spans selected by the last prefill call (persistent mechanism)")
+    ap.add_argument("--host-kv", type=int, default=0, metavar="CACHE_UNITS",
+                    help="host-memory pager: mirror evicted rows in pinned host memory and read retrieved units from a "
+                         "device cache of this many units per (layer, KV head) (the paper's 32); needs --unit-tokens. "
+                         "The mirror takes 2 x layers x KV heads x context x 256 bytes of pinned memory")
     ap.add_argument("--segment-per-unit", action="store_true",
                     help="segment every memory unit on its own, four spans kept per unit (the paper's 'Span' column); "
                          "needs --unit-tokens")
@@ -573,6 +589,12 @@ def main():
         import dataclasses
         cfg = dataclasses.replace(cfg, persist_decode=True)
         cfg.name += "[persist-decode]"
+    if args.host_kv > 0:
+        import dataclasses
+        if args.unit_tokens <= 0:
+            ap.error("--host-kv needs --unit-tokens")
+        cfg = dataclasses.replace(cfg, host_kv=True, cache_units=args.host_kv, score_decay=0.1)
+        cfg.name += f"[host-kv,cache={args.host_kv}]"
     if args.segment_per_unit:
         import dataclasses
         if args.unit_tokens <= 0:

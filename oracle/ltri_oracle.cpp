@@ -34,6 +34,9 @@
 //        alone (map, theta, votes, representatives, scores)
 //   O9'' units ranked by the weighted ballots of the layers    Sec. 3.5 "Collaborative Voting"
 //        up to this one, then by the layer's own scores
+//   O6'' every memory unit of the region segmented on its own  Sec. 3.3 (blocks divided into spans)
+// (The policy of the device-side cache of memory units, Sec. 3.4, changes no result of attention; its model,
+//  UnitCachePolicy, lives in the Python wrapper beside this file.)
 //
 // Parity status: O3/O10/O12 are pinned by softmax invariants and by the full-attention
 // equivalence; O6 is pinned by brute force, by hand-built block maps and by a library
