@@ -151,7 +151,8 @@ typedef struct {
   int64_t index_bytes;     /* N_s * n_kv_heads * head_dim * 2 */
   int64_t retrieved_tokens; /* sum of the lengths of the spans selected by the last call, over KV heads */
   int32_t last_call_spans; /* spans the last prefill call cut its region into */
-  int32_t reserved;
+  int32_t slab_slides;     /* LTRI_FLAG_HOST_KV: times the live rows of this layer's sliding K/V slabs were moved to the
+                              start of their window region (0 in a resident context) */
 } ltri_stats;
 
 /* Bytes of device memory the arena must provide for these parameters (host only; the

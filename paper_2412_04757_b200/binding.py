@@ -56,7 +56,7 @@ class LtriStats(C.Structure):
     _fields_ = [
         ("tokens", C.c_int64), ("evicted_end", C.c_int64), ("n_spans", C.c_int32), ("n_pending_regions", C.c_int32),
         ("index_bytes", C.c_int64), ("retrieved_tokens", C.c_int64), ("last_call_spans", C.c_int32),
-        ("reserved", C.c_int32),
+        ("slab_slides", C.c_int32),
     ]
 
 

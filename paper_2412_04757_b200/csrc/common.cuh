@@ -22,7 +22,13 @@ constexpr int kTokPad = 128;          // rows of slack after every K/V slab so t
 // Device-side view of one context.  Passed to kernels by value.
 struct DevCtx {
   int NL, Hq, Hkv, G, NS;
-  long long Tpad;        // row capacity of a per-(seq,layer,kv-head) K/V slab (max_tokens + slack)
+  long long Tpad;        // token capacity of a (seq, layer): max_tokens + slack (votes, host mirror of the pager)
+  long long SR;          // rows of a per-(seq, layer, KV head) K/V slab.  Resident context: Tpad, row = token.
+                         // Paged context (sliding slab): rows [0, Ls) hold the sink for good; behind them, from row
+                         // Lsp on, sits the window: the row of token tok is tok - shift, where shift = (first token
+                         // the window region holds) - Lsp moves up whenever the host compacts the slab
+  int paged;             // 1: sliding slabs (host-memory pager)
+  int Lsp;               // first row of the window region of a sliding slab
   long long Tmax;
   int chunk, W, Ls, topk, reps, C, Jmax, cap, slots;
   int rcap;              // token ranges kept per (seq, layer, KV head): 2 * top_k + 2
@@ -35,7 +41,7 @@ struct DevCtx {
   int rep_mode, ratio_kind, min_reps, max_reps;  // dynamic span index vectors (Sec. 3.3.2); rep_mode 0: static count
   float rep_lambda;
   // persistent state
-  __nv_bfloat16* Kc;     // [NS][NL][Hkv][Tpad][128]
+  __nv_bfloat16* Kc;     // [NS][NL][Hkv][SR][128]
   __nv_bfloat16* Vc;
   long long* votes;      // [NS][NL][Tpad]
   int* span_start;       // [NS][NL][cap]
@@ -98,6 +104,12 @@ struct DevCtx {
 
 __host__ __device__ inline size_t unit_of(const DevCtx& c, int seq, int layer) { return (size_t)seq * c.NL + layer; }
 
+// Row of token `tok` inside its K/V slab (see DevCtx::SR).  Sink tokens are also written to their window row while
+// they are inside the window, so a range that starts in the window may be read with window rows throughout.
+__host__ __device__ inline long long slab_row(const DevCtx& c, long long tok, long long shift) {
+  return (c.paged && tok >= c.Ls) ? tok - shift : tok;
+}
+
 #ifdef __CUDACC__
 // Retrieval head of a layer (Sec. 3.5): -1 when the layer locates evidence with all its heads.
 __device__ __forceinline__ int ret_head_of(const DevCtx& c, int layer) { return c.ret_head ? c.ret_head[layer] : -1; }
@@ -111,12 +123,14 @@ struct DecBatch {
   int pos[kDecBatch];        // position of the new token
   int loc_begin[kDecBatch];  // E' of the sequence/layer
   int src[kDecBatch];        // index into the caller's [n_seqs] arrays
+  long long shift[kDecBatch];  // sliding slabs: token - shift = row of the sequence's window tokens
 };
 
 struct EvictArgs {
   int seq, layer_begin;
   int nslots;
   int slot[8];
+  long long shift;  // sliding slabs: token - shift = row
 };
 
 struct PrefillArgs {
@@ -125,6 +139,7 @@ struct PrefillArgs {
   int sink_end, loc_begin;  // sink = [0,sink_end), local = [loc_begin,t0)
   int reg_start, m;         // region [reg_start, t0+n), m tokens
   int slot;                 // pending slot of this region (-1 if the region is empty)
+  long long shift;          // sliding slabs: token - shift = row of the window tokens (0 in a resident context)
   const __nv_bfloat16* q;   // [layer_count][n][Hq][128]
   const __nv_bfloat16* k;
   const __nv_bfloat16* v;

@@ -63,8 +63,8 @@ __global__ void __launch_bounds__(256, 1) k_attn_prefill(DevCtx c, PrefillArgs a
   }
   __syncthreads();
 
-  const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD;
-  const __nv_bfloat16* Vslab = c.Vc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD;
+  const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.SR * kD;
+  const __nv_bfloat16* Vslab = c.Vc + (unit * c.Hkv + g) * (size_t)c.SR * kD;
   const float c2 = c.scale * kLog2e;
 
   // rows of this thread
@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(128) k_map_local(DevCtx c, PrefillArgs a) {
   constexpr int TOK = 64 / G;
   const int ntiles = (a.n + TOK - 1) / TOK;
   if (tid < 64) sh_cols[tid] = 0;
-  const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD;
+  const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.SR * kD;
   load_tile_async(sK, Kslab + (size_t)kt * kD, kD, 64, nvalid, tid, 128);
   auto issue_q = [&](int stage, int t) {
     const int tok0 = t * TOK;
@@ -376,7 +376,7 @@ __global__ void __launch_bounds__(128) k_map_cur(DevCtx c, PrefillArgs a) {
                     128);
     if (h % G == 0) {
       const int g = h / G;
-      const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD;
+      const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.SR * kD;
       load_tile_async(sK + (g & 1) * 16384, Kslab + (size_t)(a.t0 + j0) * kD, kD, 64, kvalid, tid, 128);
     }
   };

@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     w.tok0 = w.mb * TOKB;
     w.unit = unit_of(c, a.seq, w.layer);
     // phase 0 reads the K/V cache of the (sequence, layer, KV head); phase 1 the packed slab of the selected spans
-    w.slab_row0 = phase == 0 ? (w.unit * c.Hkv + w.g) * (size_t)c.Tpad
+    w.slab_row0 = phase == 0 ? (w.unit * c.Hkv + w.g) * (size_t)c.SR
                              : ((size_t)w.layer * c.Hkv + w.g) * (size_t)c.Rcap;
     return w;
   };
@@ -274,9 +274,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       int pslot[16], ptok[16], pbox[16];
       while (true) {
         int np = 0;
+        // (pieces are addressed by slab row: in a sliding slab the ranges behind the sink sit at token - shift)
         if (!it.next<true>([&](int slot, int tok, int bi) {
               pslot[np] = slot;
-              ptok[np] = tok;
+              ptok[np] = (phase == 0 && c.paged && it.ri > 0) ? (int)(tok - a.shift) : tok;
               pbox[np] = bi;
               ++np;
             }))
@@ -689,7 +690,7 @@ bool tc_encode_kv_maps(const DevCtx& c, void* out_bytes) {
   EncodeFn enc = get_encode();
   if (!enc) return false;
   CUtensorMap* out = static_cast<CUtensorMap*>(out_bytes);
-  const cuuint64_t rows = (cuuint64_t)c.NS * c.NL * c.Hkv * (cuuint64_t)c.Tpad * 2;  // K slabs then V slabs
+  const cuuint64_t rows = (cuuint64_t)c.NS * c.NL * c.Hkv * (cuuint64_t)c.SR * 2;  // K slabs then V slabs
   for (int i = 0; i < kNumBoxes; ++i) {
     cuuint64_t dims[2] = {128, rows};
     cuuint64_t strides[1] = {256};
@@ -727,7 +728,7 @@ bool tc_encode_kv_maps(const DevCtx& c, void* out_bytes) {
 
 bool tc_attention_supported(const DevCtx& c) {
   // the V slabs must follow the K slabs directly (one tensor map covers both) and row indices must fit 31 bits
-  const size_t rows = (size_t)c.NS * c.NL * c.Hkv * (size_t)c.Tpad;
+  const size_t rows = (size_t)c.NS * c.NL * c.Hkv * (size_t)c.SR;
   if (c.Vc != c.Kc + rows * kD) return false;
   if (rows * 2 >= (1ull << 31)) return false;
   const size_t grows = (size_t)c.NL * c.Hkv * (size_t)c.Rcap;
@@ -755,7 +756,7 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase,
   constexpr int TOKB = 256 / G;
   const int smem = 65536 + 131072 + 1024;
   cudaFuncSetAttribute(k_attn_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  const long long v_off = phase == 0 ? (long long)c.NS * c.NL * c.Hkv * c.Tpad : (long long)c.NL * c.Hkv * c.Rcap;
+  const long long v_off = phase == 0 ? (long long)c.NS * c.NL * c.Hkv * c.SR : (long long)c.NL * c.Hkv * c.Rcap;
   static int sms = 0;
   if (sms == 0) {
     int dev = 0;

@@ -74,8 +74,9 @@ __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevC
       qa[ks][1] = r < G ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + 2 * qd) : 0u;
     }
   }
-  const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD;
-  const __nv_bfloat16* Vslab = c.Vc + (unit * c.Hkv + g) * (size_t)c.Tpad * kD;
+  // (resident contexts: row = token; paged contexts address every range through rko / rvo below)
+  const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.SR * kD;
+  const __nv_bfloat16* Vslab = c.Vc + (unit * c.Hkv + g) * (size_t)c.SR * kD;
   const uint32_t wbase = smem_u32(dsm) + warp * kDWarpBytes;
   const float c2 = c.scale * kLog2eD;
 

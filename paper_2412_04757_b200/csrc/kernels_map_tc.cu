@@ -105,7 +105,8 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     if (lane == 0) {
       mbar_expect_tx(bar(B_KFULL), (uint32_t)ntile * 32768u);
       for (int kt = 0; kt < ntile; ++kt) {
-        const long long krow = (long long)(unit * c.Hkv + g) * c.Tpad + key0_of(kt);
+        // (local and current keys: window rows of the slab)
+        const long long krow = (long long)(unit * c.Hkv + g) * c.SR + key0_of(kt) - (c.paged ? a.shift : 0);
         tma_load_2d(sK + kt * 32768, &maps.k128, 0, (int)krow, bar(B_KFULL));
         tma_load_2d(sK + kt * 32768 + 16384, &maps.k128, 64, (int)krow, bar(B_KFULL));
       }

@@ -56,10 +56,22 @@ __global__ void k_append_prefill(DevCtx c, PrefillArgs a) {
   const int r = (row / c.Hkv) % a.n;
   const int l = row / ((size_t)c.Hkv * a.n);
   const size_t unit = unit_of(c, a.seq, a.layer_begin + l);
-  const size_t dst = ((unit * c.Hkv + g) * c.Tpad + (a.t0 + r)) * kD + c16 * 8;
+  const long long tok = a.t0 + r;
+  const long long wrow = c.paged ? tok - a.shift : tok;  // window row (a sink token has one too while it is current)
+  if (wrow < 0 || wrow >= c.SR) {                         // cannot happen: the host keeps the window inside the slab
+    set_status(c, -2, (int)tok);
+    return;
+  }
+  const size_t dst = ((unit * c.Hkv + g) * c.SR + wrow) * kD + c16 * 8;
   const size_t src = row * kD + c16 * 8;
-  *reinterpret_cast<uint4*>(c.Kc + dst) = *reinterpret_cast<const uint4*>(a.k + src);
-  *reinterpret_cast<uint4*>(c.Vc + dst) = *reinterpret_cast<const uint4*>(a.v + src);
+  const uint4 kv = *reinterpret_cast<const uint4*>(a.k + src), vv = *reinterpret_cast<const uint4*>(a.v + src);
+  *reinterpret_cast<uint4*>(c.Kc + dst) = kv;
+  *reinterpret_cast<uint4*>(c.Vc + dst) = vv;
+  if (c.paged && tok < c.Ls) {  // the sink's permanent rows
+    const size_t sd = ((unit * c.Hkv + g) * c.SR + tok) * kD + c16 * 8;
+    *reinterpret_cast<uint4*>(c.Kc + sd) = kv;
+    *reinterpret_cast<uint4*>(c.Vc + sd) = vv;
+  }
   if (g == 0 && c16 == 0) c.votes[unit * c.Tpad + a.t0 + r] = 0;
 }
 
@@ -79,10 +91,22 @@ __global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer
   const int l = (row / c.Hkv) % layer_count;
   const int bi = row / ((size_t)c.Hkv * layer_count);
   const size_t unit = unit_of(c, b.seq[bi], layer_begin + l);
-  const size_t dst = ((unit * c.Hkv + g) * c.Tpad + b.pos[bi]) * kD + c16 * 8;
+  const long long tok = b.pos[bi];
+  const long long wrow = c.paged ? tok - b.shift[bi] : tok;
+  if (wrow < 0 || wrow >= c.SR) {  // cannot happen: the host keeps the window inside the slab
+    set_status(c, -2, (int)tok);
+    return;
+  }
+  const size_t dst = ((unit * c.Hkv + g) * c.SR + wrow) * kD + c16 * 8;
   const size_t src = (((size_t)b.src[bi] * layer_count + l) * c.Hkv + g) * kD + c16 * 8;
-  *reinterpret_cast<uint4*>(c.Kc + dst) = *reinterpret_cast<const uint4*>(k + src);
-  *reinterpret_cast<uint4*>(c.Vc + dst) = *reinterpret_cast<const uint4*>(v + src);
+  const uint4 kv = *reinterpret_cast<const uint4*>(k + src), vv = *reinterpret_cast<const uint4*>(v + src);
+  *reinterpret_cast<uint4*>(c.Kc + dst) = kv;
+  *reinterpret_cast<uint4*>(c.Vc + dst) = vv;
+  if (c.paged && tok < c.Ls) {  // the sink's permanent rows
+    const size_t sd = ((unit * c.Hkv + g) * c.SR + tok) * kD + c16 * 8;
+    *reinterpret_cast<uint4*>(c.Kc + sd) = kv;
+    *reinterpret_cast<uint4*>(c.Vc + sd) = vv;
+  }
   if (g == 0 && c16 == 0) {
     c.votes[unit * c.Tpad + b.pos[bi]] = 0;
     c.sel_tokens[unit] = 0;  // the retrieval kernels of this step add the tokens they select
@@ -123,10 +147,11 @@ __global__ void __launch_bounds__(1024) k_evict_index(DevCtx c, EvictArgs a) {
       int toks[kMaxReps];
       const int nrep = select_reps(votes, start, len, c.rep_mode == 1 ? c.pend_nrep[ps + i] : c.reps, toks);
       for (int g = 0; g < c.Hkv; ++g) {
-        const __nv_bfloat16* kslab = c.Kc + ((unit * c.Hkv + g) * c.Tpad) * kD;
+        const __nv_bfloat16* kslab = c.Kc + ((unit * c.Hkv + g) * c.SR) * kD;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         for (int r = 0; r < nrep; ++r) {
-          const uint2 raw = *reinterpret_cast<const uint2*>(kslab + (size_t)toks[r] * kD + lane * 4);
+          const uint2 raw =
+              *reinterpret_cast<const uint2*>(kslab + (size_t)slab_row(c, toks[r], a.shift) * kD + lane * 4);
           const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
           const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
           acc[0] += __bfloat162float(p0.x);
@@ -1216,7 +1241,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     // under the pager a decode step reads every named unit from its cache slot, so the units stay ranges of their own
     // and every range carries the row it starts at, relative to the K slabs / the V slabs (s_ko, s_vo)
     const bool paged = DECODE && c.host_kv;
-    const long long slab_row = (long long)((unit * c.Hkv + g) * (size_t)c.Tpad);
+    const long long slab0 = (long long)((unit * c.Hkv + g) * (size_t)c.SR);
     auto push = [&](int st, int ln, int slot) {
       if (ln <= 0) return;
       if (!paged && nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] >= st)  // adjacent, or (NMS with phi > 0) overlapping
@@ -1231,7 +1256,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
             s_ko[nr] = (long long)((c.Kcache - c.Kc) / kD) + crow;
             s_vo[nr] = (long long)((c.Vcache - c.Vc) / kD) + crow;
           } else {
-            s_ko[nr] = s_vo[nr] = slab_row + st;
+            s_ko[nr] = s_vo[nr] = slab0 + slab_row(c, st, DECODE ? b.shift[blockIdx.y / layer_count] : 0);
           }
         }
         ++nr;
@@ -1309,7 +1334,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     // attention kernel that continues over them reads whole 128-row tiles.  16 threads per 256-byte row, four rows
     // of K and of V in flight per thread; the rows up to the next multiple of 8 are zero-filled.
     const int nr = s_nr, R = s_pre[nr], Rz = (R + 7) & ~7;
-    const size_t slab = (unit * c.Hkv + g) * (size_t)c.Tpad;
+    const size_t slab = (unit * c.Hkv + g) * (size_t)c.SR;  // (resident contexts only: row = token)
     const uint4* Ksrc = reinterpret_cast<const uint4*>(c.Kc + slab * kD);
     const uint4* Vsrc = reinterpret_cast<const uint4*>(c.Vc + slab * kD);
     const size_t gslab = ((size_t)layer * c.Hkv + g) * (size_t)c.Rcap;

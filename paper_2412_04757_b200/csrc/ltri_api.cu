@@ -26,6 +26,8 @@ struct LayerState {
   std::deque<Region> pending;
   long long span_ub = 0;  // upper bound of the device-side span count
   int last_m = 0;
+  long long base = 0;  // sliding slabs: first token the window region of this layer's slabs holds
+  int slides = 0;      // times the live rows were moved to the start of the window region
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -105,6 +107,9 @@ size_t stage_set_bytes(const ltri_params& p) {
   return align_up(rows * p.n_q_heads * kD * 2, 256) * 2 + align_up(rows * p.n_kv_heads * kD * 2, 256) * 2;
 }
 
+// rows of the window region of a sliding slab (see layout): 2 x (window + 2 chunks) + tile slack
+long long window_rows(const ltri_params& p) { return 2ll * ((long long)p.window + 2ll * p.chunk) + 2 * kTokPad; }
+
 // fills every pointer of `d` relative to `base` (nullptr: sizing only) and returns the bytes used
 size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nullptr) {
   d.NL = p.n_layers;
@@ -145,8 +150,14 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.cache_units = d.host_kv ? p.cache_units : 0;
   d.score_decay = p.score_decay;
   const size_t cache_rows = d.host_kv ? units * d.Hkv * (size_t)d.cache_units * p.unit_tokens : 0;
-  d.Kc = cv.take<__nv_bfloat16>(units * d.Hkv * d.Tpad * kD);
-  d.Vc = cv.take<__nv_bfloat16>(units * d.Hkv * d.Tpad * kD);
+  // K/V slabs.  Resident: a row per token.  Paged: the sink, then a window region that holds twice what a call can
+  // touch (tokens since the last eviction before the call + the call + tile slack), so that when it runs full the
+  // live rows can be moved to its start without overlapping themselves.
+  d.paged = d.host_kv;
+  d.Lsp = d.paged ? (int)align_up((size_t)p.n_sink + 8, 8) : 0;
+  d.SR = d.paged ? d.Lsp + window_rows(p) + kTokPad : d.Tpad;
+  d.Kc = cv.take<__nv_bfloat16>(units * d.Hkv * d.SR * kD);
+  d.Vc = cv.take<__nv_bfloat16>(units * d.Hkv * d.SR * kD);
   d.Kcache = cv.take<__nv_bfloat16>(cache_rows * kD);
   d.Vcache = cv.take<__nv_bfloat16>(cache_rows * kD);
   d.ctag = cv.take<int>(d.host_kv ? units * d.Hkv * d.cache_units : 0);
@@ -234,6 +245,7 @@ struct ltri_ctx {
   cudaStream_t s_spill = nullptr;
   cudaEvent_t ev_pre = nullptr, ev_spill = nullptr;
   char* host_kv = nullptr;   // the caller's mirror (host address)
+  bool spilled = false;      // ev_spill has been recorded at least once
   cudaEvent_t ev_up[2][kHostGroups] = {}, ev_run[2][kHostGroups] = {}, ev_down[2][kHostGroups] = {};
   bool set_used[2] = {false, false};
   long long host_calls = 0;
@@ -393,8 +405,9 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
   ctx->use_tc = tc_attention_supported(ctx->d) && !(impl && std::strcmp(impl, "mma") == 0) &&
                 tc_encode_kv_maps(ctx->d, ctx->kv_maps);
   // unfilled tile slots and over-fetched rows must hold finite values: start from an all-zero cache
-  const size_t kv_bytes = (size_t)p->max_seqs * p->n_layers * ctx->d.Hkv * (size_t)ctx->d.Tpad * kD * 2 * sizeof(__nv_bfloat16);
-  if (!ctx->ret_head.empty() && !ctx->use_tc) {  // retrieval heads are built into the tensor-core map pass only
+  const size_t kv_bytes = (size_t)p->max_seqs * p->n_layers * ctx->d.Hkv * (size_t)ctx->d.SR * kD * 2 * sizeof(__nv_bfloat16);
+  if ((!ctx->ret_head.empty() || ctx->d.paged) && !ctx->use_tc) {
+    // retrieval heads are built into the tensor-core map pass only, sliding slabs into the tensor-core kernels only
     ltri_destroy(ctx);
     return LTRI_EINVAL;
   }
@@ -470,6 +483,34 @@ int ltri_reset_sequence(ltri_ctx* ctx, int seq, void* cuda_stream) {
   return LTRI_OK;
 }
 
+// Sliding slabs: make room for tokens up to `t_end` (exclusive) in the window region of the slabs of the given layers.
+// When the region is full, the live rows -- everything since the last eviction, [E, t) -- are moved to its start with
+// one strided device copy for K and one for V; the region is sized so that source and destination cannot overlap.
+// Rows that leave the slab this way were mirrored to the host when their region was evicted: the copy waits for that.
+static int slide_window(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, long long t_end, cudaStream_t st) {
+  const DevCtx& d = ctx->d;
+  LayerState& s0 = ctx->at(seq, layer_begin);
+  const long long cap = d.SR - d.Lsp - kTokPad;  // rows of the window region that may hold tokens
+  if (t_end - s0.base <= cap) return LTRI_OK;
+  const long long nb = s0.E, live = s0.t - nb, dist = nb - s0.base;
+  if (t_end - nb > cap || dist < live) return LTRI_ECAPACITY;  // (decode ran past what a sliding slab can hold)
+  if (ctx->spilled) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_spill, 0));
+  if (live > 0) {
+    const size_t row_bytes = kD * sizeof(__nv_bfloat16), pitch = (size_t)d.SR * row_bytes;
+    const size_t slab0 = unit_of(d, seq, layer_begin) * d.Hkv;
+    const size_t to = (slab0 * (size_t)d.SR + d.Lsp) * row_bytes, from = to + (size_t)dist * row_bytes;
+    for (__nv_bfloat16* base : {d.Kc, d.Vc})
+      LTRI_CUDA(ctx, cudaMemcpy2DAsync(reinterpret_cast<char*>(base) + to, pitch, reinterpret_cast<const char*>(base) + from,
+                                       pitch, (size_t)live * row_bytes, (size_t)layer_count * d.Hkv,
+                                       cudaMemcpyDeviceToDevice, st));
+  }
+  for (int l = 0; l < layer_count; ++l) {
+    ctx->at(seq, layer_begin + l).base = nb;
+    ctx->at(seq, layer_begin + l).slides += 1;
+  }
+  return LTRI_OK;
+}
+
 int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q,
                        const void* k, const void* v, void* out, void* cuda_stream) {
   if (!ctx) return LTRI_EINVAL;
@@ -482,10 +523,16 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   for (int l = 0; l < layer_count; ++l) {
     const LayerState& s = ctx->at(seq, layer_begin + l);
     if (s.decoding) return LTRI_ESTATE;
-    if (s.t != s0.t || s.E != s0.E || s.pending.size() != s0.pending.size()) return LTRI_ESTATE;
+    if (s.t != s0.t || s.E != s0.E || s.pending.size() != s0.pending.size() || s.base != s0.base) return LTRI_ESTATE;
   }
   if (s0.t + n_tokens > d.Tmax) return LTRI_ECAPACITY;
   const int t0 = (int)s0.t;
+  cudaStream_t st0 = static_cast<cudaStream_t>(cuda_stream);
+  if (d.paged) {
+    const int rc = slide_window(ctx, seq, layer_begin, layer_count, t0 + n_tokens, st0);
+    if (rc != LTRI_OK) return rc;
+  }
+  const long long shift = d.paged ? s0.base - d.Lsp : 0;
   // plan the evictions (host knows region boundaries; span counts live on the device)
   std::vector<Region> ev;
   int E = s0.E;
@@ -526,6 +573,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   a.reg_start = reg_start;
   a.m = m;
   a.slot = slot;
+  a.shift = shift;
   a.q = static_cast<const __nv_bfloat16*>(q);
   a.k = static_cast<const __nv_bfloat16*>(k);
   a.v = static_cast<const __nv_bfloat16*>(v);
@@ -539,6 +587,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
     Scope sc(ctx, st, LTRI_K_EVICT, 1);
     EvictArgs ea;
     ea.seq = seq;
+    ea.shift = shift;
     ea.layer_begin = layer_begin;
     ea.nslots = (int)std::min<size_t>(8, ev.size() - i);
     for (int j = 0; j < ea.nslots; ++j) ea.slot[j] = ev[i + j].slot;
@@ -551,17 +600,21 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
     // pull them back, waits for the copies
     LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_pre, st));
     LTRI_CUDA(ctx, cudaStreamWaitEvent(ctx->s_spill, ctx->ev_pre, 0));
-    const size_t half = (size_t)d.NS * d.NL * d.Hkv * (size_t)d.Tpad * kD * sizeof(__nv_bfloat16);
-    const size_t pitch = (size_t)d.Tpad * kD * sizeof(__nv_bfloat16);
+    const size_t row_bytes = kD * sizeof(__nv_bfloat16);
+    const size_t half = (size_t)d.NS * d.NL * d.Hkv * (size_t)d.Tpad * row_bytes;
+    const size_t hpitch = (size_t)d.Tpad * row_bytes, dpitch = (size_t)d.SR * row_bytes;
+    const size_t slab0 = unit_of(d, seq, layer_begin) * d.Hkv;  // first slab of the call's layers
     for (const Region& r : ev) {
-      const size_t off = ((unit_of(d, seq, layer_begin) * d.Hkv) * (size_t)d.Tpad + r.start) * kD * sizeof(__nv_bfloat16);
-      const size_t width = (size_t)(r.end - r.start) * kD * sizeof(__nv_bfloat16);
-      LTRI_CUDA(ctx, cudaMemcpy2DAsync(ctx->host_kv + off, pitch, reinterpret_cast<const char*>(d.Kc) + off, pitch, width,
-                                       (size_t)layer_count * d.Hkv, cudaMemcpyDeviceToHost, ctx->s_spill));
-      LTRI_CUDA(ctx, cudaMemcpy2DAsync(ctx->host_kv + half + off, pitch, reinterpret_cast<const char*>(d.Vc) + off, pitch,
+      const size_t hoff = (slab0 * (size_t)d.Tpad + r.start) * row_bytes;  // mirror: a row per token
+      const size_t doff = (slab0 * (size_t)d.SR + (size_t)slab_row(d, r.start, shift)) * row_bytes;
+      const size_t width = (size_t)(r.end - r.start) * row_bytes;
+      LTRI_CUDA(ctx, cudaMemcpy2DAsync(ctx->host_kv + hoff, hpitch, reinterpret_cast<const char*>(d.Kc) + doff, dpitch,
                                        width, (size_t)layer_count * d.Hkv, cudaMemcpyDeviceToHost, ctx->s_spill));
+      LTRI_CUDA(ctx, cudaMemcpy2DAsync(ctx->host_kv + half + hoff, hpitch, reinterpret_cast<const char*>(d.Vc) + doff,
+                                       dpitch, width, (size_t)layer_count * d.Hkv, cudaMemcpyDeviceToHost, ctx->s_spill));
     }
     LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_spill, ctx->s_spill));
+    ctx->spilled = true;
   }
   const bool has_index = ub > 0;
   {
@@ -685,11 +738,16 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
     if (s0.t + 1 > d.Tmax) return LTRI_ECAPACITY;
     for (int l = 0; l < layer_count; ++l) {
       const LayerState& s = ctx->at(sq, layer_begin + l);
-      if (s.t != s0.t || s.E != s0.E) return LTRI_ESTATE;
+      if (s.t != s0.t || s.E != s0.E || s.base != s0.base) return LTRI_ESTATE;
     }
     ub = std::max(ub, s0.span_ub);
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (d.paged)
+    for (int i = 0; i < n_seqs; ++i) {
+      const int rc = slide_window(ctx, seq_ids[i], layer_begin, layer_count, ctx->at(seq_ids[i], layer_begin).t + 1, st);
+      if (rc != LTRI_OK) return rc;
+    }
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
   const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
@@ -716,6 +774,7 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
       b.pos[i] = (int)s.t;
       b.loc_begin[i] = s.E;
       b.src[i] = i0 + i;
+      b.shift[i] = d.paged ? s.base - d.Lsp : 0;
     }
     const int units = b.n * layer_count * d.Hkv;
     // split count of the decode attention: three CTAs fit an SM, so the grid runs in waves of 3 x SMs CTAs.  Among
@@ -854,6 +913,7 @@ int ltri_get_stats(ltri_ctx* ctx, int seq, int layer, ltri_stats* out, void* cud
   out->n_pending_regions = (int)s.pending.size();
   out->index_bytes = (int64_t)n * d.Hkv * kD * 2;
   out->retrieved_tokens = rt;
+  out->slab_slides = s.slides;
   if (!s.pending.empty() && !s.decoding) {
     int cnt = 0;
     rc = copy_back(ctx, &cnt, d.pend_cnt + unit * d.slots + s.pending.back().slot, sizeof(int), st);

@@ -192,12 +192,48 @@ def test_host_memory_pager_is_bit_identical_to_the_resident_path():
                 assert np.array_equal(a.ltri_get_selected(0, l), b.ltri_get_selected(0, l))
             t0 += n
         assert b.ltri_debug_read(binding.BUF_CACHE_STATS, 0, 1)[1] > 0
+        # the paged context keeps sink + a sliding window in device memory: by now the live rows have been moved once
+        assert b.ltri_get_stats(0, 0).slab_slides == 1 and a.ltri_get_stats(0, 0).slab_slides == 0
         for step in range(3):      # decode steps read their units from the cache slots
             q, k, v = (x.permute(1, 0, 2, 3).contiguous().cuda() for x in st.tokens(t0 + step, 1, kind=1))
             assert torch.equal(a.ltri_decode_step([0], 0, 2, q, k, v), b.ltri_decode_step([0], 0, 2, q, k, v))
         a.ltri_reset_sequence(0)
         b.ltri_reset_sequence(0)
         assert (b.ltri_debug_read(binding.BUF_CACHE_TAGS, 0, 0) == -1).all()
+    assert a.ltri_sync_status() == 0 and b.ltri_sync_status() == 0
+    a.close()
+    b.close()
+
+
+def test_sliding_slabs_through_long_decode_and_their_capacity():
+    # a paged context holds sink + window in device memory (2 x (window + 2 chunks) + slack rows): a long decode
+    # slides the slabs once more, stays bit-identical to the resident path, and ends with a capacity error -- not a
+    # fault -- when the tokens since the last eviction no longer fit
+    cfg = small_cfg(n_layers=1, context=640, chunk=64, window=128, n_sink=16, decode_steps=900, unit_tokens=32, top_k=3,
+                    max_spans_per_region=2)
+    paged = dataclasses.replace(cfg, host_kv=True, cache_units=4, score_decay=0.1)
+    pa, pb = ph.params_of(cfg), ph.params_of(paged)
+    assert binding.ltri_arena_bytes(pb) < binding.ltri_arena_bytes(pa)
+    st = inputs.SyntheticStream(cfg)
+    a, b = binding.Ltri(pa), binding.Ltri(pb)
+    for t0, n in st.prefill_chunks():
+        q, k, v = (x.cuda() for x in st.tokens(t0, n))
+        assert torch.equal(a.ltri_prefill_chunk(0, 0, 1, q, k, v), b.ltri_prefill_chunk(0, 0, 1, q, k, v))
+    slides0 = b.ltri_get_stats(0, 0).slab_slides
+    failed_at = None
+    for step in range(cfg.decode_steps):
+        q, k, v = (x.permute(1, 0, 2, 3).contiguous().cuda() for x in st.tokens(cfg.context + step, 1, kind=1))
+        oa = a.ltri_decode_step([0], 0, 1, q, k, v)
+        try:
+            ob = b.ltri_decode_step([0], 0, 1, q, k, v)
+        except binding.LtriError as e:
+            assert e.code == binding.LTRI_ECAPACITY
+            failed_at = step
+            break
+        assert torch.equal(oa, ob), f"decode step {step}"
+    # window region: 2 * (128 + 128) + 256 = 768 rows
+    assert failed_at is not None and failed_at > 256
+    assert b.ltri_get_stats(0, 0).slab_slides == slides0 + 1
     assert a.ltri_sync_status() == 0 and b.ltri_sync_status() == 0
     a.close()
     b.close()
