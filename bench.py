@@ -388,7 +388,11 @@ def run_ltri(args, cfg):
                  "unit_misses": int(hm[1]), "hit_rate": float(hm[0] / max(1, hm[0] + hm[1])),
                  "host_to_device_bytes_per_call": float(hm[1]) * unit_bytes / max(1, len(chunks)),
                  "device_to_host_bytes_per_call": float(L * cfg.n_kv_heads * cfg.chunk * cfg.head_dim * 2 * 2),
-                 "note": "prefill calls of the whole stream; the mirror gets every evicted row once"}
+                 "note": "prefill calls of the whole stream; the mirror gets every evicted row once",
+                 "arena_bytes": int(lt.arena_bytes), "slab_slides": int(stats.slab_slides)}
+        p_res = binding.LtriParams.from_buffer_copy(p)
+        p_res.flags &= ~binding.FLAG_HOST_KV
+        pager["resident_arena_bytes"] = int(binding.ltri_arena_bytes(p_res))
     recall = {"final_chunk": needle_recall(lt, st, SQ, cfg)} if cfg.needle and rank == 0 else None
     ms = max_over_ranks(ms, world, dev)
     tokens = K * n

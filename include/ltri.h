@@ -137,9 +137,12 @@ enum {
    * (sequence, layer, KV head)'s unit cache is read from there; a missing one is pulled from host_kv over the bus by
    * the top-k kernel itself, into the slot of the unit with the lowest usage score.  Prefill calls pack the units'
    * rows from the cache slots (the unit the indexed range ends in, while still growing, straight from the mirror);
-   * decode steps attend over the cache slots in place.  Results are bit-identical to the default path.  In this
-   * version the device slabs still hold every token (sink and local window are read from them at absolute
-   * positions), so the flag exercises the whole data path of the pager but does not yet shrink the device footprint. */
+   * decode steps attend over the cache slots in place.  Results are bit-identical to the default path.
+   * The device then keeps, per (sequence, layer, KV head), only the sink and a sliding window of
+   * 2 * (window + 2 * chunk) + 256 rows instead of max_tokens rows: when the window region is full the rows since the
+   * last eviction are moved to its start (ltri_stats.slab_slides counts these moves).  Decode never evicts, so a
+   * sequence can take about window + 2 * chunk decode steps beyond that before ltri_decode_step returns
+   * LTRI_ECAPACITY.  Needs the tensor-core kernels. */
   LTRI_FLAG_HOST_KV = 16
 };
 
