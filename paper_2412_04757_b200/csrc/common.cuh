@@ -70,8 +70,8 @@ struct DevCtx {
   int* ctag;                    // [NS][NL][Hkv][cache_units]  unit held by the slot, -1 empty
   float* cscore;                // [NS][NL][Hkv][cache_units]  usage score
   unsigned long long* cstat;    // [NS][NL][2]  hits, misses
-  long long* rng_koff;          // [NS*NL][Hkv][rcap]  decode: row of a range's first token, relative to Kc
-  long long* rng_voff;          //                     and relative to Vc (slab rows or unit-cache rows)
+  int* rng_koff;                // [NS*NL][Hkv][rcap]  decode: K row of a range's first token, counted from Kc (a slab
+                                //                     row or a unit-cache row; the V row follows from it)
   // per-layer tables of the paper's configuration appendix (nullptr: the scalar holds for every layer)
   const float* theta_l;  // [NL]  theta
   const int* phi_l;      // [NL]  NMS IoU threshold in thousandths

@@ -34,8 +34,9 @@ template <int G>
 __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevCtx c, DecBatch b, int layer_begin, int layer_count,
                                                                 const __nv_bfloat16* __restrict__ q, int nsplit) {
   extern __shared__ __align__(1024) unsigned char dsm[];
+  // rs: first token of every range -- in a paged context (host-memory pager) its first K row, counted from the start
+  // of the K slabs, instead: there a range lives in a sliding slab or in a slot of the unit cache
   __shared__ int rs[kMaxRanges], rp[kMaxRanges + 1];
-  __shared__ long long rko[kMaxRanges], rvo[kMaxRanges];  // host-memory pager: first K / V row of every range
   __shared__ float sm_m[4][G], sm_l[4][G];
   __shared__ float sm_o[4][G][kD];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -47,11 +48,7 @@ __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevC
   if (tid == 0) {
     int run = 0;
     for (int i = 0; i < nr; ++i) {
-      rs[i] = c.rng_start[rb + i];
-      if (c.host_kv) {
-        rko[i] = c.rng_koff[rb + i];
-        rvo[i] = c.rng_voff[rb + i];
-      }
+      rs[i] = c.host_kv ? (int)c.rng_koff[rb + i] : c.rng_start[rb + i];
       rp[i] = run;
       run += c.rng_len[rb + i];
     }
@@ -77,6 +74,8 @@ __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevC
   // (resident contexts: row = token; paged contexts address every range through rko / rvo below)
   const __nv_bfloat16* Kslab = c.Kc + (unit * c.Hkv + g) * (size_t)c.SR * kD;
   const __nv_bfloat16* Vslab = c.Vc + (unit * c.Hkv + g) * (size_t)c.SR * kD;
+  const size_t cache_k0 = c.host_kv ? (size_t)((c.Kcache - c.Kc) / kD) : 0;
+  const size_t cache_dv = c.host_kv ? (size_t)((c.Vcache - c.Vc) / kD) - cache_k0 : 0;
   const uint32_t wbase = smem_u32(dsm) + warp * kDWarpBytes;
   const float c2 = c.scale * kLog2eD;
 
@@ -98,9 +97,11 @@ __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevC
       }
       const __nv_bfloat16* kp = Kslab + tok * kD;
       const __nv_bfloat16* vp = Vslab + tok * kD;
-      if (c.host_kv && okr) {  // the range may live in the unit cache: its rows are addressed from the slab bases
-        kp = c.Kc + (size_t)(rko[ri] + (v - rp[ri])) * kD;
-        vp = c.Vc + (size_t)(rvo[ri] + (v - rp[ri])) * kD;
+      if (c.host_kv) {
+        // tok is a K row counted from c.Kc; its V row has the same number counted from c.Vc inside the slabs and is
+        // cache_dv rows further inside the unit caches
+        kp = c.Kc + tok * kD;
+        vp = c.Vc + (tok >= cache_k0 ? tok + cache_dv : tok) * kD;
       }
       cp_async16(sk + tile_off(row, ch), kp + ch * 8, okr ? 16 : 0);
       cp_async16(sv + tile_off(row, ch), vp + ch * 8, okr ? 16 : 0);

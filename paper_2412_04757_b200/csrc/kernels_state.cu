@@ -1054,7 +1054,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
   __shared__ int s_rs[kMaxRanges], s_rl[kMaxRanges], s_pre[kMaxRanges + 1], s_nr;  // merged ranges, packed-row prefix
   __shared__ int s_sst[2 * kMaxTopK], s_sln[2 * kMaxTopK];  // extents of the selected spans
   __shared__ int s_all[2 * kMaxTopK], s_nall;            // decode: this step's selection united with the persistent one
-  __shared__ long long s_ko[kMaxRanges], s_vo[kMaxRanges];  // pager, decode: first K / V row of every range
+  __shared__ int s_ko[kMaxRanges];  // pager, decode: first K row of every range, counted from the start of the K slabs
   const int g = blockIdx.x;
   int layer, sq, pos = 0, loc_begin = 0;
   if (DECODE) {
@@ -1239,7 +1239,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     int nr = 0;
     long long tokens = 0;
     // under the pager a decode step reads every named unit from its cache slot, so the units stay ranges of their own
-    // and every range carries the row it starts at, relative to the K slabs / the V slabs (s_ko, s_vo)
+    // and every range carries the K row it starts at, counted from the start of the K slabs (the V row follows from it)
     const bool paged = DECODE && c.host_kv;
     const long long slab0 = (long long)((unit * c.Hkv + g) * (size_t)c.SR);
     auto push = [&](int st, int ln, int slot) {
@@ -1253,10 +1253,9 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
           if (slot >= 0) {
             const long long crow =
                 (long long)(((unit * c.Hkv + g) * (size_t)c.cache_units + slot) * (size_t)U) + (st - (st / U) * U);
-            s_ko[nr] = (long long)((c.Kcache - c.Kc) / kD) + crow;
-            s_vo[nr] = (long long)((c.Vcache - c.Vc) / kD) + crow;
+            s_ko[nr] = (int)((long long)((c.Kcache - c.Kc) / kD) + crow);
           } else {
-            s_ko[nr] = s_vo[nr] = slab0 + slab_row(c, st, DECODE ? b.shift[blockIdx.y / layer_count] : 0);
+            s_ko[nr] = (int)(slab0 + slab_row(c, st, DECODE ? b.shift[blockIdx.y / layer_count] : 0));
           }
         }
         ++nr;
@@ -1285,10 +1284,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     for (int t = tid; t < s_nr; t += nt) {
       c.rng_start[rb + t] = s_rs[t];
       c.rng_len[rb + t] = s_rl[t];
-      if (DECODE && c.host_kv) {
-        c.rng_koff[rb + t] = s_ko[t];
-        c.rng_voff[rb + t] = s_vo[t];
-      }
+      if (DECODE && c.host_kv) c.rng_koff[rb + t] = s_ko[t];
     }
   }
   if (!DECODE && c.host_kv) {

@@ -163,8 +163,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.ctag = cv.take<int>(d.host_kv ? units * d.Hkv * d.cache_units : 0);
   d.cscore = cv.take<float>(d.host_kv ? units * d.Hkv * d.cache_units : 0);
   d.cstat = cv.take<unsigned long long>(d.host_kv ? units * 2 : 0);
-  d.rng_koff = cv.take<long long>(d.host_kv ? units * d.Hkv * d.rcap : 0);
-  d.rng_voff = cv.take<long long>(d.host_kv ? units * d.Hkv * d.rcap : 0);
+  d.rng_koff = cv.take<int>(d.host_kv ? units * d.Hkv * d.rcap : 0);
   d.votes = cv.take<long long>(units * d.Tpad);
   d.span_start = cv.take<int>(units * d.cap);
   d.span_len = cv.take<int>(units * d.cap);
@@ -406,7 +405,10 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
                 tc_encode_kv_maps(ctx->d, ctx->kv_maps);
   // unfilled tile slots and over-fetched rows must hold finite values: start from an all-zero cache
   const size_t kv_bytes = (size_t)p->max_seqs * p->n_layers * ctx->d.Hkv * (size_t)ctx->d.SR * kD * 2 * sizeof(__nv_bfloat16);
-  if ((!ctx->ret_head.empty() || ctx->d.paged) && !ctx->use_tc) {
+  // (paged decode numbers K rows from the start of the K slabs through the unit caches in 31 bits)
+  const bool rows_fit = !ctx->d.paged ||
+                        (size_t)(ctx->d.Kcache - ctx->d.Kc) / kD + (size_t)(ctx->d.Vcache - ctx->d.Kcache) / kD < (1ull << 31);
+  if (((!ctx->ret_head.empty() || ctx->d.paged) && !ctx->use_tc) || !rows_fit) {
     // retrieval heads are built into the tensor-core map pass only, sliding slabs into the tensor-core kernels only
     ltri_destroy(ctx);
     return LTRI_EINVAL;
