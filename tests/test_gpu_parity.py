@@ -405,14 +405,17 @@ def test_state_and_capacity_errors():
     lt.close()
 
 
-def test_host_buffer_entry_matches_the_device_entry():
+@pytest.mark.parametrize("paged", [False, True])
+def test_host_buffer_entry_matches_the_device_entry(paged):
     # the same stream once through ltri_prefill_chunk (device tensors) and once through ltri_prefill_chunk_host
-    # (pinned host tensors, layer groups pipelined over internal copy streams): identical outputs and state
-    cfg = small_cfg(n_layers=6, context=1152, decode_steps=0)
+    # (pinned host tensors, layer groups pipelined over internal copy streams): identical outputs and state.
+    # paged: the host-entry context also runs the host-memory pager (each layer group spills, slides its slabs and
+    # pulls units on its own), against a resident context on the device entry
+    cfg = small_cfg(n_layers=6, context=1152 if not paged else 1920, decode_steps=0, unit_tokens=64 if paged else 0)
     dev = torch.device("cuda:0")
     st = inputs.SyntheticStream(cfg)
     lt_d = binding.Ltri(ph.params_of(cfg), device=dev)
-    p = ph.params_of(cfg)
+    p = ph.params_of(dataclasses.replace(cfg, host_kv=True, cache_units=5) if paged else cfg)
     p.flags |= binding.FLAG_HOST_STAGING
     lt_h = binding.Ltri(p, device=dev)
     outs_h = []
@@ -431,6 +434,7 @@ def test_host_buffer_entry_matches_the_device_entry():
     for layer in range(cfg.n_layers):
         assert lt_d.ltri_get_spans(0, layer).tolist() == lt_h.ltri_get_spans(0, layer).tolist()
         assert np.array_equal(lt_d.ltri_get_selected(0, layer), lt_h.ltri_get_selected(0, layer))
+        assert lt_h.ltri_get_stats(0, layer).slab_slides == (1 if paged else 0)
     # a context created without the staging flag refuses the host entry
     q, k, v = st.tokens(0, cfg.chunk)
     with pytest.raises(binding.LtriError):
