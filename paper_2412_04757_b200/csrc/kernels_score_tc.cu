@@ -16,11 +16,14 @@ namespace ltri {
 using namespace tc;
 
 constexpr int kScThreads = 192;
-constexpr int kScStages = 3;
+// index-tile stages: two when the representatives are small enough for two CTAs to share an SM (one CTA's prologue
+// -- splitting the representatives -- then overlaps the other's stream), three when only one CTA fits
 constexpr int kScMaxN = 96;  // padded query-span count the kernel supports
 
-__global__ void __launch_bounds__(kScThreads, 1)
-    k_score_tc(DevCtx c, int seq, int layer_begin, int tiles_per_cta, const __grid_constant__ CUtensorMap kr_map) {
+template <int kScStages>
+__global__ void __launch_bounds__(kScThreads, kScStages == 2 ? 2 : 1)
+    k_score_tc(DevCtx c, int seq, int layer_begin, int tiles_per_cta, int npad_lay,
+               const __grid_constant__ CUtensorMap kr_map) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * kScStages + 4];  // AFULL[3] AEMPTY[3] SFULL[2] SEMPTY[2]
   __shared__ uint32_t s_tmem_base;
@@ -38,8 +41,9 @@ __global__ void __launch_bounds__(kScThreads, 1)
   const int Npad = max(16, (J + 15) & ~15);
   const uint32_t sbase = (smem_addr(smem_raw) + 1023u) & ~1023u;
   const uint32_t sA = sbase;                          // kScStages x 32 KB: [half d][128 spans][64]
-  const uint32_t sU = sbase + kScStages * 32768;      // 3 terms x [half d][kScMaxN rows][64]
-  constexpr uint32_t kTermBytes = 2 * kScMaxN * 128;
+  const uint32_t sU = sbase + kScStages * 32768;      // 3 terms x [half d][npad_lay rows][64]
+  const uint32_t kHalfBytes = (uint32_t)npad_lay * 128;  // npad_lay: the context's largest padded query-span count
+  const uint32_t kTermBytes = 2 * kHalfBytes;
   enum { B_AFULL = 0, B_AEMPTY = kScStages, B_SFULL = 2 * kScStages, B_SEMPTY = 2 * kScStages + 2 };
   auto bar = [&](int i) { return smem_addr(&bars[i]); };
   volatile int* abortp = &s_abort;
@@ -69,7 +73,7 @@ __global__ void __launch_bounds__(kScThreads, 1)
 #pragma unroll
         for (int e = 0; e < 8; ++e) f[e] = 0.f;
       }
-      const uint32_t off = (uint32_t)(ch >> 3) * (kScMaxN * 128) + (uint32_t)j * 128 + (uint32_t)(((ch & 7) ^ (j & 7)) << 4);
+      const uint32_t off = (uint32_t)(ch >> 3) * kHalfBytes + (uint32_t)j * 128 + (uint32_t)(((ch & 7) ^ (j & 7)) << 4);
 #pragma unroll
       for (int t = 0; t < 3; ++t) {
         uint32_t w[4];
@@ -133,7 +137,7 @@ __global__ void __launch_bounds__(kScThreads, 1)
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             const uint32_t kin = (ks & 3) * 32;
-            mma_ss(tmem + buf * 128, da + (((ks >> 2) * 16384 + kin) >> 4), db + (((ks >> 2) * (kScMaxN * 128) + kin) >> 4),
+            mma_ss(tmem + buf * 128, da + (((ks >> 2) * 16384 + kin) >> 4), db + (((ks >> 2) * kHalfBytes + kin) >> 4),
                    idesc, !(t == 2 && ks == 0));
           }
         }
@@ -182,12 +186,21 @@ cudaError_t launch_score_prefill_tc(const DevCtx& c, const PrefillArgs& a, int s
   if (!score_tc_supported(c) || !kv_maps) return cudaErrorNotSupported;
   CUtensorMap kr;
   memcpy(&kr, static_cast<const CUtensorMap*>(kv_maps) + 5, sizeof(kr));
-  const int smem = kScStages * 32768 + 3 * 2 * kScMaxN * 128 + 1024;
-  cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const int npad_lay = max(16, (c.Jmax + 15) & ~15);
+  const int rep_bytes = 3 * 2 * npad_lay * 128 + 1024;
+  const bool two = 2 * (2 * 32768 + rep_bytes + 1024) <= 227 * 1024;  // two CTAs (with their reserved KB) per SM
+  const int smem = (two ? 2 : 3) * 32768 + rep_bytes;
   const int tiles = (span_bound + 127) / 128;
   const int per_cta = tiles >= 256 ? 32 : (tiles >= 48 ? 16 : 8);  // amortise the split of the representatives
   const int gx = (tiles + per_cta - 1) / per_cta;
-  k_score_tc<<<dim3(gx > 0 ? gx : 1, c.Hkv, a.layer_count), kScThreads, smem, s>>>(c, a.seq, a.layer_begin, per_cta, kr);
+  const dim3 grid(gx > 0 ? gx : 1, c.Hkv, a.layer_count);
+  if (two) {
+    cudaFuncSetAttribute(k_score_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    k_score_tc<2><<<grid, kScThreads, smem, s>>>(c, a.seq, a.layer_begin, per_cta, npad_lay, kr);
+  } else {
+    cudaFuncSetAttribute(k_score_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    k_score_tc<3><<<grid, kScThreads, smem, s>>>(c, a.seq, a.layer_begin, per_cta, npad_lay, kr);
+  }
   return cudaGetLastError();
 }
 
