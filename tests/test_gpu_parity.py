@@ -298,18 +298,24 @@ def test_irregular_call_sizes_and_single_token_calls():
     print(sp.rep)
 
 
-def test_batched_decode_independent_sequences():
-    cfg = small_cfg(n_layers=2, n_seqs=3, context=768, decode_steps=4)
+@pytest.mark.parametrize("paged", [False, True])
+def test_batched_decode_independent_sequences(paged):
+    # paged: every sequence has its own unit caches and its own sliding slabs (sequence 0 is long enough to slide once,
+    # the others are not), and a batched decode step carries one row shift per sequence
+    kw = dict(unit_tokens=32, host_kv=True, cache_units=5, window=128, chunk=64, context=1024) if paged else {}
+    cfg = small_cfg(**{**dict(n_layers=2, n_seqs=3, context=768, decode_steps=4), **kw})
     sp = ph.StreamPair(cfg, layers=[0, 1], seqs=[0, 1, 2])
     streams = [inputs.SyntheticStream(cfg, seq=s) for s in range(3)]
     for s, st in enumerate(streams):
-        upto = cfg.context - 128 * s          # different lengths per sequence
+        upto = cfg.context - (128 if not paged else 320) * s          # different lengths per sequence
         for t0, n in st.prefill_chunks():
             if t0 >= upto:
                 break
             q, k, v = st.tokens(t0, n)
             sp.prefill(s, q, k, v, check_out=(t0 + n >= upto))
-    lens = [cfg.context - 128 * s for s in range(3)]
+    lens = [cfg.context - (128 if not paged else 320) * s for s in range(3)]
+    if paged:
+        assert [sp.lt.ltri_get_stats(s, 0).slab_slides for s in range(3)] == [1, 0, 0]
     for step in range(cfg.decode_steps):
         qs, ks, vs = [], [], []
         for s, st in enumerate(streams):
