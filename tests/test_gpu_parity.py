@@ -187,7 +187,7 @@ def test_host_memory_pager_is_bit_identical_to_the_resident_path():
             q, k, v = (x.cuda() for x in st.tokens(t0, n))
             oa = a.ltri_prefill_chunk(0, 0, 2, q, k, v)
             ob = b.ltri_prefill_chunk(0, 0, 2, q, k, v)
-            assert torch.equal(oa, ob), f"round {rnd} call at {t0}"
+            assert torch.equal(oa, ob), f"pass {rnd} call at {t0}"
             for l in range(2):
                 assert np.array_equal(a.ltri_get_selected(0, l), b.ltri_get_selected(0, l))
             t0 += n
