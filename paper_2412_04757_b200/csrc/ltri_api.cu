@@ -529,12 +529,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   }
   if (s0.t + n_tokens > d.Tmax) return LTRI_ECAPACITY;
   const int t0 = (int)s0.t;
-  cudaStream_t st0 = static_cast<cudaStream_t>(cuda_stream);
-  if (d.paged) {
-    const int rc = slide_window(ctx, seq, layer_begin, layer_count, t0 + n_tokens, st0);
-    if (rc != LTRI_OK) return rc;
-  }
-  const long long shift = d.paged ? s0.base - d.Lsp : 0;
+
   // plan the evictions (host knows region boundaries; span counts live on the device)
   std::vector<Region> ev;
   int E = s0.E;
@@ -575,12 +570,18 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   a.reg_start = reg_start;
   a.m = m;
   a.slot = slot;
-  a.shift = shift;
   a.q = static_cast<const __nv_bfloat16*>(q);
   a.k = static_cast<const __nv_bfloat16*>(k);
   a.v = static_cast<const __nv_bfloat16*>(v);
   a.out = static_cast<__nv_bfloat16*>(out);
 
+  // every host-side check has passed: from here on work is enqueued
+  if (d.paged) {
+    const int rc = slide_window(ctx, seq, layer_begin, layer_count, t0 + n_tokens, st);
+    if (rc != LTRI_OK) return rc;
+  }
+  const long long shift = d.paged ? s0.base - d.Lsp : 0;
+  a.shift = shift;
   {
     Scope sc(ctx, st, LTRI_K_APPEND, 1);
     LTRI_CUDA(ctx, launch_append_prefill(d, a, st));
