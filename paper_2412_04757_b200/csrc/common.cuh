@@ -165,7 +165,7 @@ cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_be
                                 const __nv_bfloat16* q, int span_bound, cudaStream_t s);
 // decode scores + top-k + range list in one launch (span_bound <= dec_retrieve_fused_max_spans())
 cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count,
-                                      const __nv_bfloat16* q, int span_bound, bool force_cluster, cudaStream_t s);
+                                      const __nv_bfloat16* q, int span_bound, bool force_cluster, int threads, cudaStream_t s);
 int dec_retrieve_fused_max_spans();
 cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s);
 

@@ -1400,7 +1400,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   __syncthreads();
   // ---- scores
   {
-    const int hw = tid >> 4, hl = tid & 15;  // 64 half-warps
+    const int hw = tid >> 4, hl = tid & 15, nhw = nt >> 4;  // half-warps of the CTA (the launch picks its size)
     float uf[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
@@ -1409,14 +1409,14 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     auto fetch = [&](int base, uint4 (&raw)[4]) {
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
-        const int s = base + t * 64 + hw;
+        const int s = base + t * nhw + hw;
         raw[t] = s < N ? __ldg(reinterpret_cast<const uint4*>(KR + (size_t)s * kD)) : make_uint4(0, 0, 0, 0);
       }
     };
     uint4 cur[4], nxt[4];
     fetch(0, cur);
-    for (int base = 0; base < N; base += 64 * 4) {  // uniform trip count (shuffles inside)
-      fetch(base + 64 * 4, nxt);                    // past the end: zeros, no loads
+    for (int base = 0; base < N; base += nhw * 4) {  // uniform trip count (shuffles inside)
+      fetch(base + nhw * 4, nxt);                    // past the end: zeros, no loads
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&cur[t]);
@@ -1431,7 +1431,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
         d += __shfl_xor_sync(0xffffffffu, d, 2);
         d += __shfl_xor_sync(0xffffffffu, d, 4);
         d += __shfl_xor_sync(0xffffffffu, d, 8);
-        const int s = base + t * 64 + hw;
+        const int s = base + t * nhw + hw;
         if (hl == 0 && s < N) ssc[s] = d;
       }
 #pragma unroll
@@ -1783,11 +1783,12 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
 }
 
 cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count,
-                                      const __nv_bfloat16* q, int span_bound, bool force_cluster, cudaStream_t s) {
+                                      const __nv_bfloat16* q, int span_bound, bool force_cluster, int threads,
+                                      cudaStream_t s) {
   span_bound = max(span_bound, 1);
   if (span_bound <= kFusedMaxSpans && !force_cluster) {  // one CTA per head: no cluster barriers
-    k_dec_retrieve<<<dim3(c.Hkv, b.n * layer_count), 1024, (int)sizeof(float) * span_bound, s>>>(c, layer_begin, b,
-                                                                                                 layer_count, q);
+    k_dec_retrieve<<<dim3(c.Hkv, b.n * layer_count), threads, (int)sizeof(float) * span_bound, s>>>(c, layer_begin, b,
+                                                                                                    layer_count, q);
     return cudaGetLastError();
   }
   const int per = (span_bound + kRetCluster - 1) / kRetCluster;
