@@ -8,7 +8,9 @@
 // heads of a token are adjacent columns, so their sum (Eq. 4) is thread-local too and goes to the region map with one
 // integer reduction per (token, key, KV head).  Roles: warps 0-15 epilogue (four warps per lane quarter, 32 columns
 // each), warp 16 TMA producer, warp 17 MMA issuer; four TMEM accumulators and two Q stages overlap the MMAs with the
-// exp/round epilogue, which is bound by the special-function unit (one ex2 per map entry).
+// exp/round epilogue, which is bound by the special-function unit (one ex2 per map entry).  The rows' softmax
+// offsets ride along in the contraction (a ninth K step against a tile of ones), so the epilogue is one multiply,
+// one ex2, one fused scale-and-round and one integer add per entry, with no per-column operand to fetch.
 #include <cuda.h>
 
 #include <cstring>
@@ -56,7 +58,6 @@ __global__ void __launch_bounds__(kMapThreads, 1)
   __shared__ __align__(8) unsigned long long bars[1 + 4 + 8];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ __align__(16) float s_stats[16][2][32];  // per epilogue warp: offsets of its 32 columns, two blocks
   constexpr int TPB = 128 / G;  // tokens per query block
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = blockIdx.y, l = blockIdx.z, layer = a.layer_begin + l;
@@ -79,6 +80,13 @@ __global__ void __launch_bounds__(kMapThreads, 1)
   const uint32_t sbase = (smem_addr(smem_raw) + 1023u) & ~1023u;
   const uint32_t sK = sbase;                      // kMapKT x 32 KB: [tile][half d][128 keys][64]
   const uint32_t sQ = sbase + kMapKT * 32768;     // 2 stages x 32 KB: [half d][128 rows][64]
+  // One more step of the contraction carries the rows' offsets (see kMapMargin): the key side is a constant tile of
+  // ones, the query side holds off / c2 of the block's 128 rows split into four bf16 terms, so the accumulator comes
+  // out as logit + off / c2 and the epilogue needs no per-column offsets.  Both are 128 x 16 K-major tiles without
+  // swizzle: 8-row x 16-byte core matrices, the two core matrices of a row group 128 bytes apart, row groups 256.
+  const uint32_t sXa = sQ + 65536;                // 4 KB
+  const uint32_t sXb = sXa + 4096;                // 2 stages x 4 KB
+  auto xoff = [](int r, int kc) -> uint32_t { return (uint32_t)((r >> 3) * 256 + kc * 128 + (r & 7) * 16); };
   enum { B_KFULL = 0, B_QFULL = 1, B_QEMPTY = 3, B_SFULL = 5, B_SEMPTY = 9 };
   auto bar = [&](int i) { return smem_addr(&bars[i]); };
   volatile int* abortp = &s_abort;
@@ -95,6 +103,16 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     }
     fence_mbar_init();
   }
+  if (tid < 256) {  // ones in the first four K slots of every key row, zeros behind them; the query side's second
+    const int r = tid >> 1, kc = tid & 1;  // core matrix (K slots 8..15) stays zero for good
+    const uint32_t one2 = kc == 0 ? 0x3F803F80u : 0u;
+    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%2,%2};" ::"r"(sXa + xoff(r, kc)), "r"(one2), "r"(0u) : "memory");
+    if (kc == 1) {
+      asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(sXb + xoff(r, 1)), "r"(0u) : "memory");
+      asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(sXb + 4096 + xoff(r, 1)), "r"(0u) : "memory");
+    }
+  }
+  fence_async_smem();
   if (warp == 16) tmem_alloc(smem_addr(&s_tmem_base), 512);
   fence_before_sync();
   __syncthreads();
@@ -110,25 +128,60 @@ __global__ void __launch_bounds__(kMapThreads, 1)
         tma_load_2d(sK + kt * 32768, &maps.k128, 0, (int)krow, bar(B_KFULL));
         tma_load_2d(sK + kt * 32768 + 16384, &maps.k128, 64, (int)krow, bar(B_KFULL));
       }
-      bool ok = true;
-      int it = 0;
-      for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
-        const int st = it & 1;
-        if (it >= 2) ok = mbar_wait(bar(B_QEMPTY + st), ((it >> 1) - 1) & 1, abortp);
-        if (!ok) break;
+    }
+    // every lane writes the offsets of four of the block's 128 rows (row = (token, head)); lane 0 then starts the
+    // copies of the block's queries, whose barrier also publishes the offsets
+    const float* rq = c.rowq + (size_t)layer * c.chunk * c.Hq + g * G;
+    const float inv_c2 = 1.0f / (c.scale * kLog2eM);
+    int ok = 1;
+    int it = 0;
+    for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
+      const int st = it & 1;
+      if (lane == 0 && it >= 2) ok = mbar_wait(bar(B_QEMPTY + st), ((it >> 1) - 1) & 1, abortp) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int row = lane + 32 * i;
+        const int tk = blk * TPB + row / G;
+        // rows past the call's end, and (under a retrieval head) the other heads' rows, get an offset that sends
+        // every entry to zero
+        float v = -30000.f;
+        if (tk < a.n && (rh < 0 || g * G + row % G == rh)) v = fmaxf(__ldg(rq + (size_t)tk * c.Hq + row % G) * inv_c2, -30000.f);
+        uint32_t w[2];
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(v);
+          v -= __bfloat162float(h0);
+          const __nv_bfloat16 h1 = __float2bfloat16_rn(v);
+          v -= __bfloat162float(h1);
+          __nv_bfloat162 pr;
+          pr.x = h0;
+          pr.y = h1;
+          w[t] = *reinterpret_cast<uint32_t*>(&pr);
+        }
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%3};" ::"r"(sXb + st * 4096 + xoff(row, 0)), "r"(w[0]), "r"(w[1]),
+                     "r"(0u)
+                     : "memory");
+      }
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) {
         mbar_expect_tx(bar(B_QFULL + st), 32768);
         tma_load_3d(sQ + st * 32768, &maps.q, 0, g * G, l * a.n + blk * TPB, bar(B_QFULL + st));
         tma_load_3d(sQ + st * 32768 + 16384, &maps.q, 64, g * G, l * a.n + blk * TPB, bar(B_QFULL + st));
       }
+    }
+    if (lane == 0)
       for (int back = 1; back <= 2 && back <= it; ++back) {  // no copy may be in flight at exit
         const int ii = it - back;
         if (!mbar_wait(bar(B_QEMPTY + (ii & 1)), (ii >> 1) & 1, abortp)) break;
       }
-    }
   } else if (warp == 17) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(128, 128, false);
       const uint64_t dK = make_desc(sK, 16, 1024), dQ = make_desc(sQ, 16, 1024);
+      const uint64_t dXa = make_desc_noswizzle(sXa, 128, 256), dXb = make_desc_noswizzle(sXb, 128, 256);
       bool ok = mbar_wait(bar(B_KFULL), 0, abortp);
       int it = 0, seq = 0;
       for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
@@ -148,6 +201,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
             const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
             mma_ss(tmem + buf * 128, da + off, db + off, idesc, ks > 0);
           }
+          mma_ss(tmem + buf * 128, dXa, dXb + (uint64_t)((st * 4096) >> 4), idesc, true);  // + off / c2 per column
           mma_commit(bar(B_SFULL + buf));
           ++seq;
         }
@@ -161,19 +215,8 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     const int krel = (warp & 3) * 32 + lane;  // key inside its tile
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float c2 = c.scale * kLog2eM;
-    const float* rq = c.rowq + (size_t)layer * c.chunk * c.Hq + g * G;
     int* Mq = c.Mq + (size_t)layer * c.chunk * c.chunk;
     const int roff = a.t0 - a.reg_start;      // region index = call-relative token + roff
-    // per-row offsets (see kMapMargin) of the warp's 32 columns, staged per warp in shared memory one block ahead:
-    // lane e fetches the offset of column e, every lane then reads all 32 back as broadcast vector loads
-    auto load_stats = [&](int blk) -> float {
-      const int col = cq * 32 + lane;
-      const int tk = blk * TPB + col / G;
-      return tk < a.n && (rh < 0 || g * G + col % G == rh) ? __ldg(rq + (size_t)tk * c.Hq + col % G) : -INFINITY;
-    };
-    float* my_stats = &s_stats[warp][0][0];
-    if (bmin < nblocks) my_stats[lane] = load_stats(bmin);
-    __syncwarp();
     long long total[kMapKT];
 #pragma unroll
     for (int kt = 0; kt < kMapKT; ++kt) total[kt] = 0;
@@ -182,12 +225,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     const float2 c2v = make_float2(c2, c2);
     const float2 sc = make_float2(kMapScale, kMapScale), mg = make_float2(12582912.f, 12582912.f);
     for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
-      const int st = it & 1;
-      const bool more = blk + 1 < nblocks;
-      float nxt = -INFINITY;
-      if (more) nxt = load_stats(blk + 1);
       const int tokb = blk * TPB;  // first token of the block (call-relative)
-      const float* ss = my_stats + st * 32;
 #pragma unroll
       for (int kt = 0; kt < kMapKT; ++kt) {
         if (kt >= ntile || blk < blk0_of(kt)) continue;
@@ -213,17 +251,11 @@ __global__ void __launch_bounds__(kMapThreads, 1)
           uint32_t bsum = 0;
 #pragma unroll
           for (int e8 = 0; e8 < 32; e8 += 8) {
-            const float4 o0 = *reinterpret_cast<const float4*>(ss + e8);
-            const float4 o1 = *reinterpret_cast<const float4*>(ss + e8 + 4);
-            float2 x[4];
-            x[0] = __ffma2_rn(make_float2(__uint_as_float(v[e8]), __uint_as_float(v[e8 + 1])), c2v,
-                              make_float2(o0.x, o0.y));
-            x[1] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 2]), __uint_as_float(v[e8 + 3])), c2v,
-                              make_float2(o0.z, o0.w));
-            x[2] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 4]), __uint_as_float(v[e8 + 5])), c2v,
-                              make_float2(o1.x, o1.y));
-            x[3] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 6]), __uint_as_float(v[e8 + 7])), c2v,
-                              make_float2(o1.z, o1.w));
+            float2 x[4];  // (the accumulator already holds logit + off / c2)
+            x[0] = __fmul2_rn(make_float2(__uint_as_float(v[e8]), __uint_as_float(v[e8 + 1])), c2v);
+            x[1] = __fmul2_rn(make_float2(__uint_as_float(v[e8 + 2]), __uint_as_float(v[e8 + 3])), c2v);
+            x[2] = __fmul2_rn(make_float2(__uint_as_float(v[e8 + 4]), __uint_as_float(v[e8 + 5])), c2v);
+            x[3] = __fmul2_rn(make_float2(__uint_as_float(v[e8 + 6]), __uint_as_float(v[e8 + 7])), c2v);
             {
               uint32_t part = 0u - 8u * 0x4B400000u;
 #pragma unroll
@@ -246,17 +278,11 @@ __global__ void __launch_bounds__(kMapThreads, 1)
         int aq[32];
 #pragma unroll
         for (int e8 = 0; e8 < 32; e8 += 8) {
-          const float4 o0 = *reinterpret_cast<const float4*>(ss + e8);
-          const float4 o1 = *reinterpret_cast<const float4*>(ss + e8 + 4);
           float2 x[4];
-          x[0] = __ffma2_rn(make_float2(__uint_as_float(v[e8]), __uint_as_float(v[e8 + 1])), c2v,
-                            make_float2(o0.x, o0.y));
-          x[1] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 2]), __uint_as_float(v[e8 + 3])), c2v,
-                            make_float2(o0.z, o0.w));
-          x[2] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 4]), __uint_as_float(v[e8 + 5])), c2v,
-                            make_float2(o1.x, o1.y));
-          x[3] = __ffma2_rn(make_float2(__uint_as_float(v[e8 + 6]), __uint_as_float(v[e8 + 7])), c2v,
-                            make_float2(o1.z, o1.w));
+          x[0] = __fmul2_rn(make_float2(__uint_as_float(v[e8]), __uint_as_float(v[e8 + 1])), c2v);
+          x[1] = __fmul2_rn(make_float2(__uint_as_float(v[e8 + 2]), __uint_as_float(v[e8 + 3])), c2v);
+          x[2] = __fmul2_rn(make_float2(__uint_as_float(v[e8 + 4]), __uint_as_float(v[e8 + 5])), c2v);
+          x[3] = __fmul2_rn(make_float2(__uint_as_float(v[e8 + 6]), __uint_as_float(v[e8 + 7])), c2v);
           // an entry with x < 0 rounds to zero: a group of eight columns whose x is negative on every lane of the
           // warp (common under the causal diagonal) needs no exponentials at all
           const float xm = fmaxf(fmaxf(fmax3(x[0].x, x[0].y, x[1].x), fmax3(x[1].y, x[2].x, x[2].y)),
@@ -290,9 +316,6 @@ __global__ void __launch_bounds__(kMapThreads, 1)
         }
         total[kt] += bsum;
       }
-      __syncwarp();
-      if (more) my_stats[(st ^ 1) * 32 + lane] = nxt;
-      __syncwarp();
     }
     if (ok) {
 #pragma unroll
@@ -342,7 +365,7 @@ static cudaError_t launch_map_tc_g(const DevCtx& c, const PrefillArgs& a, const 
   const int nloc = (a.loc_begin >= c.Ls) ? (a.t0 - a.loc_begin + 127) / 128 : 0;
   const int ncur = (a.n + 127) / 128;
   const int gloc = (nloc + kMapKT - 1) / kMapKT, gcur = (ncur + kMapKT - 1) / kMapKT;
-  const int smem = kMapKT * 32768 + 65536 + 1024;
+  const int smem = kMapKT * 32768 + 65536 + 3 * 4096 + 1024;  // key tiles, two query stages, the offset tiles
   cudaFuncSetAttribute(k_map_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   k_map_tc<G><<<dim3(gloc + gcur, c.Hkv, a.layer_count), kMapThreads, smem, s>>>(c, a, gloc, nloc, ncur, maps);
   return cudaGetLastError();

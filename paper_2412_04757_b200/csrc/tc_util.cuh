@@ -119,6 +119,16 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
   d |= (uint64_t)2 << 61;  // SWIZZLE_128B
   return d;
 }
+// K-major tile without swizzle: 8-row x 16-byte core matrices (128 contiguous bytes each); lbo_bytes = distance
+// between the core matrices of one row group along K, sbo_bytes = distance between row groups.
+__device__ __forceinline__ uint64_t make_desc_noswizzle(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3fff);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3fff) << 32;
+  d |= (uint64_t)1 << 46;  // descriptor version (Blackwell)
+  return d;
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, M x N, optional MN-major B
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major) {
   return (1u << 4)                        // D format f32
