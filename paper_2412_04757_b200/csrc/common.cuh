@@ -76,7 +76,7 @@ struct DevCtx {
   const float* theta_l;  // [NL]  theta
   const int* phi_l;      // [NL]  NMS IoU threshold in thousandths
   const float* lambda_l; // [NL]  lambda of Eq. r_v
-  long long* sel_tokens; // [NS][NL]  retrieved tokens of the last call, summed over KV heads
+  long long* sel_tokens; // [NS][NL][Hkv]  retrieved tokens of the last call
   // per-layer scratch of the prefill call in flight
   int* Mq;               // [NL][chunk][chunk]
   long long* Rsuf;       // [NL][chunk][chunk]
@@ -165,7 +165,8 @@ cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_be
                                 const __nv_bfloat16* q, int span_bound, cudaStream_t s);
 // decode scores + top-k + range list in one launch (span_bound <= dec_retrieve_fused_max_spans())
 cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count,
-                                      const __nv_bfloat16* q, int span_bound, bool force_cluster, int threads, cudaStream_t s);
+                                      const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, int span_bound, bool force_cluster, int threads,
+                                      cudaStream_t s);
 int dec_retrieve_fused_max_spans();
 cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s);
 

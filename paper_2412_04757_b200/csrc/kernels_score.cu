@@ -18,7 +18,6 @@ __global__ void __launch_bounds__(128) k_score_mma(DevCtx c, int seq, int layer_
   const size_t unit = unit_of(c, seq, layer);
   const int N = c.n_spans[unit];
   const int J = c.Jcnt[layer];
-  if (blockIdx.x == 0 && g == 0 && tid == 0) c.sel_tokens[unit] = 0;
   const int ntiles = (N + 63) / 64;
   if ((int)blockIdx.x >= ntiles) return;
   const int njb = (J + 63) / 64;                      // blocks of 64 query spans

@@ -33,7 +33,6 @@ __global__ void __launch_bounds__(kScThreads, kScStages == 2 ? 2 : 1)
   const size_t unit = unit_of(c, seq, layer);
   const int N = c.n_spans[unit];
   const int J = c.Jcnt[layer];
-  if (blockIdx.x == 0 && g == 0 && tid == 0) c.sel_tokens[unit] = 0;
   const int ntiles = (N + 127) / 128;
   const int tile0 = blockIdx.x * tiles_per_cta;
   if (tile0 >= ntiles) return;

@@ -16,8 +16,8 @@ __global__ void k_init(DevCtx c, int seq) {
     const size_t u0 = (size_t)s * c.NL;
     for (size_t i = tid; i < (size_t)c.NL; i += stride) {
       c.n_spans[u0 + i] = 0;
-      c.sel_tokens[u0 + i] = 0;
     }
+    for (size_t i = tid; i < (size_t)c.NL * c.Hkv; i += stride) c.sel_tokens[u0 * c.Hkv + i] = 0;
     for (size_t i = tid; i < (size_t)c.NL * c.slots; i += stride) c.pend_cnt[u0 * c.slots + i] = 0;
     for (size_t i = tid; i < (size_t)c.NL * c.Hkv * c.topk; i += stride) {
       c.sel[u0 * c.Hkv * c.topk + i] = -1;
@@ -109,7 +109,6 @@ __global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer
   }
   if (g == 0 && c16 == 0) {
     c.votes[unit * c.Tpad + b.pos[bi]] = 0;
-    c.sel_tokens[unit] = 0;  // the retrieval kernels of this step add the tokens they select
   }
 }
 
@@ -830,7 +829,6 @@ __global__ void __launch_bounds__(256) k_score(DevCtx c, int seq, int layer_begi
     for (int t = threadIdx.x; t < J * kD; t += blockDim.x) su[t] = up[t];
   }
   const size_t unit = unit_of(c, sq, layer);
-  if (blockIdx.x == 0 && g == 0 && threadIdx.x == 0) c.sel_tokens[unit] = 0;
   __syncthreads();
   const int N = c.n_spans[unit];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -880,7 +878,6 @@ __global__ void __launch_bounds__(256) k_score_dec(DevCtx c, int layer_begin, De
   const int N = c.n_spans[unit];
   // a layer with a retrieval head (Sec. 3.5) scores that head's query against the index of its KV head, for every g
   const int rh = ret_head_of(c, layer), gk = rh >= 0 ? rh / c.G : g;
-  if (blockIdx.x == 0 && g == 0 && tid == 0) c.sel_tokens[unit] = 0;
   const int s0 = blockIdx.x * 256;
   if (s0 >= N) return;
   if (tid < kD) {
@@ -1275,7 +1272,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     s_pre[nr] = run;
     s_nr = nr;
     c.rng_cnt[unit * c.Hkv + g] = nr;
-    atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+    c.sel_tokens[unit * c.Hkv + g] = tokens;  // (summed over the KV heads by ltri_get_stats)
     if (!DECODE) c.gcnt[(size_t)layer * c.Hkv + g] = run;
   }
   __syncthreads();
@@ -1371,8 +1368,26 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
 // top-k there (same radix select as k_topk) and writes the selection and the token ranges of the attention kernel.
 constexpr int kFusedMaxSpans = 12288;  // scores kept in shared memory (48 KB)
 
+// a0 inside the one-launch decode retrieval: the CTA of (sequence, layer, KV head) also stores that head's new K and V
+// row (threads 0-31: sixteen 16-byte pieces each), so a decode step needs no separate append launch.  The attention
+// kernel, launched next, is the first reader of the row.  (Resident contexts only: the one-launch path is never paged.)
+__device__ __forceinline__ void append_decode_row(const DevCtx& c, const DecBatch& b, int bi, int l, int layer_count,
+                                                  size_t unit, int g, const __nv_bfloat16* __restrict__ k,
+                                                  const __nv_bfloat16* __restrict__ v) {
+  const int tid = threadIdx.x;
+  if (tid < 32) {
+    const int c16 = tid & 15;
+    const __nv_bfloat16* src = (tid < 16 ? k : v) + (((size_t)b.src[bi] * layer_count + l) * c.Hkv + g) * kD + c16 * 8;
+    __nv_bfloat16* dst = (tid < 16 ? c.Kc : c.Vc) + ((unit * c.Hkv + g) * (size_t)c.SR + b.pos[bi]) * kD + c16 * 8;
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+    if (g == 0 && tid == 0) c.votes[unit * c.Tpad + b.pos[bi]] = 0;
+  }
+}
+
 __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin, DecBatch b, int layer_count,
-                                                       const __nv_bfloat16* __restrict__ q) {
+                                                       const __nv_bfloat16* __restrict__ q,
+                                                       const __nv_bfloat16* __restrict__ knew,
+                                                       const __nv_bfloat16* __restrict__ vnew) {
   extern __shared__ float ssc[];  // [N]
   __shared__ float su[kD];
   __shared__ unsigned hist[256];
@@ -1389,6 +1404,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   const int tid = threadIdx.x, nt = blockDim.x;
   const int N = min(c.n_spans[unit], kFusedMaxSpans);
   const int rh = ret_head_of(c, layer), gk = rh >= 0 ? rh / c.G : g;  // retrieval head of the layer (Sec. 3.5)
+  append_decode_row(c, b, bi, l, layer_count, unit, g, knew, vnew);
   if (tid < kD) {
     const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + gk * c.G) * kD + tid;
     float acc = 0.f;
@@ -1551,7 +1567,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
     s_nr = nr;
     c.rng_cnt[unit * c.Hkv + g] = nr;
-    atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+    c.sel_tokens[unit * c.Hkv + g] = tokens;  // (summed over the KV heads by ltri_get_stats)
   }
   __syncthreads();
   const size_t rbb = (unit * c.Hkv + g) * (size_t)c.rcap;
@@ -1573,7 +1589,8 @@ constexpr int kRetThreads = 512;
 constexpr int kRetSliceMax = 12288;  // scores a CTA keeps in shared memory (48 KB)
 
 __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThreads)
-    k_dec_retrieve_cl(DevCtx c, int layer_begin, DecBatch b, int layer_count, const __nv_bfloat16* __restrict__ q) {
+    k_dec_retrieve_cl(DevCtx c, int layer_begin, DecBatch b, int layer_count, const __nv_bfloat16* __restrict__ q,
+                      const __nv_bfloat16* __restrict__ knew, const __nv_bfloat16* __restrict__ vnew) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ float ssc[];  // this CTA's slice of the scores
@@ -1597,6 +1614,7 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
   const int per = (N + kRetCluster - 1) / kRetCluster;
   const int lo = min(N, rank * per), hi = min(N, lo + per), nloc = hi - lo;  // this CTA's spans [lo, hi)
   const int rh = ret_head_of(c, layer), gk = rh >= 0 ? rh / c.G : g;  // retrieval head of the layer (Sec. 3.5)
+  if (rank == 0) append_decode_row(c, b, bi, l, layer_count, unit, g, knew, vnew);
   if (tid < kD) {
     const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + gk * c.G) * kD + tid;
     float acc = 0.f;
@@ -1772,7 +1790,7 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
     push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
     s_nr = nr;
     c.rng_cnt[unit * c.Hkv + g] = nr;
-    atomicAdd((unsigned long long*)&c.sel_tokens[unit], (unsigned long long)tokens);
+    c.sel_tokens[unit * c.Hkv + g] = tokens;  // (summed over the KV heads by ltri_get_stats)
   }
   __syncthreads();
   const size_t rbb = (unit * c.Hkv + g) * (size_t)c.rcap;
@@ -1783,18 +1801,18 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
 }
 
 cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count,
-                                      const __nv_bfloat16* q, int span_bound, bool force_cluster, int threads,
-                                      cudaStream_t s) {
+                                      const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                      int span_bound, bool force_cluster, int threads, cudaStream_t s) {
   span_bound = max(span_bound, 1);
   if (span_bound <= kFusedMaxSpans && !force_cluster) {  // one CTA per head: no cluster barriers
-    k_dec_retrieve<<<dim3(c.Hkv, b.n * layer_count), threads, (int)sizeof(float) * span_bound, s>>>(c, layer_begin, b,
-                                                                                                    layer_count, q);
+    k_dec_retrieve<<<dim3(c.Hkv, b.n * layer_count), threads, (int)sizeof(float) * span_bound, s>>>(
+        c, layer_begin, b, layer_count, q, k, v);
     return cudaGetLastError();
   }
   const int per = (span_bound + kRetCluster - 1) / kRetCluster;
   if (per > kRetSliceMax) return cudaErrorInvalidValue;
   k_dec_retrieve_cl<<<dim3(c.Hkv * kRetCluster, b.n * layer_count), kRetThreads, (int)sizeof(float) * per, s>>>(
-      c, layer_begin, b, layer_count, q);
+      c, layer_begin, b, layer_count, q, k, v);
   return cudaGetLastError();
 }
 int dec_retrieve_fused_max_spans() { return kRetCluster * kRetSliceMax; }

@@ -175,7 +175,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.pend_nrep = cv.take<int>(units * (d.slots + 1) * d.Jmax);
   d.sel = cv.take<int>(units * d.Hkv * d.topk);
   d.persist_sel = cv.take<int>(units * d.Hkv * d.topk);
-  d.sel_tokens = cv.take<long long>(units);
+  d.sel_tokens = cv.take<long long>(units * d.Hkv);
   {
     // (carved whether or not a layer has a retrieval head, so that the arena size does not depend on host arrays)
     int* rh = cv.take<int>(d.NL);
@@ -806,10 +806,6 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
       }
       if (ctx->dec_split > 0) nsplit = std::min(ctx->dec_split, kMaxDecSplit);
     }
-    {
-      Scope sc(ctx, st, LTRI_K_APPEND, 1);
-      LTRI_CUDA(ctx, launch_append_decode(d, b, layer_begin, layer_count, n_seqs, kb, vb, st));
-    }
     // retrieval in one launch with the scores in shared memory: one CTA per (sequence, layer, KV head) when there are
     // enough heads to fill the GPU and the index fits one CTA (12K spans), a cluster of eight CTAs per head for a larger
     // index (up to 98K spans); otherwise the scores go through global memory in two launches
@@ -817,13 +813,18 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
     // (unit-granular retrieval ranks units, which only the two-launch path does)
     const bool fused = d.unit == 0 && ub <= dec_retrieve_fused_max_spans() &&
                        (ctx->dec_fused >= 1 || (ctx->dec_fused < 0 && (!one_cta || units >= ctx->sm_count)));
+    if (!fused) {
+      Scope sc(ctx, st, LTRI_K_APPEND, 1);
+      LTRI_CUDA(ctx, launch_append_decode(d, b, layer_begin, layer_count, n_seqs, kb, vb, st));
+    }
     if (fused) {
+      // (the one-launch kernels also store the step's K/V rows: no append launch)
       Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 1);
       // CTA size of the one-CTA kernel: 1024 threads fit once per SM, 512 twice; with more CTAs than SMs the smaller
       // size keeps all of them resident instead of running a second, partly empty wave
       int ret_threads = units > ctx->sm_count ? 512 : 1024;
       if (ctx->dec_ret_threads > 0) ret_threads = ctx->dec_ret_threads;
-      LTRI_CUDA(ctx, launch_dec_retrieve_fused(d, b, layer_begin, layer_count, qb, (int)ub, ctx->dec_fused == 2,
+      LTRI_CUDA(ctx, launch_dec_retrieve_fused(d, b, layer_begin, layer_count, qb, kb, vb, (int)ub, ctx->dec_fused == 2,
                                                ret_threads, st));
     } else {
       Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, d.vote ? 3 : 2);
@@ -918,7 +919,11 @@ int ltri_get_stats(ltri_ctx* ctx, int seq, int layer, ltri_stats* out, void* cud
   long long rt = 0;
   int rc = copy_back(ctx, &n, d.n_spans + unit, sizeof(int), st);
   if (rc) return rc;
-  rc = copy_back(ctx, &rt, d.sel_tokens + unit, sizeof(long long), st);
+  {
+    std::vector<long long> per_head(d.Hkv, 0);
+    rc = copy_back(ctx, per_head.data(), d.sel_tokens + unit * d.Hkv, (size_t)d.Hkv * sizeof(long long), st);
+    for (long long v : per_head) rt += v;
+  }
   if (rc) return rc;
   out->tokens = s.t;
   out->evicted_end = s.E;
