@@ -232,33 +232,66 @@ def run_reference(args, cfg):
     steps = max(1, min(args.steps, 4))
     warm = min(args.warmup, 1)
     toks, cores, sample, per = oracle_sample(cfg, steps, warm)
+    # a step of this arm is what the oracle was actually timed on: one 512-token call of ONE layer; the all-layer
+    # figure is that time x layers and lives in `value` / `sample` only
     line = {
         "impl": "reference", "metric": METRIC, "value": toks, "unit": "tok/s", "n_gpus": args.gpus,
-        "steps": steps, "warmup": warm, "ms_per_step": per * cfg.n_layers * 1e3, "higher_is_better": True,
+        "steps": steps, "warmup": warm, "ms_per_step": per * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": cfg.name, "chunk": cfg.chunk, "window": cfg.window, "top_k": cfg.top_k},
+        "config": {**workload_config(cfg, 1, 1), "timed": "layer 0 only; value = chunk / (ms_per_step x layers)"},
         "cpu_baseline": {"value": toks, "unit": "tok/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": toks, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
 
 
+def workload_config(cfg, world, nseq):
+    return {"workload": cfg.name, "layers": cfg.n_layers, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
+            "context": cfg.context, "chunk": cfg.chunk, "window": cfg.window, "sink": cfg.n_sink, "top_k": cfg.top_k,
+            "parallelism": "replicas only" if world > 1 else "single GPU", "sequences": nseq}
+
+
 # ------------------------------------------------------------------------------------------------
-# DRAM traffic measured by Nsight Compute on small cases of the same kernels (summaries under profiles/), expressed per
-# unit so that it can be scaled to the launch this run times; traffic grows in proportion to these units.
-#  * local attention (k_attn_tc phase 0), Llama-3-8B geometry, chunk 512, window 4096 full, sink 64:
-#    101.85 MB for a 4-layer launch (profiles/k_attn_tc_cfg2_4layers_16k.md) -> bytes per layer of a launch
-ATTN_LOCAL_DRAM_BYTES_PER_LAYER = {(32, 8, 512, 4096, 64): 101.85e6 / 4}
-#  * decode retrieval + attention: 239.4 MB measured against 237.8 MB of algorithmic bytes for an 8-layer step at 64K
-#    (profiles/decode_kernels_cfg2_8layers_64k.md): every byte is read once, nothing is re-read
+# DRAM traffic measured by Nsight Compute on small cases of the same kernels, expressed per unit so that it can be
+# scaled to the launch this run times (traffic grows in proportion to these units):
+#  * local attention (k_attn_tc phase 0), Llama-3-8B geometry, chunk 512, window 4096 full, sink 64: DRAM read +
+#    write of one launch over 4 layers at 16K context -> bytes per layer of a launch
+ATTN_LOCAL_DRAM_BYTES_PER_LAYER = {(32, 8, 512, 4096, 64): (95.14e6 + 8.42e6) / 4}
+#  * decode retrieval + attention: 239.4 MB measured against 237.8 MB of algorithmic bytes for an 8-layer step at
+#    64K: every byte is read once, nothing is re-read
 DECODE_DRAM_PER_ALGORITHMIC_BYTE = 239.4 / 237.8
+NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16, per GPU
+NOMINAL_HBM_GBS = 8000.0
+
+
+def local_keys(cfg, t0, n, E):
+    """Keys a row of the call sees in the local part, averaged over the rows: sink + local + causal current."""
+    return min(cfg.n_sink, t0) + (t0 - min(E, t0)) + (n + 1) / 2.0
 
 
 def attn_local_flops(cfg, t0, n, E):
     """Algorithmic flops of the local attention kernel for one call (all layers): QK^T + PV over
     sink + local + causal current keys."""
-    keys = min(cfg.n_sink, t0) + (t0 - min(E, t0)) + (n + 1) / 2.0
-    return 4.0 * n * cfg.n_q_heads * cfg.head_dim * keys * cfg.n_layers
+    return 4.0 * n * cfg.n_q_heads * cfg.head_dim * local_keys(cfg, t0, n, E) * cfg.n_layers
+
+
+def map_pass_flops(cfg, t0, n, E):
+    """Algorithmic flops of the local-map pass for one call (all layers): QK^T over local + causal current keys."""
+    return 2.0 * n * cfg.n_q_heads * cfg.head_dim * ((t0 - min(E, t0)) + (n + 1) / 2.0) * cfg.n_layers
+
+
+def tensor_roofline(tflops, peaks, clocks):
+    """Fractions of one achieved TFLOP/s figure against every denominator on record, and which measured peak the
+    run's clocks call for: the burst figure when the SM clock stayed at (>= 95 % of) its maximum with no power cap
+    active while the kernels ran, the sustained one otherwise."""
+    sm, smax = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    at_max = bool(sm and smax and sm >= 0.95 * smax and "sw_power_cap" not in clocks.get("reasons", []))
+    peak = peaks["bf16_tflops"] if at_max else peaks["bf16_tflops_sustained"]
+    return {"achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak if tflops else None,
+            "frac_burst": tflops / peaks["bf16_tflops"] if tflops else None,
+            "frac_sustained": tflops / peaks["bf16_tflops_sustained"] if tflops else None,
+            "frac_nominal": tflops / NOMINAL_BF16_TFLOPS if tflops else None,
+            "of": f"{peaks['source']} ({'burst' if at_max else 'sustained'}: SM clock {sm} of {smax} MHz under load)"}
 
 
 def needle_recall(lt, st, seq, cfg):
@@ -289,19 +322,32 @@ def needle_recall(lt, st, seq, cfg):
     return {"needle_tokens": [int(a), int(b)], "mean_coverage": cover / units, "fully_retrieved": full / units}
 
 
-def run_ltri(args, cfg):
-    from paper_2412_04757_b200 import binding, build
+def params_of(cfg, nseq, binding):
+    return binding.make_params(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_tokens, cfg.chunk, cfg.window,
+                               cfg.n_sink, cfg.top_k, head_dim=cfg.head_dim, max_seqs=nseq,
+                               reps_per_span=cfg.reps_per_span, max_spans_per_region=cfg.max_spans_per_region,
+                               theta_mode=cfg.theta_mode, theta=cfg.theta, rep_mode=cfg.rep_mode,
+                               ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps, max_reps=cfg.max_reps,
+                               rep_lambda=cfg.rep_lambda,
+                               flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
+                                     (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0) |
+                                     (binding.FLAG_SEGMENT_PER_UNIT if cfg.segment_per_unit else 0) |
+                                     (binding.FLAG_HOST_KV if cfg.host_kv else 0),
+                               cache_units=cfg.cache_units, score_decay=cfg.score_decay,
+                               unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
+                               retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score,
+                               layer_theta=cfg.layer_theta, layer_nms_iou_milli=cfg.layer_nms_iou_milli,
+                               layer_rep_lambda=cfg.layer_rep_lambda)
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
-    rank, local, world = dist_setup(args.gpus)
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    build.build()
-    peaks = measured_peaks()
+
+def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_calls=False):
+    """Streams the workload of `cfg` up to its last W + K prefill calls, times those K calls (and the workload's decode
+    steps) with the inputs resident in HBM and, if asked, once more through the host-buffer entry.  Returns a dict
+    with everything the report lines are made of."""
+    from paper_2412_04757_b200 import binding
+
     L, n = cfg.n_layers, cfg.chunk
     chunks = list(inputs.prefill_calls(cfg))
-    K, W = args.steps, args.warmup
     if K + W > len(chunks):   # tiny workloads: fewer calls exist than were asked for
         W = min(W, max(0, len(chunks) // 2 - 1))
         K = len(chunks) - W
@@ -312,20 +358,7 @@ def run_ltri(args, cfg):
     streams = [inputs.SyntheticStream(cfg, seq=rank * NSEQ + s, device=dev) for s in range(NSEQ)]
     st = streams[-1]        # the timed prefill steps run on the last sequence; the others are streamed as set-up
     SQ = NSEQ - 1
-    p = binding.make_params(L, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_tokens, cfg.chunk, cfg.window, cfg.n_sink,
-                            cfg.top_k, head_dim=cfg.head_dim, max_seqs=NSEQ, reps_per_span=cfg.reps_per_span,
-                            max_spans_per_region=cfg.max_spans_per_region, theta_mode=cfg.theta_mode, theta=cfg.theta,
-                            rep_mode=cfg.rep_mode, ratio_kind=cfg.ratio_kind, min_reps=cfg.min_reps,
-                            max_reps=cfg.max_reps, rep_lambda=cfg.rep_lambda,
-                            flags=(binding.FLAG_PERSIST_DECODE if cfg.persist_decode else 0) |
-                                  (binding.FLAG_COLLAB_VOTE if cfg.collab_vote else 0) |
-                                  (binding.FLAG_SEGMENT_PER_UNIT if cfg.segment_per_unit else 0) |
-                                  (binding.FLAG_HOST_KV if cfg.host_kv else 0),
-                            cache_units=cfg.cache_units, score_decay=cfg.score_decay,
-                            unit_tokens=cfg.unit_tokens, nms_iou_milli=cfg.nms_iou_milli,
-                            retrieval_head=cfg.retrieval_head, retrieval_head_score=cfg.retrieval_head_score,
-                            layer_theta=cfg.layer_theta, layer_nms_iou_milli=cfg.layer_nms_iou_milli,
-                            layer_rep_lambda=cfg.layer_rep_lambda)
+    p = params_of(cfg, NSEQ, binding)
 
     def stream_until(lt, upto, keep_from):
         for s in range(NSEQ - 1):
@@ -341,10 +374,19 @@ def run_ltri(args, cfg):
                 lt.ltri_prefill_chunk(SQ, 0, L, q, k, v)
         return kept
 
+    def call(lt, qkv, out):
+        q, k, v = qkv
+        if not per_layer_calls:
+            lt.ltri_prefill_chunk(SQ, 0, L, q, k, v, out=out)
+        else:   # one layer per call, in order: what a model whose layers depend on each other has to do
+            for l in range(L):
+                lt.ltri_prefill_chunk(SQ, l, 1, q[l:l + 1], k[l:l + 1], v[l:l + 1], out=out[l:l + 1])
+
     lt = binding.Ltri(p, device=dev)
     # set-up: stream everything before the warm-up chunks, generate (and keep) warm-up + timed inputs
     kept = stream_until(lt, len(chunks), first_warm)
     outs = [torch.empty_like(kept[0][0]) for _ in range(2)]
+
     def decode_inputs(step):
         parts = [sx.tokens(cfg.context + step, 1, kind=1) for sx in streams]
         return tuple(torch.cat([pp[i].permute(1, 0, 2, 3) for pp in parts]).contiguous() for i in range(3))
@@ -355,7 +397,7 @@ def run_ltri(args, cfg):
 
     # ---- device-resident timing ------------------------------------------------------------
     for i in range(W):
-        lt.ltri_prefill_chunk(SQ, 0, L, *kept[i], out=outs[i & 1])
+        call(lt, kept[i], outs[i & 1])
     torch.cuda.synchronize(dev)
     lt.ltri_profile_read()                      # clears counters
     lt.ltri_profile_enable(True)
@@ -368,7 +410,7 @@ def run_ltri(args, cfg):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(K):
-        lt.ltri_prefill_chunk(SQ, 0, L, *kept[W + i], out=outs[i & 1])
+        call(lt, kept[W + i], outs[i & 1])
     e1.record()
     torch.cuda.synchronize(dev)
     clk_hi = sampler.mark()
@@ -379,6 +421,8 @@ def run_ltri(args, cfg):
     lt.ltri_profile_enable(False)
     assert lt.ltri_sync_status() == 0, "device-side status word reports an error"
     stats = lt.ltri_get_stats(SQ, 0)
+    # retrieved tokens of the last timed call, summed over KV heads and layers (the continuation kernel's work)
+    retrieved_all = sum(lt.ltri_get_stats(SQ, l).retrieved_tokens for l in range(L))
     pager = None
     if cfg.host_kv:
         # unit-cache traffic of all layers since the stream began (prefill calls only so far)
@@ -426,12 +470,14 @@ def run_ltri(args, cfg):
         bytes_step = NSEQ * L * (cfg.n_kv_heads * dst.n_spans * cfg.head_dim * 2 +
                                  2 * cfg.n_kv_heads * cfg.head_dim * 2 * keys)
         k_ms = dprof["decode_retrieve"][0] + dprof["decode_attn"][0]
+        gbs = bytes_step * dsteps / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
         dec = {"value": world * NSEQ * dsteps / (dms * 1e-3), "unit": "tok/s", "steps": dsteps, "sequences": NSEQ,
                "ms_per_step": dms / dsteps,
                "keys_per_head": keys, "index_spans": dst.n_spans,
-               "roofline": {"bound": "hbm", "achieved": bytes_step * dsteps / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None,
-                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                            "frac": (bytes_step * dsteps / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]) if k_ms > 0 else None,
+               "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": gbs / peaks["hbm_gbs"] if gbs else None,
+                            "frac_nominal": gbs / NOMINAL_HBM_GBS if gbs else None,
+                            "frac_whole_step": bytes_step / (dms / dsteps * 1e-3) / 1e9 / peaks["hbm_gbs"],
                             "traffic": bytes_step * DECODE_DRAM_PER_ALGORITHMIC_BYTE,
                             "traffic_note": "bytes per step, scaled from an ncu capture of an 8-layer 64K case",
                             "kernels": "decode score+top-k and split-KV attention+merge",
@@ -443,7 +489,7 @@ def run_ltri(args, cfg):
 
     # ---- end-to-end: same steps with host buffers ---------------------------------------------
     e2e = None
-    if not args.no_e2e:
+    if want_e2e:
         lt.close()
         del lt
         torch.cuda.empty_cache()
@@ -488,40 +534,115 @@ def run_ltri(args, cfg):
                "api": "ltri_prefill_chunk_host",
                "timing": "max of device events (first call -> last output copy done) and the host clock"}
     lt.close()
+    del lt
+    torch.cuda.empty_cache()
 
-    if rank != 0:
-        return
-    # ---- roofline of the dominant kernel (local attention), live CUDA-event time -------------
-    flops = sum(attn_local_flops(cfg, t0, cnt, max(cfg.n_sink, t0 - cfg.window - (t0 % cfg.chunk)))
-                for (t0, cnt) in chunks[first_timed:])
+    # ---- rooflines of the dense kernels, live CUDA-event times ---------------------------------
+    timed = chunks[first_timed:]
+    E_of = lambda t0: max(cfg.n_sink, t0 - cfg.window - (t0 % cfg.chunk))
+    f_loc = sum(attn_local_flops(cfg, t0, cnt, E_of(t0)) for (t0, cnt) in timed)
+    f_map = sum(map_pass_flops(cfg, t0, cnt, E_of(t0)) for (t0, cnt) in timed)
+    # continuation over the retrieved tokens: G query heads x n rows x R keys per (layer, KV head); R taken from
+    # the last timed call and assumed for all of them
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    f_ret = sum(4.0 * cnt * G * cfg.head_dim * retrieved_all for (_, cnt) in timed)
     a_ms, a_cnt = prof["attn_local"]
-    tf = flops / (a_ms * 1e-3) / 1e12 if a_ms > 0 else None
-    peak_tf = peaks["bf16_tflops_sustained"]
+    r_ms, _ = prof["attn_retrieved"]
     per_layer = ATTN_LOCAL_DRAM_BYTES_PER_LAYER.get((cfg.n_q_heads, cfg.n_kv_heads, cfg.chunk, cfg.window, cfg.n_sink))
-    window_full = chunks[first_timed][0] >= cfg.window + cfg.chunk
-    traffic = per_layer * L if per_layer and window_full else None
-    roof = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
-            "frac": tf / peak_tf if tf else None, "traffic": traffic,
+    window_full = timed[0][0] >= cfg.window + cfg.chunk
+    traffic = per_layer * L / max(1, a_cnt // K) if per_layer and window_full else None
+    roof = {"bound": "tensor", **tensor_roofline(f_loc / (a_ms * 1e-3) / 1e12 if a_ms > 0 else None, peaks, clocks),
+            "traffic": traffic,
             "traffic_note": "DRAM bytes per launch, ncu capture of a 4-layer case of the same geometry x layers / 4",
             "kernel": "k_attn_tc, local part (sink | local | current)",
-            "launches": a_cnt, "ms_per_launch": a_ms / max(a_cnt, 1), "of": peaks["source"] + " (sustained)"}
+            "launches": a_cnt, "ms_per_launch": a_ms / max(a_cnt, 1)}
+    roof_attn = {"bound": "tensor",
+                 **tensor_roofline((f_loc + f_ret) / ((a_ms + r_ms) * 1e-3) / 1e12 if a_ms > 0 else None, peaks, clocks),
+                 "kernels": "k_attn_tc local part + continuation over the retrieved spans (the chunked-prefill "
+                            "attention as a whole)",
+                 "ms_per_step": (a_ms + r_ms) / K, "flops_per_step": (f_loc + f_ret) / K}
+    roof_call = {"bound": "tensor",
+                 **tensor_roofline((f_loc + f_ret + f_map) / (ms * 1e-3) / 1e12, peaks, clocks),
+                 "kernels": "all dense work of a call (attention, continuation, local-map pass) over the whole step time",
+                 "flops_per_step": (f_loc + f_ret + f_map) / K}
+    return {"cfg": cfg, "K": K, "W": W, "ms": ms, "value": prefill_tps, "launches": launches, "prof": prof,
+            "stats": stats, "retrieved_per_kv_head": retrieved_all / (L * cfg.n_kv_heads), "pager": pager,
+            "recall": recall, "decode": dec, "clocks": clocks, "e2e": e2e, "roofline": roof,
+            "roofline_prefill_attention": roof_attn, "roofline_call": roof_call,
+            "timed_positions": [timed[0][0], cfg.context], "nseq": NSEQ,
+            "kernel_ms_per_step": {k: v[0] / K for k, v in prof.items() if v[1]}}
+
+
+def brief(m):
+    """The short form of a measurement, for the extra workloads reported beside the headline."""
+    d = m["decode"]
+    out = {"workload": m["cfg"].name, "prefill_tok_s": m["value"], "ms_per_step": m["ms"] / m["K"], "steps": m["K"],
+           "frac_attn_local": m["roofline"]["frac"], "frac_prefill_attention": m["roofline_prefill_attention"]["frac"],
+           "peak_tflops": m["roofline"]["peak"], "index_spans": m["stats"].n_spans,
+           "retrieved_tokens_per_kv_head": m["retrieved_per_kv_head"], "gpu_launches": m["launches"],
+           "kernel_ms_per_step": m["kernel_ms_per_step"]}
+    if d:
+        out.update({"decode_tok_s": d["value"], "decode_ms_per_step": d["ms_per_step"],
+                    "decode_frac_hbm": d["roofline"]["frac"]})
+    if m["recall"]:
+        out["needle_recall"] = m["recall"]
+    if m["pager"]:
+        out["pager"] = m["pager"]
+    return out
+
+
+def paper_setting(cfg):
+    """The paper's own setting of the optional modes on the same workload: 128-token memory units (Eq. 8 as
+    printed), dynamic representative counts with the row ratio and lambda = 3 (Sec. 3.3.2), NMS threshold 0.1
+    (App. "NMS Input Filtration"), persistent mechanism in decode (Sec. 3.5)."""
+    import dataclasses
+    c = dataclasses.replace(cfg, unit_tokens=128, rep_mode=1, ratio_kind=0, rep_lambda=3.0, min_reps=1, max_reps=4,
+                            nms_iou_milli=100, persist_decode=True)
+    c.name += "[paper-setting: unit=128,dynamic-reps,nms-iou=0.1,persist-decode]"
+    return c
+
+
+def run_ltri(args, cfg):
+    from paper_2412_04757_b200 import build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    rank, local, world = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    build.build()
+    peaks = measured_peaks()
+    m = measure(cfg, args.steps, args.warmup, rank, local, world, dev, peaks, want_e2e=not args.no_e2e)
+    extras = {}
+    if args.extras and world == 1:
+        # beside the headline: the same workload in the paper's own setting, the other single-GPU workloads, and
+        # the headline workload submitted one layer per call; few steps each, no host-buffer leg
+        ks, ws = min(8, args.steps), min(3, args.warmup)
+        extras["paper_setting"] = brief(measure(paper_setting(cfg), ks, ws, rank, local, world, dev, peaks, False))
+        if args.config == 2 and cfg.name == inputs.config(2).name:
+            extras["other_configs"] = [brief(measure(inputs.config(c), ks, ws, rank, local, world, dev, peaks, False))
+                                       for c in (1, 3, 4)]
+        pl = measure(cfg, ks, ws, rank, local, world, dev, peaks, False, per_layer_calls=True)
+        extras["per_layer_calls"] = {**brief(pl), "note": "every layer of a chunk submitted as its own call "
+                                                          "(layer_count = 1), as a model with dependent layers must"}
+    if rank != 0:
+        return
     cpu = None
     if not args.no_cpu_baseline:
         ctoks, cores, sample, _ = oracle_sample(cfg, 2, 0)
         cpu = {"value": ctoks, "unit": "tok/s", "cores": cores, "kind": "oracle", "sample": sample}
+    K = m["K"]
     line = {
-        "metric": METRIC, "value": prefill_tps, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "metric": METRIC, "value": m["value"], "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": m["W"],
+        "ms_per_step": m["ms"] / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
-                   "context": cfg.context, "chunk": cfg.chunk, "window": cfg.window, "sink": cfg.n_sink,
-                   "top_k": cfg.top_k, "timed_positions": [chunks[first_timed][0], cfg.context],
+        "config": {**workload_config(cfg, world, m["nseq"]), "timed_positions": m["timed_positions"],
                    "l2": "inputs of every step are distinct and larger than L2 (no flush needed)",
-                   "parallelism": "replicas only" if world > 1 else "single GPU", "sequences": NSEQ,
-                   "index_spans": stats.n_spans, "retrieved_tokens_per_kv_head": stats.retrieved_tokens / cfg.n_kv_heads},
-        "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "decode": dec, "roofline": roof, "cpu_baseline": cpu,
-        "needle_recall": recall, "pager": pager,
-        "kernel_ms_per_step": {k: v[0] / K for k, v in prof.items() if v[1]},
+                   "index_spans": m["stats"].n_spans, "retrieved_tokens_per_kv_head": m["retrieved_per_kv_head"]},
+        "clocks": m["clocks"], "gpu_launches": m["launches"], "e2e": m["e2e"], "decode": m["decode"],
+        "roofline": m["roofline"], "roofline_prefill_attention": m["roofline_prefill_attention"],
+        "roofline_call": m["roofline_call"], "cpu_baseline": cpu,
+        "needle_recall": m["recall"], "pager": m["pager"], "kernel_ms_per_step": m["kernel_ms_per_step"], **extras,
     }
     print(json.dumps(line))
 
@@ -565,8 +686,17 @@ def main():
                     help="generator: probability that a prefill token targets its own segment (default 0.5; 0 = the "
                          "literal 'earlier segment' reading)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--extras", dest="extras", action="store_true", default=None,
+                    help="also measure the paper's own setting, the other single-GPU workloads and per-layer calls "
+                         "(default: on for the plain default run, off when any workload option is given)")
+    ap.add_argument("--no-extras", dest="extras", action="store_false")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.extras is None:
+        workload_flags = ("--layers", "--context", "--decode-steps", "--dynamic-reps", "--unit-tokens", "--nms-iou",
+                          "--persist-decode", "--host-kv", "--segment-per-unit", "--layer-tables", "--retrieval-heads",
+                          "--collab-vote", "--p-self", "--config", "--no-e2e", "--no-cpu-baseline")
+        args.extras = not any(a.split("=")[0] in workload_flags for a in sys.argv[1:])
     cfg = inputs.config(args.config)
     if args.layers > 0 or args.context > 0 or args.decode_steps >= 0:
         import dataclasses

@@ -18,8 +18,19 @@
  *    (or be ordered by the caller).
  *  - Return value: 0 (LTRI_OK) or a negative LTRI_E* code.  Parameter, state and capacity
  *    errors are detected on the host before anything is launched and leave the context
- *    unchanged.  Device-side checks record a code in a status word read by
- *    ltri_sync_status; nothing traps or spins without bound.
+ *    unchanged (ltri_prefill_chunk_host included: it checks the whole call before its first
+ *    layer group starts).  LTRI_ECUDA means the CUDA runtime refused a launch or a copy part
+ *    of the way through a call; the sequence is then in an undefined state: reset it.
+ *    Device-side checks record a code in a status word read by ltri_sync_status; nothing
+ *    traps or spins without bound.
+ *  - Numeric range.  Inputs are finite bf16 values of any magnitude for which the scaled
+ *    logits q.k * softmax_scale stay below about 2000 in absolute value (the local-map
+ *    pass carries the row offsets -max - log2(sum) through an fp32 accumulator clamped at
+ *    that size); inside that range every softmax is exact however far a later key tile
+ *    exceeds the running maximum: the prefill attention kernel bounds the logits of a
+ *    work item by |q| |k| scale (the largest key norm of a (sequence, layer, KV head) is
+ *    tracked as keys are appended) and, where the bound is too wide for its late-moving
+ *    reference maximum, exchanges the true maximum on every tile instead.
  */
 #ifndef LTRI_H_
 #define LTRI_H_
@@ -177,7 +188,11 @@ int ltri_destroy(ltri_ctx* ctx);
 int ltri_reset_sequence(ltri_ctx* ctx, int seq, void* cuda_stream);
 
 /* One streamed prefill call (Sec. 3.4, steps 1-3) for `n_tokens` (1..chunk) new tokens of
- * sequence `seq`, for layers [layer_begin, layer_begin+layer_count).
+ * sequence `seq`, for layers [layer_begin, layer_begin+layer_count).  Every call is a region
+ * of its own (it is segmented once, while current) and stays pending until it has left the
+ * window; a context has room for window/chunk (rounded up) + 8 pending regions, so a caller
+ * that streams calls much shorter than `chunk` gets LTRI_ECAPACITY once more calls than that
+ * fit into the window (e.g. window 4096, chunk 512: the 17th 64-token call in a row).
  *   q   [layer_count][n_tokens][n_q_heads ][head_dim]
  *   k,v [layer_count][n_tokens][n_kv_heads][head_dim]   (copied into the library's cache)
  *   out [layer_count][n_tokens][n_q_heads ][head_dim]   (fully overwritten)
@@ -198,7 +213,10 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
  * group before that sends its output down on a second internal stream; two staging sets alternate between calls, so
  * the copies of one call also overlap the kernels of its neighbours.  The host inputs must stay valid, and out_host
  * must not be read, until the work is done: make a stream wait for it with ltri_host_outputs_ready (or synchronise
- * the device).  On an error return the sequence may be left with some layers advanced; reset it.
+ * the device).  All parameter, state and capacity checks of the whole call are made before the first group is
+ * enqueued, so those errors leave the sequence unchanged; only LTRI_ECUDA can leave some layers advanced (reset the
+ * sequence then).  The groups are fixed layer ranges of the context (a quarter of its layers each), so calls of any
+ * size and layer range may follow each other.
  * The streamed-context setting of Sec. 3.4 with the context memory on the host side. */
 int ltri_prefill_chunk_host(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q_host,
                             const void* k_host, const void* v_host, void* out_host, void* cuda_stream);
@@ -206,7 +224,7 @@ int ltri_prefill_chunk_host(ltri_ctx* ctx, int seq, int layer_begin, int layer_c
 /* Make `cuda_stream` wait until every output of earlier ltri_prefill_chunk_host calls has reached host memory. */
 int ltri_host_outputs_ready(ltri_ctx* ctx, void* cuda_stream);
 
-/* One decode step (the block becomes a single token, Sec. 3.5) for `n_seqs` sequences.
+/* One decode step (Sec. 3.5: during decoding the current block is one token) for `n_seqs` sequences.
  *   seq_ids  HOST array [n_seqs] of distinct sequence slots
  *   q   [n_seqs][layer_count][n_q_heads ][head_dim]
  *   k,v [n_seqs][layer_count][n_kv_heads][head_dim]
@@ -291,6 +309,27 @@ int ltri_span_capacity(const ltri_ctx* ctx);
 int ltri_debug_segment_map(ltri_ctx* ctx, const int32_t* Mq, int m, int theta_mode, float theta, int64_t theta_q,
                            int max_spans, int32_t* start_len_pairs, int cap, int* n_out, void* cuda_stream);
 
+/* Bring-up hook: replace the span table and the span index K^R of (seq, layer) -- what Sec. 3.3 builds from the
+ * evicted tokens and Sec. 3.4 step 2 (Eq. 7-8) scores against -- with a state computed elsewhere, so that retrieval
+ * and attention can be driven from spans and index vectors the library did not produce itself.
+ *   evicted_end   must equal the layer's current E (ltri_stats.evicted_end): the K/V cache, the votes and the
+ *                 pending regions are left as they are (LTRI_ESTATE otherwise)
+ *   start_len_pairs HOST int32 [n_spans][2], in token order, covering [n_sink, E) without a gap (spans may overlap,
+ *                 as those of an NMS with phi > 0 do); n_spans = 0 only if E = n_sink
+ *   index_bf16    HOST bf16 [n_kv_heads][n_spans][head_dim]
+ * n_spans beyond ltri_span_capacity is LTRI_ECAPACITY.  Synchronises `cuda_stream`; the host buffers are not kept. */
+int ltri_debug_load_index(ltri_ctx* ctx, int seq, int layer, int64_t evicted_end, const int32_t* start_len_pairs,
+                          int n_spans, const void* index_bf16, void* cuda_stream);
+
+/* Test hook for the bounded device-side waits (no counterpart in the paper; failure detection).  Runs a one-CTA
+ * kernel in which one thread waits, for at most `limit_cycles` SM clock cycles (1..10^8), on a barrier that nothing
+ * ever completes, while a second thread waits on it with the context's normal limit.  The first wait expires and
+ * raises the CTA's abort flag, which releases the second; the kernel then records LTRI_ETIMEOUT in the status word
+ * the way the tensor-core kernels do, so the next ltri_sync_status returns it (and clears it).  Nothing faults or
+ * hangs, and the context stays usable.  waited_cycles HOST int64 [2]: cycles each of the two waits lasted (-1: the
+ * wait reported success).  Synchronises `cuda_stream`. */
+int ltri_debug_wait_timeout(ltri_ctx* ctx, int64_t limit_cycles, int64_t* waited_cycles, void* cuda_stream);
+
 /* ---- allocation-free entry point ---- */
 
 /* The paper has no counterpart for this call; it exists for callers that cannot allocate device memory at the
@@ -298,9 +337,14 @@ int ltri_debug_segment_map(ltri_ctx* ctx, const int32_t* Mq, int m, int theta_mo
  * start-up, service threads that must stay off the allocator).  It runs the same segmenter as
  * ltri_debug_segment_map, but needs no context and no arena: its scratch is a fixed array inside the library
  * image (about 0.5 MiB, held by every GPU that loads the library until the process exits).
- *   Mq     DEVICE int32 [m][m] dense row-major map (lower triangle used), 1 <= m <= LTRI_STATIC_SEGMENT_MAX_M
+ *   Mq     DEVICE int32 [m][m] dense row-major map (lower triangle used), 1 <= m <= LTRI_STATIC_SEGMENT_MAX_M,
+ *          in the memory of the CURRENT device (the scratch that is used is the current device's; a pointer that
+ *          the runtime attributes to another device is LTRI_EINVAL)
  *   theta_q threshold in map units (Eq. 5), max_spans 1..64 (NMS cap)
- *   pairs  DEVICE int32 [cap_pairs][2]: {start,len} spans partitioning [0,m); n_out DEVICE int32[1]: span count
+ *   pairs  DEVICE int32 [cap_pairs][2]: {start,len} spans partitioning [0,m); n_out DEVICE int32[1]: span count.
+ *          At most cap_pairs pairs are written; *n_out is the full count even when it exceeds cap_pairs (the
+ *          segmenter yields at most 2 * max_spans + 1 spans).  If a device-side check of the segmenter fails,
+ *          *n_out is the negative LTRI_E* code instead and no pair is valid.
  * Larger m or max_spans return LTRI_ECAPACITY and launch nothing.  The call allocates nothing and returns
  * without synchronising.  The first call on each device also looks up the scratch array's device address; make
  * that first call outside any stream capture.  All calls share the one scratch array, which keeps the previous

@@ -20,8 +20,8 @@
 //   O8  similarity of query reps vs span index                Eq. 7
 //   O9  top-k spans                                           Eq. 8 (unit = span)
 //   O10 softmax attention over sink+retrieved+local+cur       Sec. 3.4 step 3
-//   O11 decode step (one query, no eviction, no votes)        Sec. 3.5 "Persistent Mechanism" (the
-//                                                             block becomes a single token)
+//   O11 decode step (one query, no eviction, no votes)        Sec. 3.5 "Persistent Mechanism" (while
+//                                                             decoding, the current block is one token)
 //   O12 full causal attention (reference for the pin
 //       "top-k covers every span => method == full attention")
 // Optional modes (off by default):
@@ -462,6 +462,22 @@ struct Stream {
     pending.clear();
     return 0;
   }
+  // test hook: replace the span table and the index vectors of the indexed prefix [n_sink, E) and leave everything
+  // else (E, the pending regions, the votes) as it is; no arithmetic of the method
+  int replace_index(int nspans, const int* start_len, const uint16_t* kr) {
+    std::vector<Span> fresh;
+    int pos = p.n_sink;
+    for (int i = 0; i < nspans; ++i) {
+      if (start_len[2 * i] != pos || start_len[2 * i + 1] < 1) return -1;
+      fresh.push_back(Span{start_len[2 * i], start_len[2 * i + 1]});
+      pos += start_len[2 * i + 1];
+    }
+    if (pos != E || !kr) return -1;
+    spans.swap(fresh);
+    KR.assign((size_t)nspans * Hkv * d, 0);
+    std::memcpy(KR.data(), kr, KR.size() * sizeof(uint16_t));
+    return 0;
+  }
   // append a region that is still inside the window, with its spans (its votes start from zero)
   int add_pending(int start, int end, int nspans, const int* start_len) {
     if (start < E || end <= start || end > t) return -1;
@@ -871,6 +887,9 @@ void orc_full_attention(void* h, int cnt, const int* pos, const uint16_t* q, flo
 int orc_append_only(void* h, int n, const uint16_t* k, const uint16_t* v) { return ((Stream*)h)->append_only(n, k, v); }
 int orc_load_state(void* h, int evicted_end, int nspans, const int* start_len, const uint16_t* kr) {
   return ((Stream*)h)->load_state(evicted_end, nspans, start_len, kr);
+}
+int orc_replace_index(void* h, int nspans, const int* start_len, const uint16_t* kr) {
+  return ((Stream*)h)->replace_index(nspans, start_len, kr);
 }
 int orc_begin_call(void* h, int n, const uint16_t* q) { return ((Stream*)h)->begin_call(n, q); }
 int orc_add_pending(void* h, int start, int end, int nspans, const int* start_len) {

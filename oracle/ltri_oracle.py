@@ -57,6 +57,7 @@ def lib():
         L.orc_load_state.argtypes = [vp, ip, ip, vp, vp]
         L.orc_begin_call.argtypes = [vp, ip, vp]
         L.orc_add_pending.argtypes = [vp, ip, ip, ip, vp]
+        L.orc_replace_index.argtypes = [vp, ip, vp, vp]
         L.orc_decode_retrieve.argtypes = [vp, vp, vp, vp]
         L.orc_decode_attend.argtypes = [vp, vp]
         L.orc_full_attention.argtypes = [vp, ip, vp, vp, vp]
@@ -188,6 +189,15 @@ class OracleStream:
         kr = None if index is None else np.ascontiguousarray(index, dtype=np.uint16)
         if lib().orc_load_state(self._h, int(evicted_end), len(sp), _ptr(sp), None if kr is None else _ptr(kr)):
             raise ValueError("inconsistent oracle state")
+
+    def replace_index(self, spans, index):
+        """Swap the span table and the index vectors ([span][Hkv][d] bf16 bits) of the indexed prefix for given
+        ones; the evicted end, the pending regions and the votes stay."""
+        sp = np.ascontiguousarray(np.asarray(spans, dtype=np.int32).reshape(-1, 2))
+        kr = np.ascontiguousarray(index, dtype=np.uint16)
+        assert kr.shape == (len(sp), self.Hkv, self.d)
+        if lib().orc_replace_index(self._h, len(sp), _ptr(sp), _ptr(kr)):
+            raise ValueError("spans do not tile the indexed prefix")
 
     def add_pending(self, start, end, spans):
         sp = np.ascontiguousarray(np.asarray(spans, dtype=np.int32).reshape(-1, 2))

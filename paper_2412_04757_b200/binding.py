@@ -30,6 +30,7 @@ EXPORTS = [
     "ltri_sync_status", "ltri_last_cuda_error", "ltri_strerror", "ltri_debug_read", "ltri_span_capacity",
     "ltri_debug_segment_map", "ltri_launch_count", "ltri_profile_enable", "ltri_profile_read",
     "ltri_segment_map_static", "ltri_prefill_chunk_host", "ltri_host_outputs_ready", "ltri_host_kv_bytes",
+    "ltri_debug_load_index", "ltri_debug_wait_timeout",
 ]
 KERNEL_CLASSES = ["append", "evict_index", "attn_local", "map_pass", "segment", "score_topk", "attn_retrieved",
                   "decode_retrieve", "decode_attn"]
@@ -104,6 +105,8 @@ def load():
         L.ltri_profile_enable.argtypes = [vp, ip]
         L.ltri_profile_read.argtypes = [vp, vp, vp, vp]
         L.ltri_segment_map_static.argtypes = [vp, ip, C.c_int64, ip, vp, ip, vp, vp]
+        L.ltri_debug_load_index.argtypes = [vp, ip, ip, C.c_int64, vp, ip, vp, vp]
+        L.ltri_debug_wait_timeout.argtypes = [vp, C.c_int64, vp, vp]
         _lib = L
     return _lib
 
@@ -352,6 +355,24 @@ class Ltri:
         if what == BUF_ROWSTAT:
             return raw.view(np.float32).reshape(p.chunk, p.n_q_heads, 2)
         return raw
+
+    def ltri_debug_load_index(self, seq, layer, evicted_end, spans: np.ndarray, index_bits: np.ndarray, stream=None):
+        """spans int32 [n][2]; index_bits uint16 [Hkv][n][d] (bf16 bit patterns), both on the host."""
+        spans = np.ascontiguousarray(spans, dtype=np.int32).reshape(-1, 2)
+        index_bits = np.ascontiguousarray(index_bits, dtype=np.uint16)
+        n = len(spans)
+        if index_bits.shape != (self.params.n_kv_heads, n, self.params.head_dim):
+            raise ValueError("index_bits must be [n_kv_heads][n_spans][head_dim]")
+        _check(self.lib.ltri_debug_load_index(self._h, seq, layer, int(evicted_end), spans.ctypes.data_as(C.c_void_p), n,
+                                              index_bits.ctypes.data_as(C.c_void_p), self._stream(stream)),
+               "ltri_debug_load_index")
+
+    def ltri_debug_wait_timeout(self, limit_cycles: int, stream=None) -> np.ndarray:
+        """Runs the bounded-wait test kernel; returns the cycles its two waits lasted."""
+        waited = np.zeros(2, dtype=np.int64)
+        _check(self.lib.ltri_debug_wait_timeout(self._h, int(limit_cycles), waited.ctypes.data_as(C.c_void_p),
+                                                self._stream(stream)), "ltri_debug_wait_timeout")
+        return waited
 
     def ltri_debug_segment_map(self, Mq: np.ndarray, theta_mode=2, theta=0.0, theta_q=0, max_spans=None, stream=None):
         Mq = np.ascontiguousarray(Mq, dtype=np.int32)

@@ -18,6 +18,7 @@ constexpr int kMaxRanges = 2 * kMaxTopK + 2;  // sink + local + the spans of thi
 constexpr float kMapMargin = 0.0078125f;          // safety margin (in log2 units) of the map pass's skip test
 constexpr float kMapScale = 0.4972997117f;         // 2^-(1 + kMapMargin)
 constexpr int kTokPad = 128;          // rows of slack after every K/V slab so tile over-reads stay inside it
+constexpr long long kDefaultWaitLimit = 2000000000ll;  // device-side waits give up after about a second
 
 // Device-side view of one context.  Passed to kernels by value.
 struct DevCtx {
@@ -100,6 +101,10 @@ struct DevCtx {
   int* rng_cnt;          // [NS*NL][Hkv]
   float* dec_part;       // [NS*NL][Hq][kMaxDecSplit][128+2]
   int* status;           // [4]: first error code, detail...
+  unsigned* kmax2;       // [NS][NL][Hkv]  largest squared norm of any key appended so far (bit pattern of a
+                         //                non-negative float, which orders like the unsigned integer): bounds every
+                         //                logit of the (sequence, layer, KV head) by |q| * sqrt(kmax2) * scale
+  long long wait_limit;  // upper bound of any single device-side wait, in SM clock cycles
 };
 
 __host__ __device__ inline size_t unit_of(const DevCtx& c, int seq, int layer) { return (size_t)seq * c.NL + layer; }
@@ -189,6 +194,9 @@ cudaError_t launch_map_pass(const DevCtx& c, const PrefillArgs& a, cudaStream_t 
 
 cudaError_t launch_decode_attn(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
                                const __nv_bfloat16* q, __nv_bfloat16* out, int nsplit, cudaStream_t s);
+
+// test kernel for the bounded waits: one wait with `short_limit` cycles on a barrier nothing completes (kernels_probe.cu)
+cudaError_t launch_wait_probe(const DevCtx& c, long long short_limit, cudaStream_t s);
 
 // ---- small device helpers --------------------------------------------------------------
 __device__ __forceinline__ void set_status(const DevCtx& c, int code, int detail) {

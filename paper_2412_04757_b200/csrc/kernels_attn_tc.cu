@@ -29,6 +29,9 @@ constexpr float kLog2eT = 1.4426950408889634f;
 constexpr int kTcThreads = 576;  // 16 softmax warps + TMA producer + MMA issuer
 constexpr int kNumBoxes = 5;  // box heights 8,16,32,64,128
 constexpr float kRescaleThreshold = 8.0f;
+// Largest exponent (log2 units) a probability may carry above the softmax reference: 2^90 times the 2^7 keys of a
+// tile, the 2^13 tiles of the longest item and values of up to 2^10 still fits fp32 (and the bf16 P operand).
+constexpr float kLazyRange = 90.0f;
 
 struct TcMaps {
   CUtensorMap q;             // [tokens][Hq][128] bf16, box {64, G, 256/G}
@@ -157,6 +160,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __shared__ int s_items_ready;       // number of work items whose key ranges the producer has published
   __shared__ float s_max[2][2][2][128];  // per tile parity, Q tile, column half, row: partial maxima
   __shared__ float s_sum[2][2][128];     // per Q tile, column half, row: partial row sums (end of an item)
+  __shared__ unsigned s_qn[2][2];        // per Q tile, column half: largest partial squared query norm of the item
   constexpr int TOKB = 256 / G;  // tokens per work item
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // persistent CTA: work items (token block, KV head, layer) are dealt round-robin
@@ -177,6 +181,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     s_abort = 0;
     s_quit[0] = s_quit[1] = 0;
     s_items_ready = 0;
+    s_qn[0][0] = s_qn[0][1] = s_qn[1][0] = s_qn[1][1] = 0u;
     rg.n = 0;
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QFREE), 1);
@@ -238,7 +243,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       const Item w = decode(item);
       if (lane == 0) {
         // the Q buffer is free once every QK^T product of the previous item has completed
-        if (wi > 0) ok = mbar_wait(bar(B_QFREE), (wi - 1) & 1, abortp) ? 1 : 0;
+        if (wi > 0) ok = mbar_wait(bar(B_QFREE), (wi - 1) & 1, abortp, c.wait_limit) ? 1 : 0;
         // the key ranges of this item (the other roles read them after they have seen its Q tile arrive)
         const int last_tok = min(a.n, w.tok0 + TOKB) - 1;
         if (phase == 0) {
@@ -287,7 +292,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         uint32_t bytes = 0;
         for (int p = 0; p < np; ++p) bytes += (uint32_t)(8 << pbox[p]) * 256u;
         if (lane == 0) {
-          if (jt >= 2) ok = mbar_wait(bar(B_KEMPTY + st), par, abortp) ? 1 : 0;
+          if (jt >= 2) ok = mbar_wait(bar(B_KEMPTY + st), par, abortp, c.wait_limit) ? 1 : 0;
           if (ok) {
             // the tile's masks travel to the softmax threads through the barrier chain KFULL -> SREADY; slot jt & 7
             // was last read for tile jt - 8, whose softmax ended before K stage jt - 2 was released
@@ -312,7 +317,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             tma_load_2d(sK + lane * 16384 + (uint32_t)pslot[p] * 128u, &kvmaps[pbox[p]], lane * 64,
                         (int)((long long)w.slab_row0 + ptok[p]), bar(B_KFULL + st));
         if (lane == 0) {
-          if (jt >= 2) ok = mbar_wait(bar(B_VEMPTY + st), par, abortp) ? 1 : 0;
+          if (jt >= 2) ok = mbar_wait(bar(B_VEMPTY + st), par, abortp, c.wait_limit) ? 1 : 0;
           if (ok) mbar_expect_tx(bar(B_VFULL + st), bytes);
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -328,7 +333,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     if (lane == 0)
       for (int back = 1; back <= 2 && back <= jt; ++back) {
         const int jj = jt - back;
-        if (!mbar_wait(bar(B_VEMPTY + (jj & 1)), (jj >> 1) & 1, abortp)) break;
+        if (!mbar_wait(bar(B_VEMPTY + (jj & 1)), (jj >> 1) & 1, abortp, c.wait_limit)) break;
       }
     __syncwarp();
   } else if (warp == 17) {
@@ -367,11 +372,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       int jt = 0;
       bool ok = true;
       for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
-        ok = mbar_wait(bar(B_QFULL), wi & 1, abortp);
+        ok = mbar_wait(bar(B_QFULL), wi & 1, abortp, c.wait_limit);
         if (!ok) break;
         const int T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
         if (T > 0) {
-          ok = mbar_wait(bar(B_KFULL + (jt & 1)), (jt >> 1) & 1, abortp);
+          ok = mbar_wait(bar(B_KFULL + (jt & 1)), (jt >> 1) & 1, abortp, c.wait_limit);
           if (!ok) break;
           fence_after_sync();
           issue_qk(0, jt & 1);
@@ -384,32 +389,32 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         for (int j = 0; ok && j < T; ++j, ++jt) {
           const int st = jt & 1, nst = st ^ 1;
           const bool acc = (j > 0) || (phase == 1);
-          ok = mbar_wait(bar(B_VFULL + st), (jt >> 1) & 1, abortp);
+          ok = mbar_wait(bar(B_VFULL + st), (jt >> 1) & 1, abortp, c.wait_limit);
           if (!ok) break;
-          ok = mbar_wait(bar(B_PREADY + 0), jt & 1, abortp);
+          ok = mbar_wait(bar(B_PREADY + 0), jt & 1, abortp, c.wait_limit);
           if (!ok) break;
           // the first P.V product of an item overwrites O: the previous item's epilogue must have read it
           if (j == 0 && wi > 0) {
-            ok = mbar_wait(bar(B_OFREE + 0), (wi - 1) & 1, abortp) && mbar_wait(bar(B_OFREE + 1), (wi - 1) & 1, abortp);
+            ok = mbar_wait(bar(B_OFREE + 0), (wi - 1) & 1, abortp, c.wait_limit) && mbar_wait(bar(B_OFREE + 1), (wi - 1) & 1, abortp, c.wait_limit);
             if (!ok) break;
           }
           fence_after_sync();
           issue_pv(0, st, acc, 0);
-          ok = mbar_wait(bar(B_PREADY + 2), jt & 1, abortp);
+          ok = mbar_wait(bar(B_PREADY + 2), jt & 1, abortp, c.wait_limit);
           if (!ok) break;
           fence_after_sync();
           issue_pv(0, st, acc, 1);
           if (j + 1 < T) {
-            ok = mbar_wait(bar(B_KFULL + nst), ((jt + 1) >> 1) & 1, abortp);
+            ok = mbar_wait(bar(B_KFULL + nst), ((jt + 1) >> 1) & 1, abortp, c.wait_limit);
             if (!ok) break;
             fence_after_sync();
             issue_qk(0, nst);
           }
-          ok = mbar_wait(bar(B_PREADY + 1), jt & 1, abortp);
+          ok = mbar_wait(bar(B_PREADY + 1), jt & 1, abortp, c.wait_limit);
           if (!ok) break;
           fence_after_sync();
           issue_pv(1, st, acc, 0);
-          ok = mbar_wait(bar(B_PREADY + 3), jt & 1, abortp);
+          ok = mbar_wait(bar(B_PREADY + 3), jt & 1, abortp, c.wait_limit);
           if (!ok) break;
           fence_after_sync();
           issue_pv(1, st, acc, 1);
@@ -446,6 +451,36 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       const int h = w.g * G + rr % G;
       const bool row_ok = tk < a.n;
       const int layer = w.layer;
+      // Bound of the item's logits: |q . k| <= |q| |k|.  This thread sums the squares of its half of its query row
+      // (eight 16-byte loads, in flight during the wait below); the largest squared key norm of the (sequence,
+      // layer, KV head) is kept up to date by the append kernels.  Every thread reads the same word, whatever its
+      // own state, because the decision taken from it below has to be the same in all 256 threads of the Q tile.
+      const unsigned kmax_bits = c.kmax2[w.unit * c.Hkv + w.g];
+      float qn2 = 0.f;
+      if (row_ok) {
+        const uint4* qp =
+            reinterpret_cast<const uint4*>(a.q + (((size_t)w.l * a.n + tk) * c.Hq + h) * kD + half * 64);
+        uint4 piece[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) piece[i] = __ldg(qp + i);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&piece[i]);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(p2[e]);
+            qn2 = fmaf(f.x, f.x, qn2);
+            qn2 = fmaf(f.y, f.y, qn2);
+          }
+        }
+      }
+      // true when some logit of the item may exceed the softmax reference by more than the exponent range leaves
+      // room for; read after the first tile's barrier, by which every thread has published its partial norm
+      auto logits_may_overflow = [&]() -> bool {
+        const float q2 = __uint_as_float(s_qn[q][0]) + __uint_as_float(s_qn[q][1]);
+        const float bound = sqrtf(q2 * __uint_as_float(kmax_bits)) * c2;   // |scaled logit| <= bound, in log2 units
+        return !(2.02f * bound + kRescaleThreshold <= kLazyRange);
+      };
       if (ok) {
         // wait (bounded) until the producer has published this item's key ranges
         const long long t0c = clock64();
@@ -454,7 +489,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             ok = false;
             break;
           }
-          if (clock64() - t0c > kWaitLimitCycles) {
+          if (clock64() - t0c > c.wait_limit) {
             *abortp = 1;
             ok = false;
             break;
@@ -497,14 +532,18 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       int j = 0;
       const int row_abs = a.t0 + tk;
       bool need_ref = true;   // no reference maximum yet: the first tile exchanges the halves' maxima
+      bool exch = false;      // the item's logits are too wide for the late reference: every tile exchanges
       float mprev = -INFINITY;
       while (j < T) {
         // after an expired wait every thread keeps walking the item's tiles (without computing) so that the named
         // barrier is still reached by all 256 threads of the tile
-        ok = ok && mbar_wait(bar(B_SREADY + q), jt & 1, abortp);
+        ok = ok && mbar_wait(bar(B_SREADY + q), jt & 1, abortp, c.wait_limit);
         if (!ok) {
-          if (need_ref) asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
-          need_ref = false;
+          if (need_ref) {
+            asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
+            if (j == 0) exch = logits_may_overflow();
+          }
+          need_ref = exch;
           ++j;
           ++jt;
           continue;
@@ -544,18 +583,27 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         // they exchange their maxima through shared memory and a named barrier.  On later tiles the reference moves
         // one tile late: it is the maximum over the previous tiles, whose partner half is already visible (the
         // partner stored it before its PREADY arrival of the previous tile, which precedes this tile's SREADY), so
-        // no barrier sits between the logits and the exponentials.  A tile that exceeds the reference is harmless
-        // (the exponent is merely positive) unless it does so by more than 2^100, which raises the status word.
+        // no barrier sits between the logits and the exponentials.  A tile that exceeds the late reference only
+        // makes the exponent positive, by at most twice the bound |q| |k| scale of the item's logits plus the lazy
+        // threshold; the first tile's barrier also settles, for the whole Q tile at once, whether that stays inside
+        // the exponent range.  If it may not, every tile of the item exchanges its maxima like the first one, so the
+        // exponent never exceeds the lazy threshold and inputs of any norm give the exact softmax.
         s_max[jt & 1][q][half][r] = mloc;
         float mt;
         if (need_ref) {
+          if (j == 0) {
+            // (qn2 >= 0: the bit patterns order like the values; lanes whose wait expired are not here)
+            const unsigned peers = __activemask();
+            const unsigned wq = __reduce_max_sync(peers, __float_as_uint(qn2));
+            if (lane == __ffs(peers) - 1) atomicMax(&s_qn[q][half], wq);
+          }
           asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
           mt = fmaxf(mloc, s_max[jt & 1][q][half ^ 1][r]) * c2;
+          if (j == 0) exch = logits_may_overflow();
         } else {
           mt = fmaxf(mprev, s_max[(jt & 1) ^ 1][q][half ^ 1][r]) * c2;
-          if (mloc * c2 > m_used + 100.f && m_used > -INFINITY) set_status(c, -5, 7000 + (int)blockIdx.x);
         }
-        need_ref = false;
+        need_ref = exch;
         mprev = mloc;
         // lazy running maximum: move it only when it grows by more than the threshold (or on first use)
         float alpha = 1.f;
@@ -609,7 +657,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       s_sum[q][half][r] = lsum;
       asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
       lsum += s_sum[q][half ^ 1][r];
-      if (ok) ok = mbar_wait(bar(B_ODONE), wi & 1, abortp);
+      if (r == 0) s_qn[q][half] = 0u;  // every thread read it after the item's first tile; the next item starts at zero
+      if (ok) ok = mbar_wait(bar(B_ODONE), wi & 1, abortp, c.wait_limit);
       if (!ok) s_quit[q] = 1;
       asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");  // also: s_sum is reused by the next item
       if (s_quit[q]) break;  // collective decision: all 256 threads of the tile leave after the same item

@@ -1,4 +1,4 @@
-// Decode attention (Sec. 3.5: the block becomes a single token): memory-bound split-KV flash-decoding over the
+// Decode attention (Sec. 3.5: while decoding, the current block is one token): memory-bound split-KV flash-decoding over the
 // token ranges [sink | selected spans | tokens since the last eviction].  Every K/V row is read once with 16-byte
 // loads and shared by the G query heads of its KV group; softmax reductions use warp shuffles.
 #include "common.cuh"

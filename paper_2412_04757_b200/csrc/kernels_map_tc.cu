@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     int it = 0;
     for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
       const int st = it & 1;
-      if (lane == 0 && it >= 2) ok = mbar_wait(bar(B_QEMPTY + st), ((it >> 1) - 1) & 1, abortp) ? 1 : 0;
+      if (lane == 0 && it >= 2) ok = mbar_wait(bar(B_QEMPTY + st), ((it >> 1) - 1) & 1, abortp, c.wait_limit) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
 #pragma unroll
@@ -175,24 +175,24 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     if (lane == 0)
       for (int back = 1; back <= 2 && back <= it; ++back) {  // no copy may be in flight at exit
         const int ii = it - back;
-        if (!mbar_wait(bar(B_QEMPTY + (ii & 1)), (ii >> 1) & 1, abortp)) break;
+        if (!mbar_wait(bar(B_QEMPTY + (ii & 1)), (ii >> 1) & 1, abortp, c.wait_limit)) break;
       }
   } else if (warp == 17) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(128, 128, false);
       const uint64_t dK = make_desc(sK, 16, 1024), dQ = make_desc(sQ, 16, 1024);
       const uint64_t dXa = make_desc_noswizzle(sXa, 128, 256), dXb = make_desc_noswizzle(sXb, 128, 256);
-      bool ok = mbar_wait(bar(B_KFULL), 0, abortp);
+      bool ok = mbar_wait(bar(B_KFULL), 0, abortp, c.wait_limit);
       int it = 0, seq = 0;
       for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
         const int st = it & 1;
-        ok = mbar_wait(bar(B_QFULL + st), (it >> 1) & 1, abortp);
+        ok = mbar_wait(bar(B_QFULL + st), (it >> 1) & 1, abortp, c.wait_limit);
         if (!ok) break;
         const uint64_t db = dQ + (uint64_t)((st * 32768) >> 4);
         for (int kt = 0; ok && kt < ntile; ++kt) {
           if (blk < blk0_of(kt)) continue;
           const int buf = seq & 3;
-          if (seq >= 4) ok = mbar_wait(bar(B_SEMPTY + buf), ((seq >> 2) - 1) & 1, abortp);
+          if (seq >= 4) ok = mbar_wait(bar(B_SEMPTY + buf), ((seq >> 2) - 1) & 1, abortp, c.wait_limit);
           if (!ok) break;
           fence_after_sync();
           const uint64_t da = dK + (uint64_t)((kt * 32768) >> 4);
@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
       for (int kt = 0; kt < kMapKT; ++kt) {
         if (kt >= ntile || blk < blk0_of(kt)) continue;
         const int buf = seq & 3;
-        ok = ok && mbar_wait(bar(B_SFULL + buf), (seq >> 2) & 1, abortp);
+        ok = ok && mbar_wait(bar(B_SFULL + buf), (seq >> 2) & 1, abortp, c.wait_limit);
         ++seq;
         if (!ok) break;
         fence_after_sync();

@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kScThreads, kScStages == 2 ? 2 : 1)
       bool ok = true;
       for (int it = 0; ok && it < my_tiles; ++it) {
         const int st = it % kScStages;
-        if (it >= kScStages) ok = mbar_wait(bar(B_AEMPTY + st), ((it / kScStages) - 1) & 1, abortp);
+        if (it >= kScStages) ok = mbar_wait(bar(B_AEMPTY + st), ((it / kScStages) - 1) & 1, abortp, c.wait_limit);
         if (!ok) break;
         const long long row = row0 + (long long)(tile0 + it) * 128;
         mbar_expect_tx(bar(B_AFULL + st), 32768);
@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(kScThreads, kScStages == 2 ? 2 : 1)
       }
       for (int back = 1; back <= kScStages && back <= my_tiles; ++back) {  // no copy in flight at exit
         const int ii = my_tiles - back;
-        if (!mbar_wait(bar(B_AEMPTY + (ii % kScStages)), (ii / kScStages) & 1, abortp)) break;
+        if (!mbar_wait(bar(B_AEMPTY + (ii % kScStages)), (ii / kScStages) & 1, abortp, c.wait_limit)) break;
       }
     }
   } else if (warp == 5) {
@@ -124,9 +124,9 @@ __global__ void __launch_bounds__(kScThreads, kScStages == 2 ? 2 : 1)
       bool ok = true;
       for (int it = 0; ok && it < my_tiles; ++it) {
         const int st = it % kScStages, buf = it & 1;
-        ok = mbar_wait(bar(B_AFULL + st), (it / kScStages) & 1, abortp);
+        ok = mbar_wait(bar(B_AFULL + st), (it / kScStages) & 1, abortp, c.wait_limit);
         if (!ok) break;
-        if (it >= 2) ok = mbar_wait(bar(B_SEMPTY + buf), ((it >> 1) - 1) & 1, abortp);
+        if (it >= 2) ok = mbar_wait(bar(B_SEMPTY + buf), ((it >> 1) - 1) & 1, abortp, c.wait_limit);
         if (!ok) break;
         fence_after_sync();
         const uint64_t da = dA + (uint64_t)((st * 32768) >> 4);
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kScThreads, kScStages == 2 ? 2 : 1)
     bool ok = true;
     for (int it = 0; it < my_tiles; ++it) {
       const int buf = it & 1;
-      ok = ok && mbar_wait(bar(B_SFULL + buf), (it >> 1) & 1, abortp);
+      ok = ok && mbar_wait(bar(B_SFULL + buf), (it >> 1) & 1, abortp, c.wait_limit);
       if (!ok) break;
       fence_after_sync();
       float best = -INFINITY;

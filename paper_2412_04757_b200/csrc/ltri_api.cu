@@ -211,6 +211,8 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.rng_cnt = cv.take<int>(units * d.Hkv);
   d.dec_part = cv.take<float>(units * d.Hq * kMaxDecSplit * (kD + 2));
   d.status = cv.take<int>(4);
+  d.kmax2 = cv.take<unsigned>(units * d.Hkv);
+  d.wait_limit = kDefaultWaitLimit;
   d.slots += 1;  // the extra slot is scratch for ltri_debug_segment_map
   if (p.flags & LTRI_FLAG_HOST_STAGING) {
     const size_t set_bytes = stage_set_bytes(p);
@@ -247,7 +249,7 @@ struct ltri_ctx {
   char* host_kv = nullptr;   // the caller's mirror (host address)
   bool spilled = false;      // ev_spill has been recorded at least once
   cudaEvent_t ev_up[2][kHostGroups] = {}, ev_run[2][kHostGroups] = {}, ev_down[2][kHostGroups] = {};
-  bool set_used[2] = {false, false};
+  bool grp_used[2][kHostGroups] = {};  // the events of (set, group) have been recorded at least once
   long long host_calls = 0;
   alignas(64) unsigned char kv_maps[kTcMapBytes];  // TMA descriptors of the K/V cache
   long long launches = 0;  // kernels launched since creation
@@ -490,6 +492,18 @@ int ltri_reset_sequence(ltri_ctx* ctx, int seq, void* cuda_stream) {
   return LTRI_OK;
 }
 
+// Sliding slabs: can tokens up to `t_end` (exclusive) be given rows in the window region of this layer's slabs?
+// Returns 0 when they already fit, 1 when the live rows have to be moved to the start of the region first, and
+// LTRI_ECAPACITY when even that would not make room (decode ran past what a sliding slab can hold).  No side effects.
+static int slide_check(const ltri_ctx* ctx, const LayerState& s0, long long t_end) {
+  const DevCtx& d = ctx->d;
+  const long long cap = d.SR - d.Lsp - kTokPad;  // rows of the window region that may hold tokens
+  if (t_end - s0.base <= cap) return 0;
+  const long long nb = s0.E, live = s0.t - nb, dist = nb - s0.base;
+  if (t_end - nb > cap || dist < live) return LTRI_ECAPACITY;
+  return 1;
+}
+
 // Sliding slabs: make room for tokens up to `t_end` (exclusive) in the window region of the slabs of the given layers.
 // When the region is full, the live rows -- everything since the last eviction, [E, t) -- are moved to its start with
 // one strided device copy for K and one for V; the region is sized so that source and destination cannot overlap.
@@ -497,10 +511,9 @@ int ltri_reset_sequence(ltri_ctx* ctx, int seq, void* cuda_stream) {
 static int slide_window(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, long long t_end, cudaStream_t st) {
   const DevCtx& d = ctx->d;
   LayerState& s0 = ctx->at(seq, layer_begin);
-  const long long cap = d.SR - d.Lsp - kTokPad;  // rows of the window region that may hold tokens
-  if (t_end - s0.base <= cap) return LTRI_OK;
+  const int need = slide_check(ctx, s0, t_end);
+  if (need <= 0) return need;
   const long long nb = s0.E, live = s0.t - nb, dist = nb - s0.base;
-  if (t_end - nb > cap || dist < live) return LTRI_ECAPACITY;  // (decode ran past what a sliding slab can hold)
   if (ctx->spilled) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_spill, 0));
   if (live > 0) {
     const size_t row_bytes = kD * sizeof(__nv_bfloat16), pitch = (size_t)d.SR * row_bytes;
@@ -518,15 +531,22 @@ static int slide_window(ltri_ctx* ctx, int seq, int layer_begin, int layer_count
   return LTRI_OK;
 }
 
-int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q,
-                       const void* k, const void* v, void* out, void* cuda_stream) {
-  if (!ctx) return LTRI_EINVAL;
+// Everything a prefill call decides on the host before it enqueues work: which regions leave the window, where the
+// indexed prefix ends afterwards, the call's own region and the pending slot it gets.
+struct PrefillPlan {
+  std::vector<Region> ev;
+  int E = 0, t0 = 0, reg_start = 0, m = 0, slot = -1;
+  long long ub = 0;
+};
+
+// All host-side checks of a prefill call over layers [layer_begin, layer_begin + layer_count); fills `plan`.
+// Changes nothing: a call that fails here leaves the context as it was.
+static int plan_prefill(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, PrefillPlan& plan) {
   const DevCtx& d = ctx->d;
   if (seq < 0 || seq >= d.NS || layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > d.NL)
     return LTRI_EINVAL;
   if (n_tokens < 1 || n_tokens > d.chunk) return LTRI_EINVAL;
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return LTRI_EINVAL;
-  LayerState& s0 = ctx->at(seq, layer_begin);
+  const LayerState& s0 = ctx->at(seq, layer_begin);
   for (int l = 0; l < layer_count; ++l) {
     const LayerState& s = ctx->at(seq, layer_begin + l);
     if (s.decoding) return LTRI_ESTATE;
@@ -534,14 +554,13 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   }
   if (s0.t + n_tokens > d.Tmax) return LTRI_ECAPACITY;
   const int t0 = (int)s0.t;
-
-  // plan the evictions (host knows region boundaries; span counts live on the device)
-  std::vector<Region> ev;
+  // the evictions (the host knows the region boundaries; the span counts live on the device)
+  plan.ev.clear();
   int E = s0.E;
   long long ub = s0.span_ub;
   for (const Region& r : s0.pending) {
     if (r.end <= t0 - d.W) {
-      ev.push_back(r);
+      plan.ev.push_back(r);
       E = r.end;
       ub += std::min(d.Jmax, r.end - r.start);
     } else
@@ -551,18 +570,42 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   const int reg_start = std::max(d.Ls, t0);
   const int m = std::max(0, t0 + n_tokens - reg_start);
   const int user_slots = d.slots - 1;
-  if (m > 0 && (int)(s0.pending.size() - ev.size()) + 1 > user_slots) return LTRI_ECAPACITY;
+  if (m > 0 && (int)(s0.pending.size() - plan.ev.size()) + 1 > user_slots) return LTRI_ECAPACITY;
   int slot = -1;
   if (m > 0) {
     // first slot not used by a region that stays pending
     std::vector<char> used(user_slots, 0);
-    for (size_t i = ev.size(); i < s0.pending.size(); ++i) used[s0.pending[i].slot] = 1;
+    for (size_t i = plan.ev.size(); i < s0.pending.size(); ++i) used[s0.pending[i].slot] = 1;
     for (int i = 0; i < user_slots; ++i)
       if (!used[i]) {
         slot = i;
         break;
       }
   }
+  if (d.paged && slide_check(ctx, s0, (long long)t0 + n_tokens) < 0) return LTRI_ECAPACITY;
+  plan.E = E;
+  plan.ub = ub;
+  plan.t0 = t0;
+  plan.reg_start = reg_start;
+  plan.m = m;
+  plan.slot = slot;
+  return LTRI_OK;
+}
+
+int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count, int n_tokens, const void* q,
+                       const void* k, const void* v, void* out, void* cuda_stream) {
+  if (!ctx) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return LTRI_EINVAL;
+  PrefillPlan plan;
+  {
+    const int rc = plan_prefill(ctx, seq, layer_begin, layer_count, n_tokens, plan);
+    if (rc != LTRI_OK) return rc;
+  }
+  LayerState& s0 = ctx->at(seq, layer_begin);
+  const std::vector<Region>& ev = plan.ev;
+  const int t0 = plan.t0, E = plan.E, reg_start = plan.reg_start, m = plan.m, slot = plan.slot;
+  const long long ub = plan.ub;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   PrefillArgs a;
   a.seq = seq;
@@ -675,9 +718,14 @@ int ltri_prefill_chunk_host(ltri_ctx* ctx, int seq, int layer_begin, int layer_c
   if (!ctx) return LTRI_EINVAL;
   if (!ctx->stage[0]) return LTRI_ESTATE;  // created without LTRI_FLAG_HOST_STAGING
   const DevCtx& d = ctx->d;
-  if (seq < 0 || seq >= d.NS || layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > d.NL)
-    return LTRI_EINVAL;
-  if (n_tokens < 1 || n_tokens > d.chunk || !q_host || !k_host || !v_host || !out_host) return LTRI_EINVAL;
+  if (!q_host || !k_host || !v_host || !out_host) return LTRI_EINVAL;
+  {
+    // every host-side check of the whole call first: the layers of a call are in the same state, so what holds for
+    // the full range holds for each layer group, and an error return leaves the sequence untouched
+    PrefillPlan plan;
+    const int rc = plan_prefill(ctx, seq, layer_begin, layer_count, n_tokens, plan);
+    if (rc != LTRI_OK) return rc;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int set = (int)(ctx->host_calls & 1);
   const size_t rows = (size_t)d.NL * d.chunk;
@@ -686,34 +734,38 @@ int ltri_prefill_chunk_host(ltri_ctx* ctx, int seq, int layer_begin, int layer_c
   char* sk = sq + qb;
   char* sv = sk + kb;
   char* so = sv + kb;
-  const int ng = std::min((int)ltri_ctx::kHostGroups, layer_count);
+  // The layer groups are those of the CONTEXT (layers [NL g / G, NL (g + 1) / G) for group g), whatever range the call
+  // covers, and a layer's staging bytes start at layer * chunk rows: a group always owns the same bytes of a staging
+  // set, so the events of (set, group) order every reuse of them, also between calls of different sizes.  Inside a
+  // group's slice the call's layers are dense (n_tokens rows apart), as the device entry wants them.
+  const int G = std::min((int)ltri_ctx::kHostGroups, d.NL);
   const size_t qrow = (size_t)n_tokens * d.Hq * kD * 2, krow = (size_t)n_tokens * d.Hkv * kD * 2;  // bytes per layer
-  for (int g = 0; g < ng; ++g) {
-    const int lo = layer_count * g / ng, hi = layer_count * (g + 1) / ng;  // layers of the group, call-relative
-    const size_t qo = lo * qrow, ko = lo * krow, qn = (hi - lo) * qrow, kn = (hi - lo) * krow;
-    // up: the kernels that read this slice two calls ago are done
-    if (ctx->set_used[set]) LTRI_CUDA(ctx, cudaStreamWaitEvent(ctx->s_up, ctx->ev_run[set][g], 0));
-    LTRI_CUDA(ctx, cudaMemcpyAsync(sq + qo, static_cast<const char*>(q_host) + qo, qn, cudaMemcpyHostToDevice, ctx->s_up));
-    LTRI_CUDA(ctx, cudaMemcpyAsync(sk + ko, static_cast<const char*>(k_host) + ko, kn, cudaMemcpyHostToDevice, ctx->s_up));
-    LTRI_CUDA(ctx, cudaMemcpyAsync(sv + ko, static_cast<const char*>(v_host) + ko, kn, cudaMemcpyHostToDevice, ctx->s_up));
+  const size_t qlay = (size_t)d.chunk * d.Hq * kD * 2, klay = (size_t)d.chunk * d.Hkv * kD * 2;     // staging stride
+  for (int g = 0; g < G; ++g) {
+    const int lo = std::max(layer_begin, d.NL * g / G), hi = std::min(layer_begin + layer_count, d.NL * (g + 1) / G);
+    if (lo >= hi) continue;
+    const size_t qs = lo * qlay, ks = lo * klay;                                  // staging offsets of the slice
+    const size_t qh = (lo - layer_begin) * qrow, kh = (lo - layer_begin) * krow;  // offsets in the caller's tensors
+    const size_t qn = (hi - lo) * qrow, kn = (hi - lo) * krow;
+    // up: the kernels that read this group's slice of the set (two calls ago) are done
+    if (ctx->grp_used[set][g]) LTRI_CUDA(ctx, cudaStreamWaitEvent(ctx->s_up, ctx->ev_run[set][g], 0));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(sq + qs, static_cast<const char*>(q_host) + qh, qn, cudaMemcpyHostToDevice, ctx->s_up));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(sk + ks, static_cast<const char*>(k_host) + kh, kn, cudaMemcpyHostToDevice, ctx->s_up));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(sv + ks, static_cast<const char*>(v_host) + kh, kn, cudaMemcpyHostToDevice, ctx->s_up));
     LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_up[set][g], ctx->s_up));
     // run: inputs are up, and the output slice written two calls ago has gone down
     LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_up[set][g], 0));
-    if (ctx->set_used[set]) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down[set][g], 0));
-    const int rc = ltri_prefill_chunk(ctx, seq, layer_begin + lo, hi - lo, n_tokens, sq + qo, sk + ko, sv + ko, so + qo, st);
+    if (ctx->grp_used[set][g]) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down[set][g], 0));
+    // (after the checks above this can only fail in the CUDA runtime)
+    const int rc = ltri_prefill_chunk(ctx, seq, lo, hi - lo, n_tokens, sq + qs, sk + ks, sv + ks, so + qs, st);
     if (rc != LTRI_OK) return rc;
     LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_run[set][g], st));
     // down
     LTRI_CUDA(ctx, cudaStreamWaitEvent(ctx->s_down, ctx->ev_run[set][g], 0));
-    LTRI_CUDA(ctx, cudaMemcpyAsync(static_cast<char*>(out_host) + qo, so + qo, qn, cudaMemcpyDeviceToHost, ctx->s_down));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(static_cast<char*>(out_host) + qh, so + qs, qn, cudaMemcpyDeviceToHost, ctx->s_down));
     LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_down[set][g], ctx->s_down));
+    ctx->grp_used[set][g] = true;
   }
-  // groups beyond ng keep their old events; make them harmless for the next use of this set
-  for (int g = ng; g < ltri_ctx::kHostGroups; ++g) {
-    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_run[set][g], st));
-    LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_down[set][g], ctx->s_down));
-  }
-  ctx->set_used[set] = true;
   ctx->host_calls += 1;
   return LTRI_OK;
 }
@@ -723,8 +775,8 @@ int ltri_host_outputs_ready(ltri_ctx* ctx, void* cuda_stream) {
   if (!ctx->stage[0]) return LTRI_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   for (int s = 0; s < 2; ++s)
-    if (ctx->set_used[s])
-      for (int g = 0; g < ltri_ctx::kHostGroups; ++g) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down[s][g], 0));
+    for (int g = 0; g < ltri_ctx::kHostGroups; ++g)
+      if (ctx->grp_used[s][g]) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down[s][g], 0));
   return LTRI_OK;
 }
 
@@ -744,6 +796,7 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
     const LayerState& s0 = ctx->at(sq, layer_begin);
     if (s0.t < 1) return LTRI_ESTATE;
     if (s0.t + 1 > d.Tmax) return LTRI_ECAPACITY;
+    if (d.paged && slide_check(ctx, s0, s0.t + 1) < 0) return LTRI_ECAPACITY;  // (before anything is enqueued)
     for (int l = 0; l < layer_count; ++l) {
       const LayerState& s = ctx->at(sq, layer_begin + l);
       if (s.t != s0.t || s.E != s0.E || s.base != s0.base) return LTRI_ESTATE;
@@ -1091,6 +1144,54 @@ int ltri_debug_segment_map(ltri_ctx* ctx, const int32_t* Mq, int m, int theta_mo
     pairs[2 * i] = a[i];
     pairs[2 * i + 1] = b[i];
   }
+  return LTRI_OK;
+}
+
+int ltri_debug_load_index(ltri_ctx* ctx, int seq, int layer, int64_t evicted_end, const int32_t* pairs, int n_spans,
+                          const void* index_bf16, void* cuda_stream) {
+  if (!ctx || seq < 0 || seq >= ctx->d.NS || layer < 0 || layer >= ctx->d.NL || n_spans < 0) return LTRI_EINVAL;
+  const DevCtx& d = ctx->d;
+  LayerState& s = ctx->at(seq, layer);
+  if (n_spans > 0 && (!pairs || !index_bf16)) return LTRI_EINVAL;
+  if (evicted_end != s.E) return LTRI_ESTATE;  // the cache, the votes and the pending regions stay as they are
+  if (n_spans > d.cap) return LTRI_ECAPACITY;
+  // the spans must cover [n_sink, E) in token order (they may overlap, as the spans of an NMS with phi > 0 do)
+  long long reach = d.Ls;
+  std::vector<int> st_(n_spans), ln_(n_spans);
+  for (int i = 0; i < n_spans; ++i) {
+    const long long a = pairs[2 * i], len = pairs[2 * i + 1];
+    if (len < 1 || a < d.Ls || a > reach || a + len > s.E || (i > 0 && a < pairs[2 * i - 2])) return LTRI_EINVAL;
+    reach = std::max(reach, a + len);
+    st_[i] = (int)a;
+    ln_[i] = (int)len;
+  }
+  if (reach != s.E) return LTRI_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t unit = unit_of(d, seq, layer);
+  if (n_spans > 0) {
+    LTRI_CUDA(ctx, cudaMemcpyAsync(d.span_start + unit * d.cap, st_.data(), n_spans * sizeof(int), cudaMemcpyHostToDevice, st));
+    LTRI_CUDA(ctx, cudaMemcpyAsync(d.span_len + unit * d.cap, ln_.data(), n_spans * sizeof(int), cudaMemcpyHostToDevice, st));
+    for (int g = 0; g < d.Hkv; ++g)
+      LTRI_CUDA(ctx, cudaMemcpyAsync(d.KR + (unit * d.Hkv + g) * (size_t)d.cap * kD,
+                                     static_cast<const __nv_bfloat16*>(index_bf16) + (size_t)g * n_spans * kD,
+                                     (size_t)n_spans * kD * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice, st));
+  }
+  LTRI_CUDA(ctx, cudaMemcpyAsync(d.n_spans + unit, &n_spans, sizeof(int), cudaMemcpyHostToDevice, st));
+  LTRI_CUDA(ctx, cudaStreamSynchronize(st));  // the host buffers (and the locals above) may go away on return
+  s.span_ub = n_spans;
+  return LTRI_OK;
+}
+
+int ltri_debug_wait_timeout(ltri_ctx* ctx, int64_t limit_cycles, int64_t* waited_cycles, void* cuda_stream) {
+  if (!ctx || !waited_cycles || limit_cycles < 1 || limit_cycles > 100000000ll) return LTRI_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->launches += 1;
+  LTRI_CUDA(ctx, launch_wait_probe(ctx->d, (long long)limit_cycles, st));
+  int w[4] = {0, 0, 0, 0};
+  const int rc = copy_back(ctx, w, ctx->d.status, sizeof(w), st);
+  if (rc) return rc;
+  waited_cycles[0] = w[2];
+  waited_cycles[1] = w[3];
   return LTRI_OK;
 }
 

@@ -39,8 +39,15 @@ std::mutex g_mu;
 void* g_scratch_addr[kMaxDevices] = {nullptr};
 
 // interleave the segmenter's {start[], len[]} arrays into the caller's {start,len} pairs
+// (status: the word the segmenter's device-side checks write; a failed check is reported through *n_out)
 __global__ void k_pack_spans(const int* __restrict__ start, const int* __restrict__ len, const int* __restrict__ cnt,
-                             int cap_pairs, int32_t* __restrict__ pairs, int32_t* __restrict__ n_out) {
+                             const int* __restrict__ status, int cap_pairs, int32_t* __restrict__ pairs,
+                             int32_t* __restrict__ n_out) {
+  const int code = *status;
+  if (code != 0) {
+    if (threadIdx.x == 0) *n_out = (code <= LTRI_EINVAL && code >= LTRI_ETIMEOUT) ? code : LTRI_EDEVICE;
+    return;
+  }
   const int n = *cnt;
   for (int i = threadIdx.x; i < n && i < cap_pairs; i += blockDim.x) {
     pairs[2 * i] = start[i];
@@ -58,6 +65,16 @@ extern "C" int ltri_segment_map_static(const int32_t* Mq, int m, int64_t theta_q
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return LTRI_ECUDA;
   if (dev < 0 || dev >= kMaxDevices) return LTRI_ECAPACITY;
+  {
+    // the scratch used below is the current device's: a map that the runtime knows to live on another device would
+    // be read across devices (or not at all), so it is refused here; pointers the runtime cannot attribute pass
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, Mq) == cudaSuccess) {
+      if (attr.type == cudaMemoryTypeDevice && attr.device != dev) return LTRI_EINVAL;
+    } else {
+      cudaGetLastError();
+    }
+  }
   unsigned char* base = nullptr;
   {
     // first call on this device: resolve the device address of the scratch array (not capturable work)
@@ -94,6 +111,6 @@ extern "C" int ltri_segment_map_static(const int32_t* Mq, int m, int64_t theta_q
   if (cudaMemsetAsync(base + kOffPendCnt, 0, kScratchBytes - kOffPendCnt, st) != cudaSuccess) return LTRI_ECUDA;
   if (launch_segment(c, 0, 0, 1, m, 0, 0, /*theta_mode=*/0, 0.f, theta_q, max_spans, 0, 0, nullptr, st) != cudaSuccess)
     return LTRI_ECUDA;
-  k_pack_spans<<<1, 128, 0, st>>>(c.pend_start, c.pend_len, c.pend_cnt, cap_pairs, pairs, n_out);
+  k_pack_spans<<<1, 128, 0, st>>>(c.pend_start, c.pend_len, c.pend_cnt, c.status, cap_pairs, pairs, n_out);
   return cudaGetLastError() == cudaSuccess ? LTRI_OK : LTRI_ECUDA;
 }

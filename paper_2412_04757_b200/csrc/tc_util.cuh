@@ -8,8 +8,9 @@
 namespace ltri {
 namespace tc {
 
-// Upper bound of any single wait, in SM clock cycles (about one second).  A wait that expires sets the CTA's abort
-// flag and the kernel's status word; every other wait of the CTA then returns at once and the CTA tears down.
+// Default upper bound of any single wait, in SM clock cycles (about one second); a context carries its own limit
+// (DevCtx::wait_limit), which every kernel hands to its waits.  A wait that expires sets the CTA's abort flag and
+// the kernel's status word; every other wait of the CTA then returns at once and the CTA tears down.
 constexpr long long kWaitLimitCycles = 2000000000ll;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -53,7 +54,7 @@ __device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity, 
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait expired, or another one did).  The abort flag and
 // the clock are looked at only between bursts of suspended tries, so a waiting warp issues few instructions.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
@@ -61,7 +62,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 8; ++i)
       if (mbar_try_suspend(bar, parity, 2000u)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       return false;
     }
