@@ -101,9 +101,6 @@ struct DevCtx {
   int* rng_cnt;          // [NS*NL][Hkv]
   float* dec_part;       // [NS*NL][Hq][kMaxDecSplit][128+2]
   int* status;           // [4]: first error code, detail...
-  unsigned* kmax2;       // [NS][NL][Hkv]  largest squared norm of any key appended so far (bit pattern of a
-                         //                non-negative float, which orders like the unsigned integer): bounds every
-                         //                logit of the (sequence, layer, KV head) by |q| * sqrt(kmax2) * scale
   long long wait_limit;  // upper bound of any single device-side wait, in SM clock cycles
 };
 
@@ -176,7 +173,8 @@ int dec_retrieve_fused_max_spans();
 cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, cudaStream_t s);
 
 // prefill attention.  phase 0: local part over sink|local|cur, stores state (+ final output if `final`);
-// phase 1: continues from the stored state over the selected spans and writes the output.
+// phase 1: continues from the stored state over the selected spans and writes the output; phase 2 (tensor-core
+// kernel only): the same result, with the selected spans accumulated from scratch and merged with the stored state.
 cudaError_t launch_attn_prefill(const DevCtx& c, const PrefillArgs& a, int phase, bool final, cudaStream_t s);
 // tcgen05/TMEM/TMA version of launch_attn_prefill (same contract) and its availability check
 // host storage for a context's tensor maps: five box heights of the K/V cache, the index, five of the packed slabs

@@ -29,8 +29,9 @@ constexpr float kLog2eT = 1.4426950408889634f;
 constexpr int kTcThreads = 576;  // 16 softmax warps + TMA producer + MMA issuer
 constexpr int kNumBoxes = 5;  // box heights 8,16,32,64,128
 constexpr float kRescaleThreshold = 8.0f;
-// Largest exponent (log2 units) a probability may carry above the softmax reference: 2^90 times the 2^7 keys of a
-// tile, the 2^13 tiles of the longest item and values of up to 2^10 still fits fp32 (and the bf16 P operand).
+// Largest exponent (log2 units) a probability may carry above the softmax reference in the first pass: 2^90 times
+// the 2^7 keys of a tile, the 2^13 tiles of the longest item and values of up to 2^10 still fits fp32 (and the bf16
+// P operand).
 constexpr float kLazyRange = 90.0f;
 
 struct TcMaps {
@@ -143,10 +144,16 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int G>
+// PHASE 0: the local part over sink | local | current keys; stores the row statistics and, unless `final_out`, the
+//          unnormalised accumulator.
+// PHASE 2: the retrieved part over the packed slab of the selected spans, accumulated from scratch; the epilogue
+//          merges it with the state phase 0 stored (log-sum-exp merge of two partial softmaxes) and writes the output.
+// PHASE 1: the retrieved part as a continuation: the stored state is loaded back into registers / TMEM first.  Kept
+//          as a cross-check of phase 2.
+template <int G, int PHASE>
 __global__ void __launch_bounds__(kTcThreads, 1)
-    k_attn_tc(DevCtx c, PrefillArgs a, int phase, int final_out, const __grid_constant__ TcMaps maps,
-              long long v_row_offset) {
+    k_attn_tc(DevCtx c, PrefillArgs a, int final_out, const __grid_constant__ TcMaps maps, long long v_row_offset) {
+  constexpr int phase = PHASE;
   const CUtensorMap* kvmaps = maps.kv;
   extern __shared__ unsigned char smem_raw[];
   // QFULL QFREE ODONE | KFULL[2] VFULL[2] KEMPTY[2] VEMPTY[2] | SREADY[2] PREADY[2][2] OFREE[2]
@@ -157,10 +164,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __shared__ int s_item_tiles[3];     // tile count of the work items in flight (roles may be up to two items apart)
   __shared__ TileDesc s_td[8];        // per-tile masks, written by the producer, read by the softmax threads
   __shared__ int s_quit[2];
+  __shared__ int s_redo;              // some tile of the first pass outran the late reference: second pass needed
   __shared__ int s_items_ready;       // number of work items whose key ranges the producer has published
   __shared__ float s_max[2][2][2][128];  // per tile parity, Q tile, column half, row: partial maxima
   __shared__ float s_sum[2][2][128];     // per Q tile, column half, row: partial row sums (end of an item)
-  __shared__ unsigned s_qn[2][2];        // per Q tile, column half: largest partial squared query norm of the item
   constexpr int TOKB = 256 / G;  // tokens per work item
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // persistent CTA: work items (token block, KV head, layer) are dealt round-robin
@@ -180,8 +187,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   if (tid == 0) {
     s_abort = 0;
     s_quit[0] = s_quit[1] = 0;
+    s_redo = 0;
     s_items_ready = 0;
-    s_qn[0][0] = s_qn[0][1] = s_qn[1][0] = s_qn[1][1] = 0u;
     rg.n = 0;
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QFREE), 1);
@@ -233,13 +240,32 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     return ((((size_t)w.layer * MB + w.mb) * c.Hkv + w.g) * 2 + q) * (size_t)(128 * kD);
   };
 
+  // Every role counts the tiles (jt) and the work items (wi) it has handled; the counters run on through the second
+  // pass, since the barrier phases do.
+  int jt = 0, wi = 0, ok = 1;
+  // Two passes over the CTA's work items.  The first uses the late-moving softmax reference (see the softmax role);
+  // a thread that meets a tile whose logits outrun that reference by more than the exponent range allows raises
+  // s_redo.  Then -- and only then -- the second pass walks the same items again with the true maximum exchanged on
+  // every tile and overwrites what the first pass stored, so inputs of any magnitude get the exact softmax; for
+  // ordinary inputs the second pass is one CTA barrier.
+#ifndef LTRI_PASSES
+#define LTRI_PASSES 2
+#endif
+#pragma unroll 1
+  for (int pass = 0; pass < LTRI_PASSES; ++pass) {
+  if (pass == 1) {
+    fence_before_sync();
+    __syncthreads();  // every thread is through its role of the first pass (also after an expired wait)
+    fence_after_sync();
+    if (!s_redo || s_abort) break;
+  }
+  const bool exch = pass == 1;
   if (warp == 16) {
     // ------------------------------------------------------------------ TMA producer
     // Every lane walks the tile list; lane 0 owns the barrier bookkeeping and lanes 0-3 issue the copies of
     // (K low half, K high half, V low half, V high half) so that many small pieces do not serialise on one thread.
-    int jt = 0, ok = 1;
-    if (lane == 0) prefetch_tmap(&maps.q);
-    for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
+    if (lane == 0 && pass == 0) prefetch_tmap(&maps.q);
+    for (int item = blockIdx.x; ok && item < nitems; item += gridDim.x, ++wi) {
       const Item w = decode(item);
       if (lane == 0) {
         // the Q buffer is free once every QK^T product of the previous item has completed
@@ -369,9 +395,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           mma_ts(d, pa + ks * 8 + (ks >> 2) * 32, db + ((ks * 2048) >> 4), idesc_pv, acc || part > 0 || i > 0);
         }
       };
-      int jt = 0;
-      bool ok = true;
-      for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
+      for (int item = blockIdx.x; ok && item < nitems; item += gridDim.x, ++wi) {
         ok = mbar_wait(bar(B_QFULL), wi & 1, abortp, c.wait_limit);
         if (!ok) break;
         const int T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
@@ -443,44 +467,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     const uint32_t tP = tS;  // its 64 probabilities (bf16 pairs) overwrite the first 32 of its own logit columns
     const uint32_t tO = tmem + lane_base + 256 + q * 128 + half * 64;
     const float c2 = c.scale * kLog2eT;
-    int jt = 0;
-    bool ok = true;
-    for (int item = blockIdx.x, wi = 0; item < nitems; item += gridDim.x, ++wi) {
+    for (int item = blockIdx.x; item < nitems; item += gridDim.x, ++wi) {
       const Item w = decode(item);
       const int tk = w.tok0 + rr / G;              // call-relative token
       const int h = w.g * G + rr % G;
       const bool row_ok = tk < a.n;
       const int layer = w.layer;
-      // Bound of the item's logits: |q . k| <= |q| |k|.  This thread sums the squares of its half of its query row
-      // (eight 16-byte loads, in flight during the wait below); the largest squared key norm of the (sequence,
-      // layer, KV head) is kept up to date by the append kernels.  Every thread reads the same word, whatever its
-      // own state, because the decision taken from it below has to be the same in all 256 threads of the Q tile.
-      const unsigned kmax_bits = c.kmax2[w.unit * c.Hkv + w.g];
-      float qn2 = 0.f;
-      if (row_ok) {
-        const uint4* qp =
-            reinterpret_cast<const uint4*>(a.q + (((size_t)w.l * a.n + tk) * c.Hq + h) * kD + half * 64);
-        uint4 piece[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) piece[i] = __ldg(qp + i);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&piece[i]);
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(p2[e]);
-            qn2 = fmaf(f.x, f.x, qn2);
-            qn2 = fmaf(f.y, f.y, qn2);
-          }
-        }
-      }
-      // true when some logit of the item may exceed the softmax reference by more than the exponent range leaves
-      // room for; read after the first tile's barrier, by which every thread has published its partial norm
-      auto logits_may_overflow = [&]() -> bool {
-        const float q2 = __uint_as_float(s_qn[q][0]) + __uint_as_float(s_qn[q][1]);
-        const float bound = sqrtf(q2 * __uint_as_float(kmax_bits)) * c2;   // |scaled logit| <= bound, in log2 units
-        return !(2.02f * bound + kRescaleThreshold <= kLazyRange);
-      };
       if (ok) {
         // wait (bounded) until the producer has published this item's key ranges
         const long long t0c = clock64();
@@ -504,6 +496,17 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       if (s_quit[q]) break;
       const int T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
       float m_used = -INFINITY, lsum = 0.f;
+      float2 stat0 = make_float2(0.f, 1.f);  // phase 2: reference maximum and row sum of the local part
+      if (phase == 2 && row_ok) {
+        // the state this item is merged with at its end: fetch the statistics now (used after the tile loop) and pull
+        // the accumulator rows into L2 (one request per 128-byte line: eight rows of a column group)
+        stat0 = c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h];
+        if ((r & 7) == 0) {
+          const float* op = c.Oacc + oacc_base(w, q) + (size_t)(half * 16) * 512 + r * 4;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) asm volatile("prefetch.global.L2 [%0];" ::"l"(op + (size_t)i * 512));
+        }
+      }
       if (ok && phase == 1) {
         // continue from the state the local pass stored: running max, row sum and the unnormalised O row
         const float* op = c.Oacc + oacc_base(w, q) + (size_t)(half * 16) * 512 + r * 4;
@@ -532,17 +535,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       int j = 0;
       const int row_abs = a.t0 + tk;
       bool need_ref = true;   // no reference maximum yet: the first tile exchanges the halves' maxima
-      bool exch = false;      // the item's logits are too wide for the late reference: every tile exchanges
       float mprev = -INFINITY;
       while (j < T) {
         // after an expired wait every thread keeps walking the item's tiles (without computing) so that the named
         // barrier is still reached by all 256 threads of the tile
         ok = ok && mbar_wait(bar(B_SREADY + q), jt & 1, abortp, c.wait_limit);
         if (!ok) {
-          if (need_ref) {
-            asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
-            if (j == 0) exch = logits_may_overflow();
-          }
+          if (need_ref) asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
           need_ref = exch;
           ++j;
           ++jt;
@@ -584,24 +583,17 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         // one tile late: it is the maximum over the previous tiles, whose partner half is already visible (the
         // partner stored it before its PREADY arrival of the previous tile, which precedes this tile's SREADY), so
         // no barrier sits between the logits and the exponentials.  A tile that exceeds the late reference only
-        // makes the exponent positive, by at most twice the bound |q| |k| scale of the item's logits plus the lazy
-        // threshold; the first tile's barrier also settles, for the whole Q tile at once, whether that stays inside
-        // the exponent range.  If it may not, every tile of the item exchanges its maxima like the first one, so the
-        // exponent never exceeds the lazy threshold and inputs of any norm give the exact softmax.
+        // makes the exponent positive; if it does so by more than kLazyRange the results of this pass are not to
+        // be trusted (the probabilities may overflow) and the thread asks for the second pass, in which every tile
+        // exchanges its maxima like the first one (exch) and the exponent never exceeds the lazy threshold.
         s_max[jt & 1][q][half][r] = mloc;
         float mt;
         if (need_ref) {
-          if (j == 0) {
-            // (qn2 >= 0: the bit patterns order like the values; lanes whose wait expired are not here)
-            const unsigned peers = __activemask();
-            const unsigned wq = __reduce_max_sync(peers, __float_as_uint(qn2));
-            if (lane == __ffs(peers) - 1) atomicMax(&s_qn[q][half], wq);
-          }
           asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
           mt = fmaxf(mloc, s_max[jt & 1][q][half ^ 1][r]) * c2;
-          if (j == 0) exch = logits_may_overflow();
         } else {
           mt = fmaxf(mprev, s_max[(jt & 1) ^ 1][q][half ^ 1][r]) * c2;
+          if (mloc > -INFINITY && !(mloc * c2 - m_used <= kLazyRange)) *reinterpret_cast<volatile int*>(&s_redo) = 1;
         }
         need_ref = exch;
         mprev = mloc;
@@ -657,7 +649,6 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       s_sum[q][half][r] = lsum;
       asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
       lsum += s_sum[q][half ^ 1][r];
-      if (r == 0) s_qn[q][half] = 0u;  // every thread read it after the item's first tile; the next item starts at zero
       if (ok) ok = mbar_wait(bar(B_ODONE), wi & 1, abortp, c.wait_limit);
       if (!ok) s_quit[q] = 1;
       asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");  // also: s_sum is reused by the next item
@@ -667,48 +658,92 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h] = make_float2(m_used, lsum);
         c.rowq[((size_t)layer * c.chunk + tk) * c.Hq + h] = -m_used - __log2f(lsum) + (21.0f + kMapMargin);
       }
-      const float inv = 1.f / lsum;
       const bool have_o = (j > 0) || (phase == 1);
-      uint32_t ov[2][32];
-      if (have_o) {
-        tmem_ld32(tO, ov[0]);
-        tmem_ld32(tO + 32, ov[1]);
-        tmem_ld_wait();
-      } else {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) ov[0][e] = ov[1][e] = 0u;
-      }
-      // O is in registers: the next item's first P.V product may overwrite the accumulator
-      fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_OFREE + q));
-      if (row_ok) {
+      if (phase == 2) {
+        // merge of two partial softmaxes: the local part (reference m0, row sum l0, accumulator O0 in global memory)
+        // and the retrieved part just computed (m_used, lsum, accumulator in TMEM)
+        const float M = fmaxf(stat0.x, m_used);
+        const float a0 = ex2(stat0.x - M), a1 = m_used == -INFINITY ? 0.f : ex2(m_used - M);
+        const float inv = 1.f / fmaf(stat0.y, a0, lsum * a1);
+        const float w0 = a0 * inv, w1 = a1 * inv;
+        const float* op0 = c.Oacc + oacc_base(w, q) + (size_t)(half * 16) * 512 + r * 4;
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
-          if (phase == 0 && !final_out) {
-            // scratch layout [4-float column group][row][4]: the 32 rows of a warp write 512 contiguous bytes
-            float* op = c.Oacc + oacc_base(w, q) + (size_t)(half * 16 + ch * 8) * 512 + r * 4;
+          float4 o0[8];
 #pragma unroll
-            for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<uint4*>(op + (size_t)(e >> 2) * 512) =
-                  make_uint4(ov[ch][e], ov[ch][e + 1], ov[ch][e + 2], ov[ch][e + 3]);
+          for (int i = 0; i < 8; ++i)
+            o0[i] = row_ok ? *reinterpret_cast<const float4*>(op0 + (size_t)(ch * 8 + i) * 512) : make_float4(0, 0, 0, 0);
+          uint32_t ov[32];
+          if (have_o) {
+            tmem_ld32(tO + ch * 32, ov);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) ov[e] = 0u;
           }
-          if (final_out) {
+          if (ch == 1) {  // O is in registers: the next item's first P.V product may overwrite the accumulator
+            fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_OFREE + q));
+          }
+          if (row_ok) {
             __nv_bfloat16* op = a.out + (((size_t)w.l * a.n + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
 #pragma unroll
             for (int e = 0; e < 32; e += 8) {
+              const float4 x0 = o0[e >> 2], x1 = o0[(e >> 2) + 1];
               uint4 wv;
-              wv.x = pack2(__uint_as_float(ov[ch][e]) * inv, __uint_as_float(ov[ch][e + 1]) * inv);
-              wv.y = pack2(__uint_as_float(ov[ch][e + 2]) * inv, __uint_as_float(ov[ch][e + 3]) * inv);
-              wv.z = pack2(__uint_as_float(ov[ch][e + 4]) * inv, __uint_as_float(ov[ch][e + 5]) * inv);
-              wv.w = pack2(__uint_as_float(ov[ch][e + 6]) * inv, __uint_as_float(ov[ch][e + 7]) * inv);
+              wv.x = pack2(fmaf(x0.x, w0, __uint_as_float(ov[e]) * w1), fmaf(x0.y, w0, __uint_as_float(ov[e + 1]) * w1));
+              wv.y = pack2(fmaf(x0.z, w0, __uint_as_float(ov[e + 2]) * w1), fmaf(x0.w, w0, __uint_as_float(ov[e + 3]) * w1));
+              wv.z = pack2(fmaf(x1.x, w0, __uint_as_float(ov[e + 4]) * w1), fmaf(x1.y, w0, __uint_as_float(ov[e + 5]) * w1));
+              wv.w = pack2(fmaf(x1.z, w0, __uint_as_float(ov[e + 6]) * w1), fmaf(x1.w, w0, __uint_as_float(ov[e + 7]) * w1));
               *reinterpret_cast<uint4*>(op + e) = wv;
+            }
+          }
+        }
+      } else {
+        const float inv = 1.f / lsum;
+        uint32_t ov[2][32];
+        if (have_o) {
+          tmem_ld32(tO, ov[0]);
+          tmem_ld32(tO + 32, ov[1]);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) ov[0][e] = ov[1][e] = 0u;
+        }
+        // O is in registers: the next item's first P.V product may overwrite the accumulator
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_OFREE + q));
+        if (row_ok) {
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) {
+            if (phase == 0 && !final_out) {
+              // scratch layout [4-float column group][row][4]: the 32 rows of a warp write 512 contiguous bytes
+              float* op = c.Oacc + oacc_base(w, q) + (size_t)(half * 16 + ch * 8) * 512 + r * 4;
+#pragma unroll
+              for (int e = 0; e < 32; e += 4)
+                *reinterpret_cast<uint4*>(op + (size_t)(e >> 2) * 512) =
+                    make_uint4(ov[ch][e], ov[ch][e + 1], ov[ch][e + 2], ov[ch][e + 3]);
+            }
+            if (final_out) {
+              __nv_bfloat16* op = a.out + (((size_t)w.l * a.n + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
+#pragma unroll
+              for (int e = 0; e < 32; e += 8) {
+                uint4 wv;
+                wv.x = pack2(__uint_as_float(ov[ch][e]) * inv, __uint_as_float(ov[ch][e + 1]) * inv);
+                wv.y = pack2(__uint_as_float(ov[ch][e + 2]) * inv, __uint_as_float(ov[ch][e + 3]) * inv);
+                wv.z = pack2(__uint_as_float(ov[ch][e + 4]) * inv, __uint_as_float(ov[ch][e + 5]) * inv);
+                wv.w = pack2(__uint_as_float(ov[ch][e + 6]) * inv, __uint_as_float(ov[ch][e + 7]) * inv);
+                *reinterpret_cast<uint4*>(op + e) = wv;
+              }
             }
           }
         }
       }
     }
   }
+  }  // pass
   // ------------------------------------------------------------------ teardown
   fence_before_sync();
   __syncthreads();
@@ -785,9 +820,10 @@ bool tc_attention_supported(const DevCtx& c) {
   return get_encode() != nullptr;
 }
 
-template <int G>
-static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out, const void* kv_maps,
+template <int G, int PHASE>
+static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, bool final_out, const void* kv_maps,
                                cudaStream_t s) {
+  constexpr int phase = PHASE;
   TcMaps maps;
   EncodeFn enc = get_encode();
   if (!enc || !kv_maps) return cudaErrorNotSupported;
@@ -804,7 +840,7 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase,
   }
   constexpr int TOKB = 256 / G;
   const int smem = 65536 + 131072 + 1024;
-  cudaFuncSetAttribute(k_attn_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(k_attn_tc<G, PHASE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   const long long v_off = phase == 0 ? (long long)c.NS * c.NL * c.Hkv * c.SR : (long long)c.NL * c.Hkv * c.Rcap;
   static int sms = 0;
   if (sms == 0) {
@@ -817,17 +853,24 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase,
   if (const char* cap = getenv("LTRI_TC_MAX_CTAS")) ctas = max(1, min(sms, atoi(cap)));
   // persistent CTAs: one per SM (the kernel needs the whole TMEM and most of the shared memory of an SM)
   const int nitems = ((a.n + TOKB - 1) / TOKB) * c.Hkv * a.layer_count;
-  k_attn_tc<G><<<min(nitems, ctas), kTcThreads, smem, s>>>(c, a, phase, final_out ? 1 : 0, maps, v_off);
+  k_attn_tc<G, PHASE><<<min(nitems, ctas), kTcThreads, smem, s>>>(c, a, final_out ? 1 : 0, maps, v_off);
   return cudaGetLastError();
+}
+
+template <int G>
+static cudaError_t launch_tc_phase(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out, const void* kv_maps,
+                                   cudaStream_t s) {
+  if (phase == 0) return launch_tc_g<G, 0>(c, a, final_out, kv_maps, s);
+  return phase == 1 ? launch_tc_g<G, 1>(c, a, final_out, kv_maps, s) : launch_tc_g<G, 2>(c, a, final_out, kv_maps, s);
 }
 
 cudaError_t launch_attn_prefill_tc(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out,
                                    const void* kv_maps, cudaStream_t s) {
   switch (c.G) {
-    case 1: return launch_tc_g<1>(c, a, phase, final_out, kv_maps, s);
-    case 2: return launch_tc_g<2>(c, a, phase, final_out, kv_maps, s);
-    case 4: return launch_tc_g<4>(c, a, phase, final_out, kv_maps, s);
-    case 8: return launch_tc_g<8>(c, a, phase, final_out, kv_maps, s);
+    case 1: return launch_tc_phase<1>(c, a, phase, final_out, kv_maps, s);
+    case 2: return launch_tc_phase<2>(c, a, phase, final_out, kv_maps, s);
+    case 4: return launch_tc_phase<4>(c, a, phase, final_out, kv_maps, s);
+    case 8: return launch_tc_phase<8>(c, a, phase, final_out, kv_maps, s);
   }
   return cudaErrorInvalidValue;
 }

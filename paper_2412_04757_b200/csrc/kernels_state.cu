@@ -17,10 +17,7 @@ __global__ void k_init(DevCtx c, int seq) {
     for (size_t i = tid; i < (size_t)c.NL; i += stride) {
       c.n_spans[u0 + i] = 0;
     }
-    for (size_t i = tid; i < (size_t)c.NL * c.Hkv; i += stride) {
-      c.sel_tokens[u0 * c.Hkv + i] = 0;
-      c.kmax2[u0 * c.Hkv + i] = 0u;
-    }
+    for (size_t i = tid; i < (size_t)c.NL * c.Hkv; i += stride) c.sel_tokens[u0 * c.Hkv + i] = 0;
     for (size_t i = tid; i < (size_t)c.NL * c.slots; i += stride) c.pend_cnt[u0 * c.slots + i] = 0;
     for (size_t i = tid; i < (size_t)c.NL * c.Hkv * c.topk; i += stride) {
       c.sel[u0 * c.Hkv * c.topk + i] = -1;
@@ -47,28 +44,6 @@ cudaError_t launch_init(const DevCtx& c, int seq, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-
-// Squared norm of a key row held as sixteen 16-byte pieces by the sixteen lanes of a half-warp, folded into the running
-// maximum of the (sequence, layer, KV head): DevCtx::kmax2 bounds every logit the attention kernels can meet.  All
-// sixteen lanes of the half-warp call it together; `piece` is this lane's eight bf16 values.
-__device__ __forceinline__ void note_key_norm(const DevCtx& c, size_t unit, int g, const uint4& piece) {
-  const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&piece);
-  float ss = 0.f;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 f = __bfloat1622float2(p2[i]);
-    ss = fmaf(f.x, f.x, ss);
-    ss = fmaf(f.y, f.y, ss);
-  }
-  const unsigned half_mask = 0xffffu << (threadIdx.x & 16);
-#pragma unroll
-  for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(half_mask, ss, o);
-  if ((threadIdx.x & 15) == 0) {
-    const unsigned bits = __float_as_uint(ss);  // ss >= 0: the bit patterns order like the values
-    unsigned* slot = c.kmax2 + unit * c.Hkv + g;
-    if (bits > *reinterpret_cast<volatile unsigned*>(slot)) atomicMax(slot, bits);
-  }
-}
 
 // ------------------------------------------------------------------------------------------
 // a0: copy the call's K/V rows into the cache slabs; 16 threads move one 256-byte row.
@@ -99,7 +74,6 @@ __global__ void k_append_prefill(DevCtx c, PrefillArgs a) {
     *reinterpret_cast<uint4*>(c.Vc + sd) = vv;
   }
   if (g == 0 && c16 == 0) c.votes[unit * c.Tpad + a.t0 + r] = 0;
-  note_key_norm(c, unit, g, kv);
 }
 
 cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
@@ -137,7 +111,6 @@ __global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer
   if (g == 0 && c16 == 0) {
     c.votes[unit * c.Tpad + b.pos[bi]] = 0;
   }
-  note_key_norm(c, unit, g, kv);
 }
 
 cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int,
@@ -1407,10 +1380,8 @@ __device__ __forceinline__ void append_decode_row(const DevCtx& c, const DecBatc
     const int c16 = tid & 15;
     const __nv_bfloat16* src = (tid < 16 ? k : v) + (((size_t)b.src[bi] * layer_count + l) * c.Hkv + g) * kD + c16 * 8;
     __nv_bfloat16* dst = (tid < 16 ? c.Kc : c.Vc) + ((unit * c.Hkv + g) * (size_t)c.SR + b.pos[bi]) * kD + c16 * 8;
-    const uint4 piece = *reinterpret_cast<const uint4*>(src);
-    *reinterpret_cast<uint4*>(dst) = piece;
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
     if (g == 0 && tid == 0) c.votes[unit * c.Tpad + b.pos[bi]] = 0;
-    if (tid < 16) note_key_norm(c, unit, g, piece);
   }
 }
 

@@ -211,7 +211,6 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.rng_cnt = cv.take<int>(units * d.Hkv);
   d.dec_part = cv.take<float>(units * d.Hq * kMaxDecSplit * (kD + 2));
   d.status = cv.take<int>(4);
-  d.kmax2 = cv.take<unsigned>(units * d.Hkv);
   d.wait_limit = kDefaultWaitLimit;
   d.slots += 1;  // the extra slot is scratch for ltri_debug_segment_map
   if (p.flags & LTRI_FLAG_HOST_STAGING) {
@@ -249,6 +248,7 @@ struct ltri_ctx {
   char* host_kv = nullptr;   // the caller's mirror (host address)
   bool spilled = false;      // ev_spill has been recorded at least once
   cudaEvent_t ev_up[2][kHostGroups] = {}, ev_run[2][kHostGroups] = {}, ev_down[2][kHostGroups] = {};
+  int ret_phase = 2;       // retrieved attention: 2 merges with the stored local state, 1 continues from it (testing aid)
   bool grp_used[2][kHostGroups] = {};  // the events of (set, group) have been recorded at least once
   long long host_calls = 0;
   alignas(64) unsigned char kv_maps[kTcMapBytes];  // TMA descriptors of the K/V cache
@@ -392,6 +392,8 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
       return LTRI_ECUDA;
     }
   }
+  if (const char* f = std::getenv("LTRI_ATTN_CONT"))  // testing aid
+    if (std::atoi(f) != 0) ctx->ret_phase = 1;
   ctx->st.resize((size_t)p->max_seqs * p->n_layers);
   for (auto& s : ctx->st) s.E = p->n_sink;
   int dev = 0;
@@ -698,7 +700,8 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
       LTRI_CUDA(ctx, launch_topk_prefill(d, a, st));
     }
     Scope sc(ctx, st, LTRI_K_ATTN_RET, 1);
-    LTRI_CUDA(ctx, ctx->use_tc ? launch_attn_prefill_tc(d, a, 1, true, ctx->kv_maps, st) : launch_attn_prefill(d, a, 1, true, st));
+    LTRI_CUDA(ctx, ctx->use_tc ? launch_attn_prefill_tc(d, a, ctx->ret_phase, true, ctx->kv_maps, st)
+                               : launch_attn_prefill(d, a, 1, true, st));
   }
   // commit the host state
   for (int l = 0; l < layer_count; ++l) {

@@ -1,4 +1,4 @@
-"""GPU paths that ordinary streams never reach: keys of very large norm (the attention kernel's exchange mode),
+"""GPU paths that ordinary streams never reach: keys of very large norm (the attention kernel's second pass),
 an expiring device-side wait, a span index loaded from outside, and host-side limits that must leave the context
 unchanged.  Everything here is finite input and bounded waiting: nothing is expected to fault, trap or hang."""
 import dataclasses
@@ -23,11 +23,12 @@ def _decode_inputs(st, pos):
 def test_keys_of_very_large_norm_give_the_exact_softmax(gain, max_ctas, monkeypatch):
     # Sec. 3.4 step 3: exact softmax over sink | retrieved | local | current for ANY finite input.  Two keys of
     # KV head 0 are scaled up so that the logits of the queries that point at their segment exceed every earlier
-    # tile's maximum by hundreds of log2 units (gain 30 and 12) or by an amount the late-moving reference still
-    # absorbs (gain 1.4: the bound of the logits stays just inside the kernel's exponent range).  The keys sit in a
-    # later tile of the local window while they are local and in the packed slab of the retrieved spans afterwards
-    # (their own votes make them their spans' representatives, so the spans are retrieved).  KV head 1 keeps
-    # ordinary keys, so one launch mixes both modes of the kernel.
+    # tile's maximum by hundreds of log2 units (gain 30 and 12: the kernel's first pass, whose softmax reference
+    # moves one tile late, notices and a second pass with the true maximum on every tile redoes the CTA's items) or
+    # by an amount the late reference still absorbs (gain 1.4).  The keys sit in a later tile of the local window
+    # while they are local and in the packed slab of the retrieved spans afterwards (their own votes make them their
+    # spans' representatives, so the spans are retrieved).  KV head 1 keeps ordinary keys, so one launch has CTAs
+    # that take the second pass and CTAs that do not; with three CTAs every CTA walks many items in both passes.
     # The map comparison is left to the ordinary tests: with logits of this size the fp32 rounding of a logit (on
     # both sides) is worth dozens of Q20 units at a probability near one, beyond the tolerance that is meant for
     # bf16-sized inputs; spans (with the oracle's tie rule), index, selections and outputs are compared as always.
@@ -215,3 +216,22 @@ def test_many_short_calls_run_out_of_pending_slots_without_changing_the_context(
     torch.cuda.synchronize()
     assert lt.ltri_sync_status() == 0
     lt.close()
+
+
+def test_retrieved_attention_merge_equals_the_continuation(monkeypatch):
+    # the retrieved part of a prefill call is accumulated from scratch and merged with the stored local state at the
+    # end of every work item; the variant that loads the state first and continues from it must agree to rounding
+    # (both are within the oracle's tolerance in the other tests; here they are compared with each other)
+    cfg = small_cfg(n_layers=2, context=1280, decode_steps=0, top_k=8)
+    st = inputs.SyntheticStream(cfg)
+    a = binding.Ltri(ph.params_of(cfg))
+    monkeypatch.setenv("LTRI_ATTN_CONT", "1")
+    b = binding.Ltri(ph.params_of(cfg))
+    worst = 0.0
+    for t0, n in st.prefill_chunks():
+        q, k, v = (x.cuda() for x in st.tokens(t0, n))
+        oa, ob = a.ltri_prefill_chunk(0, 0, 2, q, k, v), b.ltri_prefill_chunk(0, 0, 2, q, k, v)
+        worst = max(worst, float((oa.float() - ob.float()).abs().max()))
+    assert worst <= 2e-2
+    a.close()
+    b.close()
