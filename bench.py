@@ -401,6 +401,7 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
     torch.cuda.synchronize(dev)
     lt.ltri_profile_read()                      # clears counters
     lt.ltri_profile_enable(True)
+    miss_before_timed = sum(lt.ltri_debug_read(binding.BUF_CACHE_STATS, SQ, l) for l in range(L))[1] if cfg.host_kv else 0
     sampler = ClockSampler(local)
     sampler.start()
     launches0 = lt.ltri_launch_count()
@@ -437,6 +438,27 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
         p_res = binding.LtriParams.from_buffer_copy(p)
         p_res.flags &= ~binding.FLAG_HOST_KV
         pager["resident_arena_bytes"] = int(binding.ltri_arena_bytes(p_res))
+        # the pulls of the timed calls against the bus: bytes the top-k kernels asked for (misses of the timed calls,
+        # taken from the counters) over the time the pull kernels were running, next to a plain pinned-memory copy
+        miss_timed = float(hm[1]) - float(miss_before_timed)
+        pull_ms = prof["pager_pull"][0]
+        src = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
+        dst = torch.empty_like(src, device=dev)
+        best = None
+        for _ in range(4):
+            b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            b0.record()
+            dst.copy_(src, non_blocking=True)
+            b1.record()
+            torch.cuda.synchronize(dev)
+            best = min(best, b0.elapsed_time(b1)) if best else b0.elapsed_time(b1)
+        bus = src.numel() / (best * 1e-3) / 1e9
+        del src, dst
+        gbs = miss_timed * unit_bytes / (pull_ms * 1e-3) / 1e9 if pull_ms > 0 else None
+        pager["roofline"] = {"bound": "bus", "achieved": gbs, "peak": bus, "unit": "GB/s",
+                             "frac": gbs / bus if gbs else None,
+                             "note": "host-to-device bytes of the timed calls' missing units over the run time of "
+                                     "the pull kernels; peak = a 256 MiB copy from pinned memory on this box"}
     recall = {"final_chunk": needle_recall(lt, st, SQ, cfg)} if cfg.needle and rank == 0 else None
     ms = max_over_ranks(ms, world, dev)
     tokens = K * n

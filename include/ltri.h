@@ -264,6 +264,8 @@ enum {
   LTRI_K_ATTN_RET,     /* prefill attention over the retrieved spans + merge */
   LTRI_K_DEC_RETRIEVE, /* decode scores + top-k */
   LTRI_K_DEC_ATTN,     /* decode split-KV attention + merge */
+  LTRI_K_PAGER_PULL,   /* host-memory pager: pulls of missing units + gather (on the pager's own stream: overlaps
+                          the other classes) */
   LTRI_K_COUNT
 };
 /* Kernels launched by this context since it was created (host counter). */

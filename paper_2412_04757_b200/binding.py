@@ -33,7 +33,7 @@ EXPORTS = [
     "ltri_debug_load_index", "ltri_debug_wait_timeout",
 ]
 KERNEL_CLASSES = ["append", "evict_index", "attn_local", "map_pass", "segment", "score_topk", "attn_retrieved",
-                  "decode_retrieve", "decode_attn"]
+                  "decode_retrieve", "decode_attn", "pager_pull"]
 
 
 class LtriParams(C.Structure):

@@ -18,6 +18,7 @@ constexpr int kMaxRanges = 2 * kMaxTopK + 2;  // sink + local + the spans of thi
 constexpr float kMapMargin = 0.0078125f;          // safety margin (in log2 units) of the map pass's skip test
 constexpr float kMapScale = 0.4972997117f;         // 2^-(1 + kMapMargin)
 constexpr int kTokPad = 128;          // rows of slack after every K/V slab so tile over-reads stay inside it
+constexpr int kTcMaxCtas = 1024;      // most persistent CTAs the tensor-core attention kernel is launched with
 constexpr long long kDefaultWaitLimit = 2000000000ll;  // device-side waits give up after about a second
 
 // Device-side view of one context.  Passed to kernels by value.
@@ -71,6 +72,14 @@ struct DevCtx {
   int* ctag;                    // [NS][NL][Hkv][cache_units]  unit held by the slot, -1 empty
   float* cscore;                // [NS][NL][Hkv][cache_units]  usage score
   unsigned long long* cstat;    // [NS][NL][2]  hits, misses
+  // what a prefill call's top-k kernel asks k_pull_pack to move, per (seq, layer, KV head): the units named (ascending),
+  // each with the cache slot that holds it (-1: read from the mirror; bit 16: the slot has to be filled first) and
+  // its valid token range
+  int* pl_id;                   // [NS*NL][Hkv][2 * kMaxTopK]
+  int* pl_src;
+  int* pl_start;
+  int* pl_len;
+  int* pl_cnt;                  // [NS*NL][Hkv]
   int* rng_koff;                // [NS*NL][Hkv][rcap]  decode: K row of a range's first token, counted from Kc (a slab
                                 //                     row or a unit-cache row; the V row follows from it)
   // per-layer tables of the paper's configuration appendix (nullptr: the scalar holds for every layer)
@@ -101,6 +110,7 @@ struct DevCtx {
   int* rng_cnt;          // [NS*NL][Hkv]
   float* dec_part;       // [NS*NL][Hq][kMaxDecSplit][128+2]
   int* status;           // [4]: first error code, detail...
+  int* tc_redo;          // [kTcMaxCtas]  per CTA of the tensor-core attention kernel: its work has to be redone
   long long wait_limit;  // upper bound of any single device-side wait, in SM clock cycles
 };
 
@@ -163,6 +173,8 @@ cudaError_t launch_score_prefill(const DevCtx& c, const PrefillArgs& a, int span
 // tensor-core version of launch_score_prefill (split-bf16 representatives)
 cudaError_t launch_score_prefill_mma(const DevCtx& c, const PrefillArgs& a, int span_bound, cudaStream_t s);
 cudaError_t launch_topk_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
+// host-memory pager: pulls of the missing units + gather of the selected units' rows (after launch_topk_prefill)
+cudaError_t launch_pull_pack(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
                                 const __nv_bfloat16* q, int span_bound, cudaStream_t s);
 // decode scores + top-k + range list in one launch (span_bound <= dec_retrieve_fused_max_spans())
@@ -175,6 +187,8 @@ cudaError_t launch_topk_decode(const DevCtx& c, const DecBatch& b, int layer_beg
 // prefill attention.  phase 0: local part over sink|local|cur, stores state (+ final output if `final`);
 // phase 1: continues from the stored state over the selected spans and writes the output; phase 2 (tensor-core
 // kernel only): the same result, with the selected spans accumulated from scratch and merged with the stored state.
+// The tensor-core version is two launches: the second redoes, with exact per-tile maxima, the work of CTAs that met
+// logits too far above their running reference (it returns at once otherwise).
 cudaError_t launch_attn_prefill(const DevCtx& c, const PrefillArgs& a, int phase, bool final, cudaStream_t s);
 // tcgen05/TMEM/TMA version of launch_attn_prefill (same contract) and its availability check
 // host storage for a context's tensor maps: five box heights of the K/V cache, the index, five of the packed slabs

@@ -29,7 +29,7 @@ constexpr float kLog2eT = 1.4426950408889634f;
 constexpr int kTcThreads = 576;  // 16 softmax warps + TMA producer + MMA issuer
 constexpr int kNumBoxes = 5;  // box heights 8,16,32,64,128
 constexpr float kRescaleThreshold = 8.0f;
-// Largest exponent (log2 units) a probability may carry above the softmax reference in the first pass: 2^90 times
+// Largest exponent (log2 units) a probability may carry above the softmax reference in the regular launch: 2^90 times
 // the 2^7 keys of a tile, the 2^13 tiles of the longest item and values of up to 2^10 still fits fp32 (and the bf16
 // P operand).
 constexpr float kLazyRange = 90.0f;
@@ -144,16 +144,19 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// PHASE 0: the local part over sink | local | current keys; stores the row statistics and, unless `final_out`, the
-//          unnormalised accumulator.
-// PHASE 2: the retrieved part over the packed slab of the selected spans, accumulated from scratch; the epilogue
-//          merges it with the state phase 0 stored (log-sum-exp merge of two partial softmaxes) and writes the output.
-// PHASE 1: the retrieved part as a continuation: the stored state is loaded back into registers / TMEM first.  Kept
-//          as a cross-check of phase 2.
-template <int G, int PHASE>
+// MERGE: the launch may be asked for phase 2 (kept out of the instantiation that runs phases 0 and 1, whose inner
+// loop is sensitive to every register).
+template <int G, bool EXCH, bool MERGE>
 __global__ void __launch_bounds__(kTcThreads, 1)
-    k_attn_tc(DevCtx c, PrefillArgs a, int final_out, const __grid_constant__ TcMaps maps, long long v_row_offset) {
-  constexpr int phase = PHASE;
+    k_attn_tc(DevCtx c, PrefillArgs a, int phase, int final_out, int* __restrict__ redo,
+              const __grid_constant__ TcMaps maps, long long v_row_offset) {
+  constexpr int exch = EXCH ? 1 : 0;
+  // exch = 0: the regular launch.  Its softmax reference moves one tile late (see the softmax role); a CTA in which
+  // some tile outran that reference by more than the exponent range allows leaves redo[blockIdx.x] = 1.
+  // exch = 1: the launch that follows it with the same grid.  A CTA whose flag is clear returns at once; one whose
+  // flag is set walks its work items again with the true maximum exchanged on every tile and overwrites what the
+  // first launch stored, so inputs of any magnitude get the exact softmax.
+  if (exch && redo[blockIdx.x] == 0) return;
   const CUtensorMap* kvmaps = maps.kv;
   extern __shared__ unsigned char smem_raw[];
   // QFULL QFREE ODONE | KFULL[2] VFULL[2] KEMPTY[2] VEMPTY[2] | SREADY[2] PREADY[2][2] OFREE[2]
@@ -164,7 +167,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __shared__ int s_item_tiles[3];     // tile count of the work items in flight (roles may be up to two items apart)
   __shared__ TileDesc s_td[8];        // per-tile masks, written by the producer, read by the softmax threads
   __shared__ int s_quit[2];
-  __shared__ int s_redo;              // some tile of the first pass outran the late reference: second pass needed
+  __shared__ int s_redo;              // some tile of this CTA outran the late softmax reference
   __shared__ int s_items_ready;       // number of work items whose key ranges the producer has published
   __shared__ float s_max[2][2][2][128];  // per tile parity, Q tile, column half, row: partial maxima
   __shared__ float s_sum[2][2][128];     // per Q tile, column half, row: partial row sums (end of an item)
@@ -240,32 +243,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     return ((((size_t)w.layer * MB + w.mb) * c.Hkv + w.g) * 2 + q) * (size_t)(128 * kD);
   };
 
-  // Every role counts the tiles (jt) and the work items (wi) it has handled; the counters run on through the second
-  // pass, since the barrier phases do.
-  int jt = 0, wi = 0, ok = 1;
-  // Two passes over the CTA's work items.  The first uses the late-moving softmax reference (see the softmax role);
-  // a thread that meets a tile whose logits outrun that reference by more than the exponent range allows raises
-  // s_redo.  Then -- and only then -- the second pass walks the same items again with the true maximum exchanged on
-  // every tile and overwrites what the first pass stored, so inputs of any magnitude get the exact softmax; for
-  // ordinary inputs the second pass is one CTA barrier.
-#ifndef LTRI_PASSES
-#define LTRI_PASSES 2
-#endif
-#pragma unroll 1
-  for (int pass = 0; pass < LTRI_PASSES; ++pass) {
-  if (pass == 1) {
-    fence_before_sync();
-    __syncthreads();  // every thread is through its role of the first pass (also after an expired wait)
-    fence_after_sync();
-    if (!s_redo || s_abort) break;
-  }
-  const bool exch = pass == 1;
   if (warp == 16) {
     // ------------------------------------------------------------------ TMA producer
     // Every lane walks the tile list; lane 0 owns the barrier bookkeeping and lanes 0-3 issue the copies of
     // (K low half, K high half, V low half, V high half) so that many small pieces do not serialise on one thread.
-    if (lane == 0 && pass == 0) prefetch_tmap(&maps.q);
-    for (int item = blockIdx.x; ok && item < nitems; item += gridDim.x, ++wi) {
+    int jt = 0, ok = 1;
+    if (lane == 0) prefetch_tmap(&maps.q);
+    for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
       const Item w = decode(item);
       if (lane == 0) {
         // the Q buffer is free once every QK^T product of the previous item has completed
@@ -395,7 +379,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           mma_ts(d, pa + ks * 8 + (ks >> 2) * 32, db + ((ks * 2048) >> 4), idesc_pv, acc || part > 0 || i > 0);
         }
       };
-      for (int item = blockIdx.x; ok && item < nitems; item += gridDim.x, ++wi) {
+      int jt = 0;
+      bool ok = true;
+      for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
         ok = mbar_wait(bar(B_QFULL), wi & 1, abortp, c.wait_limit);
         if (!ok) break;
         const int T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
@@ -467,7 +453,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     const uint32_t tP = tS;  // its 64 probabilities (bf16 pairs) overwrite the first 32 of its own logit columns
     const uint32_t tO = tmem + lane_base + 256 + q * 128 + half * 64;
     const float c2 = c.scale * kLog2eT;
-    for (int item = blockIdx.x; item < nitems; item += gridDim.x, ++wi) {
+    int jt = 0;
+    bool ok = true;
+    for (int item = blockIdx.x, wi = 0; item < nitems; item += gridDim.x, ++wi) {
       const Item w = decode(item);
       const int tk = w.tok0 + rr / G;              // call-relative token
       const int h = w.g * G + rr % G;
@@ -497,7 +485,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       const int T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
       float m_used = -INFINITY, lsum = 0.f;
       float2 stat0 = make_float2(0.f, 1.f);  // phase 2: reference maximum and row sum of the local part
-      if (phase == 2 && row_ok) {
+      if (MERGE && phase == 2 && row_ok) {
         // the state this item is merged with at its end: fetch the statistics now (used after the tile loop) and pull
         // the accumulator rows into L2 (one request per 128-byte line: eight rows of a column group)
         stat0 = c.rowstat[((size_t)layer * c.chunk + tk) * c.Hq + h];
@@ -542,7 +530,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         ok = ok && mbar_wait(bar(B_SREADY + q), jt & 1, abortp, c.wait_limit);
         if (!ok) {
           if (need_ref) asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
-          need_ref = exch;
+          need_ref = EXCH;
           ++j;
           ++jt;
           continue;
@@ -583,9 +571,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         // one tile late: it is the maximum over the previous tiles, whose partner half is already visible (the
         // partner stored it before its PREADY arrival of the previous tile, which precedes this tile's SREADY), so
         // no barrier sits between the logits and the exponentials.  A tile that exceeds the late reference only
-        // makes the exponent positive; if it does so by more than kLazyRange the results of this pass are not to
-        // be trusted (the probabilities may overflow) and the thread asks for the second pass, in which every tile
-        // exchanges its maxima like the first one (exch) and the exponent never exceeds the lazy threshold.
+        // makes the exponent positive; if it does so by more than kLazyRange the probabilities may overflow, so the
+        // thread flags the CTA for the second launch, in which every tile exchanges its maxima like the first one
+        // and the exponent never exceeds the lazy threshold.
         s_max[jt & 1][q][half][r] = mloc;
         float mt;
         if (need_ref) {
@@ -595,7 +583,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           mt = fmaxf(mprev, s_max[(jt & 1) ^ 1][q][half ^ 1][r]) * c2;
           if (mloc > -INFINITY && !(mloc * c2 - m_used <= kLazyRange)) *reinterpret_cast<volatile int*>(&s_redo) = 1;
         }
-        need_ref = exch;
+        need_ref = EXCH;
         mprev = mloc;
         // lazy running maximum: move it only when it grows by more than the threshold (or on first use)
         float alpha = 1.f;
@@ -659,7 +647,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         c.rowq[((size_t)layer * c.chunk + tk) * c.Hq + h] = -m_used - __log2f(lsum) + (21.0f + kMapMargin);
       }
       const bool have_o = (j > 0) || (phase == 1);
-      if (phase == 2) {
+      if (MERGE && phase == 2) {
         // merge of two partial softmaxes: the local part (reference m0, row sum l0, accumulator O0 in global memory)
         // and the retrieved part just computed (m_used, lsum, accumulator in TMEM)
         const float M = fmaxf(stat0.x, m_used);
@@ -700,56 +688,56 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             }
           }
         }
+        continue;
+      }
+      const float inv = 1.f / lsum;
+      uint32_t ov[2][32];
+      if (have_o) {
+        tmem_ld32(tO, ov[0]);
+        tmem_ld32(tO + 32, ov[1]);
+        tmem_ld_wait();
       } else {
-        const float inv = 1.f / lsum;
-        uint32_t ov[2][32];
-        if (have_o) {
-          tmem_ld32(tO, ov[0]);
-          tmem_ld32(tO + 32, ov[1]);
-          tmem_ld_wait();
-        } else {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) ov[0][e] = ov[1][e] = 0u;
-        }
-        // O is in registers: the next item's first P.V product may overwrite the accumulator
-        fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(B_OFREE + q));
-        if (row_ok) {
+        for (int e = 0; e < 32; ++e) ov[0][e] = ov[1][e] = 0u;
+      }
+      // O is in registers: the next item's first P.V product may overwrite the accumulator
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_OFREE + q));
+      if (row_ok) {
 #pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
-            if (phase == 0 && !final_out) {
-              // scratch layout [4-float column group][row][4]: the 32 rows of a warp write 512 contiguous bytes
-              float* op = c.Oacc + oacc_base(w, q) + (size_t)(half * 16 + ch * 8) * 512 + r * 4;
+        for (int ch = 0; ch < 2; ++ch) {
+          if (phase == 0 && !final_out) {
+            // scratch layout [4-float column group][row][4]: the 32 rows of a warp write 512 contiguous bytes
+            float* op = c.Oacc + oacc_base(w, q) + (size_t)(half * 16 + ch * 8) * 512 + r * 4;
 #pragma unroll
-              for (int e = 0; e < 32; e += 4)
-                *reinterpret_cast<uint4*>(op + (size_t)(e >> 2) * 512) =
-                    make_uint4(ov[ch][e], ov[ch][e + 1], ov[ch][e + 2], ov[ch][e + 3]);
-            }
-            if (final_out) {
-              __nv_bfloat16* op = a.out + (((size_t)w.l * a.n + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
+            for (int e = 0; e < 32; e += 4)
+              *reinterpret_cast<uint4*>(op + (size_t)(e >> 2) * 512) =
+                  make_uint4(ov[ch][e], ov[ch][e + 1], ov[ch][e + 2], ov[ch][e + 3]);
+          }
+          if (final_out) {
+            __nv_bfloat16* op = a.out + (((size_t)w.l * a.n + tk) * c.Hq + h) * kD + half * 64 + ch * 32;
 #pragma unroll
-              for (int e = 0; e < 32; e += 8) {
-                uint4 wv;
-                wv.x = pack2(__uint_as_float(ov[ch][e]) * inv, __uint_as_float(ov[ch][e + 1]) * inv);
-                wv.y = pack2(__uint_as_float(ov[ch][e + 2]) * inv, __uint_as_float(ov[ch][e + 3]) * inv);
-                wv.z = pack2(__uint_as_float(ov[ch][e + 4]) * inv, __uint_as_float(ov[ch][e + 5]) * inv);
-                wv.w = pack2(__uint_as_float(ov[ch][e + 6]) * inv, __uint_as_float(ov[ch][e + 7]) * inv);
-                *reinterpret_cast<uint4*>(op + e) = wv;
-              }
+            for (int e = 0; e < 32; e += 8) {
+              uint4 wv;
+              wv.x = pack2(__uint_as_float(ov[ch][e]) * inv, __uint_as_float(ov[ch][e + 1]) * inv);
+              wv.y = pack2(__uint_as_float(ov[ch][e + 2]) * inv, __uint_as_float(ov[ch][e + 3]) * inv);
+              wv.z = pack2(__uint_as_float(ov[ch][e + 4]) * inv, __uint_as_float(ov[ch][e + 5]) * inv);
+              wv.w = pack2(__uint_as_float(ov[ch][e + 6]) * inv, __uint_as_float(ov[ch][e + 7]) * inv);
+              *reinterpret_cast<uint4*>(op + e) = wv;
             }
           }
         }
       }
     }
   }
-  }  // pass
   // ------------------------------------------------------------------ teardown
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
   if (warp == 16) tmem_dealloc(tmem, 512);
   if (tid == 0 && s_abort) set_status(c, -6, (int)blockIdx.x);
+  if (tid == 0) redo[blockIdx.x] = exch ? 0 : s_redo;  // (the second launch leaves the flags clear for the next call)
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -820,10 +808,9 @@ bool tc_attention_supported(const DevCtx& c) {
   return get_encode() != nullptr;
 }
 
-template <int G, int PHASE>
-static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, bool final_out, const void* kv_maps,
+template <int G, bool MERGE>
+static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out, const void* kv_maps,
                                cudaStream_t s) {
-  constexpr int phase = PHASE;
   TcMaps maps;
   EncodeFn enc = get_encode();
   if (!enc || !kv_maps) return cudaErrorNotSupported;
@@ -840,7 +827,8 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, bool final
   }
   constexpr int TOKB = 256 / G;
   const int smem = 65536 + 131072 + 1024;
-  cudaFuncSetAttribute(k_attn_tc<G, PHASE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(k_attn_tc<G, false, MERGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(k_attn_tc<G, true, MERGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   const long long v_off = phase == 0 ? (long long)c.NS * c.NL * c.Hkv * c.SR : (long long)c.NL * c.Hkv * c.Rcap;
   static int sms = 0;
   if (sms == 0) {
@@ -853,24 +841,21 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, bool final
   if (const char* cap = getenv("LTRI_TC_MAX_CTAS")) ctas = max(1, min(sms, atoi(cap)));
   // persistent CTAs: one per SM (the kernel needs the whole TMEM and most of the shared memory of an SM)
   const int nitems = ((a.n + TOKB - 1) / TOKB) * c.Hkv * a.layer_count;
-  k_attn_tc<G, PHASE><<<min(nitems, ctas), kTcThreads, smem, s>>>(c, a, final_out ? 1 : 0, maps, v_off);
+  // the regular launch, then the one that redoes the work of the CTAs that asked for it (they return at once otherwise)
+  const int grid = min(nitems, ctas);
+  if (grid > kTcMaxCtas) return cudaErrorInvalidValue;
+  k_attn_tc<G, false, MERGE><<<grid, kTcThreads, smem, s>>>(c, a, phase, final_out ? 1 : 0, c.tc_redo, maps, v_off);
+  k_attn_tc<G, true, MERGE><<<grid, kTcThreads, smem, s>>>(c, a, phase, final_out ? 1 : 0, c.tc_redo, maps, v_off);
   return cudaGetLastError();
-}
-
-template <int G>
-static cudaError_t launch_tc_phase(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out, const void* kv_maps,
-                                   cudaStream_t s) {
-  if (phase == 0) return launch_tc_g<G, 0>(c, a, final_out, kv_maps, s);
-  return phase == 1 ? launch_tc_g<G, 1>(c, a, final_out, kv_maps, s) : launch_tc_g<G, 2>(c, a, final_out, kv_maps, s);
 }
 
 cudaError_t launch_attn_prefill_tc(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out,
                                    const void* kv_maps, cudaStream_t s) {
   switch (c.G) {
-    case 1: return launch_tc_phase<1>(c, a, phase, final_out, kv_maps, s);
-    case 2: return launch_tc_phase<2>(c, a, phase, final_out, kv_maps, s);
-    case 4: return launch_tc_phase<4>(c, a, phase, final_out, kv_maps, s);
-    case 8: return launch_tc_phase<8>(c, a, phase, final_out, kv_maps, s);
+    case 1: return phase == 2 ? launch_tc_g<1, true>(c, a, phase, final_out, kv_maps, s) : launch_tc_g<1, false>(c, a, phase, final_out, kv_maps, s);
+    case 2: return phase == 2 ? launch_tc_g<2, true>(c, a, phase, final_out, kv_maps, s) : launch_tc_g<2, false>(c, a, phase, final_out, kv_maps, s);
+    case 4: return phase == 2 ? launch_tc_g<4, true>(c, a, phase, final_out, kv_maps, s) : launch_tc_g<4, false>(c, a, phase, final_out, kv_maps, s);
+    case 8: return phase == 2 ? launch_tc_g<8, true>(c, a, phase, final_out, kv_maps, s) : launch_tc_g<8, false>(c, a, phase, final_out, kv_maps, s);
   }
   return cudaErrorInvalidValue;
 }

@@ -36,6 +36,8 @@ __global__ void k_init(DevCtx c, int seq) {
   }
   if (seq < 0 && tid < 4) c.status[tid] = 0;
   if (seq < 0)
+    for (size_t i = tid; i < (size_t)kTcMaxCtas; i += stride) c.tc_redo[i] = 0;
+  if (seq < 0)
     for (size_t i = tid; i < (size_t)c.NL; i += stride) c.Jcnt[i] = 0;
 }
 
@@ -1216,22 +1218,36 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
       c.ctag[cb + tid] = s_tag[tid];
       c.cscore[cb + tid] = s_sco[tid];
     }
-    // pull the missing units: the unit's valid rows [s_sst, s_sst + s_sln) go to the same row offsets of its slot
-    const size_t hslab = (unit * c.Hkv + g) * (size_t)c.Tpad;
-    for (int t = 0; t < nall; ++t) {
-      if (!s_fill[t]) continue;
-      const int st = s_sst[t], ln = s_sln[t];
-      const size_t drow = (cb + s_src[t]) * (size_t)U + (st - ids_all[t] * U);
-      const uint4* hk = reinterpret_cast<const uint4*>(c.hostK + (hslab + st) * kD);
-      const uint4* hv = reinterpret_cast<const uint4*>(c.hostV + (hslab + st) * kD);
-      uint4* dk = reinterpret_cast<uint4*>(c.Kcache + drow * kD);
-      uint4* dv = reinterpret_cast<uint4*>(c.Vcache + drow * kD);
-      for (int i = tid; i < ln * 16; i += nt) {
-        dk[i] = hk[i];
-        dv[i] = hv[i];
+    if (!DECODE) {
+      // A prefill call leaves the data movement to k_pull_pack, which runs on a stream of its own while the kernels
+      // of the call's other layers compute: this kernel only records what has to be brought in and from where.
+      const size_t pb = (unit * c.Hkv + g) * (size_t)(2 * kMaxTopK);
+      if (tid < nall) {
+        c.pl_id[pb + tid] = ids_all[tid];
+        c.pl_src[pb + tid] = s_src[tid] < 0 ? -1 : (s_src[tid] | (s_fill[tid] ? 0x10000 : 0));
+        c.pl_start[pb + tid] = s_sst[tid];
+        c.pl_len[pb + tid] = s_sln[tid];
+      }
+      if (tid == 0) c.pl_cnt[unit * c.Hkv + g] = nall;
+    }
+    if (DECODE) {
+      // a decode step pulls its missing units here: the unit's valid rows [s_sst, s_sst + s_sln) go to the same row
+      // offsets of its slot (the attention kernel, launched next, reads the slots in place)
+      const size_t hslab = (unit * c.Hkv + g) * (size_t)c.Tpad;
+      for (int t = 0; t < nall; ++t) {
+        if (!s_fill[t]) continue;
+        const int st = s_sst[t], ln = s_sln[t];
+        const size_t drow = (cb + s_src[t]) * (size_t)U + (st - ids_all[t] * U);
+        const uint4* hk = reinterpret_cast<const uint4*>(c.hostK + (hslab + st) * kD);
+        const uint4* hv = reinterpret_cast<const uint4*>(c.hostV + (hslab + st) * kD);
+        uint4* dk = reinterpret_cast<uint4*>(c.Kcache + drow * kD);
+        uint4* dv = reinterpret_cast<uint4*>(c.Vcache + drow * kD);
+        for (int i = tid; i < ln * 16; i += nt) {
+          dk[i] = hk[i];
+          dv[i] = hv[i];
+        }
       }
     }
-    __syncthreads();  // later reads of the slots by this CTA (the prefill gather) see the rows
   }
   if (tid == 0) {
     int nr = 0;
@@ -1286,43 +1302,7 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     }
   }
   if (!DECODE && c.host_kv) {
-    const int CU = c.cache_units;
-    const size_t cb = (unit * c.Hkv + g) * (size_t)CU;
-    const size_t hslab = (unit * c.Hkv + g) * (size_t)c.Tpad;
-    // a5 gather, from the unit cache (or the host mirror) instead of the device slabs
-    const int nr = s_nr, R = s_pre[nr], Rz = (R + 7) & ~7;
-    const size_t gslab = ((size_t)layer * c.Hkv + g) * (size_t)c.Rcap;
-    uint4* Kdst = reinterpret_cast<uint4*>(c.Kg + gslab * kD);
-    uint4* Vdst = reinterpret_cast<uint4*>(c.Vg + gslab * kD);
-    const int ch = tid & 15, rpp = nt >> 4;
-    for (int r = tid >> 4; r < Rz; r += rpp) {
-      uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
-      if (r < R) {
-        int lo = 0, hi = nr - 1;  // last range whose first packed row is <= r
-        while (lo < hi) {
-          const int mid = (lo + hi + 1) >> 1;
-          if (s_pre[mid] <= r) lo = mid; else hi = mid - 1;
-        }
-        const int tok = s_rs[lo] + (r - s_pre[lo]);
-        const int uid = tok / U;
-        int a0 = 0, a1 = nall - 1;  // the selected unit (ascending ids) that holds the token
-        while (a0 < a1) {
-          const int mid = (a0 + a1) >> 1;
-          if (ids_all[mid] < uid) a0 = mid + 1; else a1 = mid;
-        }
-        const int sl = s_src[a0];
-        if (sl >= 0) {
-          const size_t row = (cb + sl) * (size_t)U + (tok - uid * U);
-          kv = *(reinterpret_cast<const uint4*>(c.Kcache + row * kD) + ch);
-          vv = *(reinterpret_cast<const uint4*>(c.Vcache + row * kD) + ch);
-        } else {
-          kv = *(reinterpret_cast<const uint4*>(c.hostK + (hslab + tok) * kD) + ch);
-          vv = *(reinterpret_cast<const uint4*>(c.hostV + (hslab + tok) * kD) + ch);
-        }
-      }
-      Kdst[(size_t)r * 16 + ch] = kv;
-      Vdst[(size_t)r * 16 + ch] = vv;
-    }
+    // (a5 gather from the unit cache / the host mirror: k_pull_pack)
   } else if (!DECODE) {
     // a5 gather: pack the K and V rows of the selected spans into one contiguous slab per (layer, KV head), so the
     // attention kernel that continues over them reads whole 128-row tiles.  16 threads per 256-byte row, four rows
@@ -1362,6 +1342,99 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
       }
     }
   }
+}
+
+// Host-memory pager (Sec. 3.4), data movement of a prefill call.  A task = one (named unit, KV head, layer): bring
+// the unit's rows to the slab the retrieved attention reads (a5 gather) -- from its cache slot, or over the bus from
+// the host mirror, in which case the rows also go into the slot the top-k kernel chose for the unit (unless the unit
+// is the one the indexed range ends in and still grows: that one is never cached).  A few small persistent CTAs
+// (128 threads, few registers, no dynamic shared memory) walk the tasks: small and few on purpose, so that each fits
+// onto an SM beside the one large CTA of the attention and map kernels and the bus transfer really runs under the
+// computation of the call's other layers instead of taking SMs away from it.  Eight 16-byte loads per thread are in
+// flight on the bus at a time, which keeps the bus busy with far fewer threads than the GPU has.
+constexpr int kPullThreads = 128;
+constexpr int kPullCtas = 32;
+
+__global__ void __launch_bounds__(kPullThreads) k_pull_pack(DevCtx c, int seq, int layer_begin, int layer_count, int max_units) {
+  __shared__ int s_off;
+  const int tid = threadIdx.x;
+  const int ntasks = max_units * c.Hkv * layer_count;
+  for (int task = blockIdx.x; task < ntasks; task += gridDim.x) {
+  const int t = task % max_units, g = (task / max_units) % c.Hkv, layer = layer_begin + task / (max_units * c.Hkv);
+  const size_t unit = unit_of(c, seq, layer);
+  const int nall = min(c.pl_cnt[unit * c.Hkv + g], 2 * kMaxTopK);
+  if (t >= nall) continue;
+  __syncthreads();  // (s_off of the previous task has been read by everyone)
+  const size_t pb = (unit * c.Hkv + g) * (size_t)(2 * kMaxTopK);
+  // first packed row of this unit: the units are packed in ascending order, every token once
+  if (tid < 32) {
+    int part = 0;
+    for (int i = tid; i < t; i += 32) part += c.pl_len[pb + i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if (tid == 0) s_off = part;
+  }
+  __syncthreads();
+  const int U = c.unit;
+  const int id = c.pl_id[pb + t], src = c.pl_src[pb + t], st = c.pl_start[pb + t], ln = c.pl_len[pb + t];
+  const size_t gslab = ((size_t)layer * c.Hkv + g) * (size_t)c.Rcap + s_off;
+  uint4* Kdst = reinterpret_cast<uint4*>(c.Kg + gslab * kD);
+  uint4* Vdst = reinterpret_cast<uint4*>(c.Vg + gslab * kD);
+  const uint4 *Ksrc, *Vsrc;
+  uint4 *Kslot = nullptr, *Vslot = nullptr;
+  const size_t hslab = (unit * c.Hkv + g) * (size_t)c.Tpad;
+  if (src >= 0) {
+    const size_t row = ((unit * c.Hkv + g) * (size_t)c.cache_units + (src & 0xffff)) * (size_t)U + (st - id * U);
+    Ksrc = reinterpret_cast<const uint4*>(c.Kcache + row * kD);
+    Vsrc = reinterpret_cast<const uint4*>(c.Vcache + row * kD);
+    if (src & 0x10000) {  // not there yet: over the bus, and into the slot as well
+      Kslot = reinterpret_cast<uint4*>(c.Kcache + row * kD);
+      Vslot = reinterpret_cast<uint4*>(c.Vcache + row * kD);
+      Ksrc = reinterpret_cast<const uint4*>(c.hostK + (hslab + st) * kD);
+      Vsrc = reinterpret_cast<const uint4*>(c.hostV + (hslab + st) * kD);
+    }
+  } else {
+    Ksrc = reinterpret_cast<const uint4*>(c.hostK + (hslab + st) * kD);
+    Vsrc = reinterpret_cast<const uint4*>(c.hostV + (hslab + st) * kD);
+  }
+  const int n16 = ln * 16;
+  for (int i0 = tid; i0 < n16; i0 += 4 * kPullThreads) {
+    uint4 kv[4], vv[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * kPullThreads;
+      if (i < n16) {
+        kv[u] = Ksrc[i];
+        vv[u] = Vsrc[i];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * kPullThreads;
+      if (i < n16) {
+        Kdst[i] = kv[u];
+        Vdst[i] = vv[u];
+        if (Kslot) {
+          Kslot[i] = kv[u];
+          Vslot[i] = vv[u];
+        }
+      }
+    }
+  }
+  if (t == nall - 1) {
+    // the packed rows up to the next multiple of eight are zero (tile pieces are eight rows high)
+    const int R = s_off + ln, pad = ((R + 7) & ~7) - R;
+    for (int i = tid; i < pad * 16; i += kPullThreads) {
+      Kdst[n16 + i] = make_uint4(0u, 0u, 0u, 0u);
+      Vdst[n16 + i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+  }  // task
+}
+
+cudaError_t launch_pull_pack(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
+  k_pull_pack<<<kPullCtas, kPullThreads, 0, s>>>(c, a.seq, a.layer_begin, a.layer_count, c.topk);
+  return cudaGetLastError();
 }
 
 // Decode retrieval in one launch: a CTA owns one (sequence, layer, KV head), streams that head's index once

@@ -164,6 +164,11 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.cscore = cv.take<float>(d.host_kv ? units * d.Hkv * d.cache_units : 0);
   d.cstat = cv.take<unsigned long long>(d.host_kv ? units * 2 : 0);
   d.rng_koff = cv.take<int>(d.host_kv ? units * d.Hkv * d.rcap : 0);
+  d.pl_id = cv.take<int>(d.host_kv ? units * d.Hkv * 2 * kMaxTopK : 0);
+  d.pl_src = cv.take<int>(d.host_kv ? units * d.Hkv * 2 * kMaxTopK : 0);
+  d.pl_start = cv.take<int>(d.host_kv ? units * d.Hkv * 2 * kMaxTopK : 0);
+  d.pl_len = cv.take<int>(d.host_kv ? units * d.Hkv * 2 * kMaxTopK : 0);
+  d.pl_cnt = cv.take<int>(d.host_kv ? units * d.Hkv : 0);
   d.votes = cv.take<long long>(units * d.Tpad);
   d.span_start = cv.take<int>(units * d.cap);
   d.span_len = cv.take<int>(units * d.cap);
@@ -211,6 +216,7 @@ size_t layout(const ltri_params& p, DevCtx& d, char* base, char** stage_out = nu
   d.rng_cnt = cv.take<int>(units * d.Hkv);
   d.dec_part = cv.take<float>(units * d.Hq * kMaxDecSplit * (kD + 2));
   d.status = cv.take<int>(4);
+  d.tc_redo = cv.take<int>(kTcMaxCtas);
   d.wait_limit = kDefaultWaitLimit;
   d.slots += 1;  // the extra slot is scratch for ltri_debug_segment_map
   if (p.flags & LTRI_FLAG_HOST_STAGING) {
@@ -245,6 +251,11 @@ struct ltri_ctx {
   // host-memory pager: evicted rows are mirrored to the host on their own stream
   cudaStream_t s_spill = nullptr;
   cudaEvent_t ev_pre = nullptr, ev_spill = nullptr;
+  // pulls of a prefill call run per layer group on their own stream (see ltri_prefill_chunk)
+  static constexpr int kMaxGroups = 4;
+  cudaStream_t s_pull = nullptr;
+  cudaEvent_t ev_sel[kMaxGroups] = {}, ev_pull[kMaxGroups] = {};
+  int pager_groups = kMaxGroups;  // layer groups of a paged prefill call (testing aid: LTRI_PAGER_GROUPS)
   char* host_kv = nullptr;   // the caller's mirror (host address)
   bool spilled = false;      // ev_spill has been recorded at least once
   cudaEvent_t ev_up[2][kHostGroups] = {}, ev_run[2][kHostGroups] = {}, ev_down[2][kHostGroups] = {};
@@ -362,12 +373,19 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
     ctx->d.hostK = host_dev;
     ctx->d.hostV = host_dev + half;
     ctx->host_kv = static_cast<char*>(p->host_kv);
-    if (cudaStreamCreateWithFlags(&ctx->s_spill, cudaStreamNonBlocking) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ctx->ev_pre, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ctx->ev_spill, cudaEventDisableTiming) != cudaSuccess) {
+    bool ok = cudaStreamCreateWithFlags(&ctx->s_spill, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&ctx->s_pull, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ctx->ev_pre, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ctx->ev_spill, cudaEventDisableTiming) == cudaSuccess;
+    for (int g = 0; g < ltri_ctx::kMaxGroups && ok; ++g)
+      ok = cudaEventCreateWithFlags(&ctx->ev_sel[g], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->ev_pull[g], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
       ltri_destroy(ctx);
       return LTRI_ECUDA;
     }
+    if (const char* f = std::getenv("LTRI_PAGER_GROUPS"))  // testing aid
+      ctx->pager_groups = std::max(1, std::min((int)ltri_ctx::kMaxGroups, std::atoi(f)));
   }
   if (p->retrieval_head) {  // the caller's arrays are read now and not kept
     ctx->ret_head.assign(p->retrieval_head, p->retrieval_head + p->n_layers);
@@ -465,6 +483,14 @@ int ltri_destroy(ltri_ctx* ctx) {
   if (ctx->s_spill) {  // copies into the caller's host mirror may still be in flight
     cudaStreamSynchronize(ctx->s_spill);
     cudaStreamDestroy(ctx->s_spill);
+  }
+  if (ctx->s_pull) {
+    cudaStreamSynchronize(ctx->s_pull);
+    cudaStreamDestroy(ctx->s_pull);
+  }
+  for (int g = 0; g < ltri_ctx::kMaxGroups; ++g) {
+    if (ctx->ev_sel[g]) cudaEventDestroy(ctx->ev_sel[g]);
+    if (ctx->ev_pull[g]) cudaEventDestroy(ctx->ev_pull[g]);
   }
   if (ctx->ev_pre) cudaEventDestroy(ctx->ev_pre);
   if (ctx->ev_spill) cudaEventDestroy(ctx->ev_spill);
@@ -670,39 +696,71 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
     ctx->spilled = true;
   }
   const bool has_index = ub > 0;
-  {
-    Scope sc(ctx, st, LTRI_K_ATTN_LOCAL, 1);
-    LTRI_CUDA(ctx, ctx->use_tc ? launch_attn_prefill_tc(d, a, 0, !has_index, ctx->kv_maps, st)
-                               : launch_attn_prefill(d, a, 0, !has_index, st));
-  }
-  {
-    // (the tensor-core pass is one kernel; the warp-MMA fallback has one for the local keys and one for the call's own)
-    Scope sc(ctx, st, LTRI_K_MAP, ctx->use_tc ? 1 : ((a.t0 - a.loc_begin > 0 && a.loc_begin >= d.Ls) ? 2 : 1));
-    LTRI_CUDA(ctx, ctx->use_tc ? launch_map_pass_tc(d, a, ctx->kv_maps, st) : launch_map_pass(d, a, st));
-  }
-  if (m > 0) {
-    Scope sc(ctx, st, LTRI_K_SEGMENT, 4);
-    long long thq_abs = 0;
-    if (d.theta_mode == 0) thq_abs = (long long)std::nearbyint((double)d.theta * (double)d.Hq * (double)kQScale);
-    LTRI_CUDA(ctx, launch_segment(d, seq, layer_begin, layer_count, m, reg_start, slot, d.theta_mode, d.theta, thq_abs,
-                                  d.C, n_tokens, t0, a.q, st, /*tables=*/true, d.seg_unit));
-  }
-  if (has_index) {
+  // Layer groups.  Resident contexts run every kernel once over all layers of the call.  Under the host-memory pager
+  // the call is issued in up to four groups of layers: a group's top-k only decides what has to come over the bus;
+  // the transfer and the gather (k_pull_pack) follow on the pager's own stream while the next groups compute, and
+  // the retrieved attention of each group is issued at the end, once its rows are in place.
+  const int NG = (d.host_kv && has_index) ? std::min(ctx->pager_groups, layer_count) : 1;
+  long long thq_abs = 0;
+  if (d.theta_mode == 0) thq_abs = (long long)std::nearbyint((double)d.theta * (double)d.Hq * (double)kQScale);
+  PrefillArgs grp[ltri_ctx::kMaxGroups];
+  for (int g = 0; g < NG; ++g) {
+    const int lo = layer_count * g / NG, hi = layer_count * (g + 1) / NG;  // call-relative layers of the group
+    PrefillArgs& ag = grp[g];
+    ag = a;
+    ag.layer_begin = layer_begin + lo;
+    ag.layer_count = hi - lo;
+    ag.q = a.q + (size_t)lo * n_tokens * d.Hq * kD;
+    ag.k = a.k + (size_t)lo * n_tokens * d.Hkv * kD;
+    ag.v = a.v + (size_t)lo * n_tokens * d.Hkv * kD;
+    ag.out = a.out + (size_t)lo * n_tokens * d.Hq * kD;
+    {
+      Scope sc(ctx, st, LTRI_K_ATTN_LOCAL, ctx->use_tc ? 2 : 1);
+      LTRI_CUDA(ctx, ctx->use_tc ? launch_attn_prefill_tc(d, ag, 0, !has_index, ctx->kv_maps, st)
+                                 : launch_attn_prefill(d, ag, 0, !has_index, st));
+    }
+    {
+      // (the tensor-core pass is one kernel; the warp-MMA fallback has one for the local keys and one for the call's own)
+      Scope sc(ctx, st, LTRI_K_MAP, ctx->use_tc ? 1 : ((a.t0 - a.loc_begin > 0 && a.loc_begin >= d.Ls) ? 2 : 1));
+      LTRI_CUDA(ctx, ctx->use_tc ? launch_map_pass_tc(d, ag, ctx->kv_maps, st) : launch_map_pass(d, ag, st));
+    }
+    if (m > 0) {
+      Scope sc(ctx, st, LTRI_K_SEGMENT, 4);
+      LTRI_CUDA(ctx, launch_segment(d, seq, ag.layer_begin, ag.layer_count, m, reg_start, slot, d.theta_mode, d.theta,
+                                    thq_abs, d.C, n_tokens, t0, ag.q, st, /*tables=*/true, d.seg_unit));
+    }
+    if (!has_index) continue;
     {
       Scope sc(ctx, st, LTRI_K_SCORE_TOPK, d.vote ? 3 : 2);
       if (ctx->use_tc && score_tc_supported(d))
-        LTRI_CUDA(ctx, launch_score_prefill_tc(d, a, (int)ub, ctx->kv_maps, st));
+        LTRI_CUDA(ctx, launch_score_prefill_tc(d, ag, (int)ub, ctx->kv_maps, st));
       else if (ctx->use_tc)
-        LTRI_CUDA(ctx, launch_score_prefill_mma(d, a, (int)ub, st));
+        LTRI_CUDA(ctx, launch_score_prefill_mma(d, ag, (int)ub, st));
       else
-        LTRI_CUDA(ctx, launch_score_prefill(d, a, (int)ub, st));
-      if (d.host_kv && !ev.empty()) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_spill, 0));
-      LTRI_CUDA(ctx, launch_topk_prefill(d, a, st));
+        LTRI_CUDA(ctx, launch_score_prefill(d, ag, (int)ub, st));
+      LTRI_CUDA(ctx, launch_topk_prefill(d, ag, st));
     }
-    Scope sc(ctx, st, LTRI_K_ATTN_RET, 1);
-    LTRI_CUDA(ctx, ctx->use_tc ? launch_attn_prefill_tc(d, a, ctx->ret_phase, true, ctx->kv_maps, st)
-                               : launch_attn_prefill(d, a, 1, true, st));
+    if (d.host_kv) {
+      // the group's selection is known: its units travel on the pager's stream (behind this call's spill copies, whose
+      // rows a pull may want back) while the caller's stream goes on with the next group
+      cudaStream_t sp = ctx->s_pull;
+      LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_sel[g], st));
+      LTRI_CUDA(ctx, cudaStreamWaitEvent(sp, ctx->ev_sel[g], 0));
+      if (!ev.empty()) LTRI_CUDA(ctx, cudaStreamWaitEvent(sp, ctx->ev_spill, 0));
+      {
+        Scope sc(ctx, sp, LTRI_K_PAGER_PULL, 1);
+        LTRI_CUDA(ctx, launch_pull_pack(d, ag, sp));
+      }
+      LTRI_CUDA(ctx, cudaEventRecord(ctx->ev_pull[g], sp));
+    }
   }
+  if (has_index)
+    for (int g = 0; g < NG; ++g) {
+      if (d.host_kv) LTRI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_pull[g], 0));
+      Scope sc(ctx, st, LTRI_K_ATTN_RET, ctx->use_tc ? 2 : 1);
+      LTRI_CUDA(ctx, ctx->use_tc ? launch_attn_prefill_tc(d, grp[g], ctx->ret_phase, true, ctx->kv_maps, st)
+                                 : launch_attn_prefill(d, grp[g], 1, true, st));
+    }
   // commit the host state
   for (int l = 0; l < layer_count; ++l) {
     LayerState& s = ctx->at(seq, layer_begin + l);
