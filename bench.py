@@ -396,6 +396,9 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
     torch.cuda.synchronize(dev)
 
     # ---- device-resident timing ------------------------------------------------------------
+    # (the library's per-class CUDA events are on during the timed steps: they give kernel_ms_per_step and the
+    # rooflines from the very launches that `value` is made of; they cost about 1 % and keep consecutive kernel
+    # classes from overlapping their launches)
     for i in range(W):
         call(lt, kept[i], outs[i & 1])
     torch.cuda.synchronize(dev)
@@ -441,7 +444,6 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
         # the pulls of the timed calls against the bus: bytes the top-k kernels asked for (misses of the timed calls,
         # taken from the counters) over the time the pull kernels were running, next to a plain pinned-memory copy
         miss_timed = float(hm[1]) - float(miss_before_timed)
-        pull_ms = prof["pager_pull"][0]
         src = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
         dst = torch.empty_like(src, device=dev)
         best = None
@@ -454,9 +456,7 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
             best = min(best, b0.elapsed_time(b1)) if best else b0.elapsed_time(b1)
         bus = src.numel() / (best * 1e-3) / 1e9
         del src, dst
-        gbs = miss_timed * unit_bytes / (pull_ms * 1e-3) / 1e9 if pull_ms > 0 else None
-        pager["roofline"] = {"bound": "bus", "achieved": gbs, "peak": bus, "unit": "GB/s",
-                             "frac": gbs / bus if gbs else None,
+        pager["roofline"] = {"bound": "bus", "pulled_bytes": miss_timed * unit_bytes, "peak": bus, "unit": "GB/s",
                              "note": "host-to-device bytes of the timed calls' missing units over the run time of "
                                      "the pull kernels; peak = a 256 MiB copy from pinned memory on this box"}
     recall = {"final_chunk": needle_recall(lt, st, SQ, cfg)} if cfg.needle and rank == 0 else None
@@ -472,19 +472,25 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
         for s in range(dw):
             lt.ltri_decode_step(seq_ids, 0, L, *dec_in[s], out=dout)
         torch.cuda.synchronize(dev)
-        lt.ltri_profile_read()
-        lt.ltri_profile_enable(True)
+        # first half of the steps plain (tok/s), second half with the per-class events on (kernel times)
+        half = dw + max(1, (cfg.decode_steps - dw) // 2)
         d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier(world)
         d0.record()
-        for s in range(dw, cfg.decode_steps):
+        for s in range(dw, half):
             lt.ltri_decode_step(seq_ids, 0, L, *dec_in[s], out=dout)
         d1.record()
         torch.cuda.synchronize(dev)
         dms = max_over_ranks(d0.elapsed_time(d1), world, dev)
+        lt.ltri_profile_read()
+        lt.ltri_profile_enable(True)
+        for s in range(half, cfg.decode_steps):
+            lt.ltri_decode_step(seq_ids, 0, L, *dec_in[s], out=dout)
+        torch.cuda.synchronize(dev)
         dprof = lt.ltri_profile_read()
         lt.ltri_profile_enable(False)
-        dsteps = cfg.decode_steps - dw
+        psteps = max(1, cfg.decode_steps - half)
+        dsteps = half - dw
         dst = lt.ltri_get_stats(SQ, 0)
         ret_tok = dst.retrieved_tokens / cfg.n_kv_heads
         keys = cfg.n_sink + ret_tok + (dst.tokens - dst.evicted_end)
@@ -492,7 +498,7 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
         bytes_step = NSEQ * L * (cfg.n_kv_heads * dst.n_spans * cfg.head_dim * 2 +
                                  2 * cfg.n_kv_heads * cfg.head_dim * 2 * keys)
         k_ms = dprof["decode_retrieve"][0] + dprof["decode_attn"][0]
-        gbs = bytes_step * dsteps / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
+        gbs = bytes_step * psteps / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
         dec = {"value": world * NSEQ * dsteps / (dms * 1e-3), "unit": "tok/s", "steps": dsteps, "sequences": NSEQ,
                "ms_per_step": dms / dsteps,
                "keys_per_head": keys, "index_spans": dst.n_spans,
@@ -504,10 +510,14 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
                             "traffic_note": "bytes per step, scaled from an ncu capture of an 8-layer 64K case",
                             "kernels": "decode score+top-k and split-KV attention+merge",
                             "of": peaks["source"]},
-               "kernel_ms_per_step": {k: v[0] / dsteps for k, v in dprof.items() if v[1]}}
+               "kernel_ms_per_step": {k: v[0] / psteps for k, v in dprof.items() if v[1]}}
         if recall is not None:
             recall["last_decode_step"] = needle_recall(lt, st, SQ, cfg)
     clocks = sampler.stop(clk_lo, clk_hi)
+    if pager is not None:
+        pull_ms = prof["pager_pull"][0]
+        gbs = pager["roofline"]["pulled_bytes"] / (pull_ms * 1e-3) / 1e9 if pull_ms > 0 else None
+        pager["roofline"].update({"achieved": gbs, "frac": gbs / pager["roofline"]["peak"] if gbs else None})
 
     # ---- end-to-end: same steps with host buffers ---------------------------------------------
     e2e = None
@@ -569,15 +579,18 @@ def measure(cfg, K, W, rank, local, world, dev, peaks, want_e2e=True, per_layer_
     G = cfg.n_q_heads // cfg.n_kv_heads
     f_ret = sum(4.0 * cnt * G * cfg.head_dim * retrieved_all for (_, cnt) in timed)
     a_ms, a_cnt = prof["attn_local"]
+    a_cnt //= 2     # (every launch of the attention kernel is followed by its redo launch, which returns at once)
     r_ms, _ = prof["attn_retrieved"]
     per_layer = ATTN_LOCAL_DRAM_BYTES_PER_LAYER.get((cfg.n_q_heads, cfg.n_kv_heads, cfg.chunk, cfg.window, cfg.n_sink))
     window_full = timed[0][0] >= cfg.window + cfg.chunk
     traffic = per_layer * L / max(1, a_cnt // K) if per_layer and window_full else None
-    roof = {"bound": "tensor", **tensor_roofline(f_loc / (a_ms * 1e-3) / 1e12 if a_ms > 0 else None, peaks, clocks),
+    roof = {"bound": "tensor",
+            **tensor_roofline(f_loc / (a_ms * 1e-3) / 1e12 if a_ms > 0 else None, peaks, clocks),
             "traffic": traffic,
             "traffic_note": "DRAM bytes per launch, ncu capture of a 4-layer case of the same geometry x layers / 4",
             "kernel": "k_attn_tc, local part (sink | local | current)",
-            "launches": a_cnt, "ms_per_launch": a_ms / max(a_cnt, 1)}
+            "launches": a_cnt, "ms_per_launch": a_ms / max(a_cnt, 1),
+            "timing": "CUDA events of the library around the launch and its redo launch (which returns at once)"}
     roof_attn = {"bound": "tensor",
                  **tensor_roofline((f_loc + f_ret) / ((a_ms + r_ms) * 1e-3) / 1e12 if a_ms > 0 else None, peaks, clocks),
                  "kernels": "k_attn_tc local part + continuation over the retrieved spans (the chunked-prefill "
@@ -664,7 +677,8 @@ def run_ltri(args, cfg):
         "clocks": m["clocks"], "gpu_launches": m["launches"], "e2e": m["e2e"], "decode": m["decode"],
         "roofline": m["roofline"], "roofline_prefill_attention": m["roofline_prefill_attention"],
         "roofline_call": m["roofline_call"], "cpu_baseline": cpu,
-        "needle_recall": m["recall"], "pager": m["pager"], "kernel_ms_per_step": m["kernel_ms_per_step"], **extras,
+        "needle_recall": m["recall"], "pager": m["pager"], "kernel_ms_per_step": m["kernel_ms_per_step"],
+        **extras,
     }
     print(json.dumps(line))
 

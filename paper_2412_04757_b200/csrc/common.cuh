@@ -210,6 +210,33 @@ cudaError_t launch_decode_attn(const DevCtx& c, const DecBatch& b, int layer_beg
 // test kernel for the bounded waits: one wait with `short_limit` cycles on a barrier nothing completes (kernels_probe.cu)
 cudaError_t launch_wait_probe(const DevCtx& c, long long short_limit, cudaStream_t s);
 
+// ---- programmatic dependent launch -------------------------------------------------------
+// The kernels of a prefill call and of a decode step form a chain on one stream.  Launched through launch_chained,
+// a kernel's launch is prepared while its predecessor is still running and its CTAs start as soon as the predecessor
+// grid has finished; it touches global memory only after chain_wait(), which returns once that grid's writes are
+// visible.  No kernel releases its successor early: with one large CTA per SM (or a tuned number of them) the
+// successor's CTAs would only take resources away from the kernel that is still working (measured: decode 0.250
+// instead of 0.225 ms per step).  Launched the ordinary way, chain_wait() does nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                  Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---- small device helpers --------------------------------------------------------------
 __device__ __forceinline__ void set_status(const DevCtx& c, int code, int detail) {
   if (atomicCAS(&c.status[0], 0, code) == 0) c.status[1] = detail;

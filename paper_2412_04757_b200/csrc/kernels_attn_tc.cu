@@ -156,7 +156,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   // exch = 1: the launch that follows it with the same grid.  A CTA whose flag is clear returns at once; one whose
   // flag is set walks its work items again with the true maximum exchanged on every tile and overwrites what the
   // first launch stored, so inputs of any magnitude get the exact softmax.
-  if (exch && redo[blockIdx.x] == 0) return;
+  if (exch) {
+    chain_wait();
+    if (redo[blockIdx.x] == 0) return;
+  }
   const CUtensorMap* kvmaps = maps.kv;
   extern __shared__ unsigned char smem_raw[];
   // QFULL QFREE ODONE | KFULL[2] VFULL[2] KEMPTY[2] VEMPTY[2] | SREADY[2] PREADY[2][2] OFREE[2]
@@ -217,6 +220,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem = s_tmem_base;
+  if (!exch) chain_wait();  // everything above set up shared memory, barriers and TMEM only
   const int causal_ri = phase == 0 ? 2 : -1;
 
   // decode a work item
@@ -844,9 +848,10 @@ static cudaError_t launch_tc_g(const DevCtx& c, const PrefillArgs& a, int phase,
   // the regular launch, then the one that redoes the work of the CTAs that asked for it (they return at once otherwise)
   const int grid = min(nitems, ctas);
   if (grid > kTcMaxCtas) return cudaErrorInvalidValue;
-  k_attn_tc<G, false, MERGE><<<grid, kTcThreads, smem, s>>>(c, a, phase, final_out ? 1 : 0, c.tc_redo, maps, v_off);
-  k_attn_tc<G, true, MERGE><<<grid, kTcThreads, smem, s>>>(c, a, phase, final_out ? 1 : 0, c.tc_redo, maps, v_off);
-  return cudaGetLastError();
+  launch_chained(k_attn_tc<G, false, MERGE>, dim3(grid), dim3(kTcThreads), smem, s, c, a, phase, final_out ? 1 : 0,
+                 c.tc_redo, maps, v_off);
+  return launch_chained(k_attn_tc<G, true, MERGE>, dim3(grid), dim3(kTcThreads), smem, s, c, a, phase, final_out ? 1 : 0,
+                        c.tc_redo, maps, v_off);
 }
 
 cudaError_t launch_attn_prefill_tc(const DevCtx& c, const PrefillArgs& a, int phase, bool final_out,

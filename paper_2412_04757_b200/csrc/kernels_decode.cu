@@ -33,6 +33,7 @@ constexpr int kDWarpBytes = kDStages * 2 * kDTile * 256;  // K and V rows of eve
 template <int G>
 __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevCtx c, DecBatch b, int layer_begin, int layer_count,
                                                                 const __nv_bfloat16* __restrict__ q, int nsplit) {
+  chain_wait();
   extern __shared__ __align__(1024) unsigned char dsm[];
   // rs: first token of every range -- in a paged context (host-memory pager) its first K row, counted from the start
   // of the K slabs, instead: there a range lives in a sliding slab or in a slot of the unit cache
@@ -214,6 +215,7 @@ __global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm) k_decode_attn(DevC
 // merge of the split partials: grid (Hq, b.n*layer_count), 128 threads (one per output dim).
 __global__ void __launch_bounds__(kD) k_decode_merge(DevCtx c, DecBatch b, int layer_begin, int layer_count,
                                                      __nv_bfloat16* __restrict__ out, int nsplit) {
+  chain_wait();
   const int h = blockIdx.x, e = threadIdx.x;
   const int bi = blockIdx.y / layer_count, l = blockIdx.y % layer_count;
   const size_t unit = unit_of(c, b.seq[bi], layer_begin + l);
@@ -235,10 +237,10 @@ static cudaError_t launch_dec_g(const DevCtx& c, const DecBatch& b, int layer_be
                                 const __nv_bfloat16* q, __nv_bfloat16* out, int nsplit, cudaStream_t s) {
   const int smem = 4 * kDWarpBytes;
   cudaFuncSetAttribute(k_decode_attn<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  k_decode_attn<G><<<dim3(nsplit, c.Hkv, b.n * layer_count), kDecThreads, smem, s>>>(c, b, layer_begin, layer_count, q,
-                                                                                    nsplit);
-  k_decode_merge<<<dim3(c.Hq, b.n * layer_count), kD, 0, s>>>(c, b, layer_begin, layer_count, out, nsplit);
-  return cudaGetLastError();
+  launch_chained(k_decode_attn<G>, dim3(nsplit, c.Hkv, b.n * layer_count), dim3(kDecThreads), smem, s, c, b, layer_begin,
+                 layer_count, q, nsplit);
+  return launch_chained(k_decode_merge, dim3(c.Hq, b.n * layer_count), dim3(kD), 0, s, c, b, layer_begin, layer_count, out,
+                        nsplit);
 }
 
 cudaError_t launch_decode_attn(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int,

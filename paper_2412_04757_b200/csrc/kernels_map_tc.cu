@@ -64,8 +64,11 @@ __global__ void __launch_bounds__(kMapThreads, 1)
   const size_t unit = unit_of(c, a.seq, layer);
   // a layer with a retrieval head (Sec. 3.5) draws its map and votes from that head alone: the other KV heads have
   // nothing to add, and in the head's own group the other heads' columns are switched off through their offsets
-  const int rh = ret_head_of(c, layer);
-  if (rh >= 0 && g != rh / G) return;
+  int rh = -1;
+  if (c.ret_head) {  // (a table in global memory, written once at ltri_create: older than any predecessor in the chain)
+    rh = c.ret_head[layer];
+    if (rh >= 0 && g != rh / G) return;
+  }
   const bool is_cur = (int)blockIdx.x >= n_local_groups;
   const int tile0 = (is_cur ? (int)blockIdx.x - n_local_groups : (int)blockIdx.x) * kMapKT;
   const int ntile = min(kMapKT, (is_cur ? n_cur_tiles : n_local_tiles) - tile0);
@@ -118,6 +121,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem = s_tmem_base;
+  chain_wait();  // everything above set up shared memory, barriers and TMEM only
 
   if (warp == 16) {
     if (lane == 0) {
@@ -367,8 +371,8 @@ static cudaError_t launch_map_tc_g(const DevCtx& c, const PrefillArgs& a, const 
   const int gloc = (nloc + kMapKT - 1) / kMapKT, gcur = (ncur + kMapKT - 1) / kMapKT;
   const int smem = kMapKT * 32768 + 65536 + 3 * 4096 + 1024;  // key tiles, two query stages, the offset tiles
   cudaFuncSetAttribute(k_map_tc<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  k_map_tc<G><<<dim3(gloc + gcur, c.Hkv, a.layer_count), kMapThreads, smem, s>>>(c, a, gloc, nloc, ncur, maps);
-  return cudaGetLastError();
+  return launch_chained(k_map_tc<G>, dim3(gloc + gcur, c.Hkv, a.layer_count), dim3(kMapThreads), smem, s, c, a, gloc, nloc,
+                        ncur, maps);
 }
 
 cudaError_t launch_map_pass_tc(const DevCtx& c, const PrefillArgs& a, const void* kv_maps, cudaStream_t s) {

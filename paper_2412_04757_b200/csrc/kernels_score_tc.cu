@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(kScThreads, kScStages == 2 ? 2 : 1)
   __shared__ __align__(8) unsigned long long bars[2 * kScStages + 4];  // AFULL[3] AEMPTY[3] SFULL[2] SEMPTY[2]
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
+  chain_wait();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = blockIdx.y, layer = layer_begin + blockIdx.z;
   const size_t unit = unit_of(c, seq, layer);
@@ -195,10 +196,10 @@ cudaError_t launch_score_prefill_tc(const DevCtx& c, const PrefillArgs& a, int s
   const dim3 grid(gx > 0 ? gx : 1, c.Hkv, a.layer_count);
   if (two) {
     cudaFuncSetAttribute(k_score_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    k_score_tc<2><<<grid, kScThreads, smem, s>>>(c, a.seq, a.layer_begin, per_cta, npad_lay, kr);
+    return launch_chained(k_score_tc<2>, grid, dim3(kScThreads), smem, s, c, a.seq, a.layer_begin, per_cta, npad_lay, kr);
   } else {
     cudaFuncSetAttribute(k_score_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    k_score_tc<3><<<grid, kScThreads, smem, s>>>(c, a.seq, a.layer_begin, per_cta, npad_lay, kr);
+    return launch_chained(k_score_tc<3>, grid, dim3(kScThreads), smem, s, c, a.seq, a.layer_begin, per_cta, npad_lay, kr);
   }
   return cudaGetLastError();
 }

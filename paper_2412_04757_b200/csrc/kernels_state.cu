@@ -50,6 +50,7 @@ cudaError_t launch_init(const DevCtx& c, int seq, cudaStream_t s) {
 // ------------------------------------------------------------------------------------------
 // a0: copy the call's K/V rows into the cache slabs; 16 threads move one 256-byte row.
 __global__ void k_append_prefill(DevCtx c, PrefillArgs a) {
+  chain_wait();
   const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int c16 = gid & 15;
   size_t row = gid >> 4;  // over [layer_count][n][Hkv]
@@ -80,12 +81,12 @@ __global__ void k_append_prefill(DevCtx c, PrefillArgs a) {
 
 cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
   const size_t threads = (size_t)a.layer_count * a.n * c.Hkv * 16;
-  k_append_prefill<<<(unsigned)((threads + 255) / 256), 256, 0, s>>>(c, a);
-  return cudaGetLastError();
+  return launch_chained(k_append_prefill, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, s, c, a);
 }
 
 __global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer_count,
                                 const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v) {
+  chain_wait();
   const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int c16 = gid & 15;
   size_t row = gid >> 4;  // over [b.n][layer_count][Hkv]
@@ -118,14 +119,15 @@ __global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer
 cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int,
                                  const __nv_bfloat16* k, const __nv_bfloat16* v, cudaStream_t s) {
   const size_t threads = (size_t)b.n * layer_count * c.Hkv * 16;
-  k_append_decode<<<(unsigned)((threads + 255) / 256), 256, 0, s>>>(c, b, layer_begin, layer_count, k, v);
-  return cudaGetLastError();
+  return launch_chained(k_append_decode, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, s, c, b, layer_begin,
+                        layer_count, k, v);
 }
 
 // ------------------------------------------------------------------------------------------
 // a1: regions that left the window: every span gets its index vector, the bf16 sum of the keys of
 // its most voted token(s), and is appended to the span table.  One CTA per layer, one warp per span (32 warps).
 __global__ void __launch_bounds__(1024) k_evict_index(DevCtx c, EvictArgs a) {
+  chain_wait();
   const int layer = a.layer_begin + blockIdx.x;
   const size_t unit = unit_of(c, a.seq, layer);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
@@ -176,8 +178,8 @@ __global__ void __launch_bounds__(1024) k_evict_index(DevCtx c, EvictArgs a) {
 }
 
 cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_count, cudaStream_t s) {
-  k_evict_index<<<layer_count, 1024, 0, s>>>(c, a);  // a warp per span: one round for a region of up to 32 spans
-  return cudaGetLastError();
+  // a warp per span: one round for a region of up to 32 spans
+  return launch_chained(k_evict_index, dim3(layer_count), dim3(1024), 0, s, c, a);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -292,6 +294,7 @@ constexpr int kThetaThreads = 512;
 
 __global__ void __cluster_dims__(kThetaCluster, 1, 1) __launch_bounds__(kThetaThreads)
     k_theta_select(DevCtx c, int layer_begin, int m, long long rank, int tables) {
+  chain_wait();
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ unsigned hist[];  // [warps][kThetaBins]
@@ -437,6 +440,7 @@ __global__ void __cluster_dims__(kThetaCluster, 1, 1) __launch_bounds__(kThetaTh
 // absolute threshold: thq in units of the map summed over all heads, thq1 in units of a single (retrieval) head's map;
 // with per-layer tables the layer's own theta, scaled here
 __global__ void k_theta_set(DevCtx c, int layer_begin, long long thq, long long thq1, int tables) {
+  chain_wait();
   const int layer = layer_begin + blockIdx.x;
   const bool one = ret_head_of(c, layer) >= 0;
   long long t = one ? thq1 : thq;
@@ -447,6 +451,7 @@ __global__ void k_theta_set(DevCtx c, int layer_begin, long long thq, long long 
 // step 2: suffix sums along each row of D = Mq - theta ("sum the right elements", Fig. 2):
 // Rsuf[i][x] = sum_{j=x..i} D[i][j].  One warp per row, 32-wide shuffle scans from the diagonal leftwards.
 __global__ void __launch_bounds__(256) k_seg_rowscan(DevCtx c, int layer_begin, int m) {
+  chain_wait();
   const int layer = layer_begin + blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int i = blockIdx.x * 8 + warp;
@@ -478,6 +483,7 @@ __global__ void __launch_bounds__(256) k_seg_rowscan(DevCtx c, int layer_begin, 
 // seg_unit > 0 (segmentation per memory unit): only intervals inside one unit of seg_unit tokens on the absolute grid
 // are candidates; `origin` is the absolute position of the region's first token.
 __global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin, int m, int seg_unit, int origin) {
+  chain_wait();
   extern __shared__ long long sm[];
   long long* part = sm;             // [32 ry][32 cx]
   long long* sbest = sm + 32 * 32;  // [m + 32]
@@ -545,6 +551,7 @@ struct NmsArgs {
 };
 
 __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
+  chain_wait();
   __shared__ long long skey[2048];
   __shared__ short scd[2048];
   __shared__ int kx[kMaxTopK], ky[kMaxTopK];
@@ -790,16 +797,18 @@ cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_
     if (rank < 0) rank = 0;
     if (rank > N - 1) rank = N - 1;
     const int hsmem = (kThetaThreads / 32) * kThetaBins * (int)sizeof(unsigned);
-    k_theta_select<<<layer_count * kThetaCluster, kThetaThreads, hsmem, s>>>(c, layer_begin, m, rank, tables);
+    launch_chained(k_theta_select, dim3(layer_count * kThetaCluster), dim3(kThetaThreads), hsmem, s, c, layer_begin, m,
+                   rank, tables ? 1 : 0);
   } else {
-    k_theta_set<<<layer_count, 1, 0, s>>>(c, layer_begin, theta_q_abs,
-                                          (long long)nearbyint((double)theta * (double)kQScale), tables);
+    launch_chained(k_theta_set, dim3(layer_count), dim3(1), 0, s, c, layer_begin, theta_q_abs,
+                   (long long)nearbyint((double)theta * (double)kQScale), tables ? 1 : 0);
   }
-  k_seg_rowscan<<<dim3((m + 7) / 8, layer_count), 256, 0, s>>>(c, layer_begin, m);
+  launch_chained(k_seg_rowscan, dim3((m + 7) / 8, layer_count), dim3(256), 0, s, c, layer_begin, m);
   const size_t smem = (size_t)(32 * 32 + m + 32) * sizeof(long long);
-  k_seg_colscan<<<dim3((m + 31) / 32, layer_count), 1024, smem, s>>>(c, layer_begin, m, seg_unit, reg_start);
+  launch_chained(k_seg_colscan, dim3((m + 31) / 32, layer_count), dim3(1024), smem, s, c, layer_begin, m, seg_unit,
+                 reg_start);
   NmsArgs a{seq, layer_begin, m, reg_start, slot, max_spans, n, t0, q, tables ? 1 : 0, seg_unit};
-  k_seg_nms<<<layer_count, 1024, 0, s>>>(c, a);
+  launch_chained(k_seg_nms, dim3(layer_count), dim3(1024), 0, s, c, a);
   return cudaGetLastError();
 }
 
@@ -873,6 +882,7 @@ cudaError_t launch_score_prefill(const DevCtx& c, const PrefillArgs& a, int span
 // Half-warp per 256-byte index row, 16 bytes per lane, four rows in flight; grid (span tiles of 256, Hkv, units).
 __global__ void __launch_bounds__(256) k_score_dec(DevCtx c, int layer_begin, DecBatch b, int layer_count,
                                                    const __nv_bfloat16* __restrict__ q) {
+  chain_wait();
   __shared__ float su[kD];
   const int g = blockIdx.y;
   const int bi = blockIdx.z / layer_count, l = blockIdx.z % layer_count, layer = layer_begin + l;
@@ -928,8 +938,8 @@ __global__ void __launch_bounds__(256) k_score_dec(DevCtx c, int layer_begin, De
 cudaError_t launch_score_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int,
                                 const __nv_bfloat16* q, int span_bound, cudaStream_t s) {
   if (span_bound <= 0) span_bound = 1;
-  k_score_dec<<<dim3((span_bound + 255) / 256, c.Hkv, b.n * layer_count), 256, 0, s>>>(c, layer_begin, b, layer_count, q);
-  return cudaGetLastError();
+  return launch_chained(k_score_dec, dim3((span_bound + 255) / 256, c.Hkv, b.n * layer_count), dim3(256), 0, s, c,
+                        layer_begin, b, layer_count, q);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1045,6 +1055,7 @@ enum { kTopkSelect = 0, kTopkBallot = 1, kTopkVote = 2 };
 template <bool DECODE>
 __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin, DecBatch b, int layer_count,
                                               int evicted_end, int mode) {
+  chain_wait();
   __shared__ unsigned hist[256];
   __shared__ unsigned s_prefix, s_need;
   __shared__ unsigned long long s_prefix64;
@@ -1462,6 +1473,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
                                                        const __nv_bfloat16* __restrict__ q,
                                                        const __nv_bfloat16* __restrict__ knew,
                                                        const __nv_bfloat16* __restrict__ vnew) {
+  chain_wait();
   extern __shared__ float ssc[];  // [N]
   __shared__ float su[kD];
   __shared__ unsigned hist[256];
@@ -1665,6 +1677,7 @@ constexpr int kRetSliceMax = 12288;  // scores a CTA keeps in shared memory (48 
 __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThreads)
     k_dec_retrieve_cl(DevCtx c, int layer_begin, DecBatch b, int layer_count, const __nv_bfloat16* __restrict__ q,
                       const __nv_bfloat16* __restrict__ knew, const __nv_bfloat16* __restrict__ vnew) {
+  chain_wait();
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ float ssc[];  // this CTA's slice of the scores
@@ -1879,15 +1892,13 @@ cudaError_t launch_dec_retrieve_fused(const DevCtx& c, const DecBatch& b, int la
                                       int span_bound, bool force_cluster, int threads, cudaStream_t s) {
   span_bound = max(span_bound, 1);
   if (span_bound <= kFusedMaxSpans && !force_cluster) {  // one CTA per head: no cluster barriers
-    k_dec_retrieve<<<dim3(c.Hkv, b.n * layer_count), threads, (int)sizeof(float) * span_bound, s>>>(
-        c, layer_begin, b, layer_count, q, k, v);
-    return cudaGetLastError();
+    return launch_chained(k_dec_retrieve, dim3(c.Hkv, b.n * layer_count), dim3(threads), sizeof(float) * span_bound, s,
+                          c, layer_begin, b, layer_count, q, k, v);
   }
   const int per = (span_bound + kRetCluster - 1) / kRetCluster;
   if (per > kRetSliceMax) return cudaErrorInvalidValue;
-  k_dec_retrieve_cl<<<dim3(c.Hkv * kRetCluster, b.n * layer_count), kRetThreads, (int)sizeof(float) * per, s>>>(
-      c, layer_begin, b, layer_count, q, k, v);
-  return cudaGetLastError();
+  return launch_chained(k_dec_retrieve_cl, dim3(c.Hkv * kRetCluster, b.n * layer_count), dim3(kRetThreads),
+                        sizeof(float) * per, s, c, layer_begin, b, layer_count, q, k, v);
 }
 int dec_retrieve_fused_max_spans() { return kRetCluster * kRetSliceMax; }
 
@@ -1911,9 +1922,10 @@ static cudaError_t launch_topk(const DevCtx& c, int seq, int layer_begin, const 
     if (e != cudaSuccess) return e;
   }
   if (c.vote)
-    k_topk<DECODE><<<dim3(c.Hkv, gy), 512, smem, s>>>(c, seq, layer_begin, b, layer_count, evicted_end, kTopkBallot);
-  k_topk<DECODE><<<dim3(c.Hkv, gy), 512, smem, s>>>(c, seq, layer_begin, b, layer_count, evicted_end,
-                                                   c.vote ? kTopkVote : kTopkSelect);
+    launch_chained(k_topk<DECODE>, dim3(c.Hkv, gy), dim3(512), smem, s, c, seq, layer_begin, b, layer_count, evicted_end,
+                   (int)kTopkBallot);
+  launch_chained(k_topk<DECODE>, dim3(c.Hkv, gy), dim3(512), smem, s, c, seq, layer_begin, b, layer_count, evicted_end,
+                 (int)(c.vote ? kTopkVote : kTopkSelect));
   return cudaGetLastError();
 }
 
