@@ -552,8 +552,7 @@ struct NmsArgs {
 
 __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   chain_wait();
-  __shared__ long long skey[2048];
-  __shared__ short scd[2048];
+  __shared__ long long skey[768];  // scratch of the query representatives: token lists and counts per span
   __shared__ int kx[kMaxTopK], ky[kMaxTopK];
   __shared__ int out_start[2 * kMaxTopK + 1], out_len[2 * kMaxTopK + 1];
   __shared__ int s_nout;
@@ -567,68 +566,82 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   const int phi_milli = a.tables && c.phi_l ? c.phi_l[layer] : c.phi_milli;
   const float rep_lambda = a.tables && c.lambda_l ? c.lambda_l[layer] : c.rep_lambda;
   const int ncand = 2 * m - 1;
-  int npow = 1;
-  while (npow < ncand) npow <<= 1;
   const long long* gbest = c.best + (size_t)layer * 2 * c.chunk;
-  for (int t = threadIdx.x; t < npow; t += blockDim.x) {
-    skey[t] = t < ncand ? gbest[t] : 0;
-    scd[t] = (short)t;
+  // Greedy NMS without a sort: the candidate the sorted sweep would reach next is the best one that is still alive
+  // (key larger, or equal key and smaller anti-diagonal), so every round takes the block-wide maximum over the alive
+  // candidates, keeps it, and lets every thread strike out its own candidates that the new span suppresses (or whose
+  // unit is full).  At most max_spans rounds of two barriers each instead of sorting up to 2047 keys.
+  // Candidate of anti-diagonal cd: key = (S << 10) | (1023 - len) > 0; x = (cd - len) / 2, y = x + len.
+  __shared__ long long s_wkey[32];
+  __shared__ int s_wcd[32];
+  const int tid = threadIdx.x, wlane = tid & 31, wid = tid >> 5;
+  long long ckey[2];
+  int cx[2], cy[2];
+  bool alive[2];
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int cd = tid + u * 1024;
+    ckey[u] = cd < ncand ? gbest[cd] : 0;
+    const int len = 1023 - (int)(ckey[u] & 1023);
+    cx[u] = (cd - len) >> 1;
+    cy[u] = cx[u] + len;
+    alive[u] = ckey[u] > 0;
+  }
+  for (int t = tid; t < kMaxTopK + 2; t += blockDim.x) s_ucnt[t] = 0;
+  int kept = 0;
+  auto better = [](long long ka, int ca, long long kb, int cb) { return ka > kb || (ka == kb && ca < cb); };
+  while (kept < cap_total) {
+    long long bk = 0;
+    int bc = 0x7fffffff;
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+      if (alive[u] && better(ckey[u], tid + u * 1024, bk, bc)) {
+        bk = ckey[u];
+        bc = tid + u * 1024;
+      }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const long long ok = shfl_xor_ll(bk, o);
+      const int oc = __shfl_xor_sync(0xffffffffu, bc, o);
+      if (better(ok, oc, bk, bc)) {
+        bk = ok;
+        bc = oc;
+      }
+    }
+    if (wlane == 0) {
+      s_wkey[wid] = bk;
+      s_wcd[wid] = bc;
+    }
+    __syncthreads();
+    bk = s_wkey[wlane];  // every warp reduces the 32 partial results itself: all threads learn the winner
+    bc = s_wcd[wlane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const long long ok = shfl_xor_ll(bk, o);
+      const int oc = __shfl_xor_sync(0xffffffffu, bc, o);
+      if (better(ok, oc, bk, bc)) {
+        bk = ok;
+        bc = oc;
+      }
+    }
+    if (bk <= 0) break;  // nothing alive is left (the same decision in every thread)
+    const int wl = 1023 - (int)(bk & 1023);
+    const int wx = (bc - wl) >> 1, wy = wx + wl;
+    if (tid == 0) {
+      kx[kept] = wx;
+      ky[kept] = wy;
+      if (SU > 0) ++s_ucnt[unit_idx(wx)];
+    }
+    ++kept;
+    __syncthreads();  // the unit counts are up to date; s_wkey may be overwritten
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+      alive[u] = alive[u] && tid + u * 1024 != bc && !nms_suppressed(cx[u], cy[u], wx, wy, phi_milli) &&
+                 (SU == 0 || s_ucnt[unit_idx(cx[u])] < a.max_spans);
   }
   __syncthreads();
-  // bitonic sort, "a before b" iff key larger, or equal key and smaller anti-diagonal
-  for (int k = 2; k <= npow; k <<= 1)
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int t = threadIdx.x; t < npow; t += blockDim.x) {
-        const int p = t ^ j;
-        if (p > t) {
-          const long long ka = skey[t], kb = skey[p];
-          const short ca = scd[t], cb = scd[p];
-          const bool a_first = ka > kb || (ka == kb && ca < cb);
-          const bool up = (t & k) == 0;
-          if (up ? !a_first : a_first) {
-            skey[t] = kb;
-            skey[p] = ka;
-            scd[t] = cb;
-            scd[p] = ca;
-          }
-        }
-      }
-      __syncthreads();
-    }
-  // greedy NMS by warp 0, 32 candidates per round
   if (threadIdx.x < 32) {
     const int lane = threadIdx.x;
-    int kept = 0;
-    for (int t = lane; t < kMaxTopK + 2; t += 32) s_ucnt[t] = 0;
-    __syncwarp();
-    for (int base = 0; base < ncand && kept < cap_total; base += 32) {
-      const int idx = base + lane;
-      const long long key = idx < ncand ? skey[idx] : 0;
-      const int len = 1023 - (int)(key & 1023);
-      const int x = ((int)scd[idx < ncand ? idx : 0] - len) >> 1;
-      const int y = x + len;
-      bool alive = key > 0;
-      if (__ballot_sync(0xffffffffu, alive) == 0) break;  // sorted: nothing positive follows
-      for (int q = 0; q < kept; ++q) alive = alive && !nms_suppressed(x, y, kx[q], ky[q], phi_milli);
-      if (SU > 0) alive = alive && s_ucnt[unit_idx(x)] < a.max_spans;  // the candidate's unit still has room
-      unsigned mask = __ballot_sync(0xffffffffu, alive);
-      while (mask && kept < cap_total) {
-        const int f = __ffs(mask) - 1;
-        const int fx = __shfl_sync(0xffffffffu, x, f), fy = __shfl_sync(0xffffffffu, y, f);
-        if (lane == 0) {
-          kx[kept] = fx;
-          ky[kept] = fy;
-          if (SU > 0) ++s_ucnt[unit_idx(fx)];
-        }
-        ++kept;
-        __syncwarp();
-        alive = alive && lane != f && !nms_suppressed(x, y, fx, fy, phi_milli);
-        if (SU > 0) alive = alive && s_ucnt[unit_idx(x)] < a.max_spans;
-        mask = __ballot_sync(0xffffffffu, alive);
-      }
-      __syncwarp();
-    }
-    __syncwarp();
     // order the kept spans by start (rank sort), then gap fill
     int rank0 = 0, rank1 = 0;
     const int x0 = lane < kept ? kx[lane] : 0x7fffffff;
@@ -688,7 +701,7 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   const long long* votes = c.votes + unit * c.Tpad;
   const __nv_bfloat16* q = a.q + (size_t)blockIdx.x * a.n * c.Hq * kD;
-  int* rep_tok = reinterpret_cast<int*>(skey);          // [Jmax][kMaxReps], the sort buffer is free now
+  int* rep_tok = reinterpret_cast<int*>(skey);          // [Jmax][kMaxReps]
   int* rep_cnt = rep_tok + (2 * kMaxTopK + 1) * kMaxReps;
   __syncthreads();
   // representative count of every span: static, or from the area ratio of Sec. 3.3.2 on the raw region map.  The
@@ -740,51 +753,67 @@ __global__ void __launch_bounds__(1024) k_seg_nms(DevCtx c, NmsArgs a) {
     }
   }
   __syncthreads();
-  for (int task = warp; task < nout * c.Hkv; task += nwarps) {
+  // a half-warp per (span, KV head): sixteen lanes x eight dimensions; the rows of the heads of the group are all in
+  // flight before they are added up, per head over the representative tokens (ascending) and then over the heads in
+  // ascending order
+  const int hw = lane >> 4, hl = lane & 15;
+  const int rh = ret_head_of(c, layer);
+  for (int task = 2 * warp + hw; task < nout * c.Hkv; task += 2 * nwarps) {
     const int j = task / c.Hkv, g = task % c.Hkv;
     const int nrep = rep_cnt[j];
-    // per head: sum over the representative tokens (ascending), then the heads of the group in ascending order
-    float qr[8][4];
-#pragma unroll
-    for (int hh = 0; hh < 8; ++hh) qr[hh][0] = qr[hh][1] = qr[hh][2] = qr[hh][3] = 0.f;
-    auto add_row = [](float (&acc)[4], const uint2& w) {
-      const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&w.x);
-      const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&w.y);
-      acc[0] += __bfloat162float(p0.x);
-      acc[1] += __bfloat162float(p0.y);
-      acc[2] += __bfloat162float(p1.x);
-      acc[3] += __bfloat162float(p1.y);
-    };
-    const __nv_bfloat16* qg = q + (size_t)g * c.G * kD + lane * 4;
+    const __nv_bfloat16* qg = q + (size_t)g * c.G * kD + hl * 8;
     // a layer with a retrieval head (Sec. 3.5) has one representative per span, that head's: the other heads add zero
-    const int rh = ret_head_of(c, layer);
     auto counts = [&](int hh) { return hh < c.G && (rh < 0 || g * c.G + hh == rh); };
-    for (int r = 0; r < nrep; ++r) {
-      const __nv_bfloat16* row = qg + (size_t)(rep_tok[j * kMaxReps + r] - a.t0) * c.Hq * kD;
-      uint2 raw[8];
+    auto add8 = [](float (&acc)[8], const uint4& w) {
+      const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&w);
 #pragma unroll
-      for (int hh = 0; hh < 8; ++hh)
-        raw[hh] = counts(hh) ? *reinterpret_cast<const uint2*>(row + (size_t)hh * kD) : make_uint2(0u, 0u);
-#pragma unroll
-      for (int hh = 0; hh < 8; ++hh) add_row(qr[hh], raw[hh]);
-    }
-    float ug[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int hh = 0; hh < 8; ++hh)
-      if (hh < c.G) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) ug[e] += qr[hh][e];
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(p2[i]);
+        acc[2 * i] += f.x;
+        acc[2 * i + 1] += f.y;
       }
-    for (int hh = 8; hh < c.G; ++hh) {  // groups wider than eight heads
-      if (!counts(hh)) continue;
-      float w[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int r = 0; r < nrep; ++r)
-        add_row(w, *reinterpret_cast<const uint2*>(qg + ((size_t)(rep_tok[j * kMaxReps + r] - a.t0) * c.Hq + hh) * kD));
+    };
+    float ug[8];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) ug[e] += w[e];
+    for (int e = 0; e < 8; ++e) ug[e] = 0.f;
+    if (nrep == 1) {
+      const __nv_bfloat16* row = qg + (size_t)(rep_tok[j * kMaxReps] - a.t0) * c.Hq * kD;
+      for (int h0 = 0; h0 < c.G; h0 += 8) {
+        uint4 raw[8];
+#pragma unroll
+        for (int hh = 0; hh < 8; ++hh)
+          raw[hh] = counts(h0 + hh) ? *reinterpret_cast<const uint4*>(row + (size_t)(h0 + hh) * kD) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int hh = 0; hh < 8; ++hh) {
+          float one[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) one[e] = 0.f;
+          add8(one, raw[hh]);  // (0 + x first, as the general path does)
+#pragma unroll
+          for (int e = 0; e < 8; ++e) ug[e] += one[e];
+        }
+      }
+    } else {
+      for (int hh = 0; hh < c.G; ++hh) {
+        if (!counts(hh)) continue;
+        uint4 raw[kMaxReps];
+#pragma unroll
+        for (int r = 0; r < kMaxReps; ++r)
+          raw[r] = r < nrep ? *reinterpret_cast<const uint4*>(qg + ((size_t)(rep_tok[j * kMaxReps + r] - a.t0) * c.Hq + hh) * kD)
+                            : make_uint4(0u, 0u, 0u, 0u);
+        float one[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) one[e] = 0.f;
+#pragma unroll
+        for (int r = 0; r < kMaxReps; ++r)
+          if (r < nrep) add8(one, raw[r]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ug[e] += one[e];
+      }
     }
-    *reinterpret_cast<float4*>(c.u + (((size_t)layer * c.Hkv + g) * c.Jmax + j) * kD + lane * 4) =
-        make_float4(ug[0], ug[1], ug[2], ug[3]);
+    float* up = c.u + (((size_t)layer * c.Hkv + g) * c.Jmax + j) * kD + hl * 8;
+    *reinterpret_cast<float4*>(up) = make_float4(ug[0], ug[1], ug[2], ug[3]);
+    *reinterpret_cast<float4*>(up + 4) = make_float4(ug[4], ug[5], ug[6], ug[7]);
   }
 }
 
@@ -1917,7 +1946,7 @@ template <bool DECODE>
 static cudaError_t launch_topk(const DevCtx& c, int seq, int layer_begin, const DecBatch& b, int layer_count, int gy,
                                int evicted_end, cudaStream_t s) {
   const int smem = topk_unit_smem(c);
-  if (smem > 48 * 1024) {
+  if (smem > 32 * 1024) {  // (static shared memory comes on top: ask for the larger limit in good time)
     cudaError_t e = cudaFuncSetAttribute(k_topk<DECODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
   }
