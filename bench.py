@@ -256,10 +256,10 @@ def workload_config(cfg, world, nseq):
 # scaled to the launch this run times (traffic grows in proportion to these units):
 #  * local attention (k_attn_tc phase 0), Llama-3-8B geometry, chunk 512, window 4096 full, sink 64: DRAM read +
 #    write of one launch over 4 layers at 16K context -> bytes per layer of a launch
-ATTN_LOCAL_DRAM_BYTES_PER_LAYER = {(32, 8, 512, 4096, 64): (95.14e6 + 8.42e6) / 4}
-#  * decode retrieval + attention: 239.4 MB measured against 237.8 MB of algorithmic bytes for an 8-layer step at
+ATTN_LOCAL_DRAM_BYTES_PER_LAYER = {(32, 8, 512, 4096, 64): (94.41e6 + 7.35e6) / 4}
+#  * decode retrieval + attention: 239.7 MB measured against 237.8 MB of algorithmic bytes for an 8-layer step at
 #    64K: every byte is read once, nothing is re-read
-DECODE_DRAM_PER_ALGORITHMIC_BYTE = 239.4 / 237.8
+DECODE_DRAM_PER_ALGORITHMIC_BYTE = 239.7 / 237.8
 NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16, per GPU
 NOMINAL_HBM_GBS = 8000.0
 

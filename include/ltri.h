@@ -27,10 +27,10 @@
  *    logits q.k * softmax_scale stay below about 2000 in absolute value (the local-map
  *    pass carries the row offsets -max - log2(sum) through an fp32 accumulator clamped at
  *    that size); inside that range every softmax is exact however far a later key tile
- *    exceeds the running maximum: the prefill attention kernel bounds the logits of a
- *    work item by |q| |k| scale (the largest key norm of a (sequence, layer, KV head) is
- *    tracked as keys are appended) and, where the bound is too wide for its late-moving
- *    reference maximum, exchanges the true maximum on every tile instead.
+ *    exceeds the running maximum: the prefill attention kernel notices when a tile's
+ *    maximum outruns its late-moving reference maximum by more than 2^90 and flags its
+ *    CTA; a second launch of the same kernel (it returns at once for CTAs without a flag)
+ *    then recomputes those CTAs' work with the true maximum exchanged on every tile.
  */
 #ifndef LTRI_H_
 #define LTRI_H_

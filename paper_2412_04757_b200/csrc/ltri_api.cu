@@ -241,8 +241,6 @@ struct ltri_ctx {
   int sm_count = 148;
   bool use_tc = false;     // tcgen05/TMEM/TMA attention kernels (default when available)
   int dec_fused = -1;      // decode retrieval in one launch: -1 auto, 0 never, 1 whenever the index fits, 2 cluster kernel
-  int dec_split = 0;       // split count of the decode attention: 0 auto (testing aid)
-  int dec_ret_threads = 0; // CTA size of the one-CTA decode retrieval kernel: 0 auto (testing aid)
   // host-buffer entry (LTRI_FLAG_HOST_STAGING): two staging sets in the arena, a copy-up and a copy-down stream, and
   // events that order every reuse of a set's layer-group slices
   static constexpr int kHostGroups = 4;
@@ -422,11 +420,6 @@ int ltri_create(const ltri_params* p, void* cuda_stream, ltri_ctx** out) {
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   // testing aid: 0 two launches, 1 one launch, 2 one launch with the cluster kernel whatever the index size
   if (const char* f = std::getenv("LTRI_DEC_FUSED")) ctx->dec_fused = std::max(0, std::min(2, std::atoi(f)));
-  if (const char* f = std::getenv("LTRI_DEC_SPLIT")) ctx->dec_split = std::max(0, std::atoi(f));    // testing aid
-  if (const char* f = std::getenv("LTRI_DEC_RET_THREADS")) {                                        // testing aid
-    const int t = std::atoi(f);
-    if (t == 256 || t == 512 || t == 1024) ctx->dec_ret_threads = t;
-  }
   const char* impl = std::getenv("LTRI_ATTN_IMPL");  // "mma" selects the warp-MMA kernels (debugging aid)
   ctx->use_tc = tc_attention_supported(ctx->d) && !(impl && std::strcmp(impl, "mma") == 0) &&
                 tc_encode_kv_maps(ctx->d, ctx->kv_maps);
@@ -918,7 +911,6 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
           nsplit = ns;
         }
       }
-      if (ctx->dec_split > 0) nsplit = std::min(ctx->dec_split, kMaxDecSplit);
     }
     // retrieval in one launch with the scores in shared memory: one CTA per (sequence, layer, KV head) when there are
     // enough heads to fill the GPU and the index fits one CTA (12K spans), a cluster of eight CTAs per head for a larger
@@ -936,8 +928,7 @@ int ltri_decode_step(ltri_ctx* ctx, const int32_t* seq_ids, int n_seqs, int laye
       Scope sc(ctx, st, LTRI_K_DEC_RETRIEVE, 1);
       // CTA size of the one-CTA kernel: 1024 threads fit once per SM, 512 twice; with more CTAs than SMs the smaller
       // size keeps all of them resident instead of running a second, partly empty wave
-      int ret_threads = units > ctx->sm_count ? 512 : 1024;
-      if (ctx->dec_ret_threads > 0) ret_threads = ctx->dec_ret_threads;
+      const int ret_threads = units > ctx->sm_count ? 512 : 1024;
       LTRI_CUDA(ctx, launch_dec_retrieve_fused(d, b, layer_begin, layer_count, qb, kb, vb, (int)ub, ctx->dec_fused == 2,
                                                ret_threads, st));
     } else {
