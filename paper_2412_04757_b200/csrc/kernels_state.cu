@@ -242,6 +242,54 @@ __device__ __forceinline__ unsigned pick_from_bottom(const unsigned* hist, int n
   return __shfl_sync(0xffffffffu, bin, src);
 }
 
+// Counting one radix digit of many keys with few shared-memory atomics.  Scores of one head share their leading bits,
+// so in the first passes nearly every key falls into the same bin and one atomic per key would serialise on it.  A
+// thread adds up runs of equal digits among its own keys; when all lanes of a warp end on the same digit, the warp
+// adds their last runs with one atomic.  flush() is called by all 32 lanes of a warp, converged.
+struct DigitRuns {
+  int cur = -1;
+  unsigned run = 0;
+  __device__ __forceinline__ void add(unsigned* hist, int d) {
+    if (d == cur) {
+      ++run;
+    } else {
+      if (run) atomicAdd(&hist[cur], run);
+      cur = d;
+      run = 1;
+    }
+  }
+  __device__ __forceinline__ void flush(unsigned* hist) {
+    const int top = __reduce_max_sync(0xffffffffu, cur);  // (-1: a lane without a matching key)
+    if (__all_sync(0xffffffffu, cur == top || cur < 0)) {
+      const unsigned sum = __reduce_add_sync(0xffffffffu, run);
+      if ((threadIdx.x & 31) == 0 && sum) atomicAdd(&hist[top], sum);
+    } else if (run) {
+      atomicAdd(&hist[cur], run);
+    }
+    cur = -1;
+    run = 0;
+  }
+};
+
+// Exclusive scan of the nt (a multiple of 32, at most 1024) counts in s_scan by the first warp of the CTA; returns the
+// total to every thread of that warp.  The caller brackets it with __syncthreads().
+__device__ __forceinline__ int warp0_exclusive_scan(int* s_scan, int nt) {
+  const int lane = threadIdx.x & 31;
+  int run = 0;
+  for (int blk = 0; blk < nt; blk += 32) {
+    const int v = s_scan[blk + lane];
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    s_scan[blk + lane] = run + inc - v;
+    run += __shfl_sync(0xffffffffu, inc, 31);
+  }
+  return run;
+}
+
 // ------------------------------------------------------------------------------------------
 // a3 segmenter, step 1: exact rank selection of theta (quantile mode) over the causal entries of Mq.
 // Pass 1 counts negatives (only hand-built maps have any) and zeros (a sparse map is mostly zeros) and builds a
@@ -1011,12 +1059,36 @@ __device__ __forceinline__ unsigned order_key(float f) {
 
 // Radix select of the K largest keys among KEY(0..N) (ties: lower index first), one 8-bit digit per pass from the top.
 // Writes the chosen indices, unordered, to s_ids and their number to *s_cnt (which the caller has zeroed).  Called by
-// every thread of the CTA; K < N.
-template <typename KT, typename KeyF>
+// every thread of the CTA; K < N.  R > 0 (keys that are expensive to read, 32-bit): up to R keys per thread are read
+// once and kept in registers (thread t holds keys t, t + nt, ...); with more keys than that, or R = 0, every pass
+// reads them through KEY.
+template <typename KT, int R, typename KeyF>
 __device__ __forceinline__ void radix_select_top(KeyF&& KEY, int N, int K, unsigned* hist, KT* s_prefix,
                                                  unsigned* s_need, int* s_scan, int* s_cnt, int* s_ids) {
+  static_assert(R == 0 || sizeof(KT) == 4, "register copies are kept of 32-bit keys only");
   const int tid = threadIdx.x, nt = blockDim.x;
   constexpr int kPasses = (int)sizeof(KT);
+  const bool inreg = R > 0 && N <= R * nt;
+  unsigned kr[R > 0 ? R : 1];
+  if (inreg) {
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+      const int s = tid + i * nt;
+      kr[i] = s < N ? (unsigned)KEY(s) : 0u;
+    }
+  }
+  // f(index, key) for every key of this thread
+  auto for_each_key = [&](auto&& f) {
+    if (inreg) {
+#pragma unroll
+      for (int i = 0; i < R; ++i) {
+        const int s = tid + i * nt;
+        if (s < N) f(s, (KT)kr[i]);
+      }
+    } else {
+      for (int s = tid; s < N; s += nt) f(s, KEY(s));
+    }
+  };
   if (tid == 0) {
     *s_prefix = 0;
     *s_need = K;  // rank from the top, 1-based: find key T with #(key > T) < K <= #(key >= T)
@@ -1027,10 +1099,11 @@ __device__ __forceinline__ void radix_select_top(KeyF&& KEY, int N, int K, unsig
     __syncthreads();
     const KT prefix = *s_prefix;
     const KT himask = pass == 0 ? (KT)0 : (KT)(~(KT)0 << (shift + 8));
-    for (int s = tid; s < N; s += nt) {
-      const KT key = KEY(s);
-      if ((key & himask) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
-    }
+    DigitRuns dr;
+    for_each_key([&](int, KT key) {
+      if ((key & himask) == prefix) dr.add(hist, (int)((unsigned)(key >> shift) & 255u));
+    });
+    dr.flush(hist);
     __syncthreads();
     if (tid < 32) {
       unsigned need = *s_need;
@@ -1044,21 +1117,25 @@ __device__ __forceinline__ void radix_select_top(KeyF&& KEY, int N, int K, unsig
   }
   const KT T = *s_prefix;
   const unsigned need_eq = *s_need;  // how many of the == T elements are taken (lowest ids first)
-  // contiguous id partition so that ties are picked in id order
+  // the last pass counted the keys equal to T in the bin of T's low digit (the histogram is still there)
+  if (hist[(unsigned)T & 255u] == need_eq) {
+    // every key equal to the threshold is taken: no order among them is needed
+    for_each_key([&](int s, KT key) {
+      if (key >= T) {
+        const int slot = atomicAdd(s_cnt, 1);
+        if (slot < kMaxTopK) s_ids[slot] = s;
+      }
+    });
+    return;
+  }
+  // ties at the cut: contiguous id partition so that they are picked in id order
   const int per = (N + nt - 1) / nt;
-  const int lo = tid * per, hi = min(N, lo + per);
+  const int lo = min(N, tid * per), hi = min(N, lo + per);
   int eq = 0;
   for (int s = lo; s < hi; ++s) eq += KEY(s) == T;
   s_scan[tid] = eq;
   __syncthreads();
-  if (tid == 0) {
-    int run = 0;
-    for (int t = 0; t < nt; ++t) {
-      const int v = s_scan[t];
-      s_scan[t] = run;
-      run += v;
-    }
-  }
+  if (tid < 32) warp0_exclusive_scan(s_scan, nt);
   __syncthreads();
   int eqrank = s_scan[tid];
   for (int s = lo; s < hi; ++s) {
@@ -1080,6 +1157,7 @@ __device__ __forceinline__ void radix_select_top(KeyF&& KEY, int N, int K, unsig
 // retrieval head; kTopkVote then ranks a layer's units by the tally of the ballots of the layers up to it before
 // their own scores and goes on like kTopkSelect.
 enum { kTopkSelect = 0, kTopkBallot = 1, kTopkVote = 2 };
+constexpr int kTopkSelRegs = 24;  // scores of up to 12K spans (512 threads) are read from global memory once
 
 template <bool DECODE>
 __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin, DecBatch b, int layer_count,
@@ -1159,9 +1237,9 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
     for (int t = tid; t < K; t += nt) s_ids[t] = t;
     if (tid == 0) s_cnt = K;
   } else if (mode == kTopkVote) {
-    radix_select_top<unsigned long long>(KEY64, N, K, hist, &s_prefix64, &s_need, s_scan, &s_cnt, s_ids);
+    radix_select_top<unsigned long long, 0>(KEY64, N, K, hist, &s_prefix64, &s_need, s_scan, &s_cnt, s_ids);
   } else {
-    radix_select_top<unsigned>(KEY, N, K, hist, &s_prefix, &s_need, s_scan, &s_cnt, s_ids);
+    radix_select_top<unsigned, kTopkSelRegs>(KEY, N, K, hist, &s_prefix, &s_need, s_scan, &s_cnt, s_ids);
   }
   __syncthreads();
   const int cnt = min(s_cnt, K);
@@ -1576,67 +1654,8 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     for (int t = tid; t < K; t += nt) s_ids[t] = t;
     if (tid == 0) s_cnt = K;
   } else {
-    if (tid == 0) {
-      s_prefix = 0;
-      s_need = K;
-    }
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      if (tid < 256) hist[tid] = 0;
-      __syncthreads();
-      const unsigned prefix = s_prefix;
-      const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-      for (int s = tid; s < N; s += nt) {
-        const unsigned key = order_key(ssc[s]);
-        if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-      }
-      __syncthreads();
-      if (tid < 32) {
-        unsigned need = s_need;
-        const int bin = pick_from_top(hist, 256, need);
-        if (tid == 0) {
-          s_need = need;
-          s_prefix = prefix | ((unsigned)bin << shift);
-        }
-      }
-      __syncthreads();
-    }
-    const unsigned T = s_prefix;
-    const unsigned need_eq = s_need;
-    const int per = (N + nt - 1) / nt;
-    const int lo = tid * per, hi = min(N, lo + per);
-    int eq = 0;
-    for (int s = lo; s < hi; ++s) eq += order_key(ssc[s]) == T;
-    s_scan[tid] = eq;
-    __syncthreads();
-    if (tid < 32) {  // exclusive scan of 1024 counts by one warp
-      int run = 0;
-      for (int blk = 0; blk < nt; blk += 32) {
-        const int v = s_scan[blk + tid];
-        int inc = v;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int t = __shfl_up_sync(0xffffffffu, inc, o);
-          if (tid >= o) inc += t;
-        }
-        s_scan[blk + tid] = run + inc - v;
-        run += __shfl_sync(0xffffffffu, inc, 31);
-      }
-    }
-    __syncthreads();
-    int eqrank = s_scan[tid];
-    for (int s = lo; s < hi; ++s) {
-      const unsigned key = order_key(ssc[s]);
-      bool take = key > T;
-      if (key == T) {
-        take = (unsigned)eqrank < need_eq;
-        ++eqrank;
-      }
-      if (take) {
-        const int slot = atomicAdd(&s_cnt, 1);
-        if (slot < kMaxTopK) s_ids[slot] = s;
-      }
-    }
+    radix_select_top<unsigned, 0>([&](int i) { return order_key(ssc[i]); }, N, K, hist, &s_prefix, &s_need, s_scan,
+                                  &s_cnt, s_ids);
   }
   __syncthreads();
   const int cnt = min(s_cnt, K);
@@ -1798,10 +1817,12 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
       __syncthreads();
       const unsigned prefix = s_prefix;
       const unsigned himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      DigitRuns dr;
       for (int s = tid; s < nloc; s += nt) {
         const unsigned key = order_key(ssc[s]);
-        if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        if ((key & himask) == prefix) dr.add(hist, (int)((key >> shift) & 255u));
       }
+      dr.flush(hist);
       cluster.sync();
       if (tid < 256) {
         unsigned sum = 0;
@@ -1828,14 +1849,9 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
     for (int s = tlo; s < thi; ++s) eq += order_key(ssc[s]) == T;
     s_scan[tid] = eq;
     __syncthreads();
-    if (tid == 0) {
-      int run = 0;
-      for (int t = 0; t < nt; ++t) {
-        const int v = s_scan[t];
-        s_scan[t] = run;
-        run += v;
-      }
-      s_eq = run;
+    if (tid < 32) {
+      const int run = warp0_exclusive_scan(s_scan, nt);
+      if (tid == 0) s_eq = run;
     }
     cluster.sync();
     int eqrank = s_scan[tid];
