@@ -54,8 +54,8 @@ __global__ void __launch_bounds__(kMapThreads, 1)
     k_map_tc(DevCtx c, PrefillArgs a, int n_local_groups, int n_local_tiles, int n_cur_tiles,
              const __grid_constant__ MapMaps maps) {
   extern __shared__ unsigned char smem_raw[];
-  // KFULL | QFULL[2] QEMPTY[2] | SFULL[4] SEMPTY[4]
-  __shared__ __align__(8) unsigned long long bars[1 + 4 + 8];
+  // KFULL[4] | QFULL[2] QEMPTY[2] | SFULL[4] SEMPTY[4]
+  __shared__ __align__(8) unsigned long long bars[4 + 4 + 8];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
   constexpr int TPB = 128 / G;  // tokens per query block
@@ -90,17 +90,17 @@ __global__ void __launch_bounds__(kMapThreads, 1)
   const uint32_t sXa = sQ + 65536;                // 4 KB
   const uint32_t sXb = sXa + 4096;                // 2 stages x 4 KB
   auto xoff = [](int r, int kc) -> uint32_t { return (uint32_t)((r >> 3) * 256 + kc * 128 + (r & 7) * 16); };
-  enum { B_KFULL = 0, B_QFULL = 1, B_QEMPTY = 3, B_SFULL = 5, B_SEMPTY = 9 };
+  enum { B_KFULL = 0, B_QFULL = 4, B_QEMPTY = 6, B_SFULL = 8, B_SEMPTY = 12 };
   auto bar = [&](int i) { return smem_addr(&bars[i]); };
   volatile int* abortp = &s_abort;
   if (tid == 0) {
     s_abort = 0;
-    mbar_init(bar(B_KFULL), 1);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(bar(B_QFULL + s), 1);
+      mbar_init(bar(B_QFULL + s), 2);  // the copies of a block's queries (with their byte count), then its offsets
       mbar_init(bar(B_QEMPTY + s), 1);
     }
     for (int s = 0; s < 4; ++s) {
+      mbar_init(bar(B_KFULL + s), 1);
       mbar_init(bar(B_SFULL + s), 1);
       mbar_init(bar(B_SEMPTY + s), 16);
     }
@@ -124,17 +124,19 @@ __global__ void __launch_bounds__(kMapThreads, 1)
   chain_wait();  // everything above set up shared memory, barriers and TMEM only
 
   if (warp == 16) {
-    if (lane == 0) {
-      mbar_expect_tx(bar(B_KFULL), (uint32_t)ntile * 32768u);
-      for (int kt = 0; kt < ntile; ++kt) {
-        // (local and current keys: window rows of the slab)
-        const long long krow = (long long)(unit * c.Hkv + g) * c.SR + key0_of(kt) - (c.paged ? a.shift : 0);
-        tma_load_2d(sK + kt * 32768, &maps.k128, 0, (int)krow, bar(B_KFULL));
-        tma_load_2d(sK + kt * 32768 + 16384, &maps.k128, 64, (int)krow, bar(B_KFULL));
-      }
-    }
-    // every lane writes the offsets of four of the block's 128 rows (row = (token, head)); lane 0 then starts the
-    // copies of the block's queries, whose barrier also publishes the offsets
+    // Every key tile has its own barrier, and the first one is asked for before anything else, the others behind the
+    // first query block: the first product starts as soon as one tile and one block have landed.
+    auto load_keys = [&](int kt) {
+      // (local and current keys: window rows of the slab)
+      const long long krow = (long long)(unit * c.Hkv + g) * c.SR + key0_of(kt) - (c.paged ? a.shift : 0);
+      mbar_expect_tx(bar(B_KFULL + kt), 32768u);
+      tma_load_2d(sK + kt * 32768, &maps.k128, 0, (int)krow, bar(B_KFULL + kt));
+      tma_load_2d(sK + kt * 32768 + 16384, &maps.k128, 64, (int)krow, bar(B_KFULL + kt));
+    };
+    if (lane == 0) load_keys(0);
+    // lane 0 starts the copies of a block's queries (and, behind the first block's, of the other key tiles); then
+    // every lane writes the offsets of four of the block's 128 rows (row = (token, head)) and lane 0 publishes them
+    // with the second arrival on the block's barrier
     const float* rq = c.rowq + (size_t)layer * c.chunk * c.Hq + g * G;
     const float inv_c2 = 1.0f / (c.scale * kLog2eM);
     int ok = 1;
@@ -144,6 +146,13 @@ __global__ void __launch_bounds__(kMapThreads, 1)
       if (lane == 0 && it >= 2) ok = mbar_wait(bar(B_QEMPTY + st), ((it >> 1) - 1) & 1, abortp, c.wait_limit) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
+      if (lane == 0) {
+        mbar_expect_tx(bar(B_QFULL + st), 32768);
+        tma_load_3d(sQ + st * 32768, &maps.q, 0, g * G, l * a.n + blk * TPB, bar(B_QFULL + st));
+        tma_load_3d(sQ + st * 32768 + 16384, &maps.q, 64, g * G, l * a.n + blk * TPB, bar(B_QFULL + st));
+        if (it == 0)
+          for (int kt = 1; kt < ntile; ++kt) load_keys(kt);
+      }
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int row = lane + 32 * i;
@@ -170,11 +179,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
       }
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) {
-        mbar_expect_tx(bar(B_QFULL + st), 32768);
-        tma_load_3d(sQ + st * 32768, &maps.q, 0, g * G, l * a.n + blk * TPB, bar(B_QFULL + st));
-        tma_load_3d(sQ + st * 32768 + 16384, &maps.q, 64, g * G, l * a.n + blk * TPB, bar(B_QFULL + st));
-      }
+      if (lane == 0) mbar_arrive(bar(B_QFULL + st));
     }
     if (lane == 0)
       for (int back = 1; back <= 2 && back <= it; ++back) {  // no copy may be in flight at exit
@@ -186,7 +191,7 @@ __global__ void __launch_bounds__(kMapThreads, 1)
       constexpr uint32_t idesc = make_idesc(128, 128, false);
       const uint64_t dK = make_desc(sK, 16, 1024), dQ = make_desc(sQ, 16, 1024);
       const uint64_t dXa = make_desc_noswizzle(sXa, 128, 256), dXb = make_desc_noswizzle(sXb, 128, 256);
-      bool ok = mbar_wait(bar(B_KFULL), 0, abortp, c.wait_limit);
+      bool ok = true;
       int it = 0, seq = 0;
       for (int blk = bmin; ok && blk < nblocks; ++blk, ++it) {
         const int st = it & 1;
@@ -195,6 +200,9 @@ __global__ void __launch_bounds__(kMapThreads, 1)
         const uint64_t db = dQ + (uint64_t)((st * 32768) >> 4);
         for (int kt = 0; ok && kt < ntile; ++kt) {
           if (blk < blk0_of(kt)) continue;
+          // the first product on a tile waits for the tile
+          if (blk == max(bmin, blk0_of(kt))) ok = mbar_wait(bar(B_KFULL + kt), 0, abortp, c.wait_limit);
+          if (!ok) break;
           const int buf = seq & 3;
           if (seq >= 4) ok = mbar_wait(bar(B_SEMPTY + buf), ((seq >> 2) - 1) & 1, abortp, c.wait_limit);
           if (!ok) break;
