@@ -146,6 +146,48 @@ def test_retrieval_and_attention_from_a_loaded_span_index(unit_tokens):
     print(sp.rep)
 
 
+@pytest.mark.parametrize("fused", ["0", "1", "2"])
+def test_equal_scores_at_the_cut_go_to_the_lower_span(fused, monkeypatch):
+    # Eq. 8 with ties: the loaded index holds only three distinct vectors per KV head (span s gets vector s mod 3),
+    # so the scores of a call take three values among the loaded spans and the top-k cut falls inside a group of
+    # exactly equal scores; the picks among them must be the lowest span ids, in the prefill retriever and in each
+    # of the three decode retrieval paths.  The harness tolerates a different pick among near-equal scores and
+    # counts it: here the count must stay zero.
+    monkeypatch.setenv("LTRI_DEC_FUSED", fused)
+    cfg = small_cfg(n_layers=2, context=1536, decode_steps=3, top_k=5)
+    sp = ph.StreamPair(cfg, [0, 1])
+    st = inputs.SyntheticStream(cfg)
+    rng = np.random.default_rng(11)
+    t0, ties_at_cut = 0, 0
+    for ci, n in enumerate([128] * 12):
+        q, k, v = st.tokens(t0, n)
+        sp.prefill(0, q, k, v)
+        t0 += n
+        if ci > 8:    # how often the cut really fell inside a group of equal scores
+            for layer in (0, 1):
+                o = sp.orc[(0, layer)]
+                sel_o, sc = o.selected()[0], o.scores()
+                for g in range(cfg.n_kv_heads):
+                    picked = [int(x) for x in sel_o[g] if x >= 0]
+                    cut = min(sc[g][i] for i in picked)
+                    ties_at_cut += sum(1 for i in range(len(sc[g])) if sc[g][i] == cut) > sum(1 for i in picked if sc[g][i] == cut)
+        if ci == 8:
+            for layer in (0, 1):
+                o = sp.orc[(0, layer)]
+                spans = np.asarray(o.spans(), dtype=np.int32)
+                assert len(spans) >= 8
+                pool = inputs.bf16_bits(torch.from_numpy(rng.standard_normal((3, cfg.n_kv_heads, 128))).to(torch.bfloat16))
+                idx = np.stack([pool[s % 3] for s in range(len(spans))])
+                o.replace_index(spans, idx)
+                sp.lt.ltri_debug_load_index(0, layer, o.evicted_end, spans, idx.transpose(1, 0, 2))
+    for s in range(cfg.decode_steps):
+        sp.decode([0], *_decode_inputs(st, cfg.context + s))
+    assert ties_at_cut > 0
+    assert sp.rep.sel_checks >= 16 and sp.rep.sel_flips == 0, sp.rep
+    sp.lt.close()
+    print(sp.rep)
+
+
 def test_host_entry_with_calls_of_different_sizes_and_layer_ranges():
     # the host-buffer entry pipelines layer groups over staging slices that calls reuse: a short call followed by
     # full ones, and calls over part of the layers, must give what the device entry gives, bit for bit
