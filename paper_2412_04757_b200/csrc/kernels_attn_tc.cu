@@ -551,12 +551,26 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           const int ctok = td.causal_tok0;
           const int lim = ctok >= 0 ? row_abs - ctok - half * 64 : 127;
           const uint2 mks = *reinterpret_cast<const uint2*>(&td.m0 + half * 2);
+          if (MERGE) {
+            // (the form that measured faster in this instantiation; the other one in the other)
+            // one bit per column: the slot holds a key and the key is visible to this row
+            const unsigned vis0 = lim >= 31 ? 0xffffffffu : (lim < 0 ? 0u : (2u << lim) - 1u);
+            const unsigned vis1 = lim >= 63 ? 0xffffffffu : (lim < 32 ? 0u : (2u << (lim - 32)) - 1u);
 #pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
-            const unsigned mk = ch == 0 ? mks.x : mks.y;
+            for (int ch = 0; ch < 2; ++ch) {
+              const unsigned mk = ch == 0 ? (mks.x & vis0) : (mks.y & vis1);
 #pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (!((mk >> e) & 1u) || ch * 32 + e > lim) v[ch][e] = 0xff800000u;  // -inf
+              for (int e = 0; e < 32; ++e)
+                if (!((mk >> e) & 1u)) v[ch][e] = 0xff800000u;  // -inf
+            }
+          } else {
+#pragma unroll
+            for (int ch = 0; ch < 2; ++ch) {
+              const unsigned mk = ch == 0 ? mks.x : mks.y;
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (!((mk >> e) & 1u) || ch * 32 + e > lim) v[ch][e] = 0xff800000u;  // -inf
+            }
           }
         }
         // maximum of this thread's 64 logits (four independent chains)
