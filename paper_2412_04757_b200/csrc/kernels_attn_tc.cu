@@ -162,8 +162,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   }
   const CUtensorMap* kvmaps = maps.kv;
   extern __shared__ unsigned char smem_raw[];
-  // QFULL QFREE ODONE | KFULL[2] VFULL[2] KEMPTY[2] VEMPTY[2] | SREADY[2] PREADY[2][2] OFREE[2]
-  __shared__ __align__(8) unsigned long long bars[3 + 8 + 8];
+  // QFULL QFREE ODONE[0] | KFULL[2] VFULL[2] KEMPTY[2] VEMPTY[2] | SREADY[2] PREADY[2][2] OFREE[2] | ODONE[1]
+  __shared__ __align__(8) unsigned long long bars[3 + 8 + 8 + 1];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
   __shared__ RangeList rg;            // key ranges of the work item the producer is walking
@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   enum {
     B_QFULL = 0, B_QFREE = 1, B_ODONE = 2, B_KFULL = 3, B_VFULL = 5, B_KEMPTY = 7, B_VEMPTY = 9, B_SREADY = 11,
     B_PREADY = 13,  // + 2 * part + q: the two 32-column chunks of a thread's probabilities are handed over separately
-    B_OFREE = 17
+    B_OFREE = 17, B_ODONE1 = 19
   };
   auto bar = [&](int i) { return smem_addr(&bars[i]); };
   volatile int* abortp = &s_abort;
@@ -199,6 +199,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QFREE), 1);
     mbar_init(bar(B_ODONE), 1);
+    mbar_init(bar(B_ODONE1), 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(B_KFULL + s), 1);
       mbar_init(bar(B_VFULL + s), 1);
@@ -385,21 +386,35 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       };
       int jt = 0;
       bool ok = true;
+      // Across work items the two Q tiles stay half a tile apart: when the last P.V product of Q tile 0 has been
+      // issued, the first QK^T product of the NEXT item's Q tile 0 follows at once if that item's queries and first
+      // key tile have landed (pre = true), so Q tile 0's logits are ready when its softmax threads come back from
+      // their epilogue, and the tensor pipe has work while Q tile 1 finishes the current item.  Each Q tile has its
+      // own "accumulator complete" barrier for the same reason.
+      bool pre = false;
+      int T_pre = 0;
       for (int item = blockIdx.x, wi = 0; ok && item < nitems; item += gridDim.x, ++wi) {
-        ok = mbar_wait(bar(B_QFULL), wi & 1, abortp, c.wait_limit);
-        if (!ok) break;
-        const int T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
-        if (T > 0) {
-          ok = mbar_wait(bar(B_KFULL + (jt & 1)), (jt >> 1) & 1, abortp, c.wait_limit);
+        int T = T_pre;
+        if (!pre) {
+          ok = mbar_wait(bar(B_QFULL), wi & 1, abortp, c.wait_limit);
           if (!ok) break;
-          fence_after_sync();
-          issue_qk(0, jt & 1);
+          T = *reinterpret_cast<volatile int*>(&s_item_tiles[wi % 3]);
+        }
+        if (T > 0) {
+          if (!pre) {
+            ok = mbar_wait(bar(B_KFULL + (jt & 1)), (jt >> 1) & 1, abortp, c.wait_limit);
+            if (!ok) break;
+            fence_after_sync();
+            issue_qk(0, jt & 1);
+          }
           issue_qk(1, jt & 1);
           mma_commit(bar(B_KEMPTY + (jt & 1)));
           if (T == 1) mma_commit(bar(B_QFREE));
         } else {
           mma_commit(bar(B_QFREE));
         }
+        pre = false;
+        const bool has_next = item + (int)gridDim.x < nitems;
         for (int j = 0; ok && j < T; ++j, ++jt) {
           const int st = jt & 1, nst = st ^ 1;
           const bool acc = (j > 0) || (phase == 1);
@@ -409,7 +424,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           if (!ok) break;
           // the first P.V product of an item overwrites O: the previous item's epilogue must have read it
           if (j == 0 && wi > 0) {
-            ok = mbar_wait(bar(B_OFREE + 0), (wi - 1) & 1, abortp, c.wait_limit) && mbar_wait(bar(B_OFREE + 1), (wi - 1) & 1, abortp, c.wait_limit);
+            ok = mbar_wait(bar(B_OFREE + 0), (wi - 1) & 1, abortp, c.wait_limit);
             if (!ok) break;
           }
           fence_after_sync();
@@ -423,9 +438,24 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             if (!ok) break;
             fence_after_sync();
             issue_qk(0, nst);
+          } else {
+            mma_commit(bar(B_ODONE));
+            if (has_next && mbar_try(bar(B_QFULL), (wi + 1) & 1)) {
+              const int Tn = *reinterpret_cast<volatile int*>(&s_item_tiles[(wi + 1) % 3]);
+              if (Tn > 0 && mbar_try(bar(B_KFULL + nst), ((jt + 1) >> 1) & 1)) {
+                fence_after_sync();
+                issue_qk(0, nst);
+                pre = true;
+                T_pre = Tn;
+              }
+            }
           }
           ok = mbar_wait(bar(B_PREADY + 1), jt & 1, abortp, c.wait_limit);
           if (!ok) break;
+          if (j == 0 && wi > 0) {
+            ok = mbar_wait(bar(B_OFREE + 1), (wi - 1) & 1, abortp, c.wait_limit);
+            if (!ok) break;
+          }
           fence_after_sync();
           issue_pv(1, st, acc, 0);
           ok = mbar_wait(bar(B_PREADY + 3), jt & 1, abortp, c.wait_limit);
@@ -440,7 +470,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           }
         }
         if (!ok) break;
-        mma_commit(bar(B_ODONE));
+        if (T == 0) mma_commit(bar(B_ODONE));
+        mma_commit(bar(B_ODONE1));
       }
     }
   } else {
@@ -655,7 +686,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       s_sum[q][half][r] = lsum;
       asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");
       lsum += s_sum[q][half ^ 1][r];
-      if (ok) ok = mbar_wait(bar(B_ODONE), wi & 1, abortp, c.wait_limit);
+      if (ok) ok = mbar_wait(bar(q ? B_ODONE1 : B_ODONE), wi & 1, abortp, c.wait_limit);
       if (!ok) s_quit[q] = 1;
       asm volatile("bar.sync %0, 256;" ::"r"(1 + q) : "memory");  // also: s_sum is reused by the next item
       if (s_quit[q]) break;  // collective decision: all 256 threads of the tile leave after the same item
