@@ -256,7 +256,7 @@ def workload_config(cfg, world, nseq):
 # scaled to the launch this run times (traffic grows in proportion to these units):
 #  * local attention (k_attn_tc phase 0), Llama-3-8B geometry, chunk 512, window 4096 full, sink 64: DRAM read +
 #    write of one launch over 4 layers at 16K context -> bytes per layer of a launch
-ATTN_LOCAL_DRAM_BYTES_PER_LAYER = {(32, 8, 512, 4096, 64): (94.41e6 + 7.35e6) / 4}
+ATTN_LOCAL_DRAM_BYTES_PER_LAYER = {(32, 8, 512, 4096, 64): (94.40e6 + 7.24e6) / 4}
 #  * decode retrieval + attention: 239.7 MB measured against 237.8 MB of algorithmic bytes for an 8-layer step at
 #    64K: every byte is read once, nothing is re-read
 DECODE_DRAM_PER_ALGORITHMIC_BYTE = 239.7 / 237.8
