@@ -160,7 +160,7 @@ struct PrefillArgs {
 
 // ---- launch wrappers (each returns the cudaError_t of the launch) -------------------
 cudaError_t launch_init(const DevCtx& c, int seq /* -1: all */, cudaStream_t s);
-cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s);
+cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, bool clear_maps, cudaStream_t s);
 cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
                                  const __nv_bfloat16* k, const __nv_bfloat16* v, cudaStream_t s);
 cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_count, cudaStream_t s);

@@ -370,10 +370,8 @@ static cudaError_t launch_map_tc_g(const DevCtx& c, const PrefillArgs& a, const 
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
-  // the region map is accumulated with integer reductions: clear it first
-  cudaError_t e = cudaMemsetAsync(c.Mq + (size_t)a.layer_begin * c.chunk * c.chunk, 0,
-                                  (size_t)a.layer_count * c.chunk * c.chunk * sizeof(int), s);
-  if (e != cudaSuccess) return e;
+  // (the region maps, which the kernel accumulates into with integer reductions, were cleared by the call's append
+  // kernel)
   const int nloc = (a.loc_begin >= c.Ls) ? (a.t0 - a.loc_begin + 127) / 128 : 0;
   const int ncur = (a.n + 127) / 128;
   const int gloc = (nloc + kMapKT - 1) / kMapKT, gcur = (ncur + kMapKT - 1) / kMapKT;

@@ -48,14 +48,22 @@ cudaError_t launch_init(const DevCtx& c, int seq, cudaStream_t s) {
 
 
 // ------------------------------------------------------------------------------------------
-// a0: copy the call's K/V rows into the cache slabs; 16 threads move one 256-byte row.
-__global__ void k_append_prefill(DevCtx c, PrefillArgs a) {
+// a0: copy the call's K/V rows into the cache slabs; 16 threads move one 256-byte row.  The threads behind the copy
+// (zero_vec of them, 16 bytes each) clear the region maps of the call's layers, which the tensor-core map pass
+// accumulates into with integer reductions: nothing reads a layer's map between the segmenter of the layer's previous
+// call and that pass, so clearing it here, in the first kernel of the call, keeps a memset out of the kernel chain.
+__global__ void k_append_prefill(DevCtx c, PrefillArgs a, unsigned long long zero_vec) {
   chain_wait();
   const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int c16 = gid & 15;
   size_t row = gid >> 4;  // over [layer_count][n][Hkv]
   const size_t nrows = (size_t)a.layer_count * a.n * c.Hkv;
-  if (row >= nrows) return;
+  if (row >= nrows) {
+    const size_t zi = gid - nrows * 16;
+    if (zi < zero_vec)
+      reinterpret_cast<uint4*>(c.Mq + (size_t)a.layer_begin * c.chunk * c.chunk)[zi] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
   const int g = row % c.Hkv;
   const int r = (row / c.Hkv) % a.n;
   const int l = row / ((size_t)c.Hkv * a.n);
@@ -79,9 +87,10 @@ __global__ void k_append_prefill(DevCtx c, PrefillArgs a) {
   if (g == 0 && c16 == 0) c.votes[unit * c.Tpad + a.t0 + r] = 0;
 }
 
-cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, cudaStream_t s) {
-  const size_t threads = (size_t)a.layer_count * a.n * c.Hkv * 16;
-  return launch_chained(k_append_prefill, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, s, c, a);
+cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, bool clear_maps, cudaStream_t s) {
+  const unsigned long long zero_vec = clear_maps ? (unsigned long long)a.layer_count * c.chunk * c.chunk / 4 : 0ull;
+  const size_t threads = (size_t)a.layer_count * a.n * c.Hkv * 16 + zero_vec;
+  return launch_chained(k_append_prefill, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, s, c, a, zero_vec);
 }
 
 __global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer_count,

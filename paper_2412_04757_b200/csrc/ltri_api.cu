@@ -653,7 +653,7 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   a.shift = shift;
   {
     Scope sc(ctx, st, LTRI_K_APPEND, 1);
-    LTRI_CUDA(ctx, launch_append_prefill(d, a, st));
+    LTRI_CUDA(ctx, launch_append_prefill(d, a, /*clear_maps=*/ctx->use_tc, st));
   }
   for (size_t i = 0; i < ev.size(); i += 8) {
     Scope sc(ctx, st, LTRI_K_EVICT, 1);
