@@ -1095,7 +1095,20 @@ __device__ __forceinline__ void radix_select_top(KeyF&& KEY, int N, int K, unsig
         if (s < N) f(s, (KT)kr[i]);
       }
     } else {
-      for (int s = tid; s < N; s += nt) f(s, KEY(s));
+      // eight keys in flight per thread (KEY may be a load from global memory)
+      for (int base = tid; base < N; base += 8 * nt) {
+        KT k8[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int s = base + u * nt;
+          k8[u] = s < N ? (KT)KEY(s) : (KT)0;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int s = base + u * nt;
+          if (s < N) f(s, k8[u]);
+        }
+      }
     }
   };
   if (tid == 0) {
