@@ -1581,6 +1581,7 @@ cudaError_t launch_pull_pack(const DevCtx& c, const PrefillArgs& a, cudaStream_t
 // (half-warp per 256-byte row, 16 bytes per lane, four rows in flight), keeps the scores in shared memory, selects the
 // top-k there (same radix select as k_topk) and writes the selection and the token ranges of the attention kernel.
 constexpr int kFusedMaxSpans = 12288;  // scores kept in shared memory (48 KB)
+constexpr int kDecSelRegs = 16;        // keys per thread the select holds in registers (8K spans at 512 threads)
 
 // a0 inside the one-launch decode retrieval: the CTA of (sequence, layer, KV head) also stores that head's new K and V
 // row (threads 0-31: sixteen 16-byte pieces each), so a decode step needs no separate append launch.  The attention
@@ -1603,7 +1604,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
                                                        const __nv_bfloat16* __restrict__ knew,
                                                        const __nv_bfloat16* __restrict__ vnew) {
   chain_wait();
-  extern __shared__ float ssc[];  // [N]
+  extern __shared__ unsigned sck[];  // [N] order-preserving keys of the scores
   __shared__ float su[kD];
   __shared__ unsigned hist[256];
   __shared__ unsigned s_prefix, s_need;
@@ -1620,6 +1621,20 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   const int N = min(c.n_spans[unit], kFusedMaxSpans);
   const int rh = ret_head_of(c, layer), gk = rh >= 0 ? rh / c.G : g;  // retrieval head of the layer (Sec. 3.5)
   append_decode_row(c, b, bi, l, layer_count, unit, g, knew, vnew);
+  // ---- scores.  The first four index rows of every half-warp are requested before the query sum below is formed,
+  // so that their latency and that of the query loads pass together.
+  const int hw = tid >> 4, hl = tid & 15, nhw = nt >> 4;  // half-warps of the CTA (the launch picks its size)
+  const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + gk) * (size_t)c.cap * kD + hl * 8;
+  // software pipeline: the next four rows are in flight while the current four are reduced
+  auto fetch = [&](int base, uint4 (&raw)[4]) {
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const int s = base + t * nhw + hw;
+      raw[t] = s < N ? __ldg(reinterpret_cast<const uint4*>(KR + (size_t)s * kD)) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  uint4 cur[4], nxt[4];
+  fetch(0, cur);
   if (tid < kD) {
     const __nv_bfloat16* qp = q + (((size_t)b.src[bi] * layer_count + l) * c.Hq + gk * c.G) * kD + tid;
     float acc = 0.f;
@@ -1629,23 +1644,10 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
   }
   if (tid == 0) s_cnt = 0;
   __syncthreads();
-  // ---- scores
   {
-    const int hw = tid >> 4, hl = tid & 15, nhw = nt >> 4;  // half-warps of the CTA (the launch picks its size)
     float uf[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) uf[e] = su[hl * 8 + e];
-    const __nv_bfloat16* KR = c.KR + (unit * c.Hkv + gk) * (size_t)c.cap * kD + hl * 8;
-    // software pipeline: the next four rows are in flight while the current four are reduced
-    auto fetch = [&](int base, uint4 (&raw)[4]) {
-#pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        const int s = base + t * nhw + hw;
-        raw[t] = s < N ? __ldg(reinterpret_cast<const uint4*>(KR + (size_t)s * kD)) : make_uint4(0, 0, 0, 0);
-      }
-    };
-    uint4 cur[4], nxt[4];
-    fetch(0, cur);
     for (int base = 0; base < N; base += nhw * 4) {  // uniform trip count (shuffles inside)
       fetch(base + nhw * 4, nxt);                    // past the end: zeros, no loads
 #pragma unroll
@@ -1663,7 +1665,7 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
         d += __shfl_xor_sync(0xffffffffu, d, 4);
         d += __shfl_xor_sync(0xffffffffu, d, 8);
         const int s = base + t * nhw + hw;
-        if (hl == 0 && s < N) ssc[s] = d;
+        if (hl == 0 && s < N) sck[s] = order_key(d);
       }
 #pragma unroll
       for (int t = 0; t < 4; ++t) cur[t] = nxt[t];
@@ -1676,8 +1678,8 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     for (int t = tid; t < K; t += nt) s_ids[t] = t;
     if (tid == 0) s_cnt = K;
   } else {
-    radix_select_top<unsigned, 0>([&](int i) { return order_key(ssc[i]); }, N, K, hist, &s_prefix, &s_need, s_scan,
-                                  &s_cnt, s_ids);
+    radix_select_top<unsigned, kDecSelRegs>([&](int i) { return sck[i]; }, N, K, hist, &s_prefix, &s_need, s_scan,
+                                            &s_cnt, s_ids);
   }
   __syncthreads();
   const int cnt = min(s_cnt, K);
