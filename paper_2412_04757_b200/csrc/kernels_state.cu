@@ -1580,6 +1580,49 @@ cudaError_t launch_pull_pack(const DevCtx& c, const PrefillArgs& a, cudaStream_t
 // Decode retrieval in one launch: a CTA owns one (sequence, layer, KV head), streams that head's index once
 // (half-warp per 256-byte row, 16 bytes per lane, four rows in flight), keeps the scores in shared memory, selects the
 // top-k there (same radix select as k_topk) and writes the selection and the token ranges of the attention kernel.
+// Token ranges of the attention kernels from M items (start, length) in ascending order of start: items of length
+// zero are dropped, an item that starts at or before the end of what came before it (adjacent spans, or overlapping
+// ones under NMS with phi > 0) extends the current range.  One warp, 32 items per round: an item opens a range iff it
+// starts beyond the largest end seen so far (a prefix maximum), its range number is the count of such items up to
+// it, and a range's end is the prefix maximum in front of the next opener.  Returns the number of ranges; s_rs / s_rl
+// receive their starts and lengths.  Called by all 32 lanes of one warp.
+template <typename ItemF>
+__device__ __forceinline__ int merge_ranges_warp(int M, ItemF&& item, int* s_rs, int* s_rl) {
+  const int lane = threadIdx.x & 31;
+  constexpr int kNone = -0x7fffffff;
+  int far = kNone, nr = 0;  // largest end so far, ranges so far
+  for (int base = 0; base < M; base += 32) {
+    const int i = base + lane;
+    int st = 0, ln = 0;
+    if (i < M) item(i, st, ln);
+    const bool valid = i < M && ln > 0;
+    const int en = valid ? st + ln : kNone;
+    int inc = en;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc = max(inc, t);
+    }
+    int before = __shfl_up_sync(0xffffffffu, inc, 1);
+    if (lane == 0) before = kNone;
+    before = max(before, far);
+    const bool opens = valid && st > before;
+    const unsigned ob = __ballot_sync(0xffffffffu, opens);
+    if (opens) {
+      const int idx = nr + __popc(ob & ((2u << lane) - 1u)) - 1;
+      s_rs[idx] = st;
+      if (idx > 0) s_rl[idx - 1] = before;  // (the end of the range before it; turned into a length below)
+    }
+    far = max(far, __shfl_sync(0xffffffffu, inc, 31));
+    nr += __popc(ob);
+  }
+  if (lane == 0 && nr > 0) s_rl[nr - 1] = far;
+  __syncwarp();
+  for (int r = lane; r < nr; r += 32) s_rl[r] -= s_rs[r];
+  __syncwarp();
+  return nr;
+}
+
 constexpr int kFusedMaxSpans = 12288;  // scores kept in shared memory (48 KB)
 constexpr int kDecSelRegs = 16;        // keys per thread the select holds in registers (8K spans at 512 threads)
 
@@ -1704,28 +1747,33 @@ __global__ void __launch_bounds__(1024) k_dec_retrieve(DevCtx c, int layer_begin
     s_sln[tid] = c.span_len[unit * c.cap + ids_all[tid]];
   }
   __syncthreads();
-  if (tid == 0) {
-    int nr = 0;
+  if (tid < 32) {
+    // items: the sink, the selected spans, the recent tokens
+    const int rb = min(loc_begin, pos + 1);
+    const int nr = merge_ranges_warp(
+        nall + 2,
+        [&](int i, int& st, int& ln) {
+          if (i == 0) {
+            st = 0;
+            ln = min(c.Ls, pos + 1);
+          } else if (i <= nall) {
+            st = s_sst[i - 1];
+            ln = s_sln[i - 1];
+          } else {
+            st = rb;
+            ln = pos + 1 - rb;
+          }
+        },
+        s_rs, s_rl);
     long long tokens = 0;
-    auto push = [&](int st, int ln) {
-      if (ln <= 0) return;
-      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] >= st)  // adjacent, or (NMS with phi > 0) overlapping: one range
-        s_rl[nr - 1] = max(s_rl[nr - 1], st + ln - s_rs[nr - 1]);
-      else {
-        s_rs[nr] = st;
-        s_rl[nr] = ln;
-        ++nr;
-      }
-    };
-    push(0, min(c.Ls, pos + 1));
-    for (int t = 0; t < nall; ++t) {
-      tokens += s_sln[t];
-      push(s_sst[t], s_sln[t]);
+    for (int t = tid; t < nall; t += 32) tokens += s_sln[t];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tokens += shfl_xor_ll(tokens, o);
+    if (tid == 0) {
+      s_nr = nr;
+      c.rng_cnt[unit * c.Hkv + g] = nr;
+      c.sel_tokens[unit * c.Hkv + g] = tokens;  // (summed over the KV heads by ltri_get_stats)
     }
-    push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
-    s_nr = nr;
-    c.rng_cnt[unit * c.Hkv + g] = nr;
-    c.sel_tokens[unit * c.Hkv + g] = tokens;  // (summed over the KV heads by ltri_get_stats)
   }
   __syncthreads();
   const size_t rbb = (unit * c.Hkv + g) * (size_t)c.rcap;
