@@ -1389,6 +1389,53 @@ __global__ void __launch_bounds__(512) k_topk(DevCtx c, int seq, int layer_begin
       }
     }
   }
+  if (!(DECODE && c.host_kv)) {
+    // (ranges in place, adjacent spans merged: one warp)
+    if (tid < 32) {
+      const int first = DECODE ? 1 : 0;  // decode: the sink in front of the spans, the recent tokens behind them
+      const int rbeg = DECODE ? min(loc_begin, pos + 1) : 0;
+      const int nr = merge_ranges_warp(
+          nall + 2 * first,
+          [&](int i, int& st, int& ln) {
+            if (i < first) {
+              st = 0;
+              ln = min(c.Ls, pos + 1);
+            } else if (i - first < nall) {
+              st = s_sst[i - first];
+              ln = s_sln[i - first];
+            } else {
+              st = rbeg;
+              ln = pos + 1 - rbeg;
+            }
+          },
+          s_rs, s_rl);
+      long long tokens = 0;
+      for (int t = tid; t < nall; t += 32) tokens += s_sln[t];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) tokens += shfl_xor_ll(tokens, o);
+      // packed-row prefix of the ranges
+      int run = 0;
+      for (int base = 0; base < nr; base += 32) {
+        const int i = base + tid;
+        const int v = i < nr ? s_rl[i] : 0;
+        int inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (tid >= o) inc += t;
+        }
+        if (i < nr) s_pre[i] = run + inc - v;
+        run += __shfl_sync(0xffffffffu, inc, 31);
+      }
+      if (tid == 0) {
+        s_pre[nr] = run;
+        s_nr = nr;
+        c.rng_cnt[unit * c.Hkv + g] = nr;
+        c.sel_tokens[unit * c.Hkv + g] = tokens;  // (summed over the KV heads by ltri_get_stats)
+        if (!DECODE) c.gcnt[(size_t)layer * c.Hkv + g] = run;
+      }
+    }
+  } else
   if (tid == 0) {
     int nr = 0;
     long long tokens = 0;
