@@ -188,6 +188,37 @@ def test_equal_scores_at_the_cut_go_to_the_lower_span(fused, monkeypatch):
     print(sp.rep)
 
 
+def test_hundreds_of_equal_scores_fall_back_to_the_radix_passes():
+    # Eq. 8 with a whole index of equal scores: every loaded span gets the same vector, so several hundred scores are
+    # exactly equal and the short cut of the select (which ranks at most 256 keys near the maximum against each
+    # other) has to hand over to the radix passes and their id-ordered tie pass; picks = the lowest span ids.
+    cfg = small_cfg(n_layers=1, context=12288, decode_steps=2, top_k=6, max_spans_per_region=8, seg_min=8, seg_max=24)
+    sp = ph.StreamPair(cfg, [0], deep=False)
+    st = inputs.SyntheticStream(cfg)
+    rng = np.random.default_rng(3)
+    chunks = list(st.prefill_chunks())
+    loaded = 0
+    for ci, (t0, n) in enumerate(chunks):
+        q, k, v = st.tokens(t0, n)
+        sp.prefill(0, q, k, v)
+        if ci == len(chunks) - 3:
+            o = sp.orc[(0, 0)]
+            spans = np.asarray(o.spans(), dtype=np.int32)
+            loaded = len(spans)
+            one = inputs.bf16_bits(torch.from_numpy(rng.standard_normal((1, cfg.n_kv_heads, 128))).to(torch.bfloat16))
+            idx = np.repeat(one, loaded, axis=0)
+            o.replace_index(spans, idx)
+            sp.lt.ltri_debug_load_index(0, 0, o.evicted_end, spans, idx.transpose(1, 0, 2))
+    assert loaded > 256 + 16, loaded      # more equal keys than the short cut ranks
+    for s in range(cfg.decode_steps):
+        sp.decode([0], *_decode_inputs(st, cfg.context + s))
+    assert sp.rep.sel_flips == 0, sp.rep
+    sel = sp.lt.ltri_get_selected(0, 0)
+    assert sel.shape[1] == cfg.top_k
+    sp.lt.close()
+    print(sp.rep)
+
+
 def test_host_entry_with_calls_of_different_sizes_and_layer_ranges():
     # the host-buffer entry pipelines layer groups over staging slices that calls reuse: a short call followed by
     # full ones, and calls over part of the layers, must give what the device entry gives, bit for bit
