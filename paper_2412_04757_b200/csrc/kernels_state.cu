@@ -1114,8 +1114,8 @@ __device__ __forceinline__ void radix_select_top(KeyF&& KEY, int N, int K, unsig
       }
     }
   };
-  if (R > 0 && inreg && nt >= 64 + kSelCand) {
-    // Short cut for register-held keys (K is small against N): with the block's largest key M known, one histogram
+  if (sizeof(KT) == 4 && s_ckey != nullptr && nt >= 64 + kSelCand) {
+    // Short cut for 32-bit keys (K is small against N): with the block's largest key M known, one histogram
     // of how far a key's upper 16 bits lie below M's (256 bins; further away: the last bin) gives the smallest
     // distance b within which at least K keys lie; those keys -- usually a few more than K -- are listed in shared
     // memory and ranked against each other (key, then lower index).  Four barriers instead of twelve and about a
