@@ -255,8 +255,9 @@ const char* ltri_strerror(int code);
 
 /* Kernel classes reported by ltri_profile_read. */
 enum {
-  LTRI_K_APPEND = 0,   /* K/V cache append */
-  LTRI_K_EVICT,        /* eviction + span index build (Eq. 6) */
+  LTRI_K_APPEND = 0,   /* K/V cache append of a call that evicts nothing (and of the two-launch decode path) */
+  LTRI_K_EVICT,        /* eviction + span index build (Eq. 6), together with the call's K/V cache append, which runs
+                          beside it */
   LTRI_K_ATTN_LOCAL,   /* prefill attention over sink | local | current */
   LTRI_K_MAP,          /* local-map pass: votes + region map (Eq. 4, Eq. 6) */
   LTRI_K_SEGMENT,      /* theta, cumulative sums, anti-diagonal filter, NMS, query representatives */

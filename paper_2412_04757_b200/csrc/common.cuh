@@ -143,6 +143,7 @@ struct EvictArgs {
   int nslots;
   int slot[8];
   long long shift;  // sliding slabs: token - shift = row
+  int release;      // let the kernel launched behind this one (the call's append kernel) start at once
 };
 
 struct PrefillArgs {
@@ -160,7 +161,7 @@ struct PrefillArgs {
 
 // ---- launch wrappers (each returns the cudaError_t of the launch) -------------------
 cudaError_t launch_init(const DevCtx& c, int seq /* -1: all */, cudaStream_t s);
-cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, bool clear_maps, cudaStream_t s);
+cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, bool clear_maps, bool late_wait, cudaStream_t s);
 cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_begin, int layer_count, int n_seqs_total,
                                  const __nv_bfloat16* k, const __nv_bfloat16* v, cudaStream_t s);
 cudaError_t launch_evict_index(const DevCtx& c, const EvictArgs& a, int layer_count, cudaStream_t s);
@@ -219,6 +220,11 @@ cudaError_t launch_wait_probe(const DevCtx& c, long long short_limit, cudaStream
 // instead of 0.225 ms per step).  Launched the ordinary way, chain_wait() does nothing.
 #ifdef __CUDACC__
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the kernel launched behind this one start now instead of when this grid has finished.  Used in one place only:
+// the eviction kernel (a few CTAs) releases the call's append kernel, which does not depend on it and whose threads
+// wait for the eviction kernel at their end instead of their beginning, so that the two run side by side and
+// everything behind the append kernel still follows both.
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,

@@ -52,8 +52,11 @@ cudaError_t launch_init(const DevCtx& c, int seq, cudaStream_t s) {
 // (zero_vec of them, 16 bytes each) clear the region maps of the call's layers, which the tensor-core map pass
 // accumulates into with integer reductions: nothing reads a layer's map between the segmenter of the layer's previous
 // call and that pass, so clearing it here, in the first kernel of the call, keeps a memset out of the kernel chain.
-__global__ void k_append_prefill(DevCtx c, PrefillArgs a, unsigned long long zero_vec) {
-  chain_wait();
+__global__ void k_append_prefill(DevCtx c, PrefillArgs a, unsigned long long zero_vec, int late_wait) {
+  // late_wait: the kernel in front of this one is the call's eviction kernel, which has released this one (see
+  // chain_release): everything older is complete and visible, the two kernels touch different data, and this one
+  // waits for the eviction kernel at its end (in its last CTA), so that whatever follows it follows both.
+  if (!late_wait) chain_wait();
   const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int c16 = gid & 15;
   size_t row = gid >> 4;  // over [layer_count][n][Hkv]
@@ -62,35 +65,40 @@ __global__ void k_append_prefill(DevCtx c, PrefillArgs a, unsigned long long zer
     const size_t zi = gid - nrows * 16;
     if (zi < zero_vec)
       reinterpret_cast<uint4*>(c.Mq + (size_t)a.layer_begin * c.chunk * c.chunk)[zi] = make_uint4(0u, 0u, 0u, 0u);
-    return;
+  } else {
+    const int g = row % c.Hkv;
+    const int r = (row / c.Hkv) % a.n;
+    const int l = row / ((size_t)c.Hkv * a.n);
+    const size_t unit = unit_of(c, a.seq, a.layer_begin + l);
+    const long long tok = a.t0 + r;
+    const long long wrow = c.paged ? tok - a.shift : tok;  // window row (a sink token has one too while it is current)
+    if (wrow < 0 || wrow >= c.SR) {                         // cannot happen: the host keeps the window inside the slab
+      set_status(c, -2, (int)tok);
+    } else {
+      const size_t dst = ((unit * c.Hkv + g) * c.SR + wrow) * kD + c16 * 8;
+      const size_t src = row * kD + c16 * 8;
+      const uint4 kv = *reinterpret_cast<const uint4*>(a.k + src), vv = *reinterpret_cast<const uint4*>(a.v + src);
+      *reinterpret_cast<uint4*>(c.Kc + dst) = kv;
+      *reinterpret_cast<uint4*>(c.Vc + dst) = vv;
+      if (c.paged && tok < c.Ls) {  // the sink's permanent rows
+        const size_t sd = ((unit * c.Hkv + g) * c.SR + tok) * kD + c16 * 8;
+        *reinterpret_cast<uint4*>(c.Kc + sd) = kv;
+        *reinterpret_cast<uint4*>(c.Vc + sd) = vv;
+      }
+      if (g == 0 && c16 == 0) c.votes[unit * c.Tpad + a.t0 + r] = 0;
+    }
   }
-  const int g = row % c.Hkv;
-  const int r = (row / c.Hkv) % a.n;
-  const int l = row / ((size_t)c.Hkv * a.n);
-  const size_t unit = unit_of(c, a.seq, a.layer_begin + l);
-  const long long tok = a.t0 + r;
-  const long long wrow = c.paged ? tok - a.shift : tok;  // window row (a sink token has one too while it is current)
-  if (wrow < 0 || wrow >= c.SR) {                         // cannot happen: the host keeps the window inside the slab
-    set_status(c, -2, (int)tok);
-    return;
-  }
-  const size_t dst = ((unit * c.Hkv + g) * c.SR + wrow) * kD + c16 * 8;
-  const size_t src = row * kD + c16 * 8;
-  const uint4 kv = *reinterpret_cast<const uint4*>(a.k + src), vv = *reinterpret_cast<const uint4*>(a.v + src);
-  *reinterpret_cast<uint4*>(c.Kc + dst) = kv;
-  *reinterpret_cast<uint4*>(c.Vc + dst) = vv;
-  if (c.paged && tok < c.Ls) {  // the sink's permanent rows
-    const size_t sd = ((unit * c.Hkv + g) * c.SR + tok) * kD + c16 * 8;
-    *reinterpret_cast<uint4*>(c.Kc + sd) = kv;
-    *reinterpret_cast<uint4*>(c.Vc + sd) = vv;
-  }
-  if (g == 0 && c16 == 0) c.votes[unit * c.Tpad + a.t0 + r] = 0;
+  // (only the last CTA waits: the grid is not complete before it is, and CTAs that sat waiting in every slot of an SM
+  // would keep the rest of the grid from starting)
+  if (late_wait && blockIdx.x == gridDim.x - 1) chain_wait();
 }
 
-cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, bool clear_maps, cudaStream_t s) {
+cudaError_t launch_append_prefill(const DevCtx& c, const PrefillArgs& a, bool clear_maps, bool late_wait,
+                                  cudaStream_t s) {
   const unsigned long long zero_vec = clear_maps ? (unsigned long long)a.layer_count * c.chunk * c.chunk / 4 : 0ull;
   const size_t threads = (size_t)a.layer_count * a.n * c.Hkv * 16 + zero_vec;
-  return launch_chained(k_append_prefill, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, s, c, a, zero_vec);
+  return launch_chained(k_append_prefill, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, s, c, a, zero_vec,
+                        late_wait ? 1 : 0);
 }
 
 __global__ void k_append_decode(DevCtx c, DecBatch b, int layer_begin, int layer_count,
@@ -137,6 +145,7 @@ cudaError_t launch_append_decode(const DevCtx& c, const DecBatch& b, int layer_b
 // its most voted token(s), and is appended to the span table.  One CTA per layer, one warp per span (32 warps).
 __global__ void __launch_bounds__(1024) k_evict_index(DevCtx c, EvictArgs a) {
   chain_wait();
+  if (a.release) chain_release();
   const int layer = a.layer_begin + blockIdx.x;
   const size_t unit = unit_of(c, a.seq, layer);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;

@@ -651,19 +651,23 @@ int ltri_prefill_chunk(ltri_ctx* ctx, int seq, int layer_begin, int layer_count,
   }
   const long long shift = d.paged ? s0.base - d.Lsp : 0;
   a.shift = shift;
+  // The eviction kernel (one CTA per layer) goes first and releases the append kernel behind it at once: the two
+  // touch different data and run side by side; the append kernel waits for the eviction kernel at its end.  They are
+  // timed together (class LTRI_K_EVICT); a call that evicts nothing times its append kernel alone (LTRI_K_APPEND).
   {
-    Scope sc(ctx, st, LTRI_K_APPEND, 1);
-    LTRI_CUDA(ctx, launch_append_prefill(d, a, /*clear_maps=*/ctx->use_tc, st));
-  }
-  for (size_t i = 0; i < ev.size(); i += 8) {
-    Scope sc(ctx, st, LTRI_K_EVICT, 1);
-    EvictArgs ea;
-    ea.seq = seq;
-    ea.shift = shift;
-    ea.layer_begin = layer_begin;
-    ea.nslots = (int)std::min<size_t>(8, ev.size() - i);
-    for (int j = 0; j < ea.nslots; ++j) ea.slot[j] = ev[i + j].slot;
-    LTRI_CUDA(ctx, launch_evict_index(d, ea, layer_count, st));
+    const int n_ev = (int)((ev.size() + 7) / 8);
+    Scope sc(ctx, st, n_ev > 0 ? LTRI_K_EVICT : LTRI_K_APPEND, n_ev + 1);
+    for (size_t i = 0; i < ev.size(); i += 8) {
+      EvictArgs ea;
+      ea.seq = seq;
+      ea.shift = shift;
+      ea.layer_begin = layer_begin;
+      ea.nslots = (int)std::min<size_t>(8, ev.size() - i);
+      ea.release = i + 8 >= ev.size() ? 1 : 0;
+      for (int j = 0; j < ea.nslots; ++j) ea.slot[j] = ev[i + j].slot;
+      LTRI_CUDA(ctx, launch_evict_index(d, ea, layer_count, st));
+    }
+    LTRI_CUDA(ctx, launch_append_prefill(d, a, /*clear_maps=*/ctx->use_tc, /*late_wait=*/n_ev > 0, st));
   }
   if (d.host_kv && !ev.empty()) {
     // mirror the rows that just left the window to the host: one strided copy for K and one for V per region (the
