@@ -548,6 +548,8 @@ __global__ void __launch_bounds__(256) k_seg_rowscan(DevCtx c, int layer_begin, 
 // supplies the offsets, and a second pass emits S.  key = (S << 10) | (1023 - (y-x)).
 // seg_unit > 0 (segmentation per memory unit): only intervals inside one unit of seg_unit tokens on the absolute grid
 // are candidates; `origin` is the absolute position of the region's first token.
+// HOLD: a thread keeps its (at most 16) entries of the column in registers between the two passes (m <= 512).
+template <bool HOLD>
 __global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin, int m, int seg_unit, int origin) {
   chain_wait();
   extern __shared__ long long sm[];
@@ -561,8 +563,18 @@ __global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin,
   for (int t = threadIdx.x; t < m + 32; t += blockDim.x) sbest[t] = 0;
   const int ylo = ry * R, yhi = min(m, ylo + R);
   long long acc = 0;
-  if (x < m)
+  long long cv[HOLD ? 16 : 1];
+  if (HOLD) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const int y = ylo + k;
+      cv[k] = (x < m && y >= x && y < yhi) ? Rs[(size_t)y * c.chunk + x] : 0;
+    }
+#pragma unroll
+    for (int k = 0; k < 16; ++k) acc += cv[k];
+  } else if (x < m) {
     for (int y = max(ylo, x); y < yhi; ++y) acc += Rs[(size_t)y * c.chunk + x];
+  }
   part[ry * 32 + cx] = acc;
   __syncthreads();
   if (ry == 0) {  // exclusive scan over ry for column cx
@@ -578,11 +590,24 @@ __global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin,
     long long S = part[ry * 32 + cx];
     // last token of the unit that holds x (region-relative)
     const int ymax = seg_unit > 0 ? ((origin + x) / seg_unit + 1) * seg_unit - origin - 1 : m;
-    for (int y = max(ylo, x); y < yhi; ++y) {
-      S += Rs[(size_t)y * c.chunk + x];
-      if (S > 0 && y <= ymax) {
-        const long long key = (S << 10) | (long long)(1023 - (y - x));
-        atomicMax(&sbest[x + y - 2 * x0], key);
+    if (HOLD) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int y = ylo + k;
+        if (y < x || y >= yhi) continue;
+        S += cv[k];
+        if (S > 0 && y <= ymax) {
+          const long long key = (S << 10) | (long long)(1023 - (y - x));
+          atomicMax(&sbest[x + y - 2 * x0], key);
+        }
+      }
+    } else {
+      for (int y = max(ylo, x); y < yhi; ++y) {
+        S += Rs[(size_t)y * c.chunk + x];
+        if (S > 0 && y <= ymax) {
+          const long long key = (S << 10) | (long long)(1023 - (y - x));
+          atomicMax(&sbest[x + y - 2 * x0], key);
+        }
       }
     }
   }
@@ -900,8 +925,12 @@ cudaError_t launch_segment(const DevCtx& c, int seq, int layer_begin, int layer_
   }
   launch_chained(k_seg_rowscan, dim3((m + 7) / 8, layer_count), dim3(256), 0, s, c, layer_begin, m);
   const size_t smem = (size_t)(32 * 32 + m + 32) * sizeof(long long);
-  launch_chained(k_seg_colscan, dim3((m + 31) / 32, layer_count), dim3(1024), smem, s, c, layer_begin, m, seg_unit,
-                 reg_start);
+  if (m <= 512)
+    launch_chained(k_seg_colscan<true>, dim3((m + 31) / 32, layer_count), dim3(1024), smem, s, c, layer_begin, m, seg_unit,
+                   reg_start);
+  else
+    launch_chained(k_seg_colscan<false>, dim3((m + 31) / 32, layer_count), dim3(1024), smem, s, c, layer_begin, m,
+                   seg_unit, reg_start);
   NmsArgs a{seq, layer_begin, m, reg_start, slot, max_spans, n, t0, q, tables ? 1 : 0, seg_unit};
   launch_chained(k_seg_nms, dim3(layer_count), dim3(1024), 0, s, c, a);
   return cudaGetLastError();
