@@ -2061,6 +2061,15 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
     }
     const unsigned T = s_prefix;
     const unsigned need_eq = s_need;  // how many of the == T elements are taken (lowest ids first, cluster-wide)
+    if (tot[T & 255u] == need_eq) {
+      // (the last pass counted the cluster's keys equal to T; every CTA holds the same tot) every key at the
+      // threshold is taken: no order among them is needed, and no exchange of counts
+      for (int s = tid; s < nloc; s += nt)
+        if (order_key(ssc[s]) >= T) {
+          const int slot = atomicAdd(&s_take, 1);
+          if (slot < kMaxTopK) s_loc[slot] = lo + s;
+        }
+    } else {
     // contiguous id partition so that ties are picked in id order: inside the CTA by thread, across CTAs by rank
     const int pt = (nloc + nt - 1) / nt;
     const int tlo = min(nloc, tid * pt), thi = min(nloc, tlo + pt);
@@ -2086,6 +2095,7 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
         const int slot = atomicAdd(&s_take, 1);
         if (slot < kMaxTopK) s_loc[slot] = lo + s;
       }
+    }
     }
   }
   __syncthreads();
@@ -2120,28 +2130,33 @@ __global__ void __cluster_dims__(kRetCluster, 1, 1) __launch_bounds__(kRetThread
     s_sln[tid] = c.span_len[unit * c.cap + ids_all[tid]];
   }
   __syncthreads();
-  if (tid == 0) {
-    int nr = 0;
+  if (tid < 32) {
+    // items: the sink, the selected spans, the recent tokens
+    const int rbeg = min(loc_begin, pos + 1);
+    const int nr = merge_ranges_warp(
+        nall + 2,
+        [&](int i, int& st, int& ln) {
+          if (i == 0) {
+            st = 0;
+            ln = min(c.Ls, pos + 1);
+          } else if (i <= nall) {
+            st = s_sst[i - 1];
+            ln = s_sln[i - 1];
+          } else {
+            st = rbeg;
+            ln = pos + 1 - rbeg;
+          }
+        },
+        s_rs, s_rl);
     long long tokens = 0;
-    auto push = [&](int st, int ln) {
-      if (ln <= 0) return;
-      if (nr > 0 && s_rs[nr - 1] + s_rl[nr - 1] >= st)  // adjacent, or (NMS with phi > 0) overlapping: one range
-        s_rl[nr - 1] = max(s_rl[nr - 1], st + ln - s_rs[nr - 1]);
-      else {
-        s_rs[nr] = st;
-        s_rl[nr] = ln;
-        ++nr;
-      }
-    };
-    push(0, min(c.Ls, pos + 1));
-    for (int t = 0; t < nall; ++t) {
-      tokens += s_sln[t];
-      push(s_sst[t], s_sln[t]);
+    for (int t = tid; t < nall; t += 32) tokens += s_sln[t];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tokens += shfl_xor_ll(tokens, o);
+    if (tid == 0) {
+      s_nr = nr;
+      c.rng_cnt[unit * c.Hkv + g] = nr;
+      c.sel_tokens[unit * c.Hkv + g] = tokens;  // (summed over the KV heads by ltri_get_stats)
     }
-    push(min(loc_begin, pos + 1), pos + 1 - min(loc_begin, pos + 1));
-    s_nr = nr;
-    c.rng_cnt[unit * c.Hkv + g] = nr;
-    c.sel_tokens[unit * c.Hkv + g] = tokens;  // (summed over the KV heads by ltri_get_stats)
   }
   __syncthreads();
   const size_t rbb = (unit * c.Hkv + g) * (size_t)c.rcap;
