@@ -188,10 +188,13 @@ def test_equal_scores_at_the_cut_go_to_the_lower_span(fused, monkeypatch):
     print(sp.rep)
 
 
-def test_hundreds_of_equal_scores_fall_back_to_the_radix_passes():
+@pytest.mark.parametrize("fused", ["1", "2"])
+def test_hundreds_of_equal_scores_fall_back_to_the_radix_passes(fused, monkeypatch):
     # Eq. 8 with a whole index of equal scores: every loaded span gets the same vector, so several hundred scores are
     # exactly equal and the short cut of the select (which ranks at most 256 keys near the maximum against each
     # other) has to hand over to the radix passes and their id-ordered tie pass; picks = the lowest span ids.
+    # (both one-launch decode retrievers: one CTA per KV head, and the cluster of eight)
+    monkeypatch.setenv("LTRI_DEC_FUSED", fused)
     cfg = small_cfg(n_layers=1, context=12288, decode_steps=2, top_k=6, max_spans_per_region=8, seg_min=8, seg_max=24)
     sp = ph.StreamPair(cfg, [0], deep=False)
     st = inputs.SyntheticStream(cfg)
