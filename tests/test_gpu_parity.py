@@ -173,9 +173,12 @@ def test_host_memory_pager(cache_units, decay, extra):
     print(rep)
 
 
-def test_host_memory_pager_is_bit_identical_to_the_resident_path():
+@pytest.mark.parametrize("groups", ["1", "2"])
+def test_host_memory_pager_is_bit_identical_to_the_resident_path(groups, monkeypatch):
     # the same stream through a paged and a resident context: every output bit and every selection equal, also
-    # with irregular call sizes (units that are still growing bypass the cache) and after a sequence reset
+    # with irregular call sizes (units that are still growing bypass the cache) and after a sequence reset; the
+    # paged call issued as one group of layers or as two whose pulls run under the other group's kernels
+    monkeypatch.setenv("LTRI_PAGER_GROUPS", groups)
     cfg = small_cfg(n_layers=2, context=1800, decode_steps=4, unit_tokens=48, top_k=5)
     paged = dataclasses.replace(cfg, host_kv=True, cache_units=7, score_decay=0.1)
     st = inputs.SyntheticStream(cfg)
