@@ -620,7 +620,7 @@ __global__ void __launch_bounds__(1024) k_seg_colscan(DevCtx c, int layer_begin,
   }
 }
 
-// step 4: sort the <= 2m-1 candidates by (S desc, length asc, start asc), greedy non-maximum suppression with
+// step 4: the <= 2m-1 candidates in the order (S desc, length asc, start asc), greedy non-maximum suppression with
 // IoU threshold 0 until max_spans are kept, gap fill, store the region's spans in its pending slot; then the
 // query representatives of every span (Sec. 3.4 step 2): u[g][j] = sum_{h in g} sum_{rep tokens} q_h[tok].
 // NMS on the squares (x, x, y+1, y+1): a candidate is suppressed by a kept span when their IoU exceeds phi_milli/1000;
