@@ -28,7 +28,7 @@ using namespace tc;
 constexpr float kLog2eT = 1.4426950408889634f;
 constexpr int kTcThreads = 576;  // 16 softmax warps + TMA producer + MMA issuer
 constexpr int kNumBoxes = 5;  // box heights 8,16,32,64,128
-constexpr float kRescaleThreshold = 8.0f;
+constexpr float kRescaleThreshold = 24.0f;
 // Largest exponent (log2 units) a probability may carry above the softmax reference in the regular launch: 2^90 times
 // the 2^7 keys of a tile, the 2^13 tiles of the longest item and values of up to 2^10 still fits fp32 (and the bf16
 // P operand).
